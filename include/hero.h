@@ -1,0 +1,245 @@
+/*
+ * hero.h - C ABI of the B200 (sm_100a) W8A8 transformer-layer forward of ZeroQuant-HERO.
+ *
+ * Every pointer named "device" is a CUDA device pointer on the GPU that was current when the
+ * handle was created; everything else is host memory or a plain value.  The caller owns every
+ * buffer and the stream.  No entry point on the hot path allocates or frees device memory, and
+ * every call is asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream).
+ * Nothing crosses this boundary but plain C types: no exceptions, no abort, no trap.
+ *
+ * Conventions (paper Sec. 2.1):
+ *   - INT8 is symmetric, range [-127, 127]; Round() is round-half-to-even.
+ *   - A linear layer is Y = X W with X [n, d] and W [d, m].  Weights are passed "column-major" as
+ *     the paper says: an array [m][d] (one output column after another, the reduction dimension d
+ *     contiguous), with one scale per output column, S_w [m] (Eq. 2).
+ *   - Activation scales follow Eq. 3-5: TWQ S_x [n] (one per token row, computed on the fly by
+ *     LN^quant and written by the library), FWQ S_x [d] (calibrated, read by the library),
+ *     SQ a single value (device pointer to one float).
+ *   - All scale / bias / gamma / beta vectors are device float32.
+ *   - Matrices are row-major with a leading dimension `ld` in elements; data pointers must be
+ *     16-byte aligned and ld * sizeof(element) a multiple of 16.
+ *
+ * Errors: every call returns a hero_status.  HERO_ERR_INVALID_ARG / _UNSUPPORTED / _ALIGNMENT are
+ * detected on the host before anything is launched.  HERO_ERR_CUDA reports a failed runtime call
+ * (text via hero_last_error()).  A device-side wait that exceeded its bound (a pipeline bug, never
+ * expected) sets a device error word; hero_check() synchronizes the stream and returns
+ * HERO_ERR_DEVICE_TIMEOUT if it is set.
+ */
+#ifndef HERO_H_
+#define HERO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  HERO_OK = 0,
+  HERO_ERR_INVALID_ARG = 1,
+  HERO_ERR_UNSUPPORTED = 2,
+  HERO_ERR_ALIGNMENT = 3,
+  HERO_ERR_WORKSPACE = 4,
+  HERO_ERR_CUDA = 5,
+  HERO_ERR_DEVICE_TIMEOUT = 6
+} hero_status;
+
+typedef enum { HERO_I8 = 0, HERO_U8 = 1, HERO_I32 = 2, HERO_F16 = 3, HERO_BF16 = 4, HERO_F32 = 5 } hero_dtype;
+
+/* Granularity of the scale attached to an INT8 tensor (Eq. 3-5). */
+typedef enum { HERO_GRAN_NONE = 0, HERO_GRAN_TWQ = 1, HERO_GRAN_FWQ = 2, HERO_GRAN_SQ = 3 } hero_gran;
+
+typedef enum { HERO_ACT_NONE = 0, HERO_ACT_GELU_ERF = 1, HERO_ACT_GELU_TANH = 2 } hero_act;
+typedef enum { HERO_MASK_NONE = 0, HERO_MASK_CAUSAL = 1 } hero_mask;
+typedef enum { HERO_POST_LN = 0, HERO_PRE_LN = 1 } hero_arch;
+/* Table 1: a module runs INT8 or stays in FP16/BF16 (the layer's fp_dtype). */
+typedef enum { HERO_MODE_INT8 = 0, HERO_MODE_FP = 1 } hero_mode;
+typedef enum { HERO_MOD_QKV = 0, HERO_MOD_ATTN = 1, HERO_MOD_ATTN_OUT = 2, HERO_MOD_FC1 = 3, HERO_MOD_FC2 = 4 } hero_module;
+typedef enum { HERO_PRESET_M1 = 1, HERO_PRESET_M2 = 2, HERO_PRESET_M3 = 3, HERO_PRESET_FP = 0 } hero_preset;
+
+/* A matrix on the device.  data == NULL means "absent" wherever a tensor is optional.
+ *   dtype : hero_dtype of the payload
+ *   gran  : hero_gran; for HERO_I8 payloads says what `scale` holds:
+ *           TWQ -> scale[rows], FWQ -> scale[cols], SQ -> scale[1], NONE -> no scale (value = code)
+ *   scale : device float32; read for inputs and for FWQ/SQ outputs, WRITTEN for TWQ outputs. */
+typedef struct {
+  void* data;
+  int32_t dtype;
+  int32_t gran;
+  int64_t rows;
+  int64_t cols;
+  int64_t ld;
+  float* scale;
+} hero_tensor;
+
+typedef struct hero_handle hero_handle;
+
+/* Create / destroy a handle on the current CUDA device.  Creation allocates the 4-byte device
+ * error word and queries the device; it is the only place the library allocates. */
+hero_status hero_create(hero_handle** out);
+hero_status hero_destroy(hero_handle* h);
+/* Text of the last error raised on the calling thread (never NULL). */
+const char* hero_last_error(void);
+/* Synchronize `stream`, read the device error word and clear it. */
+hero_status hero_check(hero_handle* h, void* stream);
+/* Number of kernels this handle has launched since creation (for benchmarks' accounting). */
+int64_t hero_launch_count(const hero_handle* h);
+
+/* ---------------------------------------------------------------------------------------------
+ * LN^quant  (Sec. 2.2.1 Eq. 6-7 embedding flavour; Sec. 2.2.2 Eq. 19 and Sec. 2.2.3 Eq. 31
+ * residual flavour).  One pass over each row:
+ *     r[i,:]  = residual[i,:] + branch[i,:] + extra[i,:]        (each dequantized in fp32)
+ *     y[i,:]  = (r - mean_i) / sqrt(biased_var_i + eps) * gamma + beta
+ *     out     = TWQ: S[i] = absmax_j |y[i,j]| / 127 (zero row -> 1), q = clip(Round(y / S[i]))
+ *               FWQ / SQ: q = clip(Round(y / S[j]))  with the given calibrated scale
+ *               F16 / BF16: y rounded to that type
+ *   residual : required.  I8 (TWQ / FWQ / SQ / NONE) or F16 / BF16, [M, H].
+ *   branch   : optional second addend, I8 (FWQ / SQ / TWQ / NONE) or F16 / BF16 (X_o S_o of Eq. 19).
+ *   extra    : optional third addend, F16 / BF16 (X_s of Eq. 7).
+ *   token_ids != NULL selects the embedding gather of Eq. 7: `residual` is then the token table
+ *       [V, H] I8 with TWQ scale [V], row ids[i]; `branch` the position table [P, H] F16/BF16, row
+ *       (i mod seq_len); `extra` the sentence-type table [T, H], row type_ids[i].  M = n_tokens.
+ *   out      : I8 (gran TWQ: out.scale[M] is written; FWQ / SQ: out.scale is read) or F16 / BF16.
+ *              out.data == NULL skips the normalisation (bare residual add into fp_out).
+ *   fp_out   : optional F16 / BF16 copy of r (the FP residual stream of a pre-LN layer); when
+ *              present the normalisation reads the stored (rounded) r.
+ * H must be a multiple of 16 and at most 16384.  M may be any size, including 0 (no launch).
+ */
+typedef struct {
+  hero_tensor residual;
+  hero_tensor branch;
+  hero_tensor extra;
+  const int32_t* token_ids; /* device [M] or NULL */
+  const int32_t* type_ids;  /* device [M]; required with token_ids when extra is present */
+  int32_t seq_len;
+  int64_t n_tokens;         /* M for the gather flavour; ignored otherwise */
+  const float* gamma;       /* device [H] */
+  const float* beta;        /* device [H] */
+  float eps;
+  hero_tensor out;
+  hero_tensor fp_out;
+} hero_ln_args;
+
+hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * GeMM^quant with fused epilogue (Sec. 2.2.2 Eq. 14, 18, 20-23; Sec. 2.2.3 Eq. 28-30, 32).
+ *     acc[i,j] = sum_k A[i,k] * W[j,k]                    exact INT32 (INT8 operands)
+ *     v        = acc * rs[i] * w_scale[j] + bias[j]       rs = TWQ scale of A, or 1
+ *     a        = act(v)                                   none | GELU(erf) | GELU(tanh)
+ *     a       *= post_scale[j]                            (1 / S_a of GELU^quant; NULL = skip)
+ *     out      = I8: clip(Round(a), -127, 127)            (Eq. 22: a bare Round once scales are folded)
+ *                F16 / BF16: a rounded to that type
+ *                I32: the raw accumulators (INT8 operands only; epilogue skipped; for verification)
+ *   A    : [M, K] I8 (gran TWQ -> row scale applied; NONE / FWQ / SQ -> none: a feature-wise or
+ *          static input scale must already be folded into W's rows, Eq. 23 / 32), or F16 / BF16
+ *          for a module left in FP mode (then W has the same type and w_scale is ignored).
+ *   W    : device [N][K], K contiguous, leading dimension ldw; same element type as A.
+ *   out  : [M, N].  A TWQ output is refused (HERO_ERR_UNSUPPORTED): the paper keeps the row
+ *          reduction out of GEMM epilogues (Sec. 2.1).
+ * K must be a multiple of 16 bytes of elements and N a multiple of 16; M is arbitrary.
+ */
+typedef struct {
+  hero_tensor A;
+  const void* W;
+  int64_t N;
+  int64_t ldw;
+  const float* w_scale;    /* device [N] (INT8 operands) */
+  const float* bias;       /* device [N] or NULL */
+  int32_t act;             /* hero_act */
+  const float* post_scale; /* device [N] or NULL */
+  hero_tensor out;
+} hero_linear_args;
+
+hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * INT8 attention core (Sec. 2.2.2 Eq. 15-17).  Per (batch b, head h), rows of one sequence:
+ *     A    = d~ (Q K^T),  d~ = s_q s_k / sqrt(dh)          INT32 -> fp32, never quantized
+ *     P    = softmax(A) over the allowed keys              fully normalised
+ *     P_u8 = clip(Round(P / s_p), 0, 255)                  unsigned ("asymmetric") INT8
+ *     acc  = P_u8 V                                        exact INT32
+ *     out  = I8: clip(Round(acc * s_p * s_v / out_scale[j]))  (FWQ [H]; SQ: one value)
+ *            F16 / BF16: acc * s_p * s_v
+ *   q, k, v : device pointers to element (0, 0) of [B*S, nh*dh] views with leading dimension ld
+ *             (e.g. the three thirds of the QKV GEMM output, ld = 3H).  dtype I8, or F16 / BF16 for
+ *             the FP attention of a module left in FP mode (then s_q, s_k, s_v, s_p are ignored and
+ *             out = softmax(Q K^T / sqrt(dh)) V, quantized by out_scale when out is I8).
+ *   mask    : HERO_MASK_NONE or HERO_MASK_CAUSAL; key_len (device int32 [B], optional) further
+ *             limits the keys of sequence b to k < key_len[b].  A fully masked row outputs 0.
+ *   dh is 64 or 128.
+ */
+typedef struct {
+  const void* q;
+  const void* k;
+  const void* v;
+  int32_t dtype;       /* hero_dtype of q, k, v */
+  int64_t ld;
+  int32_t B, S, nh, dh;
+  float s_q, s_k, s_v, s_p;
+  int32_t mask;        /* hero_mask */
+  const int32_t* key_len;
+  hero_tensor out;     /* [B*S, nh*dh]; I8 with gran FWQ (scale[H]) or SQ (scale[1]); or F16 / BF16 */
+} hero_attn_args;
+
+hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * One transformer layer (Sec. 2.2.2-2.2.3, modes of Sec. 2.3 Table 1).
+ * Post-LN (the paper's equations):  x_mid = LN1(x_in + Attn(x_in)); x_out = LN2(x_mid + MLP(x_mid)).
+ * Pre-LN (GPT-shaped): h' = h + Attn(LN1(h [+ pending])); out = h' + MLP(LN2(h')) with the residual
+ * stream h in fp_dtype.
+ * A producer emits what its consumer's mode needs; an INT8 module contracts INT8 x INT8.
+ */
+typedef struct {
+  const void* W;           /* device [N][K]: I8 when the module is INT8, else fp_dtype */
+  const float* w_scale;    /* device [N]; INT8 modules */
+  const float* bias;       /* device [N] or NULL */
+  const float* post_scale; /* device [N] or NULL: multiplies after the activation (1/S_a; 1/S_q.. for an
+                              FP QKV feeding INT8 attention) */
+} hero_linear_params;
+
+typedef struct {
+  int32_t arch;            /* hero_arch */
+  int32_t B, S, H, nh, F;
+  int32_t act;             /* hero_act of the MLP */
+  float eps;
+  int32_t mask;            /* hero_mask */
+  int32_t fp_dtype;        /* HERO_F16 or HERO_BF16: type of every FP tensor at a module border */
+  int32_t mode[5];         /* hero_mode per hero_module */
+  int32_t gran_in;         /* granularity of the INT8 tensor feeding QKV (TWQ | FWQ | SQ) */
+  int32_t gran_mid;        /* granularity of the INT8 tensor feeding FC1 */
+  int32_t gran_attn;       /* granularity of X_attn (FWQ | SQ) */
+  int32_t gran_out;        /* post-LN layer output: TWQ | FWQ | SQ, or NONE for an FP output */
+  const float* s_in;       /* device: FWQ [H] / SQ [1] scale of the tensor feeding QKV (pre-LN: LN1 output) */
+  const float* s_mid;      /* device: same for the tensor feeding FC1 */
+  const float* s_attn;     /* device: FWQ [H] / SQ [1] scale of X_attn */
+  const float* s_o;        /* device [H]: FWQ scale X_o stands for (folded into W_o; used by LN) */
+  const float* s_x2;       /* device [H]: FWQ scale X_2 stands for */
+  const float* s_out;      /* device: FWQ [H] / SQ [1] scale of a non-TWQ INT8 layer output */
+  float s_q, s_k, s_v, s_p;
+  hero_linear_params qkv, o, fc1, fc2;
+  const float* ln1_g; const float* ln1_b;
+  const float* ln2_g; const float* ln2_b;
+} hero_layer_desc;
+
+/* Fill desc->mode from a Table 1 preset (M1, M2, M3) or all-FP. */
+hero_status hero_mode_preset(int32_t preset, int32_t mode_out[5]);
+/* Scratch the layer needs for M tokens. */
+hero_status hero_layer_workspace_bytes(const hero_layer_desc* d, int64_t M, size_t* bytes);
+/*   in      : post-LN: X_in [M, H] I8 (+scale per gran_in) or fp_dtype when QKV is FP.
+ *             pre-LN : residual stream h [M, H] in fp_dtype.
+ *   pending : pre-LN only, optional: a branch (I8 FWQ or fp_dtype) still to be added to h, i.e. the
+ *             previous layer's X_2; the add is fused into LN1's kernel.
+ *   out     : post-LN: X_out (I8 TWQ -> out.scale[M] written; I8 FWQ/SQ; or fp_dtype).
+ *             pre-LN : h_out = h' + X_2 in fp_dtype (the closing add of a lone layer).
+ *   workspace: device scratch of at least hero_layer_workspace_bytes(), 256-byte aligned. */
+hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in,
+                               const hero_tensor* pending, const hero_tensor* out, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HERO_H_ */

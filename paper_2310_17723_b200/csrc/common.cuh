@@ -1,0 +1,60 @@
+// Shared host-side plumbing of the library: the handle, error reporting, argument checks.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/hero.h"
+
+struct hero_handle {
+  int device;
+  int sm_count;
+  int max_smem_optin;
+  int* d_error;        // device error word: 0 = fine, else a code saying which wait gave up
+  int64_t launches;
+  void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+namespace hero {
+
+void set_error(const char* fmt, ...);
+hero_status cuda_fail(cudaError_t e, const char* what);
+
+#define HERO_CUDA(call)                                   \
+  do {                                                    \
+    cudaError_t _e = (call);                              \
+    if (_e != cudaSuccess) return hero::cuda_fail(_e, #call); \
+  } while (0)
+
+#define HERO_REQUIRE(cond, status, ...)  \
+  do {                                   \
+    if (!(cond)) {                       \
+      hero::set_error(__VA_ARGS__);      \
+      return (status);                   \
+    }                                    \
+  } while (0)
+
+inline size_t dtype_size(int dt) {
+  switch (dt) {
+    case HERO_I8: case HERO_U8: return 1;
+    case HERO_F16: case HERO_BF16: return 2;
+    case HERO_I32: case HERO_F32: return 4;
+    default: return 0;
+  }
+}
+inline bool is_fp16ish(int dt) { return dt == HERO_F16 || dt == HERO_BF16; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// data pointer 16-byte aligned, row pitch a multiple of 16 bytes, ld >= cols
+hero_status check_matrix(const hero_tensor& t, const char* name);
+
+// 2-D TMA descriptor over a row-major matrix [rows, cols] of `elem_bytes` elements with row pitch
+// ld_bytes; box = box_cols x box_rows elements; swizzle_bytes in {0, 32, 64, 128}.
+hero_status make_tmap_2d(const hero_handle* h, CUtensorMap* out, const void* base, int elem_bytes, bool is_fp16,
+                         bool is_bf16, uint64_t rows, uint64_t cols, uint64_t ld_bytes, uint32_t box_cols,
+                         uint32_t box_rows, int swizzle_bytes);
+
+}  // namespace hero

@@ -1,0 +1,372 @@
+// GeMM^quant (Sec. 2.2.2 Eq. 14, 18, 20-23; Sec. 2.2.3 Eq. 28-30, 32): INT8 x INT8 -> INT32 on the
+// tcgen05 tensor cores with the dequantize / bias / GELU / requantize epilogue applied straight
+// from tensor memory, plus the FP16/BF16 variant for modules left in FP mode (Table 1).
+//
+// One persistent CTA per SM, 6 warps:
+//   warps 0-3  epilogue: TMEM -> registers -> fused epilogue -> global (warp w owns TMEM lanes 32w..32w+31)
+//   warp  4    TMA producer: 128-byte-swizzled K-major tiles of A [128 x 128 B] and W [BN x 128 B]
+//   warp  5    UMMA issuer (one elected lane) and owner of the TMEM allocation
+// The accumulator is double-buffered in TMEM (2 x BN columns) so the epilogue of tile t overlaps the
+// main loop of tile t+1.  Every barrier wait is bounded; on expiry the CTA records a code and unwinds.
+#include "common.cuh"
+#include "ptx.cuh"
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+
+namespace hero {
+
+constexpr int GEMM_BM = 128;
+constexpr int GEMM_BK_BYTES = 128;   // one swizzle row
+constexpr int GEMM_THREADS = 192;
+constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2;
+
+struct GemmParams {
+  int M, N, K;              // K in elements
+  int num_m_tiles, num_n_tiles, num_kb;
+  const float* rs;          // [M] or NULL
+  const float* cs;          // [N] or NULL (FP operands)
+  const float* bias;        // [N] or NULL
+  const float* post;        // [N] or NULL
+  void* out;
+  long long out_ld;         // elements
+  int out_dt;               // hero_dtype
+  uint32_t idesc;
+  int elem_bytes;           // 1 (INT8) or 2 (F16 / BF16)
+  int* err;
+};
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int A_BYTES = GEMM_BM * GEMM_BK_BYTES;
+  static constexpr int B_BYTES = BN * GEMM_BK_BYTES;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int EPI_FLOATS = 2 * 3 * BN;                 // double-buffered cs / bias / post
+  static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256 /*barriers*/;
+};
+
+__device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+__device__ __forceinline__ float gelu_tanh_f(float x) {
+  return 0.5f * x * (1.0f + tanhf(0.79788456080286535588f * (x + 0.044715f * x * x * x)));
+}
+
+__device__ __forceinline__ uint32_t pack4_i8(float a, float b, float c, float d) {
+  int ia = __float2int_rn(fminf(fmaxf(a, -127.f), 127.f));
+  int ib = __float2int_rn(fminf(fmaxf(b, -127.f), 127.f));
+  int ic = __float2int_rn(fminf(fmaxf(c, -127.f), 127.f));
+  int id = __float2int_rn(fminf(fmaxf(d, -127.f), 127.f));
+  return (uint32_t)(ia & 0xff) | ((uint32_t)(ib & 0xff) << 8) | ((uint32_t)(ic & 0xff) << 16) | ((uint32_t)id << 24);
+}
+__device__ __forceinline__ uint32_t pack2_fp(float a, float b, int dt) {
+  if (dt == HERO_F16) {
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void st16(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mt, int& nt) {
+  // grouped order: consecutive tiles sweep GROUP_M row-tiles of one column-tile strip, so that the
+  // tiles in flight at any moment share A and W panels in L2
+  constexpr int GROUP_M = 16;
+  const int width = GROUP_M * num_n;
+  const int group = t / width;
+  const int first_m = group * GROUP_M;
+  const int gsize = min(num_m - first_m, GROUP_M);
+  const int r = t - group * width;
+  mt = first_m + (r % gsize);
+  nt = r / gsize;
+}
+
+template <int BN, bool INT8, int ACT, int OUTK>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* tiles = smem;
+  float* epi = reinterpret_cast<float*>(smem + STAGES * Cfg::STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi + Cfg::EPI_FLOATS);
+  uint64_t* full = bars;                    // [STAGES]  TMA -> MMA
+  uint64_t* empty = bars + STAGES;          // [STAGES]  MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;   // [2]       MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 2;       // [2]       epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }
+    ptx::fence_mbar_init();
+  }
+  if (warp == 5) {
+    ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  if (warp == 4 && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const int kelems = GEMM_BK_BYTES / p.elem_bytes;
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x100 | stage)) { ok = false; break; }
+          uint8_t* a_dst = tiles + stage * Cfg::STAGE_BYTES;
+          uint8_t* b_dst = a_dst + Cfg::A_BYTES;
+          ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
+          ptx::tma_load_2d(a_dst, &tmA, kb * kelems, mt * GEMM_BM, &full[stage]);
+          ptx::tma_load_2d(b_dst, &tmW, kb * kelems, nt * BN, &full[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      // drain: every copy this thread started has landed before the CTA may exit
+      for (int i = 0; i < STAGES; ++i) {
+        if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x180 | stage)) break;
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      int it = 0;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+        const int as = it & 1;
+        const uint32_t aphase = (it >> 1) & 1;
+        if (!ptx::mbar_wait(&acc_empty[as], aphase ^ 1, p.err, 0x200 | as)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + as * BN;
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!ptx::mbar_wait(&full[stage], phase, p.err, 0x300 | stage)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_addr = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + Cfg::A_BYTES;
+#pragma unroll
+          for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
+            const uint64_t ad = ptx::smem_desc(desc_base, a_addr + k * 32);
+            const uint64_t bd = ptx::smem_desc(desc_base, b_addr + k * 32);
+            if constexpr (INT8) ptx::umma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            else ptx::umma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+          }
+          ptx::umma_commit(&empty[stage]);      // frees the smem stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) ptx::umma_commit(&acc_full[as]);  // accumulator of this tile complete
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3)
+    const int tid_e = threadIdx.x;            // 0..127
+    int it = 0; bool ok = true;
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+      int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+      const int as = it & 1;
+      const uint32_t aphase = (it >> 1) & 1;
+      const int n0 = nt * BN;
+      float* e_cs = epi + (it & 1) * 3 * BN;
+      float* e_bias = e_cs + BN;
+      float* e_post = e_bias + BN;
+      if constexpr (OUTK != OUT_I32) {
+        for (int j = tid_e; j < BN; j += 128) {
+          const int n = n0 + j;
+          const bool in = n < p.N;
+          e_cs[j] = (in && p.cs) ? p.cs[n] : 1.0f;
+          e_bias[j] = (in && p.bias) ? p.bias[n] : 0.0f;
+          e_post[j] = (in && p.post) ? p.post[n] : 1.0f;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+      const int m = mt * GEMM_BM + warp * 32 + lane;
+      const bool row_ok = m < p.M;
+      float rs = 1.0f;
+      if (OUTK != OUT_I32 && INT8 && p.rs && row_ok) rs = p.rs[m];
+
+      if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
+      ptx::tc_fence_after();
+      if (ok) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + as * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld32(taddr + c * 32, r);
+          ptx::tmem_ld_wait();
+          const int col0 = n0 + c * 32;
+          if constexpr (OUTK == OUT_I32) {
+            if (row_ok) {
+              int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
+#pragma unroll
+              for (int g = 0; g < 8; ++g)
+                if (col0 + 4 * g + 4 <= p.N) st16(dst + 4 * g, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+            }
+          } else {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float acc = INT8 ? (float)(int)r[j] : __uint_as_float(r[j]);
+              float x = fmaf(acc * rs, e_cs[c * 32 + j], e_bias[c * 32 + j]);
+              if constexpr (ACT == HERO_ACT_GELU_ERF) x = gelu_erf_f(x);
+              if constexpr (ACT == HERO_ACT_GELU_TANH) x = gelu_tanh_f(x);
+              v[j] = x * e_post[c * 32 + j];
+            }
+            if (row_ok) {
+              if constexpr (OUTK == OUT_I8) {
+                int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
+#pragma unroll
+                for (int g = 0; g < 2; ++g)
+                  if (col0 + 16 * g + 16 <= p.N)
+                    st16(dst + 16 * g, pack4_i8(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
+                         pack4_i8(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
+                         pack4_i8(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
+                         pack4_i8(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
+              } else {
+                uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                  if (col0 + 8 * g + 8 <= p.N)
+                    st16(dst + 8 * g, pack2_fp(v[8 * g], v[8 * g + 1], p.out_dt), pack2_fp(v[8 * g + 2], v[8 * g + 3], p.out_dt),
+                         pack2_fp(v[8 * g + 4], v[8 * g + 5], p.out_dt), pack2_fp(v[8 * g + 6], v[8 * g + 7], p.out_dt));
+              }
+            }
+          }
+        }
+      }
+      // hand the accumulator buffer back to the MMA warp
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&acc_empty[as]);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 5) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+}
+
+template <int BN, bool INT8, int ACT, int OUTK>
+static hero_status launch_gemm(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+                               cudaStream_t stream) {
+  using Cfg = GemmCfg<BN>;
+  auto kern = gemm_kernel<BN, INT8, ACT, OUTK>;
+  static bool configured = false;   // per instantiation
+  if (!configured) {
+    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    configured = true;
+  }
+  const int tiles = p.num_m_tiles * p.num_n_tiles;
+  const int grid = tiles < h->sm_count ? tiles : h->sm_count;
+  kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+  HERO_CUDA(cudaGetLastError());
+  h->launches += 1;
+  return HERO_OK;
+}
+
+template <int BN, bool INT8>
+static hero_status dispatch_epilogue(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+                                     int act, cudaStream_t s) {
+  if (p.out_dt == HERO_I32) {
+    if constexpr (INT8) return launch_gemm<BN, true, HERO_ACT_NONE, OUT_I32>(h, tmA, tmW, p, s);
+    else { set_error("raw INT32 output needs INT8 operands"); return HERO_ERR_UNSUPPORTED; }
+  }
+  const bool i8 = p.out_dt == HERO_I8;
+  switch (act) {
+    case HERO_ACT_NONE:
+      return i8 ? launch_gemm<BN, INT8, HERO_ACT_NONE, OUT_I8>(h, tmA, tmW, p, s)
+                : launch_gemm<BN, INT8, HERO_ACT_NONE, OUT_FP>(h, tmA, tmW, p, s);
+    case HERO_ACT_GELU_ERF:
+      return i8 ? launch_gemm<BN, INT8, HERO_ACT_GELU_ERF, OUT_I8>(h, tmA, tmW, p, s)
+                : launch_gemm<BN, INT8, HERO_ACT_GELU_ERF, OUT_FP>(h, tmA, tmW, p, s);
+    case HERO_ACT_GELU_TANH:
+      return i8 ? launch_gemm<BN, INT8, HERO_ACT_GELU_TANH, OUT_I8>(h, tmA, tmW, p, s)
+                : launch_gemm<BN, INT8, HERO_ACT_GELU_TANH, OUT_FP>(h, tmA, tmW, p, s);
+  }
+  set_error("unknown activation %d", act);
+  return HERO_ERR_INVALID_ARG;
+}
+
+template <int BN>
+static hero_status run_bn(hero_handle* h, const hero_linear_args* a, GemmParams& p, cudaStream_t s) {
+  const bool int8 = a->A.dtype == HERO_I8;
+  const int eb = int8 ? 1 : 2;
+  const int kbox = GEMM_BK_BYTES / eb;
+  p.num_n_tiles = (p.N + BN - 1) / BN;
+  p.idesc = int8 ? ptx::make_idesc(2, 1, 1, 0, 0, GEMM_BM, BN)
+                 : ptx::make_idesc(1, a->A.dtype == HERO_BF16 ? 1 : 0, a->A.dtype == HERO_BF16 ? 1 : 0, 0, 0, GEMM_BM, BN);
+  CUtensorMap tmA, tmW;
+  hero_status st = make_tmap_2d(h, &tmA, a->A.data, eb, a->A.dtype == HERO_F16, a->A.dtype == HERO_BF16, (uint64_t)p.M,
+                                (uint64_t)p.K, (uint64_t)a->A.ld * eb, kbox, GEMM_BM, 128);
+  if (st != HERO_OK) return st;
+  st = make_tmap_2d(h, &tmW, a->W, eb, a->A.dtype == HERO_F16, a->A.dtype == HERO_BF16, (uint64_t)p.N, (uint64_t)p.K,
+                    (uint64_t)a->ldw * eb, kbox, BN, 128);
+  if (st != HERO_OK) return st;
+  if (int8) return dispatch_epilogue<BN, true>(h, tmA, tmW, p, a->act, s);
+  return dispatch_epilogue<BN, false>(h, tmA, tmW, p, a->act, s);
+}
+
+}  // namespace hero
+
+extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(h && a, HERO_ERR_INVALID_ARG, "hero_w8a8_linear: NULL handle or args");
+  hero_status st;
+  if ((st = check_matrix(a->A, "A")) != HERO_OK) return st;
+  if ((st = check_matrix(a->out, "out")) != HERO_OK) return st;
+  const bool int8 = a->A.dtype == HERO_I8;
+  HERO_REQUIRE(int8 || is_fp16ish(a->A.dtype), HERO_ERR_UNSUPPORTED, "A dtype %d: INT8, F16 or BF16 expected", a->A.dtype);
+  const int eb = int8 ? 1 : 2;
+  HERO_REQUIRE(a->W != nullptr && aligned16(a->W), a->W ? HERO_ERR_ALIGNMENT : HERO_ERR_INVALID_ARG,
+               "W must be a 16-byte aligned device pointer");
+  HERO_REQUIRE(a->N > 0 && a->N % 16 == 0, HERO_ERR_UNSUPPORTED, "N=%lld must be a positive multiple of 16", (long long)a->N);
+  const long long K = a->A.cols;
+  HERO_REQUIRE((K * eb) % 16 == 0, HERO_ERR_UNSUPPORTED, "K=%lld: K * element size must be a multiple of 16 bytes", K);
+  HERO_REQUIRE(a->ldw >= K && (a->ldw * eb) % 16 == 0, HERO_ERR_ALIGNMENT, "ldw=%lld invalid", (long long)a->ldw);
+  HERO_REQUIRE(a->out.rows == a->A.rows && a->out.cols == a->N, HERO_ERR_INVALID_ARG, "out shape mismatch");
+  HERO_REQUIRE(a->out.dtype == HERO_I8 || is_fp16ish(a->out.dtype) || a->out.dtype == HERO_I32, HERO_ERR_UNSUPPORTED,
+               "out dtype %d", a->out.dtype);
+  HERO_REQUIRE(!(a->out.dtype == HERO_I8 && a->out.gran == HERO_GRAN_TWQ), HERO_ERR_UNSUPPORTED,
+               "a token-wise (TWQ) output needs a row reduction, which is kept out of GEMM epilogues (Sec. 2.1); "
+               "fuse it into LN^quant instead");
+  HERO_REQUIRE(a->out.dtype != HERO_I32 || int8, HERO_ERR_UNSUPPORTED, "raw INT32 output needs INT8 operands");
+  if (int8) HERO_REQUIRE(a->w_scale != nullptr || a->out.dtype == HERO_I32, HERO_ERR_INVALID_ARG, "w_scale is required");
+  HERO_REQUIRE(a->act >= HERO_ACT_NONE && a->act <= HERO_ACT_GELU_TANH, HERO_ERR_INVALID_ARG, "unknown activation %d", a->act);
+  HERO_REQUIRE(a->A.rows < (1ll << 31) && a->N < (1ll << 31) && K < (1ll << 31), HERO_ERR_UNSUPPORTED, "dimension too large");
+  if (a->A.rows == 0) return HERO_OK;
+
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = (int)a->A.rows; p.N = (int)a->N; p.K = (int)K;
+  p.num_m_tiles = (p.M + GEMM_BM - 1) / GEMM_BM;
+  p.num_kb = (int)((K * eb + GEMM_BK_BYTES - 1) / GEMM_BK_BYTES);
+  p.rs = (int8 && a->A.gran == HERO_GRAN_TWQ) ? a->A.scale : nullptr;
+  p.cs = int8 ? a->w_scale : nullptr;
+  p.bias = a->bias; p.post = a->post_scale;
+  p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
+  p.elem_bytes = eb;
+  p.err = h->d_error;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // widest column tile that still gives every SM a tile
+  const long long t256 = (long long)p.num_m_tiles * ((p.N + 255) / 256);
+  const long long t128 = (long long)p.num_m_tiles * ((p.N + 127) / 128);
+  const long long enough = (long long)h->sm_count * 6 / 10;
+  if (t256 >= enough) return run_bn<256>(h, a, p, s);
+  if (t128 >= enough) return run_bn<128>(h, a, p, s);
+  return run_bn<64>(h, a, p, s);
+}

@@ -1,0 +1,850 @@
+// LN^quant family (Sec. 2.2.1 Eq. 6-7, Sec. 2.2.2 Eq. 19, Sec. 2.2.3 Eq. 31): one pass over each row.
+//
+// HBM-bound streaming kernel.  A row of H elements is owned by G = ceil(H / VEC) threads (rounded up
+// to whole warps), each holding VEC consecutive elements in registers; a CTA of about 256 threads
+// works on RPC = 256 / G rows at once and every thread keeps R rows in flight per loop trip so that
+// enough 16-byte loads are outstanding to cover DRAM latency.  Row statistics are two-pass over the
+// registers (mean, then centred variance), reduced with warp shuffles and, when a row spans several
+// warps, one shared-memory exchange per statistic.  gamma / beta stay in registers across the
+// persistent row loop; per-feature scale vectors are re-read through L1.
+#include "common.cuh"
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+
+namespace hero {
+
+struct LnSide {           // one addend of the LayerNorm input
+  const void* data;       // NULL = absent
+  int dt;                 // hero_dtype
+  long long ld;           // elements
+  const float* row_scale; // TWQ scale [rows] or NULL
+  const float* col_scale; // FWQ [H] (stride 1) or SQ [1] (stride 0) or NULL
+  int col_stride;
+};
+
+struct LnParams {
+  LnSide res, br, ex;
+  const int* token_ids;   // embedding gather (Eq. 7) when non-NULL
+  const int* type_ids;
+  int seq_len;
+  const float* gamma;
+  const float* beta;
+  float eps;
+  void* out; int out_dt; long long out_ld; int out_gran; float* out_scale;
+  void* fp_out; int fp_dt; long long fp_ld;
+  long long M; int H;
+  int G;                  // threads per row (multiple of 32)
+  int RPC;                // rows per CTA per pass
+};
+
+template <int VEC>
+__device__ __forceinline__ void load_raw(const void* p, int bytes_per_elem, uint32_t (&w)[VEC / 2]) {
+  // VEC elements of 1 or 2 bytes -> VEC/4 or VEC/2 32-bit words, streamed past L1
+  if (bytes_per_elem == 1) {
+    if constexpr (VEC == 8) {
+      asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "l"(p));
+    } else {
+      asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(p));
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC / 8; ++i)
+      asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(w[4 * i]), "=r"(w[4 * i + 1]), "=r"(w[4 * i + 2]), "=r"(w[4 * i + 3])
+                   : "l"(reinterpret_cast<const char*>(p) + 16 * i));
+  }
+}
+
+template <int VEC>
+__device__ __forceinline__ void unpack(const uint32_t (&w)[VEC / 2], int dt, float (&v)[VEC]) {
+  if (dt == HERO_I8) {
+#pragma unroll
+    for (int i = 0; i < VEC / 4; ++i) {
+#pragma unroll
+      for (int b = 0; b < 4; ++b) v[4 * i + b] = (float)(int)(signed char)((w[i] >> (8 * b)) & 0xff);
+    }
+  } else if (dt == HERO_F16) {
+#pragma unroll
+    for (int i = 0; i < VEC / 2; ++i) {
+      float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+      v[2 * i] = f.x; v[2 * i + 1] = f.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC / 2; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_fp2(float a, float b, int dt) {
+  if (dt == HERO_F16) {
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+__device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
+  // clip(Round(.)) to [-127, 127], round-half-to-even, packed little-endian
+  int ia = __float2int_rn(fminf(fmaxf(a, -127.f), 127.f));
+  int ib = __float2int_rn(fminf(fmaxf(b, -127.f), 127.f));
+  int ic = __float2int_rn(fminf(fmaxf(c, -127.f), 127.f));
+  int id = __float2int_rn(fminf(fmaxf(d, -127.f), 127.f));
+  return (uint32_t)(ia & 0xff) | ((uint32_t)(ib & 0xff) << 8) | ((uint32_t)(ic & 0xff) << 16) | ((uint32_t)id << 24);
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_words(void* p, const uint32_t* w, int nwords) {
+  // nwords in {2, 4, 8}
+  if (nwords == 2) {
+    asm volatile("st.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(w[0]), "r"(w[1]) : "memory");
+  } else {
+#pragma unroll
+    for (int i = 0; i < nwords / 4; ++i)
+      asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(reinterpret_cast<char*>(p) + 16 * i), "r"(w[4 * i]),
+                   "r"(w[4 * i + 1]), "r"(w[4 * i + 2]), "r"(w[4 * i + 3])
+                   : "memory");
+  }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Reduce R per-thread values over the G threads of a row.  red: [RPC][R][G/32] floats.
+template <int R, bool IS_MAX>
+__device__ __forceinline__ void row_reduce(float (&v)[R], float* red, int G, int row_in_cta, int t) {
+#pragma unroll
+  for (int r = 0; r < R; ++r) v[r] = IS_MAX ? warp_max(v[r]) : warp_sum(v[r]);
+  const int nw = G >> 5;
+  if (nw == 1) return;
+  float* mine = red + (size_t)row_in_cta * R * nw;
+  if ((t & 31) == 0) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) mine[r * nw + (t >> 5)] = v[r];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    float a = mine[r * nw];
+    for (int w = 1; w < nw; ++w) a = IS_MAX ? fmaxf(a, mine[r * nw + w]) : a + mine[r * nw + w];
+    v[r] = a;
+  }
+}
+
+template <int VEC, int R, bool HAS_BR, bool HAS_EX>
+__global__ void __launch_bounds__(512) ln_quant_kernel(const LnParams p) {
+  extern __shared__ float red_smem[];
+  const int G = p.G, RPC = p.RPC, H = p.H;
+  const int nw = G >> 5;
+  float* red0 = red_smem;
+  float* red1 = red0 + RPC * R * nw;
+  float* red2 = red1 + RPC * R * nw;
+
+  const int tid = threadIdx.x;
+  const int row_in_cta = tid / G;
+  const int t = tid - row_in_cta * G;
+  const int c0 = t * VEC;
+  const bool active = c0 < H;
+  const float inv_H = 1.0f / (float)H;
+
+  float gam[VEC], bet[VEC];
+  const bool normalize = p.out != nullptr;
+  if (active && normalize) {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 4) {
+      float4 g4 = *reinterpret_cast<const float4*>(p.gamma + c0 + i);
+      float4 b4 = *reinterpret_cast<const float4*>(p.beta + c0 + i);
+      gam[i] = g4.x; gam[i + 1] = g4.y; gam[i + 2] = g4.z; gam[i + 3] = g4.w;
+      bet[i] = b4.x; bet[i + 1] = b4.y; bet[i + 2] = b4.z; bet[i + 3] = b4.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) { gam[i] = 0.f; bet[i] = 0.f; }
+  }
+
+  const int res_es = (p.res.dt == HERO_I8) ? 1 : 2;
+  const int br_es = (p.br.dt == HERO_I8) ? 1 : 2;
+  const long long rows_per_trip = (long long)RPC * R;
+
+  for (long long base = (long long)blockIdx.x * rows_per_trip; base < p.M; base += (long long)gridDim.x * rows_per_trip) {
+    float x[R][VEC];
+    uint32_t raw_res[R][VEC / 2], raw_br[HAS_BR ? R : 1][VEC / 2], raw_ex[HAS_EX ? R : 1][VEC / 2];
+    long long row[R];
+    bool valid[R];
+    float rs_res[R], rs_br[R];
+
+    // ---- issue every load of the trip before touching the data
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      row[r] = base + (long long)r * RPC + row_in_cta;
+      valid[r] = active && row[r] < p.M;
+      rs_res[r] = 1.f; rs_br[r] = 1.f;
+      if (valid[r]) {
+        long long rr = row[r], rb = row[r], re = row[r];
+        if (p.token_ids) {
+          rr = p.token_ids[row[r]];
+          rb = row[r] % p.seq_len;
+          re = p.type_ids ? p.type_ids[row[r]] : 0;
+        }
+        load_raw<VEC>(reinterpret_cast<const char*>(p.res.data) + (rr * p.res.ld + c0) * res_es, res_es, raw_res[r]);
+        if (p.res.row_scale) rs_res[r] = p.res.row_scale[rr];
+        if constexpr (HAS_BR) {
+          load_raw<VEC>(reinterpret_cast<const char*>(p.br.data) + (rb * p.br.ld + c0) * br_es, br_es, raw_br[r]);
+          if (p.br.row_scale) rs_br[r] = p.br.row_scale[rb];
+        }
+        if constexpr (HAS_EX)
+          load_raw<VEC>(reinterpret_cast<const char*>(p.ex.data) + (re * p.ex.ld + c0) * 2, 2, raw_ex[r]);
+      }
+    }
+
+    // ---- r = sum of the dequantized addends (fp32)
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (valid[r]) {
+        unpack<VEC>(raw_res[r], p.res.dt, x[r]);
+        if (p.res.dt == HERO_I8) {
+          if (p.res.col_scale) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) x[r][i] *= rs_res[r] * __ldg(p.res.col_scale + (c0 + i) * p.res.col_stride);
+          } else {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) x[r][i] *= rs_res[r];
+          }
+        }
+        if constexpr (HAS_BR) {
+          float b[VEC];
+          unpack<VEC>(raw_br[r], p.br.dt, b);
+          if (p.br.dt == HERO_I8) {
+            if (p.br.col_scale) {
+#pragma unroll
+              for (int i = 0; i < VEC; ++i)
+                x[r][i] = fmaf(b[i], rs_br[r] * __ldg(p.br.col_scale + (c0 + i) * p.br.col_stride), x[r][i]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < VEC; ++i) x[r][i] = fmaf(b[i], rs_br[r], x[r][i]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) x[r][i] += b[i];
+          }
+        }
+        if constexpr (HAS_EX) {
+          float e[VEC];
+          unpack<VEC>(raw_ex[r], p.ex.dt, e);
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) x[r][i] += e[i];
+        }
+        if (p.fp_out) {
+          // the FP residual stream carries the ROUNDED sum; normalise what is stored
+          uint32_t w[VEC / 2];
+#pragma unroll
+          for (int i = 0; i < VEC / 2; ++i) w[i] = pack_fp2(x[r][2 * i], x[r][2 * i + 1], p.fp_dt);
+          store_words<VEC>(reinterpret_cast<char*>(p.fp_out) + (row[r] * p.fp_ld + c0) * 2, w, VEC / 2);
+          unpack<VEC>(w, p.fp_dt, x[r]);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) x[r][i] = 0.f;
+      }
+    }
+    if (!normalize) continue;
+
+    // ---- mean, then centred (biased) variance, both over registers
+    float s[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float a = 0.f;
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) a += x[r][i];
+      s[r] = a;
+    }
+    row_reduce<R, false>(s, red0, G, row_in_cta, t);
+    float mean[R], rstd[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      mean[r] = s[r] * inv_H;
+      float a = 0.f;
+      if (active) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) { float d = x[r][i] - mean[r]; a = fmaf(d, d, a); }
+      }
+      s[r] = a;
+    }
+    row_reduce<R, false>(s, red1, G, row_in_cta, t);
+#pragma unroll
+    for (int r = 0; r < R; ++r) rstd[r] = 1.0f / sqrtf(s[r] * inv_H + p.eps);
+
+    // ---- y = (x - mean) * rstd * gamma + beta
+    float amax[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float m = 0.f;
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) {
+        float y = fmaf((x[r][i] - mean[r]) * rstd[r], gam[i], bet[i]);
+        x[r][i] = y;
+        m = fmaxf(m, fabsf(y));
+      }
+      amax[r] = m;
+    }
+
+    if (p.out_dt == HERO_I8) {
+      float inv[R];
+      if (p.out_gran == HERO_GRAN_TWQ) {
+        // Eq. 3: S[i] = absmax / 127 computed on the fly, in the same pass
+        row_reduce<R, true>(amax, red2, G, row_in_cta, t);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          float sc = amax[r] > 0.f ? amax[r] / 127.0f : 1.0f;
+          inv[r] = 1.0f / sc;
+          if (t == 0 && row[r] < p.M) p.out_scale[row[r]] = sc;
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (!valid[r]) continue;
+        uint32_t w[VEC / 4];
+        if (p.out_gran == HERO_GRAN_TWQ) {
+#pragma unroll
+          for (int i = 0; i < VEC / 4; ++i)
+            w[i] = quant4(x[r][4 * i] * inv[r], x[r][4 * i + 1] * inv[r], x[r][4 * i + 2] * inv[r], x[r][4 * i + 3] * inv[r]);
+        } else {
+          // Eq. 4 / 5: calibrated per-feature (stride 1) or static (stride 0) scale
+          const int st = (p.out_gran == HERO_GRAN_FWQ) ? 1 : 0;
+          float q[VEC];
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) q[i] = x[r][i] / __ldg(p.out_scale + (c0 + i) * st);
+#pragma unroll
+          for (int i = 0; i < VEC / 4; ++i) w[i] = quant4(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3]);
+        }
+        store_words<VEC>(reinterpret_cast<char*>(p.out) + row[r] * p.out_ld + c0, w, VEC / 4);
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (!valid[r]) continue;
+        uint32_t w[VEC / 2];
+#pragma unroll
+        for (int i = 0; i < VEC / 2; ++i) w[i] = pack_fp2(x[r][2 * i], x[r][2 * i + 1], p.out_dt);
+        store_words<VEC>(reinterpret_cast<char*>(p.out) + (row[r] * p.out_ld + c0) * 2, w, VEC / 2);
+      }
+    }
+  }
+}
+
+static hero_status fill_side(const hero_tensor& t, LnSide* s, const char* name, bool allow_i8, int H) {
+  s->data = nullptr; s->dt = HERO_F16; s->ld = 0; s->row_scale = nullptr; s->col_scale = nullptr; s->col_stride = 0;
+  if (t.data == nullptr) return HERO_OK;
+  hero_status st = check_matrix(t, name);
+  if (st != HERO_OK) return st;
+  HERO_REQUIRE(t.cols == H, HERO_ERR_INVALID_ARG, "%s: cols %lld != H %d", name, (long long)t.cols, H);
+  HERO_REQUIRE(is_fp16ish(t.dtype) || (allow_i8 && t.dtype == HERO_I8), HERO_ERR_UNSUPPORTED,
+               "%s: dtype %d not accepted here", name, t.dtype);
+  s->data = t.data; s->dt = t.dtype; s->ld = t.ld;
+  if (t.dtype == HERO_I8) {
+    if (t.gran == HERO_GRAN_TWQ) s->row_scale = t.scale;
+    if (t.gran == HERO_GRAN_FWQ) { s->col_scale = t.scale; s->col_stride = 1; }
+    if (t.gran == HERO_GRAN_SQ) { s->col_scale = t.scale; s->col_stride = 0; }
+  }
+  return HERO_OK;
+}
+
+template <int VEC, int R, bool HAS_BR, bool HAS_EX>
+static hero_status launch_ln2(hero_handle* h, LnParams& p, cudaStream_t stream) {
+  const int chunks = (p.H + VEC - 1) / VEC;
+  p.G = ((chunks + 31) / 32) * 32;
+  p.RPC = p.G >= 256 ? 1 : 256 / p.G;
+  const int threads = p.G * p.RPC;
+  const size_t smem = (size_t)3 * p.RPC * R * (p.G / 32) * sizeof(float);
+  const long long rows_per_trip = (long long)p.RPC * R;
+  long long want = (p.M + rows_per_trip - 1) / rows_per_trip;
+  // a few CTAs per SM, persistent over the rows
+  int occ = 1;
+  HERO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, ln_quant_kernel<VEC, R, HAS_BR, HAS_EX>, threads, smem));
+  if (occ < 1) occ = 1;
+  long long cap = (long long)h->sm_count * occ;
+  int grid = (int)(want < cap ? want : cap);
+  if (grid < 1) grid = 1;
+  ln_quant_kernel<VEC, R, HAS_BR, HAS_EX><<<grid, threads, smem, stream>>>(p);
+  HERO_CUDA(cudaGetLastError());
+  h->launches += 1;
+  return HERO_OK;
+}
+
+template <int VEC, int R>
+static hero_status launch_ln(hero_handle* h, LnParams& p, cudaStream_t stream) {
+  if (p.ex.data) return launch_ln2<VEC, R, true, true>(h, p, stream);   // embedding flavour: three addends
+  if (p.br.data) return launch_ln2<VEC, R, true, false>(h, p, stream);  // residual flavour: two addends
+  return launch_ln2<VEC, R, false, false>(h, p, stream);                // plain flavour
+}
+
+
+__device__ __forceinline__ void st_global8(void* p, uint32_t a, uint32_t b) {
+  asm volatile("st.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ void st_global16(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// =====================================================================================================
+// Fast path: types fixed at compile time, a row owned by WPR whole warps (H <= 1024 * WPR), each lane
+// holding up to four 8-element chunks.  INT8 payloads are turned into floats with byte permutes and an
+// exact float subtraction (no I2F), and the TWQ output is rounded with the 1.5 * 2^23 magic constant
+// inside one FMA (no F2I): both keep the per-element instruction count low enough for the kernel to
+// stay memory-bound.  gamma / beta / per-feature scales come through L1.
+// =====================================================================================================
+constexpr int SRC_NONE = 0, SRC_I8 = 1, SRC_FP = 2;
+constexpr int O_NONE = 0, O_TWQ = 1, O_STATIC = 2, O_FP = 3;
+constexpr int LNF_THREADS = 256;
+constexpr int LNF_MAXCH = 4;
+
+__device__ __forceinline__ void ldg8(const void* p, uint32_t& a, uint32_t& b) {
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(a), "=r"(b) : "l"(p));
+}
+__device__ __forceinline__ void ldg16(const void* p, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "l"(p));
+}
+__device__ __forceinline__ float4 ldg_f4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+
+// 8 INT8 codes (two words) -> 8 exact floats
+__device__ __forceinline__ void i8x8_to_float(uint32_t w0, uint32_t w1, float (&v)[8]) {
+  w0 ^= 0x80808080u; w1 ^= 0x80808080u;           // code + 128 in [1, 255]
+  const float off = 8388736.0f;                   // 2^23 + 128
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    v[b] = __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7440 | b)) - off;
+    v[4 + b] = __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7440 | b)) - off;
+  }
+}
+__device__ __forceinline__ void fp16x8_to_float(const uint32_t (&w)[4], int dt, float (&v)[8]) {
+  if (dt == HERO_F16) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+      v[2 * i] = f.x; v[2 * i + 1] = f.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+}
+// Round-half-to-even of |v| <= 127.x through the float adder, low byte = two's complement code
+__device__ __forceinline__ uint32_t magic_bits(float v_plus_magic) { return __float_as_uint(v_plus_magic); }
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  uint32_t ab = __byte_perm(a, b, 0x0040);        // bytes: a0, b0
+  uint32_t cd = __byte_perm(c, d, 0x0040);
+  return __byte_perm(ab, cd, 0x5410);
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int LNF_STAGES = 3;   // rows in flight per row slot (each lane prefetches its own chunks)
+
+template <int RES, int BR, bool EX, int OUT, bool FPOUT>
+__global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams p) {
+  __shared__ float red[3][8][8];                  // [statistic][row slot][warp in row]
+  extern __shared__ __align__(16) uint8_t ring[]; // [stage][row slot][res row | branch row | extra row]
+  const int WPR = p.G;                            // warps per row: 1, 2, 4 or 8
+  const int slots = 8 / WPR;                      // rows per CTA pass
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int slot = warp / WPR, wr = warp - slot * WPR;
+  const int nchunks = p.H >> 3;
+  const int stride = WPR * 32;                    // chunk stride between a lane's chunks
+  const int c_first = wr * 32 + lane;
+  const float inv_H = 1.0f / (float)p.H;
+  const float MAGIC = 12582912.0f;                // 1.5 * 2^23
+  constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2;
+  constexpr int ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
+  const int off_br = p.H * ES_RES;
+  const int off_ex = off_br + p.H * ES_BR;
+  const int slot_bytes = off_ex + (EX ? p.H * 2 : 0);
+  const int stage_bytes = slot_bytes * slots;
+
+  // A lane copies exactly the chunks it will later read, so waiting on its own copy groups is all
+  // the synchronisation the ring needs.
+  auto prefetch = [&](long long row, int st) {
+    if (row < p.M) {
+      long long r_res = row, r_br = row, r_ex = row;
+      if (p.token_ids) {
+        r_res = p.token_ids[row];
+        r_br = row % p.seq_len;
+        r_ex = p.type_ids ? p.type_ids[row] : 0;
+      }
+      uint8_t* dst = ring + st * stage_bytes + slot * slot_bytes;
+#pragma unroll
+      for (int k = 0; k < LNF_MAXCH; ++k) {
+        const int c = c_first + k * stride;
+        if (c < nchunks) {
+          if constexpr (RES == SRC_I8) cp_async8(dst + c * 8, reinterpret_cast<const char*>(p.res.data) + r_res * p.res.ld + c * 8);
+          else cp_async16(dst + c * 16, reinterpret_cast<const char*>(p.res.data) + (r_res * p.res.ld + c * 8) * 2);
+          if constexpr (BR == SRC_I8) cp_async8(dst + off_br + c * 8, reinterpret_cast<const char*>(p.br.data) + r_br * p.br.ld + c * 8);
+          if constexpr (BR == SRC_FP) cp_async16(dst + off_br + c * 16, reinterpret_cast<const char*>(p.br.data) + (r_br * p.br.ld + c * 8) * 2);
+          if constexpr (EX) cp_async16(dst + off_ex + c * 16, reinterpret_cast<const char*>(p.ex.data) + (r_ex * p.ex.ld + c * 8) * 2);
+        }
+      }
+    }
+    cp_async_commit();
+  };
+
+  const long long row_step = (long long)gridDim.x * slots;
+  const long long first = (long long)blockIdx.x * slots;
+#pragma unroll
+  for (int s0 = 0; s0 < LNF_STAGES - 1; ++s0) prefetch(first + s0 * row_step + slot, s0);
+
+  int st = 0;
+  for (long long base = first; base < p.M; base += row_step) {
+    const long long row = base + slot;
+    const bool row_ok = row < p.M;
+    {
+      int pst = st + LNF_STAGES - 1;
+      if (pst >= LNF_STAGES) pst -= LNF_STAGES;
+      prefetch(row + (LNF_STAGES - 1) * row_step, pst);
+    }
+    cp_async_wait<LNF_STAGES - 1>();
+    const uint8_t* src = ring + st * stage_bytes + slot * slot_bytes;
+    if (++st == LNF_STAGES) st = 0;
+
+    float x[LNF_MAXCH][8];
+    float rs_res = 1.f, rs_br = 1.f;
+    if (row_ok) {
+      long long r_res = row, r_br = row;
+      if (p.token_ids) { r_res = p.token_ids[row]; r_br = row % p.seq_len; }
+      if (RES == SRC_I8 && p.res.row_scale) rs_res = __ldg(p.res.row_scale + r_res);
+      if (BR == SRC_I8 && p.br.row_scale) rs_br = __ldg(p.br.row_scale + r_br);
+    }
+
+    // ---- r = sum of the dequantized addends; running row sum
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < LNF_MAXCH; ++k) {
+      const int c = c_first + k * stride;
+      if (row_ok && c < nchunks) {
+        if constexpr (RES == SRC_I8) {
+          const uint2 w = *reinterpret_cast<const uint2*>(src + c * 8);
+          i8x8_to_float(w.x, w.y, x[k]);
+          if (p.res.col_scale) {
+            float sc[8];
+            if (p.res.col_stride) {
+              float4 a = ldg_f4(p.res.col_scale + c * 8), b = ldg_f4(p.res.col_scale + c * 8 + 4);
+              sc[0] = a.x; sc[1] = a.y; sc[2] = a.z; sc[3] = a.w; sc[4] = b.x; sc[5] = b.y; sc[6] = b.z; sc[7] = b.w;
+            } else {
+              const float v = __ldg(p.res.col_scale);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) sc[i] = v;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[k][i] *= rs_res * sc[i];
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[k][i] *= rs_res;
+          }
+        } else {
+          const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+          fp16x8_to_float(ww, p.res.dt, x[k]);
+        }
+        if constexpr (BR == SRC_I8) {
+          float b[8];
+          const uint2 wb = *reinterpret_cast<const uint2*>(src + off_br + c * 8);
+          i8x8_to_float(wb.x, wb.y, b);
+          if (p.br.col_scale) {
+            float sc[8];
+            if (p.br.col_stride) {
+              float4 a = ldg_f4(p.br.col_scale + c * 8), bb = ldg_f4(p.br.col_scale + c * 8 + 4);
+              sc[0] = a.x; sc[1] = a.y; sc[2] = a.z; sc[3] = a.w; sc[4] = bb.x; sc[5] = bb.y; sc[6] = bb.z; sc[7] = bb.w;
+            } else {
+              const float v = __ldg(p.br.col_scale);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) sc[i] = v;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[k][i] = fmaf(b[i], rs_br * sc[i], x[k][i]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[k][i] = fmaf(b[i], rs_br, x[k][i]);
+          }
+        }
+        if constexpr (BR == SRC_FP) {
+          float b[8];
+          const uint4 wb = *reinterpret_cast<const uint4*>(src + off_br + c * 16);
+          const uint32_t wwb[4] = {wb.x, wb.y, wb.z, wb.w};
+          fp16x8_to_float(wwb, p.br.dt, b);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[k][i] += b[i];
+        }
+        if constexpr (EX) {
+          float e[8];
+          const uint4 we = *reinterpret_cast<const uint4*>(src + off_ex + c * 16);
+          const uint32_t wwe[4] = {we.x, we.y, we.z, we.w};
+          fp16x8_to_float(wwe, p.ex.dt, e);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[k][i] += e[i];
+        }
+        if constexpr (FPOUT) {
+          // the FP residual stream carries the ROUNDED sum; normalise what is stored
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) w[i] = pack_fp2(x[k][2 * i], x[k][2 * i + 1], p.fp_dt);
+          st_global16(reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + c * 8) * 2, w[0], w[1], w[2], w[3]);
+          fp16x8_to_float(w, p.fp_dt, x[k]);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s += x[k][i];
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[k][i] = 0.f;
+      }
+    }
+    if constexpr (OUT == O_NONE) continue;
+
+    // ---- mean
+    s = warp_sum(s);
+    if (WPR > 1) {
+      if (lane == 0) red[0][slot][wr] = s;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(stride) : "memory");
+      s = 0.f;
+      for (int w = 0; w < WPR; ++w) s += red[0][slot][w];
+    }
+    const float mean = s * inv_H;
+    // ---- centred (biased) variance over the registers
+    float q = 0.f;
+#pragma unroll
+    for (int k = 0; k < LNF_MAXCH; ++k) {
+      if (c_first + k * stride < nchunks) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { x[k][i] -= mean; q = fmaf(x[k][i], x[k][i], q); }
+      }
+    }
+    q = warp_sum(q);
+    if (WPR > 1) {
+      if (lane == 0) red[1][slot][wr] = q;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(stride) : "memory");
+      q = 0.f;
+      for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
+    }
+    const float rstd = 1.0f / sqrtf(q * inv_H + p.eps);
+
+    // ---- y = d * (rstd * gamma) + beta ; TWQ: row absmax in the same sweep
+    float amax = 0.f;
+#pragma unroll
+    for (int k = 0; k < LNF_MAXCH; ++k) {
+      const int c = c_first + k * stride;
+      if (c < nchunks) {
+        float4 g0 = ldg_f4(p.gamma + c * 8), g1 = ldg_f4(p.gamma + c * 8 + 4);
+        float4 b0 = ldg_f4(p.beta + c * 8), b1 = ldg_f4(p.beta + c * 8 + 4);
+        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+        const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          x[k][i] = fmaf(x[k][i], rstd * g[i], b[i]);
+          if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fabsf(x[k][i]));
+        }
+      }
+    }
+
+    if constexpr (OUT == O_TWQ) {
+      // Eq. 3: S[i] = absmax / 127 on the fly; the scaled value never leaves [-127, 127], so the magic add
+      // alone rounds and range-limits it
+      amax = warp_max(amax);
+      if (WPR > 1) {
+        if (lane == 0) red[2][slot][wr] = amax;
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(stride) : "memory");
+        amax = 0.f;
+        for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
+      }
+      const float sc = amax > 0.f ? amax / 127.0f : 1.0f;
+      const float inv = 1.0f / sc;
+      if (row_ok && wr == 0 && lane == 0) p.out_scale[row] = sc;
+#pragma unroll
+      for (int k = 0; k < LNF_MAXCH; ++k) {
+        const int c = c_first + k * stride;
+        if (row_ok && c < nchunks) {
+          uint32_t u[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) u[i] = magic_bits(fmaf(x[k][i], inv, MAGIC));
+          st_global8(reinterpret_cast<char*>(p.out) + row * p.out_ld + c * 8, pack_low_bytes(u[0], u[1], u[2], u[3]),
+                     pack_low_bytes(u[4], u[5], u[6], u[7]));
+        }
+      }
+    } else if constexpr (OUT == O_STATIC) {
+      // Eq. 4 / 5: calibrated per-feature (stride 1) or static (stride 0) scale; saturating
+#pragma unroll
+      for (int k = 0; k < LNF_MAXCH; ++k) {
+        const int c = c_first + k * stride;
+        if (row_ok && c < nchunks) {
+          float sc[8];
+          if (p.out_gran == HERO_GRAN_FWQ) {
+            float4 a = ldg_f4(p.out_scale + c * 8), b = ldg_f4(p.out_scale + c * 8 + 4);
+            sc[0] = a.x; sc[1] = a.y; sc[2] = a.z; sc[3] = a.w; sc[4] = b.x; sc[5] = b.y; sc[6] = b.z; sc[7] = b.w;
+          } else {
+            const float v = __ldg(p.out_scale);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sc[i] = v;
+          }
+          uint32_t u[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float v = fminf(fmaxf(x[k][i] / sc[i], -127.f), 127.f);
+            u[i] = magic_bits(v + MAGIC);
+          }
+          st_global8(reinterpret_cast<char*>(p.out) + row * p.out_ld + c * 8, pack_low_bytes(u[0], u[1], u[2], u[3]),
+                     pack_low_bytes(u[4], u[5], u[6], u[7]));
+        }
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < LNF_MAXCH; ++k) {
+        const int c = c_first + k * stride;
+        if (row_ok && c < nchunks) {
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) w[i] = pack_fp2(x[k][2 * i], x[k][2 * i + 1], p.out_dt);
+          st_global16(reinterpret_cast<char*>(p.out) + (row * p.out_ld + c * 8) * 2, w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+  }
+}
+
+template <int RES, int BR, bool EX, int OUT, bool FPOUT>
+static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream) {
+  int wpr = 1;
+  while (wpr * 1024 < p.H) wpr *= 2;
+  p.G = wpr;
+  const int slots = 8 / wpr;
+  const long long want = (p.M + slots - 1) / slots;
+  const int es_res = (RES == SRC_I8) ? 1 : 2, es_br = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
+  const size_t smem = (size_t)LNF_STAGES * slots * p.H * (es_res + es_br + (EX ? 2 : 0));
+  auto kern = ln_fast_kernel<RES, BR, EX, OUT, FPOUT>;
+  static bool configured = false;   // per instantiation
+  if (!configured) {
+    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+    configured = true;
+  }
+  int occ = 1;
+  HERO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, LNF_THREADS, smem));
+  if (occ < 1) occ = 1;
+  const long long cap = (long long)h->sm_count * occ;
+  const int grid = (int)(want < cap ? want : cap);
+  kern<<<grid, LNF_THREADS, smem, stream>>>(p);
+  HERO_CUDA(cudaGetLastError());
+  h->launches += 1;
+  return HERO_OK;
+}
+
+// Returns HERO_ERR_UNSUPPORTED (without setting an error) when the combination has no fast instantiation.
+static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
+  *taken = false;
+  if (p.H % 8 != 0 || p.H > 8192) return HERO_OK;
+  const int res = p.res.dt == HERO_I8 ? SRC_I8 : SRC_FP;
+  const int br = !p.br.data ? SRC_NONE : (p.br.dt == HERO_I8 ? SRC_I8 : SRC_FP);
+  const bool ex = p.ex.data != nullptr;
+  const int out = !p.out ? O_NONE : (p.out_dt != HERO_I8 ? O_FP : (p.out_gran == HERO_GRAN_TWQ ? O_TWQ : O_STATIC));
+  const bool fpo = p.fp_out != nullptr;
+  if (res == SRC_I8 && p.res.row_scale && p.res.col_scale) return HERO_OK;
+#define LNF_CASE(R_, B_, E_, O_, F_)                                                   \
+  if (res == R_ && br == B_ && ex == E_ && out == O_ && fpo == F_) {                   \
+    *taken = true;                                                                     \
+    return launch_fast<R_, B_, E_, O_, F_>(h, p, s);                                   \
+  }
+#define LNF_OUTS(R_, B_, E_, F_) LNF_CASE(R_, B_, E_, O_TWQ, F_) LNF_CASE(R_, B_, E_, O_STATIC, F_) LNF_CASE(R_, B_, E_, O_FP, F_)
+  LNF_OUTS(SRC_FP, SRC_NONE, false, false)   // entry LN^quant on FP activations; pre-LN LN1
+  LNF_OUTS(SRC_I8, SRC_I8, false, false)     // Eq. 19 / 31: two INT8 addends
+  LNF_OUTS(SRC_I8, SRC_FP, false, false)     // INT8 residual + FP branch (modes M1 / M2)
+  LNF_OUTS(SRC_FP, SRC_FP, false, false)     // all-FP modules
+  LNF_OUTS(SRC_FP, SRC_I8, false, false)     // FP residual + INT8 branch
+  LNF_OUTS(SRC_FP, SRC_I8, false, true)      // pre-LN: add + LN + quant, new residual stream stored
+  LNF_OUTS(SRC_FP, SRC_FP, false, true)
+  LNF_CASE(SRC_FP, SRC_I8, false, O_NONE, true)   // closing residual add of a lone pre-LN layer
+  LNF_CASE(SRC_FP, SRC_FP, false, O_NONE, true)
+  LNF_OUTS(SRC_I8, SRC_FP, true, false)      // Eq. 7: embedding gather, three addends
+#undef LNF_OUTS
+#undef LNF_CASE
+  return HERO_OK;
+}
+
+}  // namespace hero
+
+extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* a, void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(h && a, HERO_ERR_INVALID_ARG, "hero_layernorm_quant: NULL handle or args");
+  LnParams p;
+  memset(&p, 0, sizeof(p));
+  const bool gather = a->token_ids != nullptr;
+  HERO_REQUIRE(a->residual.data != nullptr || (!gather && a->residual.rows == 0), HERO_ERR_INVALID_ARG, "residual is required");
+  if (!gather && a->residual.rows == 0) return HERO_OK;
+  const int H = (int)a->residual.cols;
+  HERO_REQUIRE(H > 0 && H % 16 == 0 && H <= 16384, HERO_ERR_UNSUPPORTED, "H=%d must be a multiple of 16, at most 16384", H);
+  hero_status st;
+  if ((st = fill_side(a->residual, &p.res, "residual", true, H)) != HERO_OK) return st;
+  if ((st = fill_side(a->branch, &p.br, "branch", true, H)) != HERO_OK) return st;
+  if ((st = fill_side(a->extra, &p.ex, "extra", false, H)) != HERO_OK) return st;
+  p.M = gather ? a->n_tokens : a->residual.rows;
+  HERO_REQUIRE(p.M >= 0, HERO_ERR_INVALID_ARG, "negative row count");
+  if (gather) {
+    HERO_REQUIRE(a->residual.dtype == HERO_I8 && a->residual.gran == HERO_GRAN_TWQ, HERO_ERR_UNSUPPORTED,
+                 "embedding gather: the token table must be INT8 with one scale per row (Eq. 7)");
+    HERO_REQUIRE(a->seq_len > 0, HERO_ERR_INVALID_ARG, "embedding gather: seq_len must be positive");
+    HERO_REQUIRE(a->extra.data == nullptr || a->type_ids != nullptr, HERO_ERR_INVALID_ARG,
+                 "embedding gather: type_ids required with a sentence-type table");
+    p.token_ids = a->token_ids; p.type_ids = a->type_ids; p.seq_len = a->seq_len;
+  } else {
+    HERO_REQUIRE(a->branch.data == nullptr || a->branch.rows == p.M, HERO_ERR_INVALID_ARG, "branch rows differ");
+    HERO_REQUIRE(a->extra.data == nullptr || a->extra.rows == p.M, HERO_ERR_INVALID_ARG, "extra rows differ");
+    HERO_REQUIRE(a->extra.data == nullptr || a->branch.data != nullptr, HERO_ERR_INVALID_ARG,
+                 "extra (third addend) given without branch (second addend)");
+  }
+  p.H = H;
+  p.gamma = a->gamma; p.beta = a->beta; p.eps = a->eps;
+  if (a->out.data) {
+    if ((st = check_matrix(a->out, "out")) != HERO_OK) return st;
+    HERO_REQUIRE(a->gamma && a->beta, HERO_ERR_INVALID_ARG, "gamma and beta are required");
+    HERO_REQUIRE(aligned16(a->gamma) && aligned16(a->beta), HERO_ERR_ALIGNMENT, "gamma/beta must be 16-byte aligned");
+    HERO_REQUIRE(a->out.rows == p.M && a->out.cols == H, HERO_ERR_INVALID_ARG, "out shape mismatch");
+    HERO_REQUIRE(a->out.dtype == HERO_I8 || is_fp16ish(a->out.dtype), HERO_ERR_UNSUPPORTED, "out dtype %d", a->out.dtype);
+    if (a->out.dtype == HERO_I8)
+      HERO_REQUIRE(a->out.gran == HERO_GRAN_TWQ || a->out.gran == HERO_GRAN_FWQ || a->out.gran == HERO_GRAN_SQ,
+                   HERO_ERR_INVALID_ARG, "INT8 out needs granularity TWQ, FWQ or SQ");
+    p.out = a->out.data; p.out_dt = a->out.dtype; p.out_ld = a->out.ld; p.out_gran = a->out.gran;
+    p.out_scale = a->out.scale;
+  }
+  if (a->fp_out.data) {
+    if ((st = check_matrix(a->fp_out, "fp_out")) != HERO_OK) return st;
+    HERO_REQUIRE(is_fp16ish(a->fp_out.dtype), HERO_ERR_UNSUPPORTED, "fp_out must be F16 or BF16");
+    HERO_REQUIRE(a->fp_out.rows == p.M && a->fp_out.cols == H, HERO_ERR_INVALID_ARG, "fp_out shape mismatch");
+    p.fp_out = a->fp_out.data; p.fp_dt = a->fp_out.dtype; p.fp_ld = a->fp_out.ld;
+  }
+  HERO_REQUIRE(p.out || p.fp_out, HERO_ERR_INVALID_ARG, "neither out nor fp_out given");
+  if (p.M == 0) return HERO_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  bool taken = false;
+  st = try_fast(h, p, s, &taken);
+  if (taken || st != HERO_OK) return st;
+  // generic kernel for the remaining combinations.
+  // 16 elements per thread when rows are long (fewer, fatter threads); 8 otherwise.  VEC=16 needs H % 16 == 0.
+  if (H % 16 == 0 && H >= 2048) return launch_ln<16, 1>(h, p, s);
+  return launch_ln<8, 2>(h, p, s);
+}

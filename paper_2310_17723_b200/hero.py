@@ -1,0 +1,204 @@
+"""ctypes binding of include/hero.h.  Marshals arguments; every step runs in libhero.so.
+
+Tensors are torch CUDA tensors used purely as device buffers (data_ptr / shape / stride); the
+stream is torch's current CUDA stream unless one is passed.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libhero.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(7)
+I8, U8, I32, F16, BF16, F32 = range(6)
+GRAN_NONE, GRAN_TWQ, GRAN_FWQ, GRAN_SQ = range(4)
+ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH = range(3)
+MASK_NONE, MASK_CAUSAL = range(2)
+POST_LN, PRE_LN = range(2)
+MODE_INT8, MODE_FP = range(2)
+PRESET_FP, PRESET_M1, PRESET_M2, PRESET_M3 = range(4)
+MODULES = ("qkv", "attn", "attn_out", "fc1", "fc2")
+
+_DT = {torch.int8: I8, torch.uint8: U8, torch.int32: I32, torch.float16: F16, torch.bfloat16: BF16,
+       torch.float32: F32}
+GRAN = {"none": GRAN_NONE, "twq": GRAN_TWQ, "fwq": GRAN_FWQ, "sq": GRAN_SQ, "fp": GRAN_NONE}
+ACT = {"none": ACT_NONE, "gelu_erf": ACT_GELU_ERF, "gelu_tanh": ACT_GELU_TANH}
+MASK = {"none": MASK_NONE, "causal": MASK_CAUSAL}
+FPDT = {"f16": F16, "bf16": BF16}
+TORCH_FP = {"f16": torch.float16, "bf16": torch.bfloat16}
+
+
+class HeroError(RuntimeError):
+    def __init__(self, status, msg):
+        super().__init__("hero status %d: %s" % (status, msg))
+        self.status = status
+
+
+class Tensor(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("dtype", C.c_int32), ("gran", C.c_int32), ("rows", C.c_int64),
+                ("cols", C.c_int64), ("ld", C.c_int64), ("scale", C.c_void_p)]
+
+
+class LnArgs(C.Structure):
+    _fields_ = [("residual", Tensor), ("branch", Tensor), ("extra", Tensor), ("token_ids", C.c_void_p),
+                ("type_ids", C.c_void_p), ("seq_len", C.c_int32), ("n_tokens", C.c_int64), ("gamma", C.c_void_p),
+                ("beta", C.c_void_p), ("eps", C.c_float), ("out", Tensor), ("fp_out", Tensor)]
+
+
+class LinearArgs(C.Structure):
+    _fields_ = [("A", Tensor), ("W", C.c_void_p), ("N", C.c_int64), ("ldw", C.c_int64), ("w_scale", C.c_void_p),
+                ("bias", C.c_void_p), ("act", C.c_int32), ("post_scale", C.c_void_p), ("out", Tensor)]
+
+
+class AttnArgs(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("dtype", C.c_int32), ("ld", C.c_int64),
+                ("B", C.c_int32), ("S", C.c_int32), ("nh", C.c_int32), ("dh", C.c_int32), ("s_q", C.c_float),
+                ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float), ("mask", C.c_int32),
+                ("key_len", C.c_void_p), ("out", Tensor)]
+
+
+class LinearParams(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("w_scale", C.c_void_p), ("bias", C.c_void_p), ("post_scale", C.c_void_p)]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("arch", C.c_int32), ("B", C.c_int32), ("S", C.c_int32), ("H", C.c_int32), ("nh", C.c_int32),
+                ("F", C.c_int32), ("act", C.c_int32), ("eps", C.c_float), ("mask", C.c_int32),
+                ("fp_dtype", C.c_int32), ("mode", C.c_int32 * 5), ("gran_in", C.c_int32), ("gran_mid", C.c_int32),
+                ("gran_attn", C.c_int32), ("gran_out", C.c_int32), ("s_in", C.c_void_p), ("s_mid", C.c_void_p),
+                ("s_attn", C.c_void_p), ("s_o", C.c_void_p), ("s_x2", C.c_void_p), ("s_out", C.c_void_p),
+                ("s_q", C.c_float), ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float),
+                ("qkv", LinearParams), ("o", LinearParams), ("fc1", LinearParams), ("fc2", LinearParams),
+                ("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p)]
+
+
+EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
+           "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
+           "hero_layer_workspace_bytes", "hero_layer_forward")
+
+_lib = None
+
+
+def lib():
+    """The loaded CUDA library.  Missing library = hard error (there is no other implementation)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("libhero.so is not built (%s); run `python -m paper_2310_17723_b200.build`. "
+                               "There is no fallback path." % _LIB_PATH)
+        L = C.CDLL(_LIB_PATH)
+        L.hero_last_error.restype = C.c_char_p
+        L.hero_launch_count.restype = C.c_int64
+        L.hero_launch_count.argtypes = [C.c_void_p]
+        L.hero_create.argtypes = [C.POINTER(C.c_void_p)]
+        L.hero_destroy.argtypes = [C.c_void_p]
+        L.hero_check.argtypes = [C.c_void_p, C.c_void_p]
+        L.hero_layernorm_quant.argtypes = [C.c_void_p, C.POINTER(LnArgs), C.c_void_p]
+        L.hero_w8a8_linear.argtypes = [C.c_void_p, C.POINTER(LinearArgs), C.c_void_p]
+        L.hero_int8_attention.argtypes = [C.c_void_p, C.POINTER(AttnArgs), C.c_void_p]
+        L.hero_mode_preset.argtypes = [C.c_int32, C.POINTER(C.c_int32 * 5)]
+        L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
+        L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
+                                         C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _check(status):
+    if status != OK:
+        raise HeroError(status, lib().hero_last_error().decode())
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def tensor(t, gran="none", scale=None):
+    """hero_tensor view of a 2-D torch CUDA tensor (row-major, unit inner stride); None -> absent."""
+    if t is None:
+        return Tensor(None, 0, 0, 0, 0, 0, None)
+    assert t.is_cuda and t.dim() == 2 and t.stride(1) == 1, "need a 2-D row-major CUDA tensor"
+    if scale is not None:
+        assert scale.is_cuda and scale.dtype == torch.float32 and scale.is_contiguous()
+    g = GRAN[gran] if isinstance(gran, str) else gran
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+    T = Tensor(t.data_ptr(), _DT[t.dtype], g, t.shape[0], t.shape[1], ld, None if scale is None else scale.data_ptr())
+    T._keep = (t, scale)      # the struct holds raw pointers: keep the buffers alive as long as it lives
+    return T
+
+
+class Handle:
+    """Owns a hero_handle on the current CUDA device."""
+
+    def __init__(self):
+        if not torch.cuda.is_available():
+            raise RuntimeError("hero needs a CUDA device (sm_100a); none is visible")
+        self._h = C.c_void_p()
+        _check(lib().hero_create(C.byref(self._h)))
+
+    def close(self):
+        if self._h:
+            lib().hero_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def check(self, stream=None):
+        _check(lib().hero_check(self._h, _stream(stream)))
+
+    @property
+    def launches(self):
+        return int(lib().hero_launch_count(self._h))
+
+    # ---- the four calls of the boundary, same names as the C entry points ----
+    def hero_layernorm_quant(self, residual, gamma, beta, eps, out, branch=None, extra=None, fp_out=None,
+                             token_ids=None, type_ids=None, seq_len=0, n_tokens=0, stream=None):
+        """residual / branch / extra / out / fp_out are hero.Tensor structs (see `tensor`)."""
+        a = LnArgs(residual, branch or tensor(None), extra or tensor(None), _ptr(token_ids), _ptr(type_ids),
+                   int(seq_len), int(n_tokens), _ptr(gamma), _ptr(beta), float(eps), out or tensor(None),
+                   fp_out or tensor(None))
+        _check(lib().hero_layernorm_quant(self._h, C.byref(a), _stream(stream)))
+
+    def hero_w8a8_linear(self, A, W, out, w_scale=None, bias=None, act="none", post_scale=None, stream=None):
+        """A, out: hero.Tensor; W: torch tensor [N, K] (K contiguous)."""
+        assert W.dim() == 2 and W.stride(1) == 1
+        a = LinearArgs(A, W.data_ptr(), W.shape[0], W.stride(0), _ptr(w_scale), _ptr(bias),
+                       ACT[act] if isinstance(act, str) else act, _ptr(post_scale), out)
+        _check(lib().hero_w8a8_linear(self._h, C.byref(a), _stream(stream)))
+
+    def hero_int8_attention(self, q, k, v, B, S, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0, s_p=1.0 / 255,
+                            mask="none", key_len=None, stream=None):
+        """q, k, v: 2-D torch views [B*S, nh*dh] sharing one leading dimension; out: hero.Tensor."""
+        assert q.stride(0) == k.stride(0) == v.stride(0) and q.dtype == k.dtype == v.dtype
+        a = AttnArgs(q.data_ptr(), k.data_ptr(), v.data_ptr(), _DT[q.dtype], q.stride(0), B, S, nh, dh, s_q, s_k,
+                     s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out)
+        _check(lib().hero_int8_attention(self._h, C.byref(a), _stream(stream)))
+
+    def hero_layer_workspace_bytes(self, desc, M):
+        n = C.c_size_t()
+        _check(lib().hero_layer_workspace_bytes(C.byref(desc), int(M), C.byref(n)))
+        return int(n.value)
+
+    def hero_layer_forward(self, desc, x_in, out, workspace, pending=None, stream=None):
+        """x_in / out / pending: hero.Tensor; workspace: 1-D torch uint8 CUDA tensor."""
+        pend = C.byref(pending) if pending is not None else None
+        _check(lib().hero_layer_forward(self._h, C.byref(desc), C.byref(x_in), pend, C.byref(out),
+                                        C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)))
+
+
+def mode_preset(preset):
+    m = (C.c_int32 * 5)()
+    _check(lib().hero_mode_preset(int(preset), C.byref(m)))
+    return list(m)

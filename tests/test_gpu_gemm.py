@@ -1,0 +1,150 @@
+"""GPU parity: hero_w8a8_linear against the oracle's GeMM^quant (Eq. 14, 18, 22, 28-30)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ops as O
+from oracle import quant as Q
+from paper_2310_17723_b200 import hero, workloads as W
+from gpu_util import dev, f32, assert_int8_close, rel_err, TORCH_FP
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def h():
+    hd = hero.Handle()
+    yield hd
+    hd.check()
+    hd.close()
+
+
+def _linear(h, A, Wt, out_dtype, rs=None, cs=None, bias=None, act="none", post=None, N=None):
+    M = A.shape[0]
+    N = Wt.shape[0]
+    tA = dev(A) if A.dtype == np.int8 else A
+    tW = dev(Wt) if isinstance(Wt, np.ndarray) else Wt
+    out = torch.full((M, N), -77, dtype=out_dtype, device="cuda") if out_dtype in (torch.int8, torch.int32) else \
+        torch.full((M, N), float("nan"), dtype=out_dtype, device="cuda")
+    a_desc = hero.tensor(tA, "twq", f32(rs)) if rs is not None else hero.tensor(tA)
+    h.hero_w8a8_linear(a_desc, tW, hero.tensor(out), w_scale=None if cs is None else f32(cs),
+                       bias=None if bias is None else f32(bias), act=act, post_scale=None if post is None else f32(post))
+    h.check()
+    return out
+
+
+# shapes span one tile, several tiles, ragged M / N / K tails and every column-tile width
+SHAPES = [(128, 128, 256), (1, 64, 16), (17, 80, 48), (127, 256, 272), (129, 1024, 512), (300, 768, 2304),
+          (1000, 4096, 1024), (2500, 512, 4096), (16, 4096, 4096)]
+
+
+@pytest.mark.parametrize("M,K,N", SHAPES)
+def test_int32_accumulators_bit_exact(h, M, K, N):
+    g = W.rng(2, 1000 + M + K + N)
+    A = g.integers(-127, 128, (M, K), dtype=np.int8)
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    got = _linear(h, A, Wt, torch.int32).cpu().numpy()
+    want = O.int_matmul(A, Wt.T.copy())
+    assert np.array_equal(got, want)
+
+
+def test_int32_extreme_values_bit_exact(h):
+    M, K, N = 130, 16384, 64
+    A = np.full((M, K), 127, np.int8)
+    Wt = np.full((N, K), -127, np.int8)
+    Wt[1::2] = 127
+    got = _linear(h, A, Wt, torch.int32).cpu().numpy()
+    assert np.array_equal(got, O.int_matmul(A, Wt.T.copy()))
+
+
+@pytest.mark.parametrize("M,K,N", [(128, 1024, 4096), (333, 4096, 1024), (16, 1024, 4096), (1024, 1024, 4096)])
+def test_requant_epilogue_round_only(h, M, K, N):
+    # Eq. 22: dequantize by row and column scale, add the folded bias, Round -> INT8
+    A, Wt, rs, cs, bias = W.gemm_case(M, K, N)
+    x = O.QT("i8", A, row_scale=rs.astype(np.float64))
+    want = O.gemm_quant(x, Wt.T.copy(), cs, bias, "none", O.OutSpec("round"))
+    got = _linear(h, A, Wt, torch.int8, rs=rs, cs=cs, bias=bias).cpu().numpy()
+    assert_int8_close(got, want.data, what="requant epilogue")
+    assert np.abs(want.data.astype(int)).max() > 60      # the case exercises a wide code range
+
+
+@pytest.mark.parametrize("act", ["gelu_erf", "gelu_tanh"])
+def test_fc1_gelu_quant_epilogue(h, act):
+    # Eq. 28-29: X_1 stays FP32 on chip, GELU, then FWQ with 1 / S_a
+    M, K, N = 260, 768, 3072
+    g = W.rng(2, 555)
+    A = g.integers(-127, 128, (M, K), dtype=np.int8)
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    rs = (g.uniform(0.5, 1.5, M) * 0.02).astype(np.float32)
+    cs = (g.uniform(0.5, 1.5, N) * 1.5e-4 / np.sqrt(K / 768)).astype(np.float32)
+    bias = (g.standard_normal(N) * 0.1).astype(np.float32)
+    x = O.QT("i8", A, row_scale=rs.astype(np.float64))
+    v = O.gemm_quant(x, Wt.T.copy(), cs, bias, act, O.OutSpec("fp", dtype="f64")).data
+    S_a = Q.calib_scale(np.abs(v).max(0))
+    want = O.gemm_quant(x, Wt.T.copy(), cs, bias, act, O.OutSpec("fwq", scale=S_a))
+    inv = (1.0 / S_a).astype(np.float32)
+    got = _linear(h, A, Wt, torch.int8, rs=rs, cs=cs, bias=bias, act=act, post=inv).cpu().numpy()
+    assert_int8_close(got, want.data, what="GELU^quant")
+
+
+@pytest.mark.parametrize("fp", ["f16", "bf16"])
+def test_int8_gemm_fp_output(h, fp):
+    # an INT8 module whose consumer is in FP mode: dequantize + bias only, stored in FP16 / BF16
+    M, K, N = 200, 1024, 1024
+    A, Wt, rs, cs, bias = W.gemm_case(M, K, N)
+    x = O.QT("i8", A, row_scale=rs.astype(np.float64))
+    want = O.gemm_quant(x, Wt.T.copy(), cs, bias, "none", O.OutSpec("fp", dtype=fp))
+    got = _linear(h, A, Wt, TORCH_FP[fp], rs=rs, cs=cs, bias=bias).float().cpu().numpy()
+    assert rel_err(got, want.data) < (1e-2 if fp == "bf16" else 2e-3)
+    assert np.mean(got != want.data) < 2e-3            # equal up to rare 1-ulp rounding ties
+
+
+@pytest.mark.parametrize("fp", ["f16", "bf16"])
+@pytest.mark.parametrize("M,K,N", [(128, 64, 256), (200, 1024, 768), (77, 136, 48)])
+def test_fp_mode_gemm(h, fp, M, K, N):
+    # a module left in FP16/BF16 (Table 1): X W + b with fp32 accumulation
+    g = W.rng(2, 777 + M)
+    A = Q.round_to_storage(g.standard_normal((M, K)), fp)
+    Wm = Q.round_to_storage(g.standard_normal((K, N)) * 0.05, fp)
+    bias = (g.standard_normal(N) * 0.1).astype(np.float32)
+    want = O.gemm_fp(O.fp_tensor(A, fp), Wm, bias, "gelu_erf", O.OutSpec("fp", dtype=fp))
+    tA = dev(A, TORCH_FP[fp])
+    tW = dev(Wm.T.copy(), TORCH_FP[fp])
+    got = _linear(h, tA, tW, TORCH_FP[fp], bias=bias, act="gelu_erf").float().cpu().numpy()
+    assert rel_err(got, want.data) < (1e-2 if fp == "bf16" else 2e-3)
+    # FP GEMM that feeds an INT8 consumer: quantized in the epilogue with 1 / S
+    y = O.gemm_fp(O.fp_tensor(A, fp), Wm, bias, "none", O.OutSpec("fp", dtype="f64")).data
+    S = Q.calib_scale(np.abs(y).max(0))
+    want_q = O.gemm_fp(O.fp_tensor(A, fp), Wm, bias, "none", O.OutSpec("fwq", scale=S))
+    got_q = _linear(h, tA, tW, torch.int8, bias=bias, post=(1.0 / S).astype(np.float32)).cpu().numpy()
+    assert_int8_close(got_q, want_q.data, frac=2e-4, what="FP GEMM -> INT8")
+
+
+def test_strided_views_and_untouched_padding(h):
+    # A and out are column slices of wider buffers (ld > cols); bytes outside the view stay untouched
+    M, K, N = 150, 256, 128
+    g = W.rng(2, 888)
+    Abig = torch.from_numpy(g.integers(-127, 128, (M, K + 64), dtype=np.int8)).cuda()
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    outbig = torch.full((M, N + 32), 99, dtype=torch.int32, device="cuda")
+    h.hero_w8a8_linear(hero.tensor(Abig[:, :K]), dev(Wt), hero.tensor(outbig[:, :N]))
+    h.check()
+    want = O.int_matmul(Abig[:, :K].cpu().numpy(), Wt.T.copy())
+    assert np.array_equal(outbig[:, :N].cpu().numpy(), want)
+    assert torch.all(outbig[:, N:] == 99)
+
+
+def test_refusals(h):
+    A = torch.zeros(8, 64, dtype=torch.int8, device="cuda")
+    Wt = torch.zeros(32, 64, dtype=torch.int8, device="cuda")
+    cs = torch.ones(32, device="cuda")
+    out = torch.zeros(8, 32, dtype=torch.int8, device="cuda")
+    sc = torch.zeros(8, device="cuda")
+    with pytest.raises(hero.HeroError) as e:      # token-wise output from a GEMM epilogue: refused (Sec. 2.1)
+        h.hero_w8a8_linear(hero.tensor(A), Wt, hero.tensor(out, "twq", sc), w_scale=cs)
+    assert e.value.status == hero.ERR_UNSUPPORTED
+    with pytest.raises(hero.HeroError) as e:      # K not a multiple of 16 bytes
+        h.hero_w8a8_linear(hero.tensor(A[:, :40]), Wt[:, :40], hero.tensor(out), w_scale=cs)
+    assert e.value.status in (hero.ERR_UNSUPPORTED, hero.ERR_ALIGNMENT)
+    empty = torch.zeros(0, 64, dtype=torch.int8, device="cuda")
+    h.hero_w8a8_linear(hero.tensor(empty), Wt, hero.tensor(torch.zeros(0, 32, dtype=torch.int8, device="cuda")), w_scale=cs)
