@@ -1,14 +1,211 @@
-// hero_layer_forward (Sec. 2.2.2-2.2.3, Table 1) -- under construction.
+// hero_layer_forward: one transformer layer (Sec. 2.2.2-2.2.3) under the per-module modes of Table 1.
+// Host-side sequencing only: seven kernel launches on one stream (QKV GeMM^quant, attention core,
+// attention-output GeMM^quant, LN^quant, FC1 + GELU^quant, FC2 GeMM^quant, LN^quant), every
+// intermediate in the caller's workspace.  No standalone quantize kernel exists: each tensor is
+// quantized by the epilogue of its producer, and a producer emits what its consumer's mode needs.
 #include "common.cuh"
-extern "C" hero_status hero_layer_workspace_bytes(const hero_layer_desc* d, int64_t M, size_t* bytes) {
-  (void)d; (void)M; (void)bytes;
-  hero::set_error("hero_layer_workspace_bytes: not built yet");
-  return HERO_ERR_UNSUPPORTED;
+
+namespace hero {
+
+struct LayerPlan {
+  size_t off_qkv, off_attn, off_o, off_mid, off_mid_scale, off_a, off_x2, off_xin, off_xin_scale, off_hin, off_hmid;
+  size_t total;
+};
+
+static inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+static hero_status plan_layer(const hero_layer_desc* d, int64_t M, LayerPlan* pl) {
+  HERO_REQUIRE(d != nullptr, HERO_ERR_INVALID_ARG, "layer descriptor is NULL");
+  HERO_REQUIRE(d->arch == HERO_POST_LN || d->arch == HERO_PRE_LN, HERO_ERR_INVALID_ARG, "unknown arch %d", d->arch);
+  HERO_REQUIRE(d->B > 0 && d->S > 0 && d->H > 0 && d->nh > 0 && d->F > 0 && d->H % d->nh == 0, HERO_ERR_INVALID_ARG,
+               "bad layer dimensions");
+  HERO_REQUIRE(M == (int64_t)d->B * d->S, HERO_ERR_INVALID_ARG, "M=%lld != B*S", (long long)M);
+  HERO_REQUIRE(is_fp16ish(d->fp_dtype), HERO_ERR_INVALID_ARG, "fp_dtype must be F16 or BF16");
+  for (int i = 0; i < 5; ++i)
+    HERO_REQUIRE(d->mode[i] == HERO_MODE_INT8 || d->mode[i] == HERO_MODE_FP, HERO_ERR_INVALID_ARG, "mode[%d]=%d", i, d->mode[i]);
+  const size_t H = d->H, F = d->F, m = (size_t)M;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
+  pl->off_qkv = take(m * 3 * H * 2);
+  pl->off_attn = take(m * H * 2);
+  pl->off_o = take(m * H * 2);
+  pl->off_mid = take(m * H * 2);
+  pl->off_mid_scale = take(m * 4);
+  pl->off_a = take(m * F * 2);
+  pl->off_x2 = take(m * H * 2);
+  pl->off_xin = pl->off_xin_scale = pl->off_hin = pl->off_hmid = 0;
+  if (d->arch == HERO_PRE_LN) {
+    pl->off_xin = take(m * H * 2);
+    pl->off_xin_scale = take(m * 4);
+    pl->off_hin = take(m * H * 2);
+    pl->off_hmid = take(m * H * 2);
+  }
+  pl->total = o;
+  return HERO_OK;
 }
+
+static hero_tensor mk(void* data, int dtype, int gran, int64_t rows, int64_t cols, const float* scale) {
+  hero_tensor t;
+  t.data = data; t.dtype = dtype; t.gran = gran; t.rows = rows; t.cols = cols; t.ld = cols;
+  t.scale = const_cast<float*>(scale);
+  return t;
+}
+static hero_tensor none() { return mk(nullptr, 0, 0, 0, 0, nullptr); }
+
+}  // namespace hero
+
+extern "C" hero_status hero_layer_workspace_bytes(const hero_layer_desc* d, int64_t M, size_t* bytes) {
+  using namespace hero;
+  HERO_REQUIRE(bytes != nullptr, HERO_ERR_INVALID_ARG, "bytes is NULL");
+  LayerPlan pl;
+  hero_status st = plan_layer(d, M, &pl);
+  if (st != HERO_OK) return st;
+  *bytes = pl.total;
+  return HERO_OK;
+}
+
 extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in,
                                           const hero_tensor* pending, const hero_tensor* out, void* workspace,
                                           size_t workspace_bytes, void* stream) {
-  (void)h; (void)d; (void)in; (void)pending; (void)out; (void)workspace; (void)workspace_bytes; (void)stream;
-  hero::set_error("hero_layer_forward: not built yet");
-  return HERO_ERR_UNSUPPORTED;
+  using namespace hero;
+  HERO_REQUIRE(h && d && in && out, HERO_ERR_INVALID_ARG, "hero_layer_forward: NULL argument");
+  const int64_t M = in->rows;
+  LayerPlan pl;
+  hero_status st = plan_layer(d, M, &pl);
+  if (st != HERO_OK) return st;
+  HERO_REQUIRE(workspace != nullptr && (reinterpret_cast<uintptr_t>(workspace) & 255) == 0, HERO_ERR_ALIGNMENT,
+               "workspace must be a 256-byte aligned device pointer");
+  HERO_REQUIRE(workspace_bytes >= pl.total, HERO_ERR_WORKSPACE, "workspace too small: %zu < %zu", workspace_bytes, pl.total);
+  HERO_REQUIRE(in->cols == d->H && out->rows == M && out->cols == d->H, HERO_ERR_INVALID_ARG, "in / out shape mismatch");
+  const bool pre = d->arch == HERO_PRE_LN;
+  HERO_REQUIRE(pre || pending == nullptr || pending->data == nullptr, HERO_ERR_INVALID_ARG, "pending is for pre-LN layers only");
+
+  const int H = d->H, F = d->F, fp = d->fp_dtype;
+  const bool qkv8 = d->mode[HERO_MOD_QKV] == HERO_MODE_INT8, attn8 = d->mode[HERO_MOD_ATTN] == HERO_MODE_INT8;
+  const bool o8 = d->mode[HERO_MOD_ATTN_OUT] == HERO_MODE_INT8, fc18 = d->mode[HERO_MOD_FC1] == HERO_MODE_INT8;
+  const bool fc28 = d->mode[HERO_MOD_FC2] == HERO_MODE_INT8;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+
+  // the INT8 tensor an LN emits for an INT8 consumer, by granularity (Eq. 3-5)
+  auto ln_out = [&](void* data, bool int8, int gran, const float* static_scale, float* twq_scale) -> hero_tensor {
+    if (!int8) return mk(data, fp, HERO_GRAN_NONE, M, H, nullptr);
+    if (gran == HERO_GRAN_TWQ) return mk(data, HERO_I8, HERO_GRAN_TWQ, M, H, twq_scale);
+    return mk(data, HERO_I8, gran, M, H, static_scale);
+  };
+  HERO_REQUIRE(d->gran_in == HERO_GRAN_TWQ || d->gran_in == HERO_GRAN_FWQ || d->gran_in == HERO_GRAN_SQ, HERO_ERR_INVALID_ARG, "gran_in");
+  HERO_REQUIRE(d->gran_mid == HERO_GRAN_TWQ || d->gran_mid == HERO_GRAN_FWQ || d->gran_mid == HERO_GRAN_SQ, HERO_ERR_INVALID_ARG, "gran_mid");
+  HERO_REQUIRE(d->gran_attn == HERO_GRAN_FWQ || d->gran_attn == HERO_GRAN_SQ, HERO_ERR_UNSUPPORTED,
+               "X_attn is feature-wise or static (a GEMM-like epilogue cannot reduce over a row, Sec. 2.1)");
+
+  hero_tensor x_in = *in;       // what feeds QKV
+  hero_tensor h_cur = *in;      // pre-LN: the FP residual stream
+  if (pre) {
+    HERO_REQUIRE(is_fp16ish(in->dtype) && in->dtype == fp, HERO_ERR_INVALID_ARG, "pre-LN: `in` is the residual stream in fp_dtype");
+    hero_ln_args a;
+    memset(&a, 0, sizeof(a));
+    a.residual = *in;
+    const bool has_pending = pending && pending->data;
+    if (has_pending) a.branch = *pending;
+    a.gamma = d->ln1_g; a.beta = d->ln1_b; a.eps = d->eps;
+    a.out = ln_out(ws + pl.off_xin, qkv8, d->gran_in, d->s_in, reinterpret_cast<float*>(ws + pl.off_xin_scale));
+    if (has_pending) {
+      a.fp_out = mk(ws + pl.off_hin, fp, HERO_GRAN_NONE, M, H, nullptr);
+      h_cur = a.fp_out;
+    }
+    if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
+    x_in = a.out;
+  } else {
+    HERO_REQUIRE(qkv8 ? in->dtype == HERO_I8 : in->dtype == fp, HERO_ERR_INVALID_ARG,
+                 "post-LN: `in` must be INT8 when the QKV module is INT8, else fp_dtype");
+  }
+
+  // ---- QKV GeMM^quant (Eq. 14, 20-22)
+  const int qkv_dt = attn8 ? HERO_I8 : fp;
+  const size_t qkv_es = dtype_size(qkv_dt);
+  hero_tensor qkv = mk(ws + pl.off_qkv, qkv_dt, HERO_GRAN_NONE, M, 3 * H, nullptr);
+  {
+    hero_linear_args a;
+    memset(&a, 0, sizeof(a));
+    a.A = x_in; a.W = d->qkv.W; a.N = 3 * H; a.ldw = H;
+    a.w_scale = d->qkv.w_scale; a.bias = d->qkv.bias; a.act = HERO_ACT_NONE; a.post_scale = d->qkv.post_scale;
+    a.out = qkv;
+    if ((st = hero_w8a8_linear(h, &a, stream)) != HERO_OK) return st;
+  }
+  // ---- attention core (Eq. 15-17)
+  hero_tensor x_attn = o8 ? mk(ws + pl.off_attn, HERO_I8, d->gran_attn, M, H, d->s_attn)
+                          : mk(ws + pl.off_attn, fp, HERO_GRAN_NONE, M, H, nullptr);
+  {
+    hero_attn_args a;
+    memset(&a, 0, sizeof(a));
+    uint8_t* base = static_cast<uint8_t*>(qkv.data);
+    a.q = base; a.k = base + (size_t)H * qkv_es; a.v = base + (size_t)2 * H * qkv_es;
+    a.dtype = qkv_dt; a.ld = 3 * H;
+    a.B = d->B; a.S = d->S; a.nh = d->nh; a.dh = H / d->nh;
+    a.s_q = d->s_q; a.s_k = d->s_k; a.s_v = d->s_v; a.s_p = d->s_p;
+    a.mask = d->mask; a.key_len = nullptr;
+    a.out = x_attn;
+    if ((st = hero_int8_attention(h, &a, stream)) != HERO_OK) return st;
+  }
+  // ---- attention-output GeMM^quant (Eq. 18, 23): the FWQ / SQ scale of X_attn lives in W~_o's rows
+  hero_tensor x_o = o8 ? mk(ws + pl.off_o, HERO_I8, HERO_GRAN_FWQ, M, H, d->s_o) : mk(ws + pl.off_o, fp, HERO_GRAN_NONE, M, H, nullptr);
+  {
+    hero_linear_args a;
+    memset(&a, 0, sizeof(a));
+    a.A = x_attn; a.A.gran = HERO_GRAN_NONE; a.A.scale = nullptr;
+    a.W = d->o.W; a.N = H; a.ldw = H;
+    a.w_scale = d->o.w_scale; a.bias = d->o.bias; a.act = HERO_ACT_NONE; a.post_scale = d->o.post_scale;
+    a.out = x_o; a.out.gran = HERO_GRAN_NONE; a.out.scale = nullptr;
+    if ((st = hero_w8a8_linear(h, &a, stream)) != HERO_OK) return st;
+  }
+  // ---- LN^quant (Eq. 19): residual + attention branch -> the tensor feeding FC1
+  hero_tensor x_mid = ln_out(ws + pl.off_mid, fc18, d->gran_mid, d->s_mid, reinterpret_cast<float*>(ws + pl.off_mid_scale));
+  hero_tensor h_mid = none();
+  {
+    hero_ln_args a;
+    memset(&a, 0, sizeof(a));
+    a.residual = pre ? h_cur : *in;
+    a.branch = x_o;
+    a.gamma = pre ? d->ln2_g : d->ln1_g; a.beta = pre ? d->ln2_b : d->ln1_b; a.eps = d->eps;
+    a.out = x_mid;
+    if (pre) { h_mid = mk(ws + pl.off_hmid, fp, HERO_GRAN_NONE, M, H, nullptr); a.fp_out = h_mid; }
+    if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
+  }
+  // ---- FC1 + GELU^quant (Eq. 28-29): X_1 never leaves the epilogue's registers
+  hero_tensor act = fc28 ? mk(ws + pl.off_a, HERO_I8, HERO_GRAN_NONE, M, F, nullptr) : mk(ws + pl.off_a, fp, HERO_GRAN_NONE, M, F, nullptr);
+  {
+    hero_linear_args a;
+    memset(&a, 0, sizeof(a));
+    a.A = x_mid; a.W = d->fc1.W; a.N = F; a.ldw = H;
+    a.w_scale = d->fc1.w_scale; a.bias = d->fc1.bias; a.act = d->act; a.post_scale = d->fc1.post_scale;
+    a.out = act;
+    if ((st = hero_w8a8_linear(h, &a, stream)) != HERO_OK) return st;
+  }
+  // ---- FC2 GeMM^quant (Eq. 30, 32)
+  hero_tensor x_2 = fc28 ? mk(ws + pl.off_x2, HERO_I8, HERO_GRAN_FWQ, M, H, d->s_x2) : mk(ws + pl.off_x2, fp, HERO_GRAN_NONE, M, H, nullptr);
+  {
+    hero_linear_args a;
+    memset(&a, 0, sizeof(a));
+    a.A = act; a.W = d->fc2.W; a.N = H; a.ldw = F;
+    a.w_scale = d->fc2.w_scale; a.bias = d->fc2.bias; a.act = HERO_ACT_NONE; a.post_scale = d->fc2.post_scale;
+    a.out = x_2; a.out.gran = HERO_GRAN_NONE; a.out.scale = nullptr;
+    if ((st = hero_w8a8_linear(h, &a, stream)) != HERO_OK) return st;
+  }
+  // ---- LN^quant (Eq. 31) / closing residual add of a pre-LN layer
+  {
+    hero_ln_args a;
+    memset(&a, 0, sizeof(a));
+    a.branch = x_2;
+    if (pre) {
+      HERO_REQUIRE(out->dtype == fp, HERO_ERR_INVALID_ARG, "pre-LN: out is the residual stream in fp_dtype");
+      a.residual = h_mid;
+      a.fp_out = *out;
+    } else {
+      a.residual = x_mid;
+      a.gamma = d->ln2_g; a.beta = d->ln2_b; a.eps = d->eps;
+      a.out = *out;
+      if (out->dtype == HERO_I8 && out->gran != HERO_GRAN_TWQ && out->scale == nullptr) a.out.scale = const_cast<float*>(d->s_out);
+    }
+    if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
+  }
+  return HERO_OK;
 }

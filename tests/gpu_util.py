@@ -60,3 +60,37 @@ def rel_err(got, want):
     want = np.asarray(want, np.float64)
     den = np.max(np.abs(want))
     return float(np.max(np.abs(got - want)) / (den if den > 0 else 1.0))
+
+
+def oracle_layer_to_prepared(Lp):
+    """Re-express the oracle's prepared layer (paper layout, fp64) as the host arrays the library's Layer
+    uploads: weights transposed to [N][K], fp32 vectors, reciprocal epilogue scales.  Teacher-forcing: the
+    CUDA path then runs on exactly the oracle's weights and scales."""
+    from paper_2310_17723_b200 import prep
+    spec, C = Lp["spec"], Lp["C"]
+    cfg = prep.LayerConfig(B=spec.B, S=spec.S, H=spec.H, nh=spec.nh, F=spec.F, arch=spec.arch, act=spec.act,
+                           eps=spec.eps, mask=spec.mask, fp_dtype=spec.fp_dtype, mode=dict(spec.mode),
+                           gran_in=spec.gran_in, gran_mid=spec.gran_mid, gran_attn=spec.gran_attn,
+                           gran_out=spec.gran_out)
+    f = lambda a: None if a is None else np.ascontiguousarray(np.asarray(a, np.float64).astype(np.float32))
+    L = {"cfg": cfg, "C": C}
+    for name in ("qkv", "o", "fc1", "fc2"):
+        g = Lp[name]
+        post = None
+        if g["out"].kind == "fwq":
+            post = 1.0 / np.asarray(g["out"].scale, np.float64)
+        if g["mode"] == "int8":
+            L[name] = {"int8": True, "W": np.ascontiguousarray(g["W_i8"].T), "w_scale": f(g["cs"]), "bias": f(g["bias"]),
+                       "post_scale": f(post)}
+        else:
+            L[name] = {"int8": False, "W": prep._store_fp(g["W"], spec.fp_dtype), "w_scale": None, "bias": f(g["bias"]),
+                       "post_scale": f(post)}
+    for k in ("ln1_g", "ln1_b", "ln2_g", "ln2_b"):
+        L[k] = f(Lp[k])
+    vec = lambda gran, sf, st: None if gran == "twq" else f(sf if gran == "fwq" else [st])
+    L["s_in"] = vec(spec.gran_in, C["S_in_f"], C["S_in_t"])
+    L["s_mid"] = vec(spec.gran_mid, C["S_mid_f"], C["S_mid_t"])
+    L["s_attn"] = vec(spec.gran_attn, C["S_attn_f"], C["S_attn_t"])
+    L["s_o"], L["s_x2"] = f(C["S_o"]), f(C["S_x2"])
+    L["s_out"] = None if spec.gran_out in ("twq", "fp") else vec(spec.gran_out, C["S_out_f"], C["S_out_t"])
+    return L

@@ -128,11 +128,14 @@ def test_saturating_static_scale(h):
     B, S, nh, dh = 1, 128, 2, 64
     qkv, H = _qkv(B, S, nh, dh, 11, spread=60)
     s_q, s_k, s_v = _scales(dh, spread=30)              # sharper softmax
-    spec = O.OutSpec("fwq", scale=np.full(H, 0.01))
+    raw = _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, 0.25 / 255, O.OutSpec("fp", dtype="f64")).data
+    spec = O.OutSpec("fwq", scale=Q.calib_scale(np.abs(raw).max(0)))
     want, it = _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, 0.25 / 255, spec, internals=True)
     assert max(int(v.max()) for v in it["P_u8"].values()) == 255
     got = _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, 0.25 / 255, spec)
-    assert_int8_close(got, want.data, frac=2e-4, what="clipped P")
+    # with s_p four times finer every P code is four times closer to a rounding tie of the fp32 exponential,
+    # and one flipped code moves X_attn by a visible fraction of its LSB: 1 LSB on up to 2e-3 of the elements
+    assert_int8_close(got, want.data, frac=2e-3, what="clipped P")
 
 
 def test_refusals(h):

@@ -1,0 +1,133 @@
+"""GPU parity: hero_layer_forward against the oracle's layer, free-running (only the layer input is shared)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layer as OL
+from oracle import ops as O
+from paper_2310_17723_b200 import hero, workloads as W
+from paper_2310_17723_b200.layer import Layer
+from gpu_util import dev, f32, qt_to_device, assert_int8_close, rel_err, int8_mismatch, oracle_layer_to_prepared, TORCH_FP
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def h():
+    hd = hero.Handle()
+    yield hd
+    hd.check()
+    hd.close()
+
+
+def _spec(shape, **kw):
+    return OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, mask=shape.mask,
+                        fp_dtype=shape.fp_dtype, eps=shape.eps, **kw)
+
+
+def _build(shape, seed, **kw):
+    spec = _spec(shape, **kw)
+    p = W.layer_params(shape, seed)
+    x = W.activations(shape, seed)
+    if spec.arch == "post_ln":
+        cal_in = O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps)
+    else:
+        cal_in = x
+    C = OL.calibrate(spec, p, cal_in, shape.B)
+    Lp = OL.prepare_layer(spec, p, C)
+    if spec.arch == "post_ln":
+        x_in = OL.entry_ln(O.fp_tensor(x, "f16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+    else:
+        x_in = O.fp_tensor(x, spec.fp_dtype)
+    return spec, Lp, x_in
+
+
+def _run_layer(h, spec, Lp, x_in, pending=None):
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    M, H = spec.M, spec.H
+    _, in_desc, _ = qt_to_device(x_in)
+    pend = None if pending is None else qt_to_device(pending)[1]
+    if spec.arch == "pre_ln" or spec.gran_out == "fp":
+        out = torch.empty(M, H, dtype=TORCH_FP[spec.fp_dtype], device="cuda")
+        od, sc = hero.tensor(out), None
+    else:
+        out = torch.empty(M, H, dtype=torch.int8, device="cuda")
+        if spec.gran_out == "twq":
+            sc = torch.zeros(M, dtype=torch.float32, device="cuda")
+            od = hero.tensor(out, "twq", sc)
+        else:
+            sc = layer._bufs["s_out"]
+            od = hero.tensor(out, spec.gran_out, sc)
+    n0 = h.launches
+    layer.forward(in_desc, od, pending=pend)
+    h.check()
+    return out, sc, h.launches - n0
+
+
+SMALL = dict(B=2, S=128, H=256, nh=4, F=512)
+
+
+@pytest.mark.parametrize("gran_in,gran_attn", [("twq", "fwq"), ("fwq", "sq"), ("sq", "fwq")])
+def test_post_ln_m3_layer(h, gran_in, gran_attn):
+    shape = W.tiny_shape(**SMALL, eps=1e-5, n_outlier=2)
+    spec, Lp, x_in = _build(shape, 21, gran_in=gran_in, gran_mid=gran_in, gran_attn=gran_attn)
+    T = OL.layer_forward(Lp, x_in)
+    out, sc, launches = _run_layer(h, spec, Lp, x_in)
+    assert launches == 7                      # QKV, attention, O-proj, LN, FC1, FC2, LN: no standalone quantize kernel
+    want = T["x_out"]
+    got_real = out.cpu().numpy().astype(np.float64) * sc.cpu().numpy().astype(np.float64)[:, None]
+    # free-running: an upstream 1-LSB tie legitimately moves downstream values, so the gate is the dequantized
+    # layer output; the INT8 payload mismatch is reported alongside
+    assert rel_err(got_real, want.real()) < 1e-2
+    frac, mx = int8_mismatch(out.cpu().numpy(), want.data)
+    assert mx <= 2 and frac < 2e-2, (frac, mx)
+
+
+def test_post_ln_m3_bert_base_shape_c1(h):
+    # the BERT-base layer of the first benchmark configuration, whole batch
+    shape = W.C1
+    spec, Lp, x_in = _build(shape, 1)
+    T = OL.layer_forward(Lp, x_in)
+    out, sc, _ = _run_layer(h, spec, Lp, x_in)
+    got_real = out.cpu().numpy().astype(np.float64) * sc.cpu().numpy().astype(np.float64)[:, None]
+    assert rel_err(got_real, T["x_out"].real()) < 1e-2
+    frac, mx = int8_mismatch(out.cpu().numpy(), T["x_out"].data)
+    assert mx <= 2 and frac < 2e-2, (frac, mx)
+
+
+def test_post_ln_fp_output(h):
+    shape = W.tiny_shape(**SMALL, eps=1e-5)
+    spec, Lp, x_in = _build(shape, 22, gran_out="fp")
+    T = OL.layer_forward(Lp, x_in)
+    out, _, _ = _run_layer(h, spec, Lp, x_in)
+    assert rel_err(out.float().cpu().numpy(), T["x_out"].real()) < 1e-2
+
+
+@pytest.mark.parametrize("fp,dh", [("bf16", 64), ("f16", 128)])
+def test_pre_ln_causal_m3_layer(h, fp, dh):
+    shape = W.tiny_shape(B=2, S=256, H=256, nh=256 // dh, F=512, arch="pre_ln", mask="causal", fp_dtype=fp, eps=1e-5)
+    spec, Lp, x_in = _build(shape, 23)
+    T = OL.layer_forward(Lp, x_in)
+    out, _, launches = _run_layer(h, spec, Lp, x_in)
+    assert launches == 8                      # LN1, QKV, attention, O-proj, add+LN2, FC1, FC2, closing add
+    assert rel_err(out.float().cpu().numpy(), T["h_out"].real()) < 1e-2
+    # with a pending branch from a previous layer fused into LN1
+    g = W.rng(9, 5)
+    pend = O.QT("i8", g.integers(-127, 128, (spec.M, spec.H), dtype=np.int8),
+                col_scale=(np.abs(g.standard_normal(spec.H)) * 0.002 + 0.001).astype(np.float32).astype(np.float64))
+    T2 = OL.layer_forward(Lp, x_in, pending=pend)
+    out2, _, _ = _run_layer(h, spec, Lp, x_in, pending=pend)
+    assert rel_err(out2.float().cpu().numpy(), T2["h_out"].real()) < 1e-2
+
+
+def test_workspace_too_small_and_bad_args(h):
+    shape = W.tiny_shape(**SMALL, eps=1e-5)
+    spec, Lp, x_in = _build(shape, 24)
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    _, in_desc, _ = qt_to_device(x_in)
+    out = torch.empty(spec.M, spec.H, dtype=torch.int8, device="cuda")
+    sc = torch.zeros(spec.M, device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(hero.HeroError) as e:
+        h.hero_layer_forward(layer.desc, in_desc, hero.tensor(out, "twq", sc), small)
+    assert e.value.status == hero.ERR_WORKSPACE
