@@ -1,0 +1,392 @@
+#!/usr/bin/env python
+"""Benchmark of the W8A8 layer forward (ZeroQuant-HERO hot path) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c3|c4] [--impl reference]
+
+A step is one pass of the whole hot path over one batch of synthetic input that is already resident in
+HBM.  One JSON line is printed by rank 0.  `--impl reference` times the CPU oracle instead (a deliberately
+plain fp64 program: context, not a target).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "W8A8 layer tokens/sec"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# workloads
+# ------------------------------------------------------------------------------------------------
+def workload_spec(name):
+    """(shape, config id, [layer configs], description) for a benchmark workload."""
+    from paper_2310_17723_b200 import prep, workloads as W
+    m3 = dict(prep.PRESETS["M3"])
+
+    def cfg(shape, **kw):
+        return prep.LayerConfig(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, eps=shape.eps,
+                                mask=shape.mask, fp_dtype=shape.fp_dtype, mode=dict(m3), **kw)
+    if name == "c1":
+        s = W.C1
+        return s, 1, [cfg(s)], "C1: BERT-base layer, B1 S128 H768, post-LN, M3, TWQ"
+    if name == "c3":
+        s = W.C3
+        return s, 3, [cfg(s, gran_in="fwq", gran_attn="sq", gran_mid="twq", gran_out="twq")], \
+            "C3: BERT-large layer, B32 S384 H1024 F4096, post-LN, M3, FWQ LN->QKV (folded), SQ X_attn, TWQ elsewhere"
+    if name == "c4":
+        s = W.C4
+        return s, 4, [cfg(s)], "C4: GPT prefill layer, B8 S2048 H4096 nh32 F16384, pre-LN, causal, W8A8 everywhere"
+    raise SystemExit("unknown workload %r" % name)
+
+
+def kernel_table(shape, cfg):
+    """Per launch of one layer, in launch order: (name, family, algorithmic ops, algorithmic bytes)."""
+    M, H, F, S, nh, dh = shape.M, shape.H, shape.F, shape.S, shape.nh, shape.dh
+    causal = shape.mask == "causal"
+
+    def gemm(name, K, N):
+        return (name, "gemm", 2.0 * M * N * K, float(M * K + N * K + M * N + 4 * M + 8 * N))
+    attn_ops = 4.0 * shape.B * nh * S * S * dh * (0.5 if causal else 1.0)
+    attn = ("attention", "attn", attn_ops, float(4 * M * H))
+    rows = []
+    if shape.arch == "pre_ln":
+        rows.append(("ln1 (fp->i8 twq)", "ln", 0.0, float(M * H * 3 + 4 * M)))
+    rows += [gemm("qkv gemm", H, 3 * H), attn, gemm("attn-out gemm", H, H)]
+    if shape.arch == "pre_ln":
+        rows.append(("add+ln2 (fp+i8->fp,i8)", "ln", 0.0, float(M * H * 6 + 4 * M)))
+    else:
+        rows.append(("ln1 (i8+i8->i8 twq)", "ln", 0.0, float(M * H * 3 + 8 * M)))
+    rows += [gemm("fc1 gemm + gelu^quant", H, F), gemm("fc2 gemm", F, H)]
+    if shape.arch == "pre_ln":
+        rows.append(("closing add (fp+i8->fp)", "ln", 0.0, float(M * H * 5)))
+    else:
+        rows.append(("ln2 (i8+i8->i8 twq)", "ln", 0.0, float(M * H * 3 + 8 * M)))
+    return rows
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (also the cpu_baseline leg)
+# ------------------------------------------------------------------------------------------------
+def oracle_run(name, budget_s=12.0, repeats=1):
+    """Times the oracle, as it stands, on whole sequences of the workload.  Returns (tokens/s, cores, sample)."""
+    import numpy as np
+    from oracle import layer as OL, ops as O
+    from paper_2310_17723_b200 import workloads as W
+    shape, cid, cfgs, desc = workload_spec(name)
+    cfg = cfgs[0]
+    spec = OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, act=cfg.act, eps=cfg.eps,
+                        mask=cfg.mask, fp_dtype=cfg.fp_dtype, mode=dict(cfg.mode), gran_in=cfg.gran_in,
+                        gran_mid=cfg.gran_mid, gran_attn=cfg.gran_attn, gran_out=cfg.gran_out)
+    p = W.layer_params(shape, cid * 100)
+    x_cal = W.activations(shape, cid, n_seq=1, tensor=7).astype(np.float64)
+    cal_in = O.layernorm(x_cal, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else x_cal
+    C = OL.calibrate(spec, p, cal_in, 1)
+    Lp = OL.prepare_layer(spec, p, C)
+
+    def run(n_seq):
+        x = W.activations(shape, cid, n_seq=n_seq)
+        if spec.arch == "post_ln":
+            x_in = OL.entry_ln(O.fp_tensor(x, "f16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+        else:
+            x_in = O.fp_tensor(x, spec.fp_dtype)
+        t0 = time.perf_counter()
+        OL.layer_forward(Lp, x_in, B=n_seq)
+        return time.perf_counter() - t0
+
+    t1 = run(1)
+    n = int(max(1, min(shape.B, budget_s / max(t1, 1e-3))))
+    best = min(run(n) for _ in range(repeats)) if n > 1 else t1
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        pass
+    return n * shape.S / best, cores, "%d of %d sequences (%d tokens) of %s, one pass" % (n, shape.B, n * shape.S, shape.name), best
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape, cid, cfgs, desc = workload_spec(args.workload)
+    vals, ts = [], []
+    for i in range(args.warmup + args.steps):
+        v, cores, sample, t = oracle_run(args.workload, budget_s=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
+        if i >= args.warmup:
+            vals.append(v)
+            ts.append(t)
+    value = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sum(ts) / len(ts), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": desc, "l2": "n/a (CPU)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2310_17723_b200 import build as B
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0 or world == 1:
+        B.build()
+    if dist:
+        dist.barrier()
+    from paper_2310_17723_b200 import hero, workloads as W
+    from paper_2310_17723_b200.model import Stack
+
+    shape, cid, cfgs, desc = workload_spec(args.workload)
+    h = hero.Handle()
+    stack = Stack(h, shape, cid, cfgs, n_cal_seq=1 if shape.M * shape.H > 2 ** 25 else 2)
+    # every rank works on its own batch (replicas: the path shards by sequence, no exchange step)
+    x_host = torch.from_numpy(W.activations(shape, cid, tensor=2 + 10 * rank)).to(stack.fp_torch)
+    x_dev = x_host.cuda()
+    stack.set_input(x_dev)
+    h.check()
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.int8, device="cuda")     # > 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    def step():
+        stack.forward()
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    n0 = h.launches
+    step()
+    launches_per_step = h.launches - n0
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, each bracketed by events on the launching stream, L2 flushed in between
+    sampler = ClockSampler(local) if rank == 0 else None
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    n0 = h.launches
+    for k in range(args.steps):
+        flush.zero_()
+        ev[k][0].record(stream)
+        step()
+        ev[k][1].record(stream)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    wall = time.perf_counter() - wall0
+    gpu_launches = h.launches - n0
+    h.check()
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    if dist:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    clocks = sampler.stop() if sampler else None
+    ms_per_step = total_ms / args.steps
+    value = world * shape.M * len(cfgs) / len(cfgs) / (ms_per_step * 1e-3)
+
+    # ---- per-kernel device times (a second, instrumented pass: event pairs around every launch)
+    kern = []
+    roof = None
+    peaks, peak_kind = load_peaks()
+    if rank == 0:
+        h.profile_begin(launches_per_step * args.steps)
+        for k in range(args.steps):
+            flush.zero_()
+            step()
+        recs = h.profile_end()
+        table = []
+        for cfg in cfgs:
+            table += kernel_table(shape, cfg)
+        assert len(table) == launches_per_step, (len(table), launches_per_step)
+        int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        for i, (name, fam, ops, nbytes) in enumerate(table):
+            ms = [recs[j][1] for j in range(i, len(recs), launches_per_step)]
+            avg = sum(ms) / len(ms)
+            row = {"kernel": name, "ms": round(avg, 5), "share": None}
+            if fam == "gemm":
+                row.update(bound="tensor", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak, unit="TFLOP/s")
+            elif fam == "ln":
+                row.update(bound="hbm", achieved=nbytes / (avg * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+            else:
+                row.update(bound="alu", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak, unit="TFLOP/s")
+            row["frac"] = row["achieved"] / row["peak"]
+            kern.append(row)
+        tot = sum(r["ms"] for r in kern)
+        for r in kern:
+            r["share"] = round(r["ms"] / tot, 4)
+        dom = max(kern, key=lambda r: r["ms"])
+        roof = {"bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
+                "frac": dom["frac"], "traffic": None, "kernel": dom["kernel"],
+                "peak_source": "%s: %s" % (peak_kind, "2 x bf16_tflops_sustained (INT8 runs at twice the BF16 rate)"
+                                           if dom["bound"] != "hbm" else "hbm_gbs")}
+
+    # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
+    e2e = None
+    if len(cfgs) == 1 and shape.arch == "post_ln":
+        t_in, s_in, d_in = stack.bufs[0]
+        t_out, s_out, d_out = stack.bufs[1]
+        hin = t_in.cpu().pin_memory()
+        hout = torch.empty_like(t_out, device="cpu").pin_memory()
+        gin, gout = cfgs[0].gran_in, cfgs[0].gran_out
+        hsin = s_in.cpu().pin_memory() if s_in is not None else None
+        hsout = torch.empty_like(s_out, device="cpu").pin_memory() if s_out is not None else None
+        in_host = hero.host_tensor(hin, gin, hsin)
+        out_host = hero.host_tensor(hout, gout, hsout)
+        layer = stack.layers[0]
+
+        def e2e_step():
+            h.hero_layer_forward_host(layer.desc, in_host, out_host, d_in, d_out, layer.workspace)
+        h2d = hin.numel() + (hsin.numel() * 4 if gin == "twq" else 0)
+        d2h = hout.numel() * hout.element_size() + (hsout.numel() * 4 if gout == "twq" else 0)
+    else:
+        t_in = stack.bufs[0][0]
+        t_out = stack.bufs[-1][0]
+        hin = x_host.pin_memory()
+        hout = torch.empty_like(t_out, device="cpu").pin_memory()
+
+        def e2e_step():
+            t_in.copy_(hin, non_blocking=True)
+            stack.forward()
+            hout.copy_(t_out, non_blocking=True)
+            torch.cuda.synchronize()
+        h2d = hin.numel() * hin.element_size()
+        d2h = hout.numel() * hout.element_size()
+    for _ in range(3):
+        e2e_step()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if dist:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * shape.M * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+    h.check()
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        v, cores, sample, _t = oracle_run(args.workload)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+            "data": "synthetic",
+            "config": {"workload": desc, "tokens_per_step_per_gpu": shape.M, "l2": "flushed between timed steps (512 MiB write)",
+                       "timing": "CUDA events per step on the launching stream, max over ranks",
+                       "parallelism": "replicas x%d (sequence-sharded, no collective)" % world},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "kernels": kern,
+            "cpu_baseline": cpu, "wall_s_timed_region": wall}
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

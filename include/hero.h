@@ -239,6 +239,22 @@ hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const h
                                const hero_tensor* pending, const hero_tensor* out, void* workspace,
                                size_t workspace_bytes, void* stream);
 
+/* The same layer (Sec. 2.2.2-2.2.3) called with HOST activation buffers: copies `in_host` (payload and, for
+ * a token-wise input, its per-row scales) into the caller's device staging tensor `in_dev`, runs
+ * hero_layer_forward, copies the result back into `out_host` and synchronizes the stream.  Host buffers
+ * should be page-locked for the copies to be asynchronous.  Weights, calibrated scales, staging tensors and
+ * workspace stay device-resident and caller-owned; nothing is allocated. */
+hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
+                                    const hero_tensor* out_host, const hero_tensor* in_dev, const hero_tensor* out_dev,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* Per-launch device timing for benchmarks (no counterpart in the paper, which measured nothing): between
+ * _begin and _end every kernel the handle launches is bracketed by a pair of CUDA events on its stream.
+ * _end waits for them and returns, per launch in order, the elapsed milliseconds and the kernel family
+ * (1 = LN^quant, 2 = GeMM^quant, 3 = attention core).  Arrays must hold max_launches entries. */
+hero_status hero_profile_begin(hero_handle* h, int32_t max_launches);
+hero_status hero_profile_end(hero_handle* h, float* ms_out, int32_t* tag_out, int32_t* n_out);
+
 #ifdef __cplusplus
 }
 #endif

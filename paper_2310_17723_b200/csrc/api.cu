@@ -83,6 +83,7 @@ hero_status hero_create(hero_handle** out) {
   h->launches = 0;
   h->d_error = nullptr;
   h->encode_tiled = nullptr;
+  h->prof_on = false; h->prof_cap = 0; h->prof_n = 0; h->prof_ev = nullptr; h->prof_tag = nullptr;
   cudaError_t e = cudaMalloc(&h->d_error, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(h->d_error, 0, sizeof(int));
   if (e != cudaSuccess) {
@@ -101,8 +102,43 @@ hero_status hero_create(hero_handle** out) {
   return HERO_OK;
 }
 
+static void free_profile(hero_handle* h) {
+  for (int i = 0; i < 2 * h->prof_cap; ++i) cudaEventDestroy(h->prof_ev[i]);
+  delete[] h->prof_ev; delete[] h->prof_tag;
+  h->prof_ev = nullptr; h->prof_tag = nullptr; h->prof_cap = 0; h->prof_n = 0; h->prof_on = false;
+}
+
+hero_status hero_profile_begin(hero_handle* h, int32_t max_launches) {
+  HERO_REQUIRE(h != nullptr && max_launches > 0, HERO_ERR_INVALID_ARG, "hero_profile_begin: bad arguments");
+  if (h->prof_cap != max_launches) {
+    free_profile(h);
+    h->prof_ev = new cudaEvent_t[2 * max_launches];
+    h->prof_tag = new int32_t[max_launches];
+    for (int i = 0; i < 2 * max_launches; ++i) HERO_CUDA(cudaEventCreate(&h->prof_ev[i]));
+    h->prof_cap = max_launches;
+  }
+  h->prof_n = 0;
+  h->prof_on = true;
+  return HERO_OK;
+}
+
+hero_status hero_profile_end(hero_handle* h, float* ms_out, int32_t* tag_out, int32_t* n_out) {
+  HERO_REQUIRE(h != nullptr && n_out != nullptr, HERO_ERR_INVALID_ARG, "hero_profile_end: bad arguments");
+  h->prof_on = false;
+  for (int i = 0; i < h->prof_n; ++i) {
+    HERO_CUDA(cudaEventSynchronize(h->prof_ev[2 * i + 1]));
+    float ms = 0.f;
+    HERO_CUDA(cudaEventElapsedTime(&ms, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]));
+    if (ms_out) ms_out[i] = ms;
+    if (tag_out) tag_out[i] = h->prof_tag[i];
+  }
+  *n_out = h->prof_n;
+  return HERO_OK;
+}
+
 hero_status hero_destroy(hero_handle* h) {
   if (!h) return HERO_OK;
+  free_profile(h);
   cudaFree(h->d_error);
   delete h;
   return HERO_OK;

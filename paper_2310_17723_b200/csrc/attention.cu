@@ -392,9 +392,11 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
     configured = true;
   }
   const long long grid = (long long)p.nqt * a->nh * a->B;
-  kern<<<(unsigned)grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+  {
+    LaunchScope scope(h, stream, KERNEL_ATTN);
+    kern<<<(unsigned)grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+  }
   HERO_CUDA(cudaGetLastError());
-  h->launches += 1;
   return HERO_OK;
 }
 

@@ -16,6 +16,11 @@ struct hero_handle {
   int* d_error;        // device error word: 0 = fine, else a code saying which wait gave up
   int64_t launches;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
+  // optional per-launch timing (hero_profile_begin / _end): event pairs around every kernel launch
+  bool prof_on;
+  int prof_cap, prof_n;
+  cudaEvent_t* prof_ev;   // 2 * prof_cap events
+  int32_t* prof_tag;      // kernel family of each recorded launch
 };
 
 namespace hero {
@@ -50,6 +55,22 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // data pointer 16-byte aligned, row pitch a multiple of 16 bytes, ld >= cols
 hero_status check_matrix(const hero_tensor& t, const char* name);
+
+// Kernel families for the per-launch timing records.
+enum { KERNEL_LN = 1, KERNEL_GEMM = 2, KERNEL_ATTN = 3 };
+// Brackets one kernel launch with events when timing is on; counts the launch either way.
+struct LaunchScope {
+  hero_handle* h; cudaStream_t s; int slot;
+  LaunchScope(hero_handle* h_, cudaStream_t s_, int tag) : h(h_), s(s_), slot(-1) {
+    h->launches += 1;
+    if (h->prof_on && h->prof_n < h->prof_cap) {
+      slot = h->prof_n++;
+      h->prof_tag[slot] = tag;
+      cudaEventRecord(h->prof_ev[2 * slot], s);
+    }
+  }
+  ~LaunchScope() { if (slot >= 0) cudaEventRecord(h->prof_ev[2 * slot + 1], s); }
+};
 
 // 2-D TMA descriptor over a row-major matrix [rows, cols] of `elem_bytes` elements with row pitch
 // ld_bytes; box = box_cols x box_rows elements; swizzle_bytes in {0, 32, 64, 128}.

@@ -273,9 +273,11 @@ static hero_status launch_gemm(hero_handle* h, const CUtensorMap& tmA, const CUt
   }
   const int tiles = p.num_m_tiles * p.num_n_tiles;
   const int grid = tiles < h->sm_count ? tiles : h->sm_count;
-  kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+  {
+    LaunchScope scope(h, stream, KERNEL_GEMM);
+    kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+  }
   HERO_CUDA(cudaGetLastError());
-  h->launches += 1;
   return HERO_OK;
 }
 

@@ -209,3 +209,34 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
   }
   return HERO_OK;
 }
+
+extern "C" hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
+                                               const hero_tensor* out_host, const hero_tensor* in_dev,
+                                               const hero_tensor* out_dev, void* workspace, size_t workspace_bytes,
+                                               void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(h && d && in_host && out_host && in_dev && out_dev, HERO_ERR_INVALID_ARG, "hero_layer_forward_host: NULL argument");
+  HERO_REQUIRE(in_host->dtype == in_dev->dtype && in_host->rows == in_dev->rows && in_host->cols == in_dev->cols &&
+               out_host->dtype == out_dev->dtype && out_host->rows == out_dev->rows && out_host->cols == out_dev->cols,
+               HERO_ERR_INVALID_ARG, "host and device staging tensors must agree in type and shape");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t ies = dtype_size(in_dev->dtype), oes = dtype_size(out_dev->dtype);
+  HERO_REQUIRE(ies && oes, HERO_ERR_INVALID_ARG, "unknown dtype");
+  auto scale_len = [](const hero_tensor& t) -> size_t {
+    if (t.dtype != HERO_I8) return 0;
+    return t.gran == HERO_GRAN_TWQ ? (size_t)t.rows : 0;   // calibrated FWQ / SQ scales already live on the device
+  };
+  // host -> device: the activation payload and, for a token-wise input, its per-row scales
+  HERO_CUDA(cudaMemcpy2DAsync(in_dev->data, in_dev->ld * ies, in_host->data, in_host->ld * ies, in_dev->cols * ies,
+                              in_dev->rows, cudaMemcpyHostToDevice, s));
+  if (scale_len(*in_dev))
+    HERO_CUDA(cudaMemcpyAsync(in_dev->scale, in_host->scale, scale_len(*in_dev) * sizeof(float), cudaMemcpyHostToDevice, s));
+  hero_status st = hero_layer_forward(h, d, in_dev, nullptr, out_dev, workspace, workspace_bytes, stream);
+  if (st != HERO_OK) return st;
+  HERO_CUDA(cudaMemcpy2DAsync(out_host->data, out_host->ld * oes, out_dev->data, out_dev->ld * oes, out_dev->cols * oes,
+                              out_dev->rows, cudaMemcpyDeviceToHost, s));
+  if (scale_len(*out_dev))
+    HERO_CUDA(cudaMemcpyAsync(out_host->scale, out_dev->scale, scale_len(*out_dev) * sizeof(float), cudaMemcpyDeviceToHost, s));
+  HERO_CUDA(cudaStreamSynchronize(s));
+  return HERO_OK;
+}

@@ -377,9 +377,11 @@ static hero_status launch_ln2(hero_handle* h, LnParams& p, cudaStream_t stream) 
   long long cap = (long long)h->sm_count * occ;
   int grid = (int)(want < cap ? want : cap);
   if (grid < 1) grid = 1;
-  ln_quant_kernel<VEC, R, HAS_BR, HAS_EX><<<grid, threads, smem, stream>>>(p);
+  {
+    LaunchScope scope(h, stream, KERNEL_LN);
+    ln_quant_kernel<VEC, R, HAS_BR, HAS_EX><<<grid, threads, smem, stream>>>(p);
+  }
   HERO_CUDA(cudaGetLastError());
-  h->launches += 1;
   return HERO_OK;
 }
 
@@ -749,9 +751,11 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
   if (occ < 1) occ = 1;
   const long long cap = (long long)h->sm_count * occ;
   const int grid = (int)(want < cap ? want : cap);
-  kern<<<grid, LNF_THREADS, smem, stream>>>(p);
+  {
+    LaunchScope scope(h, stream, KERNEL_LN);
+    kern<<<grid, LNF_THREADS, smem, stream>>>(p);
+  }
   HERO_CUDA(cudaGetLastError());
-  h->launches += 1;
   return HERO_OK;
 }
 

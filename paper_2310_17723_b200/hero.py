@@ -76,7 +76,8 @@ class LayerDesc(C.Structure):
 
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
-           "hero_layer_workspace_bytes", "hero_layer_forward")
+           "hero_layer_workspace_bytes", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
+           "hero_profile_end")
 
 _lib = None
 
@@ -102,6 +103,10 @@ def lib():
         L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
         L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hero_layer_forward_host.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
+            [C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hero_profile_begin.argtypes = [C.c_void_p, C.c_int32]
+        L.hero_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         _lib = L
     return _lib
 
@@ -191,11 +196,38 @@ class Handle:
         _check(lib().hero_layer_workspace_bytes(C.byref(desc), int(M), C.byref(n)))
         return int(n.value)
 
+    def hero_layer_forward_host(self, desc, in_host, out_host, in_dev, out_dev, workspace, stream=None):
+        """Host-buffer variant: copies in, runs the layer, copies out, synchronizes."""
+        _check(lib().hero_layer_forward_host(self._h, C.byref(desc), C.byref(in_host), C.byref(out_host),
+                                             C.byref(in_dev), C.byref(out_dev), C.c_void_p(workspace.data_ptr()),
+                                             workspace.numel(), _stream(stream)))
+
+    def profile_begin(self, max_launches):
+        self._prof_cap = int(max_launches)
+        _check(lib().hero_profile_begin(self._h, self._prof_cap))
+
+    def profile_end(self):
+        """[(kernel family, milliseconds), ...] for every launch since profile_begin, in order."""
+        ms = (C.c_float * self._prof_cap)()
+        tag = (C.c_int32 * self._prof_cap)()
+        n = C.c_int32()
+        _check(lib().hero_profile_end(self._h, ms, tag, C.byref(n)))
+        return [(int(tag[i]), float(ms[i])) for i in range(n.value)]
+
     def hero_layer_forward(self, desc, x_in, out, workspace, pending=None, stream=None):
         """x_in / out / pending: hero.Tensor; workspace: 1-D torch uint8 CUDA tensor."""
         pend = C.byref(pending) if pending is not None else None
         _check(lib().hero_layer_forward(self._h, C.byref(desc), C.byref(x_in), pend, C.byref(out),
                                         C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)))
+
+
+def host_tensor(t, gran="none", scale=None):
+    """hero_tensor view of a 2-D (pinned) host torch tensor, for hero_layer_forward_host."""
+    assert not t.is_cuda and t.dim() == 2 and t.stride(1) == 1
+    g = GRAN[gran] if isinstance(gran, str) else gran
+    T = Tensor(t.data_ptr(), _DT[t.dtype], g, t.shape[0], t.shape[1], t.stride(0), None if scale is None else scale.data_ptr())
+    T._keep = (t, scale)
+    return T
 
 
 def mode_preset(preset):

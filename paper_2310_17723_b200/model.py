@@ -1,0 +1,79 @@
+"""A stack of prepared layers with its chained device buffers: the object the benchmark and the smoke
+check drive.  Construction does the offline work (seeded parameters, calibration, folding, upload); `forward`
+is pure kernel launches through the C ABI."""
+import numpy as np
+import torch
+
+from . import hero, prep, workloads
+from .layer import Layer
+
+
+def _ln_np(x, g, b, eps):
+    x = np.asarray(x, np.float64)
+    mu = x.mean(-1, keepdims=True)
+    c = x - mu
+    return c / np.sqrt((c * c).mean(-1, keepdims=True) + eps) * g + b
+
+
+class Stack:
+    def __init__(self, handle, shape, config_id, layer_cfgs, n_cal_seq=2, unit_ln=False):
+        """shape: workloads.Shape; layer_cfgs: list of prep.LayerConfig (one per layer, chained)."""
+        self.h, self.shape, self.cfgs = handle, shape, layer_cfgs
+        self.M, self.H = shape.M, shape.H
+        self.fp_torch = hero.TORCH_FP[shape.fp_dtype]
+        post = shape.arch == "post_ln"
+        x_cal = workloads.activations(shape, config_id, n_seq=n_cal_seq, tensor=7).astype(np.float64)
+        self.layers, self.params = [], []
+        cur = None
+        for li, cfg in enumerate(layer_cfgs):
+            p = workloads.layer_params(shape, config_id * 100 + li, unit_ln=unit_ln)
+            if li == 0:
+                self.ln0 = (p["ln0_g"], p["ln0_b"])
+                cur = _ln_np(x_cal, p["ln0_g"].astype(np.float64), p["ln0_b"].astype(np.float64), cfg.eps) if post else x_cal
+            C, cur = prep.calibrate(cfg, p, cur, n_cal_seq, return_output=True)
+            self.layers.append(Layer(handle, prep.prepare_layer(cfg, p, C)))
+            self.params.append((p, C))
+        # chained activation buffers: input of layer 0 .. output of the last layer
+        self.bufs = []
+        for li in range(len(layer_cfgs) + 1):
+            kind = self._edge_kind(li)
+            if kind == "fp":
+                t = torch.empty(self.M, self.H, dtype=self.fp_torch, device="cuda")
+                self.bufs.append((t, None, hero.tensor(t)))
+            else:
+                t = torch.empty(self.M, self.H, dtype=torch.int8, device="cuda")
+                if kind == "twq":
+                    s = torch.empty(self.M, dtype=torch.float32, device="cuda")
+                else:
+                    src = self.layers[li]._bufs["s_in"] if li < len(layer_cfgs) else self.layers[-1]._bufs["s_out"]
+                    s = src
+                self.bufs.append((t, s, hero.tensor(t, kind, s)))
+        g0, b0 = self.ln0
+        self.ln0_g = torch.from_numpy(np.asarray(g0, np.float32)).cuda()
+        self.ln0_b = torch.from_numpy(np.asarray(b0, np.float32)).cuda()
+
+    def _edge_kind(self, li):
+        """Type of the tensor between layer li-1 and layer li: 'fp' or an INT8 granularity."""
+        n = len(self.cfgs)
+        if self.shape.arch == "pre_ln":
+            return "fp"
+        if li < n:
+            cfg = self.cfgs[li]
+            return "fp" if cfg.mode["qkv"] == "fp" else cfg.gran_in
+        return self.cfgs[-1].gran_out
+
+    def set_input(self, x_fp):
+        """Entry LN^quant: turns the FP activation [M, H] into layer 0's input (the role of the embedding
+        LayerNorm for a lone post-LN layer); for pre-LN stacks the FP tensor is the residual stream itself."""
+        if self.shape.arch == "pre_ln":
+            self.bufs[0][0].copy_(x_fp)
+            return
+        self.h.hero_layernorm_quant(hero.tensor(x_fp), self.ln0_g, self.ln0_b, self.cfgs[0].eps, self.bufs[0][2])
+
+    def forward(self, stream=None):
+        for li, layer in enumerate(self.layers):
+            layer.forward(self.bufs[li][2], self.bufs[li + 1][2], stream=stream)
+
+    @property
+    def output(self):
+        return self.bufs[-1]

@@ -93,7 +93,7 @@ def _ln(x, g, b, eps):
     return c / np.sqrt((c * c).mean(-1, keepdims=True) + eps) * g + b
 
 
-def calibrate(cfg: LayerConfig, params, x_cal, n_seq):
+def calibrate(cfg: LayerConfig, params, x_cal, n_seq, return_output=False):
     """Forward-only pass of the un-quantized layer over calibration data, recording absmax statistics
     (no truncation tuning).  `x_cal` is what enters the layer: for post-LN the tensor feeding QKV, for
     pre-LN the residual stream.  Returns the calibrated scales."""
@@ -142,7 +142,7 @@ def calibrate(cfg: LayerConfig, params, x_cal, n_seq):
         out = h1 + mlp(_ln(h1, p["ln2_g"], p["ln2_b"], cfg.eps))
     stat["out_f"], stat["out_t"] = np.abs(out).max(0), np.abs(out).max()
     sc = scale_from_absmax
-    return {
+    scales = {
         "S_in_f": sc(stat["in_f"]), "S_in_t": float(sc(stat["in_t"])),
         "S_q": float(sc(stat["q"])), "S_k": float(sc(stat["k"])), "S_v": float(sc(stat["v"])),
         "S_p": float(sc(stat["p"], 255.0)),
@@ -152,6 +152,7 @@ def calibrate(cfg: LayerConfig, params, x_cal, n_seq):
         "S_a": sc(stat["a"]), "S_x2": sc(stat["x2"]),
         "S_out_f": sc(stat["out_f"]), "S_out_t": float(sc(stat["out_t"])),
     }
+    return (scales, out) if return_output else scales
 
 
 def _gran_vec(gran, S_f, S_t, n):
