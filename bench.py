@@ -200,9 +200,8 @@ def run_ours(args):
     import numpy as np
     import torch
     from paper_2310_17723_b200 import build as B
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2310_17723_b200 import replicas
+    rank, local, world = replicas.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -221,7 +220,7 @@ def run_ours(args):
     h = hero.Handle()
     stack = Stack(h, shape, cid, cfgs, n_cal_seq=1 if shape.M * shape.H > 2 ** 25 else 2)
     # every rank works on its own batch (replicas: the path shards by sequence, no exchange step)
-    x_host = torch.from_numpy(W.activations(shape, cid, tensor=2 + 10 * rank)).to(stack.fp_torch)
+    x_host = torch.from_numpy(W.activations(shape, cid, tensor=replicas.batch_tensor_index(rank))).to(stack.fp_torch)
     x_dev = x_host.cuda()
     stack.set_input(x_dev)
     h.check()
@@ -231,6 +230,7 @@ def run_ours(args):
     def step():
         stack.forward()
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
         flush.zero_()
         step()
@@ -241,7 +241,6 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     # ---- timed region: K steps, each bracketed by events on the launching stream, L2 flushed in between
-    sampler = ClockSampler(local) if rank == 0 else None
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     if dist:
         dist.barrier()
@@ -259,14 +258,9 @@ def run_ours(args):
     wall = time.perf_counter() - wall0
     gpu_launches = h.launches - n0
     h.check()
-    total_ms = sum(a.elapsed_time(b) for a, b in ev)
-    if dist:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    clocks = sampler.stop() if sampler else None
+    total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), dist, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * shape.M * len(cfgs) / len(cfgs) / (ms_per_step * 1e-3)
+    value = replicas.job_throughput(shape.M, args.steps, world, total_ms * 1e-3)
 
     # ---- per-kernel device times (a second, instrumented pass: event pairs around every launch)
     kern = []
@@ -278,6 +272,8 @@ def run_ours(args):
             flush.zero_()
             step()
         recs = h.profile_end()
+    clocks = sampler.stop() if sampler else None
+    if rank == 0:
         table = []
         for cfg in cfgs:
             table += kernel_table(shape, cfg)
@@ -344,12 +340,8 @@ def run_ours(args):
     for _ in range(args.steps):
         e2e_step()
     torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if dist:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * shape.M * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+    e2e_s = replicas.max_over_ranks(time.perf_counter() - t0, dist, "cuda")
+    e2e = {"value": replicas.job_throughput(shape.M, args.steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
     h.check()
 
     if rank != 0:

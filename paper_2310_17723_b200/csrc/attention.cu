@@ -9,96 +9,46 @@
 // operand layout and accumulates P_u8 V in tensor memory.  INT8 Q K^T is cheap enough (one eighth of
 // the exponential cost) that recomputing beats spilling the scores.
 //
-// One CTA per (batch, head, 128-query tile); 10 warps:
-//   warps 0-7  softmax / epilogue: row r = 32 * (w % 4) + lane, columns 64 * (w / 4) .. +63 of a block
-//   warp  8    TMA producer (Q once, K per block and sweep, V per block in sweep 2)
-//   warp  9    UMMA issuer (one lane) and owner of the TMEM allocation
-// TMEM: two score buffers of 128 columns (double-buffered against the softmax warps) + dh output columns.
-#include "common.cuh"
-#include "ptx.cuh"
-#include <climits>
-#include <cmath>
-#include <cuda_fp16.h>
-#include <cuda_bf16.h>
+// Persistent: one CTA per SM walks the (batch, head, 128-query tile) list; the K / V / Q rings and the score
+// buffers keep running across tile boundaries, so the next tile's operands load and its first Q K^T issues while
+// the current tile's epilogue is still draining.  18 warps:
+//   warps 0-15 softmax / epilogue: row r = 32 * (w % 4) + lane, columns 32 * (w / 4) .. +31 of a block
+//   warp  16   TMA producer (Q once, K per block and sweep, V per block in sweep 2)
+//   warp  17   UMMA issuer (one lane) and owner of the TMEM allocation
+// The exponentials are the binding resource (16 per clock per SM against 8192 INT8 MACs), so every other
+// conversion stays off that unit: INT32 scores become floats by an integer add into a float's mantissa
+// and an exact subtraction, and P_u8 is rounded by adding 1.5 * 2^23 inside an FMA.
+// TMEM: three score buffers of 128 columns (the UMMA issuer runs two blocks ahead of the softmax warps, which
+// hides the issue -> commit -> barrier -> tcgen05.ld round trip) + dh output columns.
+#include "attention_common.cuh"
 
 namespace hero {
-
-constexpr int ATT_BM = 128;      // queries per CTA
-constexpr int ATT_BN = 128;      // keys per block
-constexpr int ATT_THREADS = 320;
-constexpr int ATT_KSTAGES = 3;
-constexpr int ATT_VSTAGES = 2;
-
-struct AttnParams {
-  int B, S, nh, dh;
-  int nqt;                 // query tiles per sequence
-  float c2;                // d~ * log2(e),  d~ = s_q s_k / sqrt(dh)
-  float inv_sp;            // 1 / s_p
-  float pv_scale;          // s_p * s_v
-  const float* out_scale;  // FWQ [H] (stride 1) / SQ [1] (stride 0); NULL for an FP output
-  int out_scale_stride;
-  int mask;
-  const int* key_len;
-  void* out;
-  long long out_ld;
-  int out_dt;
-  uint32_t idesc_qk, idesc_pv;
-  int* err;
-};
 
 template <int DH>
 struct AttnCfg {
   static constexpr int TILE = ATT_BM * DH;                     // bytes of a Q / K / V tile (INT8)
   static constexpr int P_TILE = ATT_BM * ATT_BN;               // bytes of a P_u8 tile
-  static constexpr int OFF_K = TILE;
-  static constexpr int OFF_V = OFF_K + ATT_KSTAGES * TILE;
-  static constexpr int OFF_P = OFF_V + ATT_VSTAGES * TILE;
-  static constexpr int OFF_STATS = OFF_P + 2 * P_TILE;         // float2 [2][128]
-  static constexpr int OFF_BARS = OFF_STATS + 2 * ATT_BM * 8;
-  static constexpr int SMEM_BYTES = 1024 + OFF_BARS + 32 * 8 + 16;
+  static constexpr int KST = (DH == 64) ? 6 : 4;               // K ring depth (TMA latency ~ several block times)
+  static constexpr int VST = (DH == 64) ? 4 : 3;               // V ring depth
+  static constexpr int OFF_K = 2 * TILE;                       // Q is double-buffered across tiles
+  static constexpr int OFF_V = OFF_K + KST * TILE;
+  static constexpr int OFF_P = OFF_V + VST * TILE;
+  static constexpr int OFF_STATS = OFF_P + 2 * P_TILE;         // float2 [2][4][128]
+  static constexpr int OFF_BARS = OFF_STATS + 2 * 4 * ATT_BM * 8;
+  static constexpr int NBARS = 4 + 2 * KST + 2 * VST + 2 * ATT_NSB + 4 + 2;
+  static constexpr int SMEM_BYTES = 1024 + OFF_BARS + NBARS * 8 + 16;
   static constexpr uint32_t SWZ = (DH == 128) ? ptx::SWZ_128B : ptx::SWZ_64B;
   static constexpr uint32_t SBO = 8 * DH;                      // 8 rows of DH bytes
   static constexpr int TMEM_COLS = 512;
-  static constexpr int O_COL = 256;
+  static constexpr int O_COL = ATT_NSB * ATT_BN;
 };
-
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t sat_u8(float x) {
-  uint32_t r;
-  asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
-}
-__device__ __forceinline__ void st_shared16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ void st_g16(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ uint32_t q4(float a, float b, float c, float d) {
-  int ia = __float2int_rn(fminf(fmaxf(a, -127.f), 127.f));
-  int ib = __float2int_rn(fminf(fmaxf(b, -127.f), 127.f));
-  int ic = __float2int_rn(fminf(fmaxf(c, -127.f), 127.f));
-  int id = __float2int_rn(fminf(fmaxf(d, -127.f), 127.f));
-  return (uint32_t)(ia & 0xff) | ((uint32_t)(ib & 0xff) << 8) | ((uint32_t)(ic & 0xff) << 16) | ((uint32_t)id << 24);
-}
-__device__ __forceinline__ uint32_t fp2(float a, float b, int dt) {
-  if (dt == HERO_F16) {
-    __half2 h = __floats2half2_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&h);
-  }
-  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
 
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   using Cfg = AttnCfg<DH>;
+  constexpr int KST = Cfg::KST, VST = Cfg::VST;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
@@ -107,90 +57,90 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint8_t* sP = smem + Cfg::OFF_P;
   float2* stats = reinterpret_cast<float2*>(smem + Cfg::OFF_STATS);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::OFF_BARS);
-  uint64_t* q_full = bars;            // 1
-  uint64_t* k_full = bars + 1;        // 3
-  uint64_t* k_empty = bars + 4;       // 3
-  uint64_t* v_full = bars + 7;        // 2
-  uint64_t* v_empty = bars + 9;       // 2
-  uint64_t* s_full = bars + 11;       // 2
-  uint64_t* s_empty = bars + 13;      // 2   (8 arrivals: one per softmax warp)
-  uint64_t* p_full = bars + 15;       // 2   (8 arrivals)
-  uint64_t* p_empty = bars + 17;      // 2
-  uint64_t* o_full = bars + 19;       // 1
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+  uint64_t* q_full = bars;                      // [2]
+  uint64_t* q_empty = q_full + 2;               // [2]
+  uint64_t* k_full = q_empty + 2;               // [KST]
+  uint64_t* k_empty = k_full + KST;             // [KST]
+  uint64_t* v_full = k_empty + KST;             // [VST]
+  uint64_t* v_empty = v_full + VST;             // [VST]
+  uint64_t* s_full = v_empty + VST;             // [ATT_NSB]
+  uint64_t* s_empty = s_full + ATT_NSB;         // [ATT_NSB]  one arrival per softmax warp
+  uint64_t* p_full = s_empty + ATT_NSB;               // [2]  one arrival per softmax warp
+  uint64_t* p_empty = p_full + 2;               // [2]
+  uint64_t* o_full = p_empty + 2;               // [1]
+  uint64_t* o_empty = o_full + 1;               // [1]  one arrival per softmax warp
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  // ---- which tile: heavy (late) query tiles first so that causal work balances
-  int idx = blockIdx.x;
-  const int qt = p.nqt - 1 - (idx % p.nqt); idx /= p.nqt;
-  const int h = idx % p.nh;
-  const int b = idx / p.nh;
-  const int q0 = qt * ATT_BM;
-  int klen = p.S;
-  if (p.key_len) klen = min(p.S, max(0, p.key_len[b]));
-  int kv_end = klen;
-  if (p.mask == HERO_MASK_CAUSAL) kv_end = min(kv_end, q0 + ATT_BM);
-  const int nkv = (kv_end + ATT_BN - 1) / ATT_BN;
-  const int row_base = b * p.S;           // first row of this sequence in the [B*S, .] views
-  const int col0 = h * DH;
+  const int total_tiles = p.nqt * p.nh * p.B;
 
   if (threadIdx.x == 0) {
-    ptx::mbar_init(q_full, 1);
-    for (int i = 0; i < ATT_KSTAGES; ++i) { ptx::mbar_init(&k_full[i], 1); ptx::mbar_init(&k_empty[i], 1); }
-    for (int i = 0; i < ATT_VSTAGES; ++i) { ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1); }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_empty[i], 8);
-      ptx::mbar_init(&p_full[i], 8); ptx::mbar_init(&p_empty[i], 1);
+      ptx::mbar_init(&q_full[i], 1); ptx::mbar_init(&q_empty[i], 1);
+      ptx::mbar_init(&p_full[i], ATT_SM_WARPS); ptx::mbar_init(&p_empty[i], 1);
     }
-    ptx::mbar_init(o_full, 1);
+    for (int i = 0; i < ATT_NSB; ++i) { ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_empty[i], ATT_SM_WARPS); }
+    for (int i = 0; i < KST; ++i) { ptx::mbar_init(&k_full[i], 1); ptx::mbar_init(&k_empty[i], 1); }
+    for (int i = 0; i < VST; ++i) { ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1); }
+    ptx::mbar_init(o_full, 1); ptx::mbar_init(o_empty, ATT_SM_WARPS);
     ptx::fence_mbar_init();
   }
-  if (warp == 9) { ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS); ptx::tmem_relinquish(); }
-  if (warp == 8 && lane == 0) { ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); }
+  if (warp == ATT_MMA_WARP) { ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS); ptx::tmem_relinquish(); }
+  if (warp == ATT_TMA_WARP && lane == 0) { ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp == ATT_TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0 && nkv > 0) {
-      ptx::mbar_expect_tx(q_full, Cfg::TILE);
-      ptx::tma_load_2d(sQ, &tmQ, col0, row_base + q0, q_full);
+    // The rings run on across tile boundaries, so the next tile's Q and first K blocks are already in
+    // flight while the softmax warps finish the current tile.
+    if (lane == 0) {
+      uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
       bool ok = true;
-      for (int i = 0; i < 2 * nkv && ok; ++i) {
-        const int j = i < nkv ? i : i - nkv;
-        const int ks = i % ATT_KSTAGES;
-        const uint32_t kph = (i / ATT_KSTAGES) & 1;
-        if (!ptx::mbar_wait(&k_empty[ks], kph ^ 1, p.err, 0x1100 | ks)) { ok = false; break; }
-        ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
-        ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
-        if (i >= nkv) {
-          const int vs = j % ATT_VSTAGES;
-          const uint32_t vph = (j / ATT_VSTAGES) & 1;
-          if (!ptx::mbar_wait(&v_empty[vs], vph ^ 1, p.err, 0x1200 | vs)) { ok = false; break; }
-          ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
-          ptx::tma_load_2d(sV + vs * Cfg::TILE, &tmV, col0, row_base + j * ATT_BN, &v_full[vs]);
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+        const int nkv = attn_nkv(p, qt, b, klen);
+        if (nkv == 0) continue;
+        const int row_base = b * p.S, col0 = h * DH;
+        const int qb = wcnt & 1;
+        if (!ptx::mbar_wait(&q_empty[qb], ((wcnt >> 1) & 1) ^ 1, p.err, 0x1000 | qb)) { ok = false; break; }
+        ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
+        ptx::tma_load_2d(sQ + qb * Cfg::TILE, &tmQ, col0, row_base + qt * ATT_BM, &q_full[qb]);
+        for (int i = 0; i < 2 * nkv; ++i) {
+          const int j = i < nkv ? i : i - nkv;
+          const int ks = kcnt % KST;
+          if (!ptx::mbar_wait(&k_empty[ks], ((kcnt / KST) & 1) ^ 1, p.err, 0x1100 | ks)) { ok = false; break; }
+          ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
+          ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
+          ++kcnt;
+          if (i >= nkv) {
+            const int vs = vcnt % VST;
+            if (!ptx::mbar_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x1200 | vs)) { ok = false; break; }
+            ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
+            ptx::tma_load_2d(sV + vs * Cfg::TILE, &tmV, col0, row_base + j * ATT_BN, &v_full[vs]);
+            ++vcnt;
+          }
         }
+        ++wcnt;
       }
-      // drain: the last copies have landed (and been consumed) before the CTA may exit
-      if (ok) ptx::mbar_wait(o_full, 0, p.err, 0x1300);
     }
     __syncwarp();
-  } else if (warp == 9) {
+  } else if (warp == ATT_MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0 && nkv > 0) {
+    if (lane == 0) {
       constexpr uint64_t kmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // Q, K: K-major rows of DH bytes
       constexpr uint64_t pmaj = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);      // P: K-major rows of 128 bytes
       constexpr uint64_t vmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // V: MN-major, 8-key groups
-      bool ok = ptx::mbar_wait(q_full, 0, p.err, 0x2000);
-      const uint32_t q_addr = ptx::smem_u32(sQ);
+      uint32_t kcnt = 0, vcnt = 0, scnt = 0, pcnt = 0, wcnt = 0;
+      bool ok = true;
 
       auto issue_pv = [&](int j) -> bool {
-        const int vs = j % ATT_VSTAGES, pb = j & 1;
-        if (!ptx::mbar_wait(&v_full[vs], (j / ATT_VSTAGES) & 1, p.err, 0x2100 | vs)) return false;
-        if (!ptx::mbar_wait(&p_full[pb], (j >> 1) & 1, p.err, 0x2200 | pb)) return false;
+        if (j == 0 && !ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x2500)) return false;   // previous tile's O read out
+        const int vs = vcnt % VST, pb = pcnt & 1;
+        if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x2100 | vs)) return false;
+        if (!ptx::mbar_wait(&p_full[pb], (pcnt >> 1) & 1, p.err, 0x2200 | pb)) return false;
         ptx::tc_fence_after();
         const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
         const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
@@ -200,170 +150,207 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                        ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (j | k) != 0);
         ptx::umma_commit(&v_empty[vs]);
         ptx::umma_commit(&p_empty[pb]);
+        ++vcnt; ++pcnt;
         return true;
       };
 
-      for (int i = 0; i < 2 * nkv && ok; ++i) {
-        const int ks = i % ATT_KSTAGES, sb = i & 1;
-        if (!ptx::mbar_wait(&k_full[ks], (i / ATT_KSTAGES) & 1, p.err, 0x2300 | ks)) { ok = false; break; }
-        if (!ptx::mbar_wait(&s_empty[sb], ((i >> 1) & 1) ^ 1, p.err, 0x2400 | sb)) { ok = false; break; }
-        ptx::tc_fence_after();
-        const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+        const int nkv = attn_nkv(p, qt, b, klen);
+        if (nkv == 0) continue;
+        const int qb = wcnt & 1;
+        if (!ptx::mbar_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x2000 | qb)) { ok = false; break; }
+        const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
+        for (int i = 0; i < 2 * nkv && ok; ++i) {
+          const int ks = kcnt % KST, sb = scnt % ATT_NSB;
+          if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x2300 | ks)) { ok = false; break; }
+          if (!ptx::mbar_wait(&s_empty[sb], ((scnt / ATT_NSB) & 1) ^ 1, p.err, 0x2400 | sb)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
 #pragma unroll
-        for (int k = 0; k < DH / 32; ++k)
-          ptx::umma_i8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                       ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
-        ptx::umma_commit(&k_empty[ks]);
-        ptx::umma_commit(&s_full[sb]);
-        if (i >= nkv + 1) ok = issue_pv(i - nkv - 1);
+          for (int k = 0; k < DH / 32; ++k)
+            ptx::umma_i8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                         ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+          ptx::umma_commit(&k_empty[ks]);
+          ptx::umma_commit(&s_full[sb]);
+          ++kcnt; ++scnt;
+          if (i == 2 * nkv - 1) ptx::umma_commit(&q_empty[qb]);   // Q buffer free once these MMAs have read it
+          if (i >= nkv + 1) ok = issue_pv(i - nkv - 1);
+        }
+        if (ok) ok = issue_pv(nkv - 1);
+        if (ok) ptx::umma_commit(o_full);
+        ++wcnt;
       }
-      if (ok) ok = issue_pv(nkv - 1);
-      if (ok) ptx::umma_commit(o_full);
     }
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ softmax + epilogue warps
-    const int quarter = warp & 3, half = warp >> 2;
+    const int quarter = warp & 3, cq = warp >> 2;            // TMEM lane quarter, 32-column group of a block
     const int r_loc = quarter * 32 + lane;
-    const int q = q0 + r_loc;
-    const bool row_ok = q < p.S;
-    int kmax = klen - 1;                                     // last allowed key (inclusive)
-    if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const float c2 = p.c2;
+    uint32_t scnt = 0, pcnt = 0, wcnt = 0;
     bool ok = true;
 
-    float m = -INFINITY, l = 0.f;
-    // ---- sweep 1: running row max and row sum (log2 domain)
-    for (int i = 0; i < nkv; ++i) {
-      const int sb = i & 1;
-      if (ok && !ptx::mbar_wait(&s_full[sb], (i >> 1) & 1, p.err, 0x3000 | sb)) ok = false;
-      ptx::tc_fence_after();
-      if (ok) {
-#pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+      const int nkv = attn_nkv(p, qt, b, klen);
+      const int q0 = qt * ATT_BM, row_base = b * p.S, col0 = h * DH;
+      const int q = q0 + r_loc;
+      const bool row_ok = q < p.S;
+      int kmax = klen - 1;                                   // last allowed key (inclusive)
+      if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
+
+      float m = -INFINITY, l = 0.f;
+      // ---- sweep 1: running row max and row sum (log2 domain)
+      for (int i = 0; i < nkv; ++i, ++scnt) {
+        const int sb = scnt % ATT_NSB;
+        if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x3000 | sb)) ok = false;
+        ptx::tc_fence_after();
+        if (ok) {
           uint32_t r[32];
-          ptx::tmem_ld32(t_lane + sb * ATT_BN + half * 64 + cc * 32, r);
+          ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
           ptx::tmem_ld_wait();
-          const int kb = i * ATT_BN + half * 64 + cc * 32;
+          const int kb = i * ATT_BN + cq * 32;
           const int nvalid = min(32, kmax - kb + 1);       // keys kb .. kb + nvalid - 1 are allowed
-          if (nvalid <= 0) continue;
-          int imax = INT_MIN;
-          if (nvalid == 32) {
+          if (nvalid > 0) {
+            int imax = INT_MIN;
+            if (nvalid == 32) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) imax = max(imax, (int)r[j]);
-          } else {
+              for (int j = 0; j < 32; ++j) imax = max(imax, (int)r[j]);
+            } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) imax = max(imax, j < nvalid ? (int)r[j] : INT_MIN);
-          }
-          const float m_new = fmaxf(m, (float)imax * c2);
-          float acc = 0.f;
-          if (nvalid == 32) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc += ex2f(fmaf((float)(int)r[j], c2, -m_new));
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc += j < nvalid ? ex2f(fmaf((float)(int)r[j], c2, -m_new)) : 0.f;
-          }
-          l = l * ex2f(m - m_new) + acc;                    // m = -inf on first use: 2^-inf = 0
-          m = m_new;
-        }
-      }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
-    }
-    // ---- combine the two column halves of each row
-    stats[half * ATT_BM + r_loc] = make_float2(m, l);
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    {
-      const float2 o = stats[(half ^ 1) * ATT_BM + r_loc];
-      const float mf = fmaxf(m, o.x);
-      float lf = 0.f;
-      if (mf > -INFINITY) lf = (m > -INFINITY ? l * ex2f(m - mf) : 0.f) + (o.x > -INFINITY ? o.y * ex2f(o.x - mf) : 0.f);
-      m = mf; l = lf;
-    }
-    // P_u8 = Round(P / s_p) with P = 2^(t - m) / l
-    const float pscale = l > 0.f ? p.inv_sp / l : 0.f;
-
-    // ---- sweep 2: scores again -> P_u8 in shared memory (UMMA K-major, 128-byte swizzle)
-    for (int j = 0; j < nkv; ++j) {
-      const int i = nkv + j, sb = i & 1, pb = j & 1;
-      if (ok && !ptx::mbar_wait(&s_full[sb], (i >> 1) & 1, p.err, 0x3100 | sb)) ok = false;
-      if (ok && !ptx::mbar_wait(&p_empty[pb], ((j >> 1) & 1) ^ 1, p.err, 0x3200 | pb)) ok = false;
-      ptx::tc_fence_after();
-      if (ok) {
-        const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
-#pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
-          uint32_t r[32];
-          ptx::tmem_ld32(t_lane + sb * ATT_BN + half * 64 + cc * 32, r);
-          ptx::tmem_ld_wait();
-          const int kb = j * ATT_BN + half * 64 + cc * 32;
-          const int nvalid = min(32, kmax - kb + 1);
-          uint32_t w[8];
-#pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            uint32_t word = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int jj = 4 * g + e;
-              float pe = ex2f(fmaf((float)(int)r[jj], c2, -m)) * pscale;
-              if (jj >= nvalid) pe = 0.f;
-              word |= sat_u8(pe) << (8 * e);
+              for (int j = 0; j < 32; ++j) imax = max(imax, j < nvalid ? (int)r[j] : INT_MIN);
             }
-            w[g] = word;
+            const float m_new = fmaxf(m, (float)imax * c2);
+            float2 acc2 = make_float2(0.f, 0.f);
+            const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_new, -m_new), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
+            if (nvalid == 32) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                const float2 f = __fadd2_rn(make_float2(__uint_as_float(0x4B400000u + r[j]), __uint_as_float(0x4B400000u + r[j + 1])), mg);
+                const float2 tt = __ffma2_rn(f, c22, nm2);
+                acc2 = __fadd2_rn(acc2, make_float2(ex2f(tt.x), ex2f(tt.y)));
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) acc2.x += j < nvalid ? ex2f(fmaf(score_to_float(r[j]), c2, -m_new)) : 0.f;
+            }
+            l = l * ex2f(m - m_new) + (acc2.x + acc2.y);    // m = -inf on first use: 2^-inf = 0
+            m = m_new;
           }
-          const int c16 = half * 4 + cc * 2;                // 16-byte chunk index within the 128-byte row
-          st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
-          st_shared16(prow + (((c16 + 1) ^ (r_loc & 7)) << 4), w[4], w[5], w[6], w[7]);
         }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
       }
-      ptx::tc_fence_before();
-      ptx::fence_proxy_async_smem();                         // generic-proxy writes -> visible to the UMMA (async proxy)
-      __syncwarp();
-      if (lane == 0) { ptx::mbar_arrive(&s_empty[sb]); ptx::mbar_arrive(&p_full[pb]); }
-    }
+      // ---- combine the four column groups of each row (buffer alternates with the tile)
+      float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
+      st[cq * ATT_BM + r_loc] = make_float2(m, l);
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      {
+        float mf = -INFINITY;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
+        float lf = 0.f;
+        if (mf > -INFINITY) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const float2 o = st[g * ATT_BM + r_loc];
+            if (o.x > -INFINITY) lf += o.y * ex2f(o.x - mf);
+          }
+        }
+        m = mf; l = lf;
+      }
+      // P_u8 = Round(P / s_p) with P = 2^(t - m) / l
+      const float pscale = l > 0.f ? p.inv_sp / l : 0.f;
 
-    // ---- epilogue: X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8)
-    if (nkv > 0 && ok && !ptx::mbar_wait(o_full, 0, p.err, 0x3300)) ok = false;
-    ptx::tc_fence_after();
-    constexpr int NCH = DH / 64;                             // 32-column chunks per half
-#pragma unroll 1
-    for (int cc = 0; cc < NCH; ++cc) {
-      uint32_t r[32];
-      const int ocol = half * (DH / 2) + cc * 32;
-      if (nkv > 0 && ok) {
-        ptx::tmem_ld32(t_lane + Cfg::O_COL + ocol, r);
-        ptx::tmem_ld_wait();
-      } else {
+      // ---- sweep 2: scores again -> P_u8 in shared memory (UMMA K-major, 128-byte swizzle)
+      for (int j = 0; j < nkv; ++j, ++scnt, ++pcnt) {
+        const int sb = scnt % ATT_NSB, pb = pcnt & 1;
+        if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x3100 | sb)) ok = false;
+        if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt >> 1) & 1) ^ 1, p.err, 0x3200 | pb)) ok = false;
+        ptx::tc_fence_after();
+        if (ok) {
+          const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
+          uint32_t r[32];
+          ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
+          ptx::tmem_ld_wait();
+          const int kb = j * ATT_BN + cq * 32;
+          const int nvalid = min(32, kmax - kb + 1);
+          float y[32];
+          const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m, -m), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
+          const float2 ps2 = make_float2(pscale, pscale), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) r[j] = 0;               // every key masked: the row is zero
+          for (int e = 0; e < 32; e += 2) {
+            // Round(P / s_p) clipped to 255: round-half-to-even happens in the FMA's single rounding
+            const float2 f = __fadd2_rn(make_float2(__uint_as_float(0x4B400000u + r[e]), __uint_as_float(0x4B400000u + r[e + 1])), mg);
+            const float2 tt = __ffma2_rn(f, c22, nm2);
+            const float2 v = __ffma2_rn(make_float2(ex2f(tt.x), ex2f(tt.y)), ps2, rm2);
+            y[e] = fminf(v.x, ATT_MAGIC + 255.0f);
+            y[e + 1] = fminf(v.y, ATT_MAGIC + 255.0f);
+          }
+          if (nvalid < 32) {                                   // block straddles the mask: masked keys get code 0
+#pragma unroll
+            for (int e = 0; e < 32; ++e) if (e >= nvalid) y[e] = ATT_MAGIC;
+          }
+          const int c16 = cq * 2;                              // 16-byte chunk index within the 128-byte row
+          st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), low_bytes4_u(y[0], y[1], y[2], y[3]), low_bytes4_u(y[4], y[5], y[6], y[7]),
+                      low_bytes4_u(y[8], y[9], y[10], y[11]), low_bytes4_u(y[12], y[13], y[14], y[15]));
+          st_shared16(prow + (((c16 + 1) ^ (r_loc & 7)) << 4), low_bytes4_u(y[16], y[17], y[18], y[19]),
+                      low_bytes4_u(y[20], y[21], y[22], y[23]), low_bytes4_u(y[24], y[25], y[26], y[27]),
+                      low_bytes4_u(y[28], y[29], y[30], y[31]));
+        }
+        ptx::tc_fence_before();
+        ptx::fence_proxy_async_smem();                         // generic-proxy writes -> visible to the UMMA (async proxy)
+        __syncwarp();
+        if (lane == 0) { ptx::mbar_arrive(&s_empty[sb]); ptx::mbar_arrive(&p_full[pb]); }
       }
-      if (!row_ok) continue;
-      const long long grow = (long long)(row_base + q);
-      const int gcol = col0 + ocol;
-      if (p.out_dt == HERO_I8) {
-        float v[32];
+
+      // ---- epilogue: X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8); 32 output columns per warp
+      uint32_t r[32];
+      if (nkv > 0) {
+        if (ok && !ptx::mbar_wait(o_full, wcnt & 1, p.err, 0x3300)) ok = false;
+        ptx::tc_fence_after();
+        if (ok && cq * 32 < DH) {
+          ptx::tmem_ld32(t_lane + Cfg::O_COL + cq * 32, r);
+          ptx::tmem_ld_wait();
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(o_empty);              // the accumulator may be overwritten by the next tile
+        ++wcnt;
+      }
+      if (nkv == 0 || !ok) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          v[j] = (float)(int)r[j] * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
-        int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
+        for (int j = 0; j < 32; ++j) r[j] = 0;                 // every key masked: the row is zero
+      }
+      if (cq * 32 < DH && row_ok) {
+        const int ocol = cq * 32;
+        const long long grow = (long long)(row_base + q);
+        const int gcol = col0 + ocol;
+        if (p.out_dt == HERO_I8) {
+          float v[32];
 #pragma unroll
-        for (int g = 0; g < 2; ++g)
-          st_g16(dst + 16 * g, q4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
-                 q4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
-                 q4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
-                 q4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
-      } else {
-        uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + grow * p.out_ld + gcol;
+          for (int j = 0; j < 32; ++j)
+            v[j] = (float)(int)r[j] * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
+          int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          float v[8];
+          for (int g = 0; g < 2; ++g)
+            st_g16(dst + 16 * g, q4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
+                   q4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
+                   q4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
+                   q4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
+        } else {
+          uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + grow * p.out_ld + gcol;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * p.pv_scale;
-          st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
-                 fp2(v[6], v[7], p.out_dt));
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * p.pv_scale;
+            st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
+                   fp2(v[6], v[7], p.out_dt));
+          }
         }
       }
     }
@@ -371,7 +358,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 9) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
 template <int DH>
@@ -391,10 +378,11 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
     configured = true;
   }
-  const long long grid = (long long)p.nqt * a->nh * a->B;
+  const long long tiles = (long long)p.nqt * a->nh * a->B;
+  const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);   // persistent: one CTA per SM
   {
     LaunchScope scope(h, stream, KERNEL_ATTN);
-    kern<<<(unsigned)grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+    kern<<<grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(tq, tk, tv, p);
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
@@ -408,9 +396,11 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   HERO_REQUIRE(a->q && a->k && a->v, HERO_ERR_INVALID_ARG, "q, k, v are required");
   HERO_REQUIRE(a->B >= 0 && a->S > 0 && a->nh > 0, HERO_ERR_INVALID_ARG, "bad B / S / nh");
   HERO_REQUIRE(a->dh == 64 || a->dh == 128, HERO_ERR_UNSUPPORTED, "dh=%d: 64 or 128 supported", a->dh);
-  HERO_REQUIRE(a->dtype == HERO_I8, HERO_ERR_UNSUPPORTED, "q/k/v dtype %d: this build runs the INT8 core only", a->dtype);
-  HERO_REQUIRE(aligned16(a->q) && aligned16(a->k) && aligned16(a->v) && a->ld % 16 == 0 && a->ld >= (int64_t)a->nh * a->dh,
-               HERO_ERR_ALIGNMENT, "q/k/v must be 16-byte aligned with ld a multiple of 16 and >= nh*dh");
+  const bool fp_in = is_fp16ish(a->dtype);
+  HERO_REQUIRE(a->dtype == HERO_I8 || fp_in, HERO_ERR_UNSUPPORTED, "q/k/v dtype %d: INT8, F16 or BF16 expected", a->dtype);
+  HERO_REQUIRE(aligned16(a->q) && aligned16(a->k) && aligned16(a->v) && (a->ld * (fp_in ? 2 : 1)) % 16 == 0 &&
+               a->ld >= (int64_t)a->nh * a->dh,
+               HERO_ERR_ALIGNMENT, "q/k/v must be 16-byte aligned with a row pitch that is a multiple of 16 bytes and ld >= nh*dh");
   hero_status st;
   if ((st = check_matrix(a->out, "out")) != HERO_OK) return st;
   HERO_REQUIRE(a->out.rows == (int64_t)a->B * a->S && a->out.cols == (int64_t)a->nh * a->dh, HERO_ERR_INVALID_ARG,
@@ -419,9 +409,9 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   if (a->out.dtype == HERO_I8)
     HERO_REQUIRE((a->out.gran == HERO_GRAN_FWQ || a->out.gran == HERO_GRAN_SQ) && a->out.scale, HERO_ERR_UNSUPPORTED,
                  "INT8 X_attn is feature-wise (FWQ) or static (SQ) with a calibrated scale (Sec. 2.2.2)");
-  HERO_REQUIRE(a->s_q > 0 && a->s_k > 0 && a->s_v > 0 && a->s_p > 0, HERO_ERR_INVALID_ARG, "scales must be positive");
+  HERO_REQUIRE(fp_in || (a->s_q > 0 && a->s_k > 0 && a->s_v > 0 && a->s_p > 0), HERO_ERR_INVALID_ARG, "scales must be positive");
   HERO_REQUIRE(a->mask == HERO_MASK_NONE || a->mask == HERO_MASK_CAUSAL, HERO_ERR_INVALID_ARG, "unknown mask %d", a->mask);
-  HERO_REQUIRE((int64_t)a->S * 255 * 127 < (1ll << 31), HERO_ERR_UNSUPPORTED, "S=%d would overflow the INT32 accumulator", a->S);
+  HERO_REQUIRE(fp_in || (int64_t)a->S * 255 * 127 < (1ll << 31), HERO_ERR_UNSUPPORTED, "S=%d would overflow the INT32 accumulator", a->S);
   if (a->B == 0) return HERO_OK;
 
   AttnParams p;
@@ -438,6 +428,7 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   p.err = h->d_error;
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (fp_in) return attn_fp_dispatch(h, a, p, s);
   if (a->dh == 64) return launch_attn<64>(h, a, p, s);
   return launch_attn<128>(h, a, p, s);
 }

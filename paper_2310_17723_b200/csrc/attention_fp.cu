@@ -1,0 +1,357 @@
+// FP16 / BF16 attention for a module the mode table leaves in FP (Sec. 2.3, Table 1; Eq. 9-11):
+// P = softmax(Q K^T / sqrt(dh)), X_attn = P V with fp32 accumulation, stored in FP16 / BF16 or, when the
+// attention-output linear is INT8, quantized by the calibrated S_attn in the epilogue (no standalone
+// quantize kernel).  Same persistent, two-sweep, TMEM-resident structure as the INT8 core so that the two
+// paths differ only in operand type: kind::f16 MMAs, fp32 scores, P stored as FP16 / BF16 in the UMMA
+// operand layout.  A tile row of 128 features is 256 bytes, i.e. two 128-byte-swizzled sub-tiles.
+#include "attention_common.cuh"
+
+namespace hero {
+
+template <int DH>
+struct AttnFpCfg {
+  static constexpr int SUB = ATT_BM * 128;                     // bytes of one [128 rows x 64 elements] sub-tile
+  static constexpr int NSUB = DH / 64;                         // sub-tiles per Q / K / V tile
+  static constexpr int TILE = SUB * NSUB;
+  static constexpr int P_TILE = 2 * SUB;                       // [128 x 128 keys] FP16
+  static constexpr int QB = (DH == 64) ? 2 : 1;                // Q buffers
+  static constexpr int KST = (DH == 64) ? 4 : 2;
+  static constexpr int VST = (DH == 64) ? 3 : 2;
+  static constexpr int PB = (DH == 64) ? 2 : 1;                // P buffers
+  static constexpr int OFF_K = QB * TILE;
+  static constexpr int OFF_V = OFF_K + KST * TILE;
+  static constexpr int OFF_P = OFF_V + VST * TILE;
+  static constexpr int OFF_STATS = OFF_P + PB * P_TILE;        // float2 [2][4][128]
+  static constexpr int OFF_BARS = OFF_STATS + 2 * 4 * ATT_BM * 8;
+  static constexpr int NBARS = 2 * QB + 2 * KST + 2 * VST + 2 * ATT_NSB + 2 * PB + 2;
+  static constexpr int SMEM_BYTES = 1024 + OFF_BARS + NBARS * 8 + 16;
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int O_COL = ATT_NSB * ATT_BN;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+               const __grid_constant__ CUtensorMap tmV, const AttnParams p, const int in_dt) {
+  using Cfg = AttnFpCfg<DH>;
+  constexpr int KST = Cfg::KST, VST = Cfg::VST, QB = Cfg::QB, PB = Cfg::PB, NSUB = Cfg::NSUB;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + Cfg::OFF_K;
+  uint8_t* sV = smem + Cfg::OFF_V;
+  uint8_t* sP = smem + Cfg::OFF_P;
+  float2* stats = reinterpret_cast<float2*>(smem + Cfg::OFF_STATS);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::OFF_BARS);
+  uint64_t* q_full = bars;                      // [QB]
+  uint64_t* q_empty = q_full + QB;              // [QB]
+  uint64_t* k_full = q_empty + QB;              // [KST]
+  uint64_t* k_empty = k_full + KST;             // [KST]
+  uint64_t* v_full = k_empty + KST;             // [VST]
+  uint64_t* v_empty = v_full + VST;             // [VST]
+  uint64_t* s_full = v_empty + VST;             // [ATT_NSB]
+  uint64_t* s_empty = s_full + ATT_NSB;         // [ATT_NSB]
+  uint64_t* p_full = s_empty + ATT_NSB;               // [PB]
+  uint64_t* p_empty = p_full + PB;              // [PB]
+  uint64_t* o_full = p_empty + PB;              // [1]
+  uint64_t* o_empty = o_full + 1;               // [1]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_tiles = p.nqt * p.nh * p.B;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < QB; ++i) { ptx::mbar_init(&q_full[i], 1); ptx::mbar_init(&q_empty[i], 1); }
+    for (int i = 0; i < ATT_NSB; ++i) { ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_empty[i], ATT_SM_WARPS); }
+    for (int i = 0; i < PB; ++i) { ptx::mbar_init(&p_full[i], ATT_SM_WARPS); ptx::mbar_init(&p_empty[i], 1); }
+    for (int i = 0; i < KST; ++i) { ptx::mbar_init(&k_full[i], 1); ptx::mbar_init(&k_empty[i], 1); }
+    for (int i = 0; i < VST; ++i) { ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1); }
+    ptx::mbar_init(o_full, 1); ptx::mbar_init(o_empty, ATT_SM_WARPS);
+    ptx::fence_mbar_init();
+  }
+  if (warp == ATT_MMA_WARP) { ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS); ptx::tmem_relinquish(); }
+  if (warp == ATT_TMA_WARP && lane == 0) { ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == ATT_TMA_WARP) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+        const int nkv = attn_nkv(p, qt, b, klen);
+        if (nkv == 0) continue;
+        const int row_base = b * p.S, col0 = h * DH;
+        const int qb = wcnt % QB;
+        if (!ptx::mbar_wait(&q_empty[qb], ((wcnt / QB) & 1) ^ 1, p.err, 0x4000 | qb)) { ok = false; break; }
+        ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
+#pragma unroll
+        for (int sIdx = 0; sIdx < NSUB; ++sIdx)
+          ptx::tma_load_2d(sQ + qb * Cfg::TILE + sIdx * Cfg::SUB, &tmQ, col0 + sIdx * 64, row_base + qt * ATT_BM, &q_full[qb]);
+        for (int i = 0; i < 2 * nkv; ++i) {
+          const int j = i < nkv ? i : i - nkv;
+          const int ks = kcnt % KST;
+          if (!ptx::mbar_wait(&k_empty[ks], ((kcnt / KST) & 1) ^ 1, p.err, 0x4100 | ks)) { ok = false; break; }
+          ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
+#pragma unroll
+          for (int sIdx = 0; sIdx < NSUB; ++sIdx)
+            ptx::tma_load_2d(sK + ks * Cfg::TILE + sIdx * Cfg::SUB, &tmK, col0 + sIdx * 64, row_base + j * ATT_BN, &k_full[ks]);
+          ++kcnt;
+          if (i >= nkv) {
+            const int vs = vcnt % VST;
+            if (!ptx::mbar_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x4200 | vs)) { ok = false; break; }
+            ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
+#pragma unroll
+            for (int sIdx = 0; sIdx < NSUB; ++sIdx)
+              ptx::tma_load_2d(sV + vs * Cfg::TILE + sIdx * Cfg::SUB, &tmV, col0 + sIdx * 64, row_base + j * ATT_BN, &v_full[vs]);
+            ++vcnt;
+          }
+        }
+        ++wcnt;
+      }
+    }
+    __syncwarp();
+  } else if (warp == ATT_MMA_WARP) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint64_t kmaj = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);          // Q, K, P: K-major, 128-byte rows
+      constexpr uint64_t vmaj = ptx::smem_desc_base(Cfg::SUB, 1024, ptx::SWZ_128B);    // V: MN-major; 64-feature chunks SUB apart
+      uint32_t kcnt = 0, vcnt = 0, scnt = 0, pcnt = 0, wcnt = 0;
+      bool ok = true;
+
+      auto issue_pv = [&](int j) -> bool {
+        if (j == 0 && !ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x5500)) return false;
+        const int vs = vcnt % VST, pb = pcnt % PB;
+        if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x5100 | vs)) return false;
+        if (!ptx::mbar_wait(&p_full[pb], (pcnt / PB) & 1, p.err, 0x5200 | pb)) return false;
+        ptx::tc_fence_after();
+        const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
+        const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
+#pragma unroll
+        for (int k = 0; k < ATT_BN / 16; ++k)      // 16 keys per MMA: 2 eight-key groups of V, 32 bytes of a P row
+          ptx::umma_f16(tmem_base + Cfg::O_COL, ptx::smem_desc(kmaj, p_addr + (k >> 2) * Cfg::SUB + (k & 3) * 32),
+                        ptx::smem_desc(vmaj, v_addr + k * 2048), p.idesc_pv, (j | k) != 0);
+        ptx::umma_commit(&v_empty[vs]);
+        ptx::umma_commit(&p_empty[pb]);
+        ++vcnt; ++pcnt;
+        return true;
+      };
+
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+        const int nkv = attn_nkv(p, qt, b, klen);
+        if (nkv == 0) continue;
+        const int qb = wcnt % QB;
+        if (!ptx::mbar_wait(&q_full[qb], (wcnt / QB) & 1, p.err, 0x5000 | qb)) { ok = false; break; }
+        const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
+        for (int i = 0; i < 2 * nkv && ok; ++i) {
+          const int ks = kcnt % KST, sb = scnt % ATT_NSB;
+          if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x5300 | ks)) { ok = false; break; }
+          if (!ptx::mbar_wait(&s_empty[sb], ((scnt / ATT_NSB) & 1) ^ 1, p.err, 0x5400 | sb)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+#pragma unroll
+          for (int k = 0; k < DH / 16; ++k)
+            ptx::umma_f16(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + (k >> 2) * Cfg::SUB + (k & 3) * 32),
+                          ptx::smem_desc(kmaj, k_addr + (k >> 2) * Cfg::SUB + (k & 3) * 32), p.idesc_qk, k != 0);
+          ptx::umma_commit(&k_empty[ks]);
+          ptx::umma_commit(&s_full[sb]);
+          ++kcnt; ++scnt;
+          if (i == 2 * nkv - 1) ptx::umma_commit(&q_empty[qb]);
+          if (i >= nkv + 1) ok = issue_pv(i - nkv - 1);
+        }
+        if (ok) ok = issue_pv(nkv - 1);
+        if (ok) ptx::umma_commit(o_full);
+        ++wcnt;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue warps
+    const int quarter = warp & 3, cq = warp >> 2;
+    const int r_loc = quarter * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const float c2 = p.c2;                                   // log2(e) / sqrt(dh)
+    uint32_t scnt = 0, pcnt = 0, wcnt = 0;
+    bool ok = true;
+
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+      const int nkv = attn_nkv(p, qt, b, klen);
+      const int q0 = qt * ATT_BM, row_base = b * p.S, col0 = h * DH;
+      const int q = q0 + r_loc;
+      const bool row_ok = q < p.S;
+      int kmax = klen - 1;
+      if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
+
+      float m = -INFINITY, l = 0.f;
+      // ---- sweep 1: running row max and row sum (log2 domain)
+      for (int i = 0; i < nkv; ++i, ++scnt) {
+        const int sb = scnt % ATT_NSB;
+        if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x6000 | sb)) ok = false;
+        ptx::tc_fence_after();
+        if (ok) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
+          ptx::tmem_ld_wait();
+          const int kb = i * ATT_BN + cq * 32;
+          const int nvalid = min(32, kmax - kb + 1);
+          if (nvalid > 0) {
+            float smax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) smax = fmaxf(smax, j < nvalid ? __uint_as_float(r[j]) : -INFINITY);
+            const float m_new = fmaxf(m, smax * c2);
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc += j < nvalid ? ex2f(fmaf(__uint_as_float(r[j]), c2, -m_new)) : 0.f;
+            l = l * ex2f(m - m_new) + acc;
+            m = m_new;
+          }
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
+      }
+      float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
+      st[cq * ATT_BM + r_loc] = make_float2(m, l);
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      {
+        float mf = -INFINITY;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
+        float lf = 0.f;
+        if (mf > -INFINITY) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const float2 o = st[g * ATT_BM + r_loc];
+            if (o.x > -INFINITY) lf += o.y * ex2f(o.x - mf);
+          }
+        }
+        m = mf; l = lf;
+      }
+      const float inv_l = l > 0.f ? 1.0f / l : 0.f;
+
+      // ---- sweep 2: P = 2^(t - m) / l as FP16 / BF16 into shared memory (two 64-key sub-tiles, 128-byte swizzle)
+      for (int j = 0; j < nkv; ++j, ++scnt, ++pcnt) {
+        const int sb = scnt % ATT_NSB, pb = pcnt % PB;
+        if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x6100 | sb)) ok = false;
+        if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt / PB) & 1) ^ 1, p.err, 0x6200 | pb)) ok = false;
+        ptx::tc_fence_after();
+        if (ok) {
+          const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (cq >> 1) * Cfg::SUB + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
+          uint32_t r[32];
+          ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
+          ptx::tmem_ld_wait();
+          const int kb = j * ATT_BN + cq * 32;
+          const int nvalid = min(32, kmax - kb + 1);
+          uint32_t w[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            float a = ex2f(fmaf(__uint_as_float(r[2 * e]), c2, -m)) * inv_l;
+            float c = ex2f(fmaf(__uint_as_float(r[2 * e + 1]), c2, -m)) * inv_l;
+            if (2 * e >= nvalid) a = 0.f;
+            if (2 * e + 1 >= nvalid) c = 0.f;
+            w[e] = fp2(a, c, in_dt);
+          }
+          const int c16 = (cq & 1) * 4;                      // first 16-byte chunk of this thread's 64 bytes
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+        }
+        ptx::tc_fence_before();
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) { ptx::mbar_arrive(&s_empty[sb]); ptx::mbar_arrive(&p_full[pb]); }
+      }
+
+      // ---- epilogue
+      uint32_t r[32];
+      if (nkv > 0) {
+        if (ok && !ptx::mbar_wait(o_full, wcnt & 1, p.err, 0x6300)) ok = false;
+        ptx::tc_fence_after();
+        if (ok && cq * 32 < DH) {
+          ptx::tmem_ld32(t_lane + Cfg::O_COL + cq * 32, r);
+          ptx::tmem_ld_wait();
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(o_empty);
+        ++wcnt;
+      }
+      if (nkv == 0 || !ok) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r[j] = 0;
+      }
+      if (cq * 32 < DH && row_ok) {
+        const long long grow = (long long)(row_base + q);
+        const int gcol = col0 + cq * 32;
+        if (p.out_dt == HERO_I8) {
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride);
+          int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
+#pragma unroll
+          for (int g = 0; g < 2; ++g)
+            st_g16(dst + 16 * g, q4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
+                   q4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
+                   q4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
+                   q4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
+        } else {
+          uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + grow * p.out_ld + gcol;
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            st_g16(dst + 8 * g, fp2(__uint_as_float(r[8 * g]), __uint_as_float(r[8 * g + 1]), p.out_dt),
+                   fp2(__uint_as_float(r[8 * g + 2]), __uint_as_float(r[8 * g + 3]), p.out_dt),
+                   fp2(__uint_as_float(r[8 * g + 4]), __uint_as_float(r[8 * g + 5]), p.out_dt),
+                   fp2(__uint_as_float(r[8 * g + 6]), __uint_as_float(r[8 * g + 7]), p.out_dt));
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+}
+
+template <int DH>
+static hero_status launch_attn_fp(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
+  using Cfg = AttnFpCfg<DH>;
+  const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
+  const bool bf = a->dtype == HERO_BF16;
+  CUtensorMap tq, tk, tv;
+  hero_status st;
+  // every load is one [128 rows x 64 elements] sub-tile: 128-byte rows, 128-byte swizzle
+  if ((st = make_tmap_2d(h, &tq, a->q, 2, !bf, bf, rows, cols, (uint64_t)a->ld * 2, 64, ATT_BM, 128)) != HERO_OK) return st;
+  if ((st = make_tmap_2d(h, &tk, a->k, 2, !bf, bf, rows, cols, (uint64_t)a->ld * 2, 64, ATT_BN, 128)) != HERO_OK) return st;
+  if ((st = make_tmap_2d(h, &tv, a->v, 2, !bf, bf, rows, cols, (uint64_t)a->ld * 2, 64, ATT_BN, 128)) != HERO_OK) return st;
+  const uint32_t fmt = bf ? 1 : 0;
+  p.idesc_qk = ptx::make_idesc(1, fmt, fmt, 0, 0, ATT_BM, ATT_BN);   // F32 accumulate, both operands K-major
+  p.idesc_pv = ptx::make_idesc(1, fmt, fmt, 0, 1, ATT_BM, DH);       // V is MN-major
+  auto kern = attn_fp_kernel<DH>;
+  static bool configured = false;
+  if (!configured) {
+    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    configured = true;
+  }
+  const long long tiles = (long long)p.nqt * a->nh * a->B;
+  const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);
+  {
+    LaunchScope scope(h, stream, KERNEL_ATTN);
+    kern<<<grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(tq, tk, tv, p, a->dtype);
+  }
+  HERO_CUDA(cudaGetLastError());
+  return HERO_OK;
+}
+
+hero_status attn_fp_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
+  p.c2 = (float)(1.4426950408889634 / sqrt((double)a->dh));
+  if (a->dh == 64) return launch_attn_fp<64>(h, a, p, stream);
+  return launch_attn_fp<128>(h, a, p, stream);
+}
+
+}  // namespace hero

@@ -2,10 +2,11 @@
 // tcgen05 tensor cores with the dequantize / bias / GELU / requantize epilogue applied straight
 // from tensor memory, plus the FP16/BF16 variant for modules left in FP mode (Table 1).
 //
-// One persistent CTA per SM, 6 warps:
-//   warps 0-3  epilogue: TMEM -> registers -> fused epilogue -> global (warp w owns TMEM lanes 32w..32w+31)
-//   warp  4    TMA producer: 128-byte-swizzled K-major tiles of A [128 x 128 B] and W [BN x 128 B]
-//   warp  5    UMMA issuer (one elected lane) and owner of the TMEM allocation
+// One persistent CTA per SM, 10 warps:
+//   warps 0-7  epilogue: TMEM -> registers -> fused epilogue -> global (warp w owns TMEM lanes 32 (w & 3) ..
+//              +31 and the column half w >> 2 of the tile)
+//   warp  8    TMA producer: 128-byte-swizzled K-major tiles of A [128 x 128 B] and W [BN x 128 B]
+//   warp  9    UMMA issuer (one elected lane) and owner of the TMEM allocation
 // The accumulator is double-buffered in TMEM (2 x BN columns) so the epilogue of tile t overlaps the
 // main loop of tile t+1.  Every barrier wait is bounded; on expiry the CTA records a code and unwinds.
 #include "common.cuh"
@@ -17,7 +18,8 @@ namespace hero {
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK_BYTES = 128;   // one swizzle row
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;
+constexpr int TMA_WARP = 8, MMA_WARP = 9;
 constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2;
 
 struct GemmParams {
@@ -46,7 +48,24 @@ struct GemmCfg {
   static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256 /*barriers*/;
 };
 
-__device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+constexpr float ROUND_MAGIC = 12582912.0f;   // 1.5 * 2^23
+
+// GELU(v) = v Phi(v) = max(v, 0) - 0.5 |v| E(|v| / sqrt 2) with E(z) = erfc(z) for z >= 0, evaluated with the
+// rational-exponential form erfc(z) ~ (a1 t + ... + a5 t^5) exp(-z^2), t = 1 / (1 + p z) (absolute error
+// below 1.5e-7 for every z >= 0): branch-free, two special-function ops, no cancellation for negative v.
+__device__ __forceinline__ float gelu_erf_f(float v) {
+  const float av = fabsf(v);
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(av, 0.3275911f * 0.70710678118654752440f, 1.0f)));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  poly *= t;
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(v * v * -0.72134752044448170368f));   // exp(-v^2 / 2)
+  return fmaf(-0.5f * av, poly * e, fmaxf(v, 0.0f));
+}
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   return 0.5f * x * (1.0f + tanhf(0.79788456080286535588f * (x + 0.044715f * x * x * x)));
 }
@@ -57,6 +76,12 @@ __device__ __forceinline__ uint32_t pack4_i8(float a, float b, float c, float d)
   int ic = __float2int_rn(fminf(fmaxf(c, -127.f), 127.f));
   int id = __float2int_rn(fminf(fmaxf(d, -127.f), 127.f));
   return (uint32_t)(ia & 0xff) | ((uint32_t)(ib & 0xff) << 8) | ((uint32_t)(ic & 0xff) << 16) | ((uint32_t)id << 24);
+}
+// the low bytes of four floats already rounded with ROUND_MAGIC, packed little-endian
+__device__ __forceinline__ uint32_t low_bytes4(float a, float b, float c, float d) {
+  const uint32_t ab = __byte_perm(__float_as_uint(a), __float_as_uint(b), 0x0040);
+  const uint32_t cd = __byte_perm(__float_as_uint(c), __float_as_uint(d), 0x0040);
+  return __byte_perm(ab, cd, 0x5410);
 }
 __device__ __forceinline__ uint32_t pack2_fp(float a, float b, int dt) {
   if (dt == HERO_F16) {
@@ -105,20 +130,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 8); }
     ptx::fence_mbar_init();
   }
-  if (warp == 5) {
+  if (warp == MMA_WARP) {
     ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
     ptx::tmem_relinquish();
   }
-  if (warp == 4 && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
+  if (warp == TMA_WARP && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 4) {
+  if (warp == TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const int kelems = GEMM_BK_BYTES / p.elem_bytes;
@@ -142,7 +167,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     }
     __syncwarp();
-  } else if (warp == 5) {
+  } else if (warp == MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
     if (lane == 0) {
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
@@ -174,8 +199,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 0-3)
-    const int tid_e = threadIdx.x;            // 0..127
+    // ------------------------------------------------------------------ epilogue (warps 0-7)
+    // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
+    const int quarter = warp & 3, chalf = warp >> 2;
+    constexpr int CH = BN / 2;                 // columns per thread and tile
+    const int tid_e = threadIdx.x;             // 0..255
     int it = 0; bool ok = true;
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
       int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
@@ -186,16 +214,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       float* e_bias = e_cs + BN;
       float* e_post = e_bias + BN;
       if constexpr (OUTK != OUT_I32) {
-        for (int j = tid_e; j < BN; j += 128) {
+        for (int j = tid_e; j < BN; j += 256) {
           const int n = n0 + j;
           const bool in = n < p.N;
           e_cs[j] = (in && p.cs) ? p.cs[n] : 1.0f;
           e_bias[j] = (in && p.bias) ? p.bias[n] : 0.0f;
           e_post[j] = (in && p.post) ? p.post[n] : 1.0f;
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
       }
-      const int m = mt * GEMM_BM + warp * 32 + lane;
+      const int m = mt * GEMM_BM + quarter * 32 + lane;
       const bool row_ok = m < p.M;
       float rs = 1.0f;
       if (OUTK != OUT_I32 && INT8 && p.rs && row_ok) rs = p.rs[m];
@@ -203,13 +231,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
       ptx::tc_fence_after();
       if (ok) {
-        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + as * BN;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = 0; c < CH / 32; ++c) {
           uint32_t r[32];
           ptx::tmem_ld32(taddr + c * 32, r);
           ptx::tmem_ld_wait();
-          const int col0 = n0 + c * 32;
+          const int jc = chalf * CH + c * 32;   // column of r[0] inside the tile
+          const int col0 = n0 + jc;
           if constexpr (OUTK == OUT_I32) {
             if (row_ok) {
               int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
@@ -222,10 +251,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const float acc = INT8 ? (float)(int)r[j] : __uint_as_float(r[j]);
-              float x = fmaf(acc * rs, e_cs[c * 32 + j], e_bias[c * 32 + j]);
+              float x = fmaf(acc * rs, e_cs[jc + j], e_bias[jc + j]);
               if constexpr (ACT == HERO_ACT_GELU_ERF) x = gelu_erf_f(x);
               if constexpr (ACT == HERO_ACT_GELU_TANH) x = gelu_tanh_f(x);
-              v[j] = x * e_post[c * 32 + j];
+              if constexpr (OUTK == OUT_I8) {
+                // Round (half to even) and clip in the float adder: 1.5 * 2^23 + k keeps k in its low byte
+                const float y = fmaf(x, e_post[jc + j], ROUND_MAGIC);
+                v[j] = fminf(fmaxf(y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+              } else {
+                v[j] = x * e_post[jc + j];
+              }
             }
             if (row_ok) {
               if constexpr (OUTK == OUT_I8) {
@@ -233,10 +268,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int g = 0; g < 2; ++g)
                   if (col0 + 16 * g + 16 <= p.N)
-                    st16(dst + 16 * g, pack4_i8(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
-                         pack4_i8(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
-                         pack4_i8(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
-                         pack4_i8(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
+                    st16(dst + 16 * g, low_bytes4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
+                         low_bytes4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
+                         low_bytes4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
+                         low_bytes4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
               } else {
                 uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
 #pragma unroll
@@ -258,7 +293,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 5) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  if (warp == MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
 template <int BN, bool INT8, int ACT, int OUTK>

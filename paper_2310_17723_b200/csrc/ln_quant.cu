@@ -144,7 +144,7 @@ __device__ __forceinline__ void row_reduce(float (&v)[R], float* red, int G, int
 }
 
 template <int VEC, int R, bool HAS_BR, bool HAS_EX>
-__global__ void __launch_bounds__(512) ln_quant_kernel(const LnParams p) {
+__global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
   extern __shared__ float red_smem[];
   const int G = p.G, RPC = p.RPC, H = p.H;
   const int nw = G >> 5;
@@ -157,7 +157,6 @@ __global__ void __launch_bounds__(512) ln_quant_kernel(const LnParams p) {
   const int t = tid - row_in_cta * G;
   const int c0 = t * VEC;
   const bool active = c0 < H;
-  const float inv_H = 1.0f / (float)H;
 
   float gam[VEC], bet[VEC];
   const bool normalize = p.out != nullptr;
@@ -274,7 +273,7 @@ __global__ void __launch_bounds__(512) ln_quant_kernel(const LnParams p) {
     float mean[R], rstd[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      mean[r] = s[r] * inv_H;
+      mean[r] = s[r] / (float)H;
       float a = 0.f;
       if (active) {
 #pragma unroll
@@ -284,7 +283,7 @@ __global__ void __launch_bounds__(512) ln_quant_kernel(const LnParams p) {
     }
     row_reduce<R, false>(s, red1, G, row_in_cta, t);
 #pragma unroll
-    for (int r = 0; r < R; ++r) rstd[r] = 1.0f / sqrtf(s[r] * inv_H + p.eps);
+    for (int r = 0; r < R; ++r) rstd[r] = 1.0f / sqrtf(s[r] / (float)H + p.eps);
 
     // ---- y = (x - mean) * rstd * gamma + beta
     float amax[R];
@@ -463,20 +462,53 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-constexpr int LNF_STAGES = 3;   // rows in flight per row slot (each lane prefetches its own chunks)
+constexpr int LNF_MAX_STAGES = 8; // ring depth is chosen at launch so that ~128 KB per SM are in flight
 
-template <int RES, int BR, bool EX, int OUT, bool FPOUT>
-__global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams p) {
+// Packed FP32 pairs: sm_100 issues add / mul / fma on two floats per instruction, which halves the issue
+// slots of the arithmetic below (the kernel is bound by instruction issue, not by any one pipe).
+__device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ void load_vec8(const float* p, float2 (&v)[4]) {
+  const float4 a = ldg_f4(p), b = ldg_f4(p + 4);
+  v[0] = make_float2(a.x, a.y); v[1] = make_float2(a.z, a.w); v[2] = make_float2(b.x, b.y); v[3] = make_float2(b.z, b.w);
+}
+// 8 INT8 codes -> 4 float pairs (exact): byte + 128 into the mantissa of 2^23, then one packed subtraction
+__device__ __forceinline__ void i8x8_to_f2(uint32_t w0, uint32_t w1, float2 (&v)[4]) {
+  w0 ^= 0x80808080u; w1 ^= 0x80808080u;
+  const float2 off = f2(-8388736.0f);             // -(2^23 + 128)
+  v[0] = __fadd2_rn(make_float2(__uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7440)), __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7441))), off);
+  v[1] = __fadd2_rn(make_float2(__uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7442)), __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7443))), off);
+  v[2] = __fadd2_rn(make_float2(__uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7440)), __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7441))), off);
+  v[3] = __fadd2_rn(make_float2(__uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7442)), __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7443))), off);
+}
+__device__ __forceinline__ void fp16x8_to_f2(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, int dt, float2 (&v)[4]) {
+  const uint32_t w[4] = {w0, w1, w2, w3};
+  if (dt == HERO_F16) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
+  }
+}
+
+// NCHX = exact number of 8-element chunks per lane (H = 256 * WPR * NCHX, no tail predicates), or 0 for any H.
+template <int RES, int BR, bool EX, int OUT, bool FPOUT, int NCHX>
+__global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams p) {
+  constexpr int KMAX = NCHX ? NCHX : LNF_MAXCH;
+  // gamma / beta (and, with at most 3 chunks per lane, the branch's per-feature scale) stay in registers for
+  // the whole persistent row loop of the exact-size variants; otherwise they are re-read through L1 per row
+  constexpr bool GB_REG = NCHX != 0;
+  constexpr bool CS_REG = (NCHX == 2 || NCHX == 3) && BR == SRC_I8;
+  auto chunk_ok = [&](int c) -> bool { if constexpr (NCHX != 0) return true; else return c < (p.H >> 3); };
   __shared__ float red[3][8][8];                  // [statistic][row slot][warp in row]
   extern __shared__ __align__(16) uint8_t ring[]; // [stage][row slot][res row | branch row | extra row]
   const int WPR = p.G;                            // warps per row: 1, 2, 4 or 8
   const int slots = 8 / WPR;                      // rows per CTA pass
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int slot = warp / WPR, wr = warp - slot * WPR;
-  const int nchunks = p.H >> 3;
   const int stride = WPR * 32;                    // chunk stride between a lane's chunks
   const int c_first = wr * 32 + lane;
-  const float inv_H = 1.0f / (float)p.H;
+  const float fH = (float)p.H;
   const float MAGIC = 12582912.0f;                // 1.5 * 2^23
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2;
   constexpr int ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
@@ -484,27 +516,33 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
   const int off_ex = off_br + p.H * ES_BR;
   const int slot_bytes = off_ex + (EX ? p.H * 2 : 0);
   const int stage_bytes = slot_bytes * slots;
+  const int STAGES = p.RPC;                       // ring depth (3..8), chosen by the host
 
   // A lane copies exactly the chunks it will later read, so waiting on its own copy groups is all
   // the synchronisation the ring needs.
   auto prefetch = [&](long long row, int st) {
     if (row < p.M) {
       long long r_res = row, r_br = row, r_ex = row;
-      if (p.token_ids) {
-        r_res = p.token_ids[row];
-        r_br = row % p.seq_len;
-        r_ex = p.type_ids ? p.type_ids[row] : 0;
+      if constexpr (EX) {
+        if (p.token_ids) {
+          r_res = p.token_ids[row];
+          r_br = row % p.seq_len;
+          r_ex = p.type_ids ? p.type_ids[row] : 0;
+        }
       }
       uint8_t* dst = ring + st * stage_bytes + slot * slot_bytes;
+      const char* g_res = reinterpret_cast<const char*>(p.res.data) + r_res * p.res.ld * ES_RES;
+      const char* g_br = (BR != SRC_NONE) ? reinterpret_cast<const char*>(p.br.data) + r_br * p.br.ld * ES_BR : nullptr;
+      const char* g_ex = EX ? reinterpret_cast<const char*>(p.ex.data) + r_ex * p.ex.ld * 2 : nullptr;
 #pragma unroll
-      for (int k = 0; k < LNF_MAXCH; ++k) {
+      for (int k = 0; k < KMAX; ++k) {
         const int c = c_first + k * stride;
-        if (c < nchunks) {
-          if constexpr (RES == SRC_I8) cp_async8(dst + c * 8, reinterpret_cast<const char*>(p.res.data) + r_res * p.res.ld + c * 8);
-          else cp_async16(dst + c * 16, reinterpret_cast<const char*>(p.res.data) + (r_res * p.res.ld + c * 8) * 2);
-          if constexpr (BR == SRC_I8) cp_async8(dst + off_br + c * 8, reinterpret_cast<const char*>(p.br.data) + r_br * p.br.ld + c * 8);
-          if constexpr (BR == SRC_FP) cp_async16(dst + off_br + c * 16, reinterpret_cast<const char*>(p.br.data) + (r_br * p.br.ld + c * 8) * 2);
-          if constexpr (EX) cp_async16(dst + off_ex + c * 16, reinterpret_cast<const char*>(p.ex.data) + (r_ex * p.ex.ld + c * 8) * 2);
+        if (chunk_ok(c)) {
+          if constexpr (RES == SRC_I8) cp_async8(dst + c * 8, g_res + c * 8);
+          else cp_async16(dst + c * 16, g_res + c * 16);
+          if constexpr (BR == SRC_I8) cp_async8(dst + off_br + c * 8, g_br + c * 8);
+          if constexpr (BR == SRC_FP) cp_async16(dst + off_br + c * 16, g_br + c * 16);
+          if constexpr (EX) cp_async16(dst + off_ex + c * 16, g_ex + c * 16);
         }
       }
     }
@@ -513,156 +551,182 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
 
   const long long row_step = (long long)gridDim.x * slots;
   const long long first = (long long)blockIdx.x * slots;
+  for (int s0 = 0; s0 < STAGES - 1; ++s0) prefetch(first + s0 * row_step + slot, s0);
+
+  float2 gam[GB_REG ? KMAX : 1][4], bet[GB_REG ? KMAX : 1][4], bcs[CS_REG ? KMAX : 1][4];
+  if constexpr (GB_REG && OUT != O_NONE) {
 #pragma unroll
-  for (int s0 = 0; s0 < LNF_STAGES - 1; ++s0) prefetch(first + s0 * row_step + slot, s0);
+    for (int k = 0; k < KMAX; ++k) {
+      load_vec8(p.gamma + (c_first + k * stride) * 8, gam[k]);
+      load_vec8(p.beta + (c_first + k * stride) * 8, bet[k]);
+    }
+  }
+  if constexpr (CS_REG) {
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+      const int c8 = (c_first + k * stride) * 8;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        bcs[k][i].x = p.br.col_scale ? __ldg(p.br.col_scale + (c8 + 2 * i) * p.br.col_stride) : 1.0f;
+        bcs[k][i].y = p.br.col_scale ? __ldg(p.br.col_scale + (c8 + 2 * i + 1) * p.br.col_stride) : 1.0f;
+      }
+    }
+  }
 
   int st = 0;
   for (long long base = first; base < p.M; base += row_step) {
     const long long row = base + slot;
     const bool row_ok = row < p.M;
     {
-      int pst = st + LNF_STAGES - 1;
-      if (pst >= LNF_STAGES) pst -= LNF_STAGES;
-      prefetch(row + (LNF_STAGES - 1) * row_step, pst);
+      int pst = st + STAGES - 1;
+      if (pst >= STAGES) pst -= STAGES;
+      prefetch(row + (long long)(STAGES - 1) * row_step, pst);
     }
-    cp_async_wait<LNF_STAGES - 1>();
+    switch (STAGES) {                             // this row's copies are the oldest group still pending
+      case 3: cp_async_wait<2>(); break;
+      case 4: cp_async_wait<3>(); break;
+      case 5: cp_async_wait<4>(); break;
+      case 6: cp_async_wait<5>(); break;
+      case 7: cp_async_wait<6>(); break;
+      default: cp_async_wait<7>(); break;
+    }
     const uint8_t* src = ring + st * stage_bytes + slot * slot_bytes;
-    if (++st == LNF_STAGES) st = 0;
+    if (++st == STAGES) st = 0;
 
-    float x[LNF_MAXCH][8];
+    float2 x[KMAX][4];
     float rs_res = 1.f, rs_br = 1.f;
     if (row_ok) {
       long long r_res = row, r_br = row;
-      if (p.token_ids) { r_res = p.token_ids[row]; r_br = row % p.seq_len; }
+      if constexpr (EX) { if (p.token_ids) { r_res = p.token_ids[row]; r_br = row % p.seq_len; } }
       if (RES == SRC_I8 && p.res.row_scale) rs_res = __ldg(p.res.row_scale + r_res);
       if (BR == SRC_I8 && p.br.row_scale) rs_br = __ldg(p.br.row_scale + r_br);
     }
 
     // ---- r = sum of the dequantized addends; running row sum
-    float s = 0.f;
+    float2 s2 = f2(0.f);
 #pragma unroll
-    for (int k = 0; k < LNF_MAXCH; ++k) {
+    for (int k = 0; k < KMAX; ++k) {
       const int c = c_first + k * stride;
-      if (row_ok && c < nchunks) {
+      if (row_ok && chunk_ok(c)) {
         if constexpr (RES == SRC_I8) {
           const uint2 w = *reinterpret_cast<const uint2*>(src + c * 8);
-          i8x8_to_float(w.x, w.y, x[k]);
-          if (p.res.col_scale) {
-            float sc[8];
-            if (p.res.col_stride) {
-              float4 a = ldg_f4(p.res.col_scale + c * 8), b = ldg_f4(p.res.col_scale + c * 8 + 4);
-              sc[0] = a.x; sc[1] = a.y; sc[2] = a.z; sc[3] = a.w; sc[4] = b.x; sc[5] = b.y; sc[6] = b.z; sc[7] = b.w;
-            } else {
-              const float v = __ldg(p.res.col_scale);
+          i8x8_to_f2(w.x, w.y, x[k]);
+          if (p.res.col_scale) {                 // FWQ / SQ residual (the scale is per feature, not per row)
+            float2 sc[4];
+            if (p.res.col_stride) load_vec8(p.res.col_scale + c * 8, sc);
+            else { const float v = __ldg(p.res.col_scale); sc[0] = sc[1] = sc[2] = sc[3] = f2(v); }
 #pragma unroll
-              for (int i = 0; i < 8; ++i) sc[i] = v;
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[k][i] *= rs_res * sc[i];
+            for (int i = 0; i < 4; ++i) x[k][i] = __fmul2_rn(x[k][i], sc[i]);
           } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[k][i] *= rs_res;
+            for (int i = 0; i < 4; ++i) x[k][i] = __fmul2_rn(x[k][i], f2(rs_res));
           }
         } else {
           const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
-          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-          fp16x8_to_float(ww, p.res.dt, x[k]);
+          fp16x8_to_f2(w.x, w.y, w.z, w.w, p.res.dt, x[k]);
         }
         if constexpr (BR == SRC_I8) {
-          float b[8];
+          float2 b[4];
           const uint2 wb = *reinterpret_cast<const uint2*>(src + off_br + c * 8);
-          i8x8_to_float(wb.x, wb.y, b);
-          if (p.br.col_scale) {
-            float sc[8];
-            if (p.br.col_stride) {
-              float4 a = ldg_f4(p.br.col_scale + c * 8), bb = ldg_f4(p.br.col_scale + c * 8 + 4);
-              sc[0] = a.x; sc[1] = a.y; sc[2] = a.z; sc[3] = a.w; sc[4] = bb.x; sc[5] = bb.y; sc[6] = bb.z; sc[7] = bb.w;
+          i8x8_to_f2(wb.x, wb.y, b);
+          if constexpr (CS_REG) {
+            if (p.br.row_scale) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) x[k][i] = __ffma2_rn(b[i], __fmul2_rn(bcs[k][i], f2(rs_br)), x[k][i]);
             } else {
-              const float v = __ldg(p.br.col_scale);
 #pragma unroll
-              for (int i = 0; i < 8; ++i) sc[i] = v;
+              for (int i = 0; i < 4; ++i) x[k][i] = __ffma2_rn(b[i], bcs[k][i], x[k][i]);
             }
+          } else if (p.br.col_scale) {
+            float2 sc[4];
+            if (p.br.col_stride) load_vec8(p.br.col_scale + c * 8, sc);
+            else { const float v = __ldg(p.br.col_scale); sc[0] = sc[1] = sc[2] = sc[3] = f2(v); }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[k][i] = fmaf(b[i], rs_br * sc[i], x[k][i]);
+            for (int i = 0; i < 4; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
           } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[k][i] = fmaf(b[i], rs_br, x[k][i]);
+            for (int i = 0; i < 4; ++i) x[k][i] = __ffma2_rn(b[i], f2(rs_br), x[k][i]);
           }
         }
         if constexpr (BR == SRC_FP) {
-          float b[8];
+          float2 b[4];
           const uint4 wb = *reinterpret_cast<const uint4*>(src + off_br + c * 16);
-          const uint32_t wwb[4] = {wb.x, wb.y, wb.z, wb.w};
-          fp16x8_to_float(wwb, p.br.dt, b);
+          fp16x8_to_f2(wb.x, wb.y, wb.z, wb.w, p.br.dt, b);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[k][i] += b[i];
+          for (int i = 0; i < 4; ++i) x[k][i] = __fadd2_rn(x[k][i], b[i]);
         }
         if constexpr (EX) {
-          float e[8];
+          float2 e[4];
           const uint4 we = *reinterpret_cast<const uint4*>(src + off_ex + c * 16);
-          const uint32_t wwe[4] = {we.x, we.y, we.z, we.w};
-          fp16x8_to_float(wwe, p.ex.dt, e);
+          fp16x8_to_f2(we.x, we.y, we.z, we.w, p.ex.dt, e);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[k][i] += e[i];
+          for (int i = 0; i < 4; ++i) x[k][i] = __fadd2_rn(x[k][i], e[i]);
         }
         if constexpr (FPOUT) {
           // the FP residual stream carries the ROUNDED sum; normalise what is stored
           uint32_t w[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) w[i] = pack_fp2(x[k][2 * i], x[k][2 * i + 1], p.fp_dt);
+          for (int i = 0; i < 4; ++i) w[i] = pack_fp2(x[k][i].x, x[k][i].y, p.fp_dt);
           st_global16(reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + c * 8) * 2, w[0], w[1], w[2], w[3]);
-          fp16x8_to_float(w, p.fp_dt, x[k]);
+          fp16x8_to_f2(w[0], w[1], w[2], w[3], p.fp_dt, x[k]);
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) s += x[k][i];
+        for (int i = 0; i < 4; ++i) s2 = __fadd2_rn(s2, x[k][i]);
       } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[k][i] = 0.f;
+        for (int i = 0; i < 4; ++i) x[k][i] = f2(0.f);
       }
     }
     if constexpr (OUT == O_NONE) continue;
 
-    // ---- mean
-    s = warp_sum(s);
+    // ---- mean (true division: a constant row must give exactly zero deviations)
+    float s = warp_sum(s2.x + s2.y);
     if (WPR > 1) {
       if (lane == 0) red[0][slot][wr] = s;
       asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(stride) : "memory");
       s = 0.f;
       for (int w = 0; w < WPR; ++w) s += red[0][slot][w];
     }
-    const float mean = s * inv_H;
+    const float mean = s / fH;
     // ---- centred (biased) variance over the registers
-    float q = 0.f;
+    float2 q2 = f2(0.f);
+    const float2 nm = f2(-mean);
 #pragma unroll
-    for (int k = 0; k < LNF_MAXCH; ++k) {
-      if (c_first + k * stride < nchunks) {
+    for (int k = 0; k < KMAX; ++k) {
+      if (chunk_ok(c_first + k * stride)) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { x[k][i] -= mean; q = fmaf(x[k][i], x[k][i], q); }
+        for (int i = 0; i < 4; ++i) { x[k][i] = __fadd2_rn(x[k][i], nm); q2 = __ffma2_rn(x[k][i], x[k][i], q2); }
       }
     }
-    q = warp_sum(q);
+    float q = warp_sum(q2.x + q2.y);
     if (WPR > 1) {
       if (lane == 0) red[1][slot][wr] = q;
       asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "r"(stride) : "memory");
       q = 0.f;
       for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
     }
-    const float rstd = 1.0f / sqrtf(q * inv_H + p.eps);
+    const float rstd = 1.0f / sqrtf(q / fH + p.eps);
 
     // ---- y = d * (rstd * gamma) + beta ; TWQ: row absmax in the same sweep
     float amax = 0.f;
+    const float2 r2 = f2(rstd);
 #pragma unroll
-    for (int k = 0; k < LNF_MAXCH; ++k) {
+    for (int k = 0; k < KMAX; ++k) {
       const int c = c_first + k * stride;
-      if (c < nchunks) {
-        float4 g0 = ldg_f4(p.gamma + c * 8), g1 = ldg_f4(p.gamma + c * 8 + 4);
-        float4 b0 = ldg_f4(p.beta + c * 8), b1 = ldg_f4(p.beta + c * 8 + 4);
-        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-        const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      if constexpr (GB_REG) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          x[k][i] = fmaf(x[k][i], rstd * g[i], b[i]);
-          if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fabsf(x[k][i]));
+        for (int i = 0; i < 4; ++i) {
+          x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(gam[k][i], r2), bet[k][i]);
+          if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fmaxf(fabsf(x[k][i].x), fabsf(x[k][i].y)));
+        }
+      } else if (chunk_ok(c)) {
+        float2 g[4], b[4];
+        load_vec8(p.gamma + c * 8, g);
+        load_vec8(p.beta + c * 8, b);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(g[i], r2), b[i]);
+          if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fmaxf(fabsf(x[k][i].x), fabsf(x[k][i].y)));
         }
       }
     }
@@ -678,15 +742,18 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
         for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
       }
       const float sc = amax > 0.f ? amax / 127.0f : 1.0f;
-      const float inv = 1.0f / sc;
+      const float2 inv2 = f2(1.0f / sc), mg2 = f2(MAGIC);
       if (row_ok && wr == 0 && lane == 0) p.out_scale[row] = sc;
 #pragma unroll
-      for (int k = 0; k < LNF_MAXCH; ++k) {
+      for (int k = 0; k < KMAX; ++k) {
         const int c = c_first + k * stride;
-        if (row_ok && c < nchunks) {
+        if (row_ok && chunk_ok(c)) {
           uint32_t u[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) u[i] = magic_bits(fmaf(x[k][i], inv, MAGIC));
+          for (int i = 0; i < 4; ++i) {
+            const float2 v = __ffma2_rn(x[k][i], inv2, mg2);
+            u[2 * i] = __float_as_uint(v.x); u[2 * i + 1] = __float_as_uint(v.y);
+          }
           st_global8(reinterpret_cast<char*>(p.out) + row * p.out_ld + c * 8, pack_low_bytes(u[0], u[1], u[2], u[3]),
                      pack_low_bytes(u[4], u[5], u[6], u[7]));
         }
@@ -694,9 +761,9 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
     } else if constexpr (OUT == O_STATIC) {
       // Eq. 4 / 5: calibrated per-feature (stride 1) or static (stride 0) scale; saturating
 #pragma unroll
-      for (int k = 0; k < LNF_MAXCH; ++k) {
+      for (int k = 0; k < KMAX; ++k) {
         const int c = c_first + k * stride;
-        if (row_ok && c < nchunks) {
+        if (row_ok && chunk_ok(c)) {
           float sc[8];
           if (p.out_gran == HERO_GRAN_FWQ) {
             float4 a = ldg_f4(p.out_scale + c * 8), b = ldg_f4(p.out_scale + c * 8 + 4);
@@ -709,7 +776,8 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
           uint32_t u[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float v = fminf(fmaxf(x[k][i] / sc[i], -127.f), 127.f);
+            const float xv = (i & 1) ? x[k][i >> 1].y : x[k][i >> 1].x;
+            const float v = fminf(fmaxf(xv / sc[i], -127.f), 127.f);
             u[i] = magic_bits(v + MAGIC);
           }
           st_global8(reinterpret_cast<char*>(p.out) + row * p.out_ld + c * 8, pack_low_bytes(u[0], u[1], u[2], u[3]),
@@ -718,12 +786,12 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
       }
     } else {
 #pragma unroll
-      for (int k = 0; k < LNF_MAXCH; ++k) {
+      for (int k = 0; k < KMAX; ++k) {
         const int c = c_first + k * stride;
-        if (row_ok && c < nchunks) {
+        if (row_ok && chunk_ok(c)) {
           uint32_t w[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) w[i] = pack_fp2(x[k][2 * i], x[k][2 * i + 1], p.out_dt);
+          for (int i = 0; i < 4; ++i) w[i] = pack_fp2(x[k][i].x, x[k][i].y, p.out_dt);
           st_global16(reinterpret_cast<char*>(p.out) + (row * p.out_ld + c * 8) * 2, w[0], w[1], w[2], w[3]);
         }
       }
@@ -731,16 +799,21 @@ __global__ void __launch_bounds__(LNF_THREADS, 3) ln_fast_kernel(const LnParams 
   }
 }
 
-template <int RES, int BR, bool EX, int OUT, bool FPOUT>
+template <int RES, int BR, bool EX, int OUT, bool FPOUT, int NCHX>
 static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream) {
-  int wpr = 1;
-  while (wpr * 1024 < p.H) wpr *= 2;
-  p.G = wpr;
+  const int wpr = p.G;
   const int slots = 8 / wpr;
   const long long want = (p.M + slots - 1) / slots;
   const int es_res = (RES == SRC_I8) ? 1 : 2, es_br = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
-  const size_t smem = (size_t)LNF_STAGES * slots * p.H * (es_res + es_br + (EX ? 2 : 0));
-  auto kern = ln_fast_kernel<RES, BR, EX, OUT, FPOUT>;
+  const size_t stage = (size_t)slots * p.H * (es_res + es_br + (EX ? 2 : 0));
+  // two CTAs per SM; deep enough that about 128 KB per SM are always on their way, within 100 KB per CTA
+  int stages = 1 + (int)((64 * 1024 + stage - 1) / stage);
+  if (stages < 3) stages = 3;
+  if (stages > LNF_MAX_STAGES) stages = LNF_MAX_STAGES;
+  while (stages > 3 && stages * stage > 100 * 1024) --stages;
+  p.RPC = stages;
+  const size_t smem = (size_t)stages * stage;
+  auto kern = ln_fast_kernel<RES, BR, EX, OUT, FPOUT, NCHX>;
   static bool configured = false;   // per instantiation
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
@@ -759,6 +832,7 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
   return HERO_OK;
 }
 
+int g_ln_first_n = 2;
 // Returns HERO_ERR_UNSUPPORTED (without setting an error) when the combination has no fast instantiation.
 static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
@@ -769,12 +843,27 @@ static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* t
   const int out = !p.out ? O_NONE : (p.out_dt != HERO_I8 ? O_FP : (p.out_gran == HERO_GRAN_TWQ ? O_TWQ : O_STATIC));
   const bool fpo = p.fp_out != nullptr;
   if (res == SRC_I8 && p.res.row_scale && p.res.col_scale) return HERO_OK;
+  // rows of exactly 3 or 4 chunks per lane (H = 768, 1024, 4096, 8192, ...) take the tail-free instantiation
+  int wpr = 1, exact = 0;
+  for (int n = 4; n >= g_ln_first_n && !exact; --n)              // H = 256 * n * wpr with wpr in {1, 2, 4, 8}
+    for (int w = 1; w <= 8 && !exact; w *= 2)
+      if (p.H == 256 * n * w) { wpr = w; exact = n; }
+  if (!exact) while (wpr * 1024 < p.H) wpr *= 2;
+  p.G = wpr;
 #define LNF_CASE(R_, B_, E_, O_, F_)                                                   \
   if (res == R_ && br == B_ && ex == E_ && out == O_ && fpo == F_) {                   \
     *taken = true;                                                                     \
-    return launch_fast<R_, B_, E_, O_, F_>(h, p, s);                                   \
+    return launch_fast<R_, B_, E_, O_, F_, 0>(h, p, s);                                \
   }
-#define LNF_OUTS(R_, B_, E_, F_) LNF_CASE(R_, B_, E_, O_TWQ, F_) LNF_CASE(R_, B_, E_, O_STATIC, F_) LNF_CASE(R_, B_, E_, O_FP, F_)
+#define LNF_CASE_X(R_, B_, E_, O_, F_)                                                 \
+  if (res == R_ && br == B_ && ex == E_ && out == O_ && fpo == F_) {                   \
+    *taken = true;                                                                     \
+    if (exact == 2) return launch_fast<R_, B_, E_, O_, F_, 2>(h, p, s);                \
+    if (exact == 3) return launch_fast<R_, B_, E_, O_, F_, 3>(h, p, s);                \
+    if (exact == 4) return launch_fast<R_, B_, E_, O_, F_, 4>(h, p, s);                \
+    return launch_fast<R_, B_, E_, O_, F_, 0>(h, p, s);                                \
+  }
+#define LNF_OUTS(R_, B_, E_, F_) LNF_CASE_X(R_, B_, E_, O_TWQ, F_) LNF_CASE(R_, B_, E_, O_STATIC, F_) LNF_CASE(R_, B_, E_, O_FP, F_)
   LNF_OUTS(SRC_FP, SRC_NONE, false, false)   // entry LN^quant on FP activations; pre-LN LN1
   LNF_OUTS(SRC_I8, SRC_I8, false, false)     // Eq. 19 / 31: two INT8 addends
   LNF_OUTS(SRC_I8, SRC_FP, false, false)     // INT8 residual + FP branch (modes M1 / M2)
@@ -782,10 +871,11 @@ static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* t
   LNF_OUTS(SRC_FP, SRC_I8, false, false)     // FP residual + INT8 branch
   LNF_OUTS(SRC_FP, SRC_I8, false, true)      // pre-LN: add + LN + quant, new residual stream stored
   LNF_OUTS(SRC_FP, SRC_FP, false, true)
-  LNF_CASE(SRC_FP, SRC_I8, false, O_NONE, true)   // closing residual add of a lone pre-LN layer
+  LNF_CASE_X(SRC_FP, SRC_I8, false, O_NONE, true)   // closing residual add of a lone pre-LN layer
   LNF_CASE(SRC_FP, SRC_FP, false, O_NONE, true)
   LNF_OUTS(SRC_I8, SRC_FP, true, false)      // Eq. 7: embedding gather, three addends
 #undef LNF_OUTS
+#undef LNF_CASE_X
 #undef LNF_CASE
   return HERO_OK;
 }
@@ -852,3 +942,5 @@ extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* 
   if (H % 16 == 0 && H >= 2048) return launch_ln<16, 1>(h, p, s);
   return launch_ln<8, 2>(h, p, s);
 }
+
+extern "C" void hero_debug_ln_first_n(int n) { hero::g_ln_first_n = n; }

@@ -53,8 +53,8 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;  // polls; each try_wait itself blocks
 // Bounded wait.  Returns false (after recording `code`) when the barrier never flipped.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err_word, int code) {
   for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (i > 64) __nanosleep(64);
+    if (mbar_try_wait(bar, parity)) return true;   // try_wait itself suspends the thread for a hardware time slice
+    if (i > (1u << 16)) __nanosleep(256);           // only a wait that is already hopelessly long backs off
   }
   if (err_word) atomicExch(err_word, code);
   return false;

@@ -151,3 +151,32 @@ def test_refusals(h):
     with pytest.raises(hero.HeroError) as e:           # token-wise X_attn refused
         h.hero_int8_attention(x[:, :128], x[:, 128:256], x[:, 256:], 1, 128, 2, 64, hero.tensor(out, "twq", rs))
     assert e.value.status == hero.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ FP16 / BF16 attention (module left in FP mode, Table 1)
+@pytest.mark.parametrize("fp", ["f16", "bf16"])
+@pytest.mark.parametrize("B,S,nh,dh,mask", [(2, 128, 2, 64, "none"), (1, 384, 3, 64, "causal"), (2, 200, 2, 128, "none"),
+                                            (1, 512, 2, 128, "causal")])
+def test_fp_attention(h, fp, B, S, nh, dh, mask):
+    from gpu_util import TORCH_FP
+    g = W.rng(3, 500 + S + dh)
+    H = nh * dh
+    qkv = Q.round_to_storage(g.standard_normal((B * S, 3 * H)), fp)
+    want = O.attention_fp(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh, O.OutSpec("fp", dtype=fp), mask=mask)
+    t = dev(qkv, TORCH_FP[fp])
+    out = torch.full((B * S, H), float("nan"), dtype=TORCH_FP[fp], device="cuda")
+    h.hero_int8_attention(t[:, :H], t[:, H:2 * H], t[:, 2 * H:], B, S, nh, dh, hero.tensor(out), mask=mask)
+    h.check()
+    # P is stored in FP16 / BF16 before the second GEMM (as any fused FP attention does): that rounding, not the
+    # accumulation, sets the error
+    assert rel_err(out.float().cpu().numpy(), want.data) < (2e-3 if fp == "f16" else 1e-2)
+    # FP attention feeding an INT8 attention-output linear: quantized by S_attn in the epilogue
+    raw = O.attention_fp(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh, O.OutSpec("fp", dtype="f64"), mask=mask).data
+    S_attn = Q.calib_scale(np.abs(raw).max(0))
+    want_q = O.attention_fp(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh, O.OutSpec("fwq", scale=S_attn), mask=mask)
+    out_q = torch.full((B * S, H), -99, dtype=torch.int8, device="cuda")
+    h.hero_int8_attention(t[:, :H], t[:, H:2 * H], t[:, 2 * H:], B, S, nh, dh, hero.tensor(out_q, "fwq", f32(S_attn)), mask=mask)
+    h.check()
+    frac, mx = int8_mismatch(out_q.cpu().numpy(), want_q.data)
+    # P rounded to FP16 / BF16 perturbs X_attn by up to ~2^-11 / 2^-8 relative, i.e. a visible fraction of an INT8 step
+    assert mx <= 1 and frac < (0.02 if fp == "f16" else 0.12), (frac, mx)

@@ -36,7 +36,7 @@ def _build(shape, seed, **kw):
     C = OL.calibrate(spec, p, cal_in, shape.B)
     Lp = OL.prepare_layer(spec, p, C)
     if spec.arch == "post_ln":
-        x_in = OL.entry_ln(O.fp_tensor(x, "f16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+        x_in = OL.entry_ln(O.fp_tensor(x, spec.fp_dtype), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
     else:
         x_in = O.fp_tensor(x, spec.fp_dtype)
     return spec, Lp, x_in
@@ -118,6 +118,22 @@ def test_pre_ln_causal_m3_layer(h, fp, dh):
     T2 = OL.layer_forward(Lp, x_in, pending=pend)
     out2, _, _ = _run_layer(h, spec, Lp, x_in, pending=pend)
     assert rel_err(out2.float().cpu().numpy(), T2["h_out"].real()) < 1e-2
+
+
+@pytest.mark.parametrize("preset", ["M1", "M2", "FP"])
+@pytest.mark.parametrize("arch", ["post_ln", "pre_ln"])
+def test_mixed_precision_presets(h, preset, arch):
+    # Table 1: modules switched to FP16 keep FP operands; every INT8 <-> FP hand-off happens in a producer's epilogue
+    shape = W.tiny_shape(**SMALL, arch=arch, mask="causal" if arch == "pre_ln" else "none", eps=1e-5, n_outlier=2)
+    spec, Lp, x_in = _build(shape, 25, mode=dict(OL.MODE_PRESETS[preset]), gran_out="fp" if preset == "FP" else "twq")
+    T = OL.layer_forward(Lp, x_in)
+    out, sc, launches = _run_layer(h, spec, Lp, x_in)
+    assert launches == (8 if arch == "pre_ln" else 7)
+    if arch == "pre_ln" or preset == "FP":
+        got = out.float().cpu().numpy()
+    else:
+        got = out.cpu().numpy().astype(np.float64) * sc.cpu().numpy().astype(np.float64)[:, None]
+    assert rel_err(got, T["x_out"].real()) < 1e-2
 
 
 def test_workspace_too_small_and_bad_args(h):

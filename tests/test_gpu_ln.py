@@ -129,11 +129,14 @@ def test_pre_ln_dual_output_and_bare_add(h, fp):
               col_scale=(np.abs(g.standard_normal(H)) * 0.01 + 0.002).astype(np.float32).astype(np.float64))
     gamma, beta = np.ones(H, np.float32), np.zeros(H, np.float32)
     spec = O.OutSpec("twq")
-    want, want_r = O.ln_quant([hres, br], gamma, beta, 1e-5, spec, fp_out_dtype=fp)
+    _, want_r = O.ln_quant([hres, br], gamma, beta, 1e-5, spec, fp_out_dtype=fp)
     res = _run(h, [hres, br], gamma, beta, 1e-5, spec, M, H, fp_out=fp)
-    # the device normalises ITS stored sum; where that differs by one ulp from the oracle's the row statistics
-    # move by ~1e-7 relative, far inside the INT8 bar
-    _compare(res, want, want_r, spec)
+    # (1) the stored residual stream equals the oracle's up to rare 1-ulp ties of the fp32 sum;
+    _compare(res, None, want_r, spec)
+    # (2) the device normalises ITS stored sum (one bf16 ulp on the row's largest element would move the whole
+    # row's scale), so the quantized output is checked against the oracle applied to that same stored tensor
+    want, _ = O.ln_quant([O.fp_tensor(res["fp_out"], fp)], gamma, beta, 1e-5, spec)
+    _compare(res, want, None, spec)
     _, want_r2 = O.ln_quant([hres, br], None, None, 0.0, None, fp_out_dtype=fp, normalize=False)
     res2 = _run(h, [hres, br], gamma, beta, 0.0, spec, M, H, fp_out=fp, normalize=False)
     _compare(res2, None, want_r2, spec)
