@@ -21,6 +21,7 @@ constexpr int GEMM_BK_BYTES = 128;   // one swizzle row
 constexpr int GEMM_THREADS = 320;
 constexpr int TMA_WARP = 8, MMA_WARP = 9;
 constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2;
+extern int g_gemm_pair;   // experiment switch: CTA-pair (cta_group::2) kernel on / off
 
 struct GemmParams {
   int M, N, K;              // K in elements
@@ -106,6 +107,67 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mt
   const int r = t - group * width;
   mt = first_m + (r % gsize);
   nt = r / gsize;
+}
+
+// One thread's share of a tile's epilogue: BN / 2 columns of one output row, 32 at a time from tensor memory:
+//   v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];  INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.
+template <int BN, bool INT8, int ACT, int OUTK>
+__device__ __forceinline__ void epilogue_columns(const GemmParams& p, const float* e_cs, const float* e_bias,
+                                                 const float* e_post, uint32_t taddr, int m, bool row_ok, float rs,
+                                                 int n0, int chalf) {
+  constexpr int CH = BN / 2;
+  #pragma unroll 1
+          for (int c = 0; c < CH / 32; ++c) {
+            uint32_t r[32];
+            ptx::tmem_ld32(taddr + c * 32, r);
+            ptx::tmem_ld_wait();
+            const int jc = chalf * CH + c * 32;   // column of r[0] inside the tile
+            const int col0 = n0 + jc;
+            if constexpr (OUTK == OUT_I32) {
+              if (row_ok) {
+                int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
+  #pragma unroll
+                for (int g = 0; g < 8; ++g)
+                  if (col0 + 4 * g + 4 <= p.N) st16(dst + 4 * g, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+              }
+            } else {
+              float v[32];
+  #pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float acc = INT8 ? (float)(int)r[j] : __uint_as_float(r[j]);
+                float x = fmaf(acc * rs, e_cs[jc + j], e_bias[jc + j]);
+                if constexpr (ACT == HERO_ACT_GELU_ERF) x = gelu_erf_f(x);
+                if constexpr (ACT == HERO_ACT_GELU_TANH) x = gelu_tanh_f(x);
+                if constexpr (OUTK == OUT_I8) {
+                  // Round (half to even) and clip in the float adder: 1.5 * 2^23 + k keeps k in its low byte
+                  const float y = fmaf(x, e_post[jc + j], ROUND_MAGIC);
+                  v[j] = fminf(fmaxf(y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+                } else {
+                  v[j] = x * e_post[jc + j];
+                }
+              }
+              if (row_ok) {
+                if constexpr (OUTK == OUT_I8) {
+                  int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
+  #pragma unroll
+                  for (int g = 0; g < 2; ++g)
+                    if (col0 + 16 * g + 16 <= p.N)
+                      st16(dst + 16 * g, low_bytes4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
+                           low_bytes4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
+                           low_bytes4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
+                           low_bytes4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
+                } else {
+                  uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
+  #pragma unroll
+                  for (int g = 0; g < 4; ++g)
+                    if (col0 + 8 * g + 8 <= p.N)
+                      st16(dst + 8 * g, pack2_fp(v[8 * g], v[8 * g + 1], p.out_dt), pack2_fp(v[8 * g + 2], v[8 * g + 3], p.out_dt),
+                           pack2_fp(v[8 * g + 4], v[8 * g + 5], p.out_dt), pack2_fp(v[8 * g + 6], v[8 * g + 7], p.out_dt));
+                }
+              }
+            }
+          }
+
 }
 
 template <int BN, bool INT8, int ACT, int OUTK>
@@ -232,57 +294,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       ptx::tc_fence_after();
       if (ok) {
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
-#pragma unroll 1
-        for (int c = 0; c < CH / 32; ++c) {
-          uint32_t r[32];
-          ptx::tmem_ld32(taddr + c * 32, r);
-          ptx::tmem_ld_wait();
-          const int jc = chalf * CH + c * 32;   // column of r[0] inside the tile
-          const int col0 = n0 + jc;
-          if constexpr (OUTK == OUT_I32) {
-            if (row_ok) {
-              int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
-#pragma unroll
-              for (int g = 0; g < 8; ++g)
-                if (col0 + 4 * g + 4 <= p.N) st16(dst + 4 * g, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
-            }
-          } else {
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float acc = INT8 ? (float)(int)r[j] : __uint_as_float(r[j]);
-              float x = fmaf(acc * rs, e_cs[jc + j], e_bias[jc + j]);
-              if constexpr (ACT == HERO_ACT_GELU_ERF) x = gelu_erf_f(x);
-              if constexpr (ACT == HERO_ACT_GELU_TANH) x = gelu_tanh_f(x);
-              if constexpr (OUTK == OUT_I8) {
-                // Round (half to even) and clip in the float adder: 1.5 * 2^23 + k keeps k in its low byte
-                const float y = fmaf(x, e_post[jc + j], ROUND_MAGIC);
-                v[j] = fminf(fmaxf(y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
-              } else {
-                v[j] = x * e_post[jc + j];
-              }
-            }
-            if (row_ok) {
-              if constexpr (OUTK == OUT_I8) {
-                int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
-#pragma unroll
-                for (int g = 0; g < 2; ++g)
-                  if (col0 + 16 * g + 16 <= p.N)
-                    st16(dst + 16 * g, low_bytes4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
-                         low_bytes4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
-                         low_bytes4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
-                         low_bytes4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
-              } else {
-                uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
-#pragma unroll
-                for (int g = 0; g < 4; ++g)
-                  if (col0 + 8 * g + 8 <= p.N)
-                    st16(dst + 8 * g, pack2_fp(v[8 * g], v[8 * g + 1], p.out_dt), pack2_fp(v[8 * g + 2], v[8 * g + 3], p.out_dt),
-                         pack2_fp(v[8 * g + 4], v[8 * g + 5], p.out_dt), pack2_fp(v[8 * g + 6], v[8 * g + 7], p.out_dt));
-              }
-            }
-          }
-        }
+        epilogue_columns<BN, INT8, ACT, OUTK>(p, e_cs, e_bias, e_post, taddr, m, row_ok, rs, n0, chalf);
       }
       // hand the accumulator buffer back to the MMA warp
       ptx::tc_fence_before();
@@ -339,6 +351,237 @@ static hero_status dispatch_epilogue(hero_handle* h, const CUtensorMap& tmA, con
   return HERO_ERR_INVALID_ARG;
 }
 
+// ------------------------------------------------------------------------------------------------------
+// CTA-pair variant (tcgen05 cta_group::2): two CTAs of a cluster share one 256 x 256 tile.  Each CTA loads its
+// own 128 rows of A and its own 128 of the 256 W rows (32 KB per k-block instead of 48 KB for the same number
+// of MACs per SM, which is what the L2 -> SM path limits), the leader CTA's elected lane issues M = 256 UMMAs
+// that read both CTAs' shared memory, and each CTA's tensor memory receives its 128 accumulator rows.
+//   full[s]      (leader's copy) : the leader's producer thread loads all four half-tiles (two into the peer's
+//                                  shared memory); every copy completes on this barrier
+//   empty[s]     (every CTA)     : the leader's commit is multicast to both CTAs
+//   acc_full[a]  (every CTA)     : the leader's commit is multicast to both CTAs
+//   acc_empty[a] (leader's copy) : all 16 epilogue warps of the pair arrive on it
+// No multicast TMA load is used anywhere.
+// ------------------------------------------------------------------------------------------------------
+struct PairCfg {
+  static constexpr int BN = 256;
+  static constexpr int A_BYTES = GEMM_BM * GEMM_BK_BYTES;        // this CTA's 128 rows of A
+  static constexpr int B_BYTES = (BN / 2) * GEMM_BK_BYTES;       // this CTA's 128 rows of W
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = 6;
+  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int EPI_FLOATS = 2 * 3 * BN;
+  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256;
+};
+
+template <bool INT8, int ACT, int OUTK>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
+  using Cfg = PairCfg;
+  constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* tiles = smem;
+  float* epi = reinterpret_cast<float*>(smem + STAGES * Cfg::STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi + Cfg::EPI_FLOATS);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + STAGES;
+  uint64_t* acc_full = bars + 2 * STAGES;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
+  const int num_tiles = p.num_m_tiles * p.num_n_tiles;   // 256 x 256 tiles
+  const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 16); }
+    ptx::fence_mbar_init();
+  }
+  if (warp == MMA_WARP) {
+    ptx::tmem_alloc_pair(tmem_slot, Cfg::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  if (warp == TMA_WARP && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();                                   // both CTAs' barriers exist before any remote arrive
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == TMA_WARP) {
+    // ------------------------------------------------------------------ TMA producer (leader CTA only)
+    // One thread feeds both CTAs: its own halves of A and W go to local shared memory, the peer's halves to the
+    // peer's shared memory, all four copies completing on the leader's `full` barrier.  The peer needs no producer,
+    // so the stage hand-off costs one barrier round trip, not a cross-CTA chain.
+    if (lane == 0 && rank == 0) {
+      const int kelems = GEMM_BK_BYTES / p.elem_bytes;
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      for (int t = pair_id; t < num_tiles && ok; t += num_pairs) {
+        int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x700 | stage)) { ok = false; break; }
+          const uint32_t a_loc = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
+          const uint32_t b_loc = a_loc + Cfg::A_BYTES;
+          const uint32_t bar = ptx::mapa(ptx::smem_u32(&full[stage]), 0);
+          ptx::mbar_expect_tx(&full[stage], 2 * Cfg::STAGE_BYTES);
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            ptx::tma_load_2d_pair(ptx::mapa(a_loc, r), &tmA, kb * kelems, mt * 256 + r * GEMM_BM, bar);
+            ptx::tma_load_2d_pair(ptx::mapa(b_loc, r), &tmW, kb * kelems, nt * BN + r * (BN / 2), bar);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      for (int i = 0; i < STAGES; ++i) {                 // drain: every copy started here has been consumed
+        if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x780 | stage)) break;
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == MMA_WARP) {
+    // ------------------------------------------------------------------ UMMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      int it = 0;
+      for (int t = pair_id; t < num_tiles && ok; t += num_pairs, ++it) {
+        const int as = it & 1;
+        const uint32_t aphase = (it >> 1) & 1;
+        if (!ptx::mbar_wait(&acc_empty[as], aphase ^ 1, p.err, 0x800 | as)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + as * BN;
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!ptx::mbar_wait(&full[stage], phase, p.err, 0x900 | stage)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_addr = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + Cfg::A_BYTES;
+#pragma unroll
+          for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
+            const uint64_t ad = ptx::smem_desc(desc_base, a_addr + k * 32);
+            const uint64_t bd = ptx::smem_desc(desc_base, b_addr + k * 32);
+            if constexpr (INT8) ptx::umma_i8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            else ptx::umma_f16_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+          }
+          ptx::umma_commit_pair(&empty[stage], 3);       // frees this stage in both CTAs
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) ptx::umma_commit_pair(&acc_full[as], 3);  // both CTAs' accumulator halves are complete
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-7 of each CTA)
+    const int quarter = warp & 3, chalf = warp >> 2;
+    constexpr int CH = BN / 2;
+    const int tid_e = threadIdx.x;
+    int it = 0; bool ok = true;
+    for (int t = pair_id; t < num_tiles; t += num_pairs, ++it) {
+      int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+      const int as = it & 1;
+      const uint32_t aphase = (it >> 1) & 1;
+      const int n0 = nt * BN;
+      float* e_cs = epi + (it & 1) * 3 * BN;
+      float* e_bias = e_cs + BN;
+      float* e_post = e_bias + BN;
+      if constexpr (OUTK != OUT_I32) {
+        for (int j = tid_e; j < BN; j += 256) {
+          const int n = n0 + j;
+          const bool in = n < p.N;
+          e_cs[j] = (in && p.cs) ? p.cs[n] : 1.0f;
+          e_bias[j] = (in && p.bias) ? p.bias[n] : 0.0f;
+          e_post[j] = (in && p.post) ? p.post[n] : 1.0f;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+      }
+      const int m = mt * 256 + (int)rank * GEMM_BM + quarter * 32 + lane;
+      const bool row_ok = m < p.M;
+      float rs = 1.0f;
+      if (OUTK != OUT_I32 && INT8 && p.rs && row_ok) rs = p.rs[m];
+
+      if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0xa00 | as)) ok = false;
+      ptx::tc_fence_after();
+      if (ok) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
+        epilogue_columns<BN, INT8, ACT, OUTK>(p, e_cs, e_bias, e_post, taddr, m, row_ok, rs, n0, chalf);
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&acc_empty[as]), 0));
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();                                   // the peer may still be reading this CTA's shared memory / barriers
+  if (warp == MMA_WARP) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
+}
+
+template <bool INT8, int ACT, int OUTK>
+static hero_status launch_gemm_pair(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+                                    cudaStream_t stream) {
+  auto kern = gemm_pair_kernel<INT8, ACT, OUTK>;
+  static bool configured = false;
+  if (!configured) {
+    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg::SMEM_BYTES));
+    configured = true;
+  }
+  const int tiles = p.num_m_tiles * p.num_n_tiles;
+  const int pairs_max = h->sm_count / 2;
+  const int pairs = tiles < pairs_max ? tiles : pairs_max;
+  {
+    LaunchScope scope(h, stream, KERNEL_GEMM);
+    kern<<<2 * pairs, GEMM_THREADS, PairCfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+  }
+  HERO_CUDA(cudaGetLastError());
+  return HERO_OK;
+}
+
+template <bool INT8>
+static hero_status dispatch_epilogue_pair(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+                                          int act, cudaStream_t s) {
+  if (p.out_dt == HERO_I32) {
+    if constexpr (INT8) return launch_gemm_pair<true, HERO_ACT_NONE, OUT_I32>(h, tmA, tmW, p, s);
+    else { set_error("raw INT32 output needs INT8 operands"); return HERO_ERR_UNSUPPORTED; }
+  }
+  const bool i8 = p.out_dt == HERO_I8;
+  switch (act) {
+    case HERO_ACT_NONE:
+      return i8 ? launch_gemm_pair<INT8, HERO_ACT_NONE, OUT_I8>(h, tmA, tmW, p, s)
+                : launch_gemm_pair<INT8, HERO_ACT_NONE, OUT_FP>(h, tmA, tmW, p, s);
+    case HERO_ACT_GELU_ERF:
+      return i8 ? launch_gemm_pair<INT8, HERO_ACT_GELU_ERF, OUT_I8>(h, tmA, tmW, p, s)
+                : launch_gemm_pair<INT8, HERO_ACT_GELU_ERF, OUT_FP>(h, tmA, tmW, p, s);
+    case HERO_ACT_GELU_TANH:
+      return i8 ? launch_gemm_pair<INT8, HERO_ACT_GELU_TANH, OUT_I8>(h, tmA, tmW, p, s)
+                : launch_gemm_pair<INT8, HERO_ACT_GELU_TANH, OUT_FP>(h, tmA, tmW, p, s);
+  }
+  set_error("unknown activation %d", act);
+  return HERO_ERR_INVALID_ARG;
+}
+
+static hero_status run_pair(hero_handle* h, const hero_linear_args* a, GemmParams& p, cudaStream_t s) {
+  const bool int8 = a->A.dtype == HERO_I8;
+  const int eb = int8 ? 1 : 2;
+  const int kbox = GEMM_BK_BYTES / eb;
+  p.num_m_tiles = (p.M + 255) / 256;
+  p.num_n_tiles = (p.N + 255) / 256;
+  const bool bf = a->A.dtype == HERO_BF16;
+  p.idesc = int8 ? ptx::make_idesc(2, 1, 1, 0, 0, 256, 256) : ptx::make_idesc(1, bf ? 1 : 0, bf ? 1 : 0, 0, 0, 256, 256);
+  CUtensorMap tmA, tmW;
+  hero_status st = make_tmap_2d(h, &tmA, a->A.data, eb, a->A.dtype == HERO_F16, bf, (uint64_t)p.M, (uint64_t)p.K,
+                                (uint64_t)a->A.ld * eb, kbox, GEMM_BM, 128);
+  if (st != HERO_OK) return st;
+  st = make_tmap_2d(h, &tmW, a->W, eb, a->A.dtype == HERO_F16, bf, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)a->ldw * eb, kbox,
+                    128, 128);
+  if (st != HERO_OK) return st;
+  if (int8) return dispatch_epilogue_pair<true>(h, tmA, tmW, p, a->act, s);
+  return dispatch_epilogue_pair<false>(h, tmA, tmW, p, a->act, s);
+}
+
 template <int BN>
 static hero_status run_bn(hero_handle* h, const hero_linear_args* a, GemmParams& p, cudaStream_t s) {
   const bool int8 = a->A.dtype == HERO_I8;
@@ -358,7 +601,11 @@ static hero_status run_bn(hero_handle* h, const hero_linear_args* a, GemmParams&
   return dispatch_epilogue<BN, false>(h, tmA, tmW, p, a->act, s);
 }
 
+int g_gemm_pair = 1;
+
 }  // namespace hero
+
+extern "C" void hero_debug_gemm_pair(int on) { hero::g_gemm_pair = on; }
 
 extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* stream) {
   using namespace hero;
@@ -403,6 +650,8 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   const long long t256 = (long long)p.num_m_tiles * ((p.N + 255) / 256);
   const long long t128 = (long long)p.num_m_tiles * ((p.N + 127) / 128);
   const long long enough = (long long)h->sm_count * 6 / 10;
+  const long long tpair = (long long)((p.M + 255) / 256) * ((p.N + 255) / 256);
+  if (g_gemm_pair && tpair * 2 >= enough && p.M > GEMM_BM) return run_pair(h, a, p, s);
   if (t256 >= enough) return run_bn<256>(h, a, p, s);
   if (t128 >= enough) return run_bn<128>(h, a, p, s);
   return run_bn<64>(h, a, p, s);

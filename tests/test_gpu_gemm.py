@@ -34,8 +34,9 @@ def _linear(h, A, Wt, out_dtype, rs=None, cs=None, bias=None, act="none", post=N
 
 
 # shapes span one tile, several tiles, ragged M / N / K tails and every column-tile width
+# (the last three are large enough to take the CTA-pair kernel: 256 x 256 tiles, ragged in M and N)
 SHAPES = [(128, 128, 256), (1, 64, 16), (17, 80, 48), (127, 256, 272), (129, 1024, 512), (300, 768, 2304),
-          (1000, 4096, 1024), (2500, 512, 4096), (16, 4096, 4096)]
+          (1000, 4096, 1024), (16, 4096, 4096), (2500, 512, 4096), (600, 128, 7984), (12288, 1024, 1024)]
 
 
 @pytest.mark.parametrize("M,K,N", SHAPES)
@@ -57,7 +58,7 @@ def test_int32_extreme_values_bit_exact(h):
     assert np.array_equal(got, O.int_matmul(A, Wt.T.copy()))
 
 
-@pytest.mark.parametrize("M,K,N", [(128, 1024, 4096), (333, 4096, 1024), (16, 1024, 4096), (1024, 1024, 4096)])
+@pytest.mark.parametrize("M,K,N", [(128, 1024, 4096), (333, 4096, 1024), (16, 1024, 4096), (1024, 1024, 4096), (1500, 256, 4096)])
 def test_requant_epilogue_round_only(h, M, K, N):
     # Eq. 22: dequantize by row and column scale, add the folded bias, Round -> INT8
     A, Wt, rs, cs, bias = W.gemm_case(M, K, N)
@@ -69,9 +70,10 @@ def test_requant_epilogue_round_only(h, M, K, N):
 
 
 @pytest.mark.parametrize("act", ["gelu_erf", "gelu_tanh"])
-def test_fc1_gelu_quant_epilogue(h, act):
+@pytest.mark.parametrize("M", [260, 1100])
+def test_fc1_gelu_quant_epilogue(h, act, M):
     # Eq. 28-29: X_1 stays FP32 on chip, GELU, then FWQ with 1 / S_a
-    M, K, N = 260, 768, 3072
+    K, N = 768, 3072
     g = W.rng(2, 555)
     A = g.integers(-127, 128, (M, K), dtype=np.int8)
     Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
@@ -100,7 +102,7 @@ def test_int8_gemm_fp_output(h, fp):
 
 
 @pytest.mark.parametrize("fp", ["f16", "bf16"])
-@pytest.mark.parametrize("M,K,N", [(128, 64, 256), (200, 1024, 768), (77, 136, 48)])
+@pytest.mark.parametrize("M,K,N", [(128, 64, 256), (200, 1024, 768), (77, 136, 48), (1030, 256, 4096)])
 def test_fp_mode_gemm(h, fp, M, K, N):
     # a module left in FP16/BF16 (Table 1): X W + b with fp32 accumulation
     g = W.rng(2, 777 + M)
