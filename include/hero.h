@@ -248,6 +248,23 @@ hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, co
                                     const hero_tensor* out_host, const hero_tensor* in_dev, const hero_tensor* out_dev,
                                     void* workspace, size_t workspace_bytes, void* stream);
 
+/* The layer forward for callers that cannot allocate device memory (the paper has no counterpart: it describes
+ * no software interface).  Who needs it: code that runs inside another framework's fixed memory plan, real-time
+ * or plugin paths where an allocation might block or fail late, processes that own only the buffers they were
+ * started with.  It takes no handle and no workspace and calls no cudaMalloc / cudaFree or any other allocating
+ * routine: its scratch is a 64 MiB array built into the library image, present on every GPU that loads the
+ * library until the process exits.
+ *   - A layer whose workspace (hero_layer_workspace_bytes) exceeds 64 MiB is refused with HERO_ERR_WORKSPACE.
+ *   - The first call on a device looks up the array's device address and the driver's tensor-map encoder; make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left in it (nothing in it
+ *     needs clearing: each call overwrites what it reads).  Two calls that overlap on the GPU, e.g. on two
+ *     streams, race on it: serialize them.
+ *   - A bounded device-side wait that gives up cannot be reported here (there is no handle to hero_check).
+ * Inputs, outputs, weights and scales are passed exactly as for hero_layer_forward. */
+hero_status hero_layer_forward_static(const hero_layer_desc* d, const hero_tensor* in, const hero_tensor* pending,
+                                      const hero_tensor* out, void* stream);
+
 /* Per-launch device timing for benchmarks (no counterpart in the paper, which measured nothing): between
  * _begin and _end every kernel the handle launches is bracketed by a pair of CUDA events on its stream.
  * _end waits for them and returns, per launch in order, the elapsed milliseconds and the kernel family

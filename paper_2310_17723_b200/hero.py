@@ -77,7 +77,7 @@ class LayerDesc(C.Structure):
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
-           "hero_profile_end")
+           "hero_profile_end", "hero_layer_forward_static")
 
 _lib = None
 
@@ -105,6 +105,8 @@ def lib():
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_host.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
             [C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hero_layer_forward_static.argtypes = [C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
+                                                C.POINTER(Tensor), C.c_void_p]
         L.hero_profile_begin.argtypes = [C.c_void_p, C.c_int32]
         L.hero_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         _lib = L
@@ -228,6 +230,14 @@ def host_tensor(t, gran="none", scale=None):
     T = Tensor(t.data_ptr(), _DT[t.dtype], g, t.shape[0], t.shape[1], t.stride(0), None if scale is None else scale.data_ptr())
     T._keep = (t, scale)
     return T
+
+
+def hero_layer_forward_static(desc, x_in, out, pending=None, stream=None):
+    """The layer forward without handle or workspace, for callers that may not allocate device memory: the
+    scratch is a fixed 64 MiB array inside libhero.so (larger layers are refused).  Calls share that array, so
+    do not let two of them overlap on the GPU."""
+    pend = C.byref(pending) if pending is not None else None
+    _check(lib().hero_layer_forward_static(C.byref(desc), C.byref(x_in), pend, C.byref(out), _stream(stream)))
 
 
 def mode_preset(preset):
