@@ -53,7 +53,45 @@ def workload_spec(name):
     if name == "c4":
         s = W.C4
         return s, 4, [cfg(s)], "C4: GPT prefill layer, B8 S2048 H4096 nh32 F16384, pre-LN, causal, W8A8 everywhere"
+    if name == "c5":
+        s = W.C5
+        g = W.rng(5, 99)
+        n_layers = 24
+        fp_layers = set(int(i) for i in g.choice(n_layers, size=2, replace=False))
+        kinds = [str(k) for k in g.choice(["twq", "fwq", "sq_attn"], size=n_layers)]
+        cfgs = []
+        for li in range(n_layers):
+            if li in fp_layers:
+                c = prep.LayerConfig(B=s.B, S=s.S, H=s.H, nh=s.nh, F=s.F, arch=s.arch, eps=s.eps, mask=s.mask,
+                                     fp_dtype=s.fp_dtype, mode=dict(prep.PRESETS["FP"]))
+            elif kinds[li] == "fwq":
+                c = cfg(s, gran_in="fwq")
+            elif kinds[li] == "sq_attn":
+                c = cfg(s, gran_attn="sq")
+            else:
+                c = cfg(s)
+            cfgs.append(c)
+        for li, c in enumerate(cfgs):                      # a layer emits what the next layer's QKV consumes
+            if li + 1 < n_layers:
+                nxt = cfgs[li + 1]
+                c.gran_out = "fp" if nxt.mode["qkv"] == "fp" else nxt.gran_in
+            else:
+                c.gran_out = "fp"
+        return s, 5, cfgs, "C5: 24 x BERT-large layer, B64 S512 H1024 F4096, post-LN, seeded TWQ/FWQ/SQ mix, layers %s in FP16, FP16 output" % sorted(fp_layers)
     raise SystemExit("unknown workload %r" % name)
+
+
+def fp_variant(cfgs):
+    """The same layers with every module left in FP16/BF16 (the library's own FP path, for the W8A8 speed-up)."""
+    from paper_2310_17723_b200 import prep
+    import copy
+    out = []
+    for c in cfgs:
+        c2 = copy.deepcopy(c)
+        c2.mode = dict(prep.PRESETS["FP"])
+        c2.gran_out = "fp"
+        out.append(c2)
+    return out
 
 
 def kernel_table(shape, cfg):
@@ -61,19 +99,20 @@ def kernel_table(shape, cfg):
     M, H, F, S, nh, dh = shape.M, shape.H, shape.F, shape.S, shape.nh, shape.dh
     causal = shape.mask == "causal"
 
-    def gemm(name, K, N):
-        return (name, "gemm", 2.0 * M * N * K, float(M * K + N * K + M * N + 4 * M + 8 * N))
+    def gemm(name, K, N, module="qkv"):
+        fam = "gemm" if cfg.mode[module] == "int8" else "gemm_fp"
+        return (name, fam, 2.0 * M * N * K, float(M * K + N * K + M * N + 4 * M + 8 * N))
     attn_ops = 4.0 * shape.B * nh * S * S * dh * (0.5 if causal else 1.0)
     attn = ("attention", "attn", attn_ops, float(4 * M * H))
     rows = []
     if shape.arch == "pre_ln":
         rows.append(("ln1 (fp->i8 twq)", "ln", 0.0, float(M * H * 3 + 4 * M)))
-    rows += [gemm("qkv gemm", H, 3 * H), attn, gemm("attn-out gemm", H, H)]
+    rows += [gemm("qkv gemm", H, 3 * H, "qkv"), attn, gemm("attn-out gemm", H, H, "attn_out")]
     if shape.arch == "pre_ln":
         rows.append(("add+ln2 (fp+i8->fp,i8)", "ln", 0.0, float(M * H * 6 + 4 * M)))
     else:
         rows.append(("ln1 (i8+i8->i8 twq)", "ln", 0.0, float(M * H * 3 + 8 * M)))
-    rows += [gemm("fc1 gemm + gelu^quant", H, F), gemm("fc2 gemm", F, H)]
+    rows += [gemm("fc1 gemm + gelu^quant", H, F, "fc1"), gemm("fc2 gemm", F, H, "fc2")]
     if shape.arch == "pre_ln":
         rows.append(("closing add (fp+i8->fp)", "ln", 0.0, float(M * H * 5)))
     else:
@@ -134,29 +173,38 @@ class ClockSampler:
 # CPU oracle arm (also the cpu_baseline leg)
 # ------------------------------------------------------------------------------------------------
 def oracle_run(name, budget_s=12.0, repeats=1):
-    """Times the oracle, as it stands, on whole sequences of the workload.  Returns (tokens/s, cores, sample)."""
+    """Times the oracle, as it stands, on whole sequences of the workload (all of its layers).
+    Returns (tokens/s, cores, sample, seconds)."""
     import numpy as np
     from oracle import layer as OL, ops as O
     from paper_2310_17723_b200 import workloads as W
     shape, cid, cfgs, desc = workload_spec(name)
-    cfg = cfgs[0]
-    spec = OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, act=cfg.act, eps=cfg.eps,
-                        mask=cfg.mask, fp_dtype=cfg.fp_dtype, mode=dict(cfg.mode), gran_in=cfg.gran_in,
-                        gran_mid=cfg.gran_mid, gran_attn=cfg.gran_attn, gran_out=cfg.gran_out)
-    p = W.layer_params(shape, cid * 100)
     x_cal = W.activations(shape, cid, n_seq=1, tensor=7).astype(np.float64)
-    cal_in = O.layernorm(x_cal, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else x_cal
-    C = OL.calibrate(spec, p, cal_in, 1)
-    Lp = OL.prepare_layer(spec, p, C)
+    layers = []
+    cur = None
+    for li, cfg in enumerate(cfgs):                       # offline preparation of every layer (not timed)
+        spec = OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, act=cfg.act,
+                            eps=cfg.eps, mask=cfg.mask, fp_dtype=cfg.fp_dtype, mode=dict(cfg.mode), gran_in=cfg.gran_in,
+                            gran_mid=cfg.gran_mid, gran_attn=cfg.gran_attn, gran_out=cfg.gran_out)
+        p = W.layer_params(shape, cid * 100 + li)
+        if li == 0:
+            ln0 = (p["ln0_g"], p["ln0_b"])
+            cur = O.layernorm(x_cal, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else x_cal
+        C = OL.calibrate(spec, p, cur, 1)
+        if len(cfgs) > 1:
+            cur = OL.layer_fp64(spec, p, cur, B=1)["x_out"]
+        layers.append((spec, OL.prepare_layer(spec, p, C)))
 
     def run(n_seq):
         x = W.activations(shape, cid, n_seq=n_seq)
-        if spec.arch == "post_ln":
-            x_in = OL.entry_ln(O.fp_tensor(x, "f16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+        spec0, L0 = layers[0]
+        if spec0.arch == "post_ln":
+            cur_t = OL.entry_ln(O.fp_tensor(x, spec0.fp_dtype), ln0[0], ln0[1], spec0.eps, L0["ln_in_out"])
         else:
-            x_in = O.fp_tensor(x, spec.fp_dtype)
+            cur_t = O.fp_tensor(x, spec0.fp_dtype)
         t0 = time.perf_counter()
-        OL.layer_forward(Lp, x_in, B=n_seq)
+        for spec, Lp in layers:
+            cur_t = OL.layer_forward(Lp, cur_t, B=n_seq)["x_out"]
         return time.perf_counter() - t0
 
     t1 = run(1)
@@ -168,7 +216,8 @@ def oracle_run(name, budget_s=12.0, repeats=1):
         cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     except Exception:
         pass
-    return n * shape.S / best, cores, "%d of %d sequences (%d tokens) of %s, one pass" % (n, shape.B, n * shape.S, shape.name), best
+    sample = "%d of %d sequences (%d tokens) of %s through %d layer(s), one pass" % (n, shape.B, n * shape.S, shape.name, len(layers))
+    return n * shape.S / best, cores, sample, best
 
 
 def run_reference(args):
@@ -279,12 +328,21 @@ def run_ours(args):
             table += kernel_table(shape, cfg)
         assert len(table) == launches_per_step, (len(table), launches_per_step)
         int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        merged = {}
         for i, (name, fam, ops, nbytes) in enumerate(table):
             ms = [recs[j][1] for j in range(i, len(recs), launches_per_step)]
             avg = sum(ms) / len(ms)
-            row = {"kernel": name, "ms": round(avg, 5), "share": None}
+            key = (name, fam)
+            if key in merged:                                  # same kernel in another layer of the stack
+                merged[key] = (merged[key][0] + avg, merged[key][1] + ops, merged[key][2] + nbytes, merged[key][3] + 1)
+            else:
+                merged[key] = (avg, ops, nbytes, 1)
+        for (name, fam), (avg, ops, nbytes, cnt) in merged.items():
+            row = {"kernel": name if fam != "gemm_fp" else name + " (fp16)", "ms": round(avg, 5), "share": None, "launches_per_step": cnt}
             if fam == "gemm":
                 row.update(bound="tensor", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak, unit="TFLOP/s")
+            elif fam == "gemm_fp":
+                row.update(bound="tensor", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak / 2, unit="TFLOP/s")
             elif fam == "ln":
                 row.update(bound="hbm", achieved=nbytes / (avg * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
             else:
@@ -344,6 +402,28 @@ def run_ours(args):
     e2e = {"value": replicas.job_throughput(shape.M, args.steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
     h.check()
 
+    fp_path = None
+    if rank == 0 and world == 1 and not args.no_fp_path:
+        # the same layer(s) with every module in FP16/BF16, through the same library and the same timing loop
+        del stack
+        torch.cuda.empty_cache()
+        fstack = Stack(h, shape, cid, fp_variant(cfgs), n_cal_seq=1)
+        fstack.set_input(x_dev)
+        for _ in range(3):
+            flush.zero_()
+            fstack.forward()
+        torch.cuda.synchronize()
+        fev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for k in range(args.steps):
+            flush.zero_()
+            fev[k][0].record(stream)
+            fstack.forward()
+            fev[k][1].record(stream)
+        torch.cuda.synchronize()
+        h.check()
+        fms = sum(a.elapsed_time(b) for a, b in fev) / args.steps
+        fp_path = {"value": shape.M / (fms * 1e-3), "unit": UNIT, "ms_per_step": fms, "dtype": shape.fp_dtype,
+                   "w8a8_speedup": ms_per_step and fms / ms_per_step}
     if rank != 0:
         if dist:
             dist.destroy_process_group()
@@ -359,7 +439,7 @@ def run_ours(args):
                        "timing": "CUDA events per step on the launching stream, max over ranks",
                        "parallelism": "replicas x%d (sequence-sharded, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "kernels": kern,
-            "cpu_baseline": cpu, "wall_s_timed_region": wall}
+            "cpu_baseline": cpu, "fp16_path": fp_path, "wall_s_timed_region": wall}
     print(json.dumps(line), flush=True)
     if dist:
         dist.destroy_process_group()
@@ -371,8 +451,9 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4", "c5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fp-path", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

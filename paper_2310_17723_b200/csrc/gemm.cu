@@ -109,65 +109,186 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mt
   nt = r / gsize;
 }
 
-// One thread's share of a tile's epilogue: BN / 2 columns of one output row, 32 at a time from tensor memory:
-//   v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];  INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.
+__device__ __forceinline__ void st32(void* p, const uint32_t (&w)[8]) {   // 256-bit store, 32-byte aligned
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+               "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+
+// 32 columns of one output row: v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];
+// INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.  Per-column vectors come from shared memory four at a time,
+// the arithmetic runs on packed FP32 pairs, the row segment leaves in 32-byte stores when the output allows it.
+template <bool INT8, int ACT, int OUTK>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32_t (&r)[32], const float* e_cs,
+                                               const float* e_bias, const float* e_post, int m, bool row_ok, float rs,
+                                               int col0, bool wide) {
+  if constexpr (OUTK == OUT_I32) {
+    if (!row_ok) return;
+    int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
+    if (wide && col0 + 32 <= p.N) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const uint32_t w[8] = {r[8 * g], r[8 * g + 1], r[8 * g + 2], r[8 * g + 3], r[8 * g + 4], r[8 * g + 5], r[8 * g + 6], r[8 * g + 7]};
+        st32(dst + 8 * g, w);
+      }
+    } else {
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        if (col0 + 4 * g + 4 <= p.N) st16(dst + 4 * g, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+    }
+  } else {
+    float v[32];
+    const float2 rs2 = make_float2(rs, rs), mg2 = make_float2(ROUND_MAGIC, ROUND_MAGIC);
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      const float4 cs4 = *reinterpret_cast<const float4*>(e_cs + j);
+      const float4 b4 = *reinterpret_cast<const float4*>(e_bias + j);
+      const float4 p4 = *reinterpret_cast<const float4*>(e_post + j);
+      float2 a0, a1;
+      if constexpr (INT8) {
+        a0 = make_float2((float)(int)r[j], (float)(int)r[j + 1]);
+        a1 = make_float2((float)(int)r[j + 2], (float)(int)r[j + 3]);
+      } else {
+        a0 = make_float2(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+        a1 = make_float2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+      }
+      float2 x0 = __ffma2_rn(__fmul2_rn(a0, rs2), make_float2(cs4.x, cs4.y), make_float2(b4.x, b4.y));
+      float2 x1 = __ffma2_rn(__fmul2_rn(a1, rs2), make_float2(cs4.z, cs4.w), make_float2(b4.z, b4.w));
+      if constexpr (ACT == HERO_ACT_GELU_ERF) {
+        x0.x = gelu_erf_f(x0.x); x0.y = gelu_erf_f(x0.y); x1.x = gelu_erf_f(x1.x); x1.y = gelu_erf_f(x1.y);
+      }
+      if constexpr (ACT == HERO_ACT_GELU_TANH) {
+        x0.x = gelu_tanh_f(x0.x); x0.y = gelu_tanh_f(x0.y); x1.x = gelu_tanh_f(x1.x); x1.y = gelu_tanh_f(x1.y);
+      }
+      if constexpr (OUTK == OUT_I8) {
+        // Round (half to even) and clip in the float adder: 1.5 * 2^23 + k keeps k in its low byte
+        const float2 y0 = __ffma2_rn(x0, make_float2(p4.x, p4.y), mg2);
+        const float2 y1 = __ffma2_rn(x1, make_float2(p4.z, p4.w), mg2);
+        v[j] = fminf(fmaxf(y0.x, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+        v[j + 1] = fminf(fmaxf(y0.y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+        v[j + 2] = fminf(fmaxf(y1.x, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+        v[j + 3] = fminf(fmaxf(y1.y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+      } else {
+        const float2 y0 = __fmul2_rn(x0, make_float2(p4.x, p4.y));
+        const float2 y1 = __fmul2_rn(x1, make_float2(p4.z, p4.w));
+        v[j] = y0.x; v[j + 1] = y0.y; v[j + 2] = y1.x; v[j + 3] = y1.y;
+      }
+    }
+    if (!row_ok) return;
+    if constexpr (OUTK == OUT_I8) {
+      int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
+      uint32_t w[8];
+#pragma unroll
+      for (int g = 0; g < 8; ++g) w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+      if (wide && col0 + 32 <= p.N) {
+        st32(dst, w);
+      } else {
+        if (col0 + 16 <= p.N) st16(dst, w[0], w[1], w[2], w[3]);
+        if (col0 + 32 <= p.N) st16(dst + 16, w[4], w[5], w[6], w[7]);
+      }
+    } else {
+      uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
+      uint32_t w[16];
+#pragma unroll
+      for (int g = 0; g < 16; ++g) w[g] = pack2_fp(v[2 * g], v[2 * g + 1], p.out_dt);
+      if (wide && col0 + 32 <= p.N) {
+        const uint32_t w0[8] = {w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]};
+        const uint32_t w1[8] = {w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]};
+        st32(dst, w0);
+        st32(dst + 16, w1);
+      } else {
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          if (col0 + 8 * g + 8 <= p.N) st16(dst + 8 * g, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+      }
+    }
+  }
+}
+
+// One thread's share of a tile's epilogue: BN / 2 columns of one output row, 32 at a time from tensor memory,
+// the next 32 already loading while the current ones are processed.
 template <int BN, bool INT8, int ACT, int OUTK>
 __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const float* e_cs, const float* e_bias,
                                                  const float* e_post, uint32_t taddr, int m, bool row_ok, float rs,
                                                  int n0, int chalf) {
-  constexpr int CH = BN / 2;
-  #pragma unroll 1
-          for (int c = 0; c < CH / 32; ++c) {
-            uint32_t r[32];
-            ptx::tmem_ld32(taddr + c * 32, r);
-            ptx::tmem_ld_wait();
-            const int jc = chalf * CH + c * 32;   // column of r[0] inside the tile
-            const int col0 = n0 + jc;
-            if constexpr (OUTK == OUT_I32) {
-              if (row_ok) {
-                int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
-  #pragma unroll
-                for (int g = 0; g < 8; ++g)
-                  if (col0 + 4 * g + 4 <= p.N) st16(dst + 4 * g, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
-              }
-            } else {
-              float v[32];
-  #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float acc = INT8 ? (float)(int)r[j] : __uint_as_float(r[j]);
-                float x = fmaf(acc * rs, e_cs[jc + j], e_bias[jc + j]);
-                if constexpr (ACT == HERO_ACT_GELU_ERF) x = gelu_erf_f(x);
-                if constexpr (ACT == HERO_ACT_GELU_TANH) x = gelu_tanh_f(x);
-                if constexpr (OUTK == OUT_I8) {
-                  // Round (half to even) and clip in the float adder: 1.5 * 2^23 + k keeps k in its low byte
-                  const float y = fmaf(x, e_post[jc + j], ROUND_MAGIC);
-                  v[j] = fminf(fmaxf(y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
-                } else {
-                  v[j] = x * e_post[jc + j];
-                }
-              }
-              if (row_ok) {
-                if constexpr (OUTK == OUT_I8) {
-                  int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
-  #pragma unroll
-                  for (int g = 0; g < 2; ++g)
-                    if (col0 + 16 * g + 16 <= p.N)
-                      st16(dst + 16 * g, low_bytes4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
-                           low_bytes4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
-                           low_bytes4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
-                           low_bytes4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
-                } else {
-                  uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
-  #pragma unroll
-                  for (int g = 0; g < 4; ++g)
-                    if (col0 + 8 * g + 8 <= p.N)
-                      st16(dst + 8 * g, pack2_fp(v[8 * g], v[8 * g + 1], p.out_dt), pack2_fp(v[8 * g + 2], v[8 * g + 3], p.out_dt),
-                           pack2_fp(v[8 * g + 4], v[8 * g + 5], p.out_dt), pack2_fp(v[8 * g + 6], v[8 * g + 7], p.out_dt));
-                }
-              }
-            }
-          }
+  constexpr int CH = BN / 2, NCH = CH / 32;
+  // 32-byte stores need a 32-byte aligned row segment: base pointer and row pitch multiples of 32 bytes
+  const int es = OUTK == OUT_I8 ? 1 : (OUTK == OUT_FP ? 2 : 4);
+  const bool wide = ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0) && ((p.out_ld * es) % 32 == 0);
+  uint32_t ra[32], rb[32];
+  ptx::tmem_ld32(taddr, ra);
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    ptx::tmem_ld_wait();
+    if (c + 1 < NCH) ptx::tmem_ld32(taddr + (c + 1) * 32, (c & 1) ? ra : rb);
+    const int jc = chalf * CH + c * 32;   // column of the chunk's first element inside the tile
+    if (c & 1) epilogue_chunk<INT8, ACT, OUTK>(p, rb, e_cs + jc, e_bias + jc, e_post + jc, m, row_ok, rs, n0 + jc, wide);
+    else epilogue_chunk<INT8, ACT, OUTK>(p, ra, e_cs + jc, e_bias + jc, e_post + jc, m, row_ok, rs, n0 + jc, wide);
+  }
+}
 
+// The epilogue warps' walk over this CTA's tiles.  The per-column vectors (and the row scale) of the NEXT tile are
+// fetched from global memory into registers while the current tile is being processed, so a tile never starts by
+// waiting on them.  ROWS = output rows per tile (128, or 256 for a CTA pair of which this CTA owns rows row_off..+127).
+template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR>
+__device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, uint64_t* acc_full, uint64_t* acc_empty,
+                                              uint32_t tmem_base, int first_tile, int tile_stride, int row_off) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quarter = warp & 3, chalf = warp >> 2;
+  constexpr int CH = BN / 2;                 // columns per thread and tile
+  const int tid_e = threadIdx.x;             // 0..255: the column of the tile whose vectors this thread stages
+  const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+  bool ok = true;
+
+  float ncs = 1.0f, nbias = 0.0f, npost = 1.0f, nrs = 1.0f;
+  auto fetch = [&](int t) {                  // issue the loads for tile t; the values are consumed one tile later
+    int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+    if constexpr (OUTK != OUT_I32) {
+      const int n = nt * BN + tid_e;
+      const bool in = tid_e < BN && n < p.N;
+      ncs = (in && p.cs) ? __ldg(p.cs + n) : 1.0f;
+      nbias = (in && p.bias) ? __ldg(p.bias + n) : 0.0f;
+      npost = (in && p.post) ? __ldg(p.post + n) : 1.0f;
+      const int m = mt * ROWS + row_off + quarter * 32 + lane;
+      nrs = (INT8 && p.rs && m < p.M) ? __ldg(p.rs + m) : 1.0f;
+    }
+  };
+  auto publish = [&](int it) {               // registers -> this tile's shared-memory vectors
+    if constexpr (OUTK != OUT_I32) {
+      float* e = epi + (it & 1) * 3 * BN;
+      if (tid_e < BN) { e[tid_e] = ncs; e[BN + tid_e] = nbias; e[2 * BN + tid_e] = npost; }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
+  };
+
+  if (first_tile < num_tiles) fetch(first_tile);
+  int it = 0;
+  for (int t = first_tile; t < num_tiles; t += tile_stride, ++it) {
+    int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+    const int as = it & 1;
+    const uint32_t aphase = (it >> 1) & 1;
+    const int n0 = nt * BN;
+    const float rs = nrs;
+    publish(it);
+    if (t + tile_stride < num_tiles) fetch(t + tile_stride);
+    const float* e_cs = epi + (it & 1) * 3 * BN;
+    const int m = mt * ROWS + row_off + quarter * 32 + lane;
+    const bool row_ok = m < p.M;
+
+    if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
+    ptx::tc_fence_after();
+    if (ok) {
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
+      epilogue_columns<BN, INT8, ACT, OUTK>(p, e_cs, e_cs + BN, e_cs + 2 * BN, taddr, m, row_ok, rs, n0, chalf);
+    }
+    // hand the accumulator buffer back to the UMMA issuer
+    ptx::tc_fence_before();
+    __syncwarp();
+    if (lane == 0) {
+      if constexpr (PAIR) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&acc_empty[as]), 0));
+      else ptx::mbar_arrive(&acc_empty[as]);
+    }
+  }
 }
 
 template <int BN, bool INT8, int ACT, int OUTK>
@@ -263,44 +384,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-7)
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
-    const int quarter = warp & 3, chalf = warp >> 2;
-    constexpr int CH = BN / 2;                 // columns per thread and tile
-    const int tid_e = threadIdx.x;             // 0..255
-    int it = 0; bool ok = true;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
-      int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
-      const int as = it & 1;
-      const uint32_t aphase = (it >> 1) & 1;
-      const int n0 = nt * BN;
-      float* e_cs = epi + (it & 1) * 3 * BN;
-      float* e_bias = e_cs + BN;
-      float* e_post = e_bias + BN;
-      if constexpr (OUTK != OUT_I32) {
-        for (int j = tid_e; j < BN; j += 256) {
-          const int n = n0 + j;
-          const bool in = n < p.N;
-          e_cs[j] = (in && p.cs) ? p.cs[n] : 1.0f;
-          e_bias[j] = (in && p.bias) ? p.bias[n] : 0.0f;
-          e_post[j] = (in && p.post) ? p.post[n] : 1.0f;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-      }
-      const int m = mt * GEMM_BM + quarter * 32 + lane;
-      const bool row_ok = m < p.M;
-      float rs = 1.0f;
-      if (OUTK != OUT_I32 && INT8 && p.rs && row_ok) rs = p.rs[m];
-
-      if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
-      ptx::tc_fence_after();
-      if (ok) {
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
-        epilogue_columns<BN, INT8, ACT, OUTK>(p, e_cs, e_bias, e_post, taddr, m, row_ok, rs, n0, chalf);
-      }
-      // hand the accumulator buffer back to the MMA warp
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&acc_empty[as]);
-    }
+    epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0);
   }
 
   ptx::tc_fence_before();
@@ -475,43 +559,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-7 of each CTA)
-    const int quarter = warp & 3, chalf = warp >> 2;
-    constexpr int CH = BN / 2;
-    const int tid_e = threadIdx.x;
-    int it = 0; bool ok = true;
-    for (int t = pair_id; t < num_tiles; t += num_pairs, ++it) {
-      int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
-      const int as = it & 1;
-      const uint32_t aphase = (it >> 1) & 1;
-      const int n0 = nt * BN;
-      float* e_cs = epi + (it & 1) * 3 * BN;
-      float* e_bias = e_cs + BN;
-      float* e_post = e_bias + BN;
-      if constexpr (OUTK != OUT_I32) {
-        for (int j = tid_e; j < BN; j += 256) {
-          const int n = n0 + j;
-          const bool in = n < p.N;
-          e_cs[j] = (in && p.cs) ? p.cs[n] : 1.0f;
-          e_bias[j] = (in && p.bias) ? p.bias[n] : 0.0f;
-          e_post[j] = (in && p.post) ? p.post[n] : 1.0f;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-      }
-      const int m = mt * 256 + (int)rank * GEMM_BM + quarter * 32 + lane;
-      const bool row_ok = m < p.M;
-      float rs = 1.0f;
-      if (OUTK != OUT_I32 && INT8 && p.rs && row_ok) rs = p.rs[m];
-
-      if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0xa00 | as)) ok = false;
-      ptx::tc_fence_after();
-      if (ok) {
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
-        epilogue_columns<BN, INT8, ACT, OUTK>(p, e_cs, e_bias, e_post, taddr, m, row_ok, rs, n0, chalf);
-      }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&acc_empty[as]), 0));
-    }
+    epilogue_loop<BN, INT8, ACT, OUTK, 256, true>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM);
   }
 
   ptx::tc_fence_before();

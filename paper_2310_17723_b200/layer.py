@@ -16,7 +16,7 @@ def _up(a, dtype=None):
 
 
 class Layer:
-    def __init__(self, handle, L):
+    def __init__(self, handle, L, workspace=None):
         cfg = L["cfg"]
         C = L["C"]
         self.h, self.cfg = handle, cfg
@@ -52,7 +52,10 @@ class Layer:
             setattr(d, name, lp)
         self.desc = d
         self.workspace_bytes = handle.hero_layer_workspace_bytes(d, cfg.M)
-        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device="cuda")
+        if workspace is not None and workspace.numel() >= self.workspace_bytes:
+            self.workspace = workspace            # layers of a stack run one after another and can share scratch
+        else:
+            self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device="cuda")
 
     def forward(self, x_in, out, pending=None, stream=None):
         """x_in / out / pending are hero.Tensor structs; runs the whole layer on the current stream."""

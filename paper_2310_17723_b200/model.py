@@ -25,14 +25,17 @@ class Stack:
         x_cal = workloads.activations(shape, config_id, n_seq=n_cal_seq, tensor=7).astype(np.float64)
         self.layers, self.params = [], []
         cur = None
+        ws = None
         for li, cfg in enumerate(layer_cfgs):
             p = workloads.layer_params(shape, config_id * 100 + li, unit_ln=unit_ln)
             if li == 0:
                 self.ln0 = (p["ln0_g"], p["ln0_b"])
                 cur = _ln_np(x_cal, p["ln0_g"].astype(np.float64), p["ln0_b"].astype(np.float64), cfg.eps) if post else x_cal
             C, cur = prep.calibrate(cfg, p, cur, n_cal_seq, return_output=True)
-            self.layers.append(Layer(handle, prep.prepare_layer(cfg, p, C)))
-            self.params.append((p, C))
+            layer = Layer(handle, prep.prepare_layer(cfg, p, C), workspace=ws)
+            ws = layer.workspace
+            self.layers.append(layer)
+            self.params.append((None, C))
         # chained activation buffers: input of layer 0 .. output of the last layer
         self.bufs = []
         for li in range(len(layer_cfgs) + 1):
