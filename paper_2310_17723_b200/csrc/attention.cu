@@ -388,7 +388,11 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
   return HERO_OK;
 }
 
+int g_attn_resident = 1;
+
 }  // namespace hero
+
+extern "C" void hero_debug_attn_resident(int on) { hero::g_attn_resident = on; }
 
 extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream) {
   using namespace hero;
@@ -429,6 +433,7 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
+  if (g_attn_resident && a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory
   if (a->dh == 64) return launch_attn<64>(h, a, p, s);
   return launch_attn<128>(h, a, p, s);
 }

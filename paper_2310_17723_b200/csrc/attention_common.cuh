@@ -88,5 +88,8 @@ __device__ __forceinline__ int attn_nkv(const AttnParams& p, int qt, int b, int&
 
 // FP16 / BF16 attention for a module left in FP mode (Table 1); defined in attention_fp.cu
 hero_status attn_fp_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
+// INT8 core with the whole score row resident in tensor memory (S <= 512); defined in attention_resident.cu
+hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
+extern int g_attn_resident;   // experiment switch
 
 }  // namespace hero

@@ -1,0 +1,138 @@
+"""Single-kernel micro-benchmarks of the library (also the small cases its ncu captures are taken on).
+
+    python -m paper_2310_17723_b200.microbench ln   --M 65536 --H 1024 --kind i8       # LN^quant GB/s
+    python -m paper_2310_17723_b200.microbench gemm --M 8192 --K 4096 --N 4096        # GeMM^quant TOP/s
+    python -m paper_2310_17723_b200.microbench attn --B 8 --S 384 --nh 16 --dh 64     # INT8 attention
+    ... --sweep runs the standalone-kernel sweep of the benchmark configurations instead of one shape.
+
+Inputs are synthetic and larger than L2 (several rotating buffers), times are CUDA events around `--iters` launches.
+"""
+import argparse
+import json
+import os
+
+import torch
+
+from . import hero, workloads as W
+
+
+def _peaks():
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d["hbm_gbs"], 2.0 * d["bf16_tflops"], "measured"
+    return 6650.0, 2.0 * 1590.0, "fallback"
+
+
+def _time(fn, n_buf, iters):
+    for i in range(n_buf):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for k in range(iters):
+        fn(k % n_buf)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e-3
+
+
+def bench_ln(h, M, H, kind, iters):
+    """kind 'f16': FP16 -> INT8 TWQ (entry flavour); 'i8': INT8 TWQ + INT8 FWQ -> INT8 TWQ (Eq. 19)."""
+    n = max(2, min(32, int(400e6 // (M * H * 3)) + 1))
+    g, b = torch.ones(H, device="cuda"), torch.zeros(H, device="cuda")
+    sc = torch.empty(M, device="cuda")
+    outs = [torch.empty(M, H, device="cuda", dtype=torch.int8) for _ in range(n)]
+    if kind == "f16":
+        xs = [torch.randn(M, H, device="cuda", dtype=torch.float16) for _ in range(n)]
+        ins = [(hero.tensor(x), None) for x in xs]
+    else:
+        rs, cs = torch.rand(M, device="cuda") * 0.01 + 0.01, torch.rand(H, device="cuda") * 0.01 + 0.01
+        xs = [torch.randint(-127, 128, (M, H), device="cuda", dtype=torch.int8) for _ in range(n)]
+        ys = [torch.randint(-127, 128, (M, H), device="cuda", dtype=torch.int8) for _ in range(n)]
+        ins = [(hero.tensor(x, "twq", rs), hero.tensor(y, "fwq", cs)) for x, y in zip(xs, ys)]
+    t = _time(lambda i: h.hero_layernorm_quant(ins[i][0], g, b, 1e-5, hero.tensor(outs[i], "twq", sc), branch=ins[i][1]), n, iters)
+    hbm, _, src = _peaks()
+    gbs = M * H * 3 / t / 1e9
+    print("LN^quant %s M=%d H=%d: %.1f us, %.0f GB/s (algorithmic 3 B/element), %.2f of %s copy bandwidth"
+          % (kind, M, H, t * 1e6, gbs, gbs / hbm, src), flush=True)
+
+
+def bench_gemm(h, M, K, N, act, fp, iters):
+    dt = torch.bfloat16 if fp else torch.int8
+    n = max(2, min(8, int(300e6 // (M * K + N * K + M * N)) + 1))
+    if fp:
+        As = [torch.randn(M, K, device="cuda", dtype=dt) for _ in range(n)]
+        Ws = [torch.randn(N, K, device="cuda", dtype=dt) for _ in range(n)]
+    else:
+        As = [torch.randint(-127, 128, (M, K), device="cuda", dtype=dt) for _ in range(n)]
+        Ws = [torch.randint(-127, 128, (N, K), device="cuda", dtype=dt) for _ in range(n)]
+    outs = [torch.empty(M, N, device="cuda", dtype=dt) for _ in range(n)]
+    rs, cs = torch.rand(M, device="cuda") * 1e-3, torch.rand(N, device="cuda") * 1e-3
+    bias = torch.randn(N, device="cuda")
+
+    def run(i):
+        a = hero.tensor(As[i]) if fp else hero.tensor(As[i], "twq", rs)
+        h.hero_w8a8_linear(a, Ws[i], hero.tensor(outs[i]), w_scale=None if fp else cs, bias=bias, act=act)
+    t = _time(run, n, iters)
+    _, i8peak, src = _peaks()
+    peak = i8peak / 2 if fp else i8peak
+    tops = 2.0 * M * N * K / t / 1e12
+    print("GeMM^quant %s M=%d K=%d N=%d act=%s: %.1f us, %.0f TOP/s, %.2f of 2 x %s BF16 peak%s"
+          % ("bf16" if fp else "i8", M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else ""), flush=True)
+
+
+def bench_attn(h, B, S, nh, dh, mask, iters):
+    H = nh * dh
+    qkv = (torch.randn(B * S, 3 * H, device="cuda") * 40).clamp(-127, 127).to(torch.int8)
+    out = torch.empty(B * S, H, device="cuda", dtype=torch.int8)
+    sc = torch.full((H,), 0.02, device="cuda")
+    s = (1.5 ** 0.5) / 40
+    t = _time(lambda i: h.hero_int8_attention(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh,
+                                              hero.tensor(out, "fwq", sc), s_q=s, s_k=s, s_v=0.02, s_p=1 / 255, mask=mask), 1, iters)
+    scores = B * nh * S * S * (0.5 if mask == "causal" else 1.0)
+    print("INT8 attention B=%d S=%d nh=%d dh=%d %s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
+          % (B, S, nh, dh, mask, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("kernel", choices=["ln", "gemm", "attn"])
+    ap.add_argument("--M", type=int, default=65536)
+    ap.add_argument("--H", type=int, default=1024)
+    ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--N", type=int, default=4096)
+    ap.add_argument("--B", type=int, default=8)
+    ap.add_argument("--S", type=int, default=384)
+    ap.add_argument("--nh", type=int, default=16)
+    ap.add_argument("--dh", type=int, default=64)
+    ap.add_argument("--kind", default="i8", choices=["i8", "f16"])
+    ap.add_argument("--act", default="none")
+    ap.add_argument("--mask", default="none")
+    ap.add_argument("--fp", action="store_true")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--sweep", action="store_true")
+    a = ap.parse_args()
+    h = hero.Handle()
+    if a.kernel == "ln":
+        if a.sweep:
+            for H in W.LN_SWEEP_H:
+                for M in W.LN_SWEEP_M:
+                    bench_ln(h, M, H, a.kind, a.iters)
+        else:
+            bench_ln(h, a.M, a.H, a.kind, a.iters)
+    elif a.kernel == "gemm":
+        if a.sweep:
+            for K, N in W.GEMM_SWEEP_KN:
+                for M in W.GEMM_SWEEP_M:
+                    bench_gemm(h, M, K, N, a.act, a.fp, a.iters)
+        else:
+            bench_gemm(h, a.M, a.K, a.N, a.act, a.fp, a.iters)
+    else:
+        bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters)
+    h.check()
+
+
+if __name__ == "__main__":
+    main()
