@@ -1,16 +1,30 @@
 // INT8 attention core (Sec. 2.2.2 Eq. 15-17) for sequences of at most 512 keys: the whole score row lives in
 // tensor memory.  Q K^T is issued once for all (up to four) 128-key blocks into the 512 TMEM columns; the softmax
 // warps turn each 32-column piece into e = 2^(t - m_piece) with the piece's own maximum, write e back over the
-// scores and keep (m_piece, sum) in registers; once the row maximum and sum are known every piece is re-read,
-// scaled by 2^(m_piece - m) / (l s_p) -- one multiply, no second exponential -- rounded to P_u8 and stored as the
-// UMMA operand of P V.  One exponential per score instead of two, no second Q K^T pass, K loaded once.  The output
-// accumulator aliases the first score block's columns: P V for block 0 is issued only after every warp has consumed
-// that block.
+// scores and keep a running (max, sum); once the row maximum and sum are known every piece is re-read, scaled by
+// 2^(m_piece - m) / (l s_p) -- one multiply, no second exponential -- rounded to P_u8 and stored as the UMMA operand
+// of P V.  One exponential per score instead of two, no second Q K^T pass, K loaded once.
+//
+// The output accumulator occupies the columns of score block 3 (columns 384 ..).  With at most three key blocks it
+// is a buffer of its own.  With four, block 3 is converted to P first (the P V order is 3, 0, 1, 2), so its columns
+// are free when the first P V lands there, and the next tile's Q K^T for block 3 waits until the previous output
+// has been read.  The epilogue of tile t runs inside tile t+1, after the first three score blocks of t+1 have been
+// exponentiated: P V of tile t finishes in the shadow of that work.
 #include "attention_common.cuh"
 
 namespace hero {
 
-constexpr int RES_NB = 4;    // score blocks resident in TMEM (4 x 128 columns)
+#ifdef HERO_ATTN_PHASES
+#define PH(i) do { if (dbgon) { const long long c_ = clock64(); ph[i] += c_ - tprev; tprev = c_; } } while (0)
+#else
+#define PH(i) do {} while (0)
+#endif
+
+constexpr int RES_NB = 4;          // score blocks resident in TMEM (4 x 128 columns)
+constexpr int RES_O_COL = 384;     // output accumulator columns
+
+// the j-th block in P V order
+__device__ __forceinline__ int res_pv_block(int nkv, int i) { return nkv == RES_NB ? ((i + 3) & 3) : i; }
 
 template <int DH>
 struct AttnResCfg {
@@ -22,7 +36,9 @@ struct AttnResCfg {
   static constexpr int OFF_V = OFF_K + KST * TILE;
   static constexpr int OFF_P = OFF_V + VST * TILE;
   static constexpr int OFF_STATS = OFF_P + 2 * P_TILE;
-  static constexpr int OFF_BARS = OFF_STATS + 2 * 4 * ATT_BM * 8;
+  static constexpr int OFF_PM = OFF_STATS + 2 * 4 * ATT_BM * 8;        // per-thread piece maxima [RES_NB][512] x 2 halves
+  static constexpr int OFF_OSC = OFF_PM + RES_NB * 512 * 8;            // per-tile output factors [2][128]
+  static constexpr int OFF_BARS = OFF_OSC + 2 * 128 * 4;
   static constexpr int NBARS = 4 + 2 * KST + 2 * VST + 2 * RES_NB + 4 + 2;
   static constexpr int SMEM_BYTES = 1024 + OFF_BARS + NBARS * 8 + 16;
   static constexpr uint32_t SWZ = (DH == 128) ? ptx::SWZ_128B : ptx::SWZ_64B;
@@ -30,10 +46,68 @@ struct AttnResCfg {
   static constexpr int TMEM_COLS = 512;
 };
 
+// X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8) for the tile whose P V has been issued; frees the accumulator
+// columns.  Every softmax warp takes DH / 4 columns of its 32 rows; `osc` is the tile's per-column factor
+// s_p s_v / S_attn[j] (s_p s_v alone for an FP output) staged in shared memory.  Kept out of line: it runs once per
+// tile and its registers stay out of the sweeps' allocation.
+template <int DH>
+__device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, uint64_t* o_full, uint64_t* o_empty,
+                                          uint32_t parity, int cq, int lane, long long pend_row, int pend_col,
+                                          const float* osc, bool& ok) {
+  constexpr int CW = DH / 4;
+  uint32_t r[CW];
+  if (ok && !ptx::mbar_wait(o_full, parity, p.err, 0x9300)) ok = false;
+  ptx::tc_fence_after();
+  if (ok) {
+    if constexpr (CW == 16) ptx::tmem_ld16(t_lane + RES_O_COL + cq * CW, r);
+    else ptx::tmem_ld32(t_lane + RES_O_COL + cq * CW, r);
+    ptx::tmem_ld_wait();
+  }
+  ptx::tc_fence_before();
+  __syncwarp();
+  if (lane == 0) ptx::mbar_arrive(o_empty);
+  if (!ok) {
+#pragma unroll
+    for (int e = 0; e < CW; ++e) r[e] = 0;
+  }
+  if (pend_row >= 0) {
+    const int gcol = pend_col + cq * CW;
+    const float4* o4 = reinterpret_cast<const float4*>(osc + cq * CW);
+    if (p.out_dt == HERO_I8) {
+      int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pend_row * p.out_ld + gcol;
+#pragma unroll
+      for (int g = 0; g < CW / 16; ++g) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float4 sc = o4[4 * g + k];
+          const int c = 16 * g + 4 * k;
+          const float a = fminf(fmaxf((float)(int)r[c] * sc.x, -127.f), 127.f) + ATT_MAGIC;
+          const float b = fminf(fmaxf((float)(int)r[c + 1] * sc.y, -127.f), 127.f) + ATT_MAGIC;
+          const float cc = fminf(fmaxf((float)(int)r[c + 2] * sc.z, -127.f), 127.f) + ATT_MAGIC;
+          const float d = fminf(fmaxf((float)(int)r[c + 3] * sc.w, -127.f), 127.f) + ATT_MAGIC;
+          w[k] = low_bytes4_u(a, b, cc, d);                  // low byte of magic + x = two's-complement Round(x)
+        }
+        st_g16(dst + 16 * g, w[0], w[1], w[2], w[3]);
+      }
+    } else {
+      uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + pend_row * p.out_ld + gcol;
+#pragma unroll
+      for (int g = 0; g < CW / 8; ++g) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * p.pv_scale;
+        st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
+               fp2(v[6], v[7], p.out_dt));
+      }
+    }
+  }
+}
+
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                          const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+                          const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnParams p) {
   using Cfg = AttnResCfg<DH>;
   constexpr int KST = Cfg::KST, VST = Cfg::VST;
   extern __shared__ uint8_t smem_raw[];
@@ -43,6 +117,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   uint8_t* sV = smem + Cfg::OFF_V;
   uint8_t* sP = smem + Cfg::OFF_P;
   float2* stats = reinterpret_cast<float2*>(smem + Cfg::OFF_STATS);
+  float2* pm2 = reinterpret_cast<float2*>(smem + Cfg::OFF_PM) + (threadIdx.x & 511);
+  float* osc_s = reinterpret_cast<float*>(smem + Cfg::OFF_OSC);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::OFF_BARS);
   uint64_t* q_full = bars;                      // [2]
   uint64_t* q_empty = q_full + 2;               // [2]
@@ -80,7 +156,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == ATT_TMA_WARP) {
-    // ------------------------------------------------------------------ TMA producer: Q, every K block, every V block
+    // ------------------------------------------------------------------ TMA producer: Q, K blocks, V blocks in P V order
     if (lane == 0) {
       uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
       bool ok = true;
@@ -99,7 +175,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
           ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
         }
-        for (int j = 0; j < nkv && ok; ++j, ++vcnt) {
+        for (int i = 0; i < nkv && ok; ++i, ++vcnt) {
+          const int j = res_pv_block(nkv, i);
           const int vs = vcnt % VST;
           if (!ptx::mbar_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x7200 | vs)) { ok = false; break; }
           ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
@@ -116,7 +193,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       constexpr uint64_t pmaj = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
       constexpr uint64_t vmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);
       uint32_t kcnt = 0, vcnt = 0, pcnt = 0, wcnt = 0;
-      uint32_t used[RES_NB] = {0, 0, 0, 0};               // how often each score block has been filled so far
+      uint32_t used = 0;                                  // bit j: parity of how often score block j has been filled
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         int qt, h, b, klen; attn_tile(p, t, qt, h, b);
@@ -125,39 +202,42 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         const int qb = wcnt & 1;
         if (!ptx::mbar_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x8000 | qb)) { ok = false; break; }
         const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
-        // the output accumulator of the previous tile sits in block 0's columns: it must have been read out
-        if (!ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x8500)) { ok = false; break; }
-#pragma unroll
-        for (int j = 0; j < RES_NB; ++j) {
-          if (j < nkv && ok) {
-            const int ks = kcnt % KST;
-            if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8300 | ks)) { ok = false; }
-            if (ok && !ptx::mbar_wait(&s_free[j], (used[j] & 1) ^ 1, p.err, 0x8400 | j)) { ok = false; }
-            if (ok) {
-              ptx::tc_fence_after();
-              const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
-#pragma unroll
-              for (int k = 0; k < DH / 32; ++k)
-                ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                             ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
-              ptx::umma_commit(&k_empty[ks]);
-              ptx::umma_commit(&s_full[j]);
-              ++kcnt; ++used[j];
-            }
+        bool o_free = false;                              // previous tile's output read out of columns 384 ..
+#pragma unroll 1
+        for (int j = 0; j < nkv && ok; ++j) {
+          const int ks = kcnt % KST;
+          if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8300 | ks)) { ok = false; break; }
+          if (!ptx::mbar_wait(&s_free[j], ((used >> j) & 1) ^ 1, p.err, 0x8400 | j)) { ok = false; break; }
+          if (j == 3) {
+            if (!ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x8500)) { ok = false; break; }
+            o_free = true;
           }
+          ptx::tc_fence_after();
+          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+#pragma unroll
+          for (int k = 0; k < DH / 32; ++k)
+            ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                         ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+          ptx::umma_commit(&k_empty[ks]);
+          ptx::umma_commit(&s_full[j]);
+          ++kcnt; used ^= 1u << j;
         }
         if (ok) ptx::umma_commit(&q_empty[qb]);
-        for (int j = 0; j < nkv && ok; ++j) {
+        for (int i = 0; i < nkv && ok; ++i) {
           const int vs = vcnt % VST, pb = pcnt & 1;
           if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x8100 | vs)) { ok = false; break; }
           if (!ptx::mbar_wait(&p_full[pb], (pcnt >> 1) & 1, p.err, 0x8200 | pb)) { ok = false; break; }
+          if (!o_free) {
+            if (!ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x8600)) { ok = false; break; }
+            o_free = true;
+          }
           ptx::tc_fence_after();
           const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
           const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
 #pragma unroll
           for (int k = 0; k < ATT_BN / 32; ++k)
-            ptx::umma_i8(tmem_base, ptx::smem_desc(pmaj, p_addr + k * 32), ptx::smem_desc(vmaj, v_addr + k * 32 * DH),
-                         p.idesc_pv, (j | k) != 0);
+            ptx::umma_i8(tmem_base + RES_O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
+                         ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
           ptx::umma_commit(&v_empty[vs]);
           ptx::umma_commit(&p_empty[pb]);
           ++vcnt; ++pcnt;
@@ -173,9 +253,22 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     const int r_loc = quarter * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const float c2 = p.c2;
-    uint32_t pcnt = 0, wcnt = 0;
-    uint32_t used[RES_NB] = {0, 0, 0, 0};
+    uint32_t pcnt = 0, wcnt = 0, used = 0;
     bool ok = true;
+#ifdef HERO_ATTN_PHASES
+    const bool dbgon = p.dbg != nullptr && lane == 0;
+    long long ph[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    long long tprev = clock64();
+#endif
+    long long pend_row = -1;                                 // output row of the tile whose epilogue is pending
+    int pend_col = 0;
+    bool pend = false;
+
+    auto epilogue = [&]() {
+      res_epilogue<DH>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
+                       osc_s + ((wcnt - 1) & 1) * 128, ok);
+      pend = false;
+    };
 
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
       int qt, h, b, klen; attn_tile(p, t, qt, h, b);
@@ -183,63 +276,88 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       const int q0 = qt * ATT_BM, row_base = b * p.S, col0 = h * DH;
       const int q = q0 + r_loc;
       const bool row_ok = q < p.S;
+      if (nkv == 0) {
+        // every key masked: the rows are zero, no tensor work
+        if (cq * 32 < DH && row_ok) {
+          const long long grow = (long long)(row_base + q);
+          const int gcol = col0 + cq * 32;
+          const int es = p.out_dt == HERO_I8 ? 1 : 2;
+          uint8_t* dst = reinterpret_cast<uint8_t*>(p.out) + (grow * p.out_ld + gcol) * es;
+          for (int g = 0; g < 2 * es; ++g) st_g16(dst + 16 * g, 0u, 0u, 0u, 0u);
+        }
+        continue;
+      }
       int kmax = klen - 1;
       if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
 
-      // ---- sweep 1: per piece, e = 2^(t - m_piece) written back over the scores; (m_piece, sum) kept
-      float mj[RES_NB], lj[RES_NB];
+      // ---- sweep 1: per piece, e = 2^(t - m_piece) written back over the scores; running (m, l) in registers
+      float m = -INFINITY, l = 0.f;
+#pragma unroll 1
+      for (int j = 0; j < nkv; ++j) {
+        if (j == 3 && pend) epilogue();                      // block 3's columns hold the previous tile's output
+        PH(10);
+        if (ok && !ptx::mbar_wait(&s_full[j], (used >> j) & 1, p.err, 0x9000 | j)) ok = false;
+        ptx::tc_fence_after();
+        PH(0);
+        if (ok) {
+          const uint32_t ta = t_lane + j * ATT_BN + cq * 32;
+          const int kb = j * ATT_BN + cq * 32;
+          float mpa[2];
 #pragma unroll
-      for (int j = 0; j < RES_NB; ++j) {
-        mj[j] = -INFINITY; lj[j] = 0.f;
-        if (j < nkv) {
-          if (ok && !ptx::mbar_wait(&s_full[j], used[j] & 1, p.err, 0x9000 | j)) ok = false;
-          ptx::tc_fence_after();
-          if (ok) {
-            uint32_t r[32];
-            const uint32_t ta = t_lane + j * ATT_BN + cq * 32;
-            ptx::tmem_ld32(ta, r);
+          for (int hh = 0; hh < 2; ++hh) {                   // two 16-column pieces, each with its own maximum
+            uint32_t r[16];
+            ptx::tmem_ld16(ta + 16 * hh, r);
             ptx::tmem_ld_wait();
-            const int kb = j * ATT_BN + cq * 32;
-            const int nvalid = min(32, kmax - kb + 1);
+            PH(1);
+            const int nvalid = min(16, kmax - (kb + 16 * hh) + 1);
+            float mp = -INFINITY;
             if (nvalid > 0) {
-              int imax = INT_MIN;
-              if (nvalid == 32) {
+              if (nvalid < 16) {
+                // masked keys: a score far below every real one (|t| < 2^21) turns into e = 0 by itself
 #pragma unroll
-                for (int e = 0; e < 32; ++e) imax = max(imax, (int)r[e]);
-              } else {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) imax = max(imax, e < nvalid ? (int)r[e] : INT_MIN);
+                for (int e = 0; e < 16; ++e) if (e >= nvalid) r[e] = (uint32_t)(-(1 << 21));
               }
-              const float m = (float)imax * c2;
-              float2 acc2 = make_float2(0.f, 0.f);
-              const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m, -m), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
+              int i0 = max((int)r[0], (int)r[1]), i1 = max((int)r[2], (int)r[3]);
 #pragma unroll
-              for (int e = 0; e < 32; e += 2) {
+              for (int e = 4; e < 16; e += 4) { i0 = max(i0, max((int)r[e], (int)r[e + 1])); i1 = max(i1, max((int)r[e + 2], (int)r[e + 3])); }
+              mp = (float)max(i0, i1) * c2;
+              float2 acc2 = make_float2(0.f, 0.f);
+              const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-mp, -mp), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
+#pragma unroll
+              for (int e = 0; e < 16; e += 2) {
                 const float2 f = __fadd2_rn(make_float2(__uint_as_float(0x4B400000u + r[e]), __uint_as_float(0x4B400000u + r[e + 1])), mg);
                 const float2 tt = __ffma2_rn(f, c22, nm2);
-                float2 ev = make_float2(ex2f(tt.x), ex2f(tt.y));
-                if (nvalid < 32) { if (e >= nvalid) ev.x = 0.f; if (e + 1 >= nvalid) ev.y = 0.f; }
+                const float2 ev = make_float2(ex2f(tt.x), ex2f(tt.y));
                 acc2 = __fadd2_rn(acc2, ev);
                 r[e] = __float_as_uint(ev.x); r[e + 1] = __float_as_uint(ev.y);
               }
-              mj[j] = m; lj[j] = acc2.x + acc2.y;
+              const float mn = fmaxf(m, mp);
+              l = l * ex2f(m - mn) + (acc2.x + acc2.y) * ex2f(mp - mn);
+              m = mn;
             } else {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) r[e] = 0;         // every key of the piece masked
+              for (int e = 0; e < 16; ++e) r[e] = 0;         // every key of the piece masked
             }
-            ptx::tmem_st32(ta, r);
+            PH(2);
+            ptx::tmem_st16(ta + 16 * hh, r);
+            mpa[hh] = mp;
           }
+          pm2[j * 512] = make_float2(mpa[0], mpa[1]);
+        } else {
+          pm2[j * 512] = make_float2(-INFINITY, -INFINITY);
         }
+        PH(3);
       }
       if (ok) ptx::tmem_st_wait();
-      // ---- row maximum and sum: first over this thread's pieces, then across the four column groups
-      float m = -INFINITY, l = 0.f;
-#pragma unroll
-      for (int j = 0; j < RES_NB; ++j) m = fmaxf(m, mj[j]);
-#pragma unroll
-      for (int j = 0; j < RES_NB; ++j) if (mj[j] > -INFINITY) l += lj[j] * ex2f(mj[j] - m);
+      PH(3);
+      if (pend) epilogue();
+      PH(4);
+      // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
       st[cq * ATT_BM + r_loc] = make_float2(m, l);
+      if (p.out_dt == HERO_I8 && (int)threadIdx.x < DH)
+        osc_s[(wcnt & 1) * 128 + threadIdx.x] =
+            p.pv_scale / __ldg(p.out_scale + (long long)(col0 + (int)threadIdx.x) * p.out_scale_stride);
       asm volatile("bar.sync 1, 512;" ::: "memory");
       {
         float mf = -INFINITY;
@@ -256,88 +374,60 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         m = mf; l = lf;
       }
       const float pscale = l > 0.f ? p.inv_sp / l : 0.f;
+      PH(5);
 
       // ---- sweep 2: P_u8 = Round(e * 2^(m_piece - m) / (l s_p)), clipped to 255, into the UMMA operand tile
+#pragma unroll 1
+      for (int i = 0; i < nkv; ++i) {
+        const int j = res_pv_block(nkv, i);
+        const int pb = pcnt & 1;
+        if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt >> 1) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
+        PH(6);
+        if (ok) {
+          const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
+          const float2 mp2 = pm2[j * 512];
+          const int c16 = cq * 2;
 #pragma unroll
-      for (int j = 0; j < RES_NB; ++j) {
-        if (j < nkv) {
-          const int pb = pcnt & 1;
-          if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt >> 1) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
-          if (ok) {
-            const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
-            uint32_t r[32];
-            ptx::tmem_ld32(t_lane + j * ATT_BN + cq * 32, r);
+          for (int g = 0; g < 2; ++g) {
+            uint32_t r[16];
+            ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32 + 16 * g, r);
             ptx::tmem_ld_wait();
-            const float f = mj[j] > -INFINITY ? ex2f(mj[j] - m) * pscale : 0.f;
+            PH(7);
+            const float mp = g ? mp2.y : mp2.x;
+            const float f = mp > -INFINITY ? ex2f(mp - m) * pscale : 0.f;
             const float2 f2v = make_float2(f, f), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
-            float y[32];
+            uint32_t w[4];
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              const float2 v = __ffma2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), f2v, rm2);
-              y[e] = fminf(v.x, ATT_MAGIC + 255.0f);
-              y[e + 1] = fminf(v.y, ATT_MAGIC + 255.0f);
+            for (int k = 0; k < 4; ++k) {
+              const int e = 4 * k;
+              const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), f2v, rm2);
+              const float2 c = __ffma2_rn(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])), f2v, rm2);
+              w[k] = low_bytes4_u(fminf(a.x, ATT_MAGIC + 255.0f), fminf(a.y, ATT_MAGIC + 255.0f),
+                                  fminf(c.x, ATT_MAGIC + 255.0f), fminf(c.y, ATT_MAGIC + 255.0f));
             }
-            const int c16 = cq * 2;
-            st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), low_bytes4_u(y[0], y[1], y[2], y[3]), low_bytes4_u(y[4], y[5], y[6], y[7]),
-                        low_bytes4_u(y[8], y[9], y[10], y[11]), low_bytes4_u(y[12], y[13], y[14], y[15]));
-            st_shared16(prow + (((c16 + 1) ^ (r_loc & 7)) << 4), low_bytes4_u(y[16], y[17], y[18], y[19]),
-                        low_bytes4_u(y[20], y[21], y[22], y[23]), low_bytes4_u(y[24], y[25], y[26], y[27]),
-                        low_bytes4_u(y[28], y[29], y[30], y[31]));
+            st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
           }
-          ptx::tc_fence_before();
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) { ptx::mbar_arrive(&s_free[j]); ptx::mbar_arrive(&p_full[pb]); }
-          ++pcnt; ++used[j];
         }
-      }
-
-      // ---- epilogue: X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8); the accumulator sits in columns 0 .. DH-1
-      uint32_t r[32];
-      if (nkv > 0) {
-        if (ok && !ptx::mbar_wait(o_full, wcnt & 1, p.err, 0x9300)) ok = false;
-        ptx::tc_fence_after();
-        if (ok && cq * 32 < DH) {
-          ptx::tmem_ld32(t_lane + cq * 32, r);
-          ptx::tmem_ld_wait();
-        }
+        PH(8);
         ptx::tc_fence_before();
+        ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(o_empty);
-        ++wcnt;
+        if (lane == 0) { ptx::mbar_arrive(&s_free[j]); ptx::mbar_arrive(&p_full[pb]); }
+        PH(9);
+        ++pcnt; used ^= 1u << j;
       }
-      if (nkv == 0 || !ok) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) r[e] = 0;
-      }
-      if (cq * 32 < DH && row_ok) {
-        const long long grow = (long long)(row_base + q);
-        const int gcol = col0 + cq * 32;
-        if (p.out_dt == HERO_I8) {
-          float v[32];
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            v[e] = (float)(int)r[e] * (p.pv_scale / __ldg(p.out_scale + (gcol + e) * p.out_scale_stride));
-          int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
-#pragma unroll
-          for (int g = 0; g < 2; ++g)
-            st_g16(dst + 16 * g, q4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
-                   q4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
-                   q4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
-                   q4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
-        } else {
-          uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + grow * p.out_ld + gcol;
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * p.pv_scale;
-            st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
-                   fp2(v[6], v[7], p.out_dt));
-          }
-        }
-      }
+      pend = true;
+      pend_row = row_ok ? (long long)(row_base + q) : -1;
+      pend_col = col0;
+      ++wcnt;
     }
+    if (pend) epilogue();
+    PH(4);
+#ifdef HERO_ATTN_PHASES
+    if (dbgon && blockIdx.x == 0) {
+      for (int i = 0; i < 12; ++i) p.dbg[warp * 12 + i] = ph[i];
+    }
+#endif
   }
 
   ptx::tc_fence_before();
