@@ -195,34 +195,55 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       uint32_t kcnt = 0, vcnt = 0, pcnt = 0, wcnt = 0;
       uint32_t used = 0;                                  // bit j: parity of how often score block j has been filled
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        int qt, h, b, klen; attn_tile(p, t, qt, h, b);
-        const int nkv = attn_nkv(p, qt, b, klen);
-        if (nkv == 0) continue;
-        const int qb = wcnt & 1;
-        if (!ptx::mbar_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x8000 | qb)) { ok = false; break; }
+
+      // S_j = Q K_j^T of the tile with running index w into score block j.  K stages are consumed in issue order,
+      // which the callers keep equal to the producer's order j = 0, 1, ...
+      auto issue_qk = [&](uint32_t w, int j) {
+        const int qb = w & 1;
+        const int ks = kcnt % KST;
+        if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8300 | ks)) { ok = false; return; }
+        if (!ptx::mbar_wait(&s_free[j], ((used >> j) & 1) ^ 1, p.err, 0x8400 | j)) { ok = false; return; }
+        ptx::tc_fence_after();
         const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
+        const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+#pragma unroll
+        for (int k = 0; k < DH / 32; ++k)
+          ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                       ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+        ptx::umma_commit(&k_empty[ks]);
+        ptx::umma_commit(&s_full[j]);
+        ++kcnt; used ^= 1u << j;
+      };
+      // next tile of this CTA with at least one key block
+      auto next_tile = [&](int t, int& nkv) {
+        for (; t < total_tiles; t += gridDim.x) {
+          int qt, h, b, klen; attn_tile(p, t, qt, h, b);
+          nkv = attn_nkv(p, qt, b, klen);
+          if (nkv > 0) return t;
+        }
+        nkv = 0;
+        return total_tiles;
+      };
+
+      int nkv = 0, nkv_n = 0;
+      int t = next_tile(blockIdx.x, nkv);
+      int issued = 0;                                     // leading score blocks of the current tile already issued
+      bool q_ready = false;                               // q_full of the current tile already awaited
+      while (t < total_tiles && ok) {
+        const int tn = next_tile(t + gridDim.x, nkv_n);
+        const int qb = wcnt & 1;
+        if (!q_ready && !ptx::mbar_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x8000 | qb)) { ok = false; break; }
         bool o_free = false;                              // previous tile's output read out of columns 384 ..
-#pragma unroll 1
-        for (int j = 0; j < nkv && ok; ++j) {
-          const int ks = kcnt % KST;
-          if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8300 | ks)) { ok = false; break; }
-          if (!ptx::mbar_wait(&s_free[j], ((used >> j) & 1) ^ 1, p.err, 0x8400 | j)) { ok = false; break; }
+        for (int j = issued; j < nkv && ok; ++j) {
           if (j == 3) {
             if (!ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x8500)) { ok = false; break; }
             o_free = true;
           }
-          ptx::tc_fence_after();
-          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
-#pragma unroll
-          for (int k = 0; k < DH / 32; ++k)
-            ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                         ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
-          ptx::umma_commit(&k_empty[ks]);
-          ptx::umma_commit(&s_full[j]);
-          ++kcnt; used ^= 1u << j;
+          issue_qk(wcnt, j);
         }
-        if (ok) ptx::umma_commit(&q_empty[qb]);
+        if (!ok) break;
+        ptx::umma_commit(&q_empty[qb]);
+        issued = 0; q_ready = false;
         for (int i = 0; i < nkv && ok; ++i) {
           const int vs = vcnt % VST, pb = pcnt & 1;
           if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x8100 | vs)) { ok = false; break; }
@@ -241,9 +262,21 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           ptx::umma_commit(&v_empty[vs]);
           ptx::umma_commit(&p_empty[pb]);
           ++vcnt; ++pcnt;
+          // the block just converted to P is free: start the next tile's scores there (block 3 holds the output)
+          const int j = res_pv_block(nkv, i);
+          if (j == issued && j < 3 && j < nkv_n) {
+            if (!q_ready) {
+              const uint32_t wn = wcnt + 1;
+              if (!ptx::mbar_wait(&q_full[wn & 1], (wn >> 1) & 1, p.err, 0x8700)) { ok = false; break; }
+              q_ready = true;
+            }
+            issue_qk(wcnt + 1, j);
+            ++issued;
+          }
         }
         if (ok) ptx::umma_commit(o_full);
         ++wcnt;
+        t = tn; nkv = nkv_n;
       }
     }
     __syncwarp();
@@ -303,12 +336,14 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           const uint32_t ta = t_lane + j * ATT_BN + cq * 32;
           const int kb = j * ATT_BN + cq * 32;
           float mpa[2];
+          uint32_t ra[16], rb[16];
+          ptx::tmem_ld16(ta, ra);
+          ptx::tmem_ld16(ta + 16, rb);
+          ptx::tmem_ld_wait();
+          PH(1);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {                   // two 16-column pieces, each with its own maximum
-            uint32_t r[16];
-            ptx::tmem_ld16(ta + 16 * hh, r);
-            ptx::tmem_ld_wait();
-            PH(1);
+            uint32_t (&r)[16] = hh ? rb : ra;
             const int nvalid = min(16, kmax - (kb + 16 * hh) + 1);
             float mp = -INFINITY;
             if (nvalid > 0) {
@@ -387,12 +422,14 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
           const float2 mp2 = pm2[j * 512];
           const int c16 = cq * 2;
+          uint32_t ra[16], rb[16];
+          ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32, ra);
+          ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32 + 16, rb);
+          ptx::tmem_ld_wait();
+          PH(7);
 #pragma unroll
           for (int g = 0; g < 2; ++g) {
-            uint32_t r[16];
-            ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32 + 16 * g, r);
-            ptx::tmem_ld_wait();
-            PH(7);
+            uint32_t (&r)[16] = g ? rb : ra;
             const float mp = g ? mp2.y : mp2.x;
             const float f = mp > -INFINITY ? ex2f(mp - m) * pscale : 0.f;
             const float2 f2v = make_float2(f, f), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
