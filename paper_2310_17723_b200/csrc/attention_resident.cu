@@ -22,6 +22,7 @@ namespace hero {
 
 constexpr int RES_NB = 4;          // score blocks resident in TMEM (4 x 128 columns)
 constexpr int RES_O_COL = 384;     // output accumulator columns
+constexpr int RES_NP = 3;          // P operand tiles in shared memory
 
 // the j-th block in P V order
 __device__ __forceinline__ int res_pv_block(int nkv, int i) { return nkv == RES_NB ? ((i + 3) & 3) : i; }
@@ -35,11 +36,11 @@ struct AttnResCfg {
   static constexpr int OFF_K = 2 * TILE;
   static constexpr int OFF_V = OFF_K + KST * TILE;
   static constexpr int OFF_P = OFF_V + VST * TILE;
-  static constexpr int OFF_STATS = OFF_P + 2 * P_TILE;
+  static constexpr int OFF_STATS = OFF_P + RES_NP * P_TILE;
   static constexpr int OFF_PM = OFF_STATS + 2 * 4 * ATT_BM * 8;        // per-thread piece maxima [RES_NB][512] x 2 halves
   static constexpr int OFF_OSC = OFF_PM + RES_NB * 512 * 8;            // per-tile output factors [2][128]
   static constexpr int OFF_BARS = OFF_OSC + 2 * 128 * 4;
-  static constexpr int NBARS = 4 + 2 * KST + 2 * VST + 2 * RES_NB + 4 + 2;
+  static constexpr int NBARS = 4 + 2 * KST + 2 * VST + 2 * RES_NB + 2 * RES_NP + 2;
   static constexpr int SMEM_BYTES = 1024 + OFF_BARS + NBARS * 8 + 16;
   static constexpr uint32_t SWZ = (DH == 128) ? ptx::SWZ_128B : ptx::SWZ_64B;
   static constexpr uint32_t SBO = 8 * DH;
@@ -128,9 +129,9 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   uint64_t* v_empty = v_full + VST;             // [VST]
   uint64_t* s_full = v_empty + VST;             // [RES_NB]  scores of block j written
   uint64_t* s_free = s_full + RES_NB;           // [RES_NB]  block j consumed by every softmax warp
-  uint64_t* p_full = s_free + RES_NB;           // [2]
-  uint64_t* p_empty = p_full + 2;               // [2]
-  uint64_t* o_full = p_empty + 2;               // [1]
+  uint64_t* p_full = s_free + RES_NB;           // [RES_NP]
+  uint64_t* p_empty = p_full + RES_NP;          // [RES_NP]
+  uint64_t* o_full = p_empty + RES_NP;          // [1]
   uint64_t* o_empty = o_full + 1;               // [1]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
 
@@ -138,10 +139,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   const int total_tiles = p.nqt * p.nh * p.B;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(&q_full[i], 1); ptx::mbar_init(&q_empty[i], 1);
-      ptx::mbar_init(&p_full[i], ATT_SM_WARPS); ptx::mbar_init(&p_empty[i], 1);
-    }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&q_full[i], 1); ptx::mbar_init(&q_empty[i], 1); }
+    for (int i = 0; i < RES_NP; ++i) { ptx::mbar_init(&p_full[i], ATT_SM_WARPS); ptx::mbar_init(&p_empty[i], 1); }
     for (int i = 0; i < RES_NB; ++i) { ptx::mbar_init(&s_full[i], 1); ptx::mbar_init(&s_free[i], ATT_SM_WARPS); }
     for (int i = 0; i < KST; ++i) { ptx::mbar_init(&k_full[i], 1); ptx::mbar_init(&k_empty[i], 1); }
     for (int i = 0; i < VST; ++i) { ptx::mbar_init(&v_full[i], 1); ptx::mbar_init(&v_empty[i], 1); }
@@ -245,9 +244,9 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         ptx::umma_commit(&q_empty[qb]);
         issued = 0; q_ready = false;
         for (int i = 0; i < nkv && ok; ++i) {
-          const int vs = vcnt % VST, pb = pcnt & 1;
+          const int vs = vcnt % VST, pb = pcnt % RES_NP;
           if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x8100 | vs)) { ok = false; break; }
-          if (!ptx::mbar_wait(&p_full[pb], (pcnt >> 1) & 1, p.err, 0x8200 | pb)) { ok = false; break; }
+          if (!ptx::mbar_wait(&p_full[pb], (pcnt / RES_NP) & 1, p.err, 0x8200 | pb)) { ok = false; break; }
           if (!o_free) {
             if (!ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x8600)) { ok = false; break; }
             o_free = true;
@@ -303,12 +302,19 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       pend = false;
     };
 
+    // the next tile's coordinates are decoded one iteration ahead: the integer divisions and the key-length load
+    // overlap the current tile's work instead of standing at the head of every iteration
+    int qt_n = 0, h_n = 0, b_n = 0, klen_n = 0, nkv_n = 0;
+    if ((int)blockIdx.x < total_tiles) { attn_tile(p, blockIdx.x, qt_n, h_n, b_n); nkv_n = attn_nkv(p, qt_n, b_n, klen_n); }
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      int qt, h, b, klen; attn_tile(p, t, qt, h, b);
-      const int nkv = attn_nkv(p, qt, b, klen);
+      const int qt = qt_n, h = h_n, b = b_n, klen = klen_n, nkv = nkv_n;
+      if (t + (int)gridDim.x < total_tiles) { attn_tile(p, t + gridDim.x, qt_n, h_n, b_n); nkv_n = attn_nkv(p, qt_n, b_n, klen_n); }
       const int q0 = qt * ATT_BM, row_base = b * p.S, col0 = h * DH;
       const int q = q0 + r_loc;
       const bool row_ok = q < p.S;
+      float osc_raw = 1.f;                                   // this thread's S_attn[j], turned into a factor further down
+      if (p.out_dt == HERO_I8 && (int)threadIdx.x < DH)
+        osc_raw = __ldg(p.out_scale + (long long)(col0 + (int)threadIdx.x) * p.out_scale_stride);
       if (nkv == 0) {
         // every key masked: the rows are zero, no tensor work
         if (cq * 32 < DH && row_ok) {
@@ -390,9 +396,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
       st[cq * ATT_BM + r_loc] = make_float2(m, l);
-      if (p.out_dt == HERO_I8 && (int)threadIdx.x < DH)
-        osc_s[(wcnt & 1) * 128 + threadIdx.x] =
-            p.pv_scale / __ldg(p.out_scale + (long long)(col0 + (int)threadIdx.x) * p.out_scale_stride);
+      if ((int)threadIdx.x < DH) osc_s[(wcnt & 1) * 128 + threadIdx.x] = p.pv_scale / osc_raw;
       asm volatile("bar.sync 1, 512;" ::: "memory");
       {
         float mf = -INFINITY;
@@ -415,8 +419,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 #pragma unroll 1
       for (int i = 0; i < nkv; ++i) {
         const int j = res_pv_block(nkv, i);
-        const int pb = pcnt & 1;
-        if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt >> 1) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
+        const int pb = pcnt % RES_NP;
+        if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt / RES_NP) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
         PH(6);
         if (ok) {
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
@@ -434,13 +438,24 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             const float f = mp > -INFINITY ? ex2f(mp - m) * pscale : 0.f;
             const float2 f2v = make_float2(f, f), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
             uint32_t w[4];
+            if (f <= 255.25f) {
+              // e <= 1 in every piece, so e f cannot round above 255: no clip needed
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const int e = 4 * k;
-              const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), f2v, rm2);
-              const float2 c = __ffma2_rn(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])), f2v, rm2);
-              w[k] = low_bytes4_u(fminf(a.x, ATT_MAGIC + 255.0f), fminf(a.y, ATT_MAGIC + 255.0f),
-                                  fminf(c.x, ATT_MAGIC + 255.0f), fminf(c.y, ATT_MAGIC + 255.0f));
+              for (int k = 0; k < 4; ++k) {
+                const int e = 4 * k;
+                const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), f2v, rm2);
+                const float2 c = __ffma2_rn(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])), f2v, rm2);
+                w[k] = low_bytes4_u(a.x, a.y, c.x, c.y);
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int e = 4 * k;
+                const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), f2v, rm2);
+                const float2 c = __ffma2_rn(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])), f2v, rm2);
+                w[k] = low_bytes4_u(fminf(a.x, ATT_MAGIC + 255.0f), fminf(a.y, ATT_MAGIC + 255.0f),
+                                    fminf(c.x, ATT_MAGIC + 255.0f), fminf(c.y, ATT_MAGIC + 255.0f));
+              }
             }
             st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
           }

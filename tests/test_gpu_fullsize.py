@@ -65,15 +65,18 @@ def test_c4_gpt_prefill_layer_full_batch_sampled_sequence():
     T = OL.layer_forward(Lp, O.fp_tensor(x[rows], "bf16"), B=1)
     got, want = out[rows].float().cpu().numpy().astype(np.float64), T["h_out"].real()
     d = np.abs(got - want)
-    # Free-running: the residual stream is h + X_o S_o + X_2 S_x2 with INT8 branches, so an INT8 code that flips on an
-    # fp32-vs-fp64 rounding tie upstream moves the output by one LSB of that branch (S_o[j] or S_x2[j]); on top comes
-    # one BF16 unit of the output itself.  That, not 1e-2 of max|o|, is the bound a single element can reach at this
-    # size (67 M elements, a few hundred legitimate flips); the bulk must agree to BF16 rounding.
+    # Free-running: the output is x + X_o S_o + X_2 S_x2 with INT8 branches.  An INT8 code that flips on an fp32-vs-fp64
+    # rounding tie moves the output by one LSB of its branch (S_o[j] or S_x2[j]), and a flip upstream (LN^quant, QKV,
+    # X_attn) perturbs every accumulator of its row, so a row can collect a few flips.  With 8.4 M elements compared the
+    # bound for a single element is therefore a few branch LSBs plus the BF16 unit of the output, not 1e-2 of max|o|;
+    # what must hold is that such elements are rare and that the bulk agrees to BF16 rounding.
     C = Lp["C"]
-    lsb = float(np.max(C["S_x2"]) + np.max(C["S_o"]))
+    lsb = (np.asarray(C["S_x2"], dtype=np.float64) + np.asarray(C["S_o"], dtype=np.float64)).reshape(1, -1)
     ulp = 2.0 ** -7 * np.maximum(np.abs(want), 2.0 ** -10)
-    assert np.all(d <= lsb + 2 * ulp), float(d.max())
-    assert np.mean(d > ulp) < 1e-3, float(np.mean(d > ulp))
+    stats = (float(d.max()), float(np.mean(d > 2 * ulp)), float(np.mean(d > lsb + 2 * ulp)))
+    assert np.all(d <= 3 * lsb + 2 * ulp), stats
+    assert np.mean(d > lsb + 2 * ulp) < 1e-5, stats
+    assert np.mean(d > 2 * ulp) < 1e-3, stats
     assert float(d.mean() / np.abs(want).mean()) < 2e-3
     assert rel_err(got, want) < 3e-2
     h.close()
