@@ -22,6 +22,7 @@ constexpr int GEMM_THREADS = 320;
 constexpr int TMA_WARP = 8, MMA_WARP = 9;
 constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2;
 extern int g_gemm_pair;   // experiment switch: CTA-pair (cta_group::2) kernel on / off
+extern int g_gemm_ew;     // experiment switch: 0 = heuristic, 8 / 16 = forced epilogue warps of the pair kernel
 
 struct GemmParams {
   int M, N, K;              // K in elements
@@ -45,7 +46,7 @@ struct GemmCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int EPI_FLOATS = 2 * 3 * BN;                 // double-buffered cs / bias / post
+  static constexpr int EPI_FLOATS = 4 * 2 * 3 * BN;             // per-warp, double-buffered cs / bias / post
   static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256 /*barriers*/;
 };
 
@@ -66,6 +67,26 @@ __device__ __forceinline__ float gelu_erf_f(float v) {
   float e;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(v * v * -0.72134752044448170368f));   // exp(-v^2 / 2)
   return fmaf(-0.5f * av, poly * e, fmaxf(v, 0.0f));
+}
+// the same on a packed pair: the polynomial and the products run as FFMA2 / FMUL2, two special-function ops per element
+__device__ __forceinline__ float2 gelu_erf_f2(float2 v) {
+  const float2 av = make_float2(fabsf(v.x), fabsf(v.y));
+  const float kz = 0.3275911f * 0.70710678118654752440f;
+  const float2 d = __ffma2_rn(av, make_float2(kz, kz), make_float2(1.0f, 1.0f));
+  float2 t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.x) : "f"(d.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.y) : "f"(d.y));
+  float2 poly = __ffma2_rn(make_float2(1.061405429f, 1.061405429f), t, make_float2(-1.453152027f, -1.453152027f));
+  poly = __ffma2_rn(poly, t, make_float2(1.421413741f, 1.421413741f));
+  poly = __ffma2_rn(poly, t, make_float2(-0.284496736f, -0.284496736f));
+  poly = __ffma2_rn(poly, t, make_float2(0.254829592f, 0.254829592f));
+  poly = __fmul2_rn(poly, t);
+  const float2 q = __fmul2_rn(__fmul2_rn(v, make_float2(-0.72134752044448170368f, -0.72134752044448170368f)), v);
+  float2 e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(q.x));                // exp(-v^2 / 2)
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(q.y));
+  const float2 w = __fmul2_rn(__fmul2_rn(av, make_float2(-0.5f, -0.5f)), __fmul2_rn(poly, e));
+  return __fadd2_rn(w, make_float2(fmaxf(v.x, 0.0f), fmaxf(v.y, 0.0f)));
 }
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   return 0.5f * x * (1.0f + tanhf(0.79788456080286535588f * (x + 0.044715f * x * x * x)));
@@ -115,32 +136,32 @@ __device__ __forceinline__ void st32(void* p, const uint32_t (&w)[8]) {   // 256
                : "memory");
 }
 
-// 32 columns of one output row: v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];
+// NC (16 or 32) columns of one output row: v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];
 // INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.  Per-column vectors come from shared memory four at a time,
 // the arithmetic runs on packed FP32 pairs, the row segment leaves in 32-byte stores when the output allows it.
-template <bool INT8, int ACT, int OUTK>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32_t (&r)[32], const float* e_cs,
+template <bool INT8, int ACT, int OUTK, int NC>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32_t (&r)[NC], const float* e_cs,
                                                const float* e_bias, const float* e_post, int m, bool row_ok, float rs,
                                                int col0, bool wide) {
   if constexpr (OUTK == OUT_I32) {
     if (!row_ok) return;
     int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
-    if (wide && col0 + 32 <= p.N) {
+    if (wide && col0 + NC <= p.N) {
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
+      for (int g = 0; g < NC / 8; ++g) {
         const uint32_t w[8] = {r[8 * g], r[8 * g + 1], r[8 * g + 2], r[8 * g + 3], r[8 * g + 4], r[8 * g + 5], r[8 * g + 6], r[8 * g + 7]};
         st32(dst + 8 * g, w);
       }
     } else {
 #pragma unroll
-      for (int g = 0; g < 8; ++g)
+      for (int g = 0; g < NC / 4; ++g)
         if (col0 + 4 * g + 4 <= p.N) st16(dst + 4 * g, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
     }
   } else {
-    float v[32];
+    float v[NC];
     const float2 rs2 = make_float2(rs, rs), mg2 = make_float2(ROUND_MAGIC, ROUND_MAGIC);
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < NC; j += 4) {
       const float4 cs4 = *reinterpret_cast<const float4*>(e_cs + j);
       const float4 b4 = *reinterpret_cast<const float4*>(e_bias + j);
       const float4 p4 = *reinterpret_cast<const float4*>(e_post + j);
@@ -154,9 +175,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
       }
       float2 x0 = __ffma2_rn(__fmul2_rn(a0, rs2), make_float2(cs4.x, cs4.y), make_float2(b4.x, b4.y));
       float2 x1 = __ffma2_rn(__fmul2_rn(a1, rs2), make_float2(cs4.z, cs4.w), make_float2(b4.z, b4.w));
-      if constexpr (ACT == HERO_ACT_GELU_ERF) {
-        x0.x = gelu_erf_f(x0.x); x0.y = gelu_erf_f(x0.y); x1.x = gelu_erf_f(x1.x); x1.y = gelu_erf_f(x1.y);
-      }
+      if constexpr (ACT == HERO_ACT_GELU_ERF) { x0 = gelu_erf_f2(x0); x1 = gelu_erf_f2(x1); }
       if constexpr (ACT == HERO_ACT_GELU_TANH) {
         x0.x = gelu_tanh_f(x0.x); x0.y = gelu_tanh_f(x0.y); x1.x = gelu_tanh_f(x1.x); x1.y = gelu_tanh_f(x1.y);
       }
@@ -177,87 +196,119 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
     if (!row_ok) return;
     if constexpr (OUTK == OUT_I8) {
       int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
-      uint32_t w[8];
+      uint32_t w[NC / 4];
 #pragma unroll
-      for (int g = 0; g < 8; ++g) w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-      if (wide && col0 + 32 <= p.N) {
-        st32(dst, w);
+      for (int g = 0; g < NC / 4; ++g) w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+      if constexpr (NC == 32) {
+        if (wide && col0 + 32 <= p.N) {
+          st32(dst, w);
+        } else {
+          if (col0 + 16 <= p.N) st16(dst, w[0], w[1], w[2], w[3]);
+          if (col0 + 32 <= p.N) st16(dst + 16, w[4], w[5], w[6], w[7]);
+        }
       } else {
         if (col0 + 16 <= p.N) st16(dst, w[0], w[1], w[2], w[3]);
-        if (col0 + 32 <= p.N) st16(dst + 16, w[4], w[5], w[6], w[7]);
       }
     } else {
       uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
-      uint32_t w[16];
+      uint32_t w[NC / 2];
 #pragma unroll
-      for (int g = 0; g < 16; ++g) w[g] = pack2_fp(v[2 * g], v[2 * g + 1], p.out_dt);
-      if (wide && col0 + 32 <= p.N) {
-        const uint32_t w0[8] = {w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]};
-        const uint32_t w1[8] = {w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]};
-        st32(dst, w0);
-        st32(dst + 16, w1);
+      for (int g = 0; g < NC / 2; ++g) w[g] = pack2_fp(v[2 * g], v[2 * g + 1], p.out_dt);
+      if (wide && col0 + NC <= p.N) {
+#pragma unroll
+        for (int g = 0; g < NC / 16; ++g) {
+          const uint32_t w0[8] = {w[8 * g], w[8 * g + 1], w[8 * g + 2], w[8 * g + 3], w[8 * g + 4], w[8 * g + 5], w[8 * g + 6], w[8 * g + 7]};
+          st32(dst + 16 * g, w0);
+        }
       } else {
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
+        for (int g = 0; g < NC / 8; ++g)
           if (col0 + 8 * g + 8 <= p.N) st16(dst + 8 * g, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
       }
     }
   }
 }
 
-// One thread's share of a tile's epilogue: BN / 2 columns of one output row, 32 at a time from tensor memory,
-// the next 32 already loading while the current ones are processed.
-template <int BN, bool INT8, int ACT, int OUTK>
+// One thread's share of a tile's epilogue: BN / (EW / 4) columns of one output row (EW epilogue warps, EW / 4 per
+// tensor-memory lane quarter).  With 8 warps the columns come 32 at a time, the next 32 already loading while the
+// current ones are processed; with 16 warps (96 registers per thread) 16 at a time.
+template <int BN, bool INT8, int ACT, int OUTK, int EW>
 __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const float* e_cs, const float* e_bias,
                                                  const float* e_post, uint32_t taddr, int m, bool row_ok, float rs,
-                                                 int n0, int chalf) {
-  constexpr int CH = BN / 2, NCH = CH / 32;
+                                                 int n0, int cpart) {
+  constexpr int CH = BN / (EW / 4);
   // 32-byte stores need a 32-byte aligned row segment: base pointer and row pitch multiples of 32 bytes
   const int es = OUTK == OUT_I8 ? 1 : (OUTK == OUT_FP ? 2 : 4);
   const bool wide = ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0) && ((p.out_ld * es) % 32 == 0);
-  uint32_t ra[32], rb[32];
-  ptx::tmem_ld32(taddr, ra);
+  if constexpr (EW == 8) {
+    constexpr int NCH = CH / 32;
+    uint32_t ra[32], rb[32];
+    ptx::tmem_ld32(taddr, ra);
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    ptx::tmem_ld_wait();
-    if (c + 1 < NCH) ptx::tmem_ld32(taddr + (c + 1) * 32, (c & 1) ? ra : rb);
-    const int jc = chalf * CH + c * 32;   // column of the chunk's first element inside the tile
-    if (c & 1) epilogue_chunk<INT8, ACT, OUTK>(p, rb, e_cs + jc, e_bias + jc, e_post + jc, m, row_ok, rs, n0 + jc, wide);
-    else epilogue_chunk<INT8, ACT, OUTK>(p, ra, e_cs + jc, e_bias + jc, e_post + jc, m, row_ok, rs, n0 + jc, wide);
+    for (int c = 0; c < NCH; ++c) {
+      ptx::tmem_ld_wait();
+      if (c + 1 < NCH) ptx::tmem_ld32(taddr + (c + 1) * 32, (c & 1) ? ra : rb);
+      const int jw = c * 32;                // column of the chunk's first element among this warp's columns
+      const int jc = cpart * CH + jw;       // ... and inside the tile
+      if (c & 1) epilogue_chunk<INT8, ACT, OUTK, 32>(p, rb, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
+      else epilogue_chunk<INT8, ACT, OUTK, 32>(p, ra, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
+    }
+  } else {
+    constexpr int NCH = CH / 16;
+    uint32_t ra[16], rb[16];
+    ptx::tmem_ld16(taddr, ra);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      ptx::tmem_ld_wait();
+      if (c + 1 < NCH) ptx::tmem_ld16(taddr + (c + 1) * 16, (c & 1) ? ra : rb);
+      const int jw = c * 16;
+      const int jc = cpart * CH + jw;
+      if (c & 1) epilogue_chunk<INT8, ACT, OUTK, 16>(p, rb, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
+      else epilogue_chunk<INT8, ACT, OUTK, 16>(p, ra, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
+    }
   }
 }
 
 // The epilogue warps' walk over this CTA's tiles.  The per-column vectors (and the row scale) of the NEXT tile are
 // fetched from global memory into registers while the current tile is being processed, so a tile never starts by
 // waiting on them.  ROWS = output rows per tile (128, or 256 for a CTA pair of which this CTA owns rows row_off..+127).
-template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR>
+template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR, int EW>
 __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, uint64_t* acc_full, uint64_t* acc_empty,
                                               uint32_t tmem_base, int first_tile, int tile_stride, int row_off) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int quarter = warp & 3, chalf = warp >> 2;
-  constexpr int CH = BN / 2;                 // columns per thread and tile
-  const int tid_e = threadIdx.x;             // 0..255: the column of the tile whose vectors this thread stages
+  const int quarter = warp & 3, cpart = warp >> 2;
+  constexpr int CH = BN / (EW / 4);          // columns per thread and tile
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;
   bool ok = true;
 
-  float ncs = 1.0f, nbias = 0.0f, npost = 1.0f, nrs = 1.0f;
+  // Every warp stages the per-column vectors of its own CH columns in a shared-memory area of its own (two buffers,
+  // 3 x CH floats each), so the epilogue warps never wait for one another.
+  constexpr int NV = CH / 32;                // values per lane and vector
+  float* epi_w = epi + warp * (2 * 3 * CH);
+  float ncs[NV], nbias[NV], npost[NV], nrs = 1.0f;
   auto fetch = [&](int t) {                  // issue the loads for tile t; the values are consumed one tile later
     int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
     if constexpr (OUTK != OUT_I32) {
-      const int n = nt * BN + tid_e;
-      const bool in = tid_e < BN && n < p.N;
-      ncs = (in && p.cs) ? __ldg(p.cs + n) : 1.0f;
-      nbias = (in && p.bias) ? __ldg(p.bias + n) : 0.0f;
-      npost = (in && p.post) ? __ldg(p.post + n) : 1.0f;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const int n = nt * BN + cpart * CH + i * 32 + lane;
+        const bool in = n < p.N;
+        ncs[i] = (in && p.cs) ? __ldg(p.cs + n) : 1.0f;
+        nbias[i] = (in && p.bias) ? __ldg(p.bias + n) : 0.0f;
+        npost[i] = (in && p.post) ? __ldg(p.post + n) : 1.0f;
+      }
       const int m = mt * ROWS + row_off + quarter * 32 + lane;
       nrs = (INT8 && p.rs && m < p.M) ? __ldg(p.rs + m) : 1.0f;
     }
   };
   auto publish = [&](int it) {               // registers -> this tile's shared-memory vectors
     if constexpr (OUTK != OUT_I32) {
-      float* e = epi + (it & 1) * 3 * BN;
-      if (tid_e < BN) { e[tid_e] = ncs; e[BN + tid_e] = nbias; e[2 * BN + tid_e] = npost; }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      float* e = epi_w + (it & 1) * 3 * CH;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        e[i * 32 + lane] = ncs[i]; e[CH + i * 32 + lane] = nbias[i]; e[2 * CH + i * 32 + lane] = npost[i];
+      }
+      __syncwarp();
     }
   };
 
@@ -271,21 +322,21 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     const float rs = nrs;
     publish(it);
     if (t + tile_stride < num_tiles) fetch(t + tile_stride);
-    const float* e_cs = epi + (it & 1) * 3 * BN;
+    const float* e_cs = epi_w + (it & 1) * 3 * CH;
     const int m = mt * ROWS + row_off + quarter * 32 + lane;
     const bool row_ok = m < p.M;
 
     if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
     ptx::tc_fence_after();
     if (ok) {
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + chalf * CH;
-      epilogue_columns<BN, INT8, ACT, OUTK>(p, e_cs, e_cs + BN, e_cs + 2 * BN, taddr, m, row_ok, rs, n0, chalf);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + cpart * CH;
+      epilogue_columns<BN, INT8, ACT, OUTK, EW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart);
     }
     // hand the accumulator buffer back to the UMMA issuer
     ptx::tc_fence_before();
     __syncwarp();
     if (lane == 0) {
-      if constexpr (PAIR) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&acc_empty[as]), 0));
+      if constexpr (PAIR) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(ptx::smem_u32(&acc_empty[as]), 0));
       else ptx::mbar_arrive(&acc_empty[as]);
     }
   }
@@ -384,7 +435,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-7)
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
-    epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0);
+    epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0);
   }
 
   ptx::tc_fence_before();
@@ -454,12 +505,12 @@ struct PairCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = 6;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int EPI_FLOATS = 2 * 3 * BN;
+  static constexpr int EPI_FLOATS = 4 * 2 * 3 * BN;
   static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256;
 };
 
-template <bool INT8, int ACT, int OUTK>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+template <bool INT8, int ACT, int OUTK, int EW>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW + 2) * 32, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
   using Cfg = PairCfg;
   constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
@@ -482,21 +533,21 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 16); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 2 * EW); }
     ptx::fence_mbar_init();
   }
-  if (warp == MMA_WARP) {
+  if (warp == EW + 1) {
     ptx::tmem_alloc_pair(tmem_slot, Cfg::TMEM_COLS);
     ptx::tmem_relinquish_pair();
   }
-  if (warp == TMA_WARP && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
+  if (warp == EW && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::cluster_sync();                                   // both CTAs' barriers exist before any remote arrive
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == TMA_WARP) {
+  if (warp == EW) {
     // ------------------------------------------------------------------ TMA producer (leader CTA only)
     // One thread feeds both CTAs: its own halves of A and W go to local shared memory, the peer's halves to the
     // peer's shared memory, all four copies completing on the leader's `full` barrier.  The peer needs no producer,
@@ -526,7 +577,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == MMA_WARP) {
+  } else if (warp == EW + 1) {
     // ------------------------------------------------------------------ UMMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
@@ -558,20 +609,20 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 0-7 of each CTA)
-    epilogue_loop<BN, INT8, ACT, OUTK, 256, true>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM);
+    // ------------------------------------------------------------------ epilogue (warps 0 .. EW-1 of each CTA)
+    epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM);
   }
 
   ptx::tc_fence_before();
   __syncthreads();
   ptx::cluster_sync();                                   // the peer may still be reading this CTA's shared memory / barriers
-  if (warp == MMA_WARP) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
+  if (warp == EW + 1) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <bool INT8, int ACT, int OUTK>
-static hero_status launch_gemm_pair(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
-                                    cudaStream_t stream) {
-  auto kern = gemm_pair_kernel<INT8, ACT, OUTK>;
+template <bool INT8, int ACT, int OUTK, int EW>
+static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+                                       cudaStream_t stream) {
+  auto kern = gemm_pair_kernel<INT8, ACT, OUTK, EW>;
   static bool configured = false;
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg::SMEM_BYTES));
@@ -582,10 +633,22 @@ static hero_status launch_gemm_pair(hero_handle* h, const CUtensorMap& tmA, cons
   const int pairs = tiles < pairs_max ? tiles : pairs_max;
   {
     LaunchScope scope(h, stream, KERNEL_GEMM);
-    kern<<<2 * pairs, GEMM_THREADS, PairCfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+    kern<<<2 * pairs, (EW + 2) * 32, PairCfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
+}
+
+// 16 epilogue warps when the epilogue sets the pace (an activation and few k-blocks per tile); 8 (with twice the
+// registers and 32-column chunks) otherwise.
+template <bool INT8, int ACT, int OUTK>
+static hero_status launch_gemm_pair(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+                                    cudaStream_t stream) {
+  if constexpr (OUTK != OUT_I32) {
+    const bool wide_epi = g_gemm_ew ? g_gemm_ew == 16 : (ACT != HERO_ACT_NONE && p.num_kb <= 16);
+    if (wide_epi) return launch_gemm_pair_ew<INT8, ACT, OUTK, 16>(h, tmA, tmW, p, stream);
+  }
+  return launch_gemm_pair_ew<INT8, ACT, OUTK, 8>(h, tmA, tmW, p, stream);
 }
 
 template <bool INT8>
@@ -650,10 +713,12 @@ static hero_status run_bn(hero_handle* h, const hero_linear_args* a, GemmParams&
 }
 
 int g_gemm_pair = 1;
+int g_gemm_ew = 0;
 
 }  // namespace hero
 
 extern "C" void hero_debug_gemm_pair(int on) { hero::g_gemm_pair = on; }
+extern "C" void hero_debug_gemm_ew(int ew) { hero::g_gemm_ew = ew; }
 
 extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* stream) {
   using namespace hero;
