@@ -228,6 +228,17 @@ typedef struct {
 hero_status hero_mode_preset(int32_t preset, int32_t mode_out[5]);
 /* Scratch the layer needs for M tokens. */
 hero_status hero_layer_workspace_bytes(const hero_layer_desc* d, int64_t M, size_t* bytes);
+/* Where hero_layer_forward leaves the tensors at the operator borders (Sec. 2.2.2-2.2.3) inside the workspace: byte
+ * offsets from the workspace pointer, valid after a forward call has completed, for inspection and stage-by-stage
+ * checking.  Every tensor is row-major [M, cols] with ld = cols, INT8 or fp_dtype as the module modes dictate.
+ *   qkv [M,3H], x_attn [M,H], x_o [M,H], x_mid [M,H] (+ x_mid_scale [M] FP32 when gran_mid is TWQ), a [M,F] (the
+ *   GELU^quant output), x_2 [M,H]; pre-LN only: x_in [M,H] (+ x_in_scale [M]), h_in and h_mid [M,H] in fp_dtype
+ *   (h_in holds h + pending when a pending branch was given).  Offsets that do not apply are 0. */
+typedef struct hero_layer_layout {
+  size_t qkv, x_attn, x_o, x_mid, x_mid_scale, a, x_2, x_in, x_in_scale, h_in, h_mid;
+  size_t total;            /* = hero_layer_workspace_bytes */
+} hero_layer_layout;
+hero_status hero_layer_workspace_layout(const hero_layer_desc* d, int64_t M, hero_layer_layout* layout);
 /*   in      : post-LN: X_in [M, H] I8 (+scale per gran_in) or fp_dtype when QKV is FP.
  *             pre-LN : residual stream h [M, H] in fp_dtype.
  *   pending : pre-LN only, optional: a branch (I8 FWQ or fp_dtype) still to be added to h, i.e. the

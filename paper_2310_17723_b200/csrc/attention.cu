@@ -388,13 +388,7 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
   return HERO_OK;
 }
 
-int g_attn_resident = 1;
-long long* g_attn_dbg = nullptr;
-
 }  // namespace hero
-
-extern "C" void hero_debug_attn_resident(int on) { hero::g_attn_resident = on; }
-extern "C" void hero_debug_attn_dbg(void* ptr) { hero::g_attn_dbg = (long long*)ptr; }
 
 extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream) {
   using namespace hero;
@@ -432,11 +426,10 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   p.mask = a->mask; p.key_len = a->key_len;
   p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
   p.err = h->d_error;
-  p.dbg = g_attn_dbg;
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
-  if (g_attn_resident && a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory
+  if (a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory
   if (a->dh == 64) return launch_attn<64>(h, a, p, s);
   return launch_attn<128>(h, a, p, s);
 }

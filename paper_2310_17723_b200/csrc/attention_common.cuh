@@ -32,7 +32,6 @@ struct AttnParams {
   int out_dt;
   uint32_t idesc_qk, idesc_pv;
   int* err;
-  long long* dbg;          // phase cycle counters (experiments only; NULL otherwise)
 };
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -91,7 +90,5 @@ __device__ __forceinline__ int attn_nkv(const AttnParams& p, int qt, int b, int&
 hero_status attn_fp_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
 // INT8 core with the whole score row resident in tensor memory (S <= 512); defined in attention_resident.cu
 hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
-extern int g_attn_resident;   // experiment switch
-extern long long* g_attn_dbg;
 
 }  // namespace hero

@@ -14,11 +14,6 @@
 
 namespace hero {
 
-#ifdef HERO_ATTN_PHASES
-#define PH(i) do { if (dbgon) { const long long c_ = clock64(); ph[i] += c_ - tprev; tprev = c_; } } while (0)
-#else
-#define PH(i) do {} while (0)
-#endif
 
 constexpr int RES_NB = 4;          // score blocks resident in TMEM (4 x 128 columns)
 constexpr int RES_O_COL = 384;     // output accumulator columns
@@ -287,11 +282,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     const float c2 = p.c2;
     uint32_t pcnt = 0, wcnt = 0, used = 0;
     bool ok = true;
-#ifdef HERO_ATTN_PHASES
-    const bool dbgon = p.dbg != nullptr && lane == 0;
-    long long ph[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-    long long tprev = clock64();
-#endif
     long long pend_row = -1;                                 // output row of the tile whose epilogue is pending
     int pend_col = 0;
     bool pend = false;
@@ -334,10 +324,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 #pragma unroll 1
       for (int j = 0; j < nkv; ++j) {
         if (j == 3 && pend) epilogue();                      // block 3's columns hold the previous tile's output
-        PH(10);
         if (ok && !ptx::mbar_wait(&s_full[j], (used >> j) & 1, p.err, 0x9000 | j)) ok = false;
         ptx::tc_fence_after();
-        PH(0);
         if (ok) {
           const uint32_t ta = t_lane + j * ATT_BN + cq * 32;
           const int kb = j * ATT_BN + cq * 32;
@@ -346,7 +334,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           ptx::tmem_ld16(ta, ra);
           ptx::tmem_ld16(ta + 16, rb);
           ptx::tmem_ld_wait();
-          PH(1);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {                   // two 16-column pieces, each with its own maximum
             uint32_t (&r)[16] = hh ? rb : ra;
@@ -379,7 +366,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 #pragma unroll
               for (int e = 0; e < 16; ++e) r[e] = 0;         // every key of the piece masked
             }
-            PH(2);
             ptx::tmem_st16(ta + 16 * hh, r);
             mpa[hh] = mp;
           }
@@ -387,12 +373,9 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         } else {
           pm2[j * 512] = make_float2(-INFINITY, -INFINITY);
         }
-        PH(3);
       }
       if (ok) ptx::tmem_st_wait();
-      PH(3);
       if (pend) epilogue();
-      PH(4);
       // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
       st[cq * ATT_BM + r_loc] = make_float2(m, l);
@@ -413,7 +396,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         m = mf; l = lf;
       }
       const float pscale = l > 0.f ? p.inv_sp / l : 0.f;
-      PH(5);
 
       // ---- sweep 2: P_u8 = Round(e * 2^(m_piece - m) / (l s_p)), clipped to 255, into the UMMA operand tile
 #pragma unroll 1
@@ -421,7 +403,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         const int j = res_pv_block(nkv, i);
         const int pb = pcnt % RES_NP;
         if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt / RES_NP) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
-        PH(6);
         if (ok) {
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
           const float2 mp2 = pm2[j * 512];
@@ -430,7 +411,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32, ra);
           ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32 + 16, rb);
           ptx::tmem_ld_wait();
-          PH(7);
 #pragma unroll
           for (int g = 0; g < 2; ++g) {
             uint32_t (&r)[16] = g ? rb : ra;
@@ -460,12 +440,10 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
           }
         }
-        PH(8);
         ptx::tc_fence_before();
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) { ptx::mbar_arrive(&s_free[j]); ptx::mbar_arrive(&p_full[pb]); }
-        PH(9);
         ++pcnt; used ^= 1u << j;
       }
       pend = true;
@@ -474,12 +452,6 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       ++wcnt;
     }
     if (pend) epilogue();
-    PH(4);
-#ifdef HERO_ATTN_PHASES
-    if (dbgon && blockIdx.x == 0) {
-      for (int i = 0; i < 12; ++i) p.dbg[warp * 12 + i] = ph[i];
-    }
-#endif
   }
 
   ptx::tc_fence_before();

@@ -21,8 +21,6 @@ constexpr int GEMM_BK_BYTES = 128;   // one swizzle row
 constexpr int GEMM_THREADS = 320;
 constexpr int TMA_WARP = 8, MMA_WARP = 9;
 constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2;
-extern int g_gemm_pair;   // experiment switch: CTA-pair (cta_group::2) kernel on / off
-extern int g_gemm_ew;     // experiment switch: 0 = heuristic, 8 / 16 = forced epilogue warps of the pair kernel
 
 struct GemmParams {
   int M, N, K;              // K in elements
@@ -645,7 +643,7 @@ template <bool INT8, int ACT, int OUTK>
 static hero_status launch_gemm_pair(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
                                     cudaStream_t stream) {
   if constexpr (OUTK != OUT_I32) {
-    const bool wide_epi = g_gemm_ew ? g_gemm_ew == 16 : (ACT != HERO_ACT_NONE && p.num_kb <= 16);
+    const bool wide_epi = ACT != HERO_ACT_NONE && p.num_kb <= 16;
     if (wide_epi) return launch_gemm_pair_ew<INT8, ACT, OUTK, 16>(h, tmA, tmW, p, stream);
   }
   return launch_gemm_pair_ew<INT8, ACT, OUTK, 8>(h, tmA, tmW, p, stream);
@@ -712,13 +710,9 @@ static hero_status run_bn(hero_handle* h, const hero_linear_args* a, GemmParams&
   return dispatch_epilogue<BN, false>(h, tmA, tmW, p, a->act, s);
 }
 
-int g_gemm_pair = 1;
-int g_gemm_ew = 0;
 
 }  // namespace hero
 
-extern "C" void hero_debug_gemm_pair(int on) { hero::g_gemm_pair = on; }
-extern "C" void hero_debug_gemm_ew(int ew) { hero::g_gemm_ew = ew; }
 
 extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* stream) {
   using namespace hero;
@@ -764,7 +758,7 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   const long long t128 = (long long)p.num_m_tiles * ((p.N + 127) / 128);
   const long long enough = (long long)h->sm_count * 6 / 10;
   const long long tpair = (long long)((p.M + 255) / 256) * ((p.N + 255) / 256);
-  if (g_gemm_pair && tpair * 2 >= enough && p.M > GEMM_BM) return run_pair(h, a, p, s);
+  if (tpair * 2 >= enough && p.M > GEMM_BM) return run_pair(h, a, p, s);
   if (t256 >= enough) return run_bn<256>(h, a, p, s);
   if (t128 >= enough) return run_bn<128>(h, a, p, s);
   return run_bn<64>(h, a, p, s);

@@ -64,6 +64,19 @@ extern "C" hero_status hero_layer_workspace_bytes(const hero_layer_desc* d, int6
   return HERO_OK;
 }
 
+extern "C" hero_status hero_layer_workspace_layout(const hero_layer_desc* d, int64_t M, hero_layer_layout* layout) {
+  using namespace hero;
+  HERO_REQUIRE(layout != nullptr, HERO_ERR_INVALID_ARG, "layout is NULL");
+  LayerPlan pl;
+  hero_status st = plan_layer(d, M, &pl);
+  if (st != HERO_OK) return st;
+  layout->qkv = pl.off_qkv; layout->x_attn = pl.off_attn; layout->x_o = pl.off_o; layout->x_mid = pl.off_mid;
+  layout->x_mid_scale = pl.off_mid_scale; layout->a = pl.off_a; layout->x_2 = pl.off_x2; layout->x_in = pl.off_xin;
+  layout->x_in_scale = pl.off_xin_scale; layout->h_in = pl.off_hin; layout->h_mid = pl.off_hmid;
+  layout->total = pl.total;
+  return HERO_OK;
+}
+
 extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in,
                                           const hero_tensor* pending, const hero_tensor* out, void* workspace,
                                           size_t workspace_bytes, void* stream) {

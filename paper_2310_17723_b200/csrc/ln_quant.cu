@@ -832,7 +832,6 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
   return HERO_OK;
 }
 
-int g_ln_first_n = 2;
 // Returns HERO_ERR_UNSUPPORTED (without setting an error) when the combination has no fast instantiation.
 static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
@@ -845,7 +844,7 @@ static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* t
   if (res == SRC_I8 && p.res.row_scale && p.res.col_scale) return HERO_OK;
   // rows of exactly 3 or 4 chunks per lane (H = 768, 1024, 4096, 8192, ...) take the tail-free instantiation
   int wpr = 1, exact = 0;
-  for (int n = 4; n >= g_ln_first_n && !exact; --n)              // H = 256 * n * wpr with wpr in {1, 2, 4, 8}
+  for (int n = 4; n >= 2 && !exact; --n)              // H = 256 * n * wpr with wpr in {1, 2, 4, 8}
     for (int w = 1; w <= 8 && !exact; w *= 2)
       if (p.H == 256 * n * w) { wpr = w; exact = n; }
   if (!exact) while (wpr * 1024 < p.H) wpr *= 2;
@@ -943,4 +942,3 @@ extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* 
   return launch_ln<8, 2>(h, p, s);
 }
 
-extern "C" void hero_debug_ln_first_n(int n) { hero::g_ln_first_n = n; }

@@ -74,9 +74,14 @@ class LayerDesc(C.Structure):
                 ("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p)]
 
 
+class LayerLayout(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("qkv", "x_attn", "x_o", "x_mid", "x_mid_scale", "a", "x_2", "x_in", "x_in_scale",
+                                          "h_in", "h_mid", "total")]
+
+
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
-           "hero_layer_workspace_bytes", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
+           "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
            "hero_profile_end", "hero_layer_forward_static")
 
 _lib = None
@@ -101,6 +106,7 @@ def lib():
         L.hero_int8_attention.argtypes = [C.c_void_p, C.POINTER(AttnArgs), C.c_void_p]
         L.hero_mode_preset.argtypes = [C.c_int32, C.POINTER(C.c_int32 * 5)]
         L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
+        L.hero_layer_workspace_layout.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(LayerLayout)]
         L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_host.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
@@ -197,6 +203,11 @@ class Handle:
         n = C.c_size_t()
         _check(lib().hero_layer_workspace_bytes(C.byref(desc), int(M), C.byref(n)))
         return int(n.value)
+
+    def hero_layer_workspace_layout(self, desc, M):
+        lay = LayerLayout()
+        _check(lib().hero_layer_workspace_layout(C.byref(desc), int(M), C.byref(lay)))
+        return lay
 
     def hero_layer_forward_host(self, desc, in_host, out_host, in_dev, out_dev, workspace, stream=None):
         """Host-buffer variant: copies in, runs the layer, copies out, synchronizes."""

@@ -1,6 +1,16 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times: the whole batch runs on the
-GPU, and whole sequences sampled from it are recomputed by the oracle (a layer is independent per sequence: token-wise
-scales are per row, calibrated scales are static, attention never crosses sequences)."""
+GPU through hero_layer_forward, and whole sequences sampled from it are recomputed by the oracle (a layer is
+independent per sequence: token-wise scales are per row, calibrated scales are static, attention never crosses
+sequences).
+
+Two comparisons per sampled sequence:
+  * stage by stage (teacher-forced): every operator-border tensor the layer left in its workspace is compared with the
+    oracle's operator applied to the tensor the DEVICE produced one stage earlier.  This is the parity bar proper: INT8
+    payloads bit-exact except 1 LSB on a tiny fraction (fp32-vs-fp64 rounding ties), FP tensors to storage rounding.
+  * end to end (free-running): the layer output against the oracle's own chain.  A code that flips on a tie perturbs
+    every accumulator of its row downstream (K = 4096..16384 terms), so at these sizes several percent of the INT8
+    codes legitimately differ by one LSB at the end; the check is therefore statistical (mean and max-norm error).
+"""
 import numpy as np
 import pytest
 import torch
@@ -9,7 +19,7 @@ from oracle import layer as OL
 from oracle import ops as O
 from paper_2310_17723_b200 import hero, workloads as W
 from paper_2310_17723_b200.layer import Layer
-from gpu_util import qt_to_device, rel_err, int8_mismatch, oracle_layer_to_prepared, TORCH_FP
+from gpu_util import qt_to_device, rel_err, int8_mismatch, assert_int8_close, oracle_layer_to_prepared, TORCH_FP
 
 pytestmark = pytest.mark.gpu
 
@@ -21,6 +31,38 @@ def _oracle_layer(shape, seed, n_cal, **kw):
     xc = W.activations(shape, seed, n_seq=n_cal, tensor=7).astype(np.float64)
     cal = O.layernorm(xc, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else xc
     return spec, p, OL.prepare_layer(spec, p, OL.calibrate(spec, p, cal, n_cal))
+
+
+class Borders:
+    """Views of the operator-border tensors hero_layer_forward left in the layer's workspace."""
+
+    def __init__(self, h, layer, shape):
+        self.lay = h.hero_layer_workspace_layout(layer.desc, shape.M)
+        self.ws, self.M = layer.workspace, shape.M
+
+    def i8(self, name, cols, rows):
+        off = getattr(self.lay, name)
+        v = self.ws[off:off + self.M * cols].view(torch.int8).view(self.M, cols)
+        return v[rows].cpu().numpy()
+
+    def f32(self, name, rows):
+        off = getattr(self.lay, name)
+        return self.ws[off:off + self.M * 4].view(torch.float32)[rows].cpu().numpy().astype(np.float64)
+
+    def fp(self, name, cols, rows, dt):
+        off = getattr(self.lay, name)
+        v = self.ws[off:off + self.M * cols * 2].view(TORCH_FP[dt]).view(self.M, cols)
+        return v[rows].float().cpu().numpy().astype(np.float64)
+
+
+def _like(template, data, row_scale=None):
+    """The device's INT8 payload with the scale metadata of the oracle tensor standing at the same border."""
+    return O.QT("i8", data, row_scale=row_scale if template.row_scale is not None else None, col_scale=template.col_scale)
+
+
+def _twq_close(got_q, got_s, want, what):
+    assert_int8_close(got_q, want.data, 1e-4, what)
+    np.testing.assert_allclose(got_s, want.row_scale, rtol=2e-6, err_msg=what + " scales")
 
 
 def test_c3_bert_large_layer_full_batch_sampled_sequences():
@@ -36,15 +78,32 @@ def test_c3_bert_large_layer_full_batch_sampled_sequences():
     layer.forward(in_desc, hero.tensor(out, "twq", sc))
     h.check()
     got_q, got_s = out.cpu().numpy(), sc.cpu().numpy().astype(np.float64)
-    S = shape.S
+    bd = Borders(h, layer, shape)
+    S, H, F = shape.S, shape.H, shape.F
     for b in (0, 13, 31):                                         # first, middle, last sequence of the batch
         rows = slice(b * S, (b + 1) * S)
         xb = O.QT("i8", x_in.data[rows], col_scale=x_in.col_scale)
         T = OL.layer_forward(Lp, xb, B=1)
-        want = T["x_out"]
+        # ---- stage by stage, each oracle operator fed with what the device produced one stage earlier
+        qkv = _like(T["qkv"], bd.i8("qkv", 3 * H, rows))
+        assert_int8_close(qkv.data, T["qkv"].data, 1e-4, "qkv")                  # same input on both sides
+        x_attn = _like(T["x_attn"], bd.i8("x_attn", H, rows))
+        assert_int8_close(x_attn.data, OL._attention(Lp, qkv, 1).data, 2e-4, "x_attn")
+        x_o = _like(T["x_o"], bd.i8("x_o", H, rows))
+        assert_int8_close(x_o.data, OL._linear(Lp["o"], x_attn, "none").data, 1e-4, "x_o")
+        x_mid = _like(T["x_mid"], bd.i8("x_mid", H, rows), bd.f32("x_mid_scale", rows))
+        want, _ = O.ln_quant([xb, x_o], Lp["ln1_g"], Lp["ln1_b"], spec.eps, Lp["ln_mid_out"])
+        _twq_close(x_mid.data, x_mid.row_scale, want, "x_mid")
+        a = _like(T["a"], bd.i8("a", F, rows))
+        assert_int8_close(a.data, OL._linear(Lp["fc1"], x_mid, spec.act).data, 1e-4, "a")
+        x_2 = _like(T["x_2"], bd.i8("x_2", H, rows))
+        assert_int8_close(x_2.data, OL._linear(Lp["fc2"], a, "none").data, 1e-4, "x_2")
+        want, _ = O.ln_quant([x_mid, x_2], Lp["ln2_g"], Lp["ln2_b"], spec.eps, Lp["ln_final_out"])
+        _twq_close(got_q[rows], got_s[rows], want, "x_out")
+        # ---- end to end against the oracle's own chain
         got = got_q[rows].astype(np.float64) * got_s[rows][:, None]
-        assert rel_err(got, want.real()) < 1e-2, b
-        frac, mx = int8_mismatch(got_q[rows], want.data)
+        assert rel_err(got, T["x_out"].real()) < 1e-2, b
+        frac, mx = int8_mismatch(got_q[rows], T["x_out"].data)
         assert mx <= 2 and frac < 2e-2, (b, frac, mx)
     h.close()
 
@@ -59,24 +118,44 @@ def test_c4_gpt_prefill_layer_full_batch_sampled_sequence():
     out = torch.empty(shape.M, shape.H, dtype=torch.bfloat16, device="cuda")
     layer.forward(hero.tensor(xd), hero.tensor(out))
     h.check()
-    S = shape.S
+    bd = Borders(h, layer, shape)
+    S, H, F, fd = shape.S, shape.H, shape.F, shape.fp_dtype
     b = 5
     rows = slice(b * S, (b + 1) * S)
-    T = OL.layer_forward(Lp, O.fp_tensor(x[rows], "bf16"), B=1)
-    got, want = out[rows].float().cpu().numpy().astype(np.float64), T["h_out"].real()
-    d = np.abs(got - want)
-    # Free-running: the output is x + X_o S_o + X_2 S_x2 with INT8 branches.  An INT8 code that flips on an fp32-vs-fp64
-    # rounding tie moves the output by one LSB of its branch (S_o[j] or S_x2[j]), and a flip upstream (LN^quant, QKV,
-    # X_attn) perturbs every accumulator of its row, so a row can collect a few flips.  With 8.4 M elements compared the
-    # bound for a single element is therefore a few branch LSBs plus the BF16 unit of the output, not 1e-2 of max|o|;
-    # what must hold is that such elements are rare and that the bulk agrees to BF16 rounding.
-    C = Lp["C"]
-    lsb = (np.asarray(C["S_x2"], dtype=np.float64) + np.asarray(C["S_o"], dtype=np.float64)).reshape(1, -1)
-    ulp = 2.0 ** -7 * np.maximum(np.abs(want), 2.0 ** -10)
-    stats = (float(d.max()), float(np.mean(d > 2 * ulp)), float(np.mean(d > lsb + 2 * ulp)))
-    assert np.all(d <= 3 * lsb + 2 * ulp), stats
-    assert np.mean(d > lsb + 2 * ulp) < 1e-5, stats
-    assert np.mean(d > 2 * ulp) < 1e-3, stats
-    assert float(d.mean() / np.abs(want).mean()) < 2e-3
-    assert rel_err(got, want) < 3e-2
+    hb = O.fp_tensor(x[rows], fd)
+    T = OL.layer_forward(Lp, hb, B=1)
+    got = out[rows].float().cpu().numpy().astype(np.float64)
+    # ---- stage by stage
+    x_in = _like(T["x_in"], bd.i8("x_in", H, rows), bd.f32("x_in_scale", rows))
+    _twq_close(x_in.data, x_in.row_scale, T["x_in"], "x_in")                     # same input on both sides
+    qkv = _like(T["qkv"], bd.i8("qkv", 3 * H, rows))
+    assert_int8_close(qkv.data, OL._linear(Lp["qkv"], x_in, "none").data, 1e-4, "qkv")
+    x_attn = _like(T["x_attn"], bd.i8("x_attn", H, rows))
+    assert_int8_close(x_attn.data, OL._attention(Lp, qkv, 1).data, 2e-4, "x_attn")
+    x_o = _like(T["x_o"], bd.i8("x_o", H, rows))
+    assert_int8_close(x_o.data, OL._linear(Lp["o"], x_attn, "none").data, 1e-4, "x_o")
+    x_mid = _like(T["x_mid"], bd.i8("x_mid", H, rows), bd.f32("x_mid_scale", rows))
+    h_mid = O.QT("fp", bd.fp("h_mid", H, rows, fd), dtype=fd)
+    want, want_h = O.ln_quant([hb, x_o], Lp["ln2_g"], Lp["ln2_b"], spec.eps, Lp["ln_mid_out"], fp_out_dtype=fd)
+    # the new residual stream is stored in BF16: equal up to one storage step where fp32 and fp64 sums round apart
+    ulp = 2.0 ** -7 * np.maximum(np.abs(want_h.real()), 2.0 ** -20)
+    dh_ = np.abs(h_mid.real() - want_h.real())
+    assert np.all(dh_ <= ulp) and np.mean(dh_ > 0) < 1e-3, (float(dh_.max()), float(np.mean(dh_ > 0)))
+    # LN^quant consumes the sum it stored: compare the INT8 side against the oracle applied to the device's stream
+    want2, _ = O.ln_quant([h_mid], Lp["ln2_g"], Lp["ln2_b"], spec.eps, Lp["ln_mid_out"])
+    _twq_close(x_mid.data, x_mid.row_scale, want2, "x_mid")
+    a = _like(T["a"], bd.i8("a", F, rows))
+    assert_int8_close(a.data, OL._linear(Lp["fc1"], x_mid, spec.act).data, 1e-4, "a")
+    x_2 = _like(T["x_2"], bd.i8("x_2", H, rows))
+    assert_int8_close(x_2.data, OL._linear(Lp["fc2"], a, "none").data, 1e-4, "x_2")
+    _, want_o = O.ln_quant([h_mid, x_2], None, None, spec.eps, None, fp_out_dtype=fd, normalize=False)
+    do = np.abs(got - want_o.real())
+    ulp = 2.0 ** -7 * np.maximum(np.abs(want_o.real()), 2.0 ** -20)
+    assert np.all(do <= ulp) and np.mean(do > 0) < 1e-3, (float(do.max()), float(np.mean(do > 0)))
+    # ---- end to end against the oracle's own chain: statistical (see the module docstring)
+    ref = T["h_out"].real()
+    d = np.abs(got - ref)
+    # (measured: about 8 % of the outputs sit one branch LSB, S_x2[j] ~ 0.07, away: mean |d| / mean |o| ~ 3e-3)
+    assert float(d.mean() / np.abs(ref).mean()) < 6e-3
+    assert rel_err(got, ref) < 3e-2
     h.close()
