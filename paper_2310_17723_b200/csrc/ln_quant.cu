@@ -832,6 +832,398 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
   return HERO_OK;
 }
 
+// ------------------------------------------------------------------------------------------------------
+// Rows of exactly 1024 * WPR elements (H = 1024, 2048, 4096, 8192): everything a row needs per element is
+// decided at compile time.  A lane owns two chunks of 16 consecutive elements (one 16-byte copy per INT8
+// chunk, two per FP16 / BF16 chunk), gamma and beta live in registers, the per-feature scale vectors of the
+// INT8 addends (and of a static INT8 output) are staged once per CTA in shared memory, and the row loop has
+// no parameter-dependent branch.  Same arithmetic, in the same order, as ln_fast_kernel.
+//   RES / BR : SRC_I8 | SRC_FP (| SRC_NONE for BR);  RSC: the INT8 residual carries a per-row scale (TWQ,
+//   RS_ROW) or a per-feature vector (FWQ / SQ, RS_COL);  an INT8 branch always carries a per-feature vector;
+//   BF: the FP tensors involved are BF16 (else FP16).
+// ------------------------------------------------------------------------------------------------------
+constexpr int RS_ROW = 0, RS_COL = 1;
+
+template <bool BF>
+__device__ __forceinline__ void fpx8_to_f2(const uint4 w, float2* v) {
+  const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if constexpr (BF) v[i] = make_float2(__uint_as_float(u[i] << 16), __uint_as_float(u[i] & 0xffff0000u));
+    else v[i] = __half22float2(*reinterpret_cast<const __half2*>(&u[i]));
+  }
+}
+template <bool BF>
+__device__ __forceinline__ uint32_t pack_fpx2(float a, float b) {
+  if constexpr (BF) { __nv_bfloat162 h = __floats2bfloat162_rn(a, b); return *reinterpret_cast<uint32_t*>(&h); }
+  else { __half2 h = __floats2half2_rn(a, b); return *reinterpret_cast<uint32_t*>(&h); }
+}
+__device__ __forceinline__ void i8x16_to_f2(const uint4 w, float2* v) {
+  float2 a[4], b[4];
+  i8x8_to_f2(w.x, w.y, a);
+  i8x8_to_f2(w.z, w.w, b);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { v[i] = a[i]; v[4 + i] = b[i]; }
+}
+__device__ __forceinline__ void lds_vec16(const float* s, float2* v) {   // 16 floats from shared memory
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 q = *reinterpret_cast<const float4*>(s + 4 * i);
+    v[2 * i] = make_float2(q.x, q.y); v[2 * i + 1] = make_float2(q.z, q.w);
+  }
+}
+
+// Ring depth of ln_wide_kernel: two CTAs per SM; deep enough that about 128 KB per SM are always on their way,
+// within 100 KB per CTA (ring + staged vectors).
+__host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes) {
+  int stages = 1 + (64 * 1024 + stage_bytes - 1) / stage_bytes;
+  if (stages < 3) stages = 3;
+  if (stages > 8) stages = 8;
+  while (stages > 3 && stages * stage_bytes + vec_bytes > 100 * 1024) --stages;
+  return stages;
+}
+
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR>
+__global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
+  constexpr int H = 1024 * WPR;
+  constexpr int SLOTS = 8 / WPR;                   // rows per CTA pass
+  constexpr int STRIDE = WPR * 32;                 // chunk stride between a lane's two chunks
+  constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2;
+  constexpr int ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
+  constexpr int OFF_BR = H * ES_RES;
+  constexpr int SLOT_BYTES = OFF_BR + H * ES_BR;
+  constexpr int STAGE_BYTES = SLOT_BYTES * SLOTS;
+  constexpr bool RES_CS = RES == SRC_I8 && RSC == RS_COL;
+  constexpr bool BR_CS = BR == SRC_I8;
+  constexpr bool OUT_CS = OUT == O_STATIC;
+  constexpr int VEC_BYTES = H * 4 * ((RES_CS ? 1 : 0) + (BR_CS ? 1 : 0) + (OUT_CS ? 1 : 0));
+  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES);   // ring depth
+  __shared__ float red[3][8][8];                   // [statistic][row slot][warp in row]
+  extern __shared__ __align__(16) uint8_t dyn[];
+  float* v_rcs = reinterpret_cast<float*>(dyn);
+  float* v_bcs = v_rcs + (RES_CS ? H : 0);
+  float* v_ocs = v_bcs + (BR_CS ? H : 0);
+  uint8_t* ring = reinterpret_cast<uint8_t*>(v_ocs + (OUT_CS ? H : 0));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int slot = warp / WPR, wr = warp % WPR;
+  const int c_first = wr * 32 + lane;              // this lane's first chunk (16-element units)
+  const float MAGIC = 12582912.0f;                 // 1.5 * 2^23
+  constexpr float fH = (float)H;
+
+  const char* g_res = reinterpret_cast<const char*>(p.res.data) + c_first * 16 * ES_RES;
+  const char* g_br = (BR != SRC_NONE) ? reinterpret_cast<const char*>(p.br.data) + c_first * 16 * ES_BR : nullptr;
+  const long long pitch_res = p.res.ld * ES_RES, pitch_br = (BR != SRC_NONE) ? p.br.ld * ES_BR : 0;
+  uint8_t* my_ring = ring + slot * SLOT_BYTES + c_first * 16 * ES_RES;          // residual part of this lane's slice
+  uint8_t* my_ring_br = ring + slot * SLOT_BYTES + OFF_BR + c_first * 16 * ES_BR;
+
+  // A lane copies exactly the chunks it will later read, so waiting on its own copy groups is all the
+  // synchronisation the ring needs.
+  auto prefetch = [&](long long row, int st) {
+    if (row < p.M) {                               // rows past the end still commit an (empty) group
+      const char* gr = g_res + row * pitch_res;
+      uint8_t* d = my_ring + st * STAGE_BYTES;
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+#pragma unroll
+        for (int q = 0; q < ES_RES; ++q) cp_async16(d + k * STRIDE * 16 * ES_RES + 16 * q, gr + k * STRIDE * 16 * ES_RES + 16 * q);
+      }
+      if constexpr (BR != SRC_NONE) {
+        const char* gb = g_br + row * pitch_br;
+        uint8_t* db = my_ring_br + st * STAGE_BYTES;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+#pragma unroll
+          for (int q = 0; q < ES_BR; ++q) cp_async16(db + k * STRIDE * 16 * ES_BR + 16 * q, gb + k * STRIDE * 16 * ES_BR + 16 * q);
+        }
+      }
+    }
+    cp_async_commit();
+  };
+
+  const long long row_step = (long long)gridDim.x * SLOTS;
+  const long long first = (long long)blockIdx.x * SLOTS + slot;
+  for (int s0 = 0; s0 < STAGES - 1; ++s0) prefetch(first + s0 * row_step, s0);
+
+  // per-feature vectors: shared memory for the scales, registers for gamma / beta
+  for (int i = threadIdx.x; i < H; i += LNF_THREADS) {
+    if constexpr (RES_CS) v_rcs[i] = __ldg(p.res.col_scale + i * p.res.col_stride);
+    if constexpr (BR_CS) v_bcs[i] = __ldg(p.br.col_scale + i * p.br.col_stride);
+    if constexpr (OUT_CS) v_ocs[i] = __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));
+  }
+  float2 gam[2][8], bet[2][8];
+  if constexpr (OUT != O_NONE) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int e0 = (c_first + k * STRIDE) * 16;
+      float2 t[4];
+      load_vec8(p.gamma + e0, t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) gam[k][i] = t[i];
+      load_vec8(p.gamma + e0 + 8, t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) gam[k][4 + i] = t[i];
+      load_vec8(p.beta + e0, t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) bet[k][i] = t[i];
+      load_vec8(p.beta + e0 + 8, t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) bet[k][4 + i] = t[i];
+    }
+  }
+  __syncthreads();
+
+  int st = 0;
+  // every slot walks its own rows: nothing in the loop is shared between slots (named barriers are per slot)
+  for (long long row = first; row < p.M; row += row_step) {
+    {
+      int pst = st + STAGES - 1;
+      if (pst >= STAGES) pst -= STAGES;
+      prefetch(row + (long long)(STAGES - 1) * row_step, pst);
+    }
+    float rs_res = 1.f;
+    if constexpr (RES == SRC_I8 && RSC == RS_ROW) { rs_res = __ldg(p.res.row_scale + row); }
+    cp_async_wait<STAGES - 1>();                   // this row's copies are the oldest group still pending
+    const uint8_t* src = my_ring + st * STAGE_BYTES;
+    const uint8_t* src_br = my_ring_br + st * STAGE_BYTES;
+    if (++st == STAGES) st = 0;
+
+    // ---- r = sum of the dequantized addends; running row sum
+    float2 x[2][8];
+    float2 s2 = f2(0.f);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      {
+        if constexpr (RES == SRC_I8) {
+          i8x16_to_f2(*reinterpret_cast<const uint4*>(src + k * STRIDE * 16), x[k]);
+          if constexpr (RSC == RS_COL) {
+            float2 sc[8];
+            lds_vec16(v_rcs + (c_first + k * STRIDE) * 16, sc);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[k][i] = __fmul2_rn(x[k][i], sc[i]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[k][i] = __fmul2_rn(x[k][i], f2(rs_res));
+          }
+        } else {
+          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src + k * STRIDE * 32), x[k]);
+          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src + k * STRIDE * 32 + 16), x[k] + 4);
+        }
+        if constexpr (BR == SRC_I8) {
+          float2 b[8], sc[8];
+          i8x16_to_f2(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 16), b);
+          lds_vec16(v_bcs + (c_first + k * STRIDE) * 16, sc);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
+        }
+        if constexpr (BR == SRC_FP) {
+          float2 b[8];
+          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 32), b);
+          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 32 + 16), b + 4);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[k][i] = __fadd2_rn(x[k][i], b[i]);
+        }
+        if constexpr (FPOUT) {
+          // the FP residual stream carries the ROUNDED sum; normalise what is stored
+          uint32_t w[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
+          char* dst = reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + (c_first + k * STRIDE) * 16) * 2;
+          st_global16(dst, w[0], w[1], w[2], w[3]);
+          st_global16(dst + 16, w[4], w[5], w[6], w[7]);
+          fpx8_to_f2<BF>(make_uint4(w[0], w[1], w[2], w[3]), x[k]);
+          fpx8_to_f2<BF>(make_uint4(w[4], w[5], w[6], w[7]), x[k] + 4);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s2 = __fadd2_rn(s2, x[k][i]);
+      }
+    }
+    if constexpr (OUT == O_NONE) continue;
+
+    // ---- mean (true division: a constant row must give exactly zero deviations)
+    float s = warp_sum(s2.x + s2.y);
+    if constexpr (WPR > 1) {
+      if (lane == 0) red[0][slot][wr] = s;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
+      s = 0.f;
+#pragma unroll
+      for (int w = 0; w < WPR; ++w) s += red[0][slot][w];
+    }
+    const float mean = s / fH;
+    // ---- centred (biased) variance over the registers
+    float2 q2 = f2(0.f);
+    const float2 nm = f2(-mean);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { x[k][i] = __fadd2_rn(x[k][i], nm); q2 = __ffma2_rn(x[k][i], x[k][i], q2); }
+    }
+    float q = warp_sum(q2.x + q2.y);
+    if constexpr (WPR > 1) {
+      if (lane == 0) red[1][slot][wr] = q;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
+      q = 0.f;
+#pragma unroll
+      for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
+    }
+    const float rstd = 1.0f / sqrtf(q / fH + p.eps);
+
+    // ---- y = d * (rstd * gamma) + beta ; TWQ: row absmax in the same sweep
+    float amax = 0.f;
+    const float2 r2 = f2(rstd);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(gam[k][i], r2), bet[k][i]);
+        if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fmaxf(fabsf(x[k][i].x), fabsf(x[k][i].y)));
+      }
+    }
+
+    if constexpr (OUT == O_TWQ) {
+      // Eq. 3: S[i] = absmax / 127 on the fly; the scaled value never leaves [-127, 127], so the magic add
+      // alone rounds and range-limits it
+      amax = warp_max(amax);
+      if constexpr (WPR > 1) {
+        if (lane == 0) red[2][slot][wr] = amax;
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
+        amax = 0.f;
+#pragma unroll
+        for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
+      }
+      const float sc = amax > 0.f ? amax / 127.0f : 1.0f;
+      const float2 inv2 = f2(1.0f / sc), mg2 = f2(MAGIC);
+      if (wr == 0 && lane == 0) p.out_scale[row] = sc;
+      {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          uint32_t w[4];
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const float2 a = __ffma2_rn(x[k][2 * g], inv2, mg2), b = __ffma2_rn(x[k][2 * g + 1], inv2, mg2);
+            w[g] = pack_low_bytes(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(b.x), __float_as_uint(b.y));
+          }
+          st_global16(reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * 16, w[0], w[1], w[2], w[3]);
+        }
+      }
+    } else if constexpr (OUT == O_STATIC) {
+      // Eq. 4 / 5: calibrated per-feature or static scale; saturating; true division as the definition has it
+      {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          float2 sc[8];
+          lds_vec16(v_ocs + (c_first + k * STRIDE) * 16, sc);
+          uint32_t w[4];
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const float a = fminf(fmaxf(x[k][2 * g].x / sc[2 * g].x, -127.f), 127.f) + MAGIC;
+            const float b = fminf(fmaxf(x[k][2 * g].y / sc[2 * g].y, -127.f), 127.f) + MAGIC;
+            const float c = fminf(fmaxf(x[k][2 * g + 1].x / sc[2 * g + 1].x, -127.f), 127.f) + MAGIC;
+            const float d = fminf(fmaxf(x[k][2 * g + 1].y / sc[2 * g + 1].y, -127.f), 127.f) + MAGIC;
+            w[g] = pack_low_bytes(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d));
+          }
+          st_global16(reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * 16, w[0], w[1], w[2], w[3]);
+        }
+      }
+    } else {
+      {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          uint32_t w[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
+          char* dst = reinterpret_cast<char*>(p.out) + (row * p.out_ld + (c_first + k * STRIDE) * 16) * 2;
+          st_global16(dst, w[0], w[1], w[2], w[3]);
+          st_global16(dst + 16, w[4], w[5], w[6], w[7]);
+        }
+      }
+    }
+  }
+  cp_async_wait<0>();
+}
+
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR>
+static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream) {
+  constexpr int H = 1024 * WPR, SLOTS = 8 / WPR;
+  constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2, ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
+  constexpr size_t STAGE = (size_t)SLOTS * H * (ES_RES + ES_BR);
+  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0));
+  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC);
+  const size_t smem = (size_t)stages * STAGE + VEC;
+  auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR>;
+  static bool configured = false;   // per instantiation
+  if (!configured) {
+    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    configured = true;
+  }
+  static int occ = 0;               // per instantiation: the launch configuration never changes
+  if (occ < 1) {
+    HERO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, LNF_THREADS, smem));
+    if (occ < 1) occ = 1;
+  }
+  const long long want = (p.M + SLOTS - 1) / SLOTS;
+  const long long cap = (long long)h->sm_count * occ;
+  const int grid = (int)(want < cap ? want : cap);
+  {
+    LaunchScope scope(h, stream, KERNEL_LN);
+    kern<<<grid, LNF_THREADS, smem, stream>>>(p);
+  }
+  HERO_CUDA(cudaGetLastError());
+  return HERO_OK;
+}
+
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF>
+static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) {
+  switch (p.H) {
+    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1>(h, p, s);
+    case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2>(h, p, s);
+    case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4>(h, p, s);
+    default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8>(h, p, s);
+  }
+}
+
+// The combinations the layer forward produces on rows of 1024 * {1, 2, 4, 8} elements.
+static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
+  *taken = false;
+  if (!(p.H == 1024 || p.H == 2048 || p.H == 4096 || p.H == 8192) || p.ex.data || p.token_ids) return HERO_OK;
+  const int res = p.res.dt == HERO_I8 ? SRC_I8 : SRC_FP;
+  const int br = !p.br.data ? SRC_NONE : (p.br.dt == HERO_I8 ? SRC_I8 : SRC_FP);
+  const int out = !p.out ? O_NONE : (p.out_dt != HERO_I8 ? O_FP : (p.out_gran == HERO_GRAN_TWQ ? O_TWQ : O_STATIC));
+  const bool fpo = p.fp_out != nullptr;
+  // scale kinds the kernel is specialised for
+  int rsc = RS_ROW;
+  if (res == SRC_I8) {
+    if (p.res.row_scale && !p.res.col_scale) rsc = RS_ROW;
+    else if (!p.res.row_scale && p.res.col_scale) rsc = RS_COL;
+    else return HERO_OK;
+  }
+  if (br == SRC_I8 && (p.br.row_scale || !p.br.col_scale)) return HERO_OK;
+  if (out == O_STATIC && !(p.out_gran == HERO_GRAN_FWQ || p.out_gran == HERO_GRAN_SQ)) return HERO_OK;
+  // one FP type across the call
+  int fpt = -1;
+  auto fp_ok = [&](bool used, int dt) { if (!used) return true; if (fpt < 0) fpt = dt; return fpt == dt; };
+  if (!fp_ok(res == SRC_FP, p.res.dt) || !fp_ok(br == SRC_FP, p.br.dt) || !fp_ok(out == O_FP, p.out_dt) || !fp_ok(fpo, p.fp_dt))
+    return HERO_OK;
+  const bool bf = fpt == HERO_BF16;
+#define LNW_CASE(R_, S_, B_, O_, F_)                                                                 \
+  if (res == R_ && (R_ != SRC_I8 || rsc == S_) && br == B_ && out == O_ && fpo == F_) {               \
+    *taken = true;                                                                                   \
+    return bf ? launch_wide_wpr<R_, S_, B_, O_, F_, true>(h, p, s) : launch_wide_wpr<R_, S_, B_, O_, F_, false>(h, p, s); \
+  }
+  LNW_CASE(SRC_I8, RS_COL, SRC_I8, O_TWQ, false)      // Eq. 19: FWQ / SQ residual + FWQ branch -> TWQ
+  LNW_CASE(SRC_I8, RS_ROW, SRC_I8, O_TWQ, false)      // Eq. 31: TWQ residual + FWQ branch -> TWQ
+  LNW_CASE(SRC_I8, RS_COL, SRC_I8, O_STATIC, false)
+  LNW_CASE(SRC_I8, RS_ROW, SRC_I8, O_STATIC, false)
+  LNW_CASE(SRC_I8, RS_COL, SRC_I8, O_FP, false)
+  LNW_CASE(SRC_I8, RS_ROW, SRC_I8, O_FP, false)
+  LNW_CASE(SRC_FP, RS_ROW, SRC_NONE, O_TWQ, false)    // entry LN^quant / pre-LN LN1
+  LNW_CASE(SRC_FP, RS_ROW, SRC_NONE, O_STATIC, false)
+  LNW_CASE(SRC_FP, RS_ROW, SRC_I8, O_TWQ, true)       // pre-LN: add + LN + quant, new residual stream stored
+  LNW_CASE(SRC_FP, RS_ROW, SRC_I8, O_STATIC, true)
+  LNW_CASE(SRC_FP, RS_ROW, SRC_I8, O_NONE, true)      // closing residual add of a lone pre-LN layer
+#undef LNW_CASE
+  return HERO_OK;
+}
+
 // Returns HERO_ERR_UNSUPPORTED (without setting an error) when the combination has no fast instantiation.
 static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
@@ -934,6 +1326,8 @@ extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* 
   if (p.M == 0) return HERO_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   bool taken = false;
+  st = try_wide(h, p, s, &taken);
+  if (taken || st != HERO_OK) return st;
   st = try_fast(h, p, s, &taken);
   if (taken || st != HERO_OK) return st;
   // generic kernel for the remaining combinations.
