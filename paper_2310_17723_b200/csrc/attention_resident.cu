@@ -148,6 +148,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();                                       // the previous kernel's outputs are complete and visible from here on
 
   if (warp == ATT_TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer: Q, K blocks, V blocks in P V order
@@ -480,7 +482,7 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
   const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);
   {
     LaunchScope scope(h, stream, KERNEL_ATTN);
-    kern<<<grid, ATT_THREADS, Cfg::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+    HERO_CUDA(launch_dependent(kern, dim3(grid), dim3(ATT_THREADS), Cfg::SMEM_BYTES, stream, tq, tk, tv, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;

@@ -72,6 +72,31 @@ struct LaunchScope {
   ~LaunchScope() { if (slot >= 0) cudaEventRecord(h->prof_ev[2 * slot + 1], s); }
 };
 
+// Kernel launch with programmatic dependent launch allowed: the grid may be scheduled while the previous kernel of
+// the stream is still draining, runs its set-up (barrier init, tensor-memory allocation, descriptor prefetch) and then
+// blocks in griddepcontrol.wait until that kernel has completed and its writes are visible.  Every kernel of the
+// library executes griddepcontrol.launch_dependents first thing and griddepcontrol.wait before its first global
+// memory access, so launch latency and ramp-up overlap the predecessor's tail and nothing else changes.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+#ifdef __CUDACC__
+namespace ptx {
+// launch_dependents: the next kernel of the stream may start being scheduled.  wait: returns once the previous kernel
+// of the stream has completed and flushed its writes (immediately if there is none or the launch was an ordinary one).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+}  // namespace ptx
+#endif
+
 // 2-D TMA descriptor over a row-major matrix [rows, cols] of `elem_bytes` elements with row pitch
 // ld_bytes; box = box_cols x box_rows elements; swizzle_bytes in {0, 32, 64, 128}.
 hero_status make_tmap_2d(const hero_handle* h, CUtensorMap* out, const void* base, int elem_bytes, bool is_fp16,

@@ -374,6 +374,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();                                       // the previous kernel's outputs are complete and visible from here on
 
   if (warp == TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
@@ -455,7 +457,7 @@ static hero_status launch_gemm(hero_handle* h, const CUtensorMap& tmA, const CUt
   const int grid = tiles < h->sm_count ? tiles : h->sm_count;
   {
     LaunchScope scope(h, stream, KERNEL_GEMM);
-    kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+    HERO_CUDA(launch_dependent(kern, dim3(grid), dim3(GEMM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmW, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
@@ -544,6 +546,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   ptx::cluster_sync();                                   // both CTAs' barriers exist before any remote arrive
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();                                       // the previous kernel's outputs are complete and visible from here on
 
   if (warp == EW) {
     // ------------------------------------------------------------------ TMA producer (leader CTA only)
@@ -631,7 +635,7 @@ static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, c
   const int pairs = tiles < pairs_max ? tiles : pairs_max;
   {
     LaunchScope scope(h, stream, KERNEL_GEMM);
-    kern<<<2 * pairs, (EW + 2) * 32, PairCfg::SMEM_BYTES, stream>>>(tmA, tmW, p);
+    HERO_CUDA(launch_dependent(kern, dim3(2 * pairs), dim3((EW + 2) * 32), PairCfg::SMEM_BYTES, stream, tmA, tmW, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;

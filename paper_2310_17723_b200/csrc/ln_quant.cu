@@ -145,6 +145,8 @@ __device__ __forceinline__ void row_reduce(float (&v)[R], float* red, int G, int
 
 template <int VEC, int R, bool HAS_BR, bool HAS_EX>
 __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();                                 // the previous kernel's outputs are complete and visible
   extern __shared__ float red_smem[];
   const int G = p.G, RPC = p.RPC, H = p.H;
   const int nw = G >> 5;
@@ -378,7 +380,7 @@ static hero_status launch_ln2(hero_handle* h, LnParams& p, cudaStream_t stream) 
   if (grid < 1) grid = 1;
   {
     LaunchScope scope(h, stream, KERNEL_LN);
-    ln_quant_kernel<VEC, R, HAS_BR, HAS_EX><<<grid, threads, smem, stream>>>(p);
+    HERO_CUDA(launch_dependent(ln_quant_kernel<VEC, R, HAS_BR, HAS_EX>, dim3(grid), dim3(threads), smem, stream, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
@@ -494,6 +496,8 @@ __device__ __forceinline__ void fp16x8_to_f2(uint32_t w0, uint32_t w1, uint32_t 
 // NCHX = exact number of 8-element chunks per lane (H = 256 * WPR * NCHX, no tail predicates), or 0 for any H.
 template <int RES, int BR, bool EX, int OUT, bool FPOUT, int NCHX>
 __global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams p) {
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();                                 // the previous kernel's outputs are complete and visible
   constexpr int KMAX = NCHX ? NCHX : LNF_MAXCH;
   // gamma / beta (and, with at most 3 chunks per lane, the branch's per-feature scale) stay in registers for
   // the whole persistent row loop of the exact-size variants; otherwise they are re-read through L1 per row
@@ -826,7 +830,7 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
   const int grid = (int)(want < cap ? want : cap);
   {
     LaunchScope scope(h, stream, KERNEL_LN);
-    kern<<<grid, LNF_THREADS, smem, stream>>>(p);
+    HERO_CUDA(launch_dependent(kern, dim3(grid), dim3(LNF_THREADS), smem, stream, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
@@ -885,6 +889,8 @@ __host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes)
 
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR>
 __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();                                 // the previous kernel's outputs are complete and visible
   constexpr int H = 1024 * WPR;
   constexpr int SLOTS = 8 / WPR;                   // rows per CTA pass
   constexpr int STRIDE = WPR * 32;                 // chunk stride between a lane's two chunks
@@ -1165,7 +1171,7 @@ static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream)
   const int grid = (int)(want < cap ? want : cap);
   {
     LaunchScope scope(h, stream, KERNEL_LN);
-    kern<<<grid, LNF_THREADS, smem, stream>>>(p);
+    HERO_CUDA(launch_dependent(kern, dim3(grid), dim3(LNF_THREADS), smem, stream, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
