@@ -157,12 +157,12 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
     }
   } else {
     float v[NC];
+    float hi = -INFINITY, lo = INFINITY;
     const float2 rs2 = make_float2(rs, rs), mg2 = make_float2(ROUND_MAGIC, ROUND_MAGIC);
 #pragma unroll
     for (int j = 0; j < NC; j += 4) {
       const float4 cs4 = *reinterpret_cast<const float4*>(e_cs + j);
       const float4 b4 = *reinterpret_cast<const float4*>(e_bias + j);
-      const float4 p4 = *reinterpret_cast<const float4*>(e_post + j);
       float2 a0, a1;
       if constexpr (INT8) {
         a0 = make_float2((float)(int)r[j], (float)(int)r[j + 1]);
@@ -173,22 +173,37 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
       }
       float2 x0 = __ffma2_rn(__fmul2_rn(a0, rs2), make_float2(cs4.x, cs4.y), make_float2(b4.x, b4.y));
       float2 x1 = __ffma2_rn(__fmul2_rn(a1, rs2), make_float2(cs4.z, cs4.w), make_float2(b4.z, b4.w));
-      if constexpr (ACT == HERO_ACT_GELU_ERF) { x0 = gelu_erf_f2(x0); x1 = gelu_erf_f2(x1); }
-      if constexpr (ACT == HERO_ACT_GELU_TANH) {
-        x0.x = gelu_tanh_f(x0.x); x0.y = gelu_tanh_f(x0.y); x1.x = gelu_tanh_f(x1.x); x1.y = gelu_tanh_f(x1.y);
-      }
-      if constexpr (OUTK == OUT_I8) {
-        // Round (half to even) and clip in the float adder: 1.5 * 2^23 + k keeps k in its low byte
-        const float2 y0 = __ffma2_rn(x0, make_float2(p4.x, p4.y), mg2);
-        const float2 y1 = __ffma2_rn(x1, make_float2(p4.z, p4.w), mg2);
-        v[j] = fminf(fmaxf(y0.x, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
-        v[j + 1] = fminf(fmaxf(y0.y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
-        v[j + 2] = fminf(fmaxf(y1.x, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
-        v[j + 3] = fminf(fmaxf(y1.y, ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
+      float2 y0, y1;
+      if constexpr (ACT == HERO_ACT_NONE) {
+        // without an activation the output factor is already folded into cs and bias (see epilogue_loop)
+        if constexpr (OUTK == OUT_I8) { y0 = __fadd2_rn(x0, mg2); y1 = __fadd2_rn(x1, mg2); }
+        else { y0 = x0; y1 = x1; }
       } else {
-        const float2 y0 = __fmul2_rn(x0, make_float2(p4.x, p4.y));
-        const float2 y1 = __fmul2_rn(x1, make_float2(p4.z, p4.w));
-        v[j] = y0.x; v[j + 1] = y0.y; v[j + 2] = y1.x; v[j + 3] = y1.y;
+        const float4 p4 = *reinterpret_cast<const float4*>(e_post + j);
+        if constexpr (ACT == HERO_ACT_GELU_ERF) { x0 = gelu_erf_f2(x0); x1 = gelu_erf_f2(x1); }
+        if constexpr (ACT == HERO_ACT_GELU_TANH) {
+          x0.x = gelu_tanh_f(x0.x); x0.y = gelu_tanh_f(x0.y); x1.x = gelu_tanh_f(x1.x); x1.y = gelu_tanh_f(x1.y);
+        }
+        if constexpr (OUTK == OUT_I8) {
+          y0 = __ffma2_rn(x0, make_float2(p4.x, p4.y), mg2);
+          y1 = __ffma2_rn(x1, make_float2(p4.z, p4.w), mg2);
+        } else {
+          y0 = __fmul2_rn(x0, make_float2(p4.x, p4.y));
+          y1 = __fmul2_rn(x1, make_float2(p4.z, p4.w));
+        }
+      }
+      v[j] = y0.x; v[j + 1] = y0.y; v[j + 2] = y1.x; v[j + 3] = y1.y;
+      if constexpr (OUTK == OUT_I8) {
+        // Round (half to even) happened in the float adder: 1.5 * 2^23 + k keeps k in its low byte.  The clip to
+        // [-127, 127] is applied only if some value of the chunk needs it.
+        hi = fmaxf(fmaxf(hi, fmaxf(y0.x, y0.y)), fmaxf(y1.x, y1.y));
+        lo = fminf(fminf(lo, fminf(y0.x, y0.y)), fminf(y1.x, y1.y));
+      }
+    }
+    if constexpr (OUTK == OUT_I8) {
+      if (hi > ROUND_MAGIC + 127.0f || lo < ROUND_MAGIC - 127.0f) {
+#pragma unroll
+        for (int j = 0; j < NC; ++j) v[j] = fminf(fmaxf(v[j], ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
       }
     }
     if (!row_ok) return;
@@ -304,7 +319,11 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
       float* e = epi_w + (it & 1) * 3 * CH;
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
-        e[i * 32 + lane] = ncs[i]; e[CH + i * 32 + lane] = nbias[i]; e[2 * CH + i * 32 + lane] = npost[i];
+        if constexpr (ACT == HERO_ACT_NONE) {    // (acc rs cs + b) post = acc rs (cs post) + b post
+          e[i * 32 + lane] = ncs[i] * npost[i]; e[CH + i * 32 + lane] = nbias[i] * npost[i];
+        } else {
+          e[i * 32 + lane] = ncs[i]; e[CH + i * 32 + lane] = nbias[i]; e[2 * CH + i * 32 + lane] = npost[i];
+        }
       }
       __syncwarp();
     }
