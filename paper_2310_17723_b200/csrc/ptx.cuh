@@ -39,23 +39,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)  // suspend-time hint in ns: sleep in hardware, not in a poll loop
       : "memory");
   return ok != 0;
 }
 
-constexpr uint32_t WAIT_LIMIT = 1u << 22;  // polls; each try_wait itself blocks for a hardware time slice
+constexpr uint32_t WAIT_LIMIT = 1u << 18;  // polls; each try_wait sleeps in hardware for up to 20 us, so about 5 s in all
 
 // Bounded wait.  Returns false (after recording `code`) when the barrier never flipped.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err_word, int code) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;   // try_wait itself suspends the thread for a hardware time slice
-    if (i > (1u << 16)) __nanosleep(256);           // only a wait that is already hopelessly long backs off
-  }
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
+    if (mbar_try_wait(bar, parity)) return true;   // wakes as soon as the phase completes
   if (err_word) atomicExch(err_word, code);
   return false;
 }
