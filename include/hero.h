@@ -181,6 +181,9 @@ typedef struct {
   int32_t mask;        /* hero_mask */
   const int32_t* key_len;
   hero_tensor out;     /* [B*S, nh*dh]; I8 with gran FWQ (scale[H]) or SQ (scale[1]); or F16 / BF16 */
+  float* p_absmax;     /* optional, F16 / BF16 core only: device float[1] holding a running maximum (the caller zeroes
+                          it once); after the call it is max(old, largest softmax probability seen), from which
+                          calibration takes s_p = p_absmax / 255 (Eq. 16).  NULL: not observed. */
 } hero_attn_args;
 
 hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream);
@@ -223,6 +226,32 @@ typedef struct {
   const float* ln1_g; const float* ln1_b;
   const float* ln2_g; const float* ln2_b;
 } hero_layer_desc;
+
+/* ---------------------------------------------------------------------------------------------
+ * Calibration on the device (Sec. 2.1: the static scales of Eq. 4-5 come from statistics of the un-quantized
+ * layer over calibration data; Eq. 2 and Eq. 20-23 / 32 for the weights).  Run the layer's modules in FP mode
+ * through the entry points above and observe every tensor at an operator border with hero_absmax_observe
+ * (the softmax probabilities through hero_attn_args.p_absmax); a scale is absmax / 127 (absmax / 255 for P),
+ * 1 when the statistic is 0.
+ *
+ * hero_absmax_observe: running absolute maxima of x ([rows, cols] F16 / BF16, cols and ld multiples of 8).
+ *   col_absmax    : device float[cols] or NULL: col_absmax[j] = max(col_absmax[j], max_i |x[i][j]|)   (Eq. 4)
+ *   tensor_absmax : device float[1]    or NULL: max(old, max_ij |x[i][j]|)                            (Eq. 5)
+ *   Both accumulate, so several calibration batches can be observed one after another; zero them first.
+ *
+ * hero_quantize_weight: fold, then column-wise symmetric INT8 (Eq. 2 after Eq. 20-23 / 32), for W [N][K] FP32
+ * (row n = output feature n; K, ldw, ldq multiples of 4):
+ *     W~[n][k] = W[n][k] * in_scale[k] / out_scale[n]      in_scale [K] or NULL (the consumer-side fold of the
+ *                                                          input's FWQ / SQ scale), out_scale [N] or NULL (the
+ *                                                          producer-side fold of the output's scale)
+ *     w_scale[n] = max_k |W~[n][k]| / 127  (1 if the row is zero);   Wq[n][k] = clip(Round(W~[n][k] / w_scale[n]))
+ *     bias_out[n] = bias[n] / out_scale[n]                 when bias_out is given (bias NULL reads as 0)
+ *   All pointers are device pointers; outputs are caller-owned.  The paper gives the equations, not an interface. */
+hero_status hero_absmax_observe(hero_handle* h, const hero_tensor* x, float* col_absmax, float* tensor_absmax,
+                                void* stream);
+hero_status hero_quantize_weight(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K,
+                                 const float* in_scale, const float* out_scale, const float* bias, int8_t* Wq,
+                                 int64_t ldq, float* w_scale, float* bias_out, void* stream);
 
 /* Fill desc->mode from a Table 1 preset (M1, M2, M3) or all-FP. */
 hero_status hero_mode_preset(int32_t preset, int32_t mode_out[5]);

@@ -428,6 +428,8 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   p.mask = a->mask; p.key_len = a->key_len;
   p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
   p.err = h->d_error;
+  p.p_absmax = a->p_absmax;
+  HERO_REQUIRE(a->p_absmax == nullptr || fp_in, HERO_ERR_UNSUPPORTED, "p_absmax is observed by the F16 / BF16 attention core only");
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (fp_in) return attn_fp_dispatch(h, a, p, s);

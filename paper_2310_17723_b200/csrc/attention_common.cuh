@@ -32,6 +32,7 @@ struct AttnParams {
   int out_dt;
   uint32_t idesc_qk, idesc_pv;
   int* err;
+  float* p_absmax;         // calibration observer of the FP core: running max of the softmax probabilities, or NULL
 };
 
 __device__ __forceinline__ float ex2f(float x) {

@@ -236,6 +236,13 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         m = mf; l = lf;
       }
       const float inv_l = l > 0.f ? 1.0f / l : 0.f;
+      if (p.p_absmax != nullptr && cq == 0) {
+        // calibration observer (Eq. 16: S_p = max P / 255): the largest probability of a row is 2^0 / l
+        float pm = row_ok ? inv_l : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, o));
+        if (lane == 0 && pm > 0.f) atomicMax(reinterpret_cast<unsigned int*>(p.p_absmax), __float_as_uint(pm));
+      }
 
       // ---- sweep 2: P = 2^(t - m) / l as FP16 / BF16 into shared memory (two 64-key sub-tiles, 128-byte swizzle)
       for (int j = 0; j < nkv; ++j, ++scnt, ++pcnt) {

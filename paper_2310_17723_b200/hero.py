@@ -56,7 +56,7 @@ class AttnArgs(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("dtype", C.c_int32), ("ld", C.c_int64),
                 ("B", C.c_int32), ("S", C.c_int32), ("nh", C.c_int32), ("dh", C.c_int32), ("s_q", C.c_float),
                 ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float), ("mask", C.c_int32),
-                ("key_len", C.c_void_p), ("out", Tensor)]
+                ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p)]
 
 
 class LinearParams(C.Structure):
@@ -82,7 +82,7 @@ class LayerLayout(C.Structure):
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
-           "hero_profile_end", "hero_layer_forward_static")
+           "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight")
 
 _lib = None
 
@@ -106,6 +106,9 @@ def lib():
         L.hero_int8_attention.argtypes = [C.c_void_p, C.POINTER(AttnArgs), C.c_void_p]
         L.hero_mode_preset.argtypes = [C.c_int32, C.POINTER(C.c_int32 * 5)]
         L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
+        L.hero_absmax_observe.argtypes = [C.c_void_p, C.POINTER(Tensor), C.c_void_p, C.c_void_p, C.c_void_p]
+        L.hero_quantize_weight.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.hero_layer_workspace_layout.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(LayerLayout)]
         L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -192,12 +195,24 @@ class Handle:
         _check(lib().hero_w8a8_linear(self._h, C.byref(a), _stream(stream)))
 
     def hero_int8_attention(self, q, k, v, B, S, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0, s_p=1.0 / 255,
-                            mask="none", key_len=None, stream=None):
-        """q, k, v: 2-D torch views [B*S, nh*dh] sharing one leading dimension; out: hero.Tensor."""
+                            mask="none", key_len=None, p_absmax=None, stream=None):
+        """q, k, v: 2-D torch views [B*S, nh*dh] sharing one leading dimension; out: hero.Tensor; p_absmax: float32[1]
+        running maximum of the softmax probabilities (F16 / BF16 core only)."""
         assert q.stride(0) == k.stride(0) == v.stride(0) and q.dtype == k.dtype == v.dtype
         a = AttnArgs(q.data_ptr(), k.data_ptr(), v.data_ptr(), _DT[q.dtype], q.stride(0), B, S, nh, dh, s_q, s_k,
-                     s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out)
+                     s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out, _ptr(p_absmax))
         _check(lib().hero_int8_attention(self._h, C.byref(a), _stream(stream)))
+
+    def hero_absmax_observe(self, x, col_absmax=None, tensor_absmax=None, stream=None):
+        """x: hero.Tensor (F16 / BF16); col_absmax float32[cols] / tensor_absmax float32[1]: running maxima, updated."""
+        _check(lib().hero_absmax_observe(self._h, C.byref(x), _ptr(col_absmax), _ptr(tensor_absmax), _stream(stream)))
+
+    def hero_quantize_weight(self, W, Wq, w_scale, in_scale=None, out_scale=None, bias=None, bias_out=None, stream=None):
+        """W: float32 [N, K]; Wq: int8 [N, K]; w_scale: float32 [N]; optional folds in_scale [K], out_scale [N]."""
+        assert W.dim() == 2 and W.stride(1) == 1 and Wq.stride(1) == 1 and W.dtype == torch.float32 and Wq.dtype == torch.int8
+        _check(lib().hero_quantize_weight(self._h, C.c_void_p(W.data_ptr()), W.stride(0), W.shape[0], W.shape[1],
+                                          _ptr(in_scale), _ptr(out_scale), _ptr(bias), C.c_void_p(Wq.data_ptr()),
+                                          Wq.stride(0), _ptr(w_scale), _ptr(bias_out), _stream(stream)))
 
     def hero_layer_workspace_bytes(self, desc, M):
         n = C.c_size_t()

@@ -3,6 +3,8 @@
     python -m paper_2310_17723_b200.microbench ln   --M 65536 --H 1024 --kind i8       # LN^quant GB/s
     python -m paper_2310_17723_b200.microbench gemm --M 8192 --K 4096 --N 4096        # GeMM^quant TOP/s
     python -m paper_2310_17723_b200.microbench attn --B 8 --S 384 --nh 16 --dh 64     # INT8 attention
+    python -m paper_2310_17723_b200.microbench absmax --M 65536 --H 4096             # calibration observer GB/s
+    python -m paper_2310_17723_b200.microbench wquant --N 4096 --K 4096              # fold + Eq. 2 weight quantization GB/s
     ... --sweep runs the standalone-kernel sweep of the benchmark configurations instead of one shape.
 
 Inputs are synthetic and larger than L2 (several rotating buffers), times are CUDA events around `--iters` launches.
@@ -96,9 +98,35 @@ def bench_attn(h, B, S, nh, dh, mask, iters):
           % (B, S, nh, dh, mask, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12), flush=True)
 
 
+def bench_absmax(h, M, H, iters):
+    """Per-feature and per-tensor absmax of an FP16 tensor: one read of 2 bytes per element."""
+    n = max(2, min(16, int(400e6 // (M * H * 2)) + 1))
+    xs = [torch.randn(M, H, device="cuda", dtype=torch.float16) for _ in range(n)]
+    cf, ct = torch.zeros(H, device="cuda"), torch.zeros(1, device="cuda")
+    t = _time(lambda i: h.hero_absmax_observe(hero.tensor(xs[i]), cf, ct), n, iters)
+    hbm, _, src = _peaks()
+    gbs = M * H * 2 / t / 1e9
+    print("absmax observer f16 M=%d H=%d: %.1f us, %.0f GB/s (algorithmic 2 B/element), %.2f of %s copy bandwidth"
+          % (M, H, t * 1e6, gbs, gbs / hbm, src), flush=True)
+
+
+def bench_wquant(h, N, K, iters):
+    """W~ = Diag(in) W Diag(1/out), Eq. 2: 4 bytes read (the second sweep hits L2) + 1 written per weight."""
+    n = max(2, min(8, int(400e6 // (N * K * 5)) + 1))
+    Ws = [torch.randn(N, K, device="cuda") * 0.02 for _ in range(n)]
+    Wq = [torch.empty(N, K, device="cuda", dtype=torch.int8) for _ in range(n)]
+    si, so = torch.rand(K, device="cuda") * 0.05 + 0.01, torch.rand(N, device="cuda") * 0.05 + 0.01
+    ws, b, bo = torch.empty(N, device="cuda"), torch.randn(N, device="cuda"), torch.empty(N, device="cuda")
+    t = _time(lambda i: h.hero_quantize_weight(Ws[i], Wq[i], ws, in_scale=si, out_scale=so, bias=b, bias_out=bo), n, iters)
+    hbm, _, src = _peaks()
+    gbs = N * K * 5 / t / 1e9
+    print("weight fold + quantize N=%d K=%d: %.1f us, %.0f GB/s (algorithmic 5 B/weight), %.2f of %s copy bandwidth"
+          % (N, K, t * 1e6, gbs, gbs / hbm, src), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["ln", "gemm", "attn"])
+    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant"])
     ap.add_argument("--M", type=int, default=65536)
     ap.add_argument("--H", type=int, default=1024)
     ap.add_argument("--K", type=int, default=4096)
@@ -129,6 +157,10 @@ def main():
                     bench_gemm(h, M, K, N, a.act, a.fp, a.iters)
         else:
             bench_gemm(h, a.M, a.K, a.N, a.act, a.fp, a.iters)
+    elif a.kernel == "absmax":
+        bench_absmax(h, a.M, a.H, a.iters)
+    elif a.kernel == "wquant":
+        bench_wquant(h, a.N, a.K, a.iters)
     else:
         bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters)
     h.check()

@@ -173,9 +173,11 @@ def _store_fp(W, fp_dtype):
     return u.astype(np.uint16)          # bfloat16 bit patterns
 
 
-def prepare_layer(cfg: LayerConfig, params, C):
+def prepare_layer(cfg: LayerConfig, params, C, fold_quantize_fn=None):
     """Host arrays for one layer: per linear module {W, w_scale, bias, post_scale}, LN parameters, and the
-    activation scales the kernels read.  `C` comes from `calibrate`."""
+    activation scales the kernels read.  `C` comes from `calibrate`.  `fold_quantize_fn(W, b, in_scale, out_scale)`
+    replaces the host-side fold + Eq. 2 quantization (the device version lives in calibrate.py)."""
+    fq = fold_quantize_fn or fold_quantize
     p = {k: np.asarray(v, np.float64) for k, v in params.items()}
     H, m = cfg.H, cfg.mode
     in_vec = _gran_vec(cfg.gran_in, C["S_in_f"], C["S_in_t"], H)
@@ -189,7 +191,7 @@ def prepare_layer(cfg: LayerConfig, params, C):
     def linear(W, b, int8, in_scale, out_fold, post):
         g = {"int8": int8, "post_scale": None if post is None else _f32(post)}
         if int8:
-            g["W"], g["w_scale"], g["bias"] = fold_quantize(W, b, in_scale, out_fold)
+            g["W"], g["w_scale"], g["bias"] = fq(W, b, in_scale, out_fold)
         else:
             g["W"], g["w_scale"], g["bias"] = _store_fp(W, cfg.fp_dtype), None, _f32(b)
         return g
