@@ -33,8 +33,8 @@ struct AttnResCfg {
   static constexpr int OFF_P = OFF_V + VST * TILE;
   static constexpr int OFF_STATS = OFF_P + RES_NP * P_TILE;
   static constexpr int OFF_PM = OFF_STATS + 2 * 4 * ATT_BM * 8;        // per-thread piece maxima [RES_NB][512] x 2 halves
-  static constexpr int OFF_OSC = OFF_PM + RES_NB * 512 * 8;            // per-tile output factors [2][128]
-  static constexpr int OFF_BARS = OFF_OSC + 2 * 128 * 4;
+  static constexpr int OFF_OSC = OFF_PM + RES_NB * 512 * 8;            // per-tile output factors [lane quarter][2][128]
+  static constexpr int OFF_BARS = OFF_OSC + 4 * 2 * 128 * 4;
   static constexpr int NBARS = 4 + 2 * KST + 2 * VST + 2 * RES_NB + 2 * RES_NP + 2;
   static constexpr int SMEM_BYTES = 1024 + OFF_BARS + NBARS * 8 + 16;
   static constexpr uint32_t SWZ = (DH == 128) ? ptx::SWZ_128B : ptx::SWZ_64B;
@@ -290,7 +290,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 
     auto epilogue = [&]() {
       res_epilogue<DH>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
-                       osc_s + ((wcnt - 1) & 1) * 128, ok);
+                       osc_s + quarter * 256 + ((wcnt - 1) & 1) * 128, ok);
       pend = false;
     };
 
@@ -305,8 +305,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       const int q = q0 + r_loc;
       const bool row_ok = q < p.S;
       float osc_raw = 1.f;                                   // this thread's S_attn[j], turned into a factor further down
-      if (p.out_dt == HERO_I8 && (int)threadIdx.x < DH)
-        osc_raw = __ldg(p.out_scale + (long long)(col0 + (int)threadIdx.x) * p.out_scale_stride);
+      if (p.out_dt == HERO_I8 && cq * 32 + lane < DH)
+        osc_raw = __ldg(p.out_scale + (long long)(col0 + cq * 32 + lane) * p.out_scale_stride);
       if (nkv == 0) {
         // every key masked: the rows are zero, no tensor work
         if (cq * 32 < DH && row_ok) {
@@ -352,10 +352,10 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
               for (int e = 4; e < 16; e += 4) { i0 = max(i0, max((int)r[e], (int)r[e + 1])); i1 = max(i1, max((int)r[e + 2], (int)r[e + 3])); }
               mp = (float)max(i0, i1) * c2;
               float2 acc2 = make_float2(0.f, 0.f);
-              const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-mp, -mp), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
+              const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-mp, -mp);
 #pragma unroll
               for (int e = 0; e < 16; e += 2) {
-                const float2 f = __fadd2_rn(make_float2(__uint_as_float(0x4B400000u + r[e]), __uint_as_float(0x4B400000u + r[e + 1])), mg);
+                const float2 f = make_float2((float)(int)r[e], (float)(int)r[e + 1]);
                 const float2 tt = __ffma2_rn(f, c22, nm2);
                 const float2 ev = make_float2(ex2f(tt.x), ex2f(tt.y));
                 acc2 = __fadd2_rn(acc2, ev);
@@ -381,8 +381,9 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
       st[cq * ATT_BM + r_loc] = make_float2(m, l);
-      if ((int)threadIdx.x < DH) osc_s[(wcnt & 1) * 128 + threadIdx.x] = p.pv_scale / osc_raw;
-      asm volatile("bar.sync 1, 512;" ::: "memory");
+      if (cq * 32 + lane < DH) osc_s[quarter * 256 + (wcnt & 1) * 128 + cq * 32 + lane] = p.pv_scale / osc_raw;
+      // the four warps that share these 32 rows (one per column group) meet; the other lane quarters are not involved
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter) : "memory");
       {
         float mf = -INFINITY;
 #pragma unroll

@@ -134,6 +134,13 @@ __device__ __forceinline__ void st32(void* p, const uint32_t (&w)[8]) {   // 256
                : "memory");
 }
 
+// 16 bytes from shared memory through the shared window (a generic load would take the slower generic path)
+__device__ __forceinline__ float4 lds_f4(const float* p) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(ptx::smem_u32(p)));
+  return v;
+}
+
 // NC (16 or 32) columns of one output row: v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];
 // INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.  Per-column vectors come from shared memory four at a time,
 // the arithmetic runs on packed FP32 pairs, the row segment leaves in 32-byte stores when the output allows it.
@@ -161,8 +168,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
     const float2 rs2 = make_float2(rs, rs), mg2 = make_float2(ROUND_MAGIC, ROUND_MAGIC);
 #pragma unroll
     for (int j = 0; j < NC; j += 4) {
-      const float4 cs4 = *reinterpret_cast<const float4*>(e_cs + j);
-      const float4 b4 = *reinterpret_cast<const float4*>(e_bias + j);
+      const float4 cs4 = lds_f4(e_cs + j), b4 = lds_f4(e_bias + j);
       float2 a0, a1;
       if constexpr (INT8) {
         a0 = make_float2((float)(int)r[j], (float)(int)r[j + 1]);
@@ -179,7 +185,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
         if constexpr (OUTK == OUT_I8) { y0 = __fadd2_rn(x0, mg2); y1 = __fadd2_rn(x1, mg2); }
         else { y0 = x0; y1 = x1; }
       } else {
-        const float4 p4 = *reinterpret_cast<const float4*>(e_post + j);
+        const float4 p4 = lds_f4(e_post + j);
         if constexpr (ACT == HERO_ACT_GELU_ERF) { x0 = gelu_erf_f2(x0); x1 = gelu_erf_f2(x1); }
         if constexpr (ACT == HERO_ACT_GELU_TANH) {
           x0.x = gelu_tanh_f(x0.x); x0.y = gelu_tanh_f(x0.y); x1.x = gelu_tanh_f(x1.x); x1.y = gelu_tanh_f(x1.y);
