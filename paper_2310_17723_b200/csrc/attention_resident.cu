@@ -52,20 +52,16 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
                                           const float* osc, bool& ok) {
   constexpr int CW = DH / 4;
   uint32_t r[CW];
+  // A wait that gives up has recorded its code; the warp then runs on without waiting again (what it computes no
+  // longer matters, every access stays in bounds) so that the kernel ends promptly.
   if (ok && !ptx::mbar_wait(o_full, parity, p.err, 0x9300)) ok = false;
   ptx::tc_fence_after();
-  if (ok) {
-    if constexpr (CW == 16) ptx::tmem_ld16(t_lane + RES_O_COL + cq * CW, r);
-    else ptx::tmem_ld32(t_lane + RES_O_COL + cq * CW, r);
-    ptx::tmem_ld_wait();
-  }
+  if constexpr (CW == 16) ptx::tmem_ld16(t_lane + RES_O_COL + cq * CW, r);
+  else ptx::tmem_ld32(t_lane + RES_O_COL + cq * CW, r);
+  ptx::tmem_ld_wait();
   ptx::tc_fence_before();
   __syncwarp();
   if (lane == 0) ptx::mbar_arrive(o_empty);
-  if (!ok) {
-#pragma unroll
-    for (int e = 0; e < CW; ++e) r[e] = 0;
-  }
   if (pend_row >= 0) {
     const int gcol = pend_col + cq * CW;
     const float4* o4 = reinterpret_cast<const float4*>(osc + cq * CW);
@@ -328,7 +324,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         if (j == 3 && pend) epilogue();                      // block 3's columns hold the previous tile's output
         if (ok && !ptx::mbar_wait(&s_full[j], (used >> j) & 1, p.err, 0x9000 | j)) ok = false;
         ptx::tc_fence_after();
-        if (ok) {
+        {
           const uint32_t ta = t_lane + j * ATT_BN + cq * 32;
           const int kb = j * ATT_BN + cq * 32;
           float mpa[2];
@@ -372,11 +368,9 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             mpa[hh] = mp;
           }
           pm2[j * 512] = make_float2(mpa[0], mpa[1]);
-        } else {
-          pm2[j * 512] = make_float2(-INFINITY, -INFINITY);
         }
       }
-      if (ok) ptx::tmem_st_wait();
+      ptx::tmem_st_wait();
       if (pend) epilogue();
       // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
@@ -406,7 +400,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         const int j = res_pv_block(nkv, i);
         const int pb = pcnt % RES_NP;
         if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt / RES_NP) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
-        if (ok) {
+        {
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
           const float2 mp2 = pm2[j * 512];
           const int c16 = cq * 2;
