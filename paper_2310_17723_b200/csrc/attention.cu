@@ -209,7 +209,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int sb = scnt % ATT_NSB;
         if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x3000 | sb)) ok = false;
         ptx::tc_fence_after();
-        if (ok) {
+        {
           uint32_t r[32];
           ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
           ptx::tmem_ld_wait();
@@ -273,7 +273,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x3100 | sb)) ok = false;
         if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt >> 1) & 1) ^ 1, p.err, 0x3200 | pb)) ok = false;
         ptx::tc_fence_after();
-        if (ok) {
+        {
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
           uint32_t r[32];
           ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
@@ -314,7 +314,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (nkv > 0) {
         if (ok && !ptx::mbar_wait(o_full, wcnt & 1, p.err, 0x3300)) ok = false;
         ptx::tc_fence_after();
-        if (ok && cq * 32 < DH) {
+        if (cq * 32 < DH) {
           ptx::tmem_ld32(t_lane + Cfg::O_COL + cq * 32, r);
           ptx::tmem_ld_wait();
         }
@@ -323,7 +323,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (lane == 0) ptx::mbar_arrive(o_empty);              // the accumulator may be overwritten by the next tile
         ++wcnt;
       }
-      if (nkv == 0 || !ok) {
+      if (nkv == 0) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) r[j] = 0;                 // every key masked: the row is zero
       }

@@ -196,7 +196,7 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int sb = scnt % ATT_NSB;
         if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x6000 | sb)) ok = false;
         ptx::tc_fence_after();
-        if (ok) {
+        {
           uint32_t r[32];
           ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
           ptx::tmem_ld_wait();
@@ -250,7 +250,7 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x6100 | sb)) ok = false;
         if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt / PB) & 1) ^ 1, p.err, 0x6200 | pb)) ok = false;
         ptx::tc_fence_after();
-        if (ok) {
+        {
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (cq >> 1) * Cfg::SUB + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
           uint32_t r[32];
           ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
@@ -282,7 +282,7 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       if (nkv > 0) {
         if (ok && !ptx::mbar_wait(o_full, wcnt & 1, p.err, 0x6300)) ok = false;
         ptx::tc_fence_after();
-        if (ok && cq * 32 < DH) {
+        if (cq * 32 < DH) {
           ptx::tmem_ld32(t_lane + Cfg::O_COL + cq * 32, r);
           ptx::tmem_ld_wait();
         }
@@ -291,7 +291,7 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (lane == 0) ptx::mbar_arrive(o_empty);
         ++wcnt;
       }
-      if (nkv == 0 || !ok) {
+      if (nkv == 0) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) r[j] = 0;
       }

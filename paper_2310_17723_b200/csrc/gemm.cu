@@ -349,9 +349,10 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     const int m = mt * ROWS + row_off + quarter * 32 + lane;
     const bool row_ok = m < p.M;
 
+    // a wait that gave up has recorded its code; the warp runs on without waiting again so that the kernel ends promptly
     if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
     ptx::tc_fence_after();
-    if (ok) {
+    {
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + cpart * CH;
       epilogue_columns<BN, INT8, ACT, OUTK, EW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart);
     }
