@@ -949,6 +949,14 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   const long long row_step = (long long)gridDim.x * SLOTS;
   const long long first = (long long)blockIdx.x * SLOTS + slot;
   for (int s0 = 0; s0 < STAGES - 1; ++s0) prefetch(first + s0 * row_step, s0);
+  // the per-row scale of a TWQ residual travels STAGES - 1 rows ahead as well, in a register ring: lane i of a warp
+  // holds the scale of the i-th row ahead (STAGES <= 8 < 32)
+  constexpr bool ROW_SC = RES == SRC_I8 && RSC == RS_ROW;
+  float rs_ring = 1.f;
+  if constexpr (ROW_SC) {
+    const long long r = first + (long long)lane * row_step;
+    if (lane < STAGES - 1 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+  }
 
   // per-feature vectors: shared memory for the scales, registers for gamma / beta
   for (int i = threadIdx.x; i < H; i += LNF_THREADS) {
@@ -987,7 +995,13 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
       prefetch(row + (long long)(STAGES - 1) * row_step, pst);
     }
     float rs_res = 1.f;
-    if constexpr (RES == SRC_I8 && RSC == RS_ROW) { rs_res = __ldg(p.res.row_scale + row); }
+    if constexpr (ROW_SC) {
+      // this row's scale sits in lane 0; shift the ring by one lane and let lane STAGES - 2 fetch the newest row's
+      rs_res = __shfl_sync(0xffffffffu, rs_ring, 0);
+      rs_ring = __shfl_down_sync(0xffffffffu, rs_ring, 1);
+      const long long r = row + (long long)(STAGES - 1) * row_step;
+      if (lane == STAGES - 2 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+    }
     cp_async_wait<STAGES - 1>();                   // this row's copies are the oldest group still pending
     const uint8_t* src = my_ring + st * STAGE_BYTES;
     const uint8_t* src_br = my_ring_br + st * STAGE_BYTES;
