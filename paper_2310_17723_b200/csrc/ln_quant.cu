@@ -869,10 +869,12 @@ __device__ __forceinline__ void i8x16_to_f2(const uint4 w, float2* v) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) { v[i] = a[i]; v[4 + i] = b[i]; }
 }
-__device__ __forceinline__ void lds_vec16(const float* s, float2* v) {   // 16 floats from shared memory
+// 16 floats of one chunk from a piece-major vector in shared memory: piece i of chunk c at float4 index i * NCHUNK + c
+template <int NCHUNK>
+__device__ __forceinline__ void lds_vec16(const float* s, float2* v) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float4 q = *reinterpret_cast<const float4*>(s + 4 * i);
+    const float4 q = *reinterpret_cast<const float4*>(s + 4 * i * NCHUNK);
     v[2 * i] = make_float2(q.x, q.y); v[2 * i + 1] = make_float2(q.z, q.w);
   }
 }
@@ -959,10 +961,13 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   }
 
   // per-feature vectors: shared memory for the scales, registers for gamma / beta
+  // stored piece-major ([float4 piece q of a chunk][chunk]): consecutive lanes then read consecutive 16-byte words,
+  // free of bank conflicts
   for (int i = threadIdx.x; i < H; i += LNF_THREADS) {
-    if constexpr (RES_CS) v_rcs[i] = __ldg(p.res.col_scale + i * p.res.col_stride);
-    if constexpr (BR_CS) v_bcs[i] = __ldg(p.br.col_scale + i * p.br.col_stride);
-    if constexpr (OUT_CS) v_ocs[i] = __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));
+    const int si = (((i >> 2) & 3) * (H / 16) + (i >> 4)) * 4 + (i & 3);
+    if constexpr (RES_CS) v_rcs[si] = __ldg(p.res.col_scale + i * p.res.col_stride);
+    if constexpr (BR_CS) v_bcs[si] = __ldg(p.br.col_scale + i * p.br.col_stride);
+    if constexpr (OUT_CS) v_ocs[si] = __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));
   }
   float2 gam[2][8], bet[2][8];
   if constexpr (OUT != O_NONE) {
@@ -1017,7 +1022,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
           i8x16_to_f2(*reinterpret_cast<const uint4*>(src + k * STRIDE * 16), x[k]);
           if constexpr (RSC == RS_COL) {
             float2 sc[8];
-            lds_vec16(v_rcs + (c_first + k * STRIDE) * 16, sc);
+            lds_vec16<H / 16>(v_rcs + (c_first + k * STRIDE) * 4, sc);
 #pragma unroll
             for (int i = 0; i < 8; ++i) x[k][i] = __fmul2_rn(x[k][i], sc[i]);
           } else {
@@ -1031,7 +1036,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
         if constexpr (BR == SRC_I8) {
           float2 b[8], sc[8];
           i8x16_to_f2(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 16), b);
-          lds_vec16(v_bcs + (c_first + k * STRIDE) * 16, sc);
+          lds_vec16<H / 16>(v_bcs + (c_first + k * STRIDE) * 4, sc);
 #pragma unroll
           for (int i = 0; i < 8; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
         }
@@ -1131,7 +1136,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           float2 sc[8];
-          lds_vec16(v_ocs + (c_first + k * STRIDE) * 16, sc);
+          lds_vec16<H / 16>(v_ocs + (c_first + k * STRIDE) * 4, sc);
           uint32_t w[4];
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
