@@ -220,7 +220,7 @@ def gemm_fp(x: QT, W, bias, act, out: OutSpec, carried=None):
 # attention core (Eq. 15-17)
 # --------------------------------------------------------------------------------------
 def attention_int8(q_i8, k_i8, v_i8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutSpec,
-                   mask="none", key_len=None, return_internals=False):
+                   mask="none", key_len=None, return_internals=False, p_mode="static"):
     """INT8 attention.  q_i8/k_i8/v_i8: [B*S, nh*dh] int8 (SQ, scalar scales s_q, s_k, s_v).
 
     per (b, h):  A = d~ (Q K^T),  d~ = s_q s_k / sqrt(dh)   -- never quantized
@@ -228,7 +228,15 @@ def attention_int8(q_i8, k_i8, v_i8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutS
                  P_u8 = clip(Round(P / s_p), 0, 255)       -- asymmetric (unsigned) INT8
                  acc = P_u8 V_int8                          -- exact INT32
                  X_attn = s_p s_v acc                       -> output stage (FWQ / SQ / FP)
+
+    p_mode="rowmax" (not in the paper; the long-sequence-robust variant): the un-normalised probabilities are
+    quantized against their row maximum instead of the normalised ones against a static scale,
+                 e = exp(A - max_row A) over the allowed keys (masked: 0),   l = sum_row e
+                 P~_u8 = clip(Round(255 e), 0, 255)        -- the largest key of every row gets 255
+                 acc = P~_u8 V_int8,   X_attn = s_v acc / (255 l)
+    so nothing underflows however many keys share the mass; s_p is unused.
     """
+    assert p_mode in ("static", "rowmax")
     H = nh * dh
     d_tilde = float(s_q) * float(s_k) / np.sqrt(float(dh))
     x_attn = np.zeros((B * S, H), dtype=np.float64)
@@ -239,10 +247,20 @@ def attention_int8(q_i8, k_i8, v_i8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutS
         for h in range(nh):
             cols = slice(h * dh, (h + 1) * dh)
             A = d_tilde * int_matmul(q_i8[rows, cols], k_i8[rows, cols].T).astype(np.float64)
-            P = softmax_masked(A, allowed)
-            P_u8 = Q.quant_unsigned(P, s_p)
-            acc = int_matmul(P_u8, v_i8[rows, cols])
-            x_attn[rows, cols] = float(s_p) * float(s_v) * acc.astype(np.float64)
+            if p_mode == "static":
+                P = softmax_masked(A, allowed)
+                P_u8 = Q.quant_unsigned(P, s_p)
+                acc = int_matmul(P_u8, v_i8[rows, cols])
+                x_attn[rows, cols] = float(s_p) * float(s_v) * acc.astype(np.float64)
+            else:
+                neg = np.where(allowed, A, -np.inf)
+                m = np.max(neg, axis=-1, keepdims=True)
+                m = np.where(np.isfinite(m), m, 0.0)
+                e = np.where(allowed, np.exp(neg - m), 0.0)
+                l = np.sum(e, axis=-1, keepdims=True)
+                P_u8 = Q.quant_unsigned(e, 1.0 / Q.PMAX)
+                acc = int_matmul(P_u8, v_i8[rows, cols])
+                x_attn[rows, cols] = np.where(l > 0.0, float(s_v) * acc.astype(np.float64) / (Q.PMAX * np.where(l > 0.0, l, 1.0)), 0.0)
             if return_internals:
                 internals["P_u8"][(b, h)] = P_u8
                 internals["acc"][(b, h)] = acc

@@ -1,4 +1,5 @@
 """Pins for oracle/ops.py: brute force, closed forms and library routines (CPU only)."""
+import math
 import os
 
 import numpy as np
@@ -165,6 +166,59 @@ def test_attention_int8_tracks_fp_attention():
     got = O.attention_int8(qi, ki, vi, B, S, nh, dh, s_q, s_k, s_v, 1.0 / 255, O.OutSpec("fp", dtype="f64")).data
     ref = O.attention_fp(qi * s_q, ki * s_k, vi * s_v, B, S, nh, dh, O.OutSpec("fp", dtype="f64")).data
     assert np.max(np.abs(got - ref)) / np.max(np.abs(ref)) < 0.05
+
+
+def test_attention_int8_rowmax_variant_closed_forms_and_brute_force():
+    """The row-max-normalised P quantizer (the long-sequence-robust variant): closed forms and a scalar re-derivation."""
+    g = np.random.default_rng(70)
+    # uniform logits: e = 1 for every key -> P~ = 255, l = S -> X_attn = s_v * mean(V), for ANY S (the static
+    # quantizer rounds 1/S to zero beyond 510 keys)
+    for S in (128, 640, 1024):
+        nh, dh = 1, 8
+        q = np.zeros((S, dh), np.int8)
+        k = g.integers(-127, 128, (S, dh), dtype=np.int8)
+        v = g.integers(-127, 128, (S, dh), dtype=np.int8)
+        o, it = O.attention_int8(q, k, v, 1, S, nh, dh, 0.1, 0.1, 0.03, 1.0 / 255, O.OutSpec("fp", dtype="f64"),
+                                 return_internals=True, p_mode="rowmax")
+        assert np.all(it["P_u8"][(0, 0)] == 255)
+        assert np.allclose(o.data, np.broadcast_to(0.03 * v.astype(np.float64).mean(0), o.data.shape), rtol=1e-13)
+    stat = O.attention_int8(q, k, v, 1, S, nh, dh, 0.1, 0.1, 0.03, 1.0 / 255, O.OutSpec("fp", dtype="f64")).data
+    assert not stat.any()                           # the paper-literal quantizer has lost all the mass at S = 1024
+    # causal row 0 sees only key 0: P~ = [255, 0, ...], l = 1 -> X_attn[0] = s_v V[0]
+    S, dh = 16, 8
+    q, k, v = (g.integers(-127, 128, (S, dh), dtype=np.int8) for _ in range(3))
+    o = O.attention_int8(q, k, v, 1, S, 1, dh, 0.05, 0.05, 0.02, 1.0, O.OutSpec("fp", dtype="f64"), mask="causal", p_mode="rowmax")
+    assert np.allclose(o.data[0], 0.02 * v[0].astype(np.float64), rtol=1e-13)
+    # scalar re-derivation, key lengths included
+    S, nh, dh, klen = 12, 2, 4, 9
+    q, k, v = (g.integers(-127, 128, (S, nh * dh), dtype=np.int8) for _ in range(3))
+    s_q, s_k, s_v = 0.021, 0.017, 0.013
+    o = O.attention_int8(q, k, v, 1, S, nh, dh, s_q, s_k, s_v, 1.0, O.OutSpec("fp", dtype="f64"), mask="causal",
+                         key_len=np.array([klen]), p_mode="rowmax").data
+    for i in range(S):
+        for h in range(nh):
+            keys = [j for j in range(S) if j <= i and j < klen]
+            a = [s_q * s_k / math.sqrt(dh) * sum(int(q[i, h * dh + d]) * int(k[j, h * dh + d]) for d in range(dh)) for j in keys]
+            m = max(a)
+            e = [math.exp(x - m) for x in a]
+            pu = [min(255, max(0, round(255 * x))) for x in e]          # no ties at these magnitudes
+            for d in range(dh):
+                want = s_v * sum(p_ * int(v[j, h * dh + d]) for p_, j in zip(pu, keys)) / (255 * sum(e))
+                assert abs(o[i, h * dh + d] - want) <= 1e-12 * max(1.0, abs(want))
+
+
+def test_attention_int8_rowmax_tracks_fp_attention_better_at_long_sequences():
+    g = np.random.default_rng(71)
+    B, S, nh, dh = 1, 768, 1, 16
+    qf, kf, vf = (g.standard_normal((B * S, dh)) * c for c in (0.3, 0.3, 1.0))      # flat attention over many keys
+    s_q, s_k, s_v = (np.abs(a).max() / 127 for a in (qf, kf, vf))
+    qi, ki, vi = Q.quant_sq(qf, s_q), Q.quant_sq(kf, s_k), Q.quant_sq(vf, s_v)
+    ref = O.attention_fp(qi * s_q, ki * s_k, vi * s_v, B, S, nh, dh, O.OutSpec("fp", dtype="f64")).data
+    err = {}
+    for mode in ("static", "rowmax"):
+        got = O.attention_int8(qi, ki, vi, B, S, nh, dh, s_q, s_k, s_v, 1.0 / 255, O.OutSpec("fp", dtype="f64"), p_mode=mode).data
+        err[mode] = np.max(np.abs(got - ref)) / np.max(np.abs(ref))
+    assert err["rowmax"] < 0.02 and err["rowmax"] < 0.2 * err["static"], err
 
 
 # ------------------------------------------------------------------ GeMM^quant
