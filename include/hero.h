@@ -170,6 +170,13 @@ hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* st
  *             limits the keys of sequence b to k < key_len[b].  A fully masked row outputs 0.
  *   dh is 64 or 128.
  */
+/* How the INT8 core quantizes the softmax output.
+ *   HERO_P_STATIC (the paper, Eq. 16): P_u8 = clip(Round(P / s_p)) of the normalised probabilities, s_p calibrated.
+ *   HERO_P_ROWMAX (not in the paper; robust to long sequences, where probabilities below s_p / 2 vanish under the
+ *     static scale): P~_u8 = Round(255 * exp(A - max_row A)), row sum l of the un-quantized exponentials in FP32,
+ *     out = acc * s_v / (255 * l); s_p is ignored.  Sequences of up to 512 keys in this version. */
+typedef enum { HERO_P_STATIC = 0, HERO_P_ROWMAX = 1 } hero_p_mode;
+
 typedef struct {
   const void* q;
   const void* k;
@@ -184,6 +191,7 @@ typedef struct {
   float* p_absmax;     /* optional, F16 / BF16 core only: device float[1] holding a running maximum (the caller zeroes
                           it once); after the call it is max(old, largest softmax probability seen), from which
                           calibration takes s_p = p_absmax / 255 (Eq. 16).  NULL: not observed. */
+  int32_t p_mode;      /* hero_p_mode: how P is quantized (INT8 core only); 0 = the paper's static scale */
 } hero_attn_args;
 
 hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream);

@@ -411,7 +411,7 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   if (a->out.dtype == HERO_I8)
     HERO_REQUIRE((a->out.gran == HERO_GRAN_FWQ || a->out.gran == HERO_GRAN_SQ) && a->out.scale, HERO_ERR_UNSUPPORTED,
                  "INT8 X_attn is feature-wise (FWQ) or static (SQ) with a calibrated scale (Sec. 2.2.2)");
-  HERO_REQUIRE(fp_in || (a->s_q > 0 && a->s_k > 0 && a->s_v > 0 && a->s_p > 0), HERO_ERR_INVALID_ARG, "scales must be positive");
+  HERO_REQUIRE(fp_in || (a->s_q > 0 && a->s_k > 0 && a->s_v > 0 && (a->s_p > 0 || a->p_mode == HERO_P_ROWMAX)), HERO_ERR_INVALID_ARG, "scales must be positive");
   HERO_REQUIRE(a->mask == HERO_MASK_NONE || a->mask == HERO_MASK_CAUSAL, HERO_ERR_INVALID_ARG, "unknown mask %d", a->mask);
   HERO_REQUIRE(fp_in || (int64_t)a->S * 255 * 127 < (1ll << 31), HERO_ERR_UNSUPPORTED, "S=%d would overflow the INT32 accumulator", a->S);
   if (a->B == 0) return HERO_OK;
@@ -421,8 +421,11 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   p.B = a->B; p.S = a->S; p.nh = a->nh; p.dh = a->dh;
   p.nqt = (a->S + ATT_BM - 1) / ATT_BM;
   p.c2 = (float)((double)a->s_q * (double)a->s_k / sqrt((double)a->dh) * 1.4426950408889634);
-  p.inv_sp = 1.0f / a->s_p;
-  p.pv_scale = a->s_p * a->s_v;
+  HERO_REQUIRE(a->p_mode == HERO_P_STATIC || a->p_mode == HERO_P_ROWMAX, HERO_ERR_INVALID_ARG, "unknown p_mode %d", a->p_mode);
+  const bool rowmax = !fp_in && a->p_mode == HERO_P_ROWMAX;
+  HERO_REQUIRE(!rowmax || a->S <= 512, HERO_ERR_UNSUPPORTED, "p_mode ROWMAX handles sequences of up to 512 keys");
+  p.inv_sp = rowmax ? 255.0f : 1.0f / a->s_p;
+  p.pv_scale = rowmax ? a->s_v / 255.0f : a->s_p * a->s_v;
   p.out_scale = a->out.dtype == HERO_I8 ? a->out.scale : nullptr;
   p.out_scale_stride = a->out.gran == HERO_GRAN_FWQ ? 1 : 0;
   p.mask = a->mask; p.key_len = a->key_len;

@@ -49,7 +49,7 @@ struct AttnResCfg {
 template <int DH>
 __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, uint64_t* o_full, uint64_t* o_empty,
                                           uint32_t parity, int cq, int lane, long long pend_row, int pend_col,
-                                          const float* osc, bool& ok) {
+                                          const float* osc, float rowf, bool& ok) {
   constexpr int CW = DH / 4;
   uint32_t r[CW];
   // A wait that gives up has recorded its code; the warp then runs on without waiting again (what it computes no
@@ -74,10 +74,10 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
         for (int k = 0; k < 4; ++k) {
           const float4 sc = o4[4 * g + k];
           const int c = 16 * g + 4 * k;
-          const float a = fminf(fmaxf((float)(int)r[c] * sc.x, -127.f), 127.f) + ATT_MAGIC;
-          const float b = fminf(fmaxf((float)(int)r[c + 1] * sc.y, -127.f), 127.f) + ATT_MAGIC;
-          const float cc = fminf(fmaxf((float)(int)r[c + 2] * sc.z, -127.f), 127.f) + ATT_MAGIC;
-          const float d = fminf(fmaxf((float)(int)r[c + 3] * sc.w, -127.f), 127.f) + ATT_MAGIC;
+          const float a = fminf(fmaxf((float)(int)r[c] * rowf * sc.x, -127.f), 127.f) + ATT_MAGIC;
+          const float b = fminf(fmaxf((float)(int)r[c + 1] * rowf * sc.y, -127.f), 127.f) + ATT_MAGIC;
+          const float cc = fminf(fmaxf((float)(int)r[c + 2] * rowf * sc.z, -127.f), 127.f) + ATT_MAGIC;
+          const float d = fminf(fmaxf((float)(int)r[c + 3] * rowf * sc.w, -127.f), 127.f) + ATT_MAGIC;
           w[k] = low_bytes4_u(a, b, cc, d);                  // low byte of magic + x = two's-complement Round(x)
         }
         st_g16(dst + 16 * g, w[0], w[1], w[2], w[3]);
@@ -88,7 +88,7 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
       for (int g = 0; g < CW / 8; ++g) {
         float v[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * p.pv_scale;
+        for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * rowf * p.pv_scale;
         st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
                fp2(v[6], v[7], p.out_dt));
       }
@@ -96,7 +96,10 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
   }
 }
 
-template <int DH>
+// ROWMAX: the long-sequence-robust P quantizer (not in the paper): P~_u8 = Round(255 * 2^(t - m_row)) with the row sum
+// l of the un-quantized 2^(t - m_row) kept in FP32 and divided out in the epilogue.  Sweep 1 then only finds the row
+// maximum (integer compares, nothing written back), sweep 2 does the one exponential per score.
+template <int DH, bool ROWMAX>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnParams p) {
@@ -282,11 +285,12 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     bool ok = true;
     long long pend_row = -1;                                 // output row of the tile whose epilogue is pending
     int pend_col = 0;
+    float pend_rowf = 1.f;
     bool pend = false;
 
     auto epilogue = [&]() {
       res_epilogue<DH>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
-                       osc_s + quarter * 256 + ((wcnt - 1) & 1) * 128, ok);
+                       osc_s + quarter * 256 + ((wcnt - 1) & 1) * 128, pend_rowf, ok);
       pend = false;
     };
 
@@ -317,8 +321,38 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       int kmax = klen - 1;
       if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
 
-      // ---- sweep 1: per piece, e = 2^(t - m_piece) written back over the scores; running (m, l) in registers
       float m = -INFINITY, l = 0.f;
+      if constexpr (ROWMAX) {
+        // ---- sweep 1: the row maximum of the integer scores (the scale d~ log2 e is positive); nothing is written back
+        int imax = -(1 << 21);                               // below every real score (|t| <= 127^2 * 128 < 2^21)
+#pragma unroll 1
+        for (int j = 0; j < nkv; ++j) {
+          if (j == 3 && pend) epilogue();                    // block 3's columns hold the previous tile's output
+          if (ok && !ptx::mbar_wait(&s_full[j], (used >> j) & 1, p.err, 0x9000 | j)) ok = false;
+          ptx::tc_fence_after();
+          const uint32_t ta = t_lane + j * ATT_BN + cq * 32;
+          const int kb = j * ATT_BN + cq * 32;
+          uint32_t ra[16], rb[16];
+          ptx::tmem_ld16(ta, ra);
+          ptx::tmem_ld16(ta + 16, rb);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t (&r)[16] = hh ? rb : ra;
+            const int nvalid = min(16, kmax - (kb + 16 * hh) + 1);
+            if (nvalid < 16) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) if (e >= nvalid) r[e] = (uint32_t)(-(1 << 21));
+            }
+            int i0 = max((int)r[0], (int)r[1]), i1 = max((int)r[2], (int)r[3]);
+#pragma unroll
+            for (int e = 4; e < 16; e += 4) { i0 = max(i0, max((int)r[e], (int)r[e + 1])); i1 = max(i1, max((int)r[e + 2], (int)r[e + 3])); }
+            imax = max(imax, max(i0, i1));
+          }
+        }
+        m = (float)imax;                                     // exchanged as an (exact) integer-valued float
+      } else {
+      // ---- sweep 1: per piece, e = 2^(t - m_piece) written back over the scores; running (m, l) in registers
 #pragma unroll 1
       for (int j = 0; j < nkv; ++j) {
         if (j == 3 && pend) epilogue();                      // block 3's columns hold the previous tile's output
@@ -370,7 +404,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           pm2[j * 512] = make_float2(mpa[0], mpa[1]);
         }
       }
-      ptx::tmem_st_wait();
+      }
+      if constexpr (!ROWMAX) ptx::tmem_st_wait();
       if (pend) epilogue();
       // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
@@ -378,7 +413,14 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       if (cq * 32 + lane < DH) osc_s[quarter * 256 + (wcnt & 1) * 128 + cq * 32 + lane] = p.pv_scale / osc_raw;
       // the four warps that share these 32 rows (one per column group) meet; the other lane quarters are not involved
       asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter) : "memory");
-      {
+      float pscale = 0.f;
+      if constexpr (ROWMAX) {
+        float mf = st[r_loc].x;
+#pragma unroll
+        for (int g = 1; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
+        // a row without any allowed key: +inf makes every exponential exactly 0
+        m = mf <= (float)(-(1 << 21)) ? INFINITY : mf * c2;
+      } else {
         float mf = -INFINITY;
 #pragma unroll
         for (int g = 0; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
@@ -391,8 +433,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           }
         }
         m = mf; l = lf;
+        pscale = l > 0.f ? p.inv_sp / l : 0.f;
       }
-      const float pscale = l > 0.f ? p.inv_sp / l : 0.f;
 
       // ---- sweep 2: P_u8 = Round(e * 2^(m_piece - m) / (l s_p)), clipped to 255, into the UMMA operand tile
 #pragma unroll 1
@@ -402,12 +444,41 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         if (ok && !ptx::mbar_wait(&p_empty[pb], ((pcnt / RES_NP) & 1) ^ 1, p.err, 0x9200 | pb)) ok = false;
         {
           const uint32_t prow = ptx::smem_u32(sP + pb * Cfg::P_TILE) + (r_loc >> 3) * 1024 + (r_loc & 7) * 128;
-          const float2 mp2 = pm2[j * 512];
           const int c16 = cq * 2;
           uint32_t ra[16], rb[16];
           ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32, ra);
           ptx::tmem_ld16(t_lane + j * ATT_BN + cq * 32 + 16, rb);
           ptx::tmem_ld_wait();
+          if constexpr (ROWMAX) {
+            // P~_u8 = Round(255 * 2^(t - m)): at most 255, no clip; the un-quantized exponentials are summed for l
+            const int kb = j * ATT_BN + cq * 32;
+            const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m, -m);
+            const float2 s255 = make_float2(255.0f, 255.0f), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
+            float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+              uint32_t (&r)[16] = g ? rb : ra;
+              const int nvalid = min(16, kmax - (kb + 16 * g) + 1);
+              if (nvalid < 16) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) if (e >= nvalid) r[e] = (uint32_t)(-(1 << 21));   // 2^(very negative) = 0
+              }
+              uint32_t w[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int e = 4 * k;
+                const float2 ta = __ffma2_rn(make_float2((float)(int)r[e], (float)(int)r[e + 1]), c22, nm2);
+                const float2 tb = __ffma2_rn(make_float2((float)(int)r[e + 2], (float)(int)r[e + 3]), c22, nm2);
+                const float2 ea = make_float2(ex2f(ta.x), ex2f(ta.y)), eb = make_float2(ex2f(tb.x), ex2f(tb.y));
+                acc2 = __fadd2_rn(acc2, __fadd2_rn(ea, eb));
+                const float2 ya = __ffma2_rn(ea, s255, rm2), yb = __ffma2_rn(eb, s255, rm2);
+                w[k] = low_bytes4_u(ya.x, ya.y, yb.x, yb.y);
+              }
+              st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
+            }
+            l += acc2.x + acc2.y;
+          } else {
+          const float2 mp2 = pm2[j * 512];
 #pragma unroll
           for (int g = 0; g < 2; ++g) {
             uint32_t (&r)[16] = g ? rb : ra;
@@ -436,12 +507,22 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             }
             st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
           }
+          }
         }
         ptx::tc_fence_before();
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) { ptx::mbar_arrive(&s_free[j]); ptx::mbar_arrive(&p_full[pb]); }
         ++pcnt; used ^= 1u << j;
+      }
+      if constexpr (ROWMAX) {
+        // the row sum across the four column groups (the .y halves of this tile's statistics slots)
+        reinterpret_cast<float*>(st)[2 * (cq * ATT_BM + r_loc) + 1] = l;
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter) : "memory");
+        float lt = 0.f;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) lt += reinterpret_cast<const float*>(st)[2 * (g * ATT_BM + r_loc) + 1];
+        pend_rowf = lt > 0.f ? 1.0f / lt : 0.f;
       }
       pend = true;
       pend_row = row_ok ? (long long)(row_base + q) : -1;
@@ -456,7 +537,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <int DH>
+template <int DH, bool ROWMAX>
 static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
   using Cfg = AttnResCfg<DH>;
   const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
@@ -467,7 +548,7 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
   if ((st = make_tmap_2d(h, &tv, a->v, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BN, DH)) != HERO_OK) return st;
   p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN);
   p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);
-  auto kern = attn_int8_resident_kernel<DH>;
+  auto kern = attn_int8_resident_kernel<DH, ROWMAX>;
   static bool configured = false;
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
@@ -484,8 +565,12 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
 }
 
 hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
-  if (a->dh == 64) return launch_resident<64>(h, a, p, stream);
-  return launch_resident<128>(h, a, p, stream);
+  if (a->p_mode == HERO_P_ROWMAX) {
+    if (a->dh == 64) return launch_resident<64, true>(h, a, p, stream);
+    return launch_resident<128, true>(h, a, p, stream);
+  }
+  if (a->dh == 64) return launch_resident<64, false>(h, a, p, stream);
+  return launch_resident<128, false>(h, a, p, stream);
 }
 
 }  // namespace hero

@@ -56,7 +56,7 @@ class AttnArgs(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("dtype", C.c_int32), ("ld", C.c_int64),
                 ("B", C.c_int32), ("S", C.c_int32), ("nh", C.c_int32), ("dh", C.c_int32), ("s_q", C.c_float),
                 ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float), ("mask", C.c_int32),
-                ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p)]
+                ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p), ("p_mode", C.c_int32)]
 
 
 class LinearParams(C.Structure):
@@ -78,6 +78,8 @@ class LayerLayout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("qkv", "x_attn", "x_o", "x_mid", "x_mid_scale", "a", "x_2", "x_in", "x_in_scale",
                                           "h_in", "h_mid", "total")]
 
+
+P_MODE = {"static": 0, "rowmax": 1}
 
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
@@ -195,12 +197,13 @@ class Handle:
         _check(lib().hero_w8a8_linear(self._h, C.byref(a), _stream(stream)))
 
     def hero_int8_attention(self, q, k, v, B, S, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0, s_p=1.0 / 255,
-                            mask="none", key_len=None, p_absmax=None, stream=None):
+                            mask="none", key_len=None, p_absmax=None, p_mode="static", stream=None):
         """q, k, v: 2-D torch views [B*S, nh*dh] sharing one leading dimension; out: hero.Tensor; p_absmax: float32[1]
         running maximum of the softmax probabilities (F16 / BF16 core only)."""
         assert q.stride(0) == k.stride(0) == v.stride(0) and q.dtype == k.dtype == v.dtype
         a = AttnArgs(q.data_ptr(), k.data_ptr(), v.data_ptr(), _DT[q.dtype], q.stride(0), B, S, nh, dh, s_q, s_k,
-                     s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out, _ptr(p_absmax))
+                     s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out, _ptr(p_absmax),
+                     P_MODE[p_mode] if isinstance(p_mode, str) else p_mode)
         _check(lib().hero_int8_attention(self._h, C.byref(a), _stream(stream)))
 
     def hero_absmax_observe(self, x, col_absmax=None, tensor_absmax=None, stream=None):

@@ -85,17 +85,18 @@ def bench_gemm(h, M, K, N, act, fp, iters):
           % ("bf16" if fp else "i8", M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else ""), flush=True)
 
 
-def bench_attn(h, B, S, nh, dh, mask, iters):
+def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static"):
     H = nh * dh
     qkv = (torch.randn(B * S, 3 * H, device="cuda") * 40).clamp(-127, 127).to(torch.int8)
     out = torch.empty(B * S, H, device="cuda", dtype=torch.int8)
     sc = torch.full((H,), 0.02, device="cuda")
     s = (1.5 ** 0.5) / 40
     t = _time(lambda i: h.hero_int8_attention(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh,
-                                              hero.tensor(out, "fwq", sc), s_q=s, s_k=s, s_v=0.02, s_p=1 / 255, mask=mask), 1, iters)
+                                              hero.tensor(out, "fwq", sc), s_q=s, s_k=s, s_v=0.02, s_p=1 / 255, mask=mask,
+                                              p_mode=p_mode), 1, iters)
     scores = B * nh * S * S * (0.5 if mask == "causal" else 1.0)
-    print("INT8 attention B=%d S=%d nh=%d dh=%d %s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
-          % (B, S, nh, dh, mask, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12), flush=True)
+    print("INT8 attention B=%d S=%d nh=%d dh=%d %s P=%s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
+          % (B, S, nh, dh, mask, p_mode, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12), flush=True)
 
 
 def bench_absmax(h, M, H, iters):
@@ -138,6 +139,7 @@ def main():
     ap.add_argument("--kind", default="i8", choices=["i8", "f16"])
     ap.add_argument("--act", default="none")
     ap.add_argument("--mask", default="none")
+    ap.add_argument("--p-mode", default="static", choices=["static", "rowmax"])
     ap.add_argument("--fp", action="store_true")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--sweep", action="store_true")
@@ -162,7 +164,7 @@ def main():
     elif a.kernel == "wquant":
         bench_wquant(h, a.N, a.K, a.iters)
     else:
-        bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters)
+        bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters, a.p_mode)
     h.check()
 
 

@@ -33,7 +33,7 @@ def _scales(dh, spread=40):
     return s, s, 0.02
 
 
-def _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, s_p, out_spec, mask="none", key_len=None):
+def _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, s_p, out_spec, mask="none", key_len=None, p_mode="static"):
     H = nh * dh
     t = dev(qkv)
     if out_spec.kind == "fp":
@@ -45,15 +45,15 @@ def _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, s_p, out_spec, mask="none", key_le
         od = hero.tensor(out, out_spec.kind, sc)
     kl = None if key_len is None else dev(np.asarray(key_len, np.int32))
     h.hero_int8_attention(t[:, :H], t[:, H:2 * H], t[:, 2 * H:], B, S, nh, dh, od, s_q=s_q, s_k=s_k, s_v=s_v, s_p=s_p,
-                          mask=mask, key_len=kl)
+                          mask=mask, key_len=kl, p_mode=p_mode)
     h.check()
     return out.float().cpu().numpy() if out_spec.kind == "fp" else out.cpu().numpy()
 
 
-def _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, s_p, out_spec, mask="none", key_len=None, internals=False):
+def _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, s_p, out_spec, mask="none", key_len=None, internals=False, p_mode="static"):
     H = nh * dh
     return O.attention_int8(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh, s_q, s_k, s_v, s_p, out_spec,
-                            mask=mask, key_len=key_len, return_internals=internals)
+                            mask=mask, key_len=key_len, return_internals=internals, p_mode=p_mode)
 
 
 CASES = [  # B, S, nh, dh, mask
@@ -180,3 +180,43 @@ def test_fp_attention(h, fp, B, S, nh, dh, mask):
     frac, mx = int8_mismatch(out_q.cpu().numpy(), want_q.data)
     # P rounded to FP16 / BF16 perturbs X_attn by up to ~2^-11 / 2^-8 relative, i.e. a visible fraction of an INT8 step
     assert mx <= 1 and frac < (0.02 if fp == "f16" else 0.12), (frac, mx)
+
+
+# ------------------------------------------------------------------ row-max-normalised P (the long-sequence-robust quantizer)
+ROWMAX_CASES = [(1, 128, 2, 64, "none"), (2, 384, 4, 64, "none"), (1, 512, 2, 64, "none"), (1, 256, 2, 128, "causal"),
+                (2, 100, 3, 64, "none"), (1, 333, 2, 128, "causal"), (3, 40, 2, 64, "causal"), (1, 512, 2, 128, "none")]
+
+
+@pytest.mark.parametrize("B,S,nh,dh,mask", ROWMAX_CASES)
+def test_rowmax_p_quantizer_fwq_and_fp_output(h, B, S, nh, dh, mask):
+    qkv, H = _qkv(B, S, nh, dh, 900 + S + dh)
+    s_q, s_k, s_v = _scales(dh)
+    raw = _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, 1.0, O.OutSpec("fp", dtype="f64"), mask, p_mode="rowmax").data
+    spec = O.OutSpec("fwq", scale=Q.calib_scale(np.abs(raw).max(0)))
+    want = _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, 1.0, spec, mask, p_mode="rowmax")
+    got = _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, 0.0, spec, mask, p_mode="rowmax")      # s_p is ignored
+    assert_int8_close(got, want.data, frac=2e-4, what="X_attn (rowmax)")
+    got = _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, 0.0, O.OutSpec("fp", dtype="f16"), mask, p_mode="rowmax")
+    assert rel_err(got, raw) < 2e-3
+
+
+def test_rowmax_p_quantizer_key_lengths_and_flat_rows(h):
+    B, S, nh, dh = 3, 384, 2, 64
+    qkv, H = _qkv(B, S, nh, dh, 950)
+    s_q, s_k, s_v = _scales(dh)
+    key_len = [384, 130, 0]                                        # full, ragged inside a block, nothing allowed
+    raw = _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, 1.0, O.OutSpec("fp", dtype="f64"), "none", key_len, p_mode="rowmax").data
+    spec = O.OutSpec("fwq", scale=Q.calib_scale(np.abs(raw).max(0)))
+    want = _oracle(qkv, B, S, nh, dh, s_q, s_k, s_v, 1.0, spec, "none", key_len, p_mode="rowmax")
+    got = _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, 0.0, spec, "none", key_len, p_mode="rowmax")
+    assert_int8_close(got, want.data, frac=2e-4, what="X_attn (rowmax, key_len)")
+    assert not got[2 * S:].any()
+    # q = 0: every allowed key gets P~ = 255 and the output is the mean of V, which the static quantizer cannot do at S = 512
+    B, S, nh, dh = 1, 512, 1, 64
+    qkv, H = _qkv(B, S, nh, dh, 951)
+    qkv[:, :H] = 0
+    got = _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, 0.0, O.OutSpec("fp", dtype="f16"), p_mode="rowmax")
+    mean_v = s_v * qkv[:, 2 * H:].astype(np.float64).mean(0)
+    assert rel_err(got, np.broadcast_to(mean_v, got.shape)) < 2e-3
+    with pytest.raises(hero.HeroError):                            # longer sequences: not in this version
+        _run(h, _qkv(1, 1024, 1, 64, 952)[0], 1, 1024, 1, 64, s_q, s_k, s_v, 0.0, O.OutSpec("fp", dtype="f16"), p_mode="rowmax")
