@@ -174,7 +174,7 @@ hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* st
  *   HERO_P_STATIC (the paper, Eq. 16): P_u8 = clip(Round(P / s_p)) of the normalised probabilities, s_p calibrated.
  *   HERO_P_ROWMAX (not in the paper; robust to long sequences, where probabilities below s_p / 2 vanish under the
  *     static scale): P~_u8 = Round(255 * exp(A - max_row A)), row sum l of the un-quantized exponentials in FP32,
- *     out = acc * s_v / (255 * l); s_p is ignored.  Sequences of up to 512 keys in this version. */
+ *     out = acc * s_v / (255 * l); s_p is ignored. */
 typedef enum { HERO_P_STATIC = 0, HERO_P_ROWMAX = 1 } hero_p_mode;
 
 typedef struct {
@@ -233,6 +233,7 @@ typedef struct {
   hero_linear_params qkv, o, fc1, fc2;
   const float* ln1_g; const float* ln1_b;
   const float* ln2_g; const float* ln2_b;
+  int32_t p_mode;          /* hero_p_mode of the INT8 attention core (0 = the paper's static S_p) */
 } hero_layer_desc;
 
 /* ---------------------------------------------------------------------------------------------

@@ -44,6 +44,7 @@ class LayerSpec:
     gran_mid: str = "twq"            # granularity of the INT8 tensor feeding FC1  (twq | fwq | sq)
     gran_attn: str = "fwq"           # granularity of X_attn                        (fwq | sq)
     gran_out: str = "twq"            # post-LN layer output: twq | fwq | sq | fp
+    p_mode: str = "static"           # P quantizer of the INT8 attention core: 'static' (Eq. 16) | 'rowmax'
 
     @property
     def dh(self):
@@ -268,7 +269,8 @@ def _attention(L, qkv: QT, B):
         assert qkv.kind == "i8"
         d = qkv.data
         return attention_int8(d[:, :H], d[:, H:2 * H], d[:, 2 * H:], B, spec.S, spec.nh, spec.dh,
-                              C["S_q"], C["S_k"], C["S_v"], C["S_p"], L["attn_out_spec"], mask=spec.mask)
+                              C["S_q"], C["S_k"], C["S_v"], C["S_p"], L["attn_out_spec"], mask=spec.mask,
+                              p_mode=spec.p_mode)
     assert qkv.kind == "fp"
     d = qkv.real()
     return attention_fp(d[:, :H], d[:, H:2 * H], d[:, 2 * H:], B, spec.S, spec.nh, spec.dh,

@@ -43,7 +43,9 @@ struct AttnCfg {
   static constexpr int O_COL = ATT_NSB * ATT_BN;
 };
 
-template <int DH>
+// ROWMAX: P quantized against the row maximum (see attention_resident.cu): sweep 1 then only finds the maximum of the
+// integer scores, sweep 2 does the one exponential per score and sums the un-quantized exponentials.
+template <int DH, bool ROWMAX>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -204,6 +206,33 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
 
       float m = -INFINITY, l = 0.f;
+      if constexpr (ROWMAX) {
+        // ---- sweep 1: row maximum of the integer scores only
+        int imax = -(1 << 21);                               // below every real score
+        for (int i = 0; i < nkv; ++i, ++scnt) {
+          const int sb = scnt % ATT_NSB;
+          if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x3000 | sb)) ok = false;
+          ptx::tc_fence_after();
+          {
+            uint32_t r[32];
+            ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
+            ptx::tmem_ld_wait();
+            const int nvalid = min(32, kmax - (i * ATT_BN + cq * 32) + 1);
+            if (nvalid < 32) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (j >= nvalid) r[j] = (uint32_t)(-(1 << 21));
+            }
+            int i0 = max((int)r[0], (int)r[1]), i1 = max((int)r[2], (int)r[3]);
+#pragma unroll
+            for (int j = 4; j < 32; j += 4) { i0 = max(i0, max((int)r[j], (int)r[j + 1])); i1 = max(i1, max((int)r[j + 2], (int)r[j + 3])); }
+            imax = max(imax, max(i0, i1));
+          }
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
+        }
+        m = (float)imax;
+      } else {
       // ---- sweep 1: running row max and row sum (log2 domain)
       for (int i = 0; i < nkv; ++i, ++scnt) {
         const int sb = scnt % ATT_NSB;
@@ -246,11 +275,19 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
       }
+      }
       // ---- combine the four column groups of each row (buffer alternates with the tile)
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
       st[cq * ATT_BM + r_loc] = make_float2(m, l);
       asm volatile("bar.sync 1, 512;" ::: "memory");
-      {
+      float pscale;
+      if constexpr (ROWMAX) {
+        float mf = st[r_loc].x;
+#pragma unroll
+        for (int g = 1; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
+        m = mf <= (float)(-(1 << 21)) ? INFINITY : mf * c2;   // no allowed key: every exponential becomes exactly 0
+        pscale = 255.0f;                                      // P~_u8 = Round(255 * 2^(t - m))
+      } else {
         float mf = -INFINITY;
 #pragma unroll
         for (int g = 0; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
@@ -263,9 +300,9 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
         }
         m = mf; l = lf;
+        // P_u8 = Round(P / s_p) with P = 2^(t - m) / l
+        pscale = l > 0.f ? p.inv_sp / l : 0.f;
       }
-      // P_u8 = Round(P / s_p) with P = 2^(t - m) / l
-      const float pscale = l > 0.f ? p.inv_sp / l : 0.f;
 
       // ---- sweep 2: scores again -> P_u8 in shared memory (UMMA K-major, 128-byte swizzle)
       for (int j = 0; j < nkv; ++j, ++scnt, ++pcnt) {
@@ -283,6 +320,22 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           float y[32];
           const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m, -m), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
           const float2 ps2 = make_float2(pscale, pscale), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
+          if constexpr (ROWMAX) {
+            if (nvalid < 32) {                                 // masked keys: 2^(very negative) = 0, in P~ and in the row sum
+#pragma unroll
+              for (int e = 0; e < 32; ++e) if (e >= nvalid) r[e] = (uint32_t)(-(1 << 21));
+            }
+            float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float2 tt = __ffma2_rn(make_float2((float)(int)r[e], (float)(int)r[e + 1]), c22, nm2);
+              const float2 ev = make_float2(ex2f(tt.x), ex2f(tt.y));
+              acc2 = __fadd2_rn(acc2, ev);
+              const float2 v = __ffma2_rn(ev, ps2, rm2);       // at most 255: no clip
+              y[e] = v.x; y[e + 1] = v.y;
+            }
+            l += acc2.x + acc2.y;
+          } else {
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             // Round(P / s_p) clipped to 255: round-half-to-even happens in the FMA's single rounding
@@ -295,6 +348,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (nvalid < 32) {                                   // block straddles the mask: masked keys get code 0
 #pragma unroll
             for (int e = 0; e < 32; ++e) if (e >= nvalid) y[e] = ATT_MAGIC;
+          }
           }
           const int c16 = cq * 2;                              // 16-byte chunk index within the 128-byte row
           st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), low_bytes4_u(y[0], y[1], y[2], y[3]), low_bytes4_u(y[4], y[5], y[6], y[7]),
@@ -309,6 +363,16 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (lane == 0) { ptx::mbar_arrive(&s_empty[sb]); ptx::mbar_arrive(&p_full[pb]); }
       }
 
+      float rowf = 1.f;
+      if constexpr (ROWMAX) {
+        // the row sum across the four column groups (the .y halves of this tile's statistics slots)
+        reinterpret_cast<float*>(st)[2 * (cq * ATT_BM + r_loc) + 1] = l;
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        float lt = 0.f;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) lt += reinterpret_cast<const float*>(st)[2 * (g * ATT_BM + r_loc) + 1];
+        rowf = lt > 0.f ? 1.0f / lt : 0.f;
+      }
       // ---- epilogue: X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8); 32 output columns per warp
       uint32_t r[32];
       if (nkv > 0) {
@@ -335,7 +399,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           float v[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            v[j] = (float)(int)r[j] * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
+            v[j] = (float)(int)r[j] * rowf * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
           int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
 #pragma unroll
           for (int g = 0; g < 2; ++g)
@@ -349,7 +413,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int g = 0; g < 4; ++g) {
             float v[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * p.pv_scale;
+            for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * rowf * p.pv_scale;
             st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
                    fp2(v[6], v[7], p.out_dt));
           }
@@ -363,7 +427,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <int DH>
+template <int DH, bool ROWMAX>
 static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
   using Cfg = AttnCfg<DH>;
   const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
@@ -374,7 +438,7 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
   if ((st = make_tmap_2d(h, &tv, a->v, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BN, DH)) != HERO_OK) return st;
   p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN);   // S8 x S8 -> S32, both K-major
   p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);       // U8 x S8 -> S32, V is MN-major
-  auto kern = attn_int8_kernel<DH>;
+  auto kern = attn_int8_kernel<DH, ROWMAX>;
   static bool configured = false;
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
@@ -423,7 +487,6 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   p.c2 = (float)((double)a->s_q * (double)a->s_k / sqrt((double)a->dh) * 1.4426950408889634);
   HERO_REQUIRE(a->p_mode == HERO_P_STATIC || a->p_mode == HERO_P_ROWMAX, HERO_ERR_INVALID_ARG, "unknown p_mode %d", a->p_mode);
   const bool rowmax = !fp_in && a->p_mode == HERO_P_ROWMAX;
-  HERO_REQUIRE(!rowmax || a->S <= 512, HERO_ERR_UNSUPPORTED, "p_mode ROWMAX handles sequences of up to 512 keys");
   p.inv_sp = rowmax ? 255.0f : 1.0f / a->s_p;
   p.pv_scale = rowmax ? a->s_v / 255.0f : a->s_p * a->s_v;
   p.out_scale = a->out.dtype == HERO_I8 ? a->out.scale : nullptr;
@@ -437,6 +500,7 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
   if (a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory
-  if (a->dh == 64) return launch_attn<64>(h, a, p, s);
-  return launch_attn<128>(h, a, p, s);
+  if (rowmax) return a->dh == 64 ? launch_attn<64, true>(h, a, p, s) : launch_attn<128, true>(h, a, p, s);
+  if (a->dh == 64) return launch_attn<64, false>(h, a, p, s);
+  return launch_attn<128, false>(h, a, p, s);
 }

@@ -156,6 +156,7 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     a.B = d->B; a.S = d->S; a.nh = d->nh; a.dh = H / d->nh;
     a.s_q = d->s_q; a.s_k = d->s_k; a.s_v = d->s_v; a.s_p = d->s_p;
     a.mask = d->mask; a.key_len = nullptr;
+    a.p_mode = d->p_mode;
     a.out = x_attn;
     if ((st = hero_int8_attention(h, &a, stream)) != HERO_OK) return st;
   }

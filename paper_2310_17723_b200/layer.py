@@ -30,6 +30,7 @@ class Layer:
             d.mode[i] = hero.MODE_INT8 if cfg.mode[mname] == "int8" else hero.MODE_FP
         d.gran_in, d.gran_mid = hero.GRAN[cfg.gran_in], hero.GRAN[cfg.gran_mid]
         d.gran_attn, d.gran_out = hero.GRAN[cfg.gran_attn], hero.GRAN[cfg.gran_out]
+        d.p_mode = hero.P_MODE[getattr(cfg, "p_mode", "static")]
         for name in ("s_in", "s_mid", "s_attn", "s_o", "s_x2", "s_out", "ln1_g", "ln1_b", "ln2_g", "ln2_b"):
             t = _up(L.get(name))
             self._bufs[name] = t

@@ -37,6 +37,7 @@ class LayerConfig:
     gran_mid: str = "twq"
     gran_attn: str = "fwq"
     gran_out: str = "twq"
+    p_mode: str = "static"          # P quantizer of the INT8 attention core: "static" (the paper) | "rowmax"
 
     @property
     def dh(self):

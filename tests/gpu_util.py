@@ -71,7 +71,7 @@ def oracle_layer_to_prepared(Lp):
     cfg = prep.LayerConfig(B=spec.B, S=spec.S, H=spec.H, nh=spec.nh, F=spec.F, arch=spec.arch, act=spec.act,
                            eps=spec.eps, mask=spec.mask, fp_dtype=spec.fp_dtype, mode=dict(spec.mode),
                            gran_in=spec.gran_in, gran_mid=spec.gran_mid, gran_attn=spec.gran_attn,
-                           gran_out=spec.gran_out)
+                           gran_out=spec.gran_out, p_mode=getattr(spec, "p_mode", "static"))
     f = lambda a: None if a is None else np.ascontiguousarray(np.asarray(a, np.float64).astype(np.float32))
     L = {"cfg": cfg, "C": C}
     for name in ("qkv", "o", "fc1", "fc2"):

@@ -184,7 +184,8 @@ def test_fp_attention(h, fp, B, S, nh, dh, mask):
 
 # ------------------------------------------------------------------ row-max-normalised P (the long-sequence-robust quantizer)
 ROWMAX_CASES = [(1, 128, 2, 64, "none"), (2, 384, 4, 64, "none"), (1, 512, 2, 64, "none"), (1, 256, 2, 128, "causal"),
-                (2, 100, 3, 64, "none"), (1, 333, 2, 128, "causal"), (3, 40, 2, 64, "causal"), (1, 512, 2, 128, "none")]
+                (2, 100, 3, 64, "none"), (1, 333, 2, 128, "causal"), (3, 40, 2, 64, "causal"), (1, 512, 2, 128, "none"),
+                (1, 1024, 1, 128, "causal"), (1, 640, 2, 64, "none"), (2, 777, 1, 64, "causal")]     # the last three: two-sweep kernel
 
 
 @pytest.mark.parametrize("B,S,nh,dh,mask", ROWMAX_CASES)
@@ -218,5 +219,3 @@ def test_rowmax_p_quantizer_key_lengths_and_flat_rows(h):
     got = _run(h, qkv, B, S, nh, dh, s_q, s_k, s_v, 0.0, O.OutSpec("fp", dtype="f16"), p_mode="rowmax")
     mean_v = s_v * qkv[:, 2 * H:].astype(np.float64).mean(0)
     assert rel_err(got, np.broadcast_to(mean_v, got.shape)) < 2e-3
-    with pytest.raises(hero.HeroError):                            # longer sequences: not in this version
-        _run(h, _qkv(1, 1024, 1, 64, 952)[0], 1, 1024, 1, 64, s_q, s_k, s_v, 0.0, O.OutSpec("fp", dtype="f16"), p_mode="rowmax")

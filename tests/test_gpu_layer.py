@@ -120,6 +120,44 @@ def test_pre_ln_causal_m3_layer(h, fp, dh):
     assert rel_err(out2.float().cpu().numpy(), T2["h_out"].real()) < 1e-2
 
 
+@pytest.mark.parametrize("arch,S", [("post_ln", 128), ("pre_ln", 640)])
+def test_layer_with_rowmax_p_quantizer(h, arch, S):
+    """The long-sequence-robust P quantizer inside the layer (resident-score kernel at S = 128, two-sweep at S = 640),
+    against the oracle layer run with the same quantizer; and, at S = 640 where the static scale starts losing
+    probability mass, closer to the un-quantized layer than the paper-literal quantizer."""
+    shape = W.tiny_shape(B=2, S=S, H=256, nh=4, F=512, arch=arch, mask="causal" if arch == "pre_ln" else "none", eps=1e-5)
+    spec, Lp, x_in = _build(shape, 27, p_mode="rowmax")
+    T = OL.layer_forward(Lp, x_in)
+    out, sc, _ = _run_layer(h, spec, Lp, x_in)
+    if arch == "pre_ln":
+        got, want = out.float().cpu().numpy(), T["h_out"].real()
+    else:
+        got, want = out.cpu().numpy().astype(np.float64) * sc.cpu().numpy().astype(np.float64)[:, None], T["x_out"].real()
+    assert rel_err(got, want) < 1e-2
+
+
+def test_rowmax_p_quantizer_keeps_the_mass_of_flat_long_rows(h):
+    # attention spread evenly over 1024 keys: every normalised probability is below S_p / 2 = 1/510, the static
+    # quantizer returns zeros, the row-max quantizer returns the mean of V (compared with FP attention of the same operands)
+    B, S, nh, dh = 1, 1024, 2, 64
+    Hh = nh * dh
+    g = W.rng(9, 6)
+    qkv = np.clip(np.rint(g.standard_normal((B * S, 3 * Hh)) * 40), -127, 127).astype(np.int8)
+    qkv[:, :Hh] = 0
+    s_v = 0.02
+    t = torch.from_numpy(qkv).cuda()
+    outs = {}
+    for mode in ("static", "rowmax"):
+        o = torch.empty(B * S, Hh, dtype=torch.float16, device="cuda")
+        h.hero_int8_attention(t[:, :Hh], t[:, Hh:2 * Hh], t[:, 2 * Hh:], B, S, nh, dh, hero.tensor(o), s_q=0.03, s_k=0.03,
+                              s_v=s_v, s_p=1.0 / 255, p_mode=mode)
+        outs[mode] = o.float().cpu().numpy()
+    h.check()
+    ref = np.broadcast_to(s_v * qkv[:, 2 * Hh:].astype(np.float64).mean(0), outs["rowmax"].shape)
+    assert not outs["static"].any()
+    assert rel_err(outs["rowmax"], ref) < 2e-3
+
+
 @pytest.mark.parametrize("preset", ["M1", "M2", "FP"])
 @pytest.mark.parametrize("arch", ["post_ln", "pre_ln"])
 def test_mixed_precision_presets(h, preset, arch):
