@@ -258,6 +258,12 @@ typedef struct {
  *   All pointers are device pointers; outputs are caller-owned.  The paper gives the equations, not an interface. */
 hero_status hero_absmax_observe(hero_handle* h, const hero_tensor* x, float* col_absmax, float* tensor_absmax,
                                 void* stream);
+/* Percentile clipping of a static scale (the truncation threshold the paper leaves un-tuned, Sec. 3): adds the
+ * histogram of |x| over HERO_HIST_BINS equal bins of [0, bound) to hist (device uint64[HERO_HIST_BINS], accumulating;
+ * values >= bound fall into the last bin).  With bound = the tensor's absmax, the q-th percentile is the upper edge
+ * of the first bin at which the cumulative count reaches q of the total. */
+#define HERO_HIST_BINS 2048
+hero_status hero_abs_histogram(hero_handle* h, const hero_tensor* x, float bound, uint64_t* hist, void* stream);
 hero_status hero_quantize_weight(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K,
                                  const float* in_scale, const float* out_scale, const float* bias, int8_t* Wq,
                                  int64_t ldq, float* w_scale, float* bias_out, void* stream);

@@ -70,6 +70,39 @@ __global__ void __launch_bounds__(256) absmax_kernel(const uint16_t* __restrict_
   }
 }
 
+// Histogram of |x| / bound over NBINS equal bins (values at or above the bound land in the last bin): per-CTA counts in
+// shared memory, one global atomic per bin and CTA at the end.  The percentile clipping threshold of a static scale is
+// read off the cumulative counts on the host.
+constexpr int HIST_BINS = 2048;
+template <bool BF>
+__global__ void __launch_bounds__(256) abs_hist_kernel(const uint16_t* __restrict__ x, long long ld, long long rows, int cols,
+                                                       long long rows_per_cta, float inv_bin, unsigned long long* hist) {
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();
+  __shared__ unsigned int sh[HIST_BINS];
+  for (int i = threadIdx.x; i < HIST_BINS; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  const int nchunk = cols >> 3;
+  const long long r0 = (long long)blockIdx.x * rows_per_cta, r1 = min(rows, r0 + rows_per_cta);
+  for (long long r = r0; r < r1; ++r) {
+    for (int c = threadIdx.x; c < nchunk; c += blockDim.x) {
+      const uint4 w = __ldg(reinterpret_cast<const uint4*>(x + r * ld + (long long)c * 8));
+      const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float a, b;
+        if constexpr (BF) { a = __uint_as_float(u[i] << 16); b = __uint_as_float(u[i] & 0xffff0000u); }
+        else { const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u[i])); a = f.x; b = f.y; }
+        atomicAdd(&sh[min(HIST_BINS - 1, (int)(fabsf(a) * inv_bin))], 1u);
+        atomicAdd(&sh[min(HIST_BINS - 1, (int)(fabsf(b) * inv_bin))], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < HIST_BINS; i += blockDim.x)
+    if (sh[i]) atomicAdd(hist + i, (unsigned long long)sh[i]);
+}
+
 // One CTA per output feature n: row n of W [N][K] (FP32).
 __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __restrict__ W, long long ldw, int N, int K,
                                                               const float* __restrict__ in_scale,
@@ -150,6 +183,36 @@ extern "C" hero_status hero_absmax_observe(hero_handle* h, const hero_tensor* x,
       HERO_CUDA(launch_dependent(absmax_kernel<false>, dim3((unsigned)ctas), dim3(cx, cy), 0, s,
                                  reinterpret_cast<const uint16_t*>(x->data), (long long)x->ld, (long long)x->rows,
                                  (int)x->cols, rows_per_cta, col_absmax, tensor_absmax));
+  }
+  HERO_CUDA(cudaGetLastError());
+  return HERO_OK;
+}
+
+extern "C" hero_status hero_abs_histogram(hero_handle* h, const hero_tensor* x, float bound, uint64_t* hist, void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(h && x && hist, HERO_ERR_INVALID_ARG, "hero_abs_histogram: NULL argument");
+  HERO_REQUIRE(bound > 0.f, HERO_ERR_INVALID_ARG, "bound must be positive");
+  hero_status st;
+  if ((st = check_matrix(*x, "x")) != HERO_OK) return st;
+  HERO_REQUIRE(is_fp16ish(x->dtype), HERO_ERR_UNSUPPORTED, "observers read F16 / BF16 tensors (the un-quantized layer)");
+  HERO_REQUIRE(x->cols % 8 == 0 && x->ld % 8 == 0, HERO_ERR_ALIGNMENT, "cols and ld must be multiples of 8 elements");
+  if (x->rows == 0) return HERO_OK;
+  long long ctas = (long long)h->sm_count * 8;
+  long long rows_per_cta = (x->rows + ctas - 1) / ctas;
+  if (rows_per_cta < 8) rows_per_cta = 8;
+  ctas = (x->rows + rows_per_cta - 1) / rows_per_cta;
+  const float inv_bin = (float)HIST_BINS / bound;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  {
+    LaunchScope scope(h, s, KERNEL_LN);
+    if (x->dtype == HERO_BF16)
+      HERO_CUDA(launch_dependent(abs_hist_kernel<true>, dim3((unsigned)ctas), dim3(256), 0, s,
+                                 reinterpret_cast<const uint16_t*>(x->data), (long long)x->ld, (long long)x->rows, (int)x->cols,
+                                 rows_per_cta, inv_bin, reinterpret_cast<unsigned long long*>(hist)));
+    else
+      HERO_CUDA(launch_dependent(abs_hist_kernel<false>, dim3((unsigned)ctas), dim3(256), 0, s,
+                                 reinterpret_cast<const uint16_t*>(x->data), (long long)x->ld, (long long)x->rows, (int)x->cols,
+                                 rows_per_cta, inv_bin, reinterpret_cast<unsigned long long*>(hist)));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;

@@ -81,11 +81,12 @@ class LayerLayout(C.Structure):
 
 
 P_MODE = {"static": 0, "rowmax": 1}
+HIST_BINS = 2048
 
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
-           "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight")
+           "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram")
 
 _lib = None
 
@@ -110,6 +111,7 @@ def lib():
         L.hero_mode_preset.argtypes = [C.c_int32, C.POINTER(C.c_int32 * 5)]
         L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
         L.hero_absmax_observe.argtypes = [C.c_void_p, C.POINTER(Tensor), C.c_void_p, C.c_void_p, C.c_void_p]
+        L.hero_abs_histogram.argtypes = [C.c_void_p, C.POINTER(Tensor), C.c_float, C.c_void_p, C.c_void_p]
         L.hero_quantize_weight.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.hero_layer_workspace_layout.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(LayerLayout)]
@@ -210,6 +212,11 @@ class Handle:
     def hero_absmax_observe(self, x, col_absmax=None, tensor_absmax=None, stream=None):
         """x: hero.Tensor (F16 / BF16); col_absmax float32[cols] / tensor_absmax float32[1]: running maxima, updated."""
         _check(lib().hero_absmax_observe(self._h, C.byref(x), _ptr(col_absmax), _ptr(tensor_absmax), _stream(stream)))
+
+    def hero_abs_histogram(self, x, bound, hist, stream=None):
+        """x: hero.Tensor (F16 / BF16); hist: int64 / uint64 [2048] device tensor, accumulated."""
+        assert hist.numel() == HIST_BINS and hist.element_size() == 8
+        _check(lib().hero_abs_histogram(self._h, C.byref(x), float(bound), C.c_void_p(hist.data_ptr()), _stream(stream)))
 
     def hero_quantize_weight(self, W, Wq, w_scale, in_scale=None, out_scale=None, bias=None, bias_out=None, stream=None):
         """W: float32 [N, K]; Wq: int8 [N, K]; w_scale: float32 [N]; optional folds in_scale [K], out_scale [N]."""

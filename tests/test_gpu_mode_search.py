@@ -1,0 +1,66 @@
+"""Mode search and percentile clipping (Sec. 2.3 / Sec. 3) on the device."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ops as O
+from paper_2310_17723_b200 import hero, prep, mode_search as MS, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture
+def h():
+    hd = hero.Handle()
+    yield hd
+    hd.check()
+    hd.close()
+
+
+def test_abs_histogram_matches_numpy_and_percentile_scale(h):
+    g = np.random.default_rng(3)
+    x = torch.from_numpy(g.standard_normal((777, 1024)).astype(np.float32)).to(torch.float16).cuda()
+    x[5, 7] = 40.0                                                 # one outlier far beyond the bulk
+    ref = np.abs(x.float().cpu().numpy().astype(np.float64))
+    bound = float(ref.max())
+    hist = torch.zeros(hero.HIST_BINS, dtype=torch.int64, device="cuda")
+    h.hero_abs_histogram(hero.tensor(x), bound, hist)
+    h.check()
+    # bin index computed the way the device does it: fp32 product, truncation, last bin closed
+    idx = np.minimum(hero.HIST_BINS - 1, (ref.astype(np.float32) * np.float32(hero.HIST_BINS / np.float32(bound))).astype(np.int64))
+    want = np.bincount(idx.ravel(), minlength=hero.HIST_BINS)
+    got = hist.cpu().numpy()
+    assert got.sum() == ref.size
+    # a value that sits on a bin edge may land one bin away (reciprocal-multiply in fp32): compare cumulatively
+    assert np.abs(np.cumsum(got) - np.cumsum(want)).max() <= 2
+    # accumulation over a second call
+    h.hero_abs_histogram(hero.tensor(x), bound, hist)
+    assert hist.sum().item() == 2 * ref.size
+    # q = 1 gives absmax / 127 within one bin; q = 0.9999 cuts the outlier off
+    s1 = MS.percentile_scale(h, x, 1.0)
+    assert abs(s1 - bound / 127) <= bound / hero.HIST_BINS / 127 * 1.01
+    s2 = MS.percentile_scale(h, x, 0.9999)
+    q = np.quantile(ref, 0.9999)
+    assert q / 127 <= s2 <= (q + 2 * bound / hero.HIST_BINS) / 127 and s2 < 0.2 * s1
+
+
+def test_sensitivity_and_greedy_search(h):
+    shape = W.tiny_shape(B=2, S=128, H=256, nh=4, F=512, eps=1e-5, n_outlier=2)
+    cfg = prep.LayerConfig(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, eps=shape.eps)
+    p = W.layer_params(shape, 61)
+    x = W.activations(shape, 61)
+    cal = O.layernorm(x.astype(np.float64), p["ln0_g"], p["ln0_b"], shape.eps)
+    C = prep.calibrate(cfg, p, cal, shape.B)
+    x_in = torch.from_numpy(cal).to(torch.float16).cuda()
+    t = MS.sensitivity(h, cfg, p, C, x_in)
+    assert set(t) == set(MS.MODULES) | {"all_int8"}
+    for m in MS.MODULES:
+        # one INT8 module perturbs the layer a little, never more than a few percent; all INT8 is the largest error
+        assert 0.0 < t[m]["alone"] < 0.1 and t[m]["without"] <= t["all_int8"] * 1.5 + 1e-3
+    # a budget above the all-INT8 error keeps M3; a budget of zero walks all the way to FP
+    mode, trace = MS.search(h, cfg, p, C, x_in, budget=10.0)
+    assert mode == prep.PRESETS["M3"] and len(trace) == 1
+    mode, trace = MS.search(h, cfg, p, C, x_in, budget=t["all_int8"] * 0.5)
+    assert trace[-1][1] <= t["all_int8"] * 0.5 or all(v == "fp" for v in mode.values())
+    errs = [e for _, e in trace]
+    assert all(b <= a * 1.2 + 1e-4 for a, b in zip(errs, errs[1:]))     # releasing a module does not make it worse
