@@ -302,6 +302,12 @@ hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const h
 hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
                                     const hero_tensor* out_host, const hero_tensor* in_dev, const hero_tensor* out_dev,
                                     void* workspace, size_t workspace_bytes, void* stream);
+/* The same without the final synchronisation: the copies and the layer are only enqueued on `stream`, and `out_host`
+ * is valid once the caller has synchronised that stream.  Several calls on different streams, each with its own
+ * staging tensors, workspace and host output buffer, overlap one step's copies with another step's kernels. */
+hero_status hero_layer_forward_host_async(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
+                                          const hero_tensor* out_host, const hero_tensor* in_dev,
+                                          const hero_tensor* out_dev, void* workspace, size_t workspace_bytes, void* stream);
 
 /* The layer forward for callers that cannot allocate device memory (the paper has no counterpart: it describes
  * no software interface).  Who needs it: code that runs inside another framework's fixed memory plan, real-time

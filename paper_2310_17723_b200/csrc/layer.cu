@@ -224,10 +224,10 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
   return HERO_OK;
 }
 
-extern "C" hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
-                                               const hero_tensor* out_host, const hero_tensor* in_dev,
-                                               const hero_tensor* out_dev, void* workspace, size_t workspace_bytes,
-                                               void* stream) {
+extern "C" hero_status hero_layer_forward_host_async(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
+                                                     const hero_tensor* out_host, const hero_tensor* in_dev,
+                                                     const hero_tensor* out_dev, void* workspace, size_t workspace_bytes,
+                                                     void* stream) {
   using namespace hero;
   HERO_REQUIRE(h && d && in_host && out_host && in_dev && out_dev, HERO_ERR_INVALID_ARG, "hero_layer_forward_host: NULL argument");
   HERO_REQUIRE(in_host->dtype == in_dev->dtype && in_host->rows == in_dev->rows && in_host->cols == in_dev->cols &&
@@ -251,6 +251,15 @@ extern "C" hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_
                               out_dev->rows, cudaMemcpyDeviceToHost, s));
   if (scale_len(*out_dev))
     HERO_CUDA(cudaMemcpyAsync(out_host->scale, out_dev->scale, scale_len(*out_dev) * sizeof(float), cudaMemcpyDeviceToHost, s));
-  HERO_CUDA(cudaStreamSynchronize(s));
+  return HERO_OK;
+}
+
+extern "C" hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
+                                               const hero_tensor* out_host, const hero_tensor* in_dev,
+                                               const hero_tensor* out_dev, void* workspace, size_t workspace_bytes,
+                                               void* stream) {
+  hero_status st = hero_layer_forward_host_async(h, d, in_host, out_host, in_dev, out_dev, workspace, workspace_bytes, stream);
+  if (st != HERO_OK) return st;
+  HERO_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
   return HERO_OK;
 }

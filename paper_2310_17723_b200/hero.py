@@ -85,7 +85,7 @@ HIST_BINS = 2048
 
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
-           "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_profile_begin",
+           "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_layer_forward_host_async", "hero_profile_begin",
            "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram")
 
 _lib = None
@@ -117,6 +117,8 @@ def lib():
         L.hero_layer_workspace_layout.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(LayerLayout)]
         L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hero_layer_forward_host_async.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
+            [C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_host.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
             [C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_static.argtypes = [C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
@@ -234,6 +236,12 @@ class Handle:
         lay = LayerLayout()
         _check(lib().hero_layer_workspace_layout(C.byref(desc), int(M), C.byref(lay)))
         return lay
+
+    def hero_layer_forward_host_async(self, desc, in_host, out_host, in_dev, out_dev, workspace, stream=None):
+        """Host-buffer variant without the final synchronisation (out_host is valid after the stream is synchronised)."""
+        _check(lib().hero_layer_forward_host_async(self._h, C.byref(desc), C.byref(in_host), C.byref(out_host),
+                                                   C.byref(in_dev), C.byref(out_dev), C.c_void_p(workspace.data_ptr()),
+                                                   workspace.numel(), _stream(stream)))
 
     def hero_layer_forward_host(self, desc, in_host, out_host, in_dev, out_dev, workspace, stream=None):
         """Host-buffer variant: copies in, runs the layer, copies out, synchronizes."""

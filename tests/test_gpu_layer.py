@@ -185,3 +185,34 @@ def test_workspace_too_small_and_bad_args(h):
     with pytest.raises(hero.HeroError) as e:
         h.hero_layer_forward(layer.desc, in_desc, hero.tensor(out, "twq", sc), small)
     assert e.value.status == hero.ERR_WORKSPACE
+
+
+def test_host_buffer_entry_points_match_the_device_one(h):
+    """hero_layer_forward_host (copies in, layer, copies out, synchronise) and its _async form on side streams give
+    the bytes hero_layer_forward gives on device-resident tensors."""
+    shape = W.tiny_shape(**SMALL, eps=1e-5, n_outlier=2)
+    spec, Lp, x_in = _build(shape, 31)
+    out_ref, sc_ref, _ = _run_layer(h, spec, Lp, x_in)
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    M, H = spec.M, spec.H
+    hin = torch.from_numpy(x_in.data).pin_memory()
+    hsin = torch.from_numpy(np.asarray(x_in.row_scale, np.float32)).pin_memory()
+    in_host = hero.host_tensor(hin, "twq", hsin)
+
+    def slot():
+        ti, si = torch.empty(M, H, dtype=torch.int8, device="cuda"), torch.empty(M, dtype=torch.float32, device="cuda")
+        to, so = torch.empty(M, H, dtype=torch.int8, device="cuda"), torch.empty(M, dtype=torch.float32, device="cuda")
+        ho, hso = torch.empty(M, H, dtype=torch.int8).pin_memory(), torch.empty(M, dtype=torch.float32).pin_memory()
+        return hero.tensor(ti, "twq", si), hero.tensor(to, "twq", so), hero.host_tensor(ho, "twq", hso), ho, hso
+
+    d_in, d_out, out_host, ho, hso = slot()
+    h.hero_layer_forward_host(layer.desc, in_host, out_host, d_in, d_out, layer.workspace)
+    assert torch.equal(ho, out_ref.cpu()) and torch.equal(hso, sc_ref.cpu())
+    # three calls in flight on three streams, each with its own staging tensors and workspace
+    slots = [slot() + (torch.empty_like(layer.workspace), torch.cuda.Stream()) for _ in range(3)]
+    for d_in, d_out, out_host, ho, hso, ws, st in slots:
+        h.hero_layer_forward_host_async(layer.desc, in_host, out_host, d_in, d_out, ws, stream=st)
+    for d_in, d_out, out_host, ho, hso, ws, st in slots:
+        st.synchronize()
+        assert torch.equal(ho, out_ref.cpu()) and torch.equal(hso, sc_ref.cpu())
+    h.check()
