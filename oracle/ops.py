@@ -21,6 +21,7 @@ class QT:
 
     kind 'i8': data int8 [n, d]; row_scale [n] (TWQ) and/or col_scale [d] (FWQ; SQ is a
                constant vector) give the real value row_scale[i] * data[i, j] * col_scale[j].
+    kind 'f8': the same with an e4m3 payload (FP8 variant): data holds the e4m3 VALUES in fp64.
     kind 'fp': data fp64 holding values already rounded to the storage grid `dtype`.
     """
     kind: str
@@ -116,10 +117,13 @@ class OutSpec:
     kind 'sq'   : INT8 with the given scalar scale            (Eq. 5)
     kind 'round': INT8 = clip(Round(v)); the scale was folded into the producer (Eq. 20-22)
     kind 'fp'   : stored in `dtype` ('f16' / 'bf16' / 'f32')
+    payload 'f8' (FP8 variant): the same kinds with an e4m3 payload instead of INT8; a scale computed on the fly is
+    absmax / 448 and the quantizer is the saturating e4m3 rounding instead of clip(Round(.)).
     """
     kind: str
     scale: Optional[np.ndarray] = None
     dtype: str = "f16"
+    payload: str = "i8"
 
 
 def emit(v, spec: OutSpec, carried_col_scale=None):
@@ -127,6 +131,20 @@ def emit(v, spec: OutSpec, carried_col_scale=None):
     for when it was folded away upstream (kind 'round')."""
     if spec.kind == "fp":
         return fp_tensor(v, spec.dtype)
+    if spec.payload == "f8":
+        v = np.asarray(v, dtype=np.float64)
+        if spec.kind == "twq":
+            s = Q.f8_scale(np.max(np.abs(v), axis=1))
+            return QT("f8", Q.quant_f8(v, s[:, None]), row_scale=s)
+        if spec.kind == "fwq":
+            s = np.asarray(spec.scale, dtype=np.float64).reshape(-1)
+            return QT("f8", Q.quant_f8(v, s[None, :]), col_scale=s)
+        if spec.kind == "sq":
+            s = float(np.asarray(spec.scale).reshape(()))
+            return QT("f8", Q.quant_f8(v, s), col_scale=np.full(v.shape[1], s))
+        if spec.kind == "round":
+            return QT("f8", Q.quant_f8(v, 1.0), col_scale=carried_col_scale)
+        raise ValueError(spec.kind)
     if spec.kind == "twq":
         q, s = Q.quant_twq(v)
         return QT("i8", q, row_scale=s)
@@ -203,6 +221,32 @@ def gemm_quant(x: QT, W_i8, col_scale, bias, act, out: OutSpec, carried=None, re
     a = ACTIVATIONS[act](v)
     o = emit(a, out, carried)
     return (o, acc) if return_acc else o
+
+
+def gemm_quant_f8(x: QT, W_f8, col_scale, bias, act, out: OutSpec, carried=None):
+    """The FP8 variant of GeMM^quant: e4m3 operands, the same epilogue.
+
+    acc = X_f8 W_f8 (every product of two e4m3 values and every partial sum is exact in fp64 for d <= 2^17),
+    v = acc * rs[i] * cs[j] + b[j], a = act(v), out = emit(a).  W_f8 [d, m] holds e4m3 values, col_scale [m] the
+    column scales of Eq. 2 taken with 448 in place of 127.
+    """
+    assert x.kind == "f8"
+    assert x.data.shape[1] <= 2 ** 17
+    acc = np.asarray(x.data, np.float64) @ np.asarray(W_f8, np.float64)
+    v = acc
+    if x.row_scale is not None:
+        v = v * np.asarray(x.row_scale, np.float64)[:, None]
+    v = v * np.asarray(col_scale, np.float64)[None, :]
+    if bias is not None:
+        v = v + np.asarray(bias, np.float64)[None, :]
+    return emit(ACTIVATIONS[act](v), out, carried)
+
+
+def quant_weight_columnwise_f8(W):
+    """Eq. 2 with an e4m3 payload: per-output-column scale absmax / 448.  Returns (e4m3 values [d, m], S_w [m])."""
+    W = np.asarray(W, dtype=np.float64)
+    S_w = Q.f8_scale(np.max(np.abs(W), axis=0))
+    return Q.quant_f8(W, S_w[None, :]), S_w
 
 
 def gemm_fp(x: QT, W, bias, act, out: OutSpec, carried=None):

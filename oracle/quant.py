@@ -74,6 +74,35 @@ def dequant(q, row_scale=None, col_scale=None):
     return x
 
 
+# --------------------------------------------------------------------------------------
+# FP8 (e4m3) variant: the same fusion points with an 8-bit floating-point payload
+# --------------------------------------------------------------------------------------
+F8MAX = 448.0            # largest finite e4m3 value (1.75 * 2^8); no infinities in this format
+
+
+def e4m3_round(v):
+    """Nearest e4m3 value (1 sign, 4 exponent bits with bias 7, 3 mantissa bits), ties to even, saturating at
+    +-448 (the 'satfinite' conversion).  Normal values 2^e (1 + k/8), e in [-6, 8]; below 2^-6 the grid is the
+    subnormal one with spacing 2^-9.  Returned in fp64."""
+    x = np.asarray(v, dtype=np.float64)
+    a = np.minimum(np.abs(x), F8MAX)
+    e = np.floor(np.log2(np.where(a > 0.0, a, 1.0)))
+    e = np.clip(e, -6.0, 8.0)                   # subnormals share the spacing of the smallest normal binade
+    q = np.exp2(e - 3.0)                        # grid spacing inside the binade
+    r = np.rint(a / q) * q                      # rint: half to even; a value that rounds up to 2^(e+1) is on the next grid too
+    return np.sign(x) * np.minimum(r, F8MAX)
+
+
+def quant_f8(v, scale):
+    """Qf8(v; s) = e4m3(v / s): the 8-bit floating-point counterpart of Qs.  Returns the e4m3 VALUES in fp64."""
+    return e4m3_round(np.asarray(v, dtype=np.float64) / np.asarray(scale, dtype=np.float64))
+
+
+def f8_scale(absmax):
+    """absmax / 448 (so that the largest magnitude lands on the largest finite code), zero statistic -> 1, fp32."""
+    return _absmax_scale(absmax, F8MAX)
+
+
 def calib_scale(absmax, qmax=QMAX):
     """Calibrated FWQ / SQ scale from an absmax statistic (no truncation tuning, Sec. 3)."""
     return _absmax_scale(absmax, qmax)

@@ -221,6 +221,34 @@ def test_attention_int8_rowmax_tracks_fp_attention_better_at_long_sequences():
     assert err["rowmax"] < 0.02 and err["rowmax"] < 0.2 * err["static"], err
 
 
+def test_fp8_variant_gemm_and_ln_against_plain_definitions():
+    """FP8 GeMM^quant = the fp64 product of the dequantized e4m3 operands pushed through the same epilogue; the output
+    quantizer is e4m3 rounding of v / S; LN^quant with an e4m3 TWQ output reconstructs the LayerNorm to 2^-4 relative."""
+    g = np.random.default_rng(80)
+    n, d, m = 9, 64, 12
+    x = g.standard_normal((n, d)) * 2
+    Wm = g.standard_normal((d, m)) * 0.05
+    b = g.standard_normal(m) * 0.1
+    xq = O.emit(x, O.OutSpec("twq", payload="f8"))
+    assert xq.kind == "f8" and np.all(np.abs(xq.data).max(1) == 448.0)
+    Wq, Sw = O.quant_weight_columnwise_f8(Wm)
+    out = O.gemm_quant_f8(xq, Wq, Sw, b, "none", O.OutSpec("fp", dtype="f64"))
+    ref = xq.real() @ (Wq * Sw[None, :]) + b
+    assert np.allclose(out.data, ref, rtol=1e-13, atol=1e-13)
+    # quantized output with a feature-wise scale: e4m3(v / S) exactly, including saturation
+    S = np.abs(ref).max(0) / 448 / 2                       # half the needed range: the largest entries saturate
+    o8 = O.gemm_quant_f8(xq, Wq, Sw, b, "none", O.OutSpec("fwq", scale=S, payload="f8"))
+    assert np.array_equal(o8.data, Q.e4m3_round(ref / S[None, :])) and np.abs(o8.data).max() == 448.0
+    # closeness to the un-quantized product: e4m3 keeps 4 significant bits per operand
+    assert np.max(np.abs(out.data - (x @ Wm + b))) / np.max(np.abs(x @ Wm + b)) < 0.1
+    # LN^quant -> e4m3 TWQ
+    gam, bet = 1 + 0.1 * g.standard_normal(d), 0.1 * g.standard_normal(d)
+    y, _ = O.ln_quant([O.fp_tensor(x, "f16")], gam, bet, 1e-5, O.OutSpec("twq", payload="f8"))
+    ln = O.layernorm(O.fp_tensor(x, "f16").real(), gam, bet, 1e-5)
+    big = np.abs(ln) > np.abs(ln).max(1, keepdims=True) * 2.0 ** -6
+    assert np.all(np.abs(y.real() - ln)[big] <= np.abs(ln)[big] * 2.0 ** -4 * (1 + 1e-6))
+
+
 # ------------------------------------------------------------------ GeMM^quant
 def test_gemm_quant_equals_fake_quant_path():
     # exact INT32 + scale epilogue == fp64 product of the dequantized operands (before rounding)

@@ -97,3 +97,30 @@ def test_storage_rounding_grids():
     assert Q.round_to_storage(np.array([1.0 + 3 * 2.0 ** -8]), "bf16")[0] == 1.0 + 2.0 ** -6
     assert Q.round_to_storage(np.array([1.0 + 2.0 ** -11]), "f16")[0] == 1.0
     assert Q.round_to_storage(np.array([1.0 + 3 * 2.0 ** -11]), "f16")[0] == 1.0 + 2.0 ** -9
+
+
+# ------------------------------------------------------------------ FP8 (e4m3) quantizer
+def test_e4m3_round_matches_the_library_conversion_and_saturates():
+    import torch
+    g = np.random.default_rng(40)
+    x = np.concatenate([g.standard_normal(20000) * s for s in (1e-3, 0.05, 1.0, 30.0, 200.0)])
+    x = x[np.abs(x) <= 448.0]
+    ref = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    # the library converts through fp32 first; on values exactly representable in fp32 the two agree bit for bit
+    x32 = x.astype(np.float32).astype(np.float64)
+    ref = torch.from_numpy(x32).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(Q.e4m3_round(x32), ref)
+    # every representable e4m3 value is a fixed point
+    codes = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    codes = codes[np.isfinite(codes)]
+    assert np.array_equal(Q.e4m3_round(codes), codes) and codes.max() == 448.0
+    # ties go to the even mantissa; saturation instead of NaN / inf
+    assert Q.e4m3_round(17.0) == 16.0 and Q.e4m3_round(19.0) == 20.0 and Q.e4m3_round(2.0 ** -10) == 0.0
+    assert Q.e4m3_round(1.5 * 2.0 ** -9) == 2.0 ** -8 and Q.e4m3_round(1e9) == 448.0 and Q.e4m3_round(-460.0) == -448.0
+    # scale convention: the largest magnitude lands on 448
+    y = g.standard_normal((7, 64)) * 3
+    s = Q.f8_scale(np.abs(y).max())
+    assert np.abs(Q.quant_f8(y, s)).max() == 448.0
+    # relative reconstruction error of a normal value is at most half a mantissa step (2^-4)
+    big = np.abs(y) > s * 2.0 ** -6
+    assert np.all(np.abs(Q.quant_f8(y, s) * s - y)[big] <= np.abs(y)[big] * 2.0 ** -4 * (1 + 1e-9))
