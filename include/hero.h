@@ -45,7 +45,11 @@ typedef enum {
   HERO_ERR_DEVICE_TIMEOUT = 6
 } hero_status;
 
-typedef enum { HERO_I8 = 0, HERO_U8 = 1, HERO_I32 = 2, HERO_F16 = 3, HERO_BF16 = 4, HERO_F32 = 5 } hero_dtype;
+/* HERO_F8: e4m3 (1 sign, 4 exponent, 3 mantissa bits, largest finite value 448, no infinities): the payload of the FP8
+ * variant of the method (the paper: "the approach carries over to FP8").  An F8 tensor carries scales exactly like an
+ * I8 tensor (TWQ / FWQ / SQ); a scale computed on the fly is absmax / 448 and the quantizer is the saturating
+ * round-to-nearest-even conversion.  Accepted by hero_layernorm_quant (inputs and output) and hero_w8a8_linear. */
+typedef enum { HERO_I8 = 0, HERO_U8 = 1, HERO_I32 = 2, HERO_F16 = 3, HERO_BF16 = 4, HERO_F32 = 5, HERO_F8 = 6 } hero_dtype;
 
 /* Granularity of the scale attached to an INT8 tensor (Eq. 3-5). */
 typedef enum { HERO_GRAN_NONE = 0, HERO_GRAN_TWQ = 1, HERO_GRAN_FWQ = 2, HERO_GRAN_SQ = 3 } hero_gran;

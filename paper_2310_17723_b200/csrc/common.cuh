@@ -8,6 +8,9 @@
 #include <cstring>
 
 #include "../../include/hero.h"
+#ifdef __CUDACC__
+#include <cuda_fp16.h>
+#endif
 
 struct hero_handle {
   int device;
@@ -44,13 +47,17 @@ hero_status cuda_fail(cudaError_t e, const char* what);
 
 inline size_t dtype_size(int dt) {
   switch (dt) {
-    case HERO_I8: case HERO_U8: return 1;
+    case HERO_I8: case HERO_U8: case HERO_F8: return 1;
     case HERO_F16: case HERO_BF16: return 2;
     case HERO_I32: case HERO_F32: return 4;
     default: return 0;
   }
 }
 inline bool is_fp16ish(int dt) { return dt == HERO_F16 || dt == HERO_BF16; }
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline bool is_q8(int dt) { return dt == HERO_I8 || dt == HERO_F8; }   // 8-bit payload that carries a scale
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // data pointer 16-byte aligned, row pitch a multiple of 16 bytes, ld >= cols
@@ -90,6 +97,21 @@ inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 bloc
 
 #ifdef __CUDACC__
 namespace ptx {
+// e4m3 <-> FP32 through the conversion instructions: two values per instruction
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {   // saturating, round to nearest even
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint32_t f32x4_to_e4m3x4(float a, float b, float c, float d) {
+  return f32x2_to_e4m3x2(a, b) | (f32x2_to_e4m3x2(c, d) << 16);
+}
+__device__ __forceinline__ float2 e4m3x2_to_f32x2(uint32_t two) {          // low byte -> .x
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)two));
+  const __half2 h = *reinterpret_cast<const __half2*>(&h2);
+  return __half22float2(h);
+}
 // launch_dependents: the next kernel of the stream may start being scheduled.  wait: returns once the previous kernel
 // of the stream has completed and flushed its writes (immediately if there is none or the launch was an ordinary one).
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -20,7 +20,7 @@ constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK_BYTES = 128;   // one swizzle row
 constexpr int GEMM_THREADS = 320;
 constexpr int TMA_WARP = 8, MMA_WARP = 9;
-constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2;
+constexpr int OUT_I8 = 0, OUT_FP = 1, OUT_I32 = 2, OUT_F8 = 3;
 
 struct GemmParams {
   int M, N, K;              // K in elements
@@ -33,7 +33,8 @@ struct GemmParams {
   long long out_ld;         // elements
   int out_dt;               // hero_dtype
   uint32_t idesc;
-  int elem_bytes;           // 1 (INT8) or 2 (F16 / BF16)
+  int elem_bytes;           // 1 (INT8, e4m3) or 2 (F16 / BF16)
+  int f8;                   // operands are e4m3 (kind::f8f6f4; FP32 accumulators, scales as for INT8)
   int* err;
 };
 
@@ -183,7 +184,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
       if constexpr (ACT == HERO_ACT_NONE) {
         // without an activation the output factor is already folded into cs and bias (see epilogue_loop)
         if constexpr (OUTK == OUT_I8) { y0 = __fadd2_rn(x0, mg2); y1 = __fadd2_rn(x1, mg2); }
-        else { y0 = x0; y1 = x1; }
+        else { y0 = x0; y1 = x1; }                          // FP and e4m3 outputs: the conversion rounds
       } else {
         const float4 p4 = lds_f4(e_post + j);
         if constexpr (ACT == HERO_ACT_GELU_ERF) { x0 = gelu_erf_f2(x0); x1 = gelu_erf_f2(x1); }
@@ -213,11 +214,14 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
       }
     }
     if (!row_ok) return;
-    if constexpr (OUTK == OUT_I8) {
+    if constexpr (OUTK == OUT_I8 || OUTK == OUT_F8) {
       int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
       uint32_t w[NC / 4];
 #pragma unroll
-      for (int g = 0; g < NC / 4; ++g) w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+      for (int g = 0; g < NC / 4; ++g) {
+        if constexpr (OUTK == OUT_F8) w[g] = ptx::f32x4_to_e4m3x4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);   // saturating RNE
+        else w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+      }
       if constexpr (NC == 32) {
         if (wide && col0 + 32 <= p.N) {
           st32(dst, w);
@@ -257,7 +261,7 @@ __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const floa
                                                  int n0, int cpart) {
   constexpr int CH = BN / (EW / 4);
   // 32-byte stores need a 32-byte aligned row segment: base pointer and row pitch multiples of 32 bytes
-  const int es = OUTK == OUT_I8 ? 1 : (OUTK == OUT_FP ? 2 : 4);
+  const int es = (OUTK == OUT_I8 || OUTK == OUT_F8) ? 1 : (OUTK == OUT_FP ? 2 : 4);
   const bool wide = ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0) && ((p.out_ld * es) % 32 == 0);
   if constexpr (EW == 8) {
     constexpr int NCH = CH / 32;
@@ -317,7 +321,7 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
         npost[i] = (in && p.post) ? __ldg(p.post + n) : 1.0f;
       }
       const int m = mt * ROWS + row_off + quarter * 32 + lane;
-      nrs = (INT8 && p.rs && m < p.M) ? __ldg(p.rs + m) : 1.0f;
+      nrs = (p.rs && m < p.M) ? __ldg(p.rs + m) : 1.0f;
     }
   };
   auto publish = [&](int it) {               // registers -> this tile's shared-memory vectors
@@ -449,6 +453,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint64_t ad = ptx::smem_desc(desc_base, a_addr + k * 32);
             const uint64_t bd = ptx::smem_desc(desc_base, b_addr + k * 32);
             if constexpr (INT8) ptx::umma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            else if (p.f8) ptx::umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
             else ptx::umma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
           }
           ptx::umma_commit(&empty[stage]);      // frees the smem stage once these MMAs have read it
@@ -495,6 +500,17 @@ static hero_status dispatch_epilogue(hero_handle* h, const CUtensorMap& tmA, con
   if (p.out_dt == HERO_I32) {
     if constexpr (INT8) return launch_gemm<BN, true, HERO_ACT_NONE, OUT_I32>(h, tmA, tmW, p, s);
     else { set_error("raw INT32 output needs INT8 operands"); return HERO_ERR_UNSUPPORTED; }
+  }
+  if (p.out_dt == HERO_F8) {
+    if constexpr (!INT8) {
+      switch (act) {
+        case HERO_ACT_NONE: return launch_gemm<BN, false, HERO_ACT_NONE, OUT_F8>(h, tmA, tmW, p, s);
+        case HERO_ACT_GELU_ERF: return launch_gemm<BN, false, HERO_ACT_GELU_ERF, OUT_F8>(h, tmA, tmW, p, s);
+        case HERO_ACT_GELU_TANH: return launch_gemm<BN, false, HERO_ACT_GELU_TANH, OUT_F8>(h, tmA, tmW, p, s);
+      }
+    }
+    set_error("an e4m3 output needs e4m3 or FP operands");
+    return HERO_ERR_UNSUPPORTED;
   }
   const bool i8 = p.out_dt == HERO_I8;
   switch (act) {
@@ -627,6 +643,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t ad = ptx::smem_desc(desc_base, a_addr + k * 32);
             const uint64_t bd = ptx::smem_desc(desc_base, b_addr + k * 32);
             if constexpr (INT8) ptx::umma_i8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            else if (p.f8) ptx::umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
             else ptx::umma_f16_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
           }
           ptx::umma_commit_pair(&empty[stage], 3);       // frees this stage in both CTAs
@@ -686,6 +703,17 @@ static hero_status dispatch_epilogue_pair(hero_handle* h, const CUtensorMap& tmA
     if constexpr (INT8) return launch_gemm_pair<true, HERO_ACT_NONE, OUT_I32>(h, tmA, tmW, p, s);
     else { set_error("raw INT32 output needs INT8 operands"); return HERO_ERR_UNSUPPORTED; }
   }
+  if (p.out_dt == HERO_F8) {
+    if constexpr (!INT8) {
+      switch (act) {
+        case HERO_ACT_NONE: return launch_gemm_pair<false, HERO_ACT_NONE, OUT_F8>(h, tmA, tmW, p, s);
+        case HERO_ACT_GELU_ERF: return launch_gemm_pair<false, HERO_ACT_GELU_ERF, OUT_F8>(h, tmA, tmW, p, s);
+        case HERO_ACT_GELU_TANH: return launch_gemm_pair<false, HERO_ACT_GELU_TANH, OUT_F8>(h, tmA, tmW, p, s);
+      }
+    }
+    set_error("an e4m3 output needs e4m3 or FP operands");
+    return HERO_ERR_UNSUPPORTED;
+  }
   const bool i8 = p.out_dt == HERO_I8;
   switch (act) {
     case HERO_ACT_NONE:
@@ -703,13 +731,14 @@ static hero_status dispatch_epilogue_pair(hero_handle* h, const CUtensorMap& tmA
 }
 
 static hero_status run_pair(hero_handle* h, const hero_linear_args* a, GemmParams& p, cudaStream_t s) {
-  const bool int8 = a->A.dtype == HERO_I8;
-  const int eb = int8 ? 1 : 2;
+  const bool int8 = a->A.dtype == HERO_I8, f8 = a->A.dtype == HERO_F8;
+  const int eb = (int8 || f8) ? 1 : 2;
   const int kbox = GEMM_BK_BYTES / eb;
   p.num_m_tiles = (p.M + 255) / 256;
   p.num_n_tiles = (p.N + 255) / 256;
   const bool bf = a->A.dtype == HERO_BF16;
-  p.idesc = int8 ? ptx::make_idesc(2, 1, 1, 0, 0, 256, 256) : ptx::make_idesc(1, bf ? 1 : 0, bf ? 1 : 0, 0, 0, 256, 256);
+  p.idesc = int8 ? ptx::make_idesc(2, 1, 1, 0, 0, 256, 256)
+                 : (f8 ? ptx::make_idesc(1, 0, 0, 0, 0, 256, 256) : ptx::make_idesc(1, bf ? 1 : 0, bf ? 1 : 0, 0, 0, 256, 256));
   CUtensorMap tmA, tmW;
   hero_status st = make_tmap_2d(h, &tmA, a->A.data, eb, a->A.dtype == HERO_F16, bf, (uint64_t)p.M, (uint64_t)p.K,
                                 (uint64_t)a->A.ld * eb, kbox, GEMM_BM, 128);
@@ -723,12 +752,13 @@ static hero_status run_pair(hero_handle* h, const hero_linear_args* a, GemmParam
 
 template <int BN>
 static hero_status run_bn(hero_handle* h, const hero_linear_args* a, GemmParams& p, cudaStream_t s) {
-  const bool int8 = a->A.dtype == HERO_I8;
-  const int eb = int8 ? 1 : 2;
+  const bool int8 = a->A.dtype == HERO_I8, f8 = a->A.dtype == HERO_F8;
+  const int eb = (int8 || f8) ? 1 : 2;
   const int kbox = GEMM_BK_BYTES / eb;
   p.num_n_tiles = (p.N + BN - 1) / BN;
   p.idesc = int8 ? ptx::make_idesc(2, 1, 1, 0, 0, GEMM_BM, BN)
-                 : ptx::make_idesc(1, a->A.dtype == HERO_BF16 ? 1 : 0, a->A.dtype == HERO_BF16 ? 1 : 0, 0, 0, GEMM_BM, BN);
+                 : (f8 ? ptx::make_idesc(1, 0, 0, 0, 0, GEMM_BM, BN)
+                       : ptx::make_idesc(1, a->A.dtype == HERO_BF16 ? 1 : 0, a->A.dtype == HERO_BF16 ? 1 : 0, 0, 0, GEMM_BM, BN));
   CUtensorMap tmA, tmW;
   hero_status st = make_tmap_2d(h, &tmA, a->A.data, eb, a->A.dtype == HERO_F16, a->A.dtype == HERO_BF16, (uint64_t)p.M,
                                 (uint64_t)p.K, (uint64_t)a->A.ld * eb, kbox, GEMM_BM, 128);
@@ -750,9 +780,9 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   hero_status st;
   if ((st = check_matrix(a->A, "A")) != HERO_OK) return st;
   if ((st = check_matrix(a->out, "out")) != HERO_OK) return st;
-  const bool int8 = a->A.dtype == HERO_I8;
-  HERO_REQUIRE(int8 || is_fp16ish(a->A.dtype), HERO_ERR_UNSUPPORTED, "A dtype %d: INT8, F16 or BF16 expected", a->A.dtype);
-  const int eb = int8 ? 1 : 2;
+  const bool int8 = a->A.dtype == HERO_I8, f8 = a->A.dtype == HERO_F8, q8 = int8 || f8;
+  HERO_REQUIRE(q8 || is_fp16ish(a->A.dtype), HERO_ERR_UNSUPPORTED, "A dtype %d: INT8, e4m3, F16 or BF16 expected", a->A.dtype);
+  const int eb = q8 ? 1 : 2;
   HERO_REQUIRE(a->W != nullptr && aligned16(a->W), a->W ? HERO_ERR_ALIGNMENT : HERO_ERR_INVALID_ARG,
                "W must be a 16-byte aligned device pointer");
   HERO_REQUIRE(a->N > 0 && a->N % 16 == 0, HERO_ERR_UNSUPPORTED, "N=%lld must be a positive multiple of 16", (long long)a->N);
@@ -760,13 +790,15 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   HERO_REQUIRE((K * eb) % 16 == 0, HERO_ERR_UNSUPPORTED, "K=%lld: K * element size must be a multiple of 16 bytes", K);
   HERO_REQUIRE(a->ldw >= K && (a->ldw * eb) % 16 == 0, HERO_ERR_ALIGNMENT, "ldw=%lld invalid", (long long)a->ldw);
   HERO_REQUIRE(a->out.rows == a->A.rows && a->out.cols == a->N, HERO_ERR_INVALID_ARG, "out shape mismatch");
-  HERO_REQUIRE(a->out.dtype == HERO_I8 || is_fp16ish(a->out.dtype) || a->out.dtype == HERO_I32, HERO_ERR_UNSUPPORTED,
+  HERO_REQUIRE(is_q8(a->out.dtype) || is_fp16ish(a->out.dtype) || a->out.dtype == HERO_I32, HERO_ERR_UNSUPPORTED,
                "out dtype %d", a->out.dtype);
-  HERO_REQUIRE(!(a->out.dtype == HERO_I8 && a->out.gran == HERO_GRAN_TWQ), HERO_ERR_UNSUPPORTED,
+  HERO_REQUIRE(a->out.dtype != HERO_F8 || !int8, HERO_ERR_UNSUPPORTED, "an e4m3 output needs e4m3 or FP operands");
+  HERO_REQUIRE(a->out.dtype != HERO_I8 || !f8, HERO_ERR_UNSUPPORTED, "an INT8 output needs INT8 or FP operands");
+  HERO_REQUIRE(!(is_q8(a->out.dtype) && a->out.gran == HERO_GRAN_TWQ), HERO_ERR_UNSUPPORTED,
                "a token-wise (TWQ) output needs a row reduction, which is kept out of GEMM epilogues (Sec. 2.1); "
                "fuse it into LN^quant instead");
   HERO_REQUIRE(a->out.dtype != HERO_I32 || int8, HERO_ERR_UNSUPPORTED, "raw INT32 output needs INT8 operands");
-  if (int8) HERO_REQUIRE(a->w_scale != nullptr || a->out.dtype == HERO_I32, HERO_ERR_INVALID_ARG, "w_scale is required");
+  if (q8) HERO_REQUIRE(a->w_scale != nullptr || a->out.dtype == HERO_I32, HERO_ERR_INVALID_ARG, "w_scale is required");
   HERO_REQUIRE(a->act >= HERO_ACT_NONE && a->act <= HERO_ACT_GELU_TANH, HERO_ERR_INVALID_ARG, "unknown activation %d", a->act);
   HERO_REQUIRE(a->A.rows < (1ll << 31) && a->N < (1ll << 31) && K < (1ll << 31), HERO_ERR_UNSUPPORTED, "dimension too large");
   if (a->A.rows == 0) return HERO_OK;
@@ -776,8 +808,9 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   p.M = (int)a->A.rows; p.N = (int)a->N; p.K = (int)K;
   p.num_m_tiles = (p.M + GEMM_BM - 1) / GEMM_BM;
   p.num_kb = (int)((K * eb + GEMM_BK_BYTES - 1) / GEMM_BK_BYTES);
-  p.rs = (int8 && a->A.gran == HERO_GRAN_TWQ) ? a->A.scale : nullptr;
-  p.cs = int8 ? a->w_scale : nullptr;
+  p.rs = (q8 && a->A.gran == HERO_GRAN_TWQ) ? a->A.scale : nullptr;
+  p.cs = q8 ? a->w_scale : nullptr;
+  p.f8 = f8 ? 1 : 0;
   p.bias = a->bias; p.post = a->post_scale;
   p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
   p.elem_bytes = eb;

@@ -64,6 +64,12 @@ __device__ __forceinline__ void unpack(const uint32_t (&w)[VEC / 2], int dt, flo
 #pragma unroll
       for (int b = 0; b < 4; ++b) v[4 * i + b] = (float)(int)(signed char)((w[i] >> (8 * b)) & 0xff);
     }
+  } else if (dt == HERO_F8) {
+#pragma unroll
+    for (int i = 0; i < VEC / 4; ++i) {
+      const float2 lo = ptx::e4m3x2_to_f32x2(w[i] & 0xffffu), hi = ptx::e4m3x2_to_f32x2(w[i] >> 16);
+      v[4 * i] = lo.x; v[4 * i + 1] = lo.y; v[4 * i + 2] = hi.x; v[4 * i + 3] = hi.y;
+    }
   } else if (dt == HERO_F16) {
 #pragma unroll
     for (int i = 0; i < VEC / 2; ++i) {
@@ -175,8 +181,8 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
     for (int i = 0; i < VEC; ++i) { gam[i] = 0.f; bet[i] = 0.f; }
   }
 
-  const int res_es = (p.res.dt == HERO_I8) ? 1 : 2;
-  const int br_es = (p.br.dt == HERO_I8) ? 1 : 2;
+  const int res_es = is_q8(p.res.dt) ? 1 : 2;
+  const int br_es = is_q8(p.br.dt) ? 1 : 2;
   const long long rows_per_trip = (long long)RPC * R;
 
   for (long long base = (long long)blockIdx.x * rows_per_trip; base < p.M; base += (long long)gridDim.x * rows_per_trip) {
@@ -215,7 +221,7 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
     for (int r = 0; r < R; ++r) {
       if (valid[r]) {
         unpack<VEC>(raw_res[r], p.res.dt, x[r]);
-        if (p.res.dt == HERO_I8) {
+        if (is_q8(p.res.dt)) {
           if (p.res.col_scale) {
 #pragma unroll
             for (int i = 0; i < VEC; ++i) x[r][i] *= rs_res[r] * __ldg(p.res.col_scale + (c0 + i) * p.res.col_stride);
@@ -227,7 +233,7 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
         if constexpr (HAS_BR) {
           float b[VEC];
           unpack<VEC>(raw_br[r], p.br.dt, b);
-          if (p.br.dt == HERO_I8) {
+          if (is_q8(p.br.dt)) {
             if (p.br.col_scale) {
 #pragma unroll
               for (int i = 0; i < VEC; ++i)
@@ -301,14 +307,15 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
       amax[r] = m;
     }
 
-    if (p.out_dt == HERO_I8) {
+    if (is_q8(p.out_dt)) {
+      const bool f8 = p.out_dt == HERO_F8;
       float inv[R];
       if (p.out_gran == HERO_GRAN_TWQ) {
-        // Eq. 3: S[i] = absmax / 127 computed on the fly, in the same pass
+        // Eq. 3: S[i] = absmax / 127 (absmax / 448 for an e4m3 payload) computed on the fly, in the same pass
         row_reduce<R, true>(amax, red2, G, row_in_cta, t);
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-          float sc = amax[r] > 0.f ? amax[r] / 127.0f : 1.0f;
+          float sc = amax[r] > 0.f ? amax[r] / (f8 ? 448.0f : 127.0f) : 1.0f;
           inv[r] = 1.0f / sc;
           if (t == 0 && row[r] < p.M) p.out_scale[row[r]] = sc;
         }
@@ -319,8 +326,10 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
         uint32_t w[VEC / 4];
         if (p.out_gran == HERO_GRAN_TWQ) {
 #pragma unroll
-          for (int i = 0; i < VEC / 4; ++i)
-            w[i] = quant4(x[r][4 * i] * inv[r], x[r][4 * i + 1] * inv[r], x[r][4 * i + 2] * inv[r], x[r][4 * i + 3] * inv[r]);
+          for (int i = 0; i < VEC / 4; ++i) {
+            const float a = x[r][4 * i] * inv[r], b = x[r][4 * i + 1] * inv[r], c = x[r][4 * i + 2] * inv[r], d = x[r][4 * i + 3] * inv[r];
+            w[i] = f8 ? ptx::f32x4_to_e4m3x4(a, b, c, d) : quant4(a, b, c, d);
+          }
         } else {
           // Eq. 4 / 5: calibrated per-feature (stride 1) or static (stride 0) scale
           const int st = (p.out_gran == HERO_GRAN_FWQ) ? 1 : 0;
@@ -328,7 +337,9 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
 #pragma unroll
           for (int i = 0; i < VEC; ++i) q[i] = x[r][i] / __ldg(p.out_scale + (c0 + i) * st);
 #pragma unroll
-          for (int i = 0; i < VEC / 4; ++i) w[i] = quant4(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3]);
+          for (int i = 0; i < VEC / 4; ++i)
+            w[i] = f8 ? ptx::f32x4_to_e4m3x4(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3])
+                      : quant4(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3]);
         }
         store_words<VEC>(reinterpret_cast<char*>(p.out) + row[r] * p.out_ld + c0, w, VEC / 4);
       }
@@ -351,10 +362,10 @@ static hero_status fill_side(const hero_tensor& t, LnSide* s, const char* name, 
   hero_status st = check_matrix(t, name);
   if (st != HERO_OK) return st;
   HERO_REQUIRE(t.cols == H, HERO_ERR_INVALID_ARG, "%s: cols %lld != H %d", name, (long long)t.cols, H);
-  HERO_REQUIRE(is_fp16ish(t.dtype) || (allow_i8 && t.dtype == HERO_I8), HERO_ERR_UNSUPPORTED,
+  HERO_REQUIRE(is_fp16ish(t.dtype) || (allow_i8 && is_q8(t.dtype)), HERO_ERR_UNSUPPORTED,
                "%s: dtype %d not accepted here", name, t.dtype);
   s->data = t.data; s->dt = t.dtype; s->ld = t.ld;
-  if (t.dtype == HERO_I8) {
+  if (is_q8(t.dtype)) {
     if (t.gran == HERO_GRAN_TWQ) s->row_scale = t.scale;
     if (t.gran == HERO_GRAN_FWQ) { s->col_scale = t.scale; s->col_stride = 1; }
     if (t.gran == HERO_GRAN_SQ) { s->col_scale = t.scale; s->col_stride = 0; }
@@ -1210,6 +1221,7 @@ static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) 
 static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
   if (!(p.H == 1024 || p.H == 2048 || p.H == 4096 || p.H == 8192) || p.ex.data || p.token_ids) return HERO_OK;
+  if (p.res.dt == HERO_F8 || (p.br.data && p.br.dt == HERO_F8) || (p.out && p.out_dt == HERO_F8)) return HERO_OK;   // generic kernel
   const int res = p.res.dt == HERO_I8 ? SRC_I8 : SRC_FP;
   const int br = !p.br.data ? SRC_NONE : (p.br.dt == HERO_I8 ? SRC_I8 : SRC_FP);
   const int out = !p.out ? O_NONE : (p.out_dt != HERO_I8 ? O_FP : (p.out_gran == HERO_GRAN_TWQ ? O_TWQ : O_STATIC));
@@ -1253,6 +1265,7 @@ static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* t
 static hero_status try_fast(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
   if (p.H % 8 != 0 || p.H > 8192) return HERO_OK;
+  if (p.res.dt == HERO_F8 || (p.br.data && p.br.dt == HERO_F8) || (p.out && p.out_dt == HERO_F8)) return HERO_OK;   // generic kernel
   const int res = p.res.dt == HERO_I8 ? SRC_I8 : SRC_FP;
   const int br = !p.br.data ? SRC_NONE : (p.br.dt == HERO_I8 ? SRC_I8 : SRC_FP);
   const bool ex = p.ex.data != nullptr;
@@ -1334,10 +1347,10 @@ extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* 
     HERO_REQUIRE(a->gamma && a->beta, HERO_ERR_INVALID_ARG, "gamma and beta are required");
     HERO_REQUIRE(aligned16(a->gamma) && aligned16(a->beta), HERO_ERR_ALIGNMENT, "gamma/beta must be 16-byte aligned");
     HERO_REQUIRE(a->out.rows == p.M && a->out.cols == H, HERO_ERR_INVALID_ARG, "out shape mismatch");
-    HERO_REQUIRE(a->out.dtype == HERO_I8 || is_fp16ish(a->out.dtype), HERO_ERR_UNSUPPORTED, "out dtype %d", a->out.dtype);
-    if (a->out.dtype == HERO_I8)
+    HERO_REQUIRE(is_q8(a->out.dtype) || is_fp16ish(a->out.dtype), HERO_ERR_UNSUPPORTED, "out dtype %d", a->out.dtype);
+    if (is_q8(a->out.dtype))
       HERO_REQUIRE(a->out.gran == HERO_GRAN_TWQ || a->out.gran == HERO_GRAN_FWQ || a->out.gran == HERO_GRAN_SQ,
-                   HERO_ERR_INVALID_ARG, "INT8 out needs granularity TWQ, FWQ or SQ");
+                   HERO_ERR_INVALID_ARG, "an 8-bit out needs granularity TWQ, FWQ or SQ");
     p.out = a->out.data; p.out_dt = a->out.dtype; p.out_ld = a->out.ld; p.out_gran = a->out.gran;
     p.out_scale = a->out.scale;
   }

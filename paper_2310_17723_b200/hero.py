@@ -21,8 +21,9 @@ MODE_INT8, MODE_FP = range(2)
 PRESET_FP, PRESET_M1, PRESET_M2, PRESET_M3 = range(4)
 MODULES = ("qkv", "attn", "attn_out", "fc1", "fc2")
 
+F8 = 6                      # e4m3 payload of the FP8 variant
 _DT = {torch.int8: I8, torch.uint8: U8, torch.int32: I32, torch.float16: F16, torch.bfloat16: BF16,
-       torch.float32: F32}
+       torch.float32: F32, torch.float8_e4m3fn: F8}
 GRAN = {"none": GRAN_NONE, "twq": GRAN_TWQ, "fwq": GRAN_FWQ, "sq": GRAN_SQ, "fp": GRAN_NONE}
 ACT = {"none": ACT_NONE, "gelu_erf": ACT_GELU_ERF, "gelu_tanh": ACT_GELU_TANH}
 MASK = {"none": MASK_NONE, "causal": MASK_CAUSAL}

@@ -61,12 +61,15 @@ def bench_ln(h, M, H, kind, iters):
           % (kind, M, H, t * 1e6, gbs, gbs / hbm, src), flush=True)
 
 
-def bench_gemm(h, M, K, N, act, fp, iters):
-    dt = torch.bfloat16 if fp else torch.int8
+def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
+    dt = torch.bfloat16 if fp else (torch.float8_e4m3fn if f8 else torch.int8)
     n = max(2, min(8, int(300e6 // (M * K + N * K + M * N)) + 1))
     if fp:
         As = [torch.randn(M, K, device="cuda", dtype=dt) for _ in range(n)]
         Ws = [torch.randn(N, K, device="cuda", dtype=dt) for _ in range(n)]
+    elif f8:
+        As = [(torch.randn(M, K, device="cuda") * 100).to(dt) for _ in range(n)]
+        Ws = [(torch.randn(N, K, device="cuda") * 100).to(dt) for _ in range(n)]
     else:
         As = [torch.randint(-127, 128, (M, K), device="cuda", dtype=dt) for _ in range(n)]
         Ws = [torch.randint(-127, 128, (N, K), device="cuda", dtype=dt) for _ in range(n)]
@@ -82,7 +85,7 @@ def bench_gemm(h, M, K, N, act, fp, iters):
     peak = i8peak / 2 if fp else i8peak
     tops = 2.0 * M * N * K / t / 1e12
     print("GeMM^quant %s M=%d K=%d N=%d act=%s: %.1f us, %.0f TOP/s, %.2f of 2 x %s BF16 peak%s"
-          % ("bf16" if fp else "i8", M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else ""), flush=True)
+          % ("bf16" if fp else ("e4m3" if f8 else "i8"), M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else ""), flush=True)
 
 
 def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static"):
@@ -141,6 +144,7 @@ def main():
     ap.add_argument("--mask", default="none")
     ap.add_argument("--p-mode", default="static", choices=["static", "rowmax"])
     ap.add_argument("--fp", action="store_true")
+    ap.add_argument("--f8", action="store_true", help="e4m3 operands and output (the FP8 variant)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--sweep", action="store_true")
     a = ap.parse_args()
@@ -156,9 +160,9 @@ def main():
         if a.sweep:
             for K, N in W.GEMM_SWEEP_KN:
                 for M in W.GEMM_SWEEP_M:
-                    bench_gemm(h, M, K, N, a.act, a.fp, a.iters)
+                    bench_gemm(h, M, K, N, a.act, a.fp, a.iters, a.f8)
         else:
-            bench_gemm(h, a.M, a.K, a.N, a.act, a.fp, a.iters)
+            bench_gemm(h, a.M, a.K, a.N, a.act, a.fp, a.iters, a.f8)
     elif a.kernel == "absmax":
         bench_absmax(h, a.M, a.H, a.iters)
     elif a.kernel == "wquant":
