@@ -312,6 +312,29 @@ def attention_int8(q_i8, k_i8, v_i8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutS
     return (o, internals) if return_internals else o
 
 
+def attention_f8(q_f8, k_f8, v_f8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutSpec, mask="none", key_len=None):
+    """The FP8 variant of the attention core: e4m3 Q, K, V (values, SQ scales s_q, s_k, s_v) and an e4m3 P.
+
+    per (b, h):  A = d~ (Q K^T),  d~ = s_q s_k / sqrt(dh);  P = softmax(A) over the allowed keys;
+                 P_f8 = e4m3(P / s_p)  (s_p = max P / 448 from calibration; saturating);
+                 acc = P_f8 V_f8;  X_attn = s_p s_v acc -> output stage.
+    Every product of two e4m3 values and every partial sum here is exact in fp64.
+    """
+    H = nh * dh
+    d_tilde = float(s_q) * float(s_k) / np.sqrt(float(dh))
+    x_attn = np.zeros((B * S, H), dtype=np.float64)
+    for b in range(B):
+        allowed = attention_mask(S, mask, None if key_len is None else key_len[b])
+        rows = slice(b * S, (b + 1) * S)
+        for h in range(nh):
+            cols = slice(h * dh, (h + 1) * dh)
+            A = d_tilde * (np.asarray(q_f8[rows, cols], np.float64) @ np.asarray(k_f8[rows, cols], np.float64).T)
+            P = softmax_masked(A, allowed)
+            P_f8 = Q.quant_f8(P, s_p)
+            x_attn[rows, cols] = float(s_p) * float(s_v) * (P_f8 @ np.asarray(v_f8[rows, cols], np.float64))
+    return emit(x_attn, out)
+
+
 def attention_fp(q, k, v, B, S, nh, dh, out: OutSpec, mask="none", key_len=None):
     """FP-mode attention (Eq. 9-11): softmax(Q K^T / sqrt(dh)) V in fp64 on the stored operands."""
     H = nh * dh

@@ -249,6 +249,31 @@ def test_fp8_variant_gemm_and_ln_against_plain_definitions():
     assert np.all(np.abs(y.real() - ln)[big] <= np.abs(ln)[big] * 2.0 ** -4 * (1 + 1e-6))
 
 
+def test_fp8_attention_closed_forms_and_closeness():
+    g = np.random.default_rng(81)
+    # uniform logits: P = 1/S, P_f8 = e4m3(448 / S) for every key -> X_attn = s_p s_v e4m3(1 / (S s_p)) * column sum of V
+    S, dh = 96, 16
+    q = np.zeros((S, dh))
+    k = Q.e4m3_round(g.standard_normal((S, dh)) * 50)
+    v = Q.e4m3_round(g.standard_normal((S, dh)) * 50)
+    s_p = (1.0 / S) / 448
+    o = O.attention_f8(q, k, v, 1, S, 1, dh, 0.01, 0.01, 0.02, s_p, O.OutSpec("fp", dtype="f64")).data
+    assert np.allclose(o, np.broadcast_to(s_p * 0.02 * 448.0 * v.sum(0), o.shape), rtol=1e-13)
+    # causal row 0 sees key 0 only: P = 1 -> saturates at 448 when s_p < 1 / 448 -> X_attn[0] = s_p s_v 448 V[0]
+    q = Q.e4m3_round(g.standard_normal((S, dh)) * 50)
+    o = O.attention_f8(q, k, v, 1, S, 1, dh, 0.01, 0.01, 0.02, 1.0 / 448, O.OutSpec("fp", dtype="f64"), mask="causal").data
+    assert np.allclose(o[0], 0.02 * v[0], rtol=1e-13)
+    o2 = O.attention_f8(q, k, v, 1, S, 1, dh, 0.01, 0.01, 0.02, 0.5 / 448, O.OutSpec("fp", dtype="f64"), mask="causal").data
+    assert np.allclose(o2[0], 0.5 * 0.02 * v[0], rtol=1e-13)                    # clipped at 448: half the mass survives
+    # close to FP attention of the dequantized operands (4 significant bits in P)
+    qf, kf, vf = (g.standard_normal((64, 32)) for _ in range(3))
+    s_q, s_k, s_v = (np.abs(a).max() / 448 for a in (qf, kf, vf))
+    qi, ki, vi = Q.quant_f8(qf, s_q), Q.quant_f8(kf, s_k), Q.quant_f8(vf, s_v)
+    got = O.attention_f8(qi, ki, vi, 1, 64, 2, 16, s_q, s_k, s_v, 1.0 / 448, O.OutSpec("fp", dtype="f64")).data
+    ref = O.attention_fp(qi * s_q, ki * s_k, vi * s_v, 1, 64, 2, 16, O.OutSpec("fp", dtype="f64")).data
+    assert np.max(np.abs(got - ref)) / np.max(np.abs(ref)) < 0.05
+
+
 # ------------------------------------------------------------------ GeMM^quant
 def test_gemm_quant_equals_fake_quant_path():
     # exact INT32 + scale epilogue == fp64 product of the dequantized operands (before rounding)
