@@ -45,7 +45,8 @@ struct AttnCfg {
 
 // ROWMAX: P quantized against the row maximum (see attention_resident.cu): sweep 1 then only finds the maximum of the
 // integer scores, sweep 2 does the one exponential per score and sums the un-quantized exponentials.
-template <int DH, bool ROWMAX>
+// F8: e4m3 Q, K, V and an e4m3 P (the FP8 variant): kind::f8f6f4 MMAs, FP32 scores and accumulator, static s_p.
+template <int DH, bool ROWMAX, bool F8 = false>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -150,8 +151,10 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
 #pragma unroll
         for (int k = 0; k < ATT_BN / 32; ++k)
-          ptx::umma_i8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                       ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (j | k) != 0);
+          if constexpr (F8) ptx::umma_f8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
+                                         ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (j | k) != 0);
+          else ptx::umma_i8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
+                            ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (j | k) != 0);
         ptx::umma_commit(&v_empty[vs]);
         ptx::umma_commit(&p_empty[pb]);
         ++vcnt; ++pcnt;
@@ -173,8 +176,10 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
 #pragma unroll
           for (int k = 0; k < DH / 32; ++k)
-            ptx::umma_i8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                         ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+            if constexpr (F8) ptx::umma_f8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                                           ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+            else ptx::umma_i8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                              ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
           ptx::umma_commit(&k_empty[ks]);
           ptx::umma_commit(&s_full[sb]);
           ++kcnt; ++scnt;
@@ -245,6 +250,13 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const int kb = i * ATT_BN + cq * 32;
           const int nvalid = min(32, kmax - kb + 1);       // keys kb .. kb + nvalid - 1 are allowed
           if (nvalid > 0) {
+            float m_blk;
+            if constexpr (F8) {
+              float fm = -INFINITY;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) fm = fmaxf(fm, j < nvalid ? __uint_as_float(r[j]) : -INFINITY);
+              m_blk = fm * c2;
+            } else {
             int imax = INT_MIN;
             if (nvalid == 32) {
 #pragma unroll
@@ -253,10 +265,15 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
               for (int j = 0; j < 32; ++j) imax = max(imax, j < nvalid ? (int)r[j] : INT_MIN);
             }
-            const float m_new = fmaxf(m, (float)imax * c2);
+              m_blk = (float)imax * c2;
+            }
+            const float m_new = fmaxf(m, m_blk);
             float2 acc2 = make_float2(0.f, 0.f);
             const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_new, -m_new), mg = make_float2(-ATT_MAGIC, -ATT_MAGIC);
-            if (nvalid == 32) {
+            if constexpr (F8) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) acc2.x += j < nvalid ? ex2f(fmaf(__uint_as_float(r[j]), c2, -m_new)) : 0.f;
+            } else if (nvalid == 32) {
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
                 const float2 f = __fadd2_rn(make_float2(__uint_as_float(0x4B400000u + r[j]), __uint_as_float(0x4B400000u + r[j + 1])), mg);
@@ -335,6 +352,15 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
               y[e] = v.x; y[e + 1] = v.y;
             }
             l += acc2.x + acc2.y;
+          } else if constexpr (F8) {
+            // P / s_p as a float; the conversion to e4m3 (saturating at 448, round to nearest even) happens at the pack
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float2 tt = __ffma2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), c22, nm2);
+              const float2 v = __fmul2_rn(make_float2(ex2f(tt.x), ex2f(tt.y)), ps2);
+              y[e] = e < nvalid ? v.x : 0.f;
+              y[e + 1] = e + 1 < nvalid ? v.y : 0.f;
+            }
           } else {
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
@@ -351,11 +377,20 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
           }
           const int c16 = cq * 2;                              // 16-byte chunk index within the 128-byte row
+          if constexpr (F8) {
+            st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), ptx::f32x4_to_e4m3x4(y[0], y[1], y[2], y[3]),
+                        ptx::f32x4_to_e4m3x4(y[4], y[5], y[6], y[7]), ptx::f32x4_to_e4m3x4(y[8], y[9], y[10], y[11]),
+                        ptx::f32x4_to_e4m3x4(y[12], y[13], y[14], y[15]));
+            st_shared16(prow + (((c16 + 1) ^ (r_loc & 7)) << 4), ptx::f32x4_to_e4m3x4(y[16], y[17], y[18], y[19]),
+                        ptx::f32x4_to_e4m3x4(y[20], y[21], y[22], y[23]), ptx::f32x4_to_e4m3x4(y[24], y[25], y[26], y[27]),
+                        ptx::f32x4_to_e4m3x4(y[28], y[29], y[30], y[31]));
+          } else {
           st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), low_bytes4_u(y[0], y[1], y[2], y[3]), low_bytes4_u(y[4], y[5], y[6], y[7]),
                       low_bytes4_u(y[8], y[9], y[10], y[11]), low_bytes4_u(y[12], y[13], y[14], y[15]));
           st_shared16(prow + (((c16 + 1) ^ (r_loc & 7)) << 4), low_bytes4_u(y[16], y[17], y[18], y[19]),
                       low_bytes4_u(y[20], y[21], y[22], y[23]), low_bytes4_u(y[24], y[25], y[26], y[27]),
                       low_bytes4_u(y[28], y[29], y[30], y[31]));
+          }
         }
         ptx::tc_fence_before();
         ptx::fence_proxy_async_smem();                         // generic-proxy writes -> visible to the UMMA (async proxy)
@@ -395,11 +430,24 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int ocol = cq * 32;
         const long long grow = (long long)(row_base + q);
         const int gcol = col0 + ocol;
-        if (p.out_dt == HERO_I8) {
+        auto accf = [&](int j) -> float { return F8 ? __uint_as_float(r[j]) : (float)(int)r[j]; };
+        if (p.out_dt == HERO_F8) {
           float v[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            v[j] = (float)(int)r[j] * rowf * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
+            v[j] = accf(j) * rowf * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
+          uint8_t* dst = reinterpret_cast<uint8_t*>(p.out) + grow * p.out_ld + gcol;
+#pragma unroll
+          for (int g = 0; g < 2; ++g)
+            st_g16(dst + 16 * g, ptx::f32x4_to_e4m3x4(v[16 * g], v[16 * g + 1], v[16 * g + 2], v[16 * g + 3]),
+                   ptx::f32x4_to_e4m3x4(v[16 * g + 4], v[16 * g + 5], v[16 * g + 6], v[16 * g + 7]),
+                   ptx::f32x4_to_e4m3x4(v[16 * g + 8], v[16 * g + 9], v[16 * g + 10], v[16 * g + 11]),
+                   ptx::f32x4_to_e4m3x4(v[16 * g + 12], v[16 * g + 13], v[16 * g + 14], v[16 * g + 15]));
+        } else if (p.out_dt == HERO_I8) {
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            v[j] = accf(j) * rowf * (p.pv_scale / __ldg(p.out_scale + (gcol + j) * p.out_scale_stride));
           int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
 #pragma unroll
           for (int g = 0; g < 2; ++g)
@@ -413,7 +461,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int g = 0; g < 4; ++g) {
             float v[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * rowf * p.pv_scale;
+            for (int e = 0; e < 8; ++e) v[e] = accf(8 * g + e) * rowf * p.pv_scale;
             st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
                    fp2(v[6], v[7], p.out_dt));
           }
@@ -427,7 +475,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <int DH, bool ROWMAX>
+template <int DH, bool ROWMAX, bool F8 = false>
 static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
   using Cfg = AttnCfg<DH>;
   const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
@@ -436,9 +484,14 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
   if ((st = make_tmap_2d(h, &tq, a->q, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BM, DH)) != HERO_OK) return st;
   if ((st = make_tmap_2d(h, &tk, a->k, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BN, DH)) != HERO_OK) return st;
   if ((st = make_tmap_2d(h, &tv, a->v, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BN, DH)) != HERO_OK) return st;
-  p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN);   // S8 x S8 -> S32, both K-major
-  p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);       // U8 x S8 -> S32, V is MN-major
-  auto kern = attn_int8_kernel<DH, ROWMAX>;
+  if (F8) {
+    p.idesc_qk = ptx::make_idesc(1, 0, 0, 0, 0, ATT_BM, ATT_BN); // E4M3 x E4M3 -> F32, both K-major
+    p.idesc_pv = ptx::make_idesc(1, 0, 0, 0, 1, ATT_BM, DH);     // E4M3 x E4M3 -> F32, V is MN-major
+  } else {
+    p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN); // S8 x S8 -> S32, both K-major
+    p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);     // U8 x S8 -> S32, V is MN-major
+  }
+  auto kern = attn_int8_kernel<DH, ROWMAX, F8>;
   static bool configured = false;
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
@@ -462,8 +515,11 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   HERO_REQUIRE(a->q && a->k && a->v, HERO_ERR_INVALID_ARG, "q, k, v are required");
   HERO_REQUIRE(a->B >= 0 && a->S > 0 && a->nh > 0, HERO_ERR_INVALID_ARG, "bad B / S / nh");
   HERO_REQUIRE(a->dh == 64 || a->dh == 128, HERO_ERR_UNSUPPORTED, "dh=%d: 64 or 128 supported", a->dh);
-  const bool fp_in = is_fp16ish(a->dtype);
-  HERO_REQUIRE(a->dtype == HERO_I8 || fp_in, HERO_ERR_UNSUPPORTED, "q/k/v dtype %d: INT8, F16 or BF16 expected", a->dtype);
+  const bool fp_in = is_fp16ish(a->dtype), f8_in = a->dtype == HERO_F8;
+  HERO_REQUIRE(a->dtype == HERO_I8 || f8_in || fp_in, HERO_ERR_UNSUPPORTED, "q/k/v dtype %d: INT8, e4m3, F16 or BF16 expected", a->dtype);
+  HERO_REQUIRE(!f8_in || a->p_mode == HERO_P_STATIC, HERO_ERR_UNSUPPORTED, "the e4m3 core quantizes P with the static scale only");
+  HERO_REQUIRE(!f8_in || a->out.dtype != HERO_I8, HERO_ERR_UNSUPPORTED, "the e4m3 core emits e4m3, F16 or BF16");
+  HERO_REQUIRE(a->out.dtype != HERO_F8 || f8_in || fp_in, HERO_ERR_UNSUPPORTED, "an e4m3 X_attn needs e4m3 or FP operands");
   HERO_REQUIRE(aligned16(a->q) && aligned16(a->k) && aligned16(a->v) && (a->ld * (fp_in ? 2 : 1)) % 16 == 0 &&
                a->ld >= (int64_t)a->nh * a->dh,
                HERO_ERR_ALIGNMENT, "q/k/v must be 16-byte aligned with a row pitch that is a multiple of 16 bytes and ld >= nh*dh");
@@ -471,8 +527,9 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   if ((st = check_matrix(a->out, "out")) != HERO_OK) return st;
   HERO_REQUIRE(a->out.rows == (int64_t)a->B * a->S && a->out.cols == (int64_t)a->nh * a->dh, HERO_ERR_INVALID_ARG,
                "out must be [B*S, nh*dh]");
-  HERO_REQUIRE(a->out.dtype == HERO_I8 || is_fp16ish(a->out.dtype), HERO_ERR_UNSUPPORTED, "out dtype %d", a->out.dtype);
-  if (a->out.dtype == HERO_I8)
+  HERO_REQUIRE(is_q8(a->out.dtype) || is_fp16ish(a->out.dtype), HERO_ERR_UNSUPPORTED, "out dtype %d", a->out.dtype);
+  HERO_REQUIRE(!(fp_in && a->out.dtype == HERO_F8), HERO_ERR_UNSUPPORTED, "the FP16 / BF16 core emits INT8, F16 or BF16");
+  if (is_q8(a->out.dtype))
     HERO_REQUIRE((a->out.gran == HERO_GRAN_FWQ || a->out.gran == HERO_GRAN_SQ) && a->out.scale, HERO_ERR_UNSUPPORTED,
                  "INT8 X_attn is feature-wise (FWQ) or static (SQ) with a calibrated scale (Sec. 2.2.2)");
   HERO_REQUIRE(fp_in || (a->s_q > 0 && a->s_k > 0 && a->s_v > 0 && (a->s_p > 0 || a->p_mode == HERO_P_ROWMAX)), HERO_ERR_INVALID_ARG, "scales must be positive");
@@ -489,7 +546,7 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   const bool rowmax = !fp_in && a->p_mode == HERO_P_ROWMAX;
   p.inv_sp = rowmax ? 255.0f : 1.0f / a->s_p;
   p.pv_scale = rowmax ? a->s_v / 255.0f : a->s_p * a->s_v;
-  p.out_scale = a->out.dtype == HERO_I8 ? a->out.scale : nullptr;
+  p.out_scale = is_q8(a->out.dtype) ? a->out.scale : nullptr;
   p.out_scale_stride = a->out.gran == HERO_GRAN_FWQ ? 1 : 0;
   p.mask = a->mask; p.key_len = a->key_len;
   p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
@@ -499,6 +556,7 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
+  if (f8_in) return a->dh == 64 ? launch_attn<64, false, true>(h, a, p, s) : launch_attn<128, false, true>(h, a, p, s);
   if (a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory
   if (rowmax) return a->dh == 64 ? launch_attn<64, true>(h, a, p, s) : launch_attn<128, true>(h, a, p, s);
   if (a->dh == 64) return launch_attn<64, false>(h, a, p, s);

@@ -122,3 +122,40 @@ def test_e4m3_rejections(h):
         h.hero_w8a8_linear(hero.tensor(x, "sq", s[:1]), w, hero.tensor(o, "sq", s[:1]), w_scale=s)
     with pytest.raises(hero.HeroError):          # a token-wise output needs a row reduction: not in a GEMM epilogue
         h.hero_w8a8_linear(hero.tensor(x, "sq", s[:1]), w, hero.tensor(x.clone(), "twq", torch.ones(128, device="cuda")), w_scale=s)
+
+
+ATTN_CASES = [(1, 128, 2, 64, "none", 1.0), (2, 384, 4, 64, "none", 1.0), (1, 333, 2, 128, "causal", 1.0),
+              (1, 1024, 1, 128, "causal", 1.0), (2, 200, 2, 64, "none", 0.25)]
+
+
+@pytest.mark.parametrize("B,S,nh,dh,mask,clipf", ATTN_CASES)
+def test_attention_e4m3(h, B, S, nh, dh, mask, clipf):
+    """e4m3 Q, K, V and an e4m3 P against the oracle's FP8 attention; clipf < 1 makes s_p too small so that P saturates."""
+    g = W.rng(13, S + dh)
+    H = nh * dh
+    qkv = Q.e4m3_round(g.standard_normal((B * S, 3 * H)) * 100)
+    s = float(np.sqrt(1.5) / 100)
+    s_q, s_k, s_v, s_p = s, s, 0.02, clipf / 448
+    q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
+    raw = O.attention_f8(q, k, v, B, S, nh, dh, s_q, s_k, s_v, s_p, O.OutSpec("fp", dtype="f64"), mask=mask).data
+    t = to_f8(qkv)
+    out = torch.full((B * S, H), float("nan"), dtype=torch.float16, device="cuda")
+    h.hero_int8_attention(t[:, :H], t[:, H:2 * H], t[:, 2 * H:], B, S, nh, dh, hero.tensor(out), s_q=s_q, s_k=s_k, s_v=s_v, s_p=s_p,
+                          mask=mask)
+    h.check()
+    assert rel_err(out.float().cpu().numpy(), raw) < 3e-3
+    S_attn = Q.f8_scale(np.abs(raw).max(0))
+    want = O.attention_f8(q, k, v, B, S, nh, dh, s_q, s_k, s_v, s_p, O.OutSpec("fwq", scale=S_attn, payload="f8"), mask=mask)
+    o8 = torch.empty(B * S, H, dtype=torch.float8_e4m3fn, device="cuda")
+    h.hero_int8_attention(t[:, :H], t[:, H:2 * H], t[:, 2 * H:], B, S, nh, dh, hero.tensor(o8, "fwq", f32(S_attn)), s_q=s_q, s_k=s_k,
+                          s_v=s_v, s_p=s_p, mask=mask)
+    h.check()
+    # an e4m3 P code that flips on an fp32-vs-fp64 tie moves that probability by a whole mantissa step (6-12 % of its
+    # value, against 1/255 of full scale for the unsigned 8-bit P of the INT8 core), so an output can move by a step or,
+    # where one key dominates the row, two: almost all outputs identical, none further than two steps
+    # (the shift is absolute, a fraction of one key's contribution, so next to an output near zero it spans several
+    # of that value's fine steps: steps are counted at no less than 1/16 of the full range)
+    got, d = f8_vals(o8), np.abs(f8_vals(o8) - want.data)
+    step = np.maximum(np.abs(want.data), 448.0 / 16) * 2.0 ** -3 * 1.0001
+    stats = (float(np.mean(d > 0)), float(np.mean(d > step)), float((d / step).max()))
+    assert np.mean(d > 0) <= 5e-3 and np.mean(d > step) <= 2e-4 and np.all(d <= 2 * step), stats
