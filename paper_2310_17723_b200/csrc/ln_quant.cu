@@ -903,7 +903,6 @@ __host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes)
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR>
 __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
   ptx::pdl_launch_dependents();
-  ptx::pdl_wait();                                 // the previous kernel's outputs are complete and visible
   constexpr int H = 1024 * WPR;
   constexpr int SLOTS = 8 / WPR;                   // rows per CTA pass
   constexpr int STRIDE = WPR * 32;                 // chunk stride between a lane's two chunks
@@ -959,18 +958,8 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     cp_async_commit();
   };
 
-  const long long row_step = (long long)gridDim.x * SLOTS;
-  const long long first = (long long)blockIdx.x * SLOTS + slot;
-  for (int s0 = 0; s0 < STAGES - 1; ++s0) prefetch(first + s0 * row_step, s0);
-  // the per-row scale of a TWQ residual travels STAGES - 1 rows ahead as well, in a register ring: lane i of a warp
-  // holds the scale of the i-th row ahead (STAGES <= 8 < 32)
-  constexpr bool ROW_SC = RES == SRC_I8 && RSC == RS_ROW;
-  float rs_ring = 1.f;
-  if constexpr (ROW_SC) {
-    const long long r = first + (long long)lane * row_step;
-    if (lane < STAGES - 1 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
-  }
-
+  // Everything that does not depend on the previous kernel comes first (calibrated scale vectors, gamma, beta): with a
+  // programmatic dependent launch it overlaps that kernel's tail.
   // per-feature vectors: shared memory for the scales, registers for gamma / beta
   // stored piece-major ([float4 piece q of a chunk][chunk]): consecutive lanes then read consecutive 16-byte words,
   // free of bank conflicts
@@ -1000,6 +989,19 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
       for (int i = 0; i < 4; ++i) bet[k][4 + i] = t[i];
     }
   }
+  ptx::pdl_wait();                                 // the previous kernel's outputs are complete and visible from here on
+  const long long row_step = (long long)gridDim.x * SLOTS;
+  const long long first = (long long)blockIdx.x * SLOTS + slot;
+  for (int s0 = 0; s0 < STAGES - 1; ++s0) prefetch(first + s0 * row_step, s0);
+  // the per-row scale of a TWQ residual travels STAGES - 1 rows ahead as well, in a register ring: lane i of a warp
+  // holds the scale of the i-th row ahead (STAGES <= 8 < 32)
+  constexpr bool ROW_SC = RES == SRC_I8 && RSC == RS_ROW;
+  float rs_ring = 1.f;
+  if constexpr (ROW_SC) {
+    const long long r = first + (long long)lane * row_step;
+    if (lane < STAGES - 1 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+  }
+
   __syncthreads();
 
   int st = 0;
