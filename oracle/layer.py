@@ -14,7 +14,8 @@ import numpy as np
 
 from . import quant as Q
 from .ops import (QT, OutSpec, fp_tensor, layernorm, ACTIVATIONS, softmax_masked, attention_mask,
-                  ln_quant, gemm_quant, gemm_fp, attention_int8, attention_fp)
+                  ln_quant, gemm_quant, gemm_quant_f8, gemm_fp, attention_int8, attention_f8, attention_fp,
+                  quant_weight_columnwise_f8)
 
 MODULES = ("qkv", "attn", "attn_out", "fc1", "fc2")
 
@@ -45,6 +46,7 @@ class LayerSpec:
     gran_attn: str = "fwq"           # granularity of X_attn                        (fwq | sq)
     gran_out: str = "twq"            # post-LN layer output: twq | fwq | sq | fp
     p_mode: str = "static"           # P quantizer of the INT8 attention core: 'static' (Eq. 16) | 'rowmax'
+    payload: str = "i8"              # 8-bit type of the modules in 'int8' mode: 'i8' (the paper) | 'f8' (e4m3 variant)
 
     @property
     def dh(self):
@@ -117,17 +119,19 @@ def calibrate(spec: LayerSpec, params, x_cal, B_cal):
     t = layer_fp64(spec, params, x_cal, B=B_cal)
     am_f = lambda a: np.max(np.abs(a), axis=0)
     am_t = lambda a: np.max(np.abs(a))
+    f8 = spec.payload == "f8"
+    cs = (lambda a: Q.calib_scale(a, Q.F8MAX)) if f8 else Q.calib_scale       # absmax / 448 for an e4m3 payload
     return {
-        "S_in_f": Q.calib_scale(am_f(t["x_in"])), "S_in_t": float(Q.calib_scale(am_t(t["x_in"]))),
-        "S_q": float(Q.calib_scale(am_t(t["q"]))), "S_k": float(Q.calib_scale(am_t(t["k"]))),
-        "S_v": float(Q.calib_scale(am_t(t["v"]))),
-        "S_p": float(Q.calib_scale(t["p_max"], Q.PMAX)),
-        "S_attn_f": Q.calib_scale(am_f(t["x_attn"])), "S_attn_t": float(Q.calib_scale(am_t(t["x_attn"]))),
-        "S_o": Q.calib_scale(am_f(t["x_o"])),
-        "S_mid_f": Q.calib_scale(am_f(t["x_mid"])), "S_mid_t": float(Q.calib_scale(am_t(t["x_mid"]))),
-        "S_a": Q.calib_scale(am_f(t["a"])),
-        "S_x2": Q.calib_scale(am_f(t["x_2"])),
-        "S_out_f": Q.calib_scale(am_f(t["x_out"])), "S_out_t": float(Q.calib_scale(am_t(t["x_out"]))),
+        "S_in_f": cs(am_f(t["x_in"])), "S_in_t": float(cs(am_t(t["x_in"]))),
+        "S_q": float(cs(am_t(t["q"]))), "S_k": float(cs(am_t(t["k"]))),
+        "S_v": float(cs(am_t(t["v"]))),
+        "S_p": float(Q.calib_scale(t["p_max"], Q.F8MAX if f8 else Q.PMAX)),
+        "S_attn_f": cs(am_f(t["x_attn"])), "S_attn_t": float(cs(am_t(t["x_attn"]))),
+        "S_o": cs(am_f(t["x_o"])),
+        "S_mid_f": cs(am_f(t["x_mid"])), "S_mid_t": float(cs(am_t(t["x_mid"]))),
+        "S_a": cs(am_f(t["a"])),
+        "S_x2": cs(am_f(t["x_2"])),
+        "S_out_f": cs(am_f(t["x_out"])), "S_out_t": float(cs(am_t(t["x_out"]))),
     }
 
 
@@ -143,7 +147,7 @@ def _vec(gran, S_f, S_t, n):
     return None
 
 
-def fold_and_quantize(W, b, in_scale=None, out_scale=None):
+def fold_and_quantize(W, b, in_scale=None, out_scale=None, payload="i8"):
     """W~ = Diag(in_scale) W Diag(1/out_scale), b~ = b / out_scale, then Eq. 2 column-wise INT8.
 
     in_scale : FWQ/SQ scale vector of the GEMM's INT8 input (consumer-side fold, Eq. 23, 32)
@@ -159,7 +163,10 @@ def fold_and_quantize(W, b, in_scale=None, out_scale=None):
         W = W / np.asarray(out_scale, np.float64)[None, :]
         if b is not None:
             b = b / np.asarray(out_scale, np.float64)[None, :].reshape(-1)
-    W_i8, S_w = Q.quant_weight_columnwise(W)
+    if payload == "f8":
+        W_i8, S_w = quant_weight_columnwise_f8(W)           # e4m3 values, scales absmax / 448
+    else:
+        W_i8, S_w = Q.quant_weight_columnwise(W)
     if b is not None:
         b = b.astype(np.float32).astype(np.float64)     # biases are stored in fp32
     return W_i8, S_w, b
@@ -175,6 +182,15 @@ def prepare_layer(spec: LayerSpec, params, C):
     for k in MODULES:
         assert m[k] in ("int8", "fp")
     L = {"spec": spec, "C": C}
+    pay = spec.payload
+    assert pay in ("i8", "f8")
+    assert pay == "i8" or spec.p_mode == "static", "the e4m3 attention core has the static P quantizer only"
+
+    def out_spec(kind, **kw):                                   # every 8-bit output stage of the layer carries the payload
+        return OutSpec(kind, payload=pay, **kw)
+
+    def fold_and_quantize_(W, b, i, o):
+        return fold_and_quantize(W, b, i, o, payload=pay)
     fpW = lambda W: Q.round_to_storage(W, fd)
     f32 = lambda b: np.asarray(b, np.float64).astype(np.float32).astype(np.float64)
 
@@ -187,12 +203,12 @@ def prepare_layer(spec: LayerSpec, params, C):
     # what the LN feeding QKV / FC1 must emit
     def ln_spec(mode, gran, S_f, S_t):
         if mode == "fp":
-            return OutSpec("fp", dtype=fd)
-        return {"twq": OutSpec("twq"), "fwq": OutSpec("fwq", scale=S_f), "sq": OutSpec("sq", scale=S_t)}[gran]
+            return out_spec("fp", dtype=fd)
+        return {"twq": out_spec("twq"), "fwq": out_spec("fwq", scale=S_f), "sq": out_spec("sq", scale=S_t)}[gran]
 
     L["ln_in_out"] = ln_spec(m["qkv"], spec.gran_in, C["S_in_f"], C["S_in_t"])
     L["ln_mid_out"] = ln_spec(m["fc1"], spec.gran_mid, C["S_mid_f"], C["S_mid_t"])
-    L["ln_final_out"] = (OutSpec("fp", dtype=fd) if spec.gran_out == "fp" else
+    L["ln_final_out"] = (out_spec("fp", dtype=fd) if spec.gran_out == "fp" else
                          ln_spec("int8", spec.gran_out, C["S_out_f"], C["S_out_t"]))
 
     # QKV (Eq. 14, 20-22)
@@ -201,37 +217,37 @@ def prepare_layer(spec: LayerSpec, params, C):
     g = {"mode": m["qkv"]}
     if m["qkv"] == "int8":
         out_fold = qkv_vec if m["attn"] == "int8" else None
-        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize(Wqkv, bqkv, in_vec, out_fold)
-        g["out"] = OutSpec("round") if m["attn"] == "int8" else OutSpec("fp", dtype=fd)
+        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize_(Wqkv, bqkv, in_vec, out_fold)
+        g["out"] = out_spec("round") if m["attn"] == "int8" else out_spec("fp", dtype=fd)
         g["carried"] = out_fold
     else:
         g["W"], g["bias"] = fpW(Wqkv), f32(bqkv)
-        g["out"] = OutSpec("fwq", scale=qkv_vec) if m["attn"] == "int8" else OutSpec("fp", dtype=fd)
+        g["out"] = out_spec("fwq", scale=qkv_vec) if m["attn"] == "int8" else out_spec("fp", dtype=fd)
         g["carried"] = None
     L["qkv"] = g
 
     # attention output stage (Eq. 17): INT8 FWQ/SQ when the attention-output linear is INT8
     if m["attn_out"] == "int8":
-        L["attn_out_spec"] = (OutSpec("fwq", scale=C["S_attn_f"]) if spec.gran_attn == "fwq"
-                              else OutSpec("sq", scale=C["S_attn_t"]))
+        L["attn_out_spec"] = (out_spec("fwq", scale=C["S_attn_f"]) if spec.gran_attn == "fwq"
+                              else out_spec("sq", scale=C["S_attn_t"]))
     else:
-        L["attn_out_spec"] = OutSpec("fp", dtype=fd)
+        L["attn_out_spec"] = out_spec("fp", dtype=fd)
 
     # attention-output linear (Eq. 18, 23)
     g = {"mode": m["attn_out"]}
     if m["attn_out"] == "int8":
-        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize(p["Wo"], p["bo"], attn_vec, C["S_o"])
-        g["out"], g["carried"] = OutSpec("round"), np.asarray(C["S_o"], np.float64)
+        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize_(p["Wo"], p["bo"], attn_vec, C["S_o"])
+        g["out"], g["carried"] = out_spec("round"), np.asarray(C["S_o"], np.float64)
     else:
         g["W"], g["bias"] = fpW(p["Wo"]), f32(p["bo"])
-        g["out"], g["carried"] = OutSpec("fp", dtype=fd), None
+        g["out"], g["carried"] = out_spec("fp", dtype=fd), None
     L["o"] = g
 
     # FC1 + GELU^quant (Eq. 28-29): X_1 is never quantized; A is FWQ when FC2 is INT8
     g = {"mode": m["fc1"]}
-    a_spec = OutSpec("fwq", scale=C["S_a"]) if m["fc2"] == "int8" else OutSpec("fp", dtype=fd)
+    a_spec = out_spec("fwq", scale=C["S_a"]) if m["fc2"] == "int8" else out_spec("fp", dtype=fd)
     if m["fc1"] == "int8":
-        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize(p["W1"], p["b1"], mid_vec, None)
+        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize_(p["W1"], p["b1"], mid_vec, None)
     else:
         g["W"], g["bias"] = fpW(p["W1"]), f32(p["b1"])
     g["out"], g["carried"] = a_spec, None
@@ -240,11 +256,11 @@ def prepare_layer(spec: LayerSpec, params, C):
     # FC2 (Eq. 30, 32)
     g = {"mode": m["fc2"]}
     if m["fc2"] == "int8":
-        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize(p["W2"], p["b2"], C["S_a"], C["S_x2"])
-        g["out"], g["carried"] = OutSpec("round"), np.asarray(C["S_x2"], np.float64)
+        g["W_i8"], g["cs"], g["bias"] = fold_and_quantize_(p["W2"], p["b2"], C["S_a"], C["S_x2"])
+        g["out"], g["carried"] = out_spec("round"), np.asarray(C["S_x2"], np.float64)
     else:
         g["W"], g["bias"] = fpW(p["W2"]), f32(p["b2"])
-        g["out"], g["carried"] = OutSpec("fp", dtype=fd), None
+        g["out"], g["carried"] = out_spec("fp", dtype=fd), None
     L["fc2"] = g
 
     for k in ("ln1_g", "ln1_b", "ln2_g", "ln2_b"):
@@ -256,6 +272,9 @@ def prepare_layer(spec: LayerSpec, params, C):
 # forward
 # --------------------------------------------------------------------------------------
 def _linear(g, x: QT, act, return_acc=False):
+    if g["mode"] == "int8" and x.kind == "f8":
+        o = gemm_quant_f8(x, g["W_i8"], g["cs"], g["bias"], act, g["out"], g["carried"])
+        return (o, None) if return_acc else o
     if g["mode"] == "int8":
         return gemm_quant(x, g["W_i8"], g["cs"], g["bias"], act, g["out"], g["carried"], return_acc=return_acc)
     o = gemm_fp(x, g["W"], g["bias"], act, g["out"], g["carried"])
@@ -265,6 +284,11 @@ def _linear(g, x: QT, act, return_acc=False):
 def _attention(L, qkv: QT, B):
     spec, C = L["spec"], L["C"]
     H = spec.H
+    if spec.mode["attn"] == "int8" and spec.payload == "f8":
+        assert qkv.kind == "f8" and spec.p_mode == "static"
+        d = qkv.data
+        return attention_f8(d[:, :H], d[:, H:2 * H], d[:, 2 * H:], B, spec.S, spec.nh, spec.dh,
+                            C["S_q"], C["S_k"], C["S_v"], C["S_p"], L["attn_out_spec"], mask=spec.mask)
     if spec.mode["attn"] == "int8":
         assert qkv.kind == "i8"
         d = qkv.data

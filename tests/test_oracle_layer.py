@@ -183,3 +183,45 @@ def test_a_and_x1_are_never_rounded_to_8_bits():
     assert np.array_equal(T["a"].data, Q.quant_fwq(O.gelu_erf(x1), C["S_a"]))
     s1 = np.abs(x1).max() / 127
     assert not np.array_equal(T["a"].data, Q.quant_fwq(O.gelu_erf(Q.quant_sq(x1, s1) * s1), C["S_a"]))
+
+
+@pytest.mark.parametrize("preset", ["M2", "M3"])
+@pytest.mark.parametrize("arch", ["post_ln", "pre_ln"])
+def test_f8_payload_layer_is_close_to_unquantized_layer_and_every_border_is_e4m3(preset, arch):
+    # the FP8 variant of the layer: every 8-bit border holds e4m3 values (3 mantissa bits: relative step 2^-4 per
+    # element, averaged down by the contractions), scales are absmax / 448.  Pinned against the un-quantized layer.
+    shape = W.tiny_shape(arch=arch, mask="causal" if arch == "pre_ln" else "none", eps=1e-5, n_outlier=2)
+    spec = _spec(shape, mode=dict(L.MODE_PRESETS[preset]), payload="f8")
+    p = W.layer_params(shape, 9)
+    x = W.activations(shape, 9)
+    C = L.calibrate(spec, p, x if arch == "pre_ln" else O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps), shape.B)
+    Ci = L.calibrate(_spec(shape, mode=dict(L.MODE_PRESETS[preset])), p,
+                     x if arch == "pre_ln" else O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps), shape.B)
+    assert np.isclose(C["S_q"] * 448.0, Ci["S_q"] * 127.0, rtol=1e-6)          # same absmax, other full range
+    assert np.isclose(C["S_p"] * 448.0, Ci["S_p"] * 255.0, rtol=1e-6)
+    Lp = L.prepare_layer(spec, p, C)
+    if arch == "post_ln":
+        x_in = L.entry_ln(O.fp_tensor(x, "f16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+        ref_in = O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps)
+    else:
+        x_in, ref_in = O.fp_tensor(x, spec.fp_dtype), x
+    T = L.layer_forward(Lp, x_in)
+    R = L.layer_fp64(spec, p, ref_in)
+    err = np.max(np.abs(T["x_out"].real() - R["x_out"])) / np.max(np.abs(R["x_out"]))
+    assert err < 0.08, err
+    for key in ("x_attn", "x_o", "a", "x_2"):
+        e = np.max(np.abs(T[key].real() - R[key])) / np.max(np.abs(R[key]))
+        assert e < 0.12, (key, e)
+    m = L.MODE_PRESETS[preset]
+    for key, mod in (("x_in", "qkv"), ("qkv", "attn"), ("x_attn", "attn_out"), ("x_o", "attn_out"),
+                     ("x_mid", "fc1"), ("a", "fc2"), ("x_2", "fc2")):
+        want = "f8" if m[mod] == "int8" else "fp"
+        assert T[key].kind == want, key
+        if want == "f8":
+            d = T[key].data
+            assert np.array_equal(Q.e4m3_round(d), d) and np.max(np.abs(d)) <= 448.0, key
+    for mod in ("qkv", "o", "fc1", "fc2"):
+        if Lp[mod]["mode"] == "int8":
+            Wq = Lp[mod]["W_i8"]
+            assert np.array_equal(Q.e4m3_round(Wq), Wq)
+            assert np.allclose(np.max(np.abs(Wq), axis=0), 448.0)                  # every column uses the full range
