@@ -238,6 +238,12 @@ typedef struct {
   const float* ln1_g; const float* ln1_b;
   const float* ln2_g; const float* ln2_b;
   int32_t p_mode;          /* hero_p_mode of the INT8 attention core (0 = the paper's static S_p) */
+  int32_t payload;         /* 8-bit type of the modules in HERO_MODE_INT8: HERO_I8 (0, the paper) or HERO_F8, the FP8
+                              variant: every 8-bit tensor at a module border, the weights (W of those modules holds
+                              e4m3 bytes) and P are e4m3, every scale is absmax / 448, the contractions accumulate in
+                              FP32.  With HERO_F8: p_mode must be static, `in` (post-LN) and an 8-bit `out` are HERO_F8,
+                              and an FP attention core cannot feed an 8-bit attention-output linear
+                              (HERO_ERR_UNSUPPORTED). */
 } hero_layer_desc;
 
 /* ---------------------------------------------------------------------------------------------

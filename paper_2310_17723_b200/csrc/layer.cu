@@ -94,6 +94,8 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
   HERO_REQUIRE(pre || pending == nullptr || pending->data == nullptr, HERO_ERR_INVALID_ARG, "pending is for pre-LN layers only");
 
   const int H = d->H, F = d->F, fp = d->fp_dtype;
+  HERO_REQUIRE(d->payload == HERO_I8 || d->payload == HERO_F8, HERO_ERR_INVALID_ARG, "payload %d: HERO_I8 or HERO_F8 expected", d->payload);
+  const int q8 = d->payload;   // the 8-bit type at every border of the modules in 8-bit mode
   const bool qkv8 = d->mode[HERO_MOD_QKV] == HERO_MODE_INT8, attn8 = d->mode[HERO_MOD_ATTN] == HERO_MODE_INT8;
   const bool o8 = d->mode[HERO_MOD_ATTN_OUT] == HERO_MODE_INT8, fc18 = d->mode[HERO_MOD_FC1] == HERO_MODE_INT8;
   const bool fc28 = d->mode[HERO_MOD_FC2] == HERO_MODE_INT8;
@@ -102,8 +104,8 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
   // the INT8 tensor an LN emits for an INT8 consumer, by granularity (Eq. 3-5)
   auto ln_out = [&](void* data, bool int8, int gran, const float* static_scale, float* twq_scale) -> hero_tensor {
     if (!int8) return mk(data, fp, HERO_GRAN_NONE, M, H, nullptr);
-    if (gran == HERO_GRAN_TWQ) return mk(data, HERO_I8, HERO_GRAN_TWQ, M, H, twq_scale);
-    return mk(data, HERO_I8, gran, M, H, static_scale);
+    if (gran == HERO_GRAN_TWQ) return mk(data, q8, HERO_GRAN_TWQ, M, H, twq_scale);
+    return mk(data, q8, gran, M, H, static_scale);
   };
   HERO_REQUIRE(d->gran_in == HERO_GRAN_TWQ || d->gran_in == HERO_GRAN_FWQ || d->gran_in == HERO_GRAN_SQ, HERO_ERR_INVALID_ARG, "gran_in");
   HERO_REQUIRE(d->gran_mid == HERO_GRAN_TWQ || d->gran_mid == HERO_GRAN_FWQ || d->gran_mid == HERO_GRAN_SQ, HERO_ERR_INVALID_ARG, "gran_mid");
@@ -128,12 +130,16 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
     x_in = a.out;
   } else {
-    HERO_REQUIRE(qkv8 ? in->dtype == HERO_I8 : in->dtype == fp, HERO_ERR_INVALID_ARG,
-                 "post-LN: `in` must be INT8 when the QKV module is INT8, else fp_dtype");
+    HERO_REQUIRE(qkv8 ? in->dtype == q8 : in->dtype == fp, HERO_ERR_INVALID_ARG,
+                 "post-LN: `in` must have the layer's 8-bit payload when the QKV module is 8-bit, else fp_dtype");
   }
 
   // ---- QKV GeMM^quant (Eq. 14, 20-22)
-  const int qkv_dt = attn8 ? HERO_I8 : fp;
+  if (q8 == HERO_F8) {
+    HERO_REQUIRE(!attn8 || d->p_mode == HERO_P_STATIC, HERO_ERR_UNSUPPORTED, "the e4m3 attention core has the static P quantizer only");
+    HERO_REQUIRE(attn8 || !o8, HERO_ERR_UNSUPPORTED, "e4m3 payload: an FP attention core cannot feed an 8-bit attention-output linear");
+  }
+  const int qkv_dt = attn8 ? q8 : fp;
   const size_t qkv_es = dtype_size(qkv_dt);
   hero_tensor qkv = mk(ws + pl.off_qkv, qkv_dt, HERO_GRAN_NONE, M, 3 * H, nullptr);
   {
@@ -145,7 +151,7 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     if ((st = hero_w8a8_linear(h, &a, stream)) != HERO_OK) return st;
   }
   // ---- attention core (Eq. 15-17)
-  hero_tensor x_attn = o8 ? mk(ws + pl.off_attn, HERO_I8, d->gran_attn, M, H, d->s_attn)
+  hero_tensor x_attn = o8 ? mk(ws + pl.off_attn, q8, d->gran_attn, M, H, d->s_attn)
                           : mk(ws + pl.off_attn, fp, HERO_GRAN_NONE, M, H, nullptr);
   {
     hero_attn_args a;
@@ -161,7 +167,7 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     if ((st = hero_int8_attention(h, &a, stream)) != HERO_OK) return st;
   }
   // ---- attention-output GeMM^quant (Eq. 18, 23): the FWQ / SQ scale of X_attn lives in W~_o's rows
-  hero_tensor x_o = o8 ? mk(ws + pl.off_o, HERO_I8, HERO_GRAN_FWQ, M, H, d->s_o) : mk(ws + pl.off_o, fp, HERO_GRAN_NONE, M, H, nullptr);
+  hero_tensor x_o = o8 ? mk(ws + pl.off_o, q8, HERO_GRAN_FWQ, M, H, d->s_o) : mk(ws + pl.off_o, fp, HERO_GRAN_NONE, M, H, nullptr);
   {
     hero_linear_args a;
     memset(&a, 0, sizeof(a));
@@ -185,7 +191,7 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
   }
   // ---- FC1 + GELU^quant (Eq. 28-29): X_1 never leaves the epilogue's registers
-  hero_tensor act = fc28 ? mk(ws + pl.off_a, HERO_I8, HERO_GRAN_NONE, M, F, nullptr) : mk(ws + pl.off_a, fp, HERO_GRAN_NONE, M, F, nullptr);
+  hero_tensor act = fc28 ? mk(ws + pl.off_a, q8, HERO_GRAN_NONE, M, F, nullptr) : mk(ws + pl.off_a, fp, HERO_GRAN_NONE, M, F, nullptr);
   {
     hero_linear_args a;
     memset(&a, 0, sizeof(a));
@@ -195,7 +201,7 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     if ((st = hero_w8a8_linear(h, &a, stream)) != HERO_OK) return st;
   }
   // ---- FC2 GeMM^quant (Eq. 30, 32)
-  hero_tensor x_2 = fc28 ? mk(ws + pl.off_x2, HERO_I8, HERO_GRAN_FWQ, M, H, d->s_x2) : mk(ws + pl.off_x2, fp, HERO_GRAN_NONE, M, H, nullptr);
+  hero_tensor x_2 = fc28 ? mk(ws + pl.off_x2, q8, HERO_GRAN_FWQ, M, H, d->s_x2) : mk(ws + pl.off_x2, fp, HERO_GRAN_NONE, M, H, nullptr);
   {
     hero_linear_args a;
     memset(&a, 0, sizeof(a));
@@ -217,7 +223,7 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
       a.residual = x_mid;
       a.gamma = d->ln2_g; a.beta = d->ln2_b; a.eps = d->eps;
       a.out = *out;
-      if (out->dtype == HERO_I8 && out->gran != HERO_GRAN_TWQ && out->scale == nullptr) a.out.scale = const_cast<float*>(d->s_out);
+      if (is_q8(out->dtype) && out->gran != HERO_GRAN_TWQ && out->scale == nullptr) a.out.scale = const_cast<float*>(d->s_out);
     }
     if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
   }
@@ -237,7 +243,7 @@ extern "C" hero_status hero_layer_forward_host_async(hero_handle* h, const hero_
   const size_t ies = dtype_size(in_dev->dtype), oes = dtype_size(out_dev->dtype);
   HERO_REQUIRE(ies && oes, HERO_ERR_INVALID_ARG, "unknown dtype");
   auto scale_len = [](const hero_tensor& t) -> size_t {
-    if (t.dtype != HERO_I8) return 0;
+    if (!is_q8(t.dtype)) return 0;
     return t.gran == HERO_GRAN_TWQ ? (size_t)t.rows : 0;   // calibrated FWQ / SQ scales already live on the device
   };
   // host -> device: the activation payload and, for a token-wise input, its per-row scales

@@ -73,7 +73,7 @@ class LayerDesc(C.Structure):
                 ("s_q", C.c_float), ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float),
                 ("qkv", LinearParams), ("o", LinearParams), ("fc1", LinearParams), ("fc2", LinearParams),
                 ("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p),
-                ("p_mode", C.c_int32)]
+                ("p_mode", C.c_int32), ("payload", C.c_int32)]
 
 
 class LayerLayout(C.Structure):

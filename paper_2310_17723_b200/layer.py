@@ -31,6 +31,7 @@ class Layer:
         d.gran_in, d.gran_mid = hero.GRAN[cfg.gran_in], hero.GRAN[cfg.gran_mid]
         d.gran_attn, d.gran_out = hero.GRAN[cfg.gran_attn], hero.GRAN[cfg.gran_out]
         d.p_mode = hero.P_MODE[getattr(cfg, "p_mode", "static")]
+        d.payload = hero.F8 if getattr(cfg, "payload", "i8") == "f8" else hero.I8
         for name in ("s_in", "s_mid", "s_attn", "s_o", "s_x2", "s_out", "ln1_g", "ln1_b", "ln2_g", "ln2_b"):
             t = _up(L.get(name))
             self._bufs[name] = t

@@ -5,6 +5,7 @@
     python -m paper_2310_17723_b200.microbench attn --B 8 --S 384 --nh 16 --dh 64     # INT8 attention
     python -m paper_2310_17723_b200.microbench absmax --M 65536 --H 4096             # calibration observer GB/s
     python -m paper_2310_17723_b200.microbench wquant --N 4096 --K 4096              # fold + Eq. 2 weight quantization GB/s
+    python -m paper_2310_17723_b200.microbench layer --workload c3 [--f8 | --fp]   # one whole layer, us per forward
     ... --sweep runs the standalone-kernel sweep of the benchmark configurations instead of one shape.
 
 Inputs are synthetic and larger than L2 (several rotating buffers), times are CUDA events around `--iters` launches.
@@ -128,9 +129,35 @@ def bench_wquant(h, N, K, iters):
           % (N, K, t * 1e6, gbs, gbs / hbm, src), flush=True)
 
 
+def bench_layer(h, workload, payload, fp, iters):
+    """One forward of a single layer of a benchmark configuration (INT8, e4m3 or all-FP modules), L2 flushed between
+    forwards by a 256 MB write (its time is measured alone and subtracted)."""
+    from . import prep
+    from .model import Stack
+    shape = {"c1": W.C1, "c3": W.C3, "c4": W.C4}[workload]
+    mode = dict(prep.PRESETS["FP" if fp else "M3"])
+    kw = dict(gran_in="fwq", gran_attn="sq") if workload == "c3" else {}
+    cfg = prep.LayerConfig(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, eps=shape.eps,
+                           mask=shape.mask, fp_dtype=shape.fp_dtype, mode=mode, payload=payload, **kw)
+    if fp:
+        cfg.gran_out = "fp"
+    st = Stack(h, shape, 3, [cfg], n_cal_seq=1)
+    x = torch.randn(shape.M, shape.H, device="cuda").to(hero.TORCH_FP[shape.fp_dtype])
+    st.set_input(x)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    t_flush = _time(lambda i: flush.fill_(i & 1), 1, iters)
+
+    def step(i):
+        flush.fill_(i & 1)
+        st.forward()
+    t = _time(step, 1, iters) - t_flush
+    print("layer %s %s: %.1f us per forward, %.2f M tokens/s" % (workload, "fp" if fp else payload, t * 1e6, shape.M / t / 1e6), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant"])
+    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant", "layer"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4"])
     ap.add_argument("--M", type=int, default=65536)
     ap.add_argument("--H", type=int, default=1024)
     ap.add_argument("--K", type=int, default=4096)
@@ -167,6 +194,8 @@ def main():
         bench_absmax(h, a.M, a.H, a.iters)
     elif a.kernel == "wquant":
         bench_wquant(h, a.N, a.K, a.iters)
+    elif a.kernel == "layer":
+        bench_layer(h, a.workload, "f8" if a.f8 else "i8", a.fp, a.iters)
     else:
         bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters, a.p_mode)
     h.check()

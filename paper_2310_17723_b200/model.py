@@ -44,7 +44,8 @@ class Stack:
                 t = torch.empty(self.M, self.H, dtype=self.fp_torch, device="cuda")
                 self.bufs.append((t, None, hero.tensor(t)))
             else:
-                t = torch.empty(self.M, self.H, dtype=torch.int8, device="cuda")
+                q8 = torch.float8_e4m3fn if getattr(layer_cfgs[min(li, len(layer_cfgs) - 1)], "payload", "i8") == "f8" else torch.int8
+                t = torch.empty(self.M, self.H, dtype=q8, device="cuda")
                 if kind == "twq":
                     s = torch.empty(self.M, dtype=torch.float32, device="cuda")
                 else:

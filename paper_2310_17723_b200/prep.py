@@ -38,6 +38,7 @@ class LayerConfig:
     gran_attn: str = "fwq"
     gran_out: str = "twq"
     p_mode: str = "static"          # P quantizer of the INT8 attention core: "static" (the paper) | "rowmax"
+    payload: str = "i8"             # 8-bit type of the modules in "int8" mode: "i8" (the paper) | "f8" (e4m3 variant)
 
     @property
     def dh(self):
@@ -66,8 +67,38 @@ def quantize_columns(W):
     return np.ascontiguousarray(q.T), s.astype(np.float32)
 
 
-def fold_quantize(W, b, in_scale=None, out_scale=None):
-    """W~ = Diag(in_scale) W Diag(1 / out_scale), b~ = b / out_scale, then column-wise INT8 (fold first)."""
+F8_MAX = 448.0          # largest finite e4m3 value
+
+
+def e4m3_encode(x):
+    """Saturating round-to-nearest-even of real values to e4m3 (4 exponent bits, bias 7, 3 mantissa bits, subnormals
+    down to 2^-9, no infinities).  Returns (bytes uint8, values float64)."""
+    x = np.clip(np.asarray(x, dtype=np.float64), -F8_MAX, F8_MAX)
+    a = np.abs(x)
+    _, ex = np.frexp(a)                                    # a = m * 2^ex, m in [0.5, 1)
+    e = np.maximum(ex - 1, -6)                             # binade exponent; everything below 2^-6 is subnormal
+    step = np.ldexp(1.0, e - 3)
+    v = np.rint(a / step) * step                           # ties to even; may carry into the next binade
+    _, ex = np.frexp(v)
+    e = np.maximum(ex - 1, -6)
+    normal = v >= 2.0 ** -6
+    field = np.where(normal, e + 7, 0).astype(np.int64)
+    mant = np.where(normal, np.rint((v / np.ldexp(1.0, e) - 1.0) * 8.0), np.rint(v * 512.0)).astype(np.int64)
+    byte = (np.signbit(x).astype(np.int64) << 7) | (field << 3) | mant
+    return byte.astype(np.uint8), np.copysign(v, x)
+
+
+def quantize_columns_f8(W):
+    """Eq. 2 with an e4m3 payload on W[d, m]: per-output-column scale absmax / 448.  Returns (bytes [m][d], S_w[m])."""
+    W = np.asarray(W, dtype=np.float64)
+    s = scale_from_absmax(np.abs(W).max(axis=0), F8_MAX).astype(np.float64)
+    q, _ = e4m3_encode(W / s[None, :])
+    return np.ascontiguousarray(q.T), s.astype(np.float32)
+
+
+def fold_quantize(W, b, in_scale=None, out_scale=None, payload="i8"):
+    """W~ = Diag(in_scale) W Diag(1 / out_scale), b~ = b / out_scale, then column-wise INT8 (fold first);
+    payload "f8" quantizes the folded matrix to e4m3 instead."""
     W = np.asarray(W, dtype=np.float64)
     if in_scale is not None:
         W = W * np.asarray(in_scale, np.float64)[:, None]
@@ -77,7 +108,7 @@ def fold_quantize(W, b, in_scale=None, out_scale=None):
         W = W / o[None, :]
         if b is not None:
             b = b / o
-    Wq, s = quantize_columns(W)
+    Wq, s = quantize_columns_f8(W) if payload == "f8" else quantize_columns(W)
     return Wq, s, (None if b is None else _f32(b))
 
 
@@ -142,11 +173,12 @@ def calibrate(cfg: LayerConfig, params, x_cal, n_seq, return_output=False):
         h1 = x + attn(_ln(x, p["ln1_g"], p["ln1_b"], cfg.eps))
         out = h1 + mlp(_ln(h1, p["ln2_g"], p["ln2_b"], cfg.eps))
     stat["out_f"], stat["out_t"] = np.abs(out).max(0), np.abs(out).max()
-    sc = scale_from_absmax
+    qmax, pmax = (F8_MAX, F8_MAX) if cfg.payload == "f8" else (127.0, 255.0)
+    sc = lambda a, q=qmax: scale_from_absmax(a, q)
     scales = {
         "S_in_f": sc(stat["in_f"]), "S_in_t": float(sc(stat["in_t"])),
         "S_q": float(sc(stat["q"])), "S_k": float(sc(stat["k"])), "S_v": float(sc(stat["v"])),
-        "S_p": float(sc(stat["p"], 255.0)),
+        "S_p": float(sc(stat["p"], pmax)),
         "S_attn_f": sc(stat["attn_f"]), "S_attn_t": float(sc(stat["attn_t"])),
         "S_o": sc(stat["o"]),
         "S_mid_f": sc(stat["mid_f"]), "S_mid_t": float(sc(stat["mid_t"])),
@@ -178,7 +210,18 @@ def prepare_layer(cfg: LayerConfig, params, C, fold_quantize_fn=None):
     """Host arrays for one layer: per linear module {W, w_scale, bias, post_scale}, LN parameters, and the
     activation scales the kernels read.  `C` comes from `calibrate`.  `fold_quantize_fn(W, b, in_scale, out_scale)`
     replaces the host-side fold + Eq. 2 quantization (the device version lives in calibrate.py)."""
-    fq = fold_quantize_fn or fold_quantize
+    if cfg.payload not in ("i8", "f8"):
+        raise ValueError("payload %r" % (cfg.payload,))
+    if cfg.payload == "f8":
+        if fold_quantize_fn is not None:
+            raise NotImplementedError("the device-side fold + quantization emits INT8 weights only")
+        if cfg.p_mode != "static":
+            raise ValueError("the e4m3 attention core has the static P quantizer only")
+        if cfg.mode["attn"] != "int8" and cfg.mode["attn_out"] == "int8":
+            raise ValueError("e4m3 payload: an FP attention core cannot feed an 8-bit attention-output linear")
+        fq = lambda W, b, i, o: fold_quantize(W, b, i, o, payload="f8")
+    else:
+        fq = fold_quantize_fn or fold_quantize
     p = {k: np.asarray(v, np.float64) for k, v in params.items()}
     H, m = cfg.H, cfg.mode
     in_vec = _gran_vec(cfg.gran_in, C["S_in_f"], C["S_in_t"], H)

@@ -24,7 +24,7 @@ def qt_to_device(qt):
     if qt.kind == "fp":
         t = dev(qt.data, TORCH_FP[qt.dtype])
         return t, hero.tensor(t), None
-    t = dev(qt.data)
+    t = dev(qt.data) if qt.kind == "i8" else dev(np.asarray(qt.data, np.float32), torch.float8_e4m3fn)
     if qt.row_scale is not None:
         s = f32(qt.row_scale)
         return t, hero.tensor(t, "twq", s), s
@@ -71,7 +71,8 @@ def oracle_layer_to_prepared(Lp):
     cfg = prep.LayerConfig(B=spec.B, S=spec.S, H=spec.H, nh=spec.nh, F=spec.F, arch=spec.arch, act=spec.act,
                            eps=spec.eps, mask=spec.mask, fp_dtype=spec.fp_dtype, mode=dict(spec.mode),
                            gran_in=spec.gran_in, gran_mid=spec.gran_mid, gran_attn=spec.gran_attn,
-                           gran_out=spec.gran_out, p_mode=getattr(spec, "p_mode", "static"))
+                           gran_out=spec.gran_out, p_mode=getattr(spec, "p_mode", "static"),
+                           payload=getattr(spec, "payload", "i8"))
     f = lambda a: None if a is None else np.ascontiguousarray(np.asarray(a, np.float64).astype(np.float32))
     L = {"cfg": cfg, "C": C}
     for name in ("qkv", "o", "fc1", "fc2"):
@@ -80,7 +81,10 @@ def oracle_layer_to_prepared(Lp):
         if g["out"].kind == "fwq":
             post = 1.0 / np.asarray(g["out"].scale, np.float64)
         if g["mode"] == "int8":
-            L[name] = {"int8": True, "W": np.ascontiguousarray(g["W_i8"].T), "w_scale": f(g["cs"]), "bias": f(g["bias"]),
+            Wq = np.ascontiguousarray(g["W_i8"].T)
+            if cfg.payload == "f8":               # e4m3 values -> their bytes (the values are on the grid: exact)
+                Wq = torch.from_numpy(Wq.astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+            L[name] = {"int8": True, "W": Wq, "w_scale": f(g["cs"]), "bias": f(g["bias"]),
                        "post_scale": f(post)}
         else:
             L[name] = {"int8": False, "W": prep._store_fp(g["W"], spec.fp_dtype), "w_scale": None, "bias": f(g["bias"]),

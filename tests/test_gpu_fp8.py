@@ -159,3 +159,166 @@ def test_attention_e4m3(h, B, S, nh, dh, mask, clipf):
     step = np.maximum(np.abs(want.data), 448.0 / 16) * 2.0 ** -3 * 1.0001
     stats = (float(np.mean(d > 0)), float(np.mean(d > step)), float((d / step).max()))
     assert np.mean(d > 0) <= 5e-3 and np.mean(d > step) <= 2e-4 and np.all(d <= 2 * step), stats
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# the whole layer with an e4m3 payload (hero_layer_desc.payload = HERO_F8)
+# ------------------------------------------------------------------------------------------------------------------
+from oracle import layer as OL
+from paper_2310_17723_b200.layer import Layer
+from gpu_util import qt_to_device, oracle_layer_to_prepared, TORCH_FP
+
+
+def _f8_layer(shape, seed, **kw):
+    spec = OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, mask=shape.mask,
+                        fp_dtype=shape.fp_dtype, eps=shape.eps, payload="f8", **kw)
+    p = W.layer_params(shape, seed)
+    x = W.activations(shape, seed)
+    cal = O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else x
+    Lp = OL.prepare_layer(spec, p, OL.calibrate(spec, p, cal, shape.B))
+    if spec.arch == "post_ln":
+        x_in = OL.entry_ln(O.fp_tensor(x, spec.fp_dtype), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+    else:
+        x_in = O.fp_tensor(x, spec.fp_dtype)
+    return spec, Lp, x_in
+
+
+class _F8Borders:
+    """Views of the operator-border tensors the layer left in its workspace (e4m3 values, fp32 scales, FP tensors)."""
+
+    def __init__(self, h, layer, M):
+        self.lay, self.ws, self.M = h.hero_layer_workspace_layout(layer.desc, M), layer.workspace, M
+
+    def f8(self, name, cols):
+        off = getattr(self.lay, name)
+        return f8_vals(self.ws[off:off + self.M * cols].view(torch.float8_e4m3fn).view(self.M, cols))
+
+    def f32(self, name):
+        off = getattr(self.lay, name)
+        return self.ws[off:off + self.M * 4].view(torch.float32).cpu().numpy().astype(np.float64)
+
+    def fp(self, name, cols, dt):
+        off = getattr(self.lay, name)
+        return self.ws[off:off + self.M * cols * 2].view(TORCH_FP[dt]).view(self.M, cols).float().cpu().numpy().astype(np.float64)
+
+
+def _like8(template, values, row_scale=None):
+    return O.QT("f8", values, row_scale=row_scale if template.row_scale is not None else None, col_scale=template.col_scale)
+
+
+def _attn_close(got, want, what):
+    # the e4m3 P moves an output by up to two steps where one key dominates (see test_attention_e4m3)
+    d = np.abs(got - want)
+    step = np.maximum(np.abs(want), 448.0 / 16) * 2.0 ** -3 * 1.0001
+    stats = (float(np.mean(d > 0)), float(np.mean(d > step)), float((d / step).max()))
+    assert np.mean(d > 0) <= 5e-3 and np.mean(d > step) <= 2e-4 and np.all(d <= 2 * step), (what, stats)
+
+
+@pytest.mark.parametrize("gran_in,gran_attn", [("twq", "fwq"), ("fwq", "sq")])
+def test_post_ln_layer_e4m3_stage_by_stage(h, gran_in, gran_attn):
+    shape = W.tiny_shape(B=2, S=200, H=256, nh=4, F=512, eps=1e-5, n_outlier=2)      # ragged attention tiles
+    spec, Lp, x_in = _f8_layer(shape, 31, gran_in=gran_in, gran_mid=gran_in, gran_attn=gran_attn)
+    M, H, F = spec.M, spec.H, spec.F
+    T = OL.layer_forward(Lp, x_in)
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    _, in_desc, _ = qt_to_device(x_in)
+    out = torch.empty(M, H, dtype=torch.float8_e4m3fn, device="cuda")
+    sc = torch.zeros(M, dtype=torch.float32, device="cuda")
+    n0 = h.launches
+    layer.forward(in_desc, hero.tensor(out, "twq", sc))
+    h.check()
+    assert h.launches - n0 == 7
+    bd = _F8Borders(h, layer, M)
+    # ---- each oracle operator is fed what the device produced one stage earlier
+    qkv = _like8(T["qkv"], bd.f8("qkv", 3 * H))
+    assert_f8_close(qkv.data, T["qkv"].data, 1e-4, "qkv")
+    x_attn = _like8(T["x_attn"], bd.f8("x_attn", H))
+    _attn_close(x_attn.data, OL._attention(Lp, qkv, spec.B).data, "x_attn")
+    x_o = _like8(T["x_o"], bd.f8("x_o", H))
+    assert_f8_close(x_o.data, OL._linear(Lp["o"], x_attn, "none").data, 1e-4, "x_o")
+    x_mid = _like8(T["x_mid"], bd.f8("x_mid", H), bd.f32("x_mid_scale"))
+    want, _ = O.ln_quant([x_in, x_o], Lp["ln1_g"], Lp["ln1_b"], spec.eps, Lp["ln_mid_out"])
+    assert_f8_close(x_mid.data, want.data, 1e-4, "x_mid")
+    if gran_in == "twq":
+        np.testing.assert_allclose(x_mid.row_scale, want.row_scale, rtol=2e-6)
+    a = _like8(T["a"], bd.f8("a", F))
+    assert_f8_close(a.data, OL._linear(Lp["fc1"], x_mid, spec.act).data, 2e-4, "a")
+    x_2 = _like8(T["x_2"], bd.f8("x_2", H))
+    assert_f8_close(x_2.data, OL._linear(Lp["fc2"], a, "none").data, 1e-4, "x_2")
+    want, _ = O.ln_quant([x_mid, x_2], Lp["ln2_g"], Lp["ln2_b"], spec.eps, Lp["ln_final_out"])
+    assert_f8_close(f8_vals(out), want.data, 1e-4, "x_out")
+    np.testing.assert_allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    # ---- free-running against the oracle's own chain: an e4m3 value that flips moves by 6-12 % of itself
+    got = f8_vals(out) * sc.cpu().numpy().astype(np.float64)[:, None]
+    assert rel_err(got, T["x_out"].real()) < 6e-2
+    assert float(np.abs(got - T["x_out"].real()).mean() / np.abs(T["x_out"].real()).mean()) < 5e-3
+
+
+@pytest.mark.parametrize("preset", ["M2", "M3"])
+def test_pre_ln_causal_layer_e4m3(h, preset):
+    shape = W.tiny_shape(B=2, S=256, H=256, nh=2, F=512, arch="pre_ln", mask="causal", fp_dtype="bf16", eps=1e-5)
+    spec, Lp, x_in = _f8_layer(shape, 33, mode=dict(OL.MODE_PRESETS[preset]))
+    M, H, F, fd = spec.M, spec.H, spec.F, spec.fp_dtype
+    T = OL.layer_forward(Lp, x_in)
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    xd, in_desc, _ = qt_to_device(x_in)
+    out = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    layer.forward(in_desc, hero.tensor(out))
+    h.check()
+    bd = _F8Borders(h, layer, M)
+    x_in8 = _like8(T["x_in"], bd.f8("x_in", H), bd.f32("x_in_scale"))
+    assert_f8_close(x_in8.data, T["x_in"].data, 1e-4, "x_in")
+    np.testing.assert_allclose(x_in8.row_scale, T["x_in"].row_scale, rtol=2e-6)
+    qkv = _like8(T["qkv"], bd.f8("qkv", 3 * H))
+    assert_f8_close(qkv.data, OL._linear(Lp["qkv"], x_in8, "none").data, 1e-4, "qkv")
+    x_attn = _like8(T["x_attn"], bd.f8("x_attn", H))
+    _attn_close(x_attn.data, OL._attention(Lp, qkv, spec.B).data, "x_attn")
+    x_o = _like8(T["x_o"], bd.f8("x_o", H))
+    assert_f8_close(x_o.data, OL._linear(Lp["o"], x_attn, "none").data, 1e-4, "x_o")
+    h_mid = O.QT("fp", bd.fp("h_mid", H, fd), dtype=fd)
+    want2, _ = O.ln_quant([h_mid], Lp["ln2_g"], Lp["ln2_b"], spec.eps, Lp["ln_mid_out"])
+    x_mid = _like8(T["x_mid"], bd.f8("x_mid", H), bd.f32("x_mid_scale"))
+    assert_f8_close(x_mid.data, want2.data, 1e-4, "x_mid")
+    want_a = OL._linear(Lp["fc1"], x_mid, spec.act)
+    if preset == "M3":
+        a = _like8(T["a"], bd.f8("a", F))
+        assert_f8_close(a.data, want_a.data, 2e-4, "a")
+        x_2 = _like8(T["x_2"], bd.f8("x_2", H))
+        assert_f8_close(x_2.data, OL._linear(Lp["fc2"], a, "none").data, 1e-4, "x_2")
+    else:                                                   # FC2 left in FP: A and X_2 are BF16 tensors
+        a = O.QT("fp", bd.fp("a", F, fd), dtype=fd)
+        assert rel_err(a.data, want_a.real()) < 2.0 ** -7
+        x_2 = O.QT("fp", bd.fp("x_2", H, fd), dtype=fd)
+        assert rel_err(x_2.data, OL._linear(Lp["fc2"], a, "none").real()) < 2.0 ** -7
+    _, want_o = O.ln_quant([h_mid, x_2], None, None, spec.eps, None, fp_out_dtype=fd, normalize=False)
+    got = out.float().cpu().numpy().astype(np.float64)
+    do = np.abs(got - want_o.real())
+    assert np.all(do <= 2.0 ** -7 * np.maximum(np.abs(want_o.real()), 2.0 ** -20)) and np.mean(do > 0) < 1e-3
+    assert rel_err(got, T["h_out"].real()) < 3e-2
+
+
+def test_layer_e4m3_rejections(h):
+    shape = W.tiny_shape(B=1, S=128, H=256, nh=4, F=512, eps=1e-5)
+    spec, Lp, x_in = _f8_layer(shape, 35)
+    L = oracle_layer_to_prepared(Lp)
+    _, in_desc, _ = qt_to_device(x_in)
+    out = torch.empty(spec.M, spec.H, dtype=torch.float8_e4m3fn, device="cuda")
+    sc = torch.zeros(spec.M, dtype=torch.float32, device="cuda")
+    layer = Layer(h, L)
+    layer.desc.p_mode = hero.P_MODE["rowmax"]
+    with pytest.raises(hero.HeroError):
+        layer.forward(in_desc, hero.tensor(out, "twq", sc))
+    layer.desc.p_mode = hero.P_MODE["static"]
+    layer.desc.mode[hero.MODULES.index("attn")] = hero.MODE_FP          # FP core feeding an 8-bit attention-output linear
+    with pytest.raises(hero.HeroError):
+        layer.forward(in_desc, hero.tensor(out, "twq", sc))
+    layer.desc.mode[hero.MODULES.index("attn")] = hero.MODE_INT8
+    i8 = torch.zeros(spec.M, spec.H, dtype=torch.int8, device="cuda")   # an INT8 input to an e4m3 layer
+    with pytest.raises(hero.HeroError):
+        layer.forward(hero.tensor(i8, "twq", sc), hero.tensor(out, "twq", sc))
+    layer.desc.payload = 3
+    with pytest.raises(hero.HeroError):
+        layer.forward(in_desc, hero.tensor(out, "twq", sc))
+    layer.desc.payload = hero.F8
+    layer.forward(in_desc, hero.tensor(out, "twq", sc))
+    h.check()

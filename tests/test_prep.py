@@ -39,3 +39,30 @@ def test_prepared_layer_matches_oracle(arch, preset, gi, ga):
         else:
             assert gp["post_scale"] is None
     assert prep.PRESETS == {k: v for k, v in OL.MODE_PRESETS.items()}
+
+
+def test_e4m3_encode_matches_the_library_cast_and_saturates():
+    # the host-side e4m3 quantizer against torch's float8_e4m3fn cast (round-to-nearest-even) on values that float32
+    # holds exactly, all 256 byte patterns as fixed points, ties, subnormals and saturation
+    import torch
+    from paper_2310_17723_b200 import prep
+    g = np.random.default_rng(5)
+    x = np.concatenate([g.standard_normal(4000) * 100, g.standard_normal(4000) * 0.01, g.uniform(-448, 448, 4000),
+                        [0.0, -0.0, 2.0 ** -9, 2.0 ** -10, 3 * 2.0 ** -10, 2.0 ** -6, 17.0, 18.0, 19.0, 447.9, 464.0]])
+    x = x.astype(np.float32).astype(np.float64)
+    x = x[np.abs(x) <= 464.0]                      # beyond that the library cast yields NaN; the quantizer saturates
+    b, v = prep.e4m3_encode(x)
+    want = torch.from_numpy(x.astype(np.float32)).to(torch.float8_e4m3fn)
+    assert np.array_equal(v, want.float().numpy().astype(np.float64))
+    nz = v != 0
+    assert np.array_equal(b[nz], want.view(torch.uint8).numpy()[nz])
+    # every finite byte pattern decodes to a value that encodes back to itself
+    allb = np.array([i for i in range(256) if (i & 0x7F) != 0x7F], dtype=np.uint8)
+    vals = torch.from_numpy(allb).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    b2, v2 = prep.e4m3_encode(vals)
+    assert np.array_equal(v2, vals) and np.array_equal(b2[vals != 0], allb[vals != 0])
+    b3, v3 = prep.e4m3_encode(np.array([1e9, -1e9, 449.0]))
+    assert np.array_equal(v3, [448.0, -448.0, 448.0]) and list(b3) == [0x7E, 0xFE, 0x7E]
+    Wq, s = prep.quantize_columns_f8(g.standard_normal((64, 8)) * 0.02)
+    dec = torch.from_numpy(Wq).view(torch.float8_e4m3fn).float().numpy()
+    assert Wq.shape == (8, 64) and np.allclose(np.abs(dec).max(axis=1), 448.0)
