@@ -28,11 +28,30 @@ def _peaks():
     return 6650.0, 2.0 * 1590.0, "fallback"
 
 
+GRAPH = False       # --graph: replay the launches from a CUDA graph (kernels of a few microseconds are otherwise timed at
+                    # the rate the host can issue them)
+
+
 def _time(fn, n_buf, iters):
     for i in range(n_buf):
         fn(i)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if GRAPH:
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n_buf):
+                    fn(i)
+            reps = max(1, (iters + n_buf - 1) // n_buf)
+            g.replay()
+            e0.record()
+            for _ in range(reps):
+                g.replay()
+            e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * n_buf) * 1e-3
     e0.record()
     for k in range(iters):
         fn(k % n_buf)
@@ -64,7 +83,7 @@ def bench_ln(h, M, H, kind, iters):
 
 def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
     dt = torch.bfloat16 if fp else (torch.float8_e4m3fn if f8 else torch.int8)
-    n = max(2, min(8, int(300e6 // (M * K + N * K + M * N)) + 1))
+    n = max(2, min(64, int(300e6 // (M * K + N * K + M * N)) + 1))
     if fp:
         As = [torch.randn(M, K, device="cuda", dtype=dt) for _ in range(n)]
         Ws = [torch.randn(N, K, device="cuda", dtype=dt) for _ in range(n)]
@@ -85,8 +104,12 @@ def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
     _, i8peak, src = _peaks()
     peak = i8peak / 2 if fp else i8peak
     tops = 2.0 * M * N * K / t / 1e12
-    print("GeMM^quant %s M=%d K=%d N=%d act=%s: %.1f us, %.0f TOP/s, %.2f of 2 x %s BF16 peak%s"
-          % ("bf16" if fp else ("e4m3" if f8 else "i8"), M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else ""), flush=True)
+    es = 2 if fp else 1
+    gbs = (M * K * es + N * K * es + M * N * es + 4 * M + 8 * N) / t / 1e9
+    hbm = _peaks()[0]
+    print("GeMM^quant %s M=%d K=%d N=%d act=%s: %.1f us, %.0f TOP/s, %.2f of 2 x %s BF16 peak%s; %.0f GB/s, %.2f of copy bandwidth"
+          % ("bf16" if fp else ("e4m3" if f8 else "i8"), M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else "",
+             gbs, gbs / hbm), flush=True)
 
 
 def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static"):
@@ -174,7 +197,10 @@ def main():
     ap.add_argument("--f8", action="store_true", help="e4m3 operands and output (the FP8 variant)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="time CUDA-graph replays of the launches")
     a = ap.parse_args()
+    global GRAPH
+    GRAPH = a.graph
     h = hero.Handle()
     if a.kernel == "ln":
         if a.sweep:

@@ -150,3 +150,77 @@ def test_refusals(h):
     assert e.value.status in (hero.ERR_UNSUPPORTED, hero.ERR_ALIGNMENT)
     empty = torch.zeros(0, 64, dtype=torch.int8, device="cuda")
     h.hero_w8a8_linear(hero.tensor(empty), Wt, hero.tensor(torch.zeros(0, 32, dtype=torch.int8, device="cuda")), w_scale=cs)
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# few rows (M <= 128): the weight-streaming kernel with the K dimension split over a thread-block cluster
+# ------------------------------------------------------------------------------------------------------------------
+# (the library takes this kernel for M <= 16, and for M <= 128 when K is long and N leaves SMs idle: every case below does)
+# every row-tile width (16 / 32 / 64 / 128), 1 to 8 K splits (K = 80 .. 16384 bytes), uneven splits (33, 65, 73 K steps),
+# ragged feature tiles (N = 16, 144, 2064), ragged K (80, 9232)
+FEW_ROWS = [(1, 128, 16), (1, 16384, 4096), (5, 1024, 144), (16, 4096, 4096), (17, 4224, 768), (16, 80, 2064),
+            (33, 8320, 768), (64, 9232, 1024), (100, 16384, 256), (128, 8192, 3072)]
+
+
+@pytest.mark.parametrize("M,K,N", FEW_ROWS)
+def test_few_rows_int32_accumulators_bit_exact(h, M, K, N):
+    g = W.rng(2, 3000 + M + K + N)
+    A = g.integers(-127, 128, (M, K), dtype=np.int8)
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    got = _linear(h, A, Wt, torch.int32).cpu().numpy()
+    assert np.array_equal(got, O.int_matmul(A, Wt.T.copy()))
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 4096, 4096), (8, 1024, 3072), (16, 16384, 4096), (48, 8192, 1024), (128, 16384, 1024)])
+def test_few_rows_requant_epilogue(h, M, K, N):
+    A, Wt, rs, cs, bias = W.gemm_case(M, K, N)
+    x = O.QT("i8", A, row_scale=rs.astype(np.float64))
+    want = O.gemm_quant(x, Wt.T.copy(), cs, bias, "none", O.OutSpec("round"))
+    got = _linear(h, A, Wt, torch.int8, rs=rs, cs=cs, bias=bias).cpu().numpy()
+    assert_int8_close(got, want.data, what="few rows, requant epilogue")
+    want_fp = O.gemm_quant(x, Wt.T.copy(), cs, bias, "none", O.OutSpec("fp", dtype="bf16"))
+    got_fp = _linear(h, A, Wt, torch.bfloat16, rs=rs, cs=cs, bias=bias).float().cpu().numpy()
+    assert rel_err(got_fp, want_fp.data) < 1e-2 and np.mean(got_fp != want_fp.data) < 2e-3
+
+
+@pytest.mark.parametrize("act", ["gelu_erf", "gelu_tanh"])
+@pytest.mark.parametrize("M", [3, 16, 40, 128])
+def test_few_rows_fc1_gelu_quant(h, act, M):
+    K, N = (1024 if M <= 16 else 8192), 4096
+    g = W.rng(2, 556 + M)
+    A = g.integers(-127, 128, (M, K), dtype=np.int8)
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    rs = (g.uniform(0.5, 1.5, M) * 0.02).astype(np.float32)
+    cs = (g.uniform(0.5, 1.5, N) * 1.5e-4 / np.sqrt(K / 768)).astype(np.float32)
+    bias = (g.standard_normal(N) * 0.1).astype(np.float32)
+    x = O.QT("i8", A, row_scale=rs.astype(np.float64))
+    v = O.gemm_quant(x, Wt.T.copy(), cs, bias, act, O.OutSpec("fp", dtype="f64")).data
+    S_a = Q.calib_scale(np.abs(v).max(0))
+    want = O.gemm_quant(x, Wt.T.copy(), cs, bias, act, O.OutSpec("fwq", scale=S_a))
+    got = _linear(h, A, Wt, torch.int8, rs=rs, cs=cs, bias=bias, act=act, post=(1.0 / S_a).astype(np.float32)).cpu().numpy()
+    assert_int8_close(got, want.data, frac=3e-4, what="few rows, GELU^quant")
+
+
+@pytest.mark.parametrize("fp", ["f16", "bf16"])
+@pytest.mark.parametrize("M,K,N", [(2, 2048, 512), (20, 2048, 48), (128, 4096, 1024)])
+def test_few_rows_fp_mode_gemm(h, fp, M, K, N):
+    g = W.rng(2, 778 + M)
+    A = Q.round_to_storage(g.standard_normal((M, K)), fp)
+    Wm = Q.round_to_storage(g.standard_normal((K, N)) * 0.05, fp)
+    bias = (g.standard_normal(N) * 0.1).astype(np.float32)
+    want = O.gemm_fp(O.fp_tensor(A, fp), Wm, bias, "gelu_erf", O.OutSpec("fp", dtype=fp))
+    tA, tW = dev(A, TORCH_FP[fp]), dev(Wm.T.copy(), TORCH_FP[fp])
+    got = _linear(h, tA, tW, TORCH_FP[fp], bias=bias, act="gelu_erf").float().cpu().numpy()
+    assert rel_err(got, want.data) < (1e-2 if fp == "bf16" else 2e-3)
+
+
+def test_few_rows_strided_input_and_output(h):
+    M, K, N = 9, 1024, 384
+    g = W.rng(2, 901)
+    big_a = torch.from_numpy(g.integers(-127, 128, (M, 2 * K), dtype=np.int8)).cuda()
+    big_o = torch.full((M, 2 * N), -77, dtype=torch.int32, device="cuda")
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    h.hero_w8a8_linear(hero.tensor(big_a[:, K:]), dev(Wt), hero.tensor(big_o[:, :N]))
+    h.check()
+    assert np.array_equal(big_o[:, :N].cpu().numpy(), O.int_matmul(big_a[:, K:].cpu().numpy(), Wt.T.copy()))
+    assert bool((big_o[:, N:] == -77).all())
