@@ -312,6 +312,44 @@ def attention_int8(q_i8, k_i8, v_i8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutS
     return (o, internals) if return_internals else o
 
 
+def attention_int8_decode(q_i8, k_cache, v_cache, lens, nh, dh, s_q, s_k, s_v, s_p, out: OutSpec, p_mode="static"):
+    """One decode step of the INT8 attention core (Eq. 15-17 for a single query row per sequence, the generation
+    workload the method names) over an INT8 key / value cache.
+
+    q_i8 [B, nh*dh] int8: the current token's query; k_cache, v_cache [B, S_max, nh*dh] int8 (SQ scales s_k, s_v), of
+    which sequence b holds lens[b] valid entries, the current token's own key / value included (it attends to itself
+    and to everything before it, which is what the causal mask gives its row in a prefill).  Per (b, h):
+        A[k] = d~ (q . K[k]),  d~ = s_q s_k / sqrt(dh),  k < lens[b];   P = softmax(A);
+        P_u8 = clip(Round(P / s_p), 0, 255);   acc = sum_k P_u8[k] V[k]  (exact INT32);   X_attn = s_p s_v acc
+    then the output stage.  p_mode="rowmax": e = exp(A - max A), P~_u8 = Round(255 e), X_attn = s_v acc / (255 sum e).
+    A sequence with lens[b] = 0 yields zeros.
+    """
+    assert p_mode in ("static", "rowmax")
+    q_i8, k_cache, v_cache = np.asarray(q_i8), np.asarray(k_cache), np.asarray(v_cache)
+    assert q_i8.dtype == np.int8 and k_cache.dtype == np.int8 and v_cache.dtype == np.int8
+    B, H = q_i8.shape
+    assert H == nh * dh
+    d_tilde = float(s_q) * float(s_k) / np.sqrt(float(dh))
+    x_attn = np.zeros((B, H), dtype=np.float64)
+    for b in range(B):
+        L = int(lens[b])
+        if L == 0:
+            continue
+        for h in range(nh):
+            cols = slice(h * dh, (h + 1) * dh)
+            A = d_tilde * int_matmul(q_i8[b:b + 1, cols], k_cache[b, :L, cols].T).astype(np.float64)[0]
+            e = np.exp(A - np.max(A))
+            if p_mode == "static":
+                P_u8 = Q.quant_unsigned(e / np.sum(e), s_p)
+                acc = int_matmul(P_u8[None, :], v_cache[b, :L, cols])[0]
+                x_attn[b, cols] = float(s_p) * float(s_v) * acc.astype(np.float64)
+            else:
+                P_u8 = Q.quant_unsigned(e, 1.0 / Q.PMAX)
+                acc = int_matmul(P_u8[None, :], v_cache[b, :L, cols])[0]
+                x_attn[b, cols] = float(s_v) * acc.astype(np.float64) / (Q.PMAX * np.sum(e))
+    return emit(x_attn, out)
+
+
 def attention_f8(q_f8, k_f8, v_f8, B, S, nh, dh, s_q, s_k, s_v, s_p, out: OutSpec, mask="none", key_len=None):
     """The FP8 variant of the attention core: e4m3 Q, K, V (values, SQ scales s_q, s_k, s_v) and an e4m3 P.
 

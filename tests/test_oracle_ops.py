@@ -344,3 +344,48 @@ def test_ln_quant_fp_out_and_bare_add():
     assert np.array_equal(out.data, q)
     none, r2 = O.ln_quant([h, br], None, None, 0.0, None, fp_out_dtype="bf16", normalize=False)
     assert none is None and np.array_equal(r2.data, r.data)
+
+
+@pytest.mark.parametrize("p_mode", ["static", "rowmax"])
+def test_attention_int8_decode_is_the_last_causal_row_and_brute_force(p_mode):
+    # a decode step at position t computes row t of the causal prefill over the first t + 1 tokens (the prefill is
+    # pinned above); plus a pure-Python evaluation of the definition on one head
+    g = np.random.default_rng(40)
+    B, S, nh, dh = 3, 37, 2, 8
+    H = nh * dh
+    q = g.integers(-127, 128, (B * S, H), dtype=np.int8)
+    k = g.integers(-127, 128, (B * S, H), dtype=np.int8)
+    v = g.integers(-127, 128, (B * S, H), dtype=np.int8)
+    s_q, s_k, s_v, s_p = 0.011, 0.013, 0.02, 1.0 / 255
+    out = O.OutSpec("fp", dtype="f64")
+    full = O.attention_int8(q, k, v, B, S, nh, dh, s_q, s_k, s_v, s_p, out, mask="causal", p_mode=p_mode).data
+    kc, vc = k.reshape(B, S, H), v.reshape(B, S, H)
+    lens = np.array([S, 1, 20])
+    qd = np.stack([q[b * S + lens[b] - 1] for b in range(B)])
+    got = O.attention_int8_decode(qd, kc, vc, lens, nh, dh, s_q, s_k, s_v, s_p, out, p_mode=p_mode).data
+    for b in range(B):
+        assert np.allclose(got[b], full[b * S + lens[b] - 1], rtol=1e-12, atol=1e-15), b
+    # entries of the cache beyond lens[b] are never read
+    kc2, vc2 = kc.copy(), vc.copy()
+    kc2[2, 20:], vc2[2, 20:] = 99, -99
+    got2 = O.attention_int8_decode(qd, kc2, vc2, lens, nh, dh, s_q, s_k, s_v, s_p, out, p_mode=p_mode).data
+    assert np.array_equal(got, got2)
+    # brute force, sequence 2 head 1
+    import math
+    b, h, L = 2, 1, 20
+    A = [s_q * s_k / math.sqrt(dh) * sum(int(qd[b, h * dh + d]) * int(kc[b, t, h * dh + d]) for d in range(dh)) for t in range(L)]
+    m = max(A)
+    e = [math.exp(a - m) for a in A]
+    l = sum(e)
+    for d in range(dh):
+        if p_mode == "static":
+            acc = sum(min(255, max(0, round(e[t] / l / s_p))) * int(vc[b, t, h * dh + d]) for t in range(L))
+            want = s_p * s_v * acc
+        else:
+            acc = sum(min(255, round(255 * e[t])) * int(vc[b, t, h * dh + d]) for t in range(L))
+            want = s_v * acc / (255 * l)
+        assert math.isclose(got[b, h * dh + d], want, rel_tol=1e-12, abs_tol=1e-15)
+    # an empty sequence yields zeros; a single key yields that key's value row (P = 1 -> 255 s_p s_v V)
+    z = O.attention_int8_decode(qd, kc, vc, np.array([0, 1, 1]), nh, dh, s_q, s_k, s_v, s_p, out, p_mode=p_mode).data
+    assert np.all(z[0] == 0)
+    assert np.allclose(z[1], s_v * vc[1, 0].astype(float), rtol=1e-12)
