@@ -201,6 +201,46 @@ typedef struct {
 hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * One decode step of the INT8 attention core (Sec. 2.2.2 Eq. 15-17 for the single new token of each sequence of a
+ * generative model; Sec. 1 names GPT-style models as targets) over an INT8 key / value cache.  Per (b, h), with
+ * L = len[b] cache entries, the new token's own key and value included:
+ *     A[k] = d~ (q . K[k]),  d~ = s_q s_k / sqrt(dh),  k < L;   P = softmax(A);   P_u8 = clip(Round(P / s_p), 0, 255)
+ *     acc  = sum_k P_u8[k] V[k]   (exact INT32);   out = acc * s_p * s_v  ->  I8 by out.scale (FWQ [H] / SQ [1]) or F16 / BF16
+ *   (HERO_P_ROWMAX: P~_u8 = Round(255 exp(A - max A)), out = acc * s_v / (255 * sum exp), s_p ignored): the row the
+ *   causal prefill computes for the last of L tokens.
+ *   q            : device I8 [B][nh*dh], row pitch ld_q elements
+ *   k_cache, v_cache : device I8; entry t of sequence b starts at cache + b * batch_stride + t * ld_kv (elements), its
+ *                  nh*dh features contiguous, head h at offset h*dh.  Pointers 16-byte aligned, ld_q / ld_kv /
+ *                  batch_stride multiples of 16.  Read-only here unless k_new / v_new are given.
+ *   k_new, v_new : optional device I8 [B][nh*dh] (row pitch ld_new): the new token's key and value, e.g. the other two
+ *                  thirds of the QKV GeMM^quant output.  When given, entry len[b] - 1 of the caches is taken from them
+ *                  and the call also stores them there (the append is fused); when NULL the caches already hold it.
+ *   len          : device int32 [B]; 0 <= len[b] <= max_len; len[b] = 0 writes zeros for sequence b
+ *   max_len      : host-side upper bound on len[b] (sizes the launch); at most 98304
+ *   out          : [B][nh*dh] I8 (gran FWQ scale[H] or SQ scale[1]) or F16 / BF16; dh is 64 or 128
+ * Errors: HERO_ERR_INVALID_ARG / HERO_ERR_ALIGNMENT / HERO_ERR_UNSUPPORTED with hero_last_error() saying which.
+ */
+typedef struct {
+  const void* q;
+  int64_t ld_q;
+  void* k_cache;
+  void* v_cache;
+  int64_t ld_kv;
+  int64_t batch_stride;
+  const void* k_new;
+  const void* v_new;
+  int64_t ld_new;
+  const int32_t* len;
+  int32_t max_len;
+  int32_t B, nh, dh;
+  float s_q, s_k, s_v, s_p;
+  int32_t p_mode;      /* hero_p_mode */
+  hero_tensor out;
+} hero_decode_attn_args;
+
+hero_status hero_int8_decode_attention(hero_handle* h, const hero_decode_attn_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * One transformer layer (Sec. 2.2.2-2.2.3, modes of Sec. 2.3 Table 1).
  * Post-LN (the paper's equations):  x_mid = LN1(x_in + Attn(x_in)); x_out = LN2(x_mid + MLP(x_mid)).
  * Pre-LN (GPT-shaped): h' = h + Attn(LN1(h [+ pending])); out = h' + MLP(LN2(h')) with the residual

@@ -60,6 +60,14 @@ class AttnArgs(C.Structure):
                 ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p), ("p_mode", C.c_int32)]
 
 
+class DecodeAttnArgs(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("ld_q", C.c_int64), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("ld_kv", C.c_int64), ("batch_stride", C.c_int64), ("k_new", C.c_void_p), ("v_new", C.c_void_p),
+                ("ld_new", C.c_int64), ("len", C.c_void_p), ("max_len", C.c_int32), ("B", C.c_int32), ("nh", C.c_int32),
+                ("dh", C.c_int32), ("s_q", C.c_float), ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float),
+                ("p_mode", C.c_int32), ("out", Tensor)]
+
+
 class LinearParams(C.Structure):
     _fields_ = [("W", C.c_void_p), ("w_scale", C.c_void_p), ("bias", C.c_void_p), ("post_scale", C.c_void_p)]
 
@@ -109,6 +117,7 @@ def lib():
         L.hero_layernorm_quant.argtypes = [C.c_void_p, C.POINTER(LnArgs), C.c_void_p]
         L.hero_w8a8_linear.argtypes = [C.c_void_p, C.POINTER(LinearArgs), C.c_void_p]
         L.hero_int8_attention.argtypes = [C.c_void_p, C.POINTER(AttnArgs), C.c_void_p]
+        L.hero_int8_decode_attention.argtypes = [C.c_void_p, C.POINTER(DecodeAttnArgs), C.c_void_p]
         L.hero_mode_preset.argtypes = [C.c_int32, C.POINTER(C.c_int32 * 5)]
         L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
         L.hero_absmax_observe.argtypes = [C.c_void_p, C.POINTER(Tensor), C.c_void_p, C.c_void_p, C.c_void_p]
@@ -211,6 +220,23 @@ class Handle:
                      s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out, _ptr(p_absmax),
                      P_MODE[p_mode] if isinstance(p_mode, str) else p_mode)
         _check(lib().hero_int8_attention(self._h, C.byref(a), _stream(stream)))
+
+    def hero_int8_decode_attention(self, q, k_cache, v_cache, lens, max_len, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0,
+                                   s_p=1.0 / 255, k_new=None, v_new=None, p_mode="static", stream=None):
+        """q: int8 [B, nh*dh] view; k_cache, v_cache: int8 [B, S_max, nh*dh] views (feature stride 1, equal strides);
+        lens: int32 [B] device tensor; k_new / v_new: optional int8 [B, nh*dh] views of equal pitch (appended at
+        lens[b] - 1); out: hero.Tensor [B, nh*dh]."""
+        assert q.dim() == 2 and k_cache.dim() == 3 and k_cache.stride() == v_cache.stride() and k_cache.stride(2) == 1
+        assert q.dtype == k_cache.dtype == v_cache.dtype == torch.int8 and lens.dtype == torch.int32 and lens.is_cuda
+        ld_new = 0
+        if k_new is not None:
+            assert k_new.stride(0) == v_new.stride(0) and k_new.dtype == torch.int8
+            ld_new = k_new.stride(0) if k_new.shape[0] > 1 else max(k_new.stride(0), k_new.shape[1])
+        ld_q = q.stride(0) if q.shape[0] > 1 else max(q.stride(0), q.shape[1])
+        a = DecodeAttnArgs(q.data_ptr(), ld_q, k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(1), k_cache.stride(0),
+                           _ptr(k_new), _ptr(v_new), ld_new, lens.data_ptr(), int(max_len), q.shape[0], nh, dh, s_q, s_k, s_v,
+                           s_p, P_MODE[p_mode] if isinstance(p_mode, str) else p_mode, out)
+        _check(lib().hero_int8_decode_attention(self._h, C.byref(a), _stream(stream)))
 
     def hero_absmax_observe(self, x, col_absmax=None, tensor_absmax=None, stream=None):
         """x: hero.Tensor (F16 / BF16); col_absmax float32[cols] / tensor_absmax float32[1]: running maxima, updated."""
