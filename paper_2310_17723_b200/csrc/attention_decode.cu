@@ -23,7 +23,6 @@
 
 namespace hero {
 
-constexpr int DEC_THREADS = 128;
 constexpr int DEC_MAX_CHUNK = 12288;          // keys per CTA: 4 bytes of score + 1 byte of P each, within 64 KB
 constexpr int DEC_MAX_SPLITS = 8;             // portable cluster size
 constexpr float DEC_MAGIC = 12582912.0f;      // 1.5 * 2^23
@@ -69,17 +68,21 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-template <int DH>
-__global__ void __launch_bounds__(DEC_THREADS) attn_decode_kernel(const DecodeParams p) {
+// NT threads per CTA: 128 when the launch has CTAs to spare, 256 when (sequence, head) pairs are few and every CTA has
+// to keep more loads in flight.
+template <int DH, int NT>
+__global__ void __launch_bounds__(NT) attn_decode_kernel(const DecodeParams p) {
+  constexpr int U = 1;                         // key quads in flight per thread (two measured slower: 37 against 27 us on B8 S2048 dh128)
+  constexpr int DEC_THREADS = NT, DEC_WARPS = NT / 32;
   constexpr int TPK = DH / 16;                 // lanes per key
-  constexpr int G = DEC_THREADS / TPK;         // key quads in flight per CTA sweep
+  constexpr int G = DEC_THREADS / TPK;         // key quads per CTA sweep
   extern __shared__ __align__(16) uint8_t dsm[];
   float* sc = reinterpret_cast<float*>(dsm);                        // [chunk_cap] scores, then exponentials
   uint32_t* pw = reinterpret_cast<uint32_t*>(sc + p.chunk_cap);     // [chunk_cap / 4] four P_u8 per word
-  int* red = reinterpret_cast<int*>(pw + p.chunk_cap / 4);          // [G][DH] partial sums of the key groups
-  int* part = red + G * DH;                                         // [DH] this CTA's partial sums
+  int* red = reinterpret_cast<int*>(pw + p.chunk_cap / 4);          // [warps][DH] partial sums of the warps
+  int* part = red + DEC_WARPS * DH;                                         // [DH] this CTA's partial sums
   float* xch = reinterpret_cast<float*>(part + DH);                 // [2] (m_c, l_c)
-  float* wred = xch + 2;                                            // [4] per-warp scratch
+  float* wred = xch + 2;                                            // [DEC_WARPS] per-warp scratch
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int c = tid % TPK, g = tid / TPK;
@@ -115,24 +118,29 @@ __global__ void __launch_bounds__(DEC_THREADS) attn_decode_kernel(const DecodePa
   // ---- 1: scores
   const uint4 qv = __ldg(reinterpret_cast<const uint4*>(p.q + (long long)b * p.ld_q + col));
   float mloc = -INFINITY;
-  for (int q0 = 0; q0 < nq; q0 += G) {                      // trip count uniform over the warp: the shuffles below need every lane
-    const int qd = q0 + g;
-    uint4 kv[4];
+  for (int q0 = 0; q0 < nq; q0 += U * G) {                  // trip count uniform over the warp: the shuffles below need every lane
+    uint4 kv[U][4];                                          // U quads = 4 U keys in flight per thread
 #pragma unroll
-    for (int j = 0; j < 4; ++j) kv[j] = __ldg(krow(min(k0 + 4 * qd + j, k1 - 1)));
-    float t[4];
+    for (int u = 0; u < U; ++u)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      int a = dp4a_ss(kv[j].x, qv.x, 0);
-      a = dp4a_ss(kv[j].y, qv.y, a);
-      a = dp4a_ss(kv[j].z, qv.z, a);
-      a = dp4a_ss(kv[j].w, qv.w, a);
+      for (int j = 0; j < 4; ++j) kv[u][j] = __ldg(krow(min(k0 + 4 * (q0 + u * G + g) + j, k1 - 1)));
 #pragma unroll
-      for (int o = 1; o < TPK; o <<= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-      t[j] = (4 * qd + j < n) ? (float)a * p.score_scale : -INFINITY;
-      mloc = fmaxf(mloc, t[j]);
+    for (int u = 0; u < U; ++u) {
+      const int qd = q0 + u * G + g;
+      float t[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int a = dp4a_ss(kv[u][j].x, qv.x, 0);
+        a = dp4a_ss(kv[u][j].y, qv.y, a);
+        a = dp4a_ss(kv[u][j].z, qv.z, a);
+        a = dp4a_ss(kv[u][j].w, qv.w, a);
+#pragma unroll
+        for (int o = 1; o < TPK; o <<= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        t[j] = (4 * qd + j < n) ? (float)a * p.score_scale : -INFINITY;
+        mloc = fmaxf(mloc, t[j]);
+      }
+      if (c == 0 && qd < nq) *reinterpret_cast<float4*>(sc + 4 * qd) = make_float4(t[0], t[1], t[2], t[3]);
     }
-    if (c == 0 && qd < nq) *reinterpret_cast<float4*>(sc + 4 * qd) = make_float4(t[0], t[1], t[2], t[3]);
   }
   // rank 0 appends the new token to the cache (its own lanes cover the row once)
   if (fresh && rank == 0 && g == 0) {
@@ -142,7 +150,9 @@ __global__ void __launch_bounds__(DEC_THREADS) attn_decode_kernel(const DecodePa
   mloc = warp_max(mloc);
   if (lane == 0) wred[warp] = mloc;
   __syncthreads();
-  const float m_c = fmaxf(fmaxf(wred[0], wred[1]), fmaxf(wred[2], wred[3]));   // -inf when this CTA has no key
+  float m_c = wred[0];                                       // -inf when this CTA has no key
+#pragma unroll
+  for (int w = 1; w < DEC_WARPS; ++w) m_c = fmaxf(m_c, wred[w]);
   __syncthreads();
 
   // ---- 2: exponentials in place, CTA sum
@@ -155,7 +165,12 @@ __global__ void __launch_bounds__(DEC_THREADS) attn_decode_kernel(const DecodePa
   lloc = warp_sum(lloc);
   if (lane == 0) wred[warp] = lloc;
   __syncthreads();
-  if (tid == 0) { xch[0] = m_c; xch[1] = (wred[0] + wred[1]) + (wred[2] + wred[3]); }
+  if (tid == 0) {
+    float lc = 0.f;
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) lc += wred[w];
+    xch[0] = m_c; xch[1] = lc;
+  }
   ptx::cluster_sync();
   float m = -INFINITY, l = 0.f;
   {
@@ -189,32 +204,49 @@ __global__ void __launch_bounds__(DEC_THREADS) attn_decode_kernel(const DecodePa
   int acc[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) acc[i] = 0;
-  for (int qd = g; qd < nq; qd += G) {
-    const uint32_t p4 = pw[qd];
-    if (p4 == 0) continue;
-    uint4 vv[4];
+  for (int q0 = g; q0 < nq; q0 += U * G) {
+    uint32_t p4[U], any = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) vv[j] = __ldg(vrow(min(k0 + 4 * qd + j, k1 - 1)));
-    const uint32_t x[4][4] = {{vv[0].x, vv[1].x, vv[2].x, vv[3].x}, {vv[0].y, vv[1].y, vv[2].y, vv[3].y},
-                              {vv[0].z, vv[1].z, vv[2].z, vv[3].z}, {vv[0].w, vv[1].w, vv[2].w, vv[3].w}};
+    for (int u = 0; u < U; ++u) { p4[u] = (q0 + u * G < nq) ? pw[q0 + u * G] : 0u; any |= p4[u]; }
+    if (any == 0) continue;
+    uint4 vv[U][4];
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {                              // features 4 w .. 4 w + 3 of this lane's slice
-      const uint32_t ab = __byte_perm(x[w][0], x[w][1], 0x5140), cd = __byte_perm(x[w][2], x[w][3], 0x5140);
-      const uint32_t ef = __byte_perm(x[w][0], x[w][1], 0x7362), gh = __byte_perm(x[w][2], x[w][3], 0x7362);
-      acc[4 * w + 0] = dp4a_su(__byte_perm(ab, cd, 0x5410), p4, acc[4 * w + 0]);
-      acc[4 * w + 1] = dp4a_su(__byte_perm(ab, cd, 0x7632), p4, acc[4 * w + 1]);
-      acc[4 * w + 2] = dp4a_su(__byte_perm(ef, gh, 0x5410), p4, acc[4 * w + 2]);
-      acc[4 * w + 3] = dp4a_su(__byte_perm(ef, gh, 0x7632), p4, acc[4 * w + 3]);
+    for (int u = 0; u < U; ++u)
+      if (p4[u] != 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) vv[u][j] = __ldg(vrow(min(k0 + 4 * (q0 + u * G) + j, k1 - 1)));
+      }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (p4[u] == 0) continue;
+      const uint32_t x[4][4] = {{vv[u][0].x, vv[u][1].x, vv[u][2].x, vv[u][3].x}, {vv[u][0].y, vv[u][1].y, vv[u][2].y, vv[u][3].y},
+                                {vv[u][0].z, vv[u][1].z, vv[u][2].z, vv[u][3].z}, {vv[u][0].w, vv[u][1].w, vv[u][2].w, vv[u][3].w}};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {                            // features 4 w .. 4 w + 3 of this lane's slice
+        const uint32_t ab = __byte_perm(x[w][0], x[w][1], 0x5140), cd = __byte_perm(x[w][2], x[w][3], 0x5140);
+        const uint32_t ef = __byte_perm(x[w][0], x[w][1], 0x7362), gh = __byte_perm(x[w][2], x[w][3], 0x7362);
+        acc[4 * w + 0] = dp4a_su(__byte_perm(ab, cd, 0x5410), p4[u], acc[4 * w + 0]);
+        acc[4 * w + 1] = dp4a_su(__byte_perm(ab, cd, 0x7632), p4[u], acc[4 * w + 1]);
+        acc[4 * w + 2] = dp4a_su(__byte_perm(ef, gh, 0x5410), p4[u], acc[4 * w + 2]);
+        acc[4 * w + 3] = dp4a_su(__byte_perm(ef, gh, 0x7632), p4[u], acc[4 * w + 3]);
+      }
     }
   }
-  // ---- 5: key groups -> CTA -> cluster -> output stage
+  // ---- 5: key groups of a warp (shuffles) -> warps (shared memory) -> cluster -> output stage
 #pragma unroll
-  for (int i = 0; i < 16; i += 4)
-    *reinterpret_cast<int4*>(red + g * DH + c * 16 + i) = make_int4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+  for (int i = 0; i < 16; ++i)
+#pragma unroll
+    for (int o = TPK; o < 32; o <<= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+  if (lane < TPK) {
+#pragma unroll
+    for (int i = 0; i < 16; i += 4)
+      *reinterpret_cast<int4*>(red + warp * DH + c * 16 + i) = make_int4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+  }
   __syncthreads();
   if (tid < DH) {
     int s = 0;
-    for (int gg = 0; gg < G; ++gg) s += red[gg * DH + tid];
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) s += red[w * DH + tid];
     part[tid] = s;
   }
   ptx::cluster_sync();
@@ -239,11 +271,10 @@ __global__ void __launch_bounds__(DEC_THREADS) attn_decode_kernel(const DecodePa
   ptx::cluster_sync();                                       // nobody leaves while rank 0 may still read its sums
 }
 
-template <int DH>
+template <int DH, int NT>
 static hero_status launch_decode(hero_handle* h, const DecodeParams& p, int B, int splits, cudaStream_t stream) {
-  auto kern = attn_decode_kernel<DH>;
-  constexpr int G = DEC_THREADS / (DH / 16);
-  const size_t smem = (size_t)p.chunk_cap * 5 + (size_t)(G * DH + DH) * 4 + 32;
+  auto kern = attn_decode_kernel<DH, NT>;
+  const size_t smem = (size_t)p.chunk_cap * 5 + (size_t)(NT / 32 * DH + DH) * 4 + 8 + NT / 32 * 4 + 16;
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -251,7 +282,7 @@ static hero_status launch_decode(hero_handle* h, const DecodeParams& p, int B, i
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)splits, (unsigned)p.nh, (unsigned)B);
-  cfg.blockDim = dim3(DEC_THREADS);
+  cfg.blockDim = dim3(NT);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute at[2];
@@ -311,12 +342,15 @@ extern "C" hero_status hero_int8_decode_attention(hero_handle* h, const hero_dec
   p.out_scale = a->out.dtype == HERO_I8 ? a->out.scale : nullptr;
   p.out_scale_stride = a->out.gran == HERO_GRAN_FWQ ? 1 : 0;
   p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
-  // key splits: enough CTAs for about four per SM, at least 256 keys each, as many as the score buffer requires
+  // key splits: enough CTAs for about four per SM, at least 512 keys each, as many as the score buffer requires
   int splits = 1;
   const long long heads = (long long)a->B * a->nh;
-  while (splits < DEC_MAX_SPLITS && (heads * splits < 4ll * h->sm_count && a->max_len / (splits * 2) >= 256)) splits *= 2;
+  while (splits < DEC_MAX_SPLITS && (heads * splits < 4ll * h->sm_count && a->max_len / (splits * 2) >= 512)) splits *= 2;
   while (splits < DEC_MAX_SPLITS && (a->max_len + splits - 1) / splits > DEC_MAX_CHUNK) splits *= 2;
   p.chunk_cap = (((a->max_len + splits - 1) / splits) + 4 + 15) & ~15;   // multiple of 16: the arrays behind it stay 16-byte aligned
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return a->dh == 64 ? launch_decode<64>(h, p, a->B, splits, s) : launch_decode<128>(h, p, a->B, splits, s);
+  // few (sequence, head) pairs: wider CTAs keep more loads in flight per SM (38 against 59 us on B1 S16384 dh128)
+  if (heads * splits <= 2ll * h->sm_count)
+    return a->dh == 64 ? launch_decode<64, 256>(h, p, a->B, splits, s) : launch_decode<128, 256>(h, p, a->B, splits, s);
+  return a->dh == 64 ? launch_decode<64, 128>(h, p, a->B, splits, s) : launch_decode<128, 128>(h, p, a->B, splits, s);
 }

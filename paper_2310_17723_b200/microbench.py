@@ -5,6 +5,7 @@
     python -m paper_2310_17723_b200.microbench attn --B 8 --S 384 --nh 16 --dh 64     # INT8 attention
     python -m paper_2310_17723_b200.microbench absmax --M 65536 --H 4096             # calibration observer GB/s
     python -m paper_2310_17723_b200.microbench wquant --N 4096 --K 4096              # fold + Eq. 2 weight quantization GB/s
+    python -m paper_2310_17723_b200.microbench decode --B 8 --S 2048 --nh 32 --dh 128 --graph   # decode attention GB/s
     python -m paper_2310_17723_b200.microbench layer --workload c3 [--f8 | --fp]   # one whole layer, us per forward
     ... --sweep runs the standalone-kernel sweep of the benchmark configurations instead of one shape.
 
@@ -152,6 +153,31 @@ def bench_wquant(h, N, K, iters):
           % (N, K, t * 1e6, gbs, gbs / hbm, src), flush=True)
 
 
+def bench_decode(h, B, S, nh, dh, iters, p_mode="static"):
+    """One decode step of the INT8 attention core: every sequence holds S cache entries.  Algorithmic bytes: every key
+    and value once (2 B S H); several caches are rotated so that the reads come from HBM.  The kernel does not fetch value
+    rows whose probabilities quantize to zero, so the timed query is all zeros: a flat softmax, under which the row-max
+    quantizer gives every key the code 255 and every value row is read (the worst case; the static quantizer of Eq. 16
+    rounds 1 / S to zero for S > 510 and then reads the keys only)."""
+    H = nh * dh
+    n = max(2, min(32, int(400e6 // (2 * B * S * H)) + 1))
+    q = torch.zeros(B, H, device="cuda", dtype=torch.int8)
+    ks = [torch.randint(-127, 128, (B, S, H), device="cuda", dtype=torch.int8) for _ in range(n)]
+    vs = [torch.randint(-127, 128, (B, S, H), device="cuda", dtype=torch.int8) for _ in range(n)]
+    lens = torch.full((B,), S, device="cuda", dtype=torch.int32)
+    out = torch.empty(B, H, device="cuda", dtype=torch.int8)
+    osc = torch.full((H,), 0.01, device="cuda")
+    s = 0.03
+    t = _time(lambda i: h.hero_int8_decode_attention(q, ks[i], vs[i], lens, S, nh, dh, hero.tensor(out, "fwq", osc), s_q=s, s_k=s,
+                                                     s_v=0.02, s_p=1.0 / 255, p_mode=p_mode), n, iters)
+    hbm, _, src = _peaks()
+    keys_only = p_mode == "static" and S > 510            # P = 1 / S rounds to zero: no value row is fetched
+    gbs = (1.0 if keys_only else 2.0) * B * S * H / t / 1e9
+    print("decode attention B=%d S=%d nh=%d dh=%d %s: %.1f us, %.0f GB/s (%s), %.2f of %s copy bandwidth"
+          % (B, S, nh, dh, p_mode, t * 1e6, gbs, "keys once; all P_u8 = 0" if keys_only else "keys and values once", gbs / hbm, src),
+          flush=True)
+
+
 def bench_layer(h, workload, payload, fp, iters):
     """One forward of a single layer of a benchmark configuration (INT8, e4m3 or all-FP modules), L2 flushed between
     forwards by a 256 MB write (its time is measured alone and subtracted)."""
@@ -179,7 +205,7 @@ def bench_layer(h, workload, payload, fp, iters):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant", "layer"])
+    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant", "layer", "decode"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4"])
     ap.add_argument("--M", type=int, default=65536)
     ap.add_argument("--H", type=int, default=1024)
@@ -220,6 +246,8 @@ def main():
         bench_absmax(h, a.M, a.H, a.iters)
     elif a.kernel == "wquant":
         bench_wquant(h, a.N, a.K, a.iters)
+    elif a.kernel == "decode":
+        bench_decode(h, a.B, a.S, a.nh, a.dh, a.iters, a.p_mode)
     elif a.kernel == "layer":
         bench_layer(h, a.workload, "f8" if a.f8 else "i8", a.fp, a.iters)
     else:
