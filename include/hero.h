@@ -344,6 +344,26 @@ hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const h
                                const hero_tensor* pending, const hero_tensor* out, void* workspace,
                                size_t workspace_bytes, void* stream);
 
+/* One decode step of the layer: the new token of each of the B sequences (in: [B, H], typed as for hero_layer_forward)
+ * goes through the same modules, the attention core in its decode form (hero_int8_decode_attention) against this
+ * layer's INT8 key / value cache.  The step stores the new token's key and value at entry len[b] - 1 of the caches
+ * (the caller increments len before the call and owns the caches) and writes out: [B, H].  The attention module must
+ * be HERO_MODE_INT8 with the INT8 payload; desc->S is not used; the workspace is the one of a forward pass or at least
+ * hero_layer_workspace_bytes(desc, B).  The result equals row len[b] - 1 of a causal forward pass over the sequence
+ * so far (up to rounding ties). */
+typedef struct {
+  void* k_cache;           /* device I8, entry t of sequence b at k_cache + b * batch_stride + t * ld_kv, H features */
+  void* v_cache;
+  int64_t ld_kv;
+  int64_t batch_stride;
+  const int32_t* len;      /* device int32 [B]: cache entries including the new token */
+  int32_t max_len;         /* host-side upper bound on len[b] */
+} hero_kv_cache;
+
+hero_status hero_layer_decode(hero_handle* h, const hero_layer_desc* desc, const hero_kv_cache* kv, const hero_tensor* in,
+                              const hero_tensor* pending, const hero_tensor* out, void* workspace, size_t workspace_bytes,
+                              void* stream);
+
 /* The same layer (Sec. 2.2.2-2.2.3) called with HOST activation buffers: copies `in_host` (payload and, for
  * a token-wise input, its per-row scales) into the caller's device staging tensor `in_dev`, runs
  * hero_layer_forward, copies the result back into `out_host` and synchronizes the stream.  Host buffers

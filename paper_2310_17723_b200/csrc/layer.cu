@@ -19,7 +19,8 @@ static hero_status plan_layer(const hero_layer_desc* d, int64_t M, LayerPlan* pl
   HERO_REQUIRE(d->arch == HERO_POST_LN || d->arch == HERO_PRE_LN, HERO_ERR_INVALID_ARG, "unknown arch %d", d->arch);
   HERO_REQUIRE(d->B > 0 && d->S > 0 && d->H > 0 && d->nh > 0 && d->F > 0 && d->H % d->nh == 0, HERO_ERR_INVALID_ARG,
                "bad layer dimensions");
-  HERO_REQUIRE(M == (int64_t)d->B * d->S, HERO_ERR_INVALID_ARG, "M=%lld != B*S", (long long)M);
+  HERO_REQUIRE(M == (int64_t)d->B * d->S || M == (int64_t)d->B, HERO_ERR_INVALID_ARG, "M=%lld is neither B*S (a forward pass) nor B (a decode step)",
+               (long long)M);
   HERO_REQUIRE(is_fp16ish(d->fp_dtype), HERO_ERR_INVALID_ARG, "fp_dtype must be F16 or BF16");
   for (int i = 0; i < 5; ++i)
     HERO_REQUIRE(d->mode[i] == HERO_MODE_INT8 || d->mode[i] == HERO_MODE_FP, HERO_ERR_INVALID_ARG, "mode[%d]=%d", i, d->mode[i]);
@@ -77,12 +78,16 @@ extern "C" hero_status hero_layer_workspace_layout(const hero_layer_desc* d, int
   return HERO_OK;
 }
 
-extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in,
-                                          const hero_tensor* pending, const hero_tensor* out, void* workspace,
-                                          size_t workspace_bytes, void* stream) {
-  using namespace hero;
+namespace hero {
+// The layer on M = B*S tokens (kv == NULL), or one decode step on M = B new tokens against the layer's key / value
+// cache: the same launches with the attention core replaced by its decode form.
+static hero_status layer_impl(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in, const hero_tensor* pending,
+                              const hero_tensor* out, void* workspace, size_t workspace_bytes, void* stream,
+                              const hero_kv_cache* kv) {
   HERO_REQUIRE(h && d && in && out, HERO_ERR_INVALID_ARG, "hero_layer_forward: NULL argument");
   const int64_t M = in->rows;
+  HERO_REQUIRE(M == (kv ? (int64_t)d->B : (int64_t)d->B * d->S), HERO_ERR_INVALID_ARG, "in has %lld rows: %s expected", (long long)M,
+               kv ? "B (one new token per sequence)" : "B*S");
   LayerPlan pl;
   hero_status st = plan_layer(d, M, &pl);
   if (st != HERO_OK) return st;
@@ -153,7 +158,22 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
   // ---- attention core (Eq. 15-17)
   hero_tensor x_attn = o8 ? mk(ws + pl.off_attn, q8, d->gran_attn, M, H, d->s_attn)
                           : mk(ws + pl.off_attn, fp, HERO_GRAN_NONE, M, H, nullptr);
-  {
+  if (kv) {
+    // decode: the query and the new key / value are the thirds of the QKV rows; the step appends them to the cache
+    HERO_REQUIRE(attn8 && q8 == HERO_I8, HERO_ERR_UNSUPPORTED, "a decode step needs the INT8 attention core");
+    hero_decode_attn_args a;
+    memset(&a, 0, sizeof(a));
+    const int8_t* base = static_cast<const int8_t*>(qkv.data);
+    a.q = base; a.ld_q = 3 * H;
+    a.k_new = base + H; a.v_new = base + 2 * H; a.ld_new = 3 * H;
+    a.k_cache = kv->k_cache; a.v_cache = kv->v_cache; a.ld_kv = kv->ld_kv; a.batch_stride = kv->batch_stride;
+    a.len = kv->len; a.max_len = kv->max_len;
+    a.B = d->B; a.nh = d->nh; a.dh = H / d->nh;
+    a.s_q = d->s_q; a.s_k = d->s_k; a.s_v = d->s_v; a.s_p = d->s_p;
+    a.p_mode = d->p_mode;
+    a.out = x_attn;
+    if ((st = hero_int8_decode_attention(h, &a, stream)) != HERO_OK) return st;
+  } else {
     hero_attn_args a;
     memset(&a, 0, sizeof(a));
     uint8_t* base = static_cast<uint8_t*>(qkv.data);
@@ -228,6 +248,21 @@ extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc*
     if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
   }
   return HERO_OK;
+}
+}  // namespace hero
+
+extern "C" hero_status hero_layer_forward(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in,
+                                          const hero_tensor* pending, const hero_tensor* out, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
+  return hero::layer_impl(h, d, in, pending, out, workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" hero_status hero_layer_decode(hero_handle* h, const hero_layer_desc* d, const hero_kv_cache* kv, const hero_tensor* in,
+                                         const hero_tensor* pending, const hero_tensor* out, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(kv && kv->k_cache && kv->v_cache && kv->len, HERO_ERR_INVALID_ARG, "hero_layer_decode: the key / value cache is required");
+  return layer_impl(h, d, in, pending, out, workspace, workspace_bytes, stream, kv);
 }
 
 extern "C" hero_status hero_layer_forward_host_async(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,

@@ -84,6 +84,11 @@ class LayerDesc(C.Structure):
                 ("p_mode", C.c_int32), ("payload", C.c_int32)]
 
 
+class KvCache(C.Structure):
+    _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("ld_kv", C.c_int64), ("batch_stride", C.c_int64),
+                ("len", C.c_void_p), ("max_len", C.c_int32)]
+
+
 class LayerLayout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("qkv", "x_attn", "x_o", "x_mid", "x_mid_scale", "a", "x_2", "x_in", "x_in_scale",
                                           "h_in", "h_mid", "total")]
@@ -127,6 +132,8 @@ def lib():
         L.hero_layer_workspace_layout.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(LayerLayout)]
         L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hero_layer_decode.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(KvCache), C.POINTER(Tensor), C.POINTER(Tensor),
+                                        C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_host_async.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
             [C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_host.argtypes = [C.c_void_p, C.POINTER(LayerDesc)] + [C.POINTER(Tensor)] * 4 + \
@@ -293,6 +300,16 @@ class Handle:
         pend = C.byref(pending) if pending is not None else None
         _check(lib().hero_layer_forward(self._h, C.byref(desc), C.byref(x_in), pend, C.byref(out),
                                         C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)))
+
+    def hero_layer_decode(self, desc, k_cache, v_cache, lens, max_len, x_in, out, workspace, pending=None, stream=None):
+        """One decode step: k_cache / v_cache int8 [B, S_max, H] views of equal strides (the new key / value are stored at
+        lens[b] - 1), lens int32 [B]; x_in / out / pending: hero.Tensor with B rows."""
+        assert k_cache.dim() == 3 and k_cache.stride() == v_cache.stride() and k_cache.stride(2) == 1
+        assert k_cache.dtype == v_cache.dtype == torch.int8 and lens.dtype == torch.int32 and lens.is_cuda
+        kv = KvCache(k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(1), k_cache.stride(0), lens.data_ptr(), int(max_len))
+        pend = C.byref(pending) if pending is not None else None
+        _check(lib().hero_layer_decode(self._h, C.byref(desc), C.byref(kv), C.byref(x_in), pend, C.byref(out),
+                                       C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)))
 
 
 def host_tensor(t, gran="none", scale=None):

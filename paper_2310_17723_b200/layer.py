@@ -62,3 +62,8 @@ class Layer:
     def forward(self, x_in, out, pending=None, stream=None):
         """x_in / out / pending are hero.Tensor structs; runs the whole layer on the current stream."""
         self.h.hero_layer_forward(self.desc, x_in, out, self.workspace, pending=pending, stream=stream)
+
+    def decode(self, k_cache, v_cache, lens, max_len, x_in, out, pending=None, stream=None):
+        """One decode step against this layer's INT8 key / value cache (x_in / out have B rows)."""
+        self.h.hero_layer_decode(self.desc, k_cache, v_cache, lens, max_len, x_in, out, self.workspace, pending=pending,
+                                 stream=stream)

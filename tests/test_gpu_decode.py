@@ -158,3 +158,72 @@ def test_decode_attention_refusals(h):
                                 tl.data_ptr(), 64, 2, 2, 64, 1.0, 1.0, 1.0, 1.0 / 255, 0, hero.tensor(out))
         hero._check(hero.lib().hero_int8_decode_attention(h._h, hero.C.byref(a), hero._stream(None)))
     h.check()
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# the whole layer, one decode step at a time, against the oracle's causal forward pass over the sequence so far
+# ------------------------------------------------------------------------------------------------------------------
+from oracle import layer as OL
+from paper_2310_17723_b200.layer import Layer
+from gpu_util import qt_to_device, oracle_layer_to_prepared, TORCH_FP
+
+
+@pytest.mark.parametrize("arch,dh,p_mode", [("pre_ln", 64, "static"), ("pre_ln", 128, "rowmax"), ("post_ln", 64, "static")])
+def test_layer_decode_steps_match_causal_forward_rows(h, arch, dh, p_mode):
+    B, S, H, F = 3, 131, 256, 512                        # the last two tokens of each sequence are decoded one by one
+    shape = W.tiny_shape(B=B, S=S, H=H, nh=H // dh, F=F, arch=arch, mask="causal", fp_dtype="bf16", eps=1e-5)
+    spec = OL.LayerSpec(B=B, S=S, H=H, nh=H // dh, F=F, arch=arch, mask="causal", fp_dtype="bf16", eps=1e-5, p_mode=p_mode,
+                        gran_out="fp")
+    p = W.layer_params(shape, 61)
+    x = W.activations(shape, 61)
+    cal = O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps) if arch == "post_ln" else x
+    Lp = OL.prepare_layer(spec, p, OL.calibrate(spec, p, cal, B))
+    if arch == "post_ln":
+        x_in = OL.entry_ln(O.fp_tensor(x, "bf16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"])
+    else:
+        x_in = O.fp_tensor(x, "bf16")
+    T = OL.layer_forward(Lp, x_in)                       # causal forward pass over all S tokens (the oracle)
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    qkv = T["qkv"].data.reshape(B, S, 3 * H)
+    kc = torch.from_numpy(np.ascontiguousarray(qkv[:, :, H:2 * H])).cuda()
+    vc = torch.from_numpy(np.ascontiguousarray(qkv[:, :, 2 * H:])).cuda()
+    kc[:, S - 2:], vc[:, S - 2:] = 77, -77               # the two positions to be decoded hold garbage
+    want_out = T["x_out"].real().reshape(B, S, H)
+    for t in (S - 2, S - 1):
+        rows = [b * S + t for b in range(B)]
+        if arch == "post_ln":
+            xin_t = O.QT("i8", x_in.data[rows], row_scale=x_in.row_scale[rows])
+        else:
+            xin_t = O.QT("fp", x_in.data[rows], dtype="bf16")
+        _, in_desc, _ = qt_to_device(xin_t)
+        out = torch.full((B, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lens = dev(np.full(B, t + 1, np.int32))
+        n0 = h.launches
+        layer.decode(kc, vc, lens, S, in_desc, hero.tensor(out))
+        h.check()
+        assert h.launches - n0 == (8 if arch == "pre_ln" else 7)
+        got = out.float().cpu().numpy().astype(np.float64)
+        assert rel_err(got, want_out[:, t]) < 1e-2, t
+        # the step appended the token's key and value (the QKV GeMM^quant output of the few-row kernel)
+        assert_int8_close(kc[:, t].cpu().numpy(), qkv[:, t, H:2 * H], frac=1e-3, what="appended keys")
+        assert_int8_close(vc[:, t].cpu().numpy(), qkv[:, t, 2 * H:], frac=1e-3, what="appended values")
+    assert np.array_equal(kc[:, :S - 2].cpu().numpy(), qkv[:, :S - 2, H:2 * H])
+
+
+def test_layer_decode_refusals(h):
+    shape = W.tiny_shape(B=2, S=64, H=256, nh=4, F=512, arch="pre_ln", mask="causal", fp_dtype="bf16", eps=1e-5)
+    spec = OL.LayerSpec(B=2, S=64, H=256, nh=4, F=512, arch="pre_ln", mask="causal", fp_dtype="bf16", eps=1e-5,
+                        mode=dict(OL.MODE_PRESETS["M1"]))
+    p = W.layer_params(shape, 62)
+    x = W.activations(shape, 62)
+    Lp = OL.prepare_layer(spec, p, OL.calibrate(spec, p, x, 2))
+    layer = Layer(h, oracle_layer_to_prepared(Lp))
+    kc = torch.zeros(2, 64, 256, dtype=torch.int8, device="cuda")
+    xin = torch.zeros(2, 256, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty_like(xin)
+    lens = dev(np.asarray([5, 6], np.int32))
+    with pytest.raises(hero.HeroError):                  # M1 leaves the attention core in FP: no decode form
+        layer.decode(kc, kc.clone(), lens, 64, hero.tensor(xin), hero.tensor(out))
+    with pytest.raises(hero.HeroError):                  # one row per sequence
+        layer.decode(kc, kc.clone(), lens, 64, hero.tensor(torch.zeros(4, 256, dtype=torch.bfloat16, device="cuda")), hero.tensor(out))
+    h.check()
