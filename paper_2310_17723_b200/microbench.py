@@ -6,6 +6,7 @@
     python -m paper_2310_17723_b200.microbench absmax --M 65536 --H 4096             # calibration observer GB/s
     python -m paper_2310_17723_b200.microbench wquant --N 4096 --K 4096              # fold + Eq. 2 weight quantization GB/s
     python -m paper_2310_17723_b200.microbench decode --B 8 --S 2048 --nh 32 --dh 128 --graph   # decode attention GB/s
+    python -m paper_2310_17723_b200.microbench layer-decode --workload c4 --B 8 --S 2048 --graph   # one decode step of a layer
     python -m paper_2310_17723_b200.microbench layer --workload c3 [--f8 | --fp]   # one whole layer, us per forward
     ... --sweep runs the standalone-kernel sweep of the benchmark configurations instead of one shape.
 
@@ -178,6 +179,43 @@ def bench_decode(h, B, S, nh, dh, iters, p_mode="static"):
           flush=True)
 
 
+def bench_layer_decode(h, workload, B, S, iters, p_mode="rowmax"):
+    """One decode step of a layer of the named configuration's width: B sequences with S cache entries each.  What bounds
+    it is reading the layer's INT8 weights and the key / value caches once: bytes = 12 H^2 (F = 4H) + 2 B S H.  Several
+    caches are rotated; the row-max quantizer is timed because it reads every value row (see bench_decode)."""
+    from . import prep
+    from .layer import Layer
+    full = {"c3": W.C3, "c4": W.C4}[workload]
+    shape = W.tiny_shape(B=B, S=128, H=full.H, nh=full.nh, F=full.F, arch=full.arch, mask="causal", fp_dtype=full.fp_dtype,
+                         eps=full.eps)
+    cfg = prep.LayerConfig(B=B, S=128, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, eps=shape.eps, mask="causal",
+                           fp_dtype=shape.fp_dtype, mode=dict(prep.PRESETS["M3"]), p_mode=p_mode,
+                           gran_out="fp" if shape.arch == "pre_ln" else "twq")
+    p = W.layer_params(shape, 4)
+    x_cal = W.activations(shape, 4, n_seq=1, tensor=7).astype("float64")
+    if shape.arch == "post_ln":
+        from .model import _ln_np
+        x_cal = _ln_np(x_cal, p["ln0_g"].astype("float64"), p["ln0_b"].astype("float64"), cfg.eps)
+    layer = Layer(h, prep.prepare_layer(cfg, p, prep.calibrate(cfg, p, x_cal, 1)))
+    H = shape.H
+    n = max(2, min(16, int(400e6 // (2 * B * S * H)) + 1))
+    ks = [torch.randint(-127, 128, (B, S, H), device="cuda", dtype=torch.int8) for _ in range(n)]
+    vs = [torch.randint(-127, 128, (B, S, H), device="cuda", dtype=torch.int8) for _ in range(n)]
+    lens = torch.full((B,), S, device="cuda", dtype=torch.int32)
+    if shape.arch == "pre_ln":
+        x = torch.randn(B, H, device="cuda").to(hero.TORCH_FP[shape.fp_dtype])
+        xin, out = hero.tensor(x), hero.tensor(torch.empty_like(x))
+    else:
+        xq = torch.randint(-127, 128, (B, H), device="cuda", dtype=torch.int8)
+        xin = hero.tensor(xq, "twq", torch.full((B,), 0.02, device="cuda"))
+        out = hero.tensor(torch.empty_like(xq), "twq", torch.empty(B, device="cuda"))
+    t = _time(lambda i: layer.decode(ks[i], vs[i], lens, S, xin, out), n, iters)
+    hbm, _, src = _peaks()
+    byts = 4.0 * H * H + 2.0 * H * shape.F + 2.0 * B * S * H
+    print("layer decode step %s B=%d S=%d %s: %.1f us, %.0f tokens/s, %.0f GB/s (weights + caches once), %.2f of %s copy bandwidth"
+          % (workload, B, S, p_mode, t * 1e6, B / t, byts / t / 1e9, byts / t / 1e9 / hbm, src), flush=True)
+
+
 def bench_layer(h, workload, payload, fp, iters):
     """One forward of a single layer of a benchmark configuration (INT8, e4m3 or all-FP modules), L2 flushed between
     forwards by a 256 MB write (its time is measured alone and subtracted)."""
@@ -205,7 +243,7 @@ def bench_layer(h, workload, payload, fp, iters):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant", "layer", "decode"])
+    ap.add_argument("kernel", choices=["ln", "gemm", "attn", "absmax", "wquant", "layer", "decode", "layer-decode"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4"])
     ap.add_argument("--M", type=int, default=65536)
     ap.add_argument("--H", type=int, default=1024)
@@ -246,6 +284,8 @@ def main():
         bench_absmax(h, a.M, a.H, a.iters)
     elif a.kernel == "wquant":
         bench_wquant(h, a.N, a.K, a.iters)
+    elif a.kernel == "layer-decode":
+        bench_layer_decode(h, a.workload, a.B, a.S, a.iters, a.p_mode)
     elif a.kernel == "decode":
         bench_decode(h, a.B, a.S, a.nh, a.dh, a.iters, a.p_mode)
     elif a.kernel == "layer":
