@@ -855,7 +855,8 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
 // no parameter-dependent branch.  Same arithmetic, in the same order, as ln_fast_kernel.
 //   RES / BR : SRC_I8 | SRC_FP (| SRC_NONE for BR);  RSC: the INT8 residual carries a per-row scale (TWQ,
 //   RS_ROW) or a per-feature vector (FWQ / SQ, RS_COL);  an INT8 branch always carries a per-feature vector;
-//   BF: the FP tensors involved are BF16 (else FP16).
+//   BF: the FP tensors involved are BF16 (else FP16);  F8: the 8-bit tensors involved hold e4m3 values instead of INT8
+//   (FP8 variant: scale absmax / 448, saturating conversion instead of round + clip).
 // ------------------------------------------------------------------------------------------------------
 constexpr int RS_ROW = 0, RS_COL = 1;
 
@@ -880,6 +881,16 @@ __device__ __forceinline__ void i8x16_to_f2(const uint4 w, float2* v) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) { v[i] = a[i]; v[4 + i] = b[i]; }
 }
+// 16 e4m3 bytes -> 8 float pairs (the conversion instruction takes two bytes at a time)
+__device__ __forceinline__ void e4m3x16_to_f2(const uint4 w, float2* v) {
+  const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { v[2 * i] = ptx::e4m3x2_to_f32x2(u[i] & 0xffffu); v[2 * i + 1] = ptx::e4m3x2_to_f32x2(u[i] >> 16); }
+}
+template <bool F8>
+__device__ __forceinline__ void q8x16_to_f2(const uint4 w, float2* v) {
+  if constexpr (F8) e4m3x16_to_f2(w, v); else i8x16_to_f2(w, v);
+}
 // 16 floats of one chunk from a piece-major vector in shared memory: piece i of chunk c at float4 index i * NCHUNK + c
 template <int NCHUNK>
 __device__ __forceinline__ void lds_vec16(const float* s, float2* v) {
@@ -900,7 +911,7 @@ __host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes)
   return stages;
 }
 
-template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR>
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8>
 __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
   ptx::pdl_launch_dependents();
   constexpr int H = 1024 * WPR;
@@ -1032,7 +1043,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     for (int k = 0; k < 2; ++k) {
       {
         if constexpr (RES == SRC_I8) {
-          i8x16_to_f2(*reinterpret_cast<const uint4*>(src + k * STRIDE * 16), x[k]);
+          q8x16_to_f2<F8>(*reinterpret_cast<const uint4*>(src + k * STRIDE * 16), x[k]);
           if constexpr (RSC == RS_COL) {
             float2 sc[8];
             lds_vec16<H / 16>(v_rcs + (c_first + k * STRIDE) * 4, sc);
@@ -1048,7 +1059,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
         }
         if constexpr (BR == SRC_I8) {
           float2 b[8], sc[8];
-          i8x16_to_f2(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 16), b);
+          q8x16_to_f2<F8>(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 16), b);
           lds_vec16<H / 16>(v_bcs + (c_first + k * STRIDE) * 4, sc);
 #pragma unroll
           for (int i = 0; i < 8; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
@@ -1128,7 +1139,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 #pragma unroll
         for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
       }
-      const float sc = amax > 0.f ? amax / 127.0f : 1.0f;
+      const float sc = amax > 0.f ? amax / (F8 ? 448.0f : 127.0f) : 1.0f;
       const float2 inv2 = f2(1.0f / sc), mg2 = f2(MAGIC);
       if (wr == 0 && lane == 0) p.out_scale[row] = sc;
       {
@@ -1137,8 +1148,13 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
           uint32_t w[4];
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            const float2 a = __ffma2_rn(x[k][2 * g], inv2, mg2), b = __ffma2_rn(x[k][2 * g + 1], inv2, mg2);
-            w[g] = pack_low_bytes(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(b.x), __float_as_uint(b.y));
+            if constexpr (F8) {
+              const float2 a = __fmul2_rn(x[k][2 * g], inv2), b = __fmul2_rn(x[k][2 * g + 1], inv2);
+              w[g] = ptx::f32x4_to_e4m3x4(a.x, a.y, b.x, b.y);
+            } else {
+              const float2 a = __ffma2_rn(x[k][2 * g], inv2, mg2), b = __ffma2_rn(x[k][2 * g + 1], inv2, mg2);
+              w[g] = pack_low_bytes(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(b.x), __float_as_uint(b.y));
+            }
           }
           st_global16(reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * 16, w[0], w[1], w[2], w[3]);
         }
@@ -1153,6 +1169,11 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
           uint32_t w[4];
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
+            if constexpr (F8) {
+              w[g] = ptx::f32x4_to_e4m3x4(x[k][2 * g].x / sc[2 * g].x, x[k][2 * g].y / sc[2 * g].y, x[k][2 * g + 1].x / sc[2 * g + 1].x,
+                                          x[k][2 * g + 1].y / sc[2 * g + 1].y);
+              continue;
+            }
             const float a = fminf(fmaxf(x[k][2 * g].x / sc[2 * g].x, -127.f), 127.f) + MAGIC;
             const float b = fminf(fmaxf(x[k][2 * g].y / sc[2 * g].y, -127.f), 127.f) + MAGIC;
             const float c = fminf(fmaxf(x[k][2 * g + 1].x / sc[2 * g + 1].x, -127.f), 127.f) + MAGIC;
@@ -1179,7 +1200,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   cp_async_wait<0>();
 }
 
-template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR>
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8>
 static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream) {
   constexpr int H = 1024 * WPR, SLOTS = 8 / WPR;
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2, ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
@@ -1187,7 +1208,7 @@ static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream)
   constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0));
   constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC);
   const size_t smem = (size_t)stages * STAGE + VEC;
-  auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR>;
+  auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8>;
   static bool configured = false;   // per instantiation
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
@@ -1209,13 +1230,13 @@ static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream)
   return HERO_OK;
 }
 
-template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF>
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, bool F8>
 static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) {
   switch (p.H) {
-    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1>(h, p, s);
-    case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2>(h, p, s);
-    case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4>(h, p, s);
-    default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8>(h, p, s);
+    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8>(h, p, s);
+    case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2, F8>(h, p, s);
+    case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4, F8>(h, p, s);
+    default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8, F8>(h, p, s);
   }
 }
 
@@ -1223,10 +1244,14 @@ static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) 
 static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
   if (!(p.H == 1024 || p.H == 2048 || p.H == 4096 || p.H == 8192) || p.ex.data || p.token_ids) return HERO_OK;
-  if (p.res.dt == HERO_F8 || (p.br.data && p.br.dt == HERO_F8) || (p.out && p.out_dt == HERO_F8)) return HERO_OK;   // generic kernel
-  const int res = p.res.dt == HERO_I8 ? SRC_I8 : SRC_FP;
-  const int br = !p.br.data ? SRC_NONE : (p.br.dt == HERO_I8 ? SRC_I8 : SRC_FP);
-  const int out = !p.out ? O_NONE : (p.out_dt != HERO_I8 ? O_FP : (p.out_gran == HERO_GRAN_TWQ ? O_TWQ : O_STATIC));
+  // one 8-bit payload across the call (INT8, or e4m3 for the FP8 variant); a mix takes the generic kernel
+  int q8t = -1;
+  auto q8_ok = [&](bool used, int dt) { if (!used || !is_q8(dt)) return true; if (q8t < 0) q8t = dt; return q8t == dt; };
+  if (!q8_ok(true, p.res.dt) || !q8_ok(p.br.data != nullptr, p.br.dt) || !q8_ok(p.out != nullptr, p.out_dt)) return HERO_OK;
+  const bool f8 = q8t == HERO_F8;
+  const int res = is_q8(p.res.dt) ? SRC_I8 : SRC_FP;
+  const int br = !p.br.data ? SRC_NONE : (is_q8(p.br.dt) ? SRC_I8 : SRC_FP);
+  const int out = !p.out ? O_NONE : (!is_q8(p.out_dt) ? O_FP : (p.out_gran == HERO_GRAN_TWQ ? O_TWQ : O_STATIC));
   const bool fpo = p.fp_out != nullptr;
   // scale kinds the kernel is specialised for
   int rsc = RS_ROW;
@@ -1246,7 +1271,8 @@ static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* t
 #define LNW_CASE(R_, S_, B_, O_, F_)                                                                 \
   if (res == R_ && (R_ != SRC_I8 || rsc == S_) && br == B_ && out == O_ && fpo == F_) {               \
     *taken = true;                                                                                   \
-    return bf ? launch_wide_wpr<R_, S_, B_, O_, F_, true>(h, p, s) : launch_wide_wpr<R_, S_, B_, O_, F_, false>(h, p, s); \
+    if (f8) return bf ? launch_wide_wpr<R_, S_, B_, O_, F_, true, true>(h, p, s) : launch_wide_wpr<R_, S_, B_, O_, F_, false, true>(h, p, s); \
+    return bf ? launch_wide_wpr<R_, S_, B_, O_, F_, true, false>(h, p, s) : launch_wide_wpr<R_, S_, B_, O_, F_, false, false>(h, p, s); \
   }
   LNW_CASE(SRC_I8, RS_COL, SRC_I8, O_TWQ, false)      // Eq. 19: FWQ / SQ residual + FWQ branch -> TWQ
   LNW_CASE(SRC_I8, RS_ROW, SRC_I8, O_TWQ, false)      // Eq. 31: TWQ residual + FWQ branch -> TWQ

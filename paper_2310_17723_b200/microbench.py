@@ -239,6 +239,12 @@ def bench_layer(h, workload, payload, fp, iters):
         st.forward()
     t = _time(step, 1, iters) - t_flush
     print("layer %s %s: %.1f us per forward, %.2f M tokens/s" % (workload, "fp" if fp else payload, t * 1e6, shape.M / t / 1e6), flush=True)
+    # per-launch times of one forward (event pairs around every launch: the sum exceeds the un-instrumented time)
+    h.profile_begin(64)
+    st.forward()
+    torch.cuda.synchronize()
+    fam = {1: "ln", 2: "gemm", 3: "attention"}
+    print("  launches: " + ", ".join("%s %.1f us" % (fam.get(k, "?"), ms * 1e3) for k, ms in h.profile_end()), flush=True)
 
 
 def main():

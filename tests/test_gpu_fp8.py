@@ -214,9 +214,11 @@ def _attn_close(got, want, what):
     assert np.mean(d > 0) <= 5e-3 and np.mean(d > step) <= 2e-4 and np.all(d <= 2 * step), (what, stats)
 
 
-@pytest.mark.parametrize("gran_in,gran_attn", [("twq", "fwq"), ("fwq", "sq")])
-def test_post_ln_layer_e4m3_stage_by_stage(h, gran_in, gran_attn):
-    shape = W.tiny_shape(B=2, S=200, H=256, nh=4, F=512, eps=1e-5, n_outlier=2)      # ragged attention tiles
+# H = 1024 rows take the specialised LN^quant kernel, H = 256 the generic one
+@pytest.mark.parametrize("gran_in,gran_attn,H,nh", [("twq", "fwq", 256, 4), ("fwq", "sq", 256, 4), ("twq", "fwq", 1024, 8),
+                                                    ("fwq", "sq", 1024, 16)])
+def test_post_ln_layer_e4m3_stage_by_stage(h, gran_in, gran_attn, H, nh):
+    shape = W.tiny_shape(B=2, S=200, H=H, nh=nh, F=2 * H, eps=1e-5, n_outlier=2)      # ragged attention tiles
     spec, Lp, x_in = _f8_layer(shape, 31, gran_in=gran_in, gran_mid=gran_in, gran_attn=gran_attn)
     M, H, F = spec.M, spec.H, spec.F
     T = OL.layer_forward(Lp, x_in)
@@ -254,9 +256,9 @@ def test_post_ln_layer_e4m3_stage_by_stage(h, gran_in, gran_attn):
     assert float(np.abs(got - T["x_out"].real()).mean() / np.abs(T["x_out"].real()).mean()) < 5e-3
 
 
-@pytest.mark.parametrize("preset", ["M2", "M3"])
-def test_pre_ln_causal_layer_e4m3(h, preset):
-    shape = W.tiny_shape(B=2, S=256, H=256, nh=2, F=512, arch="pre_ln", mask="causal", fp_dtype="bf16", eps=1e-5)
+@pytest.mark.parametrize("preset,H", [("M2", 256), ("M3", 256), ("M3", 1024)])
+def test_pre_ln_causal_layer_e4m3(h, preset, H):
+    shape = W.tiny_shape(B=2, S=256, H=H, nh=H // 128, F=2 * H, arch="pre_ln", mask="causal", fp_dtype="bf16", eps=1e-5)
     spec, Lp, x_in = _f8_layer(shape, 33, mode=dict(OL.MODE_PRESETS[preset]))
     M, H, F, fd = spec.M, spec.H, spec.F, spec.fp_dtype
     T = OL.layer_forward(Lp, x_in)
