@@ -320,6 +320,23 @@ def run_ours(args):
     step()
     launches_per_step = h.launches - n0
     torch.cuda.synchronize()
+    eager_step = step
+    replayed = [0]
+    if args.graph:
+        # the same launches through the C ABI, captured once; a replay issues them without host work in between
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                stack.forward()
+        torch.cuda.synchronize()
+
+        def step():
+            graph.replay()
+            replayed[0] += launches_per_step           # the handle counts launches as they are issued, i.e. at capture
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
 
     # ---- timed region: K steps, each bracketed by events on the launching stream, L2 flushed in between
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -328,6 +345,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
     n0 = h.launches
+    replayed[0] = 0
     for k in range(args.steps):
         flush.zero_()
         ev[k][0].record(stream)
@@ -337,7 +355,7 @@ def run_ours(args):
     if dist:
         dist.barrier()
     wall = time.perf_counter() - wall0
-    gpu_launches = h.launches - n0
+    gpu_launches = h.launches - n0 + replayed[0]
     h.check()
     total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), dist, "cuda")
     ms_per_step = total_ms / args.steps
@@ -351,7 +369,7 @@ def run_ours(args):
         h.profile_begin(launches_per_step * args.steps)
         for k in range(args.steps):
             flush.zero_()
-            step()
+            eager_step()
         recs = h.profile_end()
     clocks = sampler.stop() if sampler else None
     if rank == 0:
@@ -491,6 +509,7 @@ def run_ours(args):
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
             "data": "synthetic",
             "config": {"workload": desc, "tokens_per_step_per_gpu": shape.M, "l2": "flushed between timed steps (512 MiB write)",
+                       "launch": "CUDA graph replay of the step's launches" if args.graph else "one C-ABI call per layer, 7-8 kernel launches each",
                        "timing": "CUDA events per step on the launching stream, max over ranks",
                        "parallelism": "replicas x%d (sequence-sharded, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "kernels": kern,
@@ -509,6 +528,7 @@ def main():
     ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4", "c5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp-path", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="replay the step's launches from a CUDA graph (latency-bound workloads)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
