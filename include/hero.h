@@ -216,7 +216,7 @@ hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* s
  *                  thirds of the QKV GeMM^quant output.  When given, entry len[b] - 1 of the caches is taken from them
  *                  and the call also stores them there (the append is fused); when NULL the caches already hold it.
  *   len          : device int32 [B]; 0 <= len[b] <= max_len; len[b] = 0 writes zeros for sequence b
- *   max_len      : host-side upper bound on len[b] (sizes the launch); at most 98304
+ *   max_len      : host-side upper bound on len[b] (sizes the launch; a larger len[b] is treated as max_len); at most 98304
  *   out          : [B][nh*dh] I8 (gran FWQ scale[H] or SQ scale[1]) or F16 / BF16; dh is 64 or 128
  * Errors: HERO_ERR_INVALID_ARG / HERO_ERR_ALIGNMENT / HERO_ERR_UNSUPPORTED with hero_last_error() saying which.
  */

@@ -32,6 +32,7 @@ struct DecodeParams {
   int8_t* kc; int8_t* vc; long long ld_kv, bstride;
   const int8_t* k_new; const int8_t* v_new; long long ld_new;
   const int* len;
+  int max_len;              // the launch is sized for this many keys: a larger len[b] is clamped to it
   int nh;
   float score_scale;        // d~ log2(e)
   float pv_scale;           // static: s_p s_v; row-max: s_v / 255
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(NT) attn_decode_kernel(const DecodeParams p) {
   const int h = blockIdx.y, b = blockIdx.z;
   ptx::pdl_launch_dependents();
   ptx::pdl_wait();
-  const int L = __ldg(p.len + b);
+  const int L = min(__ldg(p.len + b), p.max_len);
   const int col = h * DH + c * 16;
 
   if (L <= 0) {                                                     // uniform over the cluster: nobody reaches a barrier
@@ -334,7 +335,7 @@ extern "C" hero_status hero_int8_decode_attention(hero_handle* h, const hero_dec
   p.q = static_cast<const int8_t*>(a->q); p.ld_q = a->ld_q;
   p.kc = static_cast<int8_t*>(a->k_cache); p.vc = static_cast<int8_t*>(a->v_cache); p.ld_kv = a->ld_kv; p.bstride = a->batch_stride;
   p.k_new = static_cast<const int8_t*>(a->k_new); p.v_new = static_cast<const int8_t*>(a->v_new); p.ld_new = a->ld_new;
-  p.len = a->len; p.nh = a->nh;
+  p.len = a->len; p.max_len = a->max_len; p.nh = a->nh;
   p.score_scale = a->s_q * a->s_k / sqrtf((float)a->dh) * 1.4426950408889634f;
   p.rowmax = a->p_mode == HERO_P_ROWMAX;
   p.pv_scale = p.rowmax ? a->s_v / 255.0f : a->s_p * a->s_v;

@@ -891,13 +891,46 @@ template <bool F8>
 __device__ __forceinline__ void q8x16_to_f2(const uint4 w, float2* v) {
   if constexpr (F8) e4m3x16_to_f2(w, v); else i8x16_to_f2(w, v);
 }
-// 16 floats of one chunk from a piece-major vector in shared memory: piece i of chunk c at float4 index i * NCHUNK + c
-template <int NCHUNK>
-__device__ __forceinline__ void lds_vec16(const float* s, float2* v) {
+// The CE (16 or 8) floats of one chunk from a piece-major vector in shared memory: piece i of chunk c at float4 index
+// i * NCHUNK + c
+template <int NCHUNK, int CE>
+__device__ __forceinline__ void lds_vec(const float* s, float2* v) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < CE / 4; ++i) {
     const float4 q = *reinterpret_cast<const float4*>(s + 4 * i * NCHUNK);
     v[2 * i] = make_float2(q.x, q.y); v[2 * i + 1] = make_float2(q.z, q.w);
+  }
+}
+// one chunk of CE 8-bit codes (INT8 or e4m3) / CE FP16-BF16 values from the ring -> CE / 2 float pairs
+template <int CE, bool F8>
+__device__ __forceinline__ void ring_q8(const uint8_t* src, float2* v) {
+  if constexpr (CE == 16) {
+    q8x16_to_f2<F8>(*reinterpret_cast<const uint4*>(src), v);
+  } else {
+    const uint2 w = *reinterpret_cast<const uint2*>(src);
+    if constexpr (F8) {
+      v[0] = ptx::e4m3x2_to_f32x2(w.x & 0xffffu); v[1] = ptx::e4m3x2_to_f32x2(w.x >> 16);
+      v[2] = ptx::e4m3x2_to_f32x2(w.y & 0xffffu); v[3] = ptx::e4m3x2_to_f32x2(w.y >> 16);
+    } else {
+      float2 t[4];
+      i8x8_to_f2(w.x, w.y, t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) v[i] = t[i];
+    }
+  }
+}
+template <int CE, bool BF>
+__device__ __forceinline__ void ring_fp(const uint8_t* src, float2* v) {
+  fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src), v);
+  if constexpr (CE == 16) fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src + 16), v + 4);
+}
+// BYTES (8, 16 or 32) of one chunk: global -> ring
+template <int BYTES>
+__device__ __forceinline__ void copy_chunk(uint8_t* dst, const char* src) {
+  if constexpr (BYTES == 8) cp_async8(dst, src);
+  else {
+    cp_async16(dst, src);
+    if constexpr (BYTES == 32) cp_async16(dst + 16, src + 16);
   }
 }
 
@@ -911,12 +944,16 @@ __host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes)
   return stages;
 }
 
-template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8>
+// GEO 0: a lane owns two chunks of 16 elements (H = 1024 * WPR); GEO 1: three chunks of 8 (H = 768 * WPR).
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
 __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
   ptx::pdl_launch_dependents();
-  constexpr int H = 1024 * WPR;
+  constexpr int CE = GEO == 0 ? 16 : 8;            // elements per chunk
+  constexpr int CPL = GEO == 0 ? 2 : 3;            // chunks per lane
+  constexpr int NP = CE / 2;                       // float pairs per chunk
+  constexpr int H = CE * 32 * CPL * WPR;
   constexpr int SLOTS = 8 / WPR;                   // rows per CTA pass
-  constexpr int STRIDE = WPR * 32;                 // chunk stride between a lane's two chunks
+  constexpr int STRIDE = WPR * 32;                 // chunk stride between a lane's chunks
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2;
   constexpr int ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
   constexpr int OFF_BR = H * ES_RES;
@@ -939,11 +976,11 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   const float MAGIC = 12582912.0f;                 // 1.5 * 2^23
   constexpr float fH = (float)H;
 
-  const char* g_res = reinterpret_cast<const char*>(p.res.data) + c_first * 16 * ES_RES;
-  const char* g_br = (BR != SRC_NONE) ? reinterpret_cast<const char*>(p.br.data) + c_first * 16 * ES_BR : nullptr;
+  const char* g_res = reinterpret_cast<const char*>(p.res.data) + c_first * CE * ES_RES;
+  const char* g_br = (BR != SRC_NONE) ? reinterpret_cast<const char*>(p.br.data) + c_first * CE * ES_BR : nullptr;
   const long long pitch_res = p.res.ld * ES_RES, pitch_br = (BR != SRC_NONE) ? p.br.ld * ES_BR : 0;
-  uint8_t* my_ring = ring + slot * SLOT_BYTES + c_first * 16 * ES_RES;          // residual part of this lane's slice
-  uint8_t* my_ring_br = ring + slot * SLOT_BYTES + OFF_BR + c_first * 16 * ES_BR;
+  uint8_t* my_ring = ring + slot * SLOT_BYTES + c_first * CE * ES_RES;          // residual part of this lane's slice
+  uint8_t* my_ring_br = ring + slot * SLOT_BYTES + OFF_BR + c_first * CE * ES_BR;
 
   // A lane copies exactly the chunks it will later read, so waiting on its own copy groups is all the
   // synchronisation the ring needs.
@@ -952,18 +989,12 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
       const char* gr = g_res + row * pitch_res;
       uint8_t* d = my_ring + st * STAGE_BYTES;
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
-#pragma unroll
-        for (int q = 0; q < ES_RES; ++q) cp_async16(d + k * STRIDE * 16 * ES_RES + 16 * q, gr + k * STRIDE * 16 * ES_RES + 16 * q);
-      }
+      for (int k = 0; k < CPL; ++k) copy_chunk<CE * ES_RES>(d + k * STRIDE * CE * ES_RES, gr + k * STRIDE * CE * ES_RES);
       if constexpr (BR != SRC_NONE) {
         const char* gb = g_br + row * pitch_br;
         uint8_t* db = my_ring_br + st * STAGE_BYTES;
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-#pragma unroll
-          for (int q = 0; q < ES_BR; ++q) cp_async16(db + k * STRIDE * 16 * ES_BR + 16 * q, gb + k * STRIDE * 16 * ES_BR + 16 * q);
-        }
+        for (int k = 0; k < CPL; ++k) copy_chunk<CE * ES_BR>(db + k * STRIDE * CE * ES_BR, gb + k * STRIDE * CE * ES_BR);
       }
     }
     cp_async_commit();
@@ -975,29 +1006,26 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   // stored piece-major ([float4 piece q of a chunk][chunk]): consecutive lanes then read consecutive 16-byte words,
   // free of bank conflicts
   for (int i = threadIdx.x; i < H; i += LNF_THREADS) {
-    const int si = (((i >> 2) & 3) * (H / 16) + (i >> 4)) * 4 + (i & 3);
+    const int si = ((((i % CE) >> 2) * (H / CE)) + i / CE) * 4 + (i & 3);
     if constexpr (RES_CS) v_rcs[si] = __ldg(p.res.col_scale + i * p.res.col_stride);
     if constexpr (BR_CS) v_bcs[si] = __ldg(p.br.col_scale + i * p.br.col_stride);
     if constexpr (OUT_CS) v_ocs[si] = __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));
   }
-  float2 gam[2][8], bet[2][8];
+  float2 gam[CPL][NP], bet[CPL][NP];
   if constexpr (OUT != O_NONE) {
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int e0 = (c_first + k * STRIDE) * 16;
-      float2 t[4];
-      load_vec8(p.gamma + e0, t);
+    for (int k = 0; k < CPL; ++k) {
+      const int e0 = (c_first + k * STRIDE) * CE;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) gam[k][i] = t[i];
-      load_vec8(p.gamma + e0 + 8, t);
+      for (int j = 0; j < CE / 8; ++j) {
+        float2 t[4];
+        load_vec8(p.gamma + e0 + 8 * j, t);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) gam[k][4 + i] = t[i];
-      load_vec8(p.beta + e0, t);
+        for (int i = 0; i < 4; ++i) gam[k][4 * j + i] = t[i];
+        load_vec8(p.beta + e0 + 8 * j, t);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) bet[k][i] = t[i];
-      load_vec8(p.beta + e0 + 8, t);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) bet[k][4 + i] = t[i];
+        for (int i = 0; i < 4; ++i) bet[k][4 * j + i] = t[i];
+      }
     }
   }
   ptx::pdl_wait();                                 // the previous kernel's outputs are complete and visible from here on
@@ -1037,53 +1065,52 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     if (++st == STAGES) st = 0;
 
     // ---- r = sum of the dequantized addends; running row sum
-    float2 x[2][8];
+    float2 x[CPL][NP];
     float2 s2 = f2(0.f);
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < CPL; ++k) {
       {
         if constexpr (RES == SRC_I8) {
-          q8x16_to_f2<F8>(*reinterpret_cast<const uint4*>(src + k * STRIDE * 16), x[k]);
+          ring_q8<CE, F8>(src + k * STRIDE * CE, x[k]);
           if constexpr (RSC == RS_COL) {
-            float2 sc[8];
-            lds_vec16<H / 16>(v_rcs + (c_first + k * STRIDE) * 4, sc);
+            float2 sc[NP];
+            lds_vec<H / CE, CE>(v_rcs + (c_first + k * STRIDE) * 4, sc);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[k][i] = __fmul2_rn(x[k][i], sc[i]);
+            for (int i = 0; i < NP; ++i) x[k][i] = __fmul2_rn(x[k][i], sc[i]);
           } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[k][i] = __fmul2_rn(x[k][i], f2(rs_res));
+            for (int i = 0; i < NP; ++i) x[k][i] = __fmul2_rn(x[k][i], f2(rs_res));
           }
         } else {
-          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src + k * STRIDE * 32), x[k]);
-          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src + k * STRIDE * 32 + 16), x[k] + 4);
+          ring_fp<CE, BF>(src + k * STRIDE * CE * 2, x[k]);
         }
         if constexpr (BR == SRC_I8) {
-          float2 b[8], sc[8];
-          q8x16_to_f2<F8>(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 16), b);
-          lds_vec16<H / 16>(v_bcs + (c_first + k * STRIDE) * 4, sc);
+          float2 b[NP], sc[NP];
+          ring_q8<CE, F8>(src_br + k * STRIDE * CE, b);
+          lds_vec<H / CE, CE>(v_bcs + (c_first + k * STRIDE) * 4, sc);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
+          for (int i = 0; i < NP; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
         }
         if constexpr (BR == SRC_FP) {
-          float2 b[8];
-          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 32), b);
-          fpx8_to_f2<BF>(*reinterpret_cast<const uint4*>(src_br + k * STRIDE * 32 + 16), b + 4);
+          float2 b[NP];
+          ring_fp<CE, BF>(src_br + k * STRIDE * CE * 2, b);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[k][i] = __fadd2_rn(x[k][i], b[i]);
+          for (int i = 0; i < NP; ++i) x[k][i] = __fadd2_rn(x[k][i], b[i]);
         }
         if constexpr (FPOUT) {
           // the FP residual stream carries the ROUNDED sum; normalise what is stored
-          uint32_t w[8];
+          uint32_t w[NP];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
-          char* dst = reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + (c_first + k * STRIDE) * 16) * 2;
-          st_global16(dst, w[0], w[1], w[2], w[3]);
-          st_global16(dst + 16, w[4], w[5], w[6], w[7]);
-          fpx8_to_f2<BF>(make_uint4(w[0], w[1], w[2], w[3]), x[k]);
-          fpx8_to_f2<BF>(make_uint4(w[4], w[5], w[6], w[7]), x[k] + 4);
+          for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
+          char* dst = reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + (c_first + k * STRIDE) * CE) * 2;
+#pragma unroll
+          for (int j = 0; j < CE / 8; ++j) {
+            st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            fpx8_to_f2<BF>(make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]), x[k] + 4 * j);
+          }
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) s2 = __fadd2_rn(s2, x[k][i]);
+        for (int i = 0; i < NP; ++i) s2 = __fadd2_rn(s2, x[k][i]);
       }
     }
     if constexpr (OUT == O_NONE) continue;
@@ -1102,9 +1129,9 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     float2 q2 = f2(0.f);
     const float2 nm = f2(-mean);
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < CPL; ++k) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { x[k][i] = __fadd2_rn(x[k][i], nm); q2 = __ffma2_rn(x[k][i], x[k][i], q2); }
+      for (int i = 0; i < NP; ++i) { x[k][i] = __fadd2_rn(x[k][i], nm); q2 = __ffma2_rn(x[k][i], x[k][i], q2); }
     }
     float q = warp_sum(q2.x + q2.y);
     if constexpr (WPR > 1) {
@@ -1120,9 +1147,9 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     float amax = 0.f;
     const float2 r2 = f2(rstd);
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < CPL; ++k) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < NP; ++i) {
         x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(gam[k][i], r2), bet[k][i]);
         if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fmaxf(fabsf(x[k][i].x), fabsf(x[k][i].y)));
       }
@@ -1144,10 +1171,10 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
       if (wr == 0 && lane == 0) p.out_scale[row] = sc;
       {
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          uint32_t w[4];
+        for (int k = 0; k < CPL; ++k) {
+          uint32_t w[CE / 4];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
+          for (int g = 0; g < CE / 4; ++g) {
             if constexpr (F8) {
               const float2 a = __fmul2_rn(x[k][2 * g], inv2), b = __fmul2_rn(x[k][2 * g + 1], inv2);
               w[g] = ptx::f32x4_to_e4m3x4(a.x, a.y, b.x, b.y);
@@ -1156,19 +1183,21 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
               w[g] = pack_low_bytes(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(b.x), __float_as_uint(b.y));
             }
           }
-          st_global16(reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * 16, w[0], w[1], w[2], w[3]);
+          char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
+          if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
+          else st_global8(dst, w[0], w[1]);
         }
       }
     } else if constexpr (OUT == O_STATIC) {
       // Eq. 4 / 5: calibrated per-feature or static scale; saturating; true division as the definition has it
       {
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          float2 sc[8];
-          lds_vec16<H / 16>(v_ocs + (c_first + k * STRIDE) * 4, sc);
-          uint32_t w[4];
+        for (int k = 0; k < CPL; ++k) {
+          float2 sc[NP];
+          lds_vec<H / CE, CE>(v_ocs + (c_first + k * STRIDE) * 4, sc);
+          uint32_t w[CE / 4];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
+          for (int g = 0; g < CE / 4; ++g) {
             if constexpr (F8) {
               w[g] = ptx::f32x4_to_e4m3x4(x[k][2 * g].x / sc[2 * g].x, x[k][2 * g].y / sc[2 * g].y, x[k][2 * g + 1].x / sc[2 * g + 1].x,
                                           x[k][2 * g + 1].y / sc[2 * g + 1].y);
@@ -1180,19 +1209,21 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
             const float d = fminf(fmaxf(x[k][2 * g + 1].y / sc[2 * g + 1].y, -127.f), 127.f) + MAGIC;
             w[g] = pack_low_bytes(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d));
           }
-          st_global16(reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * 16, w[0], w[1], w[2], w[3]);
+          char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
+          if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
+          else st_global8(dst, w[0], w[1]);
         }
       }
     } else {
       {
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          uint32_t w[8];
+        for (int k = 0; k < CPL; ++k) {
+          uint32_t w[NP];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
-          char* dst = reinterpret_cast<char*>(p.out) + (row * p.out_ld + (c_first + k * STRIDE) * 16) * 2;
-          st_global16(dst, w[0], w[1], w[2], w[3]);
-          st_global16(dst + 16, w[4], w[5], w[6], w[7]);
+          for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
+          char* dst = reinterpret_cast<char*>(p.out) + (row * p.out_ld + (c_first + k * STRIDE) * CE) * 2;
+#pragma unroll
+          for (int j = 0; j < CE / 8; ++j) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         }
       }
     }
@@ -1200,15 +1231,15 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   cp_async_wait<0>();
 }
 
-template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8>
+template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
 static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream) {
-  constexpr int H = 1024 * WPR, SLOTS = 8 / WPR;
+  constexpr int H = (GEO == 0 ? 1024 : 768) * WPR, SLOTS = 8 / WPR;
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2, ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
   constexpr size_t STAGE = (size_t)SLOTS * H * (ES_RES + ES_BR);
   constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0));
   constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC);
   const size_t smem = (size_t)stages * STAGE + VEC;
-  auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8>;
+  auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8, GEO>;
   static bool configured = false;   // per instantiation
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
@@ -1233,17 +1264,18 @@ static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream)
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, bool F8>
 static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) {
   switch (p.H) {
-    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8>(h, p, s);
-    case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2, F8>(h, p, s);
-    case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4, F8>(h, p, s);
-    default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8, F8>(h, p, s);
+    case 768: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 1>(h, p, s);
+    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 0>(h, p, s);
+    case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2, F8, 0>(h, p, s);
+    case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4, F8, 0>(h, p, s);
+    default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8, F8, 0>(h, p, s);
   }
 }
 
 // The combinations the layer forward produces on rows of 1024 * {1, 2, 4, 8} elements.
 static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* taken) {
   *taken = false;
-  if (!(p.H == 1024 || p.H == 2048 || p.H == 4096 || p.H == 8192) || p.ex.data || p.token_ids) return HERO_OK;
+  if (!(p.H == 768 || p.H == 1024 || p.H == 2048 || p.H == 4096 || p.H == 8192) || p.ex.data || p.token_ids) return HERO_OK;
   // one 8-bit payload across the call (INT8, or e4m3 for the FP8 variant); a mix takes the generic kernel
   int q8t = -1;
   auto q8_ok = [&](bool used, int dt) { if (!used || !is_q8(dt)) return true; if (q8t < 0) q8t = dt; return q8t == dt; };

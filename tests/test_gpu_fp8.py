@@ -39,7 +39,7 @@ def assert_f8_close(got, want, frac, what):
     assert f <= max(frac, 1.0 / want.size), "%s: %.3g of the elements differ" % (what, f)
 
 
-@pytest.mark.parametrize("M,H", [(7, 768), (300, 1024), (65, 4096)])
+@pytest.mark.parametrize("M,H", [(7, 768), (300, 1024), (65, 4096), (300, 768), (9, 1280)])
 def test_ln_quant_fp16_to_e4m3_twq_and_static(h, M, H):
     g = W.rng(11, M + H)
     x = g.standard_normal((M, H)) * 2

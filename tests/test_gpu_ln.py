@@ -69,7 +69,7 @@ def _compare(res, want, want_r, out_spec):
         assert np.mean(d != 0) < 1e-3 and rel_err(res["fp_out"], want_r.data) < 8e-3
 
 
-@pytest.mark.parametrize("M,H", [(128, 768), (37, 1024), (1, 768), (300, 4096), (65, 8192), (129, 80), (7, 16384), (40, 2048), (33, 5120)])
+@pytest.mark.parametrize("M,H", [(128, 768), (37, 1024), (1, 768), (2100, 768), (300, 4096), (65, 8192), (129, 80), (7, 16384), (40, 2048), (33, 5120)])
 def test_plain_fp16_to_twq(h, M, H):
     x, gamma, beta = W.ln_case(M, H)
     spec = O.OutSpec("twq")
@@ -98,8 +98,9 @@ def test_residual_int8_twq_plus_int8_fwq(h, out_kind, H):
 
 @pytest.mark.parametrize("res_kind,br_kind", [("i8_twq", "f16"), ("f16", "f16"), ("bf16", "i8_fwq"), ("i8_fwq", "i8_fwq"),
                                               ("i8_sq", "bf16")])
-def test_mixed_input_types(h, res_kind, br_kind):
-    M, H = 96, 1024
+@pytest.mark.parametrize("H", [1024, 768])        # two chunks of 16 elements per lane / three chunks of 8
+def test_mixed_input_types(h, res_kind, br_kind, H):
+    M = 96
     g = W.rng(2, 99)
     x, gamma, beta = W.ln_case(M, H)
 
@@ -121,8 +122,9 @@ def test_mixed_input_types(h, res_kind, br_kind):
 
 
 @pytest.mark.parametrize("fp", ["f16", "bf16"])
-def test_pre_ln_dual_output_and_bare_add(h, fp):
-    M, H = 150, 4096
+@pytest.mark.parametrize("H", [4096, 768])
+def test_pre_ln_dual_output_and_bare_add(h, fp, H):
+    M = 150
     g = W.rng(2, 123)
     hres = O.fp_tensor(g.standard_normal((M, H)), fp)
     br = O.QT("i8", g.integers(-127, 128, (M, H), dtype=np.int8),
