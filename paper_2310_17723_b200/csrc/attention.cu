@@ -556,8 +556,8 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
+  if (a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory (INT8 or e4m3)
   if (f8_in) return a->dh == 64 ? launch_attn<64, false, true>(h, a, p, s) : launch_attn<128, false, true>(h, a, p, s);
-  if (a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory
   if (rowmax) return a->dh == 64 ? launch_attn<64, true>(h, a, p, s) : launch_attn<128, true>(h, a, p, s);
   if (a->dh == 64) return launch_attn<64, false>(h, a, p, s);
   return launch_attn<128, false>(h, a, p, s);

@@ -46,7 +46,7 @@ struct AttnResCfg {
 // columns.  Every softmax warp takes DH / 4 columns of its 32 rows; `osc` is the tile's per-column factor
 // s_p s_v / S_attn[j] (s_p s_v alone for an FP output) staged in shared memory.  Kept out of line: it runs once per
 // tile and its registers stay out of the sweeps' allocation.
-template <int DH>
+template <int DH, bool F8>
 __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, uint64_t* o_full, uint64_t* o_empty,
                                           uint32_t parity, int cq, int lane, long long pend_row, int pend_col,
                                           const float* osc, float rowf, bool& ok) {
@@ -65,7 +65,22 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
   if (pend_row >= 0) {
     const int gcol = pend_col + cq * CW;
     const float4* o4 = reinterpret_cast<const float4*>(osc + cq * CW);
-    if (p.out_dt == HERO_I8) {
+    auto acc = [&](int c) -> float { if constexpr (F8) return __uint_as_float(r[c]); else return (float)(int)r[c]; };
+    if (p.out_dt == HERO_F8) {
+      // e4m3 X_attn (FP8 variant): the conversion saturates and rounds to nearest even
+      int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pend_row * p.out_ld + gcol;
+#pragma unroll
+      for (int g = 0; g < CW / 16; ++g) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float4 sc = o4[4 * g + k];
+          const int c = 16 * g + 4 * k;
+          w[k] = ptx::f32x4_to_e4m3x4(acc(c) * rowf * sc.x, acc(c + 1) * rowf * sc.y, acc(c + 2) * rowf * sc.z, acc(c + 3) * rowf * sc.w);
+        }
+        st_g16(dst + 16 * g, w[0], w[1], w[2], w[3]);
+      }
+    } else if (p.out_dt == HERO_I8) {
       int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pend_row * p.out_ld + gcol;
 #pragma unroll
       for (int g = 0; g < CW / 16; ++g) {
@@ -88,7 +103,7 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
       for (int g = 0; g < CW / 8; ++g) {
         float v[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) v[e] = (float)(int)r[8 * g + e] * rowf * p.pv_scale;
+        for (int e = 0; e < 8; ++e) v[e] = acc(8 * g + e) * rowf * p.pv_scale;
         st_g16(dst + 8 * g, fp2(v[0], v[1], p.out_dt), fp2(v[2], v[3], p.out_dt), fp2(v[4], v[5], p.out_dt),
                fp2(v[6], v[7], p.out_dt));
       }
@@ -99,7 +114,9 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
 // ROWMAX: the long-sequence-robust P quantizer (not in the paper): P~_u8 = Round(255 * 2^(t - m_row)) with the row sum
 // l of the un-quantized 2^(t - m_row) kept in FP32 and divided out in the epilogue.  Sweep 1 then only finds the row
 // maximum (integer compares, nothing written back), sweep 2 does the one exponential per score.
-template <int DH, bool ROWMAX>
+// F8: e4m3 Q, K, V and an e4m3 P (the FP8 variant; static P quantizer only): kind::f8f6f4 products, FP32 scores and
+// accumulator in tensor memory, P formed by the saturating conversion instead of round + clip.
+template <int DH, bool ROWMAX, bool F8>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnParams p) {
@@ -202,9 +219,12 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
         const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
 #pragma unroll
-        for (int k = 0; k < DH / 32; ++k)
-          ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                       ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+        for (int k = 0; k < DH / 32; ++k) {
+          if constexpr (F8) ptx::umma_f8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                                         ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+          else ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
+                            ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+        }
         ptx::umma_commit(&k_empty[ks]);
         ptx::umma_commit(&s_full[j]);
         ++kcnt; used ^= 1u << j;
@@ -251,9 +271,12 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
           const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
 #pragma unroll
-          for (int k = 0; k < ATT_BN / 32; ++k)
-            ptx::umma_i8(tmem_base + RES_O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                         ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
+          for (int k = 0; k < ATT_BN / 32; ++k) {
+            if constexpr (F8) ptx::umma_f8(tmem_base + RES_O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
+                                           ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
+            else ptx::umma_i8(tmem_base + RES_O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
+                              ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
+          }
           ptx::umma_commit(&v_empty[vs]);
           ptx::umma_commit(&p_empty[pb]);
           ++vcnt; ++pcnt;
@@ -289,7 +312,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     bool pend = false;
 
     auto epilogue = [&]() {
-      res_epilogue<DH>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
+      res_epilogue<DH, F8>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
                        osc_s + quarter * 256 + ((wcnt - 1) & 1) * 128, pend_rowf, ok);
       pend = false;
     };
@@ -305,14 +328,14 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       const int q = q0 + r_loc;
       const bool row_ok = q < p.S;
       float osc_raw = 1.f;                                   // this thread's S_attn[j], turned into a factor further down
-      if (p.out_dt == HERO_I8 && cq * 32 + lane < DH)
+      if (is_q8(p.out_dt) && cq * 32 + lane < DH)
         osc_raw = __ldg(p.out_scale + (long long)(col0 + cq * 32 + lane) * p.out_scale_stride);
       if (nkv == 0) {
         // every key masked: the rows are zero, no tensor work
         if (cq * 32 < DH && row_ok) {
           const long long grow = (long long)(row_base + q);
           const int gcol = col0 + cq * 32;
-          const int es = p.out_dt == HERO_I8 ? 1 : 2;
+          const int es = is_q8(p.out_dt) ? 1 : 2;
           uint8_t* dst = reinterpret_cast<uint8_t*>(p.out) + (grow * p.out_ld + gcol) * es;
           for (int g = 0; g < 2 * es; ++g) st_g16(dst + 16 * g, 0u, 0u, 0u, 0u);
         }
@@ -375,17 +398,28 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
               if (nvalid < 16) {
                 // masked keys: a score far below every real one (|t| < 2^21) turns into e = 0 by itself
 #pragma unroll
-                for (int e = 0; e < 16; ++e) if (e >= nvalid) r[e] = (uint32_t)(-(1 << 21));
+                for (int e = 0; e < 16; ++e) if (e >= nvalid) r[e] = F8 ? __float_as_uint(-1.0e30f) : (uint32_t)(-(1 << 21));
               }
-              int i0 = max((int)r[0], (int)r[1]), i1 = max((int)r[2], (int)r[3]);
+              if constexpr (F8) {
+                float f0 = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), f1 = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
 #pragma unroll
-              for (int e = 4; e < 16; e += 4) { i0 = max(i0, max((int)r[e], (int)r[e + 1])); i1 = max(i1, max((int)r[e + 2], (int)r[e + 3])); }
-              mp = (float)max(i0, i1) * c2;
+                for (int e = 4; e < 16; e += 4) {
+                  f0 = fmaxf(f0, fmaxf(__uint_as_float(r[e]), __uint_as_float(r[e + 1])));
+                  f1 = fmaxf(f1, fmaxf(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])));
+                }
+                mp = fmaxf(f0, f1) * c2;
+              } else {
+                int i0 = max((int)r[0], (int)r[1]), i1 = max((int)r[2], (int)r[3]);
+#pragma unroll
+                for (int e = 4; e < 16; e += 4) { i0 = max(i0, max((int)r[e], (int)r[e + 1])); i1 = max(i1, max((int)r[e + 2], (int)r[e + 3])); }
+                mp = (float)max(i0, i1) * c2;
+              }
               float2 acc2 = make_float2(0.f, 0.f);
               const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-mp, -mp);
 #pragma unroll
               for (int e = 0; e < 16; e += 2) {
-                const float2 f = make_float2((float)(int)r[e], (float)(int)r[e + 1]);
+                const float2 f = F8 ? make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1]))
+                                    : make_float2((float)(int)r[e], (float)(int)r[e + 1]);
                 const float2 tt = __ffma2_rn(f, c22, nm2);
                 const float2 ev = make_float2(ex2f(tt.x), ex2f(tt.y));
                 acc2 = __fadd2_rn(acc2, ev);
@@ -486,7 +520,16 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             const float f = mp > -INFINITY ? ex2f(mp - m) * pscale : 0.f;
             const float2 f2v = make_float2(f, f), rm2 = make_float2(ATT_MAGIC, ATT_MAGIC);
             uint32_t w[4];
-            if (f <= 255.25f) {
+            if constexpr (F8) {
+              // P_f8 = e4m3(e f): the conversion saturates at 448 (s_p = max P / 448)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int e = 4 * k;
+                const float2 a = __fmul2_rn(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), f2v);
+                const float2 c = __fmul2_rn(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])), f2v);
+                w[k] = ptx::f32x4_to_e4m3x4(a.x, a.y, c.x, c.y);
+              }
+            } else if (f <= 255.25f) {
               // e <= 1 in every piece, so e f cannot round above 255: no clip needed
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
@@ -537,7 +580,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <int DH, bool ROWMAX>
+template <int DH, bool ROWMAX, bool F8>
 static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
   using Cfg = AttnResCfg<DH>;
   const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
@@ -546,9 +589,14 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
   if ((st = make_tmap_2d(h, &tq, a->q, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BM, DH)) != HERO_OK) return st;
   if ((st = make_tmap_2d(h, &tk, a->k, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BN, DH)) != HERO_OK) return st;
   if ((st = make_tmap_2d(h, &tv, a->v, 1, false, false, rows, cols, (uint64_t)a->ld, DH, ATT_BN, DH)) != HERO_OK) return st;
-  p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN);
-  p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);
-  auto kern = attn_int8_resident_kernel<DH, ROWMAX>;
+  if (F8) {
+    p.idesc_qk = ptx::make_idesc(1, 0, 0, 0, 0, ATT_BM, ATT_BN);   // E4M3 x E4M3 -> F32, both K-major
+    p.idesc_pv = ptx::make_idesc(1, 0, 0, 0, 1, ATT_BM, DH);       // E4M3 x E4M3 -> F32, V is MN-major
+  } else {
+    p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN);   // S8 x S8 -> S32
+    p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);       // U8 x S8 -> S32
+  }
+  auto kern = attn_int8_resident_kernel<DH, ROWMAX, F8>;
   static bool configured = false;
   if (!configured) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
@@ -565,12 +613,16 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
 }
 
 hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
-  if (a->p_mode == HERO_P_ROWMAX) {
-    if (a->dh == 64) return launch_resident<64, true>(h, a, p, stream);
-    return launch_resident<128, true>(h, a, p, stream);
+  if (a->dtype == HERO_F8) {                               // static P quantizer only (checked by the caller)
+    if (a->dh == 64) return launch_resident<64, false, true>(h, a, p, stream);
+    return launch_resident<128, false, true>(h, a, p, stream);
   }
-  if (a->dh == 64) return launch_resident<64, false>(h, a, p, stream);
-  return launch_resident<128, false>(h, a, p, stream);
+  if (a->p_mode == HERO_P_ROWMAX) {
+    if (a->dh == 64) return launch_resident<64, true, false>(h, a, p, stream);
+    return launch_resident<128, true, false>(h, a, p, stream);
+  }
+  if (a->dh == 64) return launch_resident<64, false, false>(h, a, p, stream);
+  return launch_resident<128, false, false>(h, a, p, stream);
 }
 
 }  // namespace hero

@@ -141,6 +141,15 @@ def test_decode_step_equals_causal_prefill_row_on_device(h):
     assert rel_err(a, b_) < 2e-3
 
 
+def test_decode_attention_clamps_lengths_beyond_the_launch_bound(h):
+    # len[b] > max_len (a caller's mistake) is treated as max_len: nothing outside the sized buffers is touched
+    q, kc, vc, sc = _case(2, 96, 2, 64, 11)
+    spec = O.OutSpec("fp", dtype="f16")
+    want, _, _ = _run(h, q, kc, vc, [64, 10], 2, 64, sc, 1.0 / 255, spec, max_len=64)
+    got, _, _ = _run(h, q, kc, vc, [90, 10], 2, 64, sc, 1.0 / 255, spec, max_len=64)
+    assert np.array_equal(got, want)
+
+
 def test_decode_attention_refusals(h):
     q, kc, vc, sc = _case(2, 64, 2, 64, 3)
     tq, tk, tv, tl = dev(q), dev(kc), dev(vc), dev(np.asarray([3, 4], np.int32))
