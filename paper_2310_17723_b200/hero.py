@@ -100,7 +100,8 @@ HIST_BINS = 2048
 EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero_launch_count",
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_layer_forward_host_async", "hero_profile_begin",
-           "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram")
+           "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram",
+           "hero_int8_decode_attention", "hero_layer_decode")
 
 _lib = None
 
