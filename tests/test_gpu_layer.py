@@ -158,12 +158,17 @@ def test_rowmax_p_quantizer_keeps_the_mass_of_flat_long_rows(h):
     assert rel_err(outs["rowmax"], ref) < 2e-3
 
 
-@pytest.mark.parametrize("preset", ["M1", "M2", "FP"])
+# "ATTN_LN_FP": attention and the LN outputs in FP (so QKV and FC1 run FP), attention-output linear and FC2 INT8: the
+# comparison variant of the GPT prefill configuration
+MODES = dict(OL.MODE_PRESETS, ATTN_LN_FP=dict(qkv="fp", attn="fp", attn_out="int8", fc1="fp", fc2="int8"))
+
+
+@pytest.mark.parametrize("preset", ["M1", "M2", "FP", "ATTN_LN_FP"])
 @pytest.mark.parametrize("arch", ["post_ln", "pre_ln"])
 def test_mixed_precision_presets(h, preset, arch):
     # Table 1: modules switched to FP16 keep FP operands; every INT8 <-> FP hand-off happens in a producer's epilogue
     shape = W.tiny_shape(**SMALL, arch=arch, mask="causal" if arch == "pre_ln" else "none", eps=1e-5, n_outlier=2)
-    spec, Lp, x_in = _build(shape, 25, mode=dict(OL.MODE_PRESETS[preset]), gran_out="fp" if preset == "FP" else "twq")
+    spec, Lp, x_in = _build(shape, 25, mode=dict(MODES[preset]), gran_out="fp" if preset == "FP" else "twq")
     T = OL.layer_forward(Lp, x_in)
     out, sc, launches = _run_layer(h, spec, Lp, x_in)
     assert launches == (8 if arch == "pre_ln" else 7)
