@@ -282,14 +282,21 @@ extern "C" hero_status hero_layer_forward_host_async(hero_handle* h, const hero_
     return t.gran == HERO_GRAN_TWQ ? (size_t)t.rows : 0;   // calibrated FWQ / SQ scales already live on the device
   };
   // host -> device: the activation payload and, for a token-wise input, its per-row scales
-  HERO_CUDA(cudaMemcpy2DAsync(in_dev->data, in_dev->ld * ies, in_host->data, in_host->ld * ies, in_dev->cols * ies,
-                              in_dev->rows, cudaMemcpyHostToDevice, s));
+  // contiguous on both sides: one linear copy (the pitched form is kept for strided views)
+  if (in_dev->ld == in_dev->cols && in_host->ld == in_host->cols)
+    HERO_CUDA(cudaMemcpyAsync(in_dev->data, in_host->data, (size_t)in_dev->rows * in_dev->cols * ies, cudaMemcpyHostToDevice, s));
+  else
+    HERO_CUDA(cudaMemcpy2DAsync(in_dev->data, in_dev->ld * ies, in_host->data, in_host->ld * ies, in_dev->cols * ies,
+                                in_dev->rows, cudaMemcpyHostToDevice, s));
   if (scale_len(*in_dev))
     HERO_CUDA(cudaMemcpyAsync(in_dev->scale, in_host->scale, scale_len(*in_dev) * sizeof(float), cudaMemcpyHostToDevice, s));
   hero_status st = hero_layer_forward(h, d, in_dev, nullptr, out_dev, workspace, workspace_bytes, stream);
   if (st != HERO_OK) return st;
-  HERO_CUDA(cudaMemcpy2DAsync(out_host->data, out_host->ld * oes, out_dev->data, out_dev->ld * oes, out_dev->cols * oes,
-                              out_dev->rows, cudaMemcpyDeviceToHost, s));
+  if (out_dev->ld == out_dev->cols && out_host->ld == out_host->cols)
+    HERO_CUDA(cudaMemcpyAsync(out_host->data, out_dev->data, (size_t)out_dev->rows * out_dev->cols * oes, cudaMemcpyDeviceToHost, s));
+  else
+    HERO_CUDA(cudaMemcpy2DAsync(out_host->data, out_host->ld * oes, out_dev->data, out_dev->ld * oes, out_dev->cols * oes,
+                                out_dev->rows, cudaMemcpyDeviceToHost, s));
   if (scale_len(*out_dev))
     HERO_CUDA(cudaMemcpyAsync(out_host->scale, out_dev->scale, scale_len(*out_dev) * sizeof(float), cudaMemcpyDeviceToHost, s));
   return HERO_OK;
