@@ -139,7 +139,9 @@ hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* a, void* st
  *   A    : [M, K] I8 (gran TWQ -> row scale applied; NONE / FWQ / SQ -> none: a feature-wise or
  *          static input scale must already be folded into W's rows, Eq. 23 / 32), or F16 / BF16
  *          for a module left in FP mode (then W has the same type and w_scale is ignored).
- *   W    : device [N][K], K contiguous, leading dimension ldw; same element type as A.
+ *   W    : device [N][K], K contiguous, leading dimension ldw; same element type as A.  W is a constant of the model:
+ *          kernels may fetch it before earlier work on the stream has completed, so it must not be written by work
+ *          still in flight when the call is made (hero_quantize_weight takes care of this for its own outputs).
  *   out  : [M, N].  A TWQ output is refused (HERO_ERR_UNSUPPORTED): the paper keeps the row
  *          reduction out of GEMM epilogues (Sec. 2.1).
  * K must be a multiple of 16 bytes of elements and N a multiple of 16; M is arbitrary.

@@ -1,4 +1,6 @@
 // Handle life cycle, error text, tensor-map construction, Table 1 presets.
+#include <mutex>
+#include <unordered_set>
 #include "common.cuh"
 
 namespace hero {
@@ -10,6 +12,18 @@ void set_error(const char* fmt, ...) {
   va_start(ap, fmt);
   vsnprintf(g_err, sizeof(g_err), fmt, ap);
   va_end(ap);
+}
+
+// streams on which a library call has just written model constants (see launch_dependent)
+static std::mutex g_fence_mutex;
+static std::unordered_set<cudaStream_t> g_fenced;
+void pdl_fence_stream(cudaStream_t s) {
+  std::lock_guard<std::mutex> lock(g_fence_mutex);
+  g_fenced.insert(s);
+}
+bool pdl_take_fence(cudaStream_t s) {
+  std::lock_guard<std::mutex> lock(g_fence_mutex);
+  return g_fenced.erase(s) != 0;
 }
 
 hero_status cuda_fail(cudaError_t e, const char* what) {

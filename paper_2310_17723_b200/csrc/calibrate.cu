@@ -234,6 +234,7 @@ extern "C" hero_status hero_quantize_weight(hero_handle* h, const float* W, int6
     HERO_CUDA(launch_dependent(quantize_weight_kernel, dim3((unsigned)N), dim3(256), 0, s, W, (long long)ldw, (int)N, (int)K,
                                in_scale, out_scale, bias, Wq, (long long)ldq, w_scale, bias_out));
   }
+  pdl_fence_stream(s);   // Wq, w_scale and bias_out are model constants to whatever runs next on this stream
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
 }

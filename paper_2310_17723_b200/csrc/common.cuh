@@ -84,6 +84,13 @@ struct LaunchScope {
 // blocks in griddepcontrol.wait until that kernel has completed and its writes are visible.  Every kernel of the
 // library executes griddepcontrol.launch_dependents first thing and griddepcontrol.wait before its first global
 // memory access, so launch latency and ramp-up overlap the predecessor's tail and nothing else changes.
+//
+// Model constants (weight matrices) may be fetched BEFORE the dependency wait: they are not produced by the layer's own
+// kernels.  A library call that writes such constants on a stream (hero_quantize_weight) therefore fences the stream:
+// the next launch on it is an ordinary, fully serialised one, and with it everything launched after.
+void pdl_fence_stream(cudaStream_t s);     // the next launch on `s` must not start before earlier work has completed
+bool pdl_take_fence(cudaStream_t s);       // true once after pdl_fence_stream(s)
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
@@ -91,7 +98,7 @@ inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 bloc
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = 1;
+  cfg.attrs = at; cfg.numAttrs = pdl_take_fence(s) ? 0 : 1;
   return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 

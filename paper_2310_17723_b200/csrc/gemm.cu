@@ -327,22 +327,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   ptx::pdl_launch_dependents();
-  ptx::pdl_wait();                                       // the previous kernel's outputs are complete and visible from here on
 
   if (warp == TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const int kelems = GEMM_BK_BYTES / p.elem_bytes;
       int stage = 0; uint32_t phase = 0; bool ok = true;
+      // The weights are constants of the model: the W tiles of the first tile's first stages are requested before the
+      // dependency wait, the activation tiles after it (both complete the same barrier).
+      int pre = 0;
+      if ((int)blockIdx.x < num_tiles) {
+        int mt, nt; tile_coords(blockIdx.x, p.num_m_tiles, p.num_n_tiles, mt, nt);
+        pre = min(p.num_kb, STAGES);
+        for (int kb = 0; kb < pre; ++kb) {
+          ptx::mbar_expect_tx(&full[kb], Cfg::STAGE_BYTES);
+          ptx::tma_load_2d(tiles + kb * Cfg::STAGE_BYTES + Cfg::A_BYTES, &tmW, kb * kelems, nt * BN, &full[kb]);
+        }
+      }
+      ptx::pdl_wait();                                   // the previous kernel's outputs are complete and visible from here on
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
         for (int kb = 0; kb < p.num_kb; ++kb) {
-          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x100 | stage)) { ok = false; break; }
+          const bool early = t == (int)blockIdx.x && kb < pre;   // barrier armed and W requested above
+          if (!early && !ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x100 | stage)) { ok = false; break; }
           uint8_t* a_dst = tiles + stage * Cfg::STAGE_BYTES;
           uint8_t* b_dst = a_dst + Cfg::A_BYTES;
-          ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
+          if (!early) ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
           ptx::tma_load_2d(a_dst, &tmA, kb * kelems, mt * GEMM_BM, &full[stage]);
-          ptx::tma_load_2d(b_dst, &tmW, kb * kelems, nt * BN, &full[stage]);
+          if (!early) ptx::tma_load_2d(b_dst, &tmW, kb * kelems, nt * BN, &full[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -355,6 +367,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp == MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
+    ptx::pdl_wait();
     if (lane == 0) {
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
       int stage = 0; uint32_t phase = 0; bool ok = true;
@@ -388,6 +401,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-7)
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
+    ptx::pdl_wait();                                     // before this warp's first global access
     epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0);
   }
 
@@ -511,7 +525,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   ptx::pdl_launch_dependents();
-  ptx::pdl_wait();                                       // the previous kernel's outputs are complete and visible from here on
 
   if (warp == EW) {
     // ------------------------------------------------------------------ TMA producer (leader CTA only)
@@ -521,18 +534,34 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (lane == 0 && rank == 0) {
       const int kelems = GEMM_BK_BYTES / p.elem_bytes;
       int stage = 0; uint32_t phase = 0; bool ok = true;
+      // The weights are constants of the model: the W halves of the first tile's first stages are requested before the
+      // dependency wait, the activation halves after it (all complete the same barrier).
+      int pre = 0;
+      if (pair_id < num_tiles) {
+        int mt, nt; tile_coords(pair_id, p.num_m_tiles, p.num_n_tiles, mt, nt);
+        pre = min(p.num_kb, STAGES);
+        for (int kb = 0; kb < pre; ++kb) {
+          const uint32_t b_loc = ptx::smem_u32(tiles + kb * Cfg::STAGE_BYTES) + Cfg::A_BYTES;
+          const uint32_t bar = ptx::mapa(ptx::smem_u32(&full[kb]), 0);
+          ptx::mbar_expect_tx(&full[kb], 2 * Cfg::STAGE_BYTES);
+#pragma unroll
+          for (int r = 0; r < 2; ++r) ptx::tma_load_2d_pair(ptx::mapa(b_loc, r), &tmW, kb * kelems, nt * BN + r * (BN / 2), bar);
+        }
+      }
+      ptx::pdl_wait();                                   // the previous kernel's outputs are complete and visible from here on
       for (int t = pair_id; t < num_tiles && ok; t += num_pairs) {
         int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
         for (int kb = 0; kb < p.num_kb; ++kb) {
-          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x700 | stage)) { ok = false; break; }
+          const bool early = t == pair_id && kb < pre;   // barrier armed and W requested above
+          if (!early && !ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x700 | stage)) { ok = false; break; }
           const uint32_t a_loc = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
           const uint32_t b_loc = a_loc + Cfg::A_BYTES;
           const uint32_t bar = ptx::mapa(ptx::smem_u32(&full[stage]), 0);
-          ptx::mbar_expect_tx(&full[stage], 2 * Cfg::STAGE_BYTES);
+          if (!early) ptx::mbar_expect_tx(&full[stage], 2 * Cfg::STAGE_BYTES);
 #pragma unroll
           for (int r = 0; r < 2; ++r) {
             ptx::tma_load_2d_pair(ptx::mapa(a_loc, r), &tmA, kb * kelems, mt * 256 + r * GEMM_BM, bar);
-            ptx::tma_load_2d_pair(ptx::mapa(b_loc, r), &tmW, kb * kelems, nt * BN + r * (BN / 2), bar);
+            if (!early) ptx::tma_load_2d_pair(ptx::mapa(b_loc, r), &tmW, kb * kelems, nt * BN + r * (BN / 2), bar);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -545,6 +574,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncwarp();
   } else if (warp == EW + 1) {
     // ------------------------------------------------------------------ UMMA issuer (leader CTA only)
+    ptx::pdl_wait();
     if (lane == 0 && rank == 0) {
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
       int stage = 0; uint32_t phase = 0; bool ok = true;
@@ -576,6 +606,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     __syncwarp();
   } else {
+    ptx::pdl_wait();                                     // before this warp's first global access
     // ------------------------------------------------------------------ epilogue (warps 0 .. EW-1 of each CTA)
     epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM);
   }
