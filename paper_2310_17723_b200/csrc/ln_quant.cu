@@ -1318,6 +1318,18 @@ static hero_status try_wide(hero_handle* h, LnParams& p, cudaStream_t s, bool* t
   LNW_CASE(SRC_FP, RS_ROW, SRC_I8, O_STATIC, true)
   LNW_CASE(SRC_FP, RS_ROW, SRC_I8, O_NONE, true)      // closing residual add of a lone pre-LN layer
 #undef LNW_CASE
+  // modules left in FP16 / BF16 (Table 1): no 8-bit tensor in the call
+#define LNW_FP_CASE(B_, O_, F_)                                                                       \
+  if (res == SRC_FP && br == B_ && out == O_ && fpo == F_) {                                            \
+    *taken = true;                                                                                   \
+    return bf ? launch_wide_wpr<SRC_FP, RS_ROW, B_, O_, F_, true, false>(h, p, s)                       \
+              : launch_wide_wpr<SRC_FP, RS_ROW, B_, O_, F_, false, false>(h, p, s);                     \
+  }
+  LNW_FP_CASE(SRC_FP, O_FP, false)                    // post-LN: residual + branch -> FP
+  LNW_FP_CASE(SRC_NONE, O_FP, false)                  // pre-LN LN1 feeding an FP QKV
+  LNW_FP_CASE(SRC_FP, O_FP, true)                     // pre-LN: add + LN, new residual stream stored
+  LNW_FP_CASE(SRC_FP, O_NONE, true)                   // closing residual add
+#undef LNW_FP_CASE
   return HERO_OK;
 }
 
