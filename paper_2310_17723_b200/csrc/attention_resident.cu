@@ -444,7 +444,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       // ---- row maximum and sum across the four column groups
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
       st[cq * ATT_BM + r_loc] = make_float2(m, l);
-      if (cq * 32 + lane < DH) osc_s[quarter * 256 + (wcnt & 1) * 128 + cq * 32 + lane] = p.pv_scale / osc_raw;
+      if (cq * 32 + lane < DH) osc_s[quarter * 256 + (wcnt & 1) * 128 + cq * 32 + lane] = __fdividef(p.pv_scale, osc_raw);
       // the four warps that share these 32 rows (one per column group) meet; the other lane quarters are not involved
       asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter) : "memory");
       float pscale = 0.f;
@@ -467,7 +467,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           }
         }
         m = mf; l = lf;
-        pscale = l > 0.f ? p.inv_sp / l : 0.f;
+        pscale = l > 0.f ? __fdividef(p.inv_sp, l) : 0.f;   // 2 ulp: far below the rounding step of P
       }
 
       // ---- sweep 2: P_u8 = Round(e * 2^(m_piece - m) / (l s_p)), clipped to 255, into the UMMA operand tile
