@@ -720,7 +720,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams 
       q = 0.f;
       for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
     }
-    const float rstd = 1.0f / sqrtf(q / fH + p.eps);
+    const float rstd = rsqrtf(q / fH + p.eps);
 
     // ---- y = d * (rstd * gamma) + beta ; TWQ: row absmax in the same sweep
     float amax = 0.f;
@@ -756,8 +756,8 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams 
         amax = 0.f;
         for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
       }
-      const float sc = amax > 0.f ? amax / 127.0f : 1.0f;
-      const float2 inv2 = f2(1.0f / sc), mg2 = f2(MAGIC);
+      const float sc = amax > 0.f ? amax * (1.0f / 127.0f) : 1.0f;
+      const float2 inv2 = f2(__fdividef(1.0f, sc)), mg2 = f2(MAGIC);
       if (row_ok && wr == 0 && lane == 0) p.out_scale[row] = sc;
 #pragma unroll
       for (int k = 0; k < KMAX; ++k) {
@@ -1141,7 +1141,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 #pragma unroll
       for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
     }
-    const float rstd = 1.0f / sqrtf(q / fH + p.eps);
+    const float rstd = rsqrtf(q / fH + p.eps);   // 2 ulp: far below the rounding step of the output
 
     // ---- y = d * (rstd * gamma) + beta ; TWQ: row absmax in the same sweep
     float amax = 0.f;
@@ -1166,8 +1166,8 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 #pragma unroll
         for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
       }
-      const float sc = amax > 0.f ? amax / (F8 ? 448.0f : 127.0f) : 1.0f;
-      const float2 inv2 = f2(1.0f / sc), mg2 = f2(MAGIC);
+      const float sc = amax > 0.f ? amax * (F8 ? 1.0f / 448.0f : 1.0f / 127.0f) : 1.0f;   // within 1 ulp of the quotient
+      const float2 inv2 = f2(__fdividef(1.0f, sc)), mg2 = f2(MAGIC);
       if (wr == 0 && lane == 0) p.out_scale[row] = sc;
       {
 #pragma unroll
