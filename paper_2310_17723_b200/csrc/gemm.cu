@@ -51,6 +51,24 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mt
   nt = r / gsize;
 }
 
+// The same order walked tile by tile without integer divisions: the epilogue threads advance by the grid's stride and
+// read the coordinates off (group, r); only a last, shorter group of row-tiles needs a division.
+struct TileWalk {
+  int group, r, width, num_m;
+  __device__ __forceinline__ void init(int t, int num_m_, int num_n) {
+    num_m = num_m_; width = 16 * num_n; group = t / width; r = t - group * width;
+  }
+  __device__ __forceinline__ void advance(int stride) {
+    r += stride;
+    while (r >= width) { r -= width; ++group; }
+  }
+  __device__ __forceinline__ void coords(int& mt, int& nt) const {
+    const int first_m = group * 16, gsize = min(num_m - first_m, 16);
+    if (gsize == 16) { mt = first_m + (r & 15); nt = r >> 4; }
+    else { mt = first_m + r % gsize; nt = r / gsize; }
+  }
+};
+
 __device__ __forceinline__ void st32(void* p, const uint32_t (&w)[8]) {   // 256-bit store, 32-byte aligned
   asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
                "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
@@ -231,8 +249,13 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
   constexpr int NV = CH / 32;                // values per lane and vector
   float* epi_w = epi + warp * (2 * 3 * CH);
   float ncs[NV], nbias[NV], npost[NV], nrs = 1.0f;
-  auto fetch = [&](int t) {                  // issue the loads for tile t; the values are consumed one tile later
-    int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+  TileWalk walk;                             // stands at the tile whose vectors are fetched next
+  walk.init(first_tile, p.num_m_tiles, p.num_n_tiles);
+  int nmt = 0, nnt = 0;                      // its coordinates, consumed one tile later like the vectors
+  auto fetch = [&]() {                       // issue the loads for the walker's tile, then step on
+    int mt, nt; walk.coords(mt, nt);
+    nmt = mt; nnt = nt;
+    walk.advance(tile_stride);
     if constexpr (OUTK != OUT_I32) {
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
@@ -261,16 +284,16 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     }
   };
 
-  if (first_tile < num_tiles) fetch(first_tile);
+  if (first_tile < num_tiles) fetch();
   int it = 0;
   for (int t = first_tile; t < num_tiles; t += tile_stride, ++it) {
-    int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+    const int mt = nmt, nt = nnt;
     const int as = it & 1;
     const uint32_t aphase = (it >> 1) & 1;
     const int n0 = nt * BN;
     const float rs = nrs;
     publish(it);
-    if (t + tile_stride < num_tiles) fetch(t + tile_stride);
+    if (t + tile_stride < num_tiles) fetch();
     const float* e_cs = epi_w + (it & 1) * 3 * CH;
     const int m = mt * ROWS + row_off + quarter * 32 + lane;
     const bool row_ok = m < p.M;
