@@ -792,7 +792,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams 
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float xv = (i & 1) ? x[k][i >> 1].y : x[k][i >> 1].x;
-            const float v = fminf(fmaxf(xv / sc[i], -127.f), 127.f);
+            const float v = fminf(fmaxf(__fdividef(xv, sc[i]), -127.f), 127.f);   // 2 ulp: far below the rounding step
             u[i] = magic_bits(v + MAGIC);
           }
           st_global8(reinterpret_cast<char*>(p.out) + row * p.out_ld + c * 8, pack_low_bytes(u[0], u[1], u[2], u[3]),
@@ -1009,7 +1009,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     const int si = ((((i % CE) >> 2) * (H / CE)) + i / CE) * 4 + (i & 3);
     if constexpr (RES_CS) v_rcs[si] = __ldg(p.res.col_scale + i * p.res.col_stride);
     if constexpr (BR_CS) v_bcs[si] = __ldg(p.br.col_scale + i * p.br.col_stride);
-    if constexpr (OUT_CS) v_ocs[si] = __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));
+    if constexpr (OUT_CS) v_ocs[si] = 1.0f / __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));   // reciprocal, see the output stage
   }
   float2 gam[CPL][NP], bet[CPL][NP];
   if constexpr (OUT != O_NONE) {
@@ -1189,8 +1189,10 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
         }
       }
     } else if constexpr (OUT == O_STATIC) {
-      // Eq. 4 / 5: calibrated per-feature or static scale; saturating; true division as the definition has it
+      // Eq. 4 / 5: calibrated per-feature or static scale, saturating.  The staged vector holds the reciprocals (one true
+      // division per feature and CTA): the product is within one ulp of the quotient
       {
+        const float2 lo2 = f2(-127.f), hi2 = f2(127.f), mg2 = f2(MAGIC);
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
           float2 sc[NP];
@@ -1198,16 +1200,14 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
           uint32_t w[CE / 4];
 #pragma unroll
           for (int g = 0; g < CE / 4; ++g) {
+            const float2 a = __fmul2_rn(x[k][2 * g], sc[2 * g]), b = __fmul2_rn(x[k][2 * g + 1], sc[2 * g + 1]);
             if constexpr (F8) {
-              w[g] = ptx::f32x4_to_e4m3x4(x[k][2 * g].x / sc[2 * g].x, x[k][2 * g].y / sc[2 * g].y, x[k][2 * g + 1].x / sc[2 * g + 1].x,
-                                          x[k][2 * g + 1].y / sc[2 * g + 1].y);
-              continue;
+              w[g] = ptx::f32x4_to_e4m3x4(a.x, a.y, b.x, b.y);
+            } else {
+              const float a0 = fminf(fmaxf(a.x, lo2.x), hi2.x) + mg2.x, a1 = fminf(fmaxf(a.y, lo2.x), hi2.x) + mg2.x;
+              const float b0 = fminf(fmaxf(b.x, lo2.x), hi2.x) + mg2.x, b1 = fminf(fmaxf(b.y, lo2.x), hi2.x) + mg2.x;
+              w[g] = pack_low_bytes(__float_as_uint(a0), __float_as_uint(a1), __float_as_uint(b0), __float_as_uint(b1));
             }
-            const float a = fminf(fmaxf(x[k][2 * g].x / sc[2 * g].x, -127.f), 127.f) + MAGIC;
-            const float b = fminf(fmaxf(x[k][2 * g].y / sc[2 * g].y, -127.f), 127.f) + MAGIC;
-            const float c = fminf(fmaxf(x[k][2 * g + 1].x / sc[2 * g + 1].x, -127.f), 127.f) + MAGIC;
-            const float d = fminf(fmaxf(x[k][2 * g + 1].y / sc[2 * g + 1].y, -127.f), 127.f) + MAGIC;
-            w[g] = pack_low_bytes(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d));
           }
           char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
           if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);

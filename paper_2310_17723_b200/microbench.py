@@ -62,8 +62,9 @@ def _time(fn, n_buf, iters):
     return e0.elapsed_time(e1) / iters * 1e-3
 
 
-def bench_ln(h, M, H, kind, iters):
-    """kind 'f16': FP16 -> INT8 TWQ (entry flavour); 'i8': INT8 TWQ + INT8 FWQ -> INT8 TWQ (Eq. 19)."""
+def bench_ln(h, M, H, kind, iters, out_gran="twq"):
+    """kind 'f16': FP16 -> INT8 TWQ (entry flavour); 'i8': INT8 TWQ + INT8 FWQ -> INT8 TWQ (Eq. 19); out_gran 'fwq': the
+    output is quantized with a calibrated per-feature scale instead (Eq. 4)."""
     n = max(2, min(32, int(400e6 // (M * H * 3)) + 1))
     g, b = torch.ones(H, device="cuda"), torch.zeros(H, device="cuda")
     sc = torch.empty(M, device="cuda")
@@ -76,11 +77,13 @@ def bench_ln(h, M, H, kind, iters):
         xs = [torch.randint(-127, 128, (M, H), device="cuda", dtype=torch.int8) for _ in range(n)]
         ys = [torch.randint(-127, 128, (M, H), device="cuda", dtype=torch.int8) for _ in range(n)]
         ins = [(hero.tensor(x, "twq", rs), hero.tensor(y, "fwq", cs)) for x, y in zip(xs, ys)]
-    t = _time(lambda i: h.hero_layernorm_quant(ins[i][0], g, b, 1e-5, hero.tensor(outs[i], "twq", sc), branch=ins[i][1]), n, iters)
+    if out_gran == "fwq":
+        sc = torch.rand(H, device="cuda") * 0.01 + 0.02
+    t = _time(lambda i: h.hero_layernorm_quant(ins[i][0], g, b, 1e-5, hero.tensor(outs[i], out_gran, sc), branch=ins[i][1]), n, iters)
     hbm, _, src = _peaks()
     gbs = M * H * 3 / t / 1e9
-    print("LN^quant %s M=%d H=%d: %.1f us, %.0f GB/s (algorithmic 3 B/element), %.2f of %s copy bandwidth"
-          % (kind, M, H, t * 1e6, gbs, gbs / hbm, src), flush=True)
+    print("LN^quant %s%s M=%d H=%d: %.1f us, %.0f GB/s (algorithmic 3 B/element), %.2f of %s copy bandwidth"
+          % (kind, "" if out_gran == "twq" else " -> " + out_gran, M, H, t * 1e6, gbs, gbs / hbm, src), flush=True)
 
 
 def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
@@ -267,6 +270,7 @@ def main():
     ap.add_argument("--f8", action="store_true", help="e4m3 operands and output (the FP8 variant)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--out-gran", default="twq", choices=["twq", "fwq"], help="LN^quant output quantizer")
     ap.add_argument("--graph", action="store_true", help="time CUDA-graph replays of the launches")
     a = ap.parse_args()
     global GRAPH
@@ -278,7 +282,7 @@ def main():
                 for M in W.LN_SWEEP_M:
                     bench_ln(h, M, H, a.kind, a.iters)
         else:
-            bench_ln(h, a.M, a.H, a.kind, a.iters)
+            bench_ln(h, a.M, a.H, a.kind, a.iters, a.out_gran)
     elif a.kernel == "gemm":
         if a.sweep:
             for K, N in W.GEMM_SWEEP_KN:
