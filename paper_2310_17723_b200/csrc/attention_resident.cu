@@ -11,6 +11,7 @@
 // has been read.  The epilogue of tile t runs inside tile t+1, after the first three score blocks of t+1 have been
 // exponentiated: P V of tile t finishes in the shadow of that work.
 #include "attention_common.cuh"
+#include <type_traits>
 
 namespace hero {
 
@@ -375,7 +376,11 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         }
         m = (float)imax;                                     // exchanged as an (exact) integer-valued float
       } else {
-      // ---- sweep 1: per piece, e = 2^(t - m_piece) written back over the scores; running (m, l) in registers
+      // ---- sweep 1: per piece, e = 2^(t - m_piece) written back over the scores; running (m, l) in registers.
+      // FULL: every key of every block is valid for every row of the tile (no mask, no short sequence): the loop then
+      // carries no per-piece validity logic at all.
+      auto sweep1 = [&](auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll 1
       for (int j = 0; j < nkv; ++j) {
         if (j == 3 && pend) epilogue();                      // block 3's columns hold the previous tile's output
@@ -392,10 +397,10 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {                   // two 16-column pieces, each with its own maximum
             uint32_t (&r)[16] = hh ? rb : ra;
-            const int nvalid = min(16, kmax - (kb + 16 * hh) + 1);
+            const int nvalid = FULL ? 16 : min(16, kmax - (kb + 16 * hh) + 1);
             float mp = -INFINITY;
-            if (nvalid > 0) {
-              if (nvalid < 16) {
+            if (FULL || nvalid > 0) {
+              if (!FULL && nvalid < 16) {
                 // masked keys: a score far below every real one (|t| < 2^21) turns into e = 0 by itself
 #pragma unroll
                 for (int e = 0; e < 16; ++e) if (e >= nvalid) r[e] = F8 ? __float_as_uint(-1.0e30f) : (uint32_t)(-(1 << 21));
@@ -438,6 +443,8 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           pm2[j * 512] = make_float2(mpa[0], mpa[1]);
         }
       }
+      };
+      if (p.mask != HERO_MASK_CAUSAL && klen >= nkv * ATT_BN) sweep1(std::true_type{}); else sweep1(std::false_type{});
       }
       if constexpr (!ROWMAX) ptx::tmem_st_wait();
       if (pend) epilogue();
