@@ -538,6 +538,8 @@ def run_ours(args):
                        "timing": "CUDA events per step on the launching stream, max over ranks",
                        "parallelism": "replicas x%d (sequence-sharded, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "kernels": kern,
+            "kernels_note": "per-launch times come from a second pass with an event pair around every launch, which serialises the "
+                            "launches (no programmatic overlap): their sum exceeds ms_per_step, so the fractions are lower bounds",
             "cpu_baseline": cpu, "fp16_path": fp_path, "wall_s_timed_region": wall}
     if mixed_path:
         line["attention_and_ln_bf16_path"] = mixed_path
