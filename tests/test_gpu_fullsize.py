@@ -207,3 +207,63 @@ def test_c5_stack_full_batch_sampled_sequence():
     assert dev_vs_oracle < 0.75 * q_err and rel_err(got, want) < 0.15, (dev_vs_oracle, q_err)
     assert mean_rel(got, plain) < 1.25 * q_err                       # and the device is as close to the un-quantized stack
     h.close()
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# the largest points of the standalone-kernel sweep: the whole launch on the device, sampled outputs from the oracle
+# ------------------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,K,N", [(32768, 4096, 16384), (32768, 16384, 4096), (8192, 1024, 4096)])
+def test_sweep_gemm_full_size_sampled_rows_and_columns(M, K, N):
+    from oracle import quant as Q
+    from gpu_util import f32
+    A, Wt, rs, cs, bias = W.gemm_case(M, K, N)
+    h = hero.Handle()
+    tA, tW = torch.from_numpy(A).cuda(), torch.from_numpy(Wt).cuda()
+    out = torch.full((M, N), -77, dtype=torch.int8, device="cuda")
+    h.hero_w8a8_linear(hero.tensor(tA, "twq", f32(rs)), tW, hero.tensor(out), w_scale=f32(cs), bias=f32(bias))
+    h.check()
+    g = W.rng(2, 4242)
+    rows = np.sort(np.concatenate([[0, 127, 128, 255, 256, M - 1], g.choice(M, 58, replace=False)]))
+    cols = np.sort(np.concatenate([[0, 255, 256, N - 1], g.choice(N, 60, replace=False)]))
+    # sampled rows x all columns
+    want = O.gemm_quant(O.QT("i8", A[rows], row_scale=rs[rows].astype(np.float64)), Wt.T.copy(), cs, bias, "none", O.OutSpec("round"))
+    assert_int8_close(out[torch.from_numpy(rows).cuda()].cpu().numpy(), want.data, what="sampled rows")
+    # all rows x sampled columns
+    want = O.gemm_quant(O.QT("i8", A, row_scale=rs.astype(np.float64)), np.ascontiguousarray(Wt[cols].T), cs[cols], bias[cols],
+                        "none", O.OutSpec("round"))
+    assert_int8_close(out[:, torch.from_numpy(cols).cuda()].cpu().numpy(), want.data, what="sampled columns")
+    assert np.abs(want.data.astype(int)).max() > 60
+    h.close()
+
+
+@pytest.mark.parametrize("M,H,kind", [(65536, 8192, "f16"), (65536, 4096, "i8"), (65536, 768, "i8")])
+def test_sweep_ln_full_size_sampled_rows(M, H, kind):
+    from gpu_util import f32
+    g = W.rng(2, 77 + H)
+    torch.manual_seed(77 + H)                          # the large tensors are drawn on the device, seeded
+    gamma, beta = (1 + 0.1 * g.standard_normal(H)).astype(np.float32), (0.1 * g.standard_normal(H)).astype(np.float32)
+    rows = np.sort(np.concatenate([[0, 7, 8, M - 1], g.choice(M, 60, replace=False)]))
+    trows = torch.from_numpy(rows).cuda()
+    h = hero.Handle()
+    out = torch.full((M, H), -77, dtype=torch.int8, device="cuda")
+    sc = torch.zeros(M, dtype=torch.float32, device="cuda")
+    if kind == "f16":
+        x = torch.randn(M, H, device="cuda", dtype=torch.float16)
+        x[:, 5] *= 20
+        h.hero_layernorm_quant(hero.tensor(x), f32(gamma), f32(beta), 1e-5, hero.tensor(out, "twq", sc))
+        ins = [O.QT("fp", x[trows].float().cpu().numpy().astype(np.float64), dtype="f16")]
+    else:
+        xr = torch.randint(-127, 128, (M, H), device="cuda", dtype=torch.int8)
+        xb = torch.randint(-127, 128, (M, H), device="cuda", dtype=torch.int8)
+        rs = (torch.rand(M, device="cuda") * 0.02 + 0.01)
+        cs = (np.abs(g.standard_normal(H)) * 0.01 + 0.005).astype(np.float32)
+        h.hero_layernorm_quant(hero.tensor(xr, "twq", rs), f32(gamma), f32(beta), 1e-5, hero.tensor(out, "twq", sc),
+                               branch=hero.tensor(xb, "fwq", f32(cs)))
+        ins = [O.QT("i8", xr[trows].cpu().numpy(), row_scale=rs[trows].cpu().numpy().astype(np.float64)),
+               O.QT("i8", xb[trows].cpu().numpy(), col_scale=cs.astype(np.float64))]
+    h.check()
+    want, _ = O.ln_quant(ins, gamma, beta, 1e-5, O.OutSpec("twq"))
+    assert_int8_close(out[trows].cpu().numpy(), want.data, 1e-4, "sampled rows")
+    np.testing.assert_allclose(sc[trows].cpu().numpy(), want.row_scale, rtol=2e-6)
+    assert bool((sc > 0).all())                                                      # every row was written
+    h.close()
