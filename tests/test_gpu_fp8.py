@@ -82,7 +82,9 @@ def test_ln_quant_e4m3_residual_plus_e4m3_branch(h):
 
 
 GEMM_CASES = [(200, 512, 256, "none"), (1024, 1024, 2048, "none"), (1024, 1024, 2048, "gelu_erf"), (129, 4096, 1024, "none"),
-              (2000, 768, 3072, "gelu_erf")]
+              (2000, 768, 3072, "gelu_erf"),
+              # few rows: the kernel with the operands swapped on the tensor core and K split over a cluster
+              (1, 4096, 1024, "none"), (16, 8192, 512, "gelu_erf"), (40, 16384, 1024, "none"), (128, 8192, 256, "gelu_erf")]
 
 
 @pytest.mark.parametrize("M,K,N,act", GEMM_CASES)
