@@ -23,7 +23,9 @@
  * detected on the host before anything is launched.  HERO_ERR_CUDA reports a failed runtime call
  * (text via hero_last_error()).  A device-side wait that exceeded its bound (a pipeline bug, never
  * expected) sets a device error word; hero_check() synchronizes the stream and returns
- * HERO_ERR_DEVICE_TIMEOUT if it is set.
+ * HERO_ERR_DEVICE_TIMEOUT if it is set.  The same word reports an embedding id outside its table (the gather of
+ * hero_layernorm_quant clamps such an id, so nothing is read out of bounds): hero_check() then returns
+ * HERO_ERR_INVALID_ARG.
  */
 #ifndef HERO_H_
 #define HERO_H_
@@ -104,6 +106,8 @@ int64_t hero_launch_count(const hero_handle* h);
  *   token_ids != NULL selects the embedding gather of Eq. 7: `residual` is then the token table
  *       [V, H] I8 with TWQ scale [V], row ids[i]; `branch` the position table [P, H] F16/BF16, row
  *       (i mod seq_len); `extra` the sentence-type table [T, H], row type_ids[i].  M = n_tokens.
+ *       P >= seq_len is required.  An id outside [0, V) or [0, T) is clamped to the nearest valid row and reported
+ *       by the next hero_check() as HERO_ERR_INVALID_ARG.
  *   out      : I8 (gran TWQ: out.scale[M] is written; FWQ / SQ: out.scale is read) or F16 / BF16.
  *              out.data == NULL skips the normalisation (bare residual add into fp_out).
  *   fp_out   : optional F16 / BF16 copy of r (the FP residual stream of a pre-LN layer); when
@@ -393,10 +397,17 @@ hero_status hero_layer_forward_host_async(hero_handle* h, const hero_layer_desc*
  *   - All calls on a device share the one array, and it keeps whatever the last call left in it (nothing in it
  *     needs clearing: each call overwrites what it reads).  Two calls that overlap on the GPU, e.g. on two
  *     streams, race on it: serialize them.
- *   - A bounded device-side wait that gives up cannot be reported here (there is no handle to hero_check).
+ *   - Host threads may call it concurrently as far as the host side goes, but their kernels share the one array:
+ *     unless the caller serializes them on the GPU (one stream, or events between streams) they race on it.
+ *   - A bounded device-side wait that gives up is recorded in a device word of the library image (there is no
+ *     handle for hero_check to look at); hero_static_check reads it.
  * Inputs, outputs, weights and scales are passed exactly as for hero_layer_forward. */
 hero_status hero_layer_forward_static(const hero_layer_desc* d, const hero_tensor* in, const hero_tensor* pending,
                                       const hero_tensor* out, void* stream);
+/* hero_check for hero_layer_forward_static (the paper has no counterpart either): synchronizes `stream`, reads the
+ * device error word of the current device, clears it, and returns HERO_OK or HERO_ERR_DEVICE_TIMEOUT.  Allocates
+ * nothing (a symbol copy). */
+hero_status hero_static_check(void* stream);
 
 /* Per-launch device timing for benchmarks (no counterpart in the paper, which measured nothing): between
  * _begin and _end every kernel the handle launches is bracketed by a pair of CUDA events on its stream.

@@ -41,8 +41,8 @@ hero_status check_matrix(const hero_tensor& t, const char* name) {
   HERO_REQUIRE(aligned16(t.data), HERO_ERR_ALIGNMENT, "%s: data pointer is not 16-byte aligned", name);
   HERO_REQUIRE((t.ld * es) % 16 == 0, HERO_ERR_ALIGNMENT, "%s: row pitch %lld bytes is not a multiple of 16", name,
                (long long)(t.ld * es));
-  if (t.dtype == HERO_I8 && t.gran != HERO_GRAN_NONE)
-    HERO_REQUIRE(t.scale != nullptr, HERO_ERR_INVALID_ARG, "%s: INT8 tensor with granularity %d needs a scale", name,
+  if (is_q8(t.dtype) && t.gran != HERO_GRAN_NONE)
+    HERO_REQUIRE(t.scale != nullptr, HERO_ERR_INVALID_ARG, "%s: 8-bit tensor with granularity %d needs a scale", name,
                  t.gran);
   return HERO_OK;
 }
@@ -94,7 +94,7 @@ hero_status hero_create(hero_handle** out) {
   h->device = dev;
   h->sm_count = prop.multiProcessorCount;
   h->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
-  h->launches = 0;
+  h->launches.store(0);
   h->d_error = nullptr;
   h->encode_tiled = nullptr;
   h->prof_on = false; h->prof_cap = 0; h->prof_n = 0; h->prof_ev = nullptr; h->prof_tag = nullptr;
@@ -166,13 +166,17 @@ hero_status hero_check(hero_handle* h, void* stream) {
   HERO_CUDA(cudaMemcpy(&code, h->d_error, sizeof(int), cudaMemcpyDeviceToHost));
   if (code != 0) {
     cudaMemset(h->d_error, 0, sizeof(int));
+    if (code == hero::ERR_BAD_ID) {
+      hero::set_error("an embedding id was outside its table; it was clamped to the nearest valid row");
+      return HERO_ERR_INVALID_ARG;
+    }
     hero::set_error("a bounded device-side wait gave up (code 0x%x)", code);
     return HERO_ERR_DEVICE_TIMEOUT;
   }
   return HERO_OK;
 }
 
-int64_t hero_launch_count(const hero_handle* h) { return h ? h->launches : 0; }
+int64_t hero_launch_count(const hero_handle* h) { return h ? h->launches.load(std::memory_order_relaxed) : 0; }
 
 hero_status hero_mode_preset(int32_t preset, int32_t mode_out[5]) {
   HERO_REQUIRE(mode_out != nullptr, HERO_ERR_INVALID_ARG, "hero_mode_preset: mode_out is NULL");

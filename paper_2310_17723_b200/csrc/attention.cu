@@ -492,11 +492,7 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
     p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);     // U8 x S8 -> S32, V is MN-major
   }
   auto kern = attn_int8_kernel<DH, ROWMAX, F8>;
-  static bool configured = false;
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    configured = true;
-  }
+  HERO_SMEM_OPT_IN(h, kern, Cfg::SMEM_BYTES);
   const long long tiles = (long long)p.nqt * a->nh * a->B;
   const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);   // persistent: one CTA per SM
   {

@@ -276,10 +276,10 @@ template <int DH, int NT>
 static hero_status launch_decode(hero_handle* h, const DecodeParams& p, int B, int splits, cudaStream_t stream) {
   auto kern = attn_decode_kernel<DH, NT>;
   const size_t smem = (size_t)p.chunk_cap * 5 + (size_t)(NT / 32 * DH + DH) * 4 + 8 + NT / 32 * 4 + 16;
-  static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
+  static PerDeviceInt configured;    // largest opt-in made so far, per device
+  if (smem > 48 * 1024 && (int)smem > configured.get(h->device)) {
     HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    configured = smem;
+    configured.set(h->device, (int)smem);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)splits, (unsigned)p.nh, (unsigned)B);

@@ -342,11 +342,7 @@ static hero_status launch_attn_fp(hero_handle* h, const hero_attn_args* a, AttnP
   p.idesc_qk = ptx::make_idesc(1, fmt, fmt, 0, 0, ATT_BM, ATT_BN);   // F32 accumulate, both operands K-major
   p.idesc_pv = ptx::make_idesc(1, fmt, fmt, 0, 1, ATT_BM, DH);       // V is MN-major
   auto kern = attn_fp_kernel<DH>;
-  static bool configured = false;
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    configured = true;
-  }
+  HERO_SMEM_OPT_IN(h, kern, Cfg::SMEM_BYTES);
   const long long tiles = (long long)p.nqt * a->nh * a->B;
   const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);
   {

@@ -6,6 +6,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 
 #include "../../include/hero.h"
 #ifdef __CUDACC__
@@ -17,7 +18,7 @@ struct hero_handle {
   int sm_count;
   int max_smem_optin;
   int* d_error;        // device error word: 0 = fine, else a code saying which wait gave up
-  int64_t launches;
+  std::atomic<int64_t> launches;   // bumped by every launch; several host threads may share a handle's counter
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
   // optional per-launch timing (hero_profile_begin / _end): event pairs around every kernel launch
   bool prof_on;
@@ -63,13 +64,17 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // data pointer 16-byte aligned, row pitch a multiple of 16 bytes, ld >= cols
 hero_status check_matrix(const hero_tensor& t, const char* name);
 
+// Codes a kernel may leave in the device error word besides "a bounded wait gave up" (those carry the place in
+// their low 16 bits and nothing above): an embedding id outside its table, clamped by LN^quant's gather.
+constexpr int ERR_BAD_ID = 0x1D000001;
+
 // Kernel families for the per-launch timing records.
 enum { KERNEL_LN = 1, KERNEL_GEMM = 2, KERNEL_ATTN = 3 };
 // Brackets one kernel launch with events when timing is on; counts the launch either way.
 struct LaunchScope {
   hero_handle* h; cudaStream_t s; int slot;
   LaunchScope(hero_handle* h_, cudaStream_t s_, int tag) : h(h_), s(s_), slot(-1) {
-    h->launches += 1;
+    h->launches.fetch_add(1, std::memory_order_relaxed);
     if (h->prof_on && h->prof_n < h->prof_cap) {
       slot = h->prof_n++;
       h->prof_tag[slot] = tag;
@@ -78,6 +83,31 @@ struct LaunchScope {
   }
   ~LaunchScope() { if (slot >= 0) cudaEventRecord(h->prof_ev[2 * slot + 1], s); }
 };
+
+// Function attributes (the opt-in to more than 48 KB of dynamic shared memory) and occupancy figures belong to a
+// (kernel, device) pair, not to the process.  One of these per kernel instantiation (a function-local static)
+// remembers per device ordinal what has been set; lock-free, and a lost race only repeats an idempotent call.
+constexpr int MAX_DEVICES = 64;
+struct PerDeviceOnce {
+  std::atomic<uint64_t> mask{0};
+  bool done(int dev) const { return dev >= 0 && dev < MAX_DEVICES && ((mask.load(std::memory_order_acquire) >> dev) & 1); }
+  void set(int dev) { if (dev >= 0 && dev < MAX_DEVICES) mask.fetch_or(1ull << dev, std::memory_order_release); }
+};
+struct PerDeviceInt {
+  std::atomic<int> v[MAX_DEVICES];
+  PerDeviceInt() { for (auto& x : v) x.store(0, std::memory_order_relaxed); }
+  int get(int dev) const { return dev >= 0 && dev < MAX_DEVICES ? v[dev].load(std::memory_order_acquire) : 0; }
+  void set(int dev, int x) { if (dev >= 0 && dev < MAX_DEVICES) v[dev].store(x, std::memory_order_release); }
+};
+// Opts `kern` in to `bytes` of dynamic shared memory on the handle's device, once per device.
+#define HERO_SMEM_OPT_IN(h, kern, bytes)                                                                 \
+  do {                                                                                                   \
+    static hero::PerDeviceOnce _once;                                                                    \
+    if (!_once.done((h)->device)) {                                                                      \
+      HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes))); \
+      _once.set((h)->device);                                                                            \
+    }                                                                                                    \
+  } while (0)
 
 // Kernel launch with programmatic dependent launch allowed: the grid may be scheduled while the previous kernel of
 // the stream is still draining, runs its set-up (barrier init, tensor-memory allocation, descriptor prefetch) and then

@@ -438,11 +438,7 @@ static hero_status launch_gemm(hero_handle* h, const CUtensorMap& tmA, const CUt
                                cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
   auto kern = gemm_kernel<BN, INT8, ACT, OUTK>;
-  static bool configured = false;   // per instantiation
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    configured = true;
-  }
+  HERO_SMEM_OPT_IN(h, kern, Cfg::SMEM_BYTES);
   const int tiles = p.num_m_tiles * p.num_n_tiles;
   const int grid = tiles < h->sm_count ? tiles : h->sm_count;
   {
@@ -644,11 +640,7 @@ template <bool INT8, int ACT, int OUTK, int EW>
 static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
                                        cudaStream_t stream) {
   auto kern = gemm_pair_kernel<INT8, ACT, OUTK, EW>;
-  static bool configured = false;
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg::SMEM_BYTES));
-    configured = true;
-  }
+  HERO_SMEM_OPT_IN(h, kern, PairCfg::SMEM_BYTES);
   const int tiles = p.num_m_tiles * p.num_n_tiles;
   const int pairs_max = h->sm_count / 2;
   const int pairs = tiles < pairs_max ? tiles : pairs_max;

@@ -232,11 +232,7 @@ static hero_status launch_skinny(hero_handle* h, const CUtensorMap& tmW, const C
                                  int splits, cudaStream_t stream) {
   using Cfg = SkinnyCfg<MT>;
   auto kern = gemm_skinny_kernel<MT, INT8>;
-  static bool configured = false;   // per instantiation
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    configured = true;
-  }
+  HERO_SMEM_OPT_IN(h, kern, Cfg::SMEM_BYTES);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)splits, (unsigned)p.num_n_tiles);
   cfg.blockDim = dim3(SK_THREADS);

@@ -24,8 +24,7 @@ struct StaticState {
   hero_handle handle;
   void* scratch = nullptr;
 };
-constexpr int MAX_DEVICES = 64;
-StaticState g_state[MAX_DEVICES];
+StaticState g_state[hero::MAX_DEVICES];
 std::mutex g_mutex;
 
 // One-time set-up for the current device: no allocation, only queries and symbol look-ups.
@@ -47,7 +46,9 @@ hero_status setup_device(int dev, StaticState** out) {
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &encode, cudaEnableDefault, &qres);
     HERO_REQUIRE(e == cudaSuccess && qres == cudaDriverEntryPointSuccess && encode != nullptr, HERO_ERR_CUDA,
                  "cuTensorMapEncodeTiled could not be resolved");
-    memset(&s.handle, 0, sizeof(s.handle));
+    s.handle.launches.store(0);
+    s.handle.prof_on = false; s.handle.prof_cap = 0; s.handle.prof_n = 0;
+    s.handle.prof_ev = nullptr; s.handle.prof_tag = nullptr;
     s.handle.device = dev;
     s.handle.sm_count = prop.multiProcessorCount;
     s.handle.max_smem_optin = (int)prop.sharedMemPerBlockOptin;
@@ -79,10 +80,27 @@ extern "C" hero_status hero_layer_forward_static(const hero_layer_desc* d, const
                need, STATIC_SCRATCH_BYTES);
   int dev = 0;
   HERO_CUDA(cudaGetDevice(&dev));
-  HERO_REQUIRE(dev >= 0 && dev < MAX_DEVICES, HERO_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+  HERO_REQUIRE(dev >= 0 && dev < hero::MAX_DEVICES, HERO_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
   StaticState* s = nullptr;
   if ((st = setup_device(dev, &s)) != HERO_OK) return st;
   // Every intermediate the layer reads is written by an earlier kernel of the same call, so nothing in the
   // scratch has to start at zero; what a previous call left there is simply overwritten.
   return hero_layer_forward(&s->handle, d, in, pending, out, s->scratch, STATIC_SCRATCH_BYTES, stream);
+}
+
+// The device error word of hero_layer_forward_static (the entry point has no handle for hero_check to look at).
+// Synchronizes `stream`, copies the word back with a symbol copy (no allocation), clears it and reports what it held.
+extern "C" hero_status hero_static_check(void* stream) {
+  HERO_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  int code = 0;
+  HERO_CUDA(cudaMemcpyFromSymbol(&code, g_static_error_word, sizeof(int)));
+  if (code == 0) return HERO_OK;
+  const int zero = 0;
+  HERO_CUDA(cudaMemcpyToSymbol(g_static_error_word, &zero, sizeof(int)));
+  if (code == hero::ERR_BAD_ID) {
+    hero::set_error("an embedding id was outside its table; it was clamped to the nearest valid row");
+    return HERO_ERR_INVALID_ARG;
+  }
+  hero::set_error("a bounded device-side wait gave up (code 0x%x)", code);
+  return HERO_ERR_DEVICE_TIMEOUT;
 }

@@ -27,6 +27,8 @@ struct LnParams {
   const int* token_ids;   // embedding gather (Eq. 7) when non-NULL
   const int* type_ids;
   int seq_len;
+  int n_tok_rows, n_type_rows;   // rows of the token / sentence-type tables: ids are clamped into them
+  int* err;                      // device error word: an out-of-range id records ERR_BAD_ID there
   const float* gamma;
   const float* beta;
   float eps;
@@ -36,6 +38,17 @@ struct LnParams {
   int G;                  // threads per row (multiple of 32)
   int RPC;                // rows per CTA per pass
 };
+
+// Row of an embedding table named by ids[row].  An id outside [0, n_rows) must not become an out-of-bounds read:
+// it is clamped into the table and a code is left in the device error word for hero_check to report.
+__device__ __forceinline__ long long table_row(const int* ids, long long row, int n_rows, int* err) {
+  int id = ids[row];
+  if ((unsigned)id >= (unsigned)n_rows) {
+    if (err) atomicExch(err, ERR_BAD_ID);
+    id = id < 0 ? 0 : n_rows - 1;
+  }
+  return id;
+}
 
 template <int VEC>
 __device__ __forceinline__ void load_raw(const void* p, int bytes_per_elem, uint32_t (&w)[VEC / 2]) {
@@ -201,9 +214,9 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
       if (valid[r]) {
         long long rr = row[r], rb = row[r], re = row[r];
         if (p.token_ids) {
-          rr = p.token_ids[row[r]];
+          rr = table_row(p.token_ids, row[r], p.n_tok_rows, p.err);
           rb = row[r] % p.seq_len;
-          re = p.type_ids ? p.type_ids[row[r]] : 0;
+          re = p.type_ids ? table_row(p.type_ids, row[r], p.n_type_rows, p.err) : 0;
         }
         load_raw<VEC>(reinterpret_cast<const char*>(p.res.data) + (rr * p.res.ld + c0) * res_es, res_es, raw_res[r]);
         if (p.res.row_scale) rs_res[r] = p.res.row_scale[rr];
@@ -540,9 +553,9 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams 
       long long r_res = row, r_br = row, r_ex = row;
       if constexpr (EX) {
         if (p.token_ids) {
-          r_res = p.token_ids[row];
+          r_res = table_row(p.token_ids, row, p.n_tok_rows, p.err);
           r_br = row % p.seq_len;
-          r_ex = p.type_ids ? p.type_ids[row] : 0;
+          r_ex = p.type_ids ? table_row(p.type_ids, row, p.n_type_rows, p.err) : 0;
         }
       }
       uint8_t* dst = ring + st * stage_bytes + slot * slot_bytes;
@@ -612,7 +625,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_fast_kernel(const LnParams 
     float rs_res = 1.f, rs_br = 1.f;
     if (row_ok) {
       long long r_res = row, r_br = row;
-      if constexpr (EX) { if (p.token_ids) { r_res = p.token_ids[row]; r_br = row % p.seq_len; } }
+      if constexpr (EX) { if (p.token_ids) { r_res = table_row(p.token_ids, row, p.n_tok_rows, nullptr); r_br = row % p.seq_len; } }
       if (RES == SRC_I8 && p.res.row_scale) rs_res = __ldg(p.res.row_scale + r_res);
       if (BR == SRC_I8 && p.br.row_scale) rs_br = __ldg(p.br.row_scale + r_br);
     }
@@ -829,11 +842,7 @@ static hero_status launch_fast(hero_handle* h, LnParams& p, cudaStream_t stream)
   p.RPC = stages;
   const size_t smem = (size_t)stages * stage;
   auto kern = ln_fast_kernel<RES, BR, EX, OUT, FPOUT, NCHX>;
-  static bool configured = false;   // per instantiation
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-    configured = true;
-  }
+  HERO_SMEM_OPT_IN(h, kern, 160 * 1024);
   int occ = 1;
   HERO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, LNF_THREADS, smem));
   if (occ < 1) occ = 1;
@@ -1241,15 +1250,13 @@ static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream)
   constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR);
   const size_t smem = (size_t)stages * STAGE + VEC;
   auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8, GEO>;
-  static bool configured = false;   // per instantiation
-  if (!configured) {
-    HERO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    configured = true;
-  }
-  static int occ = 0;               // per instantiation: the launch configuration never changes
+  HERO_SMEM_OPT_IN(h, kern, 200 * 1024);
+  static PerDeviceInt occ_cache;     // per instantiation and device: the launch configuration never changes
+  int occ = occ_cache.get(h->device);
   if (occ < 1) {
     HERO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, LNF_THREADS, smem));
     if (occ < 1) occ = 1;
+    occ_cache.set(h->device, occ);
   }
   const long long want = (p.M + SLOTS - 1) / SLOTS;
   const long long cap = (long long)h->sm_count * occ;
@@ -1406,7 +1413,14 @@ extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* 
     HERO_REQUIRE(a->seq_len > 0, HERO_ERR_INVALID_ARG, "embedding gather: seq_len must be positive");
     HERO_REQUIRE(a->extra.data == nullptr || a->type_ids != nullptr, HERO_ERR_INVALID_ARG,
                  "embedding gather: type_ids required with a sentence-type table");
+    HERO_REQUIRE(a->residual.rows > 0 && a->residual.rows < (1ll << 31), HERO_ERR_INVALID_ARG, "embedding gather: the token table needs 1 .. 2^31-1 rows");
+    HERO_REQUIRE(a->branch.data == nullptr || a->branch.rows >= a->seq_len, HERO_ERR_INVALID_ARG,
+                 "embedding gather: the position table has %lld rows, seq_len is %d", (long long)a->branch.rows, a->seq_len);
+    HERO_REQUIRE(a->extra.data == nullptr || (a->extra.rows > 0 && a->extra.rows < (1ll << 31)), HERO_ERR_INVALID_ARG,
+                 "embedding gather: the sentence-type table needs at least one row");
     p.token_ids = a->token_ids; p.type_ids = a->type_ids; p.seq_len = a->seq_len;
+    p.n_tok_rows = (int)a->residual.rows; p.n_type_rows = a->extra.data ? (int)a->extra.rows : 1;
+    p.err = h->d_error;
   } else {
     HERO_REQUIRE(a->branch.data == nullptr || a->branch.rows == p.M, HERO_ERR_INVALID_ARG, "branch rows differ");
     HERO_REQUIRE(a->extra.data == nullptr || a->extra.rows == p.M, HERO_ERR_INVALID_ARG, "extra rows differ");

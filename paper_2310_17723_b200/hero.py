@@ -101,7 +101,7 @@ EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_layer_forward_host_async", "hero_profile_begin",
            "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram",
-           "hero_int8_decode_attention", "hero_layer_decode")
+           "hero_int8_decode_attention", "hero_layer_decode", "hero_static_check")
 
 _lib = None
 
@@ -141,6 +141,7 @@ def lib():
             [C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_layer_forward_static.argtypes = [C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                                 C.POINTER(Tensor), C.c_void_p]
+        L.hero_static_check.argtypes = [C.c_void_p]
         L.hero_profile_begin.argtypes = [C.c_void_p, C.c_int32]
         L.hero_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         _lib = L
@@ -328,6 +329,11 @@ def hero_layer_forward_static(desc, x_in, out, pending=None, stream=None):
     do not let two of them overlap on the GPU."""
     pend = C.byref(pending) if pending is not None else None
     _check(lib().hero_layer_forward_static(C.byref(desc), C.byref(x_in), pend, C.byref(out), _stream(stream)))
+
+
+def hero_static_check(stream=None):
+    """Synchronizes the stream and raises if a kernel of hero_layer_forward_static left a code in its error word."""
+    _check(lib().hero_static_check(_stream(stream)))
 
 
 def mode_preset(preset):

@@ -1,4 +1,6 @@
 """Helpers for the GPU parity tests: move oracle tensors to the device, compare within the stated bars."""
+import os
+
 import numpy as np
 import torch
 
@@ -46,12 +48,25 @@ def int8_mismatch(got, want):
     return float(np.mean(d != 0)), int(d.max()) if d.size else 0
 
 
+def report(what, text):
+    """One line per passed parity check (shown by `pytest -s`; appended to the file HERO_PARITY_LOG names, if set),
+    so that every bar's headroom is on record."""
+    line = "parity %-44s %s" % (what or "(unnamed)", text)
+    print(line)
+    path = os.environ.get("HERO_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+
+
 def assert_int8_close(got, want, frac=1e-4, what=""):
-    """The INT8 bar: bit-exact except at most 1 LSB on at most `frac` of the elements."""
+    """The INT8 bar: bit-exact except at most 1 LSB on at most `frac` of the elements.  The measured mismatch
+    fraction and largest difference are reported on success too."""
     f, m = int8_mismatch(got, want)
     assert m <= 1, "%s: max INT8 difference %d LSB" % (what, m)
     # small tensors: allow a single tie
     assert f <= max(frac, 1.0 / max(np.asarray(want).size, 1)), "%s: %.3g of elements differ" % (what, f)
+    report(what, "mismatch %.3g of %d elements (bar %.1g), max %d LSB" % (f, np.asarray(want).size, frac, m))
 
 
 def rel_err(got, want):

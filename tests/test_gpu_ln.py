@@ -167,6 +167,41 @@ def test_embedding_gather_flavour(h):
     assert np.allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
 
 
+def test_embedding_gather_clamps_out_of_range_ids_and_reports_them(h):
+    # a bad id from upstream must not become an out-of-bounds read: the row is taken from the nearest valid table row
+    # and the next hero_check() says so
+    V, P, T, H, S, B = 50, 32, 2, 768, 32, 2
+    g = W.rng(0, 43)
+    tok, pos, typ = W.embedding_tables(V, P, T, H)
+    tok_q, tok_s = Q.quant_twq(tok)
+    ids = g.integers(0, V, B * S).astype(np.int32)
+    tids = g.integers(0, T, B * S).astype(np.int32)
+    bad_ids, bad_tids = ids.copy(), tids.copy()
+    bad_ids[3], bad_ids[40], bad_tids[17] = V + 100000, -5, T + 7
+    ids[3], ids[40], tids[17] = V - 1, 0, T - 1                       # what the clamp makes of them
+    gamma = (1 + 0.1 * g.standard_normal(H)).astype(np.float32)
+    beta = (0.1 * g.standard_normal(H)).astype(np.float32)
+    want = O.embedding_ln_quant(ids, tids, tok_q, tok_s, pos, typ, S, gamma, beta, 1e-12, O.OutSpec("twq"))
+    t_tok, t_pos, t_typ = dev(tok_q), dev(pos, torch.float16), dev(typ, torch.float16)
+    out = torch.empty(B * S, H, dtype=torch.int8, device="cuda")
+    sc = torch.zeros(B * S, dtype=torch.float32, device="cuda")
+    h.hero_layernorm_quant(hero.tensor(t_tok, "twq", f32(tok_s)), f32(gamma), f32(beta), 1e-12, hero.tensor(out, "twq", sc),
+                           branch=hero.tensor(t_pos), extra=hero.tensor(t_typ), token_ids=dev(bad_ids), type_ids=dev(bad_tids),
+                           seq_len=S, n_tokens=B * S)
+    with pytest.raises(hero.HeroError) as e:
+        h.check()
+    assert e.value.status == hero.ERR_INVALID_ARG and "embedding id" in str(e.value)
+    h.check()                                                          # the word was cleared
+    assert_int8_close(out.cpu().numpy(), want.data, what="embedding LN, clamped ids")
+    assert np.allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    # a position table shorter than the sequence is refused on the host
+    with pytest.raises(hero.HeroError) as e:
+        h.hero_layernorm_quant(hero.tensor(t_tok, "twq", f32(tok_s)), f32(gamma), f32(beta), 1e-12, hero.tensor(out, "twq", sc),
+                               branch=hero.tensor(t_pos), extra=hero.tensor(t_typ), token_ids=dev(ids), type_ids=dev(tids),
+                               seq_len=P + 1, n_tokens=B * S)
+    assert e.value.status == hero.ERR_INVALID_ARG
+
+
 def test_constant_rows_and_empty_input(h):
     H = 768
     x = np.full((4, H), 2.5, np.float32)
@@ -191,3 +226,18 @@ def test_argument_errors(h):
     with pytest.raises(hero.HeroError) as e:
         h.hero_layernorm_quant(hero.tensor(x), g, g, 1e-5, hero.tensor(out, "none", None))
     assert e.value.status == hero.ERR_INVALID_ARG
+    # an 8-bit output of either payload without its scale pointer is an argument error, caught before any launch
+    n0 = h.launches
+    for dt in (torch.int8, torch.float8_e4m3fn):
+        o8 = torch.empty(4, H, dtype=dt, device="cuda")
+        for gran in ("twq", "fwq", "sq"):
+            with pytest.raises(hero.HeroError) as e:
+                h.hero_layernorm_quant(hero.tensor(x), g, g, 1e-5, hero.tensor(o8, gran, None))
+            assert e.value.status == hero.ERR_INVALID_ARG, (dt, gran)
+    a8 = torch.zeros(4, H, dtype=torch.float8_e4m3fn, device="cuda")
+    w8 = torch.zeros(64, H, dtype=torch.float8_e4m3fn, device="cuda")
+    o16 = torch.empty(4, 64, dtype=torch.float16, device="cuda")
+    with pytest.raises(hero.HeroError) as e:                          # e4m3 input declared token-wise, no scale given
+        h.hero_w8a8_linear(hero.tensor(a8, "twq", None), w8, hero.tensor(o16), w_scale=torch.ones(64, device="cuda"))
+    assert e.value.status == hero.ERR_INVALID_ARG
+    assert h.launches == n0

@@ -225,3 +225,33 @@ def test_f8_payload_layer_is_close_to_unquantized_layer_and_every_border_is_e4m3
             Wq = Lp[mod]["W_i8"]
             assert np.array_equal(Q.e4m3_round(Wq), Wq)
             assert np.allclose(np.max(np.abs(Wq), axis=0), 448.0)                  # every column uses the full range
+
+
+@pytest.mark.parametrize("preset", ["M2", "M3"])
+def test_pre_ln_pending_branch_equals_the_closing_add(preset):
+    # Two chained pre-LN layers.  Layer 1 closes with h_out = Round_fp(h_mid + X_2) (the lone-layer add).  Layer 2 can
+    # be fed either that h_out, or the un-added pair (h_mid, pending = X_2), in which case its LN1 step forms the same
+    # sum itself.  The residual stream is rounded to the storage type exactly once either way, so every tensor of
+    # layer 2 must be bit-identical between the two forms; and the `pending` form must report the sum as its h_in.
+    shape = W.tiny_shape(arch="pre_ln", mask="causal", eps=1e-5, n_outlier=2)
+    spec = _spec(shape, mode=dict(L.MODE_PRESETS[preset]))
+    p1, p2 = W.layer_params(shape, 21), W.layer_params(shape, 22)
+    x = W.activations(shape, 21)
+    L1 = L.prepare_layer(spec, p1, L.calibrate(spec, p1, x, shape.B))
+    T1 = L.layer_forward(L1, O.fp_tensor(x, spec.fp_dtype))
+    h1 = T1["h_out"]
+    assert h1.kind == "fp" and np.array_equal(Q.round_to_storage(T1["h_mid"].real() + T1["x_2"].real(), spec.fp_dtype), h1.data)
+    assert np.max(np.abs(T1["x_2"].real())) > 0            # the pending branch is not trivially zero
+    L2 = L.prepare_layer(spec, p2, L.calibrate(spec, p2, L.layer_fp64(spec, p1, x)["x_out"], shape.B))
+    Ta = L.layer_forward(L2, h1)                                        # closing-add form
+    Tb = L.layer_forward(L2, T1["h_mid"], pending=T1["x_2"])            # pending form
+    assert np.array_equal(Tb["h_in"].data, h1.data)
+    for key in ("x_in", "qkv", "x_attn", "x_o", "x_mid", "h_mid", "a", "x_2", "h_out"):
+        a, b = Ta[key], Tb[key]
+        assert a.kind == b.kind, key
+        assert np.array_equal(a.data, b.data), key
+        for sa, sb in ((a.row_scale, b.row_scale), (a.col_scale, b.col_scale)):
+            assert (sa is None) == (sb is None) and (sa is None or np.array_equal(sa, sb)), key
+    # and the branch matters: dropping it changes the layer's input
+    Tc = L.layer_forward(L2, T1["h_mid"])
+    assert not np.array_equal(Tc["x_in"].data, Ta["x_in"].data)

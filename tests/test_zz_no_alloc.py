@@ -43,8 +43,16 @@ def test_static_scratch_entry_point_matches_the_workspace_one_twice():
             h.check()
         out = torch.full((M, H), -100, dtype=torch.int8, device="cuda")
         out_s = torch.zeros(M, dtype=torch.float32, device="cuda")
-        hero.hero_layer_forward_static(layer.desc, hero.tensor(x_in, "twq", s_in), hero.tensor(out, "twq", out_s))
+        x_d, o_d = hero.tensor(x_in, "twq", s_in), hero.tensor(out, "twq", out_s)
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        hero.hero_layer_forward_static(layer.desc, x_d, o_d)
+        hero.hero_static_check()                 # synchronizes; raises if a bounded device-side wait gave up
+        free_after = torch.cuda.mem_get_info()[0]
+        if call == 1:
+            # the entry point's promise: the device's free memory is what it was before the call (the first call
+            # may still make the driver load kernels; by the second everything is in place)
+            assert free_after == free_before, "device free memory moved by %d bytes" % (free_before - free_after)
         # same kernels on the same inputs: identical INT8 codes and scales, not merely within the 1-LSB bar
         assert torch.equal(out, ref), "call %d: INT8 output differs" % call
         assert torch.equal(out_s, ref_s), "call %d: row scales differ" % call
