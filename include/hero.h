@@ -206,6 +206,23 @@ typedef struct {
 
 hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream);
 
+/* The same core with its on-chip intermediates written out, for verification (Sec. 2.2.2 Eq. 15-17 name three
+ * quantities that never leave the chip in hero_int8_attention: the INT32 result of Q K^T, the unsigned codes P_u8 and
+ * the INT32 result of P_u8 V).  INT8 operands only, either p_mode; `a->out` is written as usual.  Slow (scalar stores):
+ * for tests, not for the hot path.  Each pointer may be NULL.
+ *   scores  : device int32 [B*nh][S][S]: scores[(b*nh + h)][i][k] = sum_c Q[i][c] K[k][c] (before the factor d~).
+ *   p_codes : device uint8 [B*nh][S][S]: P_u8 of Eq. 16 (HERO_P_ROWMAX: P~_u8); a masked key inside a visited block holds 0.
+ *             Both arrays are written for query row i at every key k < S of the 128-key blocks the kernel visits
+ *             for that row (under a causal mask: blocks up to the one holding the diagonal); other entries are untouched.
+ *   acc     : device int32 [B*S][nh*dh]: acc[i][j] = sum_k P_u8[i][k] V[k][j] of Eq. 17, before s_p s_v / S_attn;
+ *             rows of a sequence without any allowed key are untouched. */
+typedef struct {
+  int32_t* scores;
+  uint8_t* p_codes;
+  int32_t* acc;
+} hero_attn_probe;
+hero_status hero_int8_attention_probe(hero_handle* h, const hero_attn_args* a, const hero_attn_probe* probe, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * One decode step of the INT8 attention core (Sec. 2.2.2 Eq. 15-17 for the single new token of each sequence of a
  * generative model; Sec. 1 names GPT-style models as targets) over an INT8 key / value cache.  Per (b, h), with

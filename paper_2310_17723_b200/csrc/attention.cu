@@ -46,7 +46,8 @@ struct AttnCfg {
 // ROWMAX: P quantized against the row maximum (see attention_resident.cu): sweep 1 then only finds the maximum of the
 // integer scores, sweep 2 does the one exponential per score and sums the un-quantized exponentials.
 // F8: e4m3 Q, K, V and an e4m3 P (the FP8 variant): kind::f8f6f4 MMAs, FP32 scores and accumulator, static s_p.
-template <int DH, bool ROWMAX, bool F8 = false>
+// PROBE: also writes the raw scores, the P codes and the raw accumulators to global memory (verification only).
+template <int DH, bool ROWMAX, bool F8 = false, bool PROBE = false>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -210,6 +211,17 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       int kmax = klen - 1;                                   // last allowed key (inclusive)
       if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
 
+      // verification outputs: row (b, h, q) of the [B*nh][S][S] score / code arrays
+      const long long probe_row = ((long long)(b * p.nh + h) * p.S + q) * p.S;
+      auto probe_scores = [&](const uint32_t (&r)[32], int key0) {
+        if constexpr (PROBE) {
+          if (p.dbg_scores && row_ok) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) if (key0 + e < p.S) p.dbg_scores[probe_row + key0 + e] = (int)r[e];
+          }
+        }
+      };
+
       float m = -INFINITY, l = 0.f;
       if constexpr (ROWMAX) {
         // ---- sweep 1: row maximum of the integer scores only
@@ -222,6 +234,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             uint32_t r[32];
             ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
             ptx::tmem_ld_wait();
+            probe_scores(r, i * ATT_BN + cq * 32);
             const int nvalid = min(32, kmax - (i * ATT_BN + cq * 32) + 1);
             if (nvalid < 32) {
 #pragma unroll
@@ -248,6 +261,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           ptx::tmem_ld32(t_lane + sb * ATT_BN + cq * 32, r);
           ptx::tmem_ld_wait();
           const int kb = i * ATT_BN + cq * 32;
+          probe_scores(r, kb);
           const int nvalid = min(32, kmax - kb + 1);       // keys kb .. kb + nvalid - 1 are allowed
           if (nvalid > 0) {
             float m_blk;
@@ -377,6 +391,12 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
           }
           const int c16 = cq * 2;                              // 16-byte chunk index within the 128-byte row
+          if constexpr (PROBE) {
+            if (p.dbg_p && row_ok) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) if (kb + e < p.S) p.dbg_p[probe_row + kb + e] = (uint8_t)(__float_as_uint(y[e]) & 0xffu);
+            }
+          }
           if constexpr (F8) {
             st_shared16(prow + (((c16) ^ (r_loc & 7)) << 4), ptx::f32x4_to_e4m3x4(y[0], y[1], y[2], y[3]),
                         ptx::f32x4_to_e4m3x4(y[4], y[5], y[6], y[7]), ptx::f32x4_to_e4m3x4(y[8], y[9], y[10], y[11]),
@@ -430,6 +450,12 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int ocol = cq * 32;
         const long long grow = (long long)(row_base + q);
         const int gcol = col0 + ocol;
+        if constexpr (PROBE) {
+          if (p.dbg_acc) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) p.dbg_acc[grow * ((long long)p.nh * p.dh) + gcol + j] = (int)r[j];
+          }
+        }
         auto accf = [&](int j) -> float { return F8 ? __uint_as_float(r[j]) : (float)(int)r[j]; };
         if (p.out_dt == HERO_F8) {
           float v[32];
@@ -475,7 +501,7 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <int DH, bool ROWMAX, bool F8 = false>
+template <int DH, bool ROWMAX, bool F8 = false, bool PROBE = false>
 static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
   using Cfg = AttnCfg<DH>;
   const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
@@ -491,7 +517,7 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
     p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN); // S8 x S8 -> S32, both K-major
     p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);     // U8 x S8 -> S32, V is MN-major
   }
-  auto kern = attn_int8_kernel<DH, ROWMAX, F8>;
+  auto kern = attn_int8_kernel<DH, ROWMAX, F8, PROBE>;
   HERO_SMEM_OPT_IN(h, kern, Cfg::SMEM_BYTES);
   const long long tiles = (long long)p.nqt * a->nh * a->B;
   const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);   // persistent: one CTA per SM
@@ -505,8 +531,8 @@ static hero_status launch_attn(hero_handle* h, const hero_attn_args* a, AttnPara
 
 }  // namespace hero
 
-extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream) {
-  using namespace hero;
+namespace hero {
+static hero_status attention_impl(hero_handle* h, const hero_attn_args* a, const hero_attn_probe* probe, void* stream) {
   HERO_REQUIRE(h && a, HERO_ERR_INVALID_ARG, "hero_int8_attention: NULL handle or args");
   HERO_REQUIRE(a->q && a->k && a->v, HERO_ERR_INVALID_ARG, "q, k, v are required");
   HERO_REQUIRE(a->B >= 0 && a->S > 0 && a->nh > 0, HERO_ERR_INVALID_ARG, "bad B / S / nh");
@@ -551,10 +577,28 @@ extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args*
   HERO_REQUIRE(a->p_absmax == nullptr || fp_in, HERO_ERR_UNSUPPORTED, "p_absmax is observed by the F16 / BF16 attention core only");
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (probe) {
+    HERO_REQUIRE(a->dtype == HERO_I8, HERO_ERR_UNSUPPORTED, "the verification outputs exist for the INT8 core only");
+    p.dbg_scores = probe->scores; p.dbg_p = probe->p_codes; p.dbg_acc = probe->acc;
+    if (a->S <= 512) return attn_resident_dispatch(h, a, p, s, true);
+    if (rowmax) return a->dh == 64 ? launch_attn<64, true, false, true>(h, a, p, s) : launch_attn<128, true, false, true>(h, a, p, s);
+    return a->dh == 64 ? launch_attn<64, false, false, true>(h, a, p, s) : launch_attn<128, false, false, true>(h, a, p, s);
+  }
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
-  if (a->S <= 512) return attn_resident_dispatch(h, a, p, s);   // the score row fits tensor memory (INT8 or e4m3)
+  if (a->S <= 512) return attn_resident_dispatch(h, a, p, s, false);   // the score row fits tensor memory (INT8 or e4m3)
   if (f8_in) return a->dh == 64 ? launch_attn<64, false, true>(h, a, p, s) : launch_attn<128, false, true>(h, a, p, s);
   if (rowmax) return a->dh == 64 ? launch_attn<64, true>(h, a, p, s) : launch_attn<128, true>(h, a, p, s);
   if (a->dh == 64) return launch_attn<64, false>(h, a, p, s);
   return launch_attn<128, false>(h, a, p, s);
+}
+}  // namespace hero
+
+extern "C" hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream) {
+  return hero::attention_impl(h, a, nullptr, stream);
+}
+
+extern "C" hero_status hero_int8_attention_probe(hero_handle* h, const hero_attn_args* a, const hero_attn_probe* probe,
+                                                 void* stream) {
+  HERO_REQUIRE(probe != nullptr, HERO_ERR_INVALID_ARG, "hero_int8_attention_probe: probe is NULL");
+  return hero::attention_impl(h, a, probe, stream);
 }

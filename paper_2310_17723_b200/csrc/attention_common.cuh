@@ -33,6 +33,11 @@ struct AttnParams {
   uint32_t idesc_qk, idesc_pv;
   int* err;
   float* p_absmax;         // calibration observer of the FP core: running max of the softmax probabilities, or NULL
+  // verification outputs (hero_int8_attention_probe; kernels compiled with PROBE only): raw Q K^T accumulators and
+  // P codes [B*nh][S][S], raw P V accumulators [B*S][nh*dh]; each may be NULL
+  int* dbg_scores;
+  uint8_t* dbg_p;
+  int* dbg_acc;
 };
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -90,6 +95,6 @@ __device__ __forceinline__ int attn_nkv(const AttnParams& p, int qt, int b, int&
 // FP16 / BF16 attention for a module left in FP mode (Table 1); defined in attention_fp.cu
 hero_status attn_fp_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
 // INT8 core with the whole score row resident in tensor memory (S <= 512); defined in attention_resident.cu
-hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
+hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream, bool probe);
 
 }  // namespace hero

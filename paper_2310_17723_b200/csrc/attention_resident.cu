@@ -47,7 +47,7 @@ struct AttnResCfg {
 // columns.  Every softmax warp takes DH / 4 columns of its 32 rows; `osc` is the tile's per-column factor
 // s_p s_v / S_attn[j] (s_p s_v alone for an FP output) staged in shared memory.  Kept out of line: it runs once per
 // tile and its registers stay out of the sweeps' allocation.
-template <int DH, bool F8>
+template <int DH, bool F8, bool PROBE>
 __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, uint64_t* o_full, uint64_t* o_empty,
                                           uint32_t parity, int cq, int lane, long long pend_row, int pend_col,
                                           const float* osc, float rowf, bool& ok) {
@@ -65,6 +65,13 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
   if (lane == 0) ptx::mbar_arrive(o_empty);
   if (pend_row >= 0) {
     const int gcol = pend_col + cq * CW;
+    if constexpr (PROBE) {
+      if (p.dbg_acc) {
+        int* dst = p.dbg_acc + pend_row * ((long long)p.nh * p.dh) + gcol;
+#pragma unroll
+        for (int c = 0; c < CW; ++c) dst[c] = (int)r[c];
+      }
+    }
     const float4* o4 = reinterpret_cast<const float4*>(osc + cq * CW);
     auto acc = [&](int c) -> float { if constexpr (F8) return __uint_as_float(r[c]); else return (float)(int)r[c]; };
     if (p.out_dt == HERO_F8) {
@@ -117,7 +124,8 @@ __device__ __noinline__ void res_epilogue(const AttnParams& p, uint32_t t_lane, 
 // maximum (integer compares, nothing written back), sweep 2 does the one exponential per score.
 // F8: e4m3 Q, K, V and an e4m3 P (the FP8 variant; static P quantizer only): kind::f8f6f4 products, FP32 scores and
 // accumulator in tensor memory, P formed by the saturating conversion instead of round + clip.
-template <int DH, bool ROWMAX, bool F8>
+// PROBE: also writes the raw scores, the P codes and the raw accumulators to global memory (verification only).
+template <int DH, bool ROWMAX, bool F8, bool PROBE>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnParams p) {
@@ -313,7 +321,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     bool pend = false;
 
     auto epilogue = [&]() {
-      res_epilogue<DH, F8>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
+      res_epilogue<DH, F8, PROBE>(p, t_lane, o_full, o_empty, (wcnt - 1) & 1, cq, lane, pend_row, pend_col,
                        osc_s + quarter * 256 + ((wcnt - 1) & 1) * 128, pend_rowf, ok);
       pend = false;
     };
@@ -344,6 +352,24 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       }
       int kmax = klen - 1;
       if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
+      // verification outputs: row (b, h, q) of the [B*nh][S][S] score / code arrays
+      const long long probe_row = ((long long)(b * p.nh + h) * p.S + q) * p.S;
+      auto probe_scores = [&](const uint32_t (&r)[16], int key0) {
+        if constexpr (PROBE) {
+          if (p.dbg_scores && row_ok) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) if (key0 + e < p.S) p.dbg_scores[probe_row + key0 + e] = (int)r[e];
+          }
+        }
+      };
+      auto probe_codes = [&](const uint32_t (&w)[4], int key0) {
+        if constexpr (PROBE) {
+          if (p.dbg_p && row_ok) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) if (key0 + e < p.S) p.dbg_p[probe_row + key0 + e] = (uint8_t)(w[e >> 2] >> (8 * (e & 3)));
+          }
+        }
+      };
 
       float m = -INFINITY, l = 0.f;
       if constexpr (ROWMAX) {
@@ -360,6 +386,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           ptx::tmem_ld16(ta, ra);
           ptx::tmem_ld16(ta + 16, rb);
           ptx::tmem_ld_wait();
+          probe_scores(ra, kb); probe_scores(rb, kb + 16);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             uint32_t (&r)[16] = hh ? rb : ra;
@@ -394,6 +421,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           ptx::tmem_ld16(ta, ra);
           ptx::tmem_ld16(ta + 16, rb);
           ptx::tmem_ld_wait();
+          probe_scores(ra, kb); probe_scores(rb, kb + 16);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {                   // two 16-column pieces, each with its own maximum
             uint32_t (&r)[16] = hh ? rb : ra;
@@ -515,6 +543,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                 const float2 ya = __ffma2_rn(ea, s255, rm2), yb = __ffma2_rn(eb, s255, rm2);
                 w[k] = low_bytes4_u(ya.x, ya.y, yb.x, yb.y);
               }
+              probe_codes(w, kb + 16 * g);
               st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
             }
             l += acc2.x + acc2.y;
@@ -555,6 +584,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                                     fminf(c.x, ATT_MAGIC + 255.0f), fminf(c.y, ATT_MAGIC + 255.0f));
               }
             }
+            probe_codes(w, j * ATT_BN + cq * 32 + 16 * g);
             st_shared16(prow + (((c16 + g) ^ (r_loc & 7)) << 4), w[0], w[1], w[2], w[3]);
           }
           }
@@ -587,7 +617,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   if (warp == ATT_MMA_WARP) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
-template <int DH, bool ROWMAX, bool F8>
+template <int DH, bool ROWMAX, bool F8, bool PROBE = false>
 static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
   using Cfg = AttnResCfg<DH>;
   const uint64_t rows = (uint64_t)a->B * a->S, cols = (uint64_t)a->nh * DH;
@@ -603,7 +633,7 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
     p.idesc_qk = ptx::make_idesc(2, 1, 1, 0, 0, ATT_BM, ATT_BN);   // S8 x S8 -> S32
     p.idesc_pv = ptx::make_idesc(2, 0, 1, 0, 1, ATT_BM, DH);       // U8 x S8 -> S32
   }
-  auto kern = attn_int8_resident_kernel<DH, ROWMAX, F8>;
+  auto kern = attn_int8_resident_kernel<DH, ROWMAX, F8, PROBE>;
   HERO_SMEM_OPT_IN(h, kern, Cfg::SMEM_BYTES);
   const long long tiles = (long long)p.nqt * a->nh * a->B;
   const int grid = (int)(tiles < h->sm_count ? tiles : h->sm_count);
@@ -615,7 +645,12 @@ static hero_status launch_resident(hero_handle* h, const hero_attn_args* a, Attn
   return HERO_OK;
 }
 
-hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream) {
+hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream, bool probe) {
+  if (probe) {                                               // INT8 operands only (checked by the caller)
+    if (a->p_mode == HERO_P_ROWMAX)
+      return a->dh == 64 ? launch_resident<64, true, false, true>(h, a, p, stream) : launch_resident<128, true, false, true>(h, a, p, stream);
+    return a->dh == 64 ? launch_resident<64, false, false, true>(h, a, p, stream) : launch_resident<128, false, false, true>(h, a, p, stream);
+  }
   if (a->dtype == HERO_F8) {                               // static P quantizer only (checked by the caller)
     if (a->dh == 64) return launch_resident<64, false, true>(h, a, p, stream);
     return launch_resident<128, false, true>(h, a, p, stream);

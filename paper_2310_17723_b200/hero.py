@@ -60,6 +60,10 @@ class AttnArgs(C.Structure):
                 ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p), ("p_mode", C.c_int32)]
 
 
+class AttnProbe(C.Structure):
+    _fields_ = [("scores", C.c_void_p), ("p_codes", C.c_void_p), ("acc", C.c_void_p)]
+
+
 class DecodeAttnArgs(C.Structure):
     _fields_ = [("q", C.c_void_p), ("ld_q", C.c_int64), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
                 ("ld_kv", C.c_int64), ("batch_stride", C.c_int64), ("k_new", C.c_void_p), ("v_new", C.c_void_p),
@@ -101,7 +105,7 @@ EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_layer_forward_host_async", "hero_profile_begin",
            "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram",
-           "hero_int8_decode_attention", "hero_layer_decode", "hero_static_check")
+           "hero_int8_decode_attention", "hero_layer_decode", "hero_static_check", "hero_int8_attention_probe")
 
 _lib = None
 
@@ -123,6 +127,7 @@ def lib():
         L.hero_layernorm_quant.argtypes = [C.c_void_p, C.POINTER(LnArgs), C.c_void_p]
         L.hero_w8a8_linear.argtypes = [C.c_void_p, C.POINTER(LinearArgs), C.c_void_p]
         L.hero_int8_attention.argtypes = [C.c_void_p, C.POINTER(AttnArgs), C.c_void_p]
+        L.hero_int8_attention_probe.argtypes = [C.c_void_p, C.POINTER(AttnArgs), C.POINTER(AttnProbe), C.c_void_p]
         L.hero_int8_decode_attention.argtypes = [C.c_void_p, C.POINTER(DecodeAttnArgs), C.c_void_p]
         L.hero_mode_preset.argtypes = [C.c_int32, C.POINTER(C.c_int32 * 5)]
         L.hero_layer_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(C.c_size_t)]
@@ -221,13 +226,19 @@ class Handle:
         _check(lib().hero_w8a8_linear(self._h, C.byref(a), _stream(stream)))
 
     def hero_int8_attention(self, q, k, v, B, S, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0, s_p=1.0 / 255,
-                            mask="none", key_len=None, p_absmax=None, p_mode="static", stream=None):
+                            mask="none", key_len=None, p_absmax=None, p_mode="static", probe=None, stream=None):
         """q, k, v: 2-D torch views [B*S, nh*dh] sharing one leading dimension; out: hero.Tensor; p_absmax: float32[1]
-        running maximum of the softmax probabilities (F16 / BF16 core only)."""
+        running maximum of the softmax probabilities (F16 / BF16 core only).  probe = (scores int32 [B*nh, S, S] | None,
+        p_codes uint8 [B*nh, S, S] | None, acc int32 [B*S, nh*dh] | None) calls hero_int8_attention_probe instead."""
         assert q.stride(0) == k.stride(0) == v.stride(0) and q.dtype == k.dtype == v.dtype
         a = AttnArgs(q.data_ptr(), k.data_ptr(), v.data_ptr(), _DT[q.dtype], q.stride(0), B, S, nh, dh, s_q, s_k,
                      s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out, _ptr(p_absmax),
                      P_MODE[p_mode] if isinstance(p_mode, str) else p_mode)
+        if probe is not None:
+            scores, codes, acc = probe
+            pr = AttnProbe(_ptr(scores), _ptr(codes), _ptr(acc))
+            _check(lib().hero_int8_attention_probe(self._h, C.byref(a), C.byref(pr), _stream(stream)))
+            return
         _check(lib().hero_int8_attention(self._h, C.byref(a), _stream(stream)))
 
     def hero_int8_decode_attention(self, q, k_cache, v_cache, lens, max_len, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0,

@@ -16,8 +16,10 @@ def _ln_np(x, g, b, eps):
 
 
 class Stack:
-    def __init__(self, handle, shape, config_id, layer_cfgs, n_cal_seq=2, unit_ln=False):
-        """shape: workloads.Shape; layer_cfgs: list of prep.LayerConfig (one per layer, chained)."""
+    def __init__(self, handle, shape, config_id, layer_cfgs, n_cal_seq=2, unit_ln=False, prepared=None):
+        """shape: workloads.Shape; layer_cfgs: list of prep.LayerConfig (one per layer, chained).  `prepared`: optional
+        list of already prepared layers (the dictionaries `prep.prepare_layer` returns), one per config, used instead
+        of this constructor's own calibration and folding."""
         self.h, self.shape, self.cfgs = handle, shape, layer_cfgs
         self.M, self.H = shape.M, shape.H
         self.fp_torch = hero.TORCH_FP[shape.fp_dtype]
@@ -31,8 +33,12 @@ class Stack:
             if li == 0:
                 self.ln0 = (p["ln0_g"], p["ln0_b"])
                 cur = _ln_np(x_cal, p["ln0_g"].astype(np.float64), p["ln0_b"].astype(np.float64), cfg.eps) if post else x_cal
-            C, cur = prep.calibrate(cfg, p, cur, n_cal_seq, return_output=True)
-            layer = Layer(handle, prep.prepare_layer(cfg, p, C), workspace=ws)
+            if prepared is not None:
+                C = prepared[li]["C"]
+                layer = Layer(handle, prepared[li], workspace=ws)
+            else:
+                C, cur = prep.calibrate(cfg, p, cur, n_cal_seq, return_output=True)
+                layer = Layer(handle, prep.prepare_layer(cfg, p, C), workspace=ws)
             ws = layer.workspace
             self.layers.append(layer)
             self.params.append((None, C))

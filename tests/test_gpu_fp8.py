@@ -7,7 +7,7 @@ import torch
 from oracle import ops as O
 from oracle import quant as Q
 from paper_2310_17723_b200 import hero, workloads as W
-from gpu_util import f32, rel_err
+from gpu_util import f32, rel_err, assert_scales_close
 
 pytestmark = pytest.mark.gpu
 
@@ -52,7 +52,7 @@ def test_ln_quant_fp16_to_e4m3_twq_and_static(h, M, H):
     sc = torch.zeros(M, dtype=torch.float32, device="cuda")
     h.hero_layernorm_quant(hero.tensor(xd), f32(gam), f32(bet), 1e-5, hero.tensor(out, "twq", sc))
     h.check()
-    np.testing.assert_allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    assert_scales_close(sc.cpu().numpy(), want.row_scale, 1e-6, "e4m3 LN row scales")
     assert_f8_close(f8_vals(out), want.data, 1e-4, "LN^quant e4m3 TWQ")
     # static feature-wise scale, half the needed range so that the largest entries saturate at 448
     S = np.abs(O.layernorm(xin.real(), gam, bet, 1e-5)).max(0) / 448 / 2
@@ -77,7 +77,7 @@ def test_ln_quant_e4m3_residual_plus_e4m3_branch(h):
     h.hero_layernorm_quant(hero.tensor(to_f8(res.data), "twq", f32(res.row_scale)), f32(gam), f32(bet), 1e-5,
                            hero.tensor(out, "twq", sc), branch=hero.tensor(to_f8(br.data), "fwq", f32(S_o)))
     h.check()
-    np.testing.assert_allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    assert_scales_close(sc.cpu().numpy(), want.row_scale, 1e-6, "e4m3 LN row scales")
     assert_f8_close(f8_vals(out), want.data, 1e-4, "LN^quant e4m3 + e4m3")
 
 
@@ -244,14 +244,14 @@ def test_post_ln_layer_e4m3_stage_by_stage(h, gran_in, gran_attn, H, nh):
     want, _ = O.ln_quant([x_in, x_o], Lp["ln1_g"], Lp["ln1_b"], spec.eps, Lp["ln_mid_out"])
     assert_f8_close(x_mid.data, want.data, 1e-4, "x_mid")
     if gran_in == "twq":
-        np.testing.assert_allclose(x_mid.row_scale, want.row_scale, rtol=2e-6)
+        assert_scales_close(x_mid.row_scale, want.row_scale, 1e-6, "e4m3 x_mid scales")
     a = _like8(T["a"], bd.f8("a", F))
     assert_f8_close(a.data, OL._linear(Lp["fc1"], x_mid, spec.act).data, 2e-4, "a")
     x_2 = _like8(T["x_2"], bd.f8("x_2", H))
     assert_f8_close(x_2.data, OL._linear(Lp["fc2"], a, "none").data, 1e-4, "x_2")
     want, _ = O.ln_quant([x_mid, x_2], Lp["ln2_g"], Lp["ln2_b"], spec.eps, Lp["ln_final_out"])
     assert_f8_close(f8_vals(out), want.data, 1e-4, "x_out")
-    np.testing.assert_allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    assert_scales_close(sc.cpu().numpy(), want.row_scale, 1e-6, "e4m3 LN row scales")
     # ---- free-running against the oracle's own chain: an e4m3 value that flips moves by 6-12 % of itself
     got = f8_vals(out) * sc.cpu().numpy().astype(np.float64)[:, None]
     assert rel_err(got, T["x_out"].real()) < 6e-2
@@ -272,7 +272,7 @@ def test_pre_ln_causal_layer_e4m3(h, preset, H):
     bd = _F8Borders(h, layer, M)
     x_in8 = _like8(T["x_in"], bd.f8("x_in", H), bd.f32("x_in_scale"))
     assert_f8_close(x_in8.data, T["x_in"].data, 1e-4, "x_in")
-    np.testing.assert_allclose(x_in8.row_scale, T["x_in"].row_scale, rtol=2e-6)
+    assert_scales_close(x_in8.row_scale, T["x_in"].row_scale, 1e-6, "e4m3 x_in scales")
     qkv = _like8(T["qkv"], bd.f8("qkv", 3 * H))
     assert_f8_close(qkv.data, OL._linear(Lp["qkv"], x_in8, "none").data, 1e-4, "qkv")
     x_attn = _like8(T["x_attn"], bd.f8("x_attn", H))

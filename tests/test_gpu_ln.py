@@ -6,7 +6,7 @@ import torch
 from oracle import ops as O
 from oracle import quant as Q
 from paper_2310_17723_b200 import hero, workloads as W
-from gpu_util import dev, f32, qt_to_device, assert_int8_close, rel_err, TORCH_FP
+from gpu_util import dev, f32, qt_to_device, assert_int8_close, assert_scales_close, rel_err, TORCH_FP
 
 pytestmark = pytest.mark.gpu
 
@@ -62,7 +62,7 @@ def _compare(res, want, want_r, out_spec):
         else:
             assert_int8_close(res["out"], want.data, what="LN out")
             if out_spec.kind == "twq":
-                assert np.allclose(res["scale"], want.row_scale, rtol=2e-6, atol=0)
+                assert_scales_close(res["scale"], want.row_scale, 1e-6, "LN row scales")
     if want_r is not None:
         # fp16/bf16 store of an fp32 sum vs the oracle's fp64 sum: equal except rare 1-ulp ties
         d = np.abs(res["fp_out"] - want_r.data)
@@ -164,7 +164,7 @@ def test_embedding_gather_flavour(h):
                            seq_len=S, n_tokens=B * S)
     h.check()
     assert_int8_close(out.cpu().numpy(), want.data, what="embedding LN")
-    assert np.allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    assert_scales_close(sc.cpu().numpy(), want.row_scale, 1e-6, "embedding LN row scales")
 
 
 def test_embedding_gather_clamps_out_of_range_ids_and_reports_them(h):
@@ -193,7 +193,7 @@ def test_embedding_gather_clamps_out_of_range_ids_and_reports_them(h):
     assert e.value.status == hero.ERR_INVALID_ARG and "embedding id" in str(e.value)
     h.check()                                                          # the word was cleared
     assert_int8_close(out.cpu().numpy(), want.data, what="embedding LN, clamped ids")
-    assert np.allclose(sc.cpu().numpy(), want.row_scale, rtol=2e-6)
+    assert_scales_close(sc.cpu().numpy(), want.row_scale, 1e-6, "embedding LN row scales")
     # a position table shorter than the sequence is refused on the host
     with pytest.raises(hero.HeroError) as e:
         h.hero_layernorm_quant(hero.tensor(t_tok, "twq", f32(tok_s)), f32(gamma), f32(beta), 1e-12, hero.tensor(out, "twq", sc),
