@@ -1,11 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the W8A8 layer forward (ZeroQuant-HERO hot path) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c3|c4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5|c4|c3|c1] [--impl reference]
 
-A step is one pass of the whole hot path over one batch of synthetic input that is already resident in
-HBM.  One JSON line is printed by rank 0.  `--impl reference` times the CPU oracle instead (a deliberately
-plain fp64 program: context, not a target).
+A step is one pass of the whole hot path (the entry LN^quant and every layer of the workload) over one batch of
+synthetic input that is already resident in HBM.  The default workload is the largest single-GPU configuration, the
+24-layer BERT-large-shaped stack.  One JSON line is printed by rank 0.  With --gpus N > 1 and no torchrun environment
+the script starts its own N ranks (replicas: the path shards by sequence, nothing is exchanged).  `--impl reference`
+times the CPU oracle instead (a deliberately plain fp64 program: context, not a target).
 """
 import argparse
 import json
@@ -106,45 +108,71 @@ def attn_ln_fp_variant(cfgs):
     return out
 
 
-def kernel_table(shape, cfg):
-    """Per launch of one layer, in launch order: (name, family, algorithmic ops, algorithmic bytes)."""
+def kernel_table(shape, cfg, first=False):
+    """Per launch of one layer, in launch order: (name, family, algorithmic ops, algorithmic bytes); `first`: the
+    layer is preceded by the entry LN^quant of a post-LN workload."""
     M, H, F, S, nh, dh = shape.M, shape.H, shape.F, shape.S, shape.nh, shape.dh
     causal = shape.mask == "causal"
+    i8 = lambda module: cfg.mode[module] == "int8"
+    es = lambda is8: 1 if is8 else 2                          # bytes per element at a border
 
-    def gemm(name, K, N, module="qkv"):
-        fam = "gemm" if cfg.mode[module] == "int8" else "gemm_fp"
-        return (name, fam, 2.0 * M * N * K, float(M * K + N * K + M * N + 4 * M + 8 * N))
+    def gemm(name, K, N, module, out8):
+        fam = "gemm" if i8(module) else "gemm_fp"
+        e = es(i8(module))
+        return (name, fam, 2.0 * M * N * K, float(M * K * e + N * K * e + M * N * es(out8) + 4 * M + 8 * N))
+
+    def ln(name, res8, br8, out8, fp_out=False):
+        per = es(res8) + (es(br8) if br8 is not None else 0) + (es(out8) if out8 is not None else 0) + (2 if fp_out else 0)
+        return ("%s (%s%s->%s%s)" % (name, "i8" if res8 else "fp", "" if br8 is None else ("+i8" if br8 else "+fp"),
+                                      "" if out8 is None else ("i8" if out8 else "fp"), ",fp" if fp_out else ""),
+                "ln", 0.0, float(M * H * per + 8 * M))
     attn_ops = 4.0 * shape.B * nh * S * S * dh * (0.5 if causal else 1.0)
-    attn = ("attention", "attn", attn_ops, float(4 * M * H))
+    attn = ("attention" if i8("attn") else "attention (fp16)", "attn" if i8("attn") else "attn_fp", attn_ops,
+            float(M * H * (3 * es(i8("attn")) + es(i8("attn_out")))))
+    pre = shape.arch == "pre_ln"
     rows = []
-    if shape.arch == "pre_ln":
-        rows.append(("ln1 (fp->i8 twq)", "ln", 0.0, float(M * H * 3 + 4 * M)))
-    rows += [gemm("qkv gemm", H, 3 * H, "qkv"), attn, gemm("attn-out gemm", H, H, "attn_out")]
-    if shape.arch == "pre_ln":
-        rows.append(("add+ln2 (fp+i8->fp,i8)", "ln", 0.0, float(M * H * 6 + 4 * M)))
+    if first and not pre:
+        rows.append(ln("entry ln", False, None, i8("qkv")))
+    if pre:
+        rows.append(ln("ln1", False, None, i8("qkv")))
+    rows += [gemm("qkv gemm", H, 3 * H, "qkv", i8("attn")), attn, gemm("attn-out gemm", H, H, "attn_out", i8("attn_out"))]
+    if pre:
+        rows.append(ln("add+ln2", False, i8("attn_out"), i8("fc1"), fp_out=True))
     else:
-        rows.append(("ln1 (i8+i8->i8 twq)", "ln", 0.0, float(M * H * 3 + 8 * M)))
-    rows += [gemm("fc1 gemm + gelu^quant", H, F, "fc1"), gemm("fc2 gemm", F, H, "fc2")]
-    if shape.arch == "pre_ln":
-        rows.append(("closing add (fp+i8->fp)", "ln", 0.0, float(M * H * 5)))
+        rows.append(ln("ln1", i8("qkv"), i8("attn_out"), i8("fc1")))
+    rows += [gemm("fc1 gemm + gelu^quant", H, F, "fc1", i8("fc2")), gemm("fc2 gemm", F, H, "fc2", i8("fc2"))]
+    if pre:
+        rows.append(ln("closing add", False, i8("fc2"), None, fp_out=True))
     else:
-        rows.append(("ln2 (i8+i8->i8 twq)", "ln", 0.0, float(M * H * 3 + 8 * M)))
+        rows.append(ln("ln2", i8("fc1"), i8("fc2"), cfg.gran_out != "fp"))
     return rows
 
 
-
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the default workload's kernels, from one
-# ncu pass over this script (see profiles/dram_traffic_c3_layer.md).  ncu flushes L2 before every captured launch, so
-# reads equal the algorithmic input bytes and the outputs (all smaller than L2) are still cached when the kernel ends.
-NCU_TRAFFIC_C3 = {"qkv gemm": 15.8e6, "attention": 38.1e6, "attn-out gemm": 13.7e6, "ln1 (i8+i8->i8 twq)": 25.2e6,
-                  "fc1 gemm + gelu^quant": 18.6e6, "fc2 gemm": 54.8e6, "ln2 (i8+i8->i8 twq)": 25.3e6}
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernel function that dominates a
+# workload's step, each from one small ncu capture (one kernel, a few launches) recorded under profiles/; keyed by
+# (workload, kernel function).  These are constants of a recorded capture, not values this run measures.
+NCU_TRAFFIC = {}
 KERNEL_FUNCTION = {"qkv gemm": "gemm_pair_kernel<int8, no activation>", "attn-out gemm": "gemm_pair_kernel<int8, no activation>",
                    "fc2 gemm": "gemm_pair_kernel<int8, no activation>"}
+INT8_NOMINAL_TOPS = 4500.0          # dense INT8 rate of the part (datasheet figure without sparsity), for context
+
+
+def peak_regime(clocks, peaks):
+    """Which measured BF16 figure the timed region compares with: 'sustained' when the sampled clocks show the power
+    cap biting (reason active, or the median SM clock well below the maximum), else 'burst'."""
+    if not clocks or not clocks.get("sm_mhz"):
+        return "burst", "no clock samples"
+    mx = clocks.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0)
+    if "sw_power_cap" in (clocks.get("reasons") or []):
+        return "sustained", "sw_power_cap active during the timed region"
+    if clocks["sm_mhz"] < 0.93 * mx:
+        return "sustained", "median SM clock %.0f MHz below 0.93 x %.0f" % (clocks["sm_mhz"], mx)
+    return "burst", "SM clock at %.0f of %.0f MHz, no power cap" % (clocks["sm_mhz"], mx)
 
 
 def dominant_kernel(kern, workload, peaks, peak_kind, clocks):
     """The roofline object: rows of `kern` grouped by kernel function (the three GEMMs without activation are one
-    function launched three times per step), the group with the largest time share, aggregated over its launches."""
+    function launched three times per layer), the group with the largest time share, aggregated over its launches."""
     groups = {}
     for r in kern:
         key = KERNEL_FUNCTION.get(r["kernel"], r["kernel"])
@@ -153,64 +181,88 @@ def dominant_kernel(kern, workload, peaks, peak_kind, clocks):
     ms = sum(r["ms"] for r in rows)
     launches = sum(r["launches_per_step"] for r in rows)
     achieved = sum(r["achieved"] * r["ms"] for r in rows) / ms            # total work / total time
-    peak = rows[0]["peak"]
-    traffic = None
-    if workload == "c3" and all(r["kernel"] in NCU_TRAFFIC_C3 for r in rows):
-        traffic = sum(NCU_TRAFFIC_C3[r["kernel"]] for r in rows) / launches
-    src = {"tensor": "2 x bf16_tflops_sustained (INT8 runs at twice the BF16 rate; sustained: the kernel runs inside a long step)",
-           "hbm": "hbm_gbs", "alu": "148 SMs x 16 ex2 per clock x sampled SM clock"}[rows[0]["bound"]]
-    return {"bound": rows[0]["bound"], "achieved": achieved, "peak": peak, "unit": rows[0]["unit"], "frac": achieved / peak,
-            "traffic": traffic, "kernel": key, "members": [r["kernel"] for r in rows], "launches_per_step": launches,
-            "ms_per_step": round(ms, 5), "share": round(sum(r["share"] for r in rows), 4),
-            "peak_source": "%s: %s" % (peak_kind if rows[0]["bound"] != "alu" else "derived", src)}
+    bound = rows[0]["bound"]
+    out = {"bound": bound, "achieved": achieved, "peak": rows[0]["peak"], "unit": rows[0]["unit"], "frac": achieved / rows[0]["peak"],
+           "traffic": None, "kernel": key, "members": sorted(set(r["kernel"] for r in rows)), "launches_per_step": launches,
+           "ms_per_step": round(ms, 5), "share": round(sum(r["share"] for r in rows), 4)}
+    if bound == "tensor":
+        regime, why = peak_regime(clocks, peaks)
+        burst, sust = 2.0 * peaks["bf16_tflops"], 2.0 * peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        out.update(regime=regime, regime_why=why, frac_of_burst=achieved / burst, frac_of_sustained=achieved / sust,
+                   frac_of_nominal=achieved / INT8_NOMINAL_TOPS, peak_burst=burst, peak_sustained=sust, peak_nominal=INT8_NOMINAL_TOPS,
+                   peak_source="%s: 2 x bf16_tflops%s (INT8 runs at twice the BF16 rate of the same tensor cores; no INT8 figure is "
+                               "measured by the driver)" % (peak_kind, "_sustained" if regime == "sustained" else ""))
+    elif bound == "hbm":
+        out["peak_source"] = "%s: hbm_gbs" % peak_kind
+    else:
+        out["peak_source"] = "derived: 148 SMs x 16 ex2 per clock x sampled SM clock"
+    t = NCU_TRAFFIC.get((workload, key))
+    if t:
+        out["traffic"] = t["bytes_per_launch"]
+        out["traffic_source"] = t["source"]
+    return out
+
 
 # ------------------------------------------------------------------------------------------------
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
+    """nvidia-smi queries (read-only) every 100 ms in a child process; `stop` summarises the samples that fell inside
+    the window the caller marks with `begin()` .. `stop()`, i.e. while the GPU was working."""
     Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
 
     def __init__(self, index):
-        self.rows, self.proc = [], None
+        self.rows, self.proc, self.t_begin = [], None, None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
                                           "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
+            t0 = time.time()
+            while not self.rows and time.time() - t0 < 5.0:      # the first sample takes a moment: wait for it
+                time.sleep(0.02)
         except Exception:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.time(), line.strip()))
+
+    def begin(self):
+        self.t_begin = time.time()
 
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        t_end = time.time()
         time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
+        sm, mx, reasons, power = [], None, set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for t, r in self.rows:
+            if self.t_begin is not None and not (self.t_begin <= t <= t_end + 0.05):
+                continue
             f = [x.strip() for x in r.split(",")]
             if len(f) < 7:
                 continue
             try:
                 sm.append(float(f[0]))
                 mx = float(f[1])
+                power.append(float(f[2]))
             except ValueError:
                 continue
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm),
+                "power_w_max": max(power) if power else None, "window": "warm-up through the per-kernel pass (GPU busy throughout)"}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -242,11 +294,11 @@ def oracle_run(name, budget_s=12.0, repeats=1):
     def run(n_seq):
         x = W.activations(shape, cid, n_seq=n_seq)
         spec0, L0 = layers[0]
+        t0 = time.perf_counter()                              # a step = the entry LN^quant and every layer, as on the GPU
         if spec0.arch == "post_ln":
             cur_t = OL.entry_ln(O.fp_tensor(x, spec0.fp_dtype), ln0[0], ln0[1], spec0.eps, L0["ln_in_out"])
         else:
             cur_t = O.fp_tensor(x, spec0.fp_dtype)
-        t0 = time.perf_counter()
         for spec, Lp in layers:
             cur_t = OL.layer_forward(Lp, cur_t, B=n_seq)["x_out"]
         return time.perf_counter() - t0
@@ -289,6 +341,50 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
+def sweep_extra(h, peaks):
+    """The metric's second and third parts on the standalone-kernel sweep: INT8 GeMM^quant TOP/s at M >= 8192 and
+    LN^quant GB/s at 65536 rows, as fractions of the measured peaks (burst: each kernel is timed alone)."""
+    import torch
+    from paper_2310_17723_b200 import microbench as MB, workloads as W
+    MB.QUIET = True
+    i8_burst = 2.0 * peaks["bf16_tflops"]
+    out = {"gemm_int8": [], "ln_quant": [], "peaks": {"int8_tops_burst": i8_burst, "int8_tops_nominal": INT8_NOMINAL_TOPS, "hbm_gbs": peaks["hbm_gbs"]},
+           "note": "each kernel timed alone over rotating buffers larger than L2, CUDA events; GEMM epilogue = dequant + bias + "
+                   "requant to INT8; LN^quant algorithmic bytes 3 per element"}
+    for K, N in W.GEMM_SWEEP_KN:
+        for M in (8192, 32768):
+            r = MB.bench_gemm(h, M, K, N, "none", False, 10)
+            out["gemm_int8"].append({"M": M, "K": K, "N": N, "tops": round(r["tops"], 1), "frac_of_burst": round(r["tops"] / i8_burst, 3),
+                                     "frac_of_nominal": round(r["tops"] / INT8_NOMINAL_TOPS, 3)})
+            torch.cuda.empty_cache()
+    for H in W.LN_SWEEP_H:
+        for kind in ("f16", "i8"):
+            r = MB.bench_ln(h, 65536, H, kind, 20)
+            out["ln_quant"].append({"M": 65536, "H": H, "inputs": "fp16" if kind == "f16" else "int8 twq + int8 fwq", "gbs": round(r["gbs"], 0),
+                                    "frac_of_hbm": round(r["gbs"] / peaks["hbm_gbs"], 3)})
+            torch.cuda.empty_cache()
+    try:
+        # a library INT8 GEMM of the same size as the driver's BF16 probe, for a MEASURED INT8 figure beside the derived
+        # 2 x BF16 one (measurement only: nothing of the product path goes through it)
+        a = torch.randint(-127, 128, (8192, 8192), device="cuda", dtype=torch.int8)
+        b = torch.randint(-127, 128, (8192, 8192), device="cuda", dtype=torch.int8).t()
+        for _ in range(3):
+            torch._int_mm(a, b)
+        best = 1e9
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); torch._int_mm(a, b); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        out["peaks"]["int8_tops_library_gemm_8192"] = round(2.0 * 8192 ** 3 / (best * 1e-3) / 1e12, 1)
+        del a, b
+    except Exception as e:                                     # the figure is optional context
+        out["peaks"]["int8_tops_library_gemm_8192"] = None
+        out["peaks"]["int8_library_gemm_note"] = "torch._int_mm unavailable: %s" % str(e)[:80]
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -310,24 +406,35 @@ def run_ours(args):
     from paper_2310_17723_b200.model import Stack
 
     shape, cid, cfgs, desc = workload_spec(args.workload)
+    post = shape.arch == "post_ln"
     h = hero.Handle()
     stack = Stack(h, shape, cid, cfgs, n_cal_seq=1 if shape.M * shape.H > 2 ** 25 else 2)
     # every rank works on its own batch (replicas: the path shards by sequence, no exchange step)
     x_host = torch.from_numpy(W.activations(shape, cid, tensor=replicas.batch_tensor_index(rank))).to(stack.fp_torch)
     x_dev = x_host.cuda()
-    stack.set_input(x_dev)
-    h.check()
     flush = torch.empty(512 * 1024 * 1024, dtype=torch.int8, device="cuda")     # > 126 MB L2
     stream = torch.cuda.current_stream()
+    # a step = the whole hot path on one batch: the entry LN^quant (post-LN workloads: it stands for the embedding
+    # LayerNorm of Eq. 6-7 and turns the FP16 activations into layer 0's INT8 input) and every layer
+    sd_full = stack.desc(entry_in=hero.tensor(x_dev)) if post else stack.desc()
+    sd_layers = stack.desc()
+    if not post:
+        stack.set_input(x_dev)
 
     def step():
-        stack.forward()
+        h.hero_stack_forward(sd_full, stack.workspace)
+
+    def step_layers_only():
+        h.hero_stack_forward(sd_layers, stack.workspace)
 
     sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.begin()
     for _ in range(max(args.warmup, 3)):
         flush.zero_()
         step()
     torch.cuda.synchronize()
+    h.check()
     n0 = h.launches
     step()
     launches_per_step = h.launches - n0
@@ -340,7 +447,7 @@ def run_ours(args):
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
             with torch.cuda.graph(graph, stream=side):
-                stack.forward()
+                eager_step()
         torch.cuda.synchronize()
 
         def step():
@@ -350,28 +457,36 @@ def run_ours(args):
             step()
         torch.cuda.synchronize()
 
-    # ---- timed region: K steps, each bracketed by events on the launching stream, L2 flushed in between
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    def timed(fn, steps):
+        """`steps` calls of fn, each bracketed by events on the launching stream, L2 flushed before each (outside the
+        event pairs).  Returns the summed device milliseconds."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for k in range(steps):
+            flush.zero_()
+            ev[k][0].record(stream)
+            fn()
+            ev[k][1].record(stream)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in ev)
+
+    # ---- timed region: K steps
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
     n0 = h.launches
     replayed[0] = 0
-    for k in range(args.steps):
-        flush.zero_()
-        ev[k][0].record(stream)
-        step()
-        ev[k][1].record(stream)
-    torch.cuda.synchronize()
+    my_ms = timed(step, args.steps)
     if dist:
         dist.barrier()
     wall = time.perf_counter() - wall0
     gpu_launches = h.launches - n0 + replayed[0]
     h.check()
-    total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), dist, "cuda")
+    total_ms = replicas.max_over_ranks(my_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
     value = replicas.job_throughput(shape.M, args.steps, world, total_ms * 1e-3)
+    # the same steps without the entry LN^quant (the layers alone, their INT8 input already in place)
+    layers_only_ms = timed(step_layers_only, args.steps) / args.steps if post else None
 
     # ---- per-kernel device times (a second, instrumented pass: event pairs around every launch)
     kern = []
@@ -386,10 +501,11 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     if rank == 0:
         table = []
-        for cfg in cfgs:
-            table += kernel_table(shape, cfg)
+        for li, cfg in enumerate(cfgs):
+            table += kernel_table(shape, cfg, first=(li == 0))
         assert len(table) == launches_per_step, (len(table), launches_per_step)
-        int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        regime, _why = peak_regime(clocks, peaks)
+        int8_peak = 2.0 * (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) if regime == "sustained" else peaks["bf16_tflops"])
         merged = {}
         for i, (name, fam, ops, nbytes) in enumerate(table):
             ms = [recs[j][1] for j in range(i, len(recs), launches_per_step)]
@@ -399,10 +515,11 @@ def run_ours(args):
                 merged[key] = (merged[key][0] + avg, merged[key][1] + ops, merged[key][2] + nbytes, merged[key][3] + 1)
             else:
                 merged[key] = (avg, ops, nbytes, 1)
+        mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
         for (name, fam), (avg, ops, nbytes, cnt) in merged.items():
             row = {"kernel": name if fam != "gemm_fp" else name + " (fp16)", "ms": round(avg, 5), "share": None, "launches_per_step": cnt}
             if fam == "gemm":
-                row.update(bound="tensor", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak, unit="TFLOP/s")
+                row.update(bound="tensor", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak, unit="TOP/s")
             elif fam == "gemm_fp":
                 row.update(bound="tensor", achieved=ops / (avg * 1e-3) / 1e12, peak=int8_peak / 2, unit="TFLOP/s")
             elif fam == "ln":
@@ -411,7 +528,6 @@ def run_ours(args):
                 # bound by the special-function unit: one exponential per score and sweep that needs it
                 # (ops = 4 dh per score, so scores = ops / (4 dh)); peak = 16 ex2 per clock and SM at the sampled clock
                 scores = ops / (4.0 * shape.dh)
-                mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
                 row.update(bound="alu", achieved=scores / (avg * 1e-3) / 1e12, peak=148 * 16 * mhz * 1e6 / 1e12,
                            unit="Texp/s", tensor_tops=ops / (avg * 1e-3) / 1e12)
             row["frac"] = row["achieved"] / row["peak"]
@@ -421,97 +537,80 @@ def run_ours(args):
             r["share"] = round(r["ms"] / tot, 4)
         roof = dominant_kernel(kern, args.workload, peaks, peak_kind, clocks)
 
-    # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
-    e2e = None
-    if len(cfgs) == 1 and shape.arch == "post_ln":
-        t_in, s_in, d_in = stack.bufs[0]
-        t_out, s_out, d_out = stack.bufs[1]
-        hin = t_in.cpu().pin_memory()
-        hout = torch.empty_like(t_out, device="cpu").pin_memory()
-        gin, gout = cfgs[0].gran_in, cfgs[0].gran_out
-        hsin = s_in.cpu().pin_memory() if s_in is not None else None
-        hsout = torch.empty_like(s_out, device="cpu").pin_memory() if s_out is not None else None
-        in_host = hero.host_tensor(hin, gin, hsin)
-        out_host = hero.host_tensor(hout, gout, hsout)
-        layer = stack.layers[0]
+    # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region:
+    # hero_stack_forward_host_async = H2D of the FP activations, entry LN^quant, every layer, D2H of the output
+    # (payload and, for a token-wise output, its row scales).  Three steps in flight, each on its own stream with its
+    # own chained device buffers, staging tensor, workspace and pinned output: one step's copies overlap another's
+    # kernels.  A slot is synchronised (its result is then in host memory) before it is reused.
+    DEPTH = 3 if shape.M * shape.H * 2 <= (1 << 28) else 2
+    hin = x_host.pin_memory()
+    t_out, s_out, _d = stack.bufs[-1]
+    g_out = "fp" if t_out.dtype in (torch.float16, torch.bfloat16) else cfgs[-1].gran_out
+    slots = []
+    for _ in range(DEPTH):
+        edges = stack.make_edges()
+        stage = torch.empty_like(x_dev)
+        if post:
+            sd = stack.desc(entry_in=hero.tensor(stage), edges=edges)
+        else:
+            edges[0] = (stage, None, hero.tensor(stage))
+            sd = stack.desc(edges=edges)
+        ho = torch.empty_like(edges[-1][0], device="cpu").pin_memory()
+        hso = torch.empty(shape.M, dtype=torch.float32).pin_memory() if g_out == "twq" else None
+        slots.append({"sd": sd, "host": hero.host_tensor(ho, g_out, hso if g_out == "twq" else None), "keep": (edges, stage, ho, hso),
+                      "ws": torch.empty_like(stack.workspace), "stream": torch.cuda.Stream(), "busy": False})
+    in_host = hero.host_tensor(hin)
+    e2e_k = [0]
 
-        # three steps in flight, each on its own stream with its own device staging tensors, workspace and pinned
-        # output buffer: one step's copies overlap another step's kernels.  A slot is synchronised (its result is
-        # then in host memory) before it is reused, so every step's input is copied in and its output read back.
-        DEPTH = 3
-        slots = []
-        for _ in range(DEPTH):
-            ti = torch.empty_like(t_in)
-            si = torch.empty_like(s_in) if (s_in is not None and gin == "twq") else s_in
-            to = torch.empty_like(t_out)
-            so = torch.empty_like(s_out) if (s_out is not None and gout == "twq") else s_out
-            ho = torch.empty_like(t_out, device="cpu").pin_memory()
-            hso = torch.empty_like(s_out, device="cpu").pin_memory() if s_out is not None else None
-            slots.append({"in": hero.tensor(ti, gin, si), "out": hero.tensor(to, gout, so), "host": hero.host_tensor(ho, gout, hso),
-                          "ws": torch.empty_like(layer.workspace), "stream": torch.cuda.Stream(), "busy": False})
-        e2e_k = [0]
-
-        def e2e_step():
-            sl = slots[e2e_k[0] % DEPTH]
-            e2e_k[0] += 1
-            if sl["busy"]:
-                sl["stream"].synchronize()
-            h.hero_layer_forward_host_async(layer.desc, in_host, sl["host"], sl["in"], sl["out"], sl["ws"], stream=sl["stream"])
-            sl["busy"] = True
-        h2d = hin.numel() + (hsin.numel() * 4 if gin == "twq" else 0)
-        d2h = hout.numel() * hout.element_size() + (hsout.numel() * 4 if gout == "twq" else 0)
-    else:
-        t_in = stack.bufs[0][0]
-        t_out = stack.bufs[-1][0]
-        hin = x_host.pin_memory()
-        hout = torch.empty_like(t_out, device="cpu").pin_memory()
-
-        def e2e_step():
-            t_in.copy_(hin, non_blocking=True)
-            stack.forward()
-            hout.copy_(t_out, non_blocking=True)
-            torch.cuda.synchronize()
-        h2d = hin.numel() * hin.element_size()
-        d2h = hout.numel() * hout.element_size()
+    def e2e_step():
+        sl = slots[e2e_k[0] % DEPTH]
+        e2e_k[0] += 1
+        if sl["busy"]:
+            sl["stream"].synchronize()
+        h.hero_stack_forward_host_async(sl["sd"], in_host, sl["host"], sl["ws"], stream=sl["stream"])
+        sl["busy"] = True
+    h2d = hin.numel() * hin.element_size()
+    d2h = t_out.numel() * t_out.element_size() + (shape.M * 4 if g_out == "twq" else 0)
     for _ in range(3):
         e2e_step()
+    torch.cuda.synchronize()
     if dist:
         dist.barrier()
-    torch.cuda.synchronize()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         e2e_step()
     torch.cuda.synchronize()
     e2e_s = replicas.max_over_ranks(time.perf_counter() - t0, dist, "cuda")
-    e2e = {"value": replicas.job_throughput(shape.M, args.steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-           "steps_in_flight": 3 if (len(cfgs) == 1 and shape.arch == "post_ln") else 1}
+    e2e = {"value": replicas.job_throughput(shape.M, args.steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(d2h), "steps_in_flight": DEPTH, "api": "hero_stack_forward_host_async (pinned host buffers)",
+           "ms_per_step": 1e3 * e2e_s / args.steps}
     h.check()
+    del slots
+    torch.cuda.empty_cache()
 
     fp_path = None
     mixed_path = None
+    extra = None
     if rank == 0 and world == 1 and not args.no_fp_path:
         # the same layer(s) in other module modes, through the same library and the same timing loop
-        del stack
+        del stack, sd_full, sd_layers
         torch.cuda.empty_cache()
 
         def time_variant(vcfgs):
             vstack = Stack(h, shape, cid, vcfgs, n_cal_seq=1)
-            vstack.set_input(x_dev)
+            vsd = vstack.desc(entry_in=hero.tensor(x_dev)) if post else vstack.desc()
+            if not post:
+                vstack.set_input(x_dev)
+            run = lambda: h.hero_stack_forward(vsd, vstack.workspace)
             for _ in range(3):
                 flush.zero_()
-                vstack.forward()
+                run()
             torch.cuda.synchronize()
-            fev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-            for k in range(args.steps):
-                flush.zero_()
-                fev[k][0].record(stream)
-                vstack.forward()
-                fev[k][1].record(stream)
-            torch.cuda.synchronize()
+            ms = timed(run, args.steps) / args.steps
             h.check()
-            del vstack
+            del vstack, vsd
             torch.cuda.empty_cache()
-            return sum(a.elapsed_time(b) for a, b in fev) / args.steps
+            return ms
 
         fms = time_variant(fp_variant(cfgs))                 # every module in FP16 / BF16
         fp_path = {"value": shape.M / (fms * 1e-3), "unit": UNIT, "ms_per_step": fms, "dtype": shape.fp_dtype,
@@ -522,6 +621,8 @@ def run_ours(args):
             mms = time_variant(attn_ln_fp_variant(cfgs))
             mixed_path = {"modes": "qkv, attention, fc1 in BF16; attention-output linear, fc2 INT8", "value": shape.M / (mms * 1e-3),
                           "unit": UNIT, "ms_per_step": mms, "w8a8_speedup": ms_per_step and mms / ms_per_step}
+    if rank == 0 and world == 1 and not args.no_extra:
+        extra = sweep_extra(h, peaks)
     if rank != 0:
         if dist:
             dist.destroy_process_group()
@@ -534,17 +635,60 @@ def run_ours(args):
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
             "data": "synthetic",
             "config": {"workload": desc, "tokens_per_step_per_gpu": shape.M, "l2": "flushed between timed steps (512 MiB write)",
-                       "launch": "CUDA graph replay of the step's launches" if args.graph else "one C-ABI call per layer, 7-8 kernel launches each",
+                       "step": ("entry LN^quant + %d layer(s)" % len(cfgs)) if post else "%d pre-LN layer(s)" % len(cfgs),
+                       "launch": "CUDA graph replay of the step's launches" if args.graph else
+                                 "one C-ABI call per step (hero_stack_forward), %d kernel launches" % launches_per_step,
                        "timing": "CUDA events per step on the launching stream, max over ranks",
                        "parallelism": "replicas x%d (sequence-sharded, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "kernels": kern,
             "kernels_note": "per-launch times come from a second pass with an event pair around every launch, which serialises the "
                             "launches (no programmatic overlap): their sum exceeds ms_per_step, so the fractions are lower bounds",
             "cpu_baseline": cpu, "fp16_path": fp_path, "wall_s_timed_region": wall}
+    if layers_only_ms is not None:
+        line["without_entry_ln"] = {"ms_per_step": layers_only_ms, "value": shape.M / (layers_only_ms * 1e-3), "unit": UNIT,
+                                    "note": "the layers alone, their INT8 input already in place (one rank's device time)"}
     if mixed_path:
         line["attention_and_ln_bf16_path"] = mixed_path
+    if extra:
+        line["extra"] = extra
     print(json.dumps(line), flush=True)
     if dist:
+        dist.destroy_process_group()
+
+
+def self_spawn(args):
+    """`--gpus N` with N > 1 outside a torchrun environment: start N ranks of this script (one per GPU, rendezvous on
+    127.0.0.1); rank 0 prints the JSON line.  Returns the launcher's exit code."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_rendezvous_only(args):
+    """The multi-rank plumbing without the workload (also what the CPU test drives): process group, barrier, maximum
+    over ranks, one JSON line from rank 0.  NCCL when a GPU per rank is visible, gloo otherwise."""
+    import torch
+    import torch.distributed as dist
+    from paper_2310_17723_b200 import replicas
+    rank, local, world = replicas.rank_info()
+    use_cuda = torch.cuda.is_available() and torch.cuda.device_count() >= world
+    if world > 1:
+        if use_cuda:
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group("gloo")
+        dist.barrier()
+    t = replicas.max_over_ranks(1.0 + rank, dist if world > 1 else None, "cuda" if use_cuda else "cpu")
+    if rank == 0:
+        print(json.dumps({"rendezvous": "ok", "n_gpus": world, "backend": "nccl" if use_cuda else "gloo", "max_over_ranks": t,
+                          "value": replicas.job_throughput(100, 1, world, t)}), flush=True)
+    if world > 1:
         dist.destroy_process_group()
 
 
@@ -554,12 +698,18 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c1", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c3", "c4", "c5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp-path", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the standalone-kernel sweep figures")
     ap.add_argument("--graph", action="store_true", help="replay the step's launches from a CUDA graph (latency-bound workloads)")
+    ap.add_argument("--rendezvous-only", action="store_true", help="only start the ranks, meet and print (no workload)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(self_spawn(args))
+    if args.rendezvous_only:
+        run_rendezvous_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

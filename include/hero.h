@@ -402,6 +402,33 @@ hero_status hero_layer_forward_host_async(hero_handle* h, const hero_layer_desc*
                                           const hero_tensor* out_host, const hero_tensor* in_dev,
                                           const hero_tensor* out_dev, void* workspace, size_t workspace_bytes, void* stream);
 
+/* A stack of layers (the paper's models are stacks of the layer of Sec. 2.2.2-2.2.3 behind the embedding LN^quant of
+ * Sec. 2.2.1): host-side sequencing only, one hero_layer_forward per layer on `stream`, layer i reading edges[i] and
+ * writing edges[i + 1], all layers sharing one workspace (at least the largest hero_layer_workspace_bytes among them).
+ *   layers   : host array [n_layers] of layer descriptors
+ *   edges    : host array [n_layers + 1] of DEVICE tensors, typed as each layer's `in` / `out` (hero_layer_forward)
+ *   pending  : host array [n_layers] or NULL: pre-LN only, the branch still to be added to layer i's input
+ *   entry_in : optional DEVICE tensor [M, H] F16 / BF16; when present the entry LN^quant (plain flavour of Eq. 6-7,
+ *              entry_gamma / entry_beta / entry_eps) turns it into edges[0] before layer 0 runs. */
+typedef struct {
+  int32_t n_layers;
+  const hero_layer_desc* layers;
+  const hero_tensor* edges;
+  const hero_tensor* pending;
+  hero_tensor entry_in;
+  const float* entry_gamma;
+  const float* entry_beta;
+  float entry_eps;
+} hero_stack_desc;
+hero_status hero_stack_forward(hero_handle* h, const hero_stack_desc* stack, void* workspace, size_t workspace_bytes,
+                               void* stream);
+/* The same with HOST activation buffers, enqueued on `stream` without a final synchronisation: in_host is copied into
+ * entry_in (when the stack has an entry LN^quant) or into edges[0] (payload and, for a token-wise tensor, its row
+ * scales), the stack runs, and edges[n_layers] is copied into out_host, which is valid once the caller has
+ * synchronised the stream.  Host buffers should be page-locked.  Nothing is allocated. */
+hero_status hero_stack_forward_host_async(hero_handle* h, const hero_stack_desc* stack, const hero_tensor* in_host,
+                                          const hero_tensor* out_host, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The layer forward for callers that cannot allocate device memory (the paper has no counterpart: it describes
  * no software interface).  Who needs it: code that runs inside another framework's fixed memory plan, real-time
  * or plugin paths where an allocation might block or fail late, processes that own only the buffers they were

@@ -302,6 +302,60 @@ extern "C" hero_status hero_layer_forward_host_async(hero_handle* h, const hero_
   return HERO_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------------------
+// A stack of layers: host-side sequencing of hero_layer_forward over chained edge tensors, with an optional entry LN^quant.
+namespace hero {
+static hero_status copy_tensor(const hero_tensor& dst, const hero_tensor& src, cudaMemcpyKind kind, cudaStream_t s, const char* what) {
+  HERO_REQUIRE(dst.data && src.data && dst.dtype == src.dtype && dst.rows == src.rows && dst.cols == src.cols, HERO_ERR_INVALID_ARG,
+               "%s: host and device tensors must agree in type and shape", what);
+  const size_t es = dtype_size(dst.dtype);
+  HERO_REQUIRE(es != 0, HERO_ERR_INVALID_ARG, "%s: unknown dtype", what);
+  if (dst.ld == dst.cols && src.ld == src.cols)
+    HERO_CUDA(cudaMemcpyAsync(dst.data, src.data, (size_t)dst.rows * dst.cols * es, kind, s));
+  else
+    HERO_CUDA(cudaMemcpy2DAsync(dst.data, dst.ld * es, src.data, src.ld * es, dst.cols * es, dst.rows, kind, s));
+  if (is_q8(dst.dtype) && dst.gran == HERO_GRAN_TWQ) {      // token-wise scales travel with the payload; calibrated ones live on the device
+    HERO_REQUIRE(dst.scale && src.scale, HERO_ERR_INVALID_ARG, "%s: a token-wise tensor needs its row scales on both sides", what);
+    HERO_CUDA(cudaMemcpyAsync(dst.scale, src.scale, (size_t)dst.rows * sizeof(float), kind, s));
+  }
+  return HERO_OK;
+}
+}  // namespace hero
+
+extern "C" hero_status hero_stack_forward(hero_handle* h, const hero_stack_desc* sd, void* workspace, size_t workspace_bytes,
+                                          void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(h && sd && sd->n_layers > 0 && sd->layers && sd->edges, HERO_ERR_INVALID_ARG, "hero_stack_forward: bad stack descriptor");
+  hero_status st;
+  if (sd->entry_in.data) {
+    hero_ln_args a;
+    memset(&a, 0, sizeof(a));
+    a.residual = sd->entry_in;
+    a.gamma = sd->entry_gamma; a.beta = sd->entry_beta; a.eps = sd->entry_eps;
+    a.out = sd->edges[0];
+    if ((st = hero_layernorm_quant(h, &a, stream)) != HERO_OK) return st;
+  }
+  for (int32_t i = 0; i < sd->n_layers; ++i) {
+    const hero_tensor* pend = (sd->pending && sd->pending[i].data) ? &sd->pending[i] : nullptr;
+    if ((st = hero_layer_forward(h, &sd->layers[i], &sd->edges[i], pend, &sd->edges[i + 1], workspace, workspace_bytes, stream)) != HERO_OK)
+      return st;
+  }
+  return HERO_OK;
+}
+
+extern "C" hero_status hero_stack_forward_host_async(hero_handle* h, const hero_stack_desc* sd, const hero_tensor* in_host,
+                                                     const hero_tensor* out_host, void* workspace, size_t workspace_bytes,
+                                                     void* stream) {
+  using namespace hero;
+  HERO_REQUIRE(h && sd && in_host && out_host && sd->n_layers > 0 && sd->edges, HERO_ERR_INVALID_ARG,
+               "hero_stack_forward_host: NULL argument");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  hero_status st;
+  if ((st = copy_tensor(sd->entry_in.data ? sd->entry_in : sd->edges[0], *in_host, cudaMemcpyHostToDevice, s, "stack input")) != HERO_OK) return st;
+  if ((st = hero_stack_forward(h, sd, workspace, workspace_bytes, stream)) != HERO_OK) return st;
+  return copy_tensor(*out_host, sd->edges[sd->n_layers], cudaMemcpyDeviceToHost, s, "stack output");
+}
+
 extern "C" hero_status hero_layer_forward_host(hero_handle* h, const hero_layer_desc* d, const hero_tensor* in_host,
                                                const hero_tensor* out_host, const hero_tensor* in_dev,
                                                const hero_tensor* out_dev, void* workspace, size_t workspace_bytes,

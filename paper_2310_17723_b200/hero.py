@@ -88,6 +88,12 @@ class LayerDesc(C.Structure):
                 ("p_mode", C.c_int32), ("payload", C.c_int32)]
 
 
+class StackDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("layers", C.POINTER(LayerDesc)), ("edges", C.POINTER(Tensor)),
+                ("pending", C.POINTER(Tensor)), ("entry_in", Tensor), ("entry_gamma", C.c_void_p), ("entry_beta", C.c_void_p),
+                ("entry_eps", C.c_float)]
+
+
 class KvCache(C.Structure):
     _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("ld_kv", C.c_int64), ("batch_stride", C.c_int64),
                 ("len", C.c_void_p), ("max_len", C.c_int32)]
@@ -105,7 +111,8 @@ EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero
            "hero_layernorm_quant", "hero_w8a8_linear", "hero_int8_attention", "hero_mode_preset",
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_layer_forward_host_async", "hero_profile_begin",
            "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram",
-           "hero_int8_decode_attention", "hero_layer_decode", "hero_static_check", "hero_int8_attention_probe")
+           "hero_int8_decode_attention", "hero_layer_decode", "hero_static_check", "hero_int8_attention_probe", "hero_stack_forward",
+           "hero_stack_forward_host_async")
 
 _lib = None
 
@@ -147,6 +154,9 @@ def lib():
         L.hero_layer_forward_static.argtypes = [C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                                 C.POINTER(Tensor), C.c_void_p]
         L.hero_static_check.argtypes = [C.c_void_p]
+        L.hero_stack_forward.argtypes = [C.c_void_p, C.POINTER(StackDesc), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hero_stack_forward_host_async.argtypes = [C.c_void_p, C.POINTER(StackDesc), C.POINTER(Tensor), C.POINTER(Tensor),
+                                                    C.c_void_p, C.c_size_t, C.c_void_p]
         L.hero_profile_begin.argtypes = [C.c_void_p, C.c_int32]
         L.hero_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         _lib = L
@@ -296,6 +306,16 @@ class Handle:
                                              C.byref(in_dev), C.byref(out_dev), C.c_void_p(workspace.data_ptr()),
                                              workspace.numel(), _stream(stream)))
 
+    def hero_stack_forward(self, stack_desc, workspace, stream=None):
+        """stack_desc: hero.StackDesc (see `stack_desc`); one C call runs the entry LN^quant (if any) and every layer."""
+        _check(lib().hero_stack_forward(self._h, C.byref(stack_desc), C.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                        _stream(stream)))
+
+    def hero_stack_forward_host_async(self, stack_desc, in_host, out_host, workspace, stream=None):
+        """Host-buffer variant: H2D of in_host, the stack, D2H into out_host, all enqueued on the stream."""
+        _check(lib().hero_stack_forward_host_async(self._h, C.byref(stack_desc), C.byref(in_host), C.byref(out_host),
+                                                   C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)))
+
     def profile_begin(self, max_launches):
         self._prof_cap = int(max_launches)
         _check(lib().hero_profile_begin(self._h, self._prof_cap))
@@ -323,6 +343,20 @@ class Handle:
         pend = C.byref(pending) if pending is not None else None
         _check(lib().hero_layer_decode(self._h, C.byref(desc), C.byref(kv), C.byref(x_in), pend, C.byref(out),
                                        C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(stream)))
+
+
+def stack_desc(layer_descs, edges, entry_in=None, entry_gamma=None, entry_beta=None, entry_eps=0.0):
+    """hero_stack_desc over a list of LayerDesc and a list of len(layer_descs) + 1 hero.Tensor edges (device tensors)."""
+    n = len(layer_descs)
+    assert len(edges) == n + 1
+    sd = StackDesc()
+    layers = (LayerDesc * n)(*layer_descs)
+    e = (Tensor * (n + 1))(*edges)
+    sd.n_layers, sd.layers, sd.edges, sd.pending = n, layers, e, None
+    sd.entry_in = entry_in if entry_in is not None else tensor(None)
+    sd.entry_gamma, sd.entry_beta, sd.entry_eps = _ptr(entry_gamma), _ptr(entry_beta), float(entry_eps)
+    sd._keep = (layers, e, list(layer_descs), list(edges), entry_in, entry_gamma, entry_beta)
+    return sd
 
 
 def host_tensor(t, gran="none", scale=None):

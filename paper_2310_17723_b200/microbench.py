@@ -62,6 +62,14 @@ def _time(fn, n_buf, iters):
     return e0.elapsed_time(e1) / iters * 1e-3
 
 
+QUIET = False       # set by callers that only want the returned figures (bench.py prints one JSON line and nothing else)
+
+
+def _say(text):
+    if not QUIET:
+        print(text, flush=True)
+
+
 def bench_ln(h, M, H, kind, iters, out_gran="twq"):
     """kind 'f16': FP16 -> INT8 TWQ (entry flavour); 'i8': INT8 TWQ + INT8 FWQ -> INT8 TWQ (Eq. 19); out_gran 'fwq': the
     output is quantized with a calibrated per-feature scale instead (Eq. 4)."""
@@ -82,8 +90,9 @@ def bench_ln(h, M, H, kind, iters, out_gran="twq"):
     t = _time(lambda i: h.hero_layernorm_quant(ins[i][0], g, b, 1e-5, hero.tensor(outs[i], out_gran, sc), branch=ins[i][1]), n, iters)
     hbm, _, src = _peaks()
     gbs = M * H * 3 / t / 1e9
-    print("LN^quant %s%s M=%d H=%d: %.1f us, %.0f GB/s (algorithmic 3 B/element), %.2f of %s copy bandwidth"
-          % (kind, "" if out_gran == "twq" else " -> " + out_gran, M, H, t * 1e6, gbs, gbs / hbm, src), flush=True)
+    _say("LN^quant %s%s M=%d H=%d: %.1f us, %.0f GB/s (algorithmic 3 B/element), %.2f of %s copy bandwidth"
+         % (kind, "" if out_gran == "twq" else " -> " + out_gran, M, H, t * 1e6, gbs, gbs / hbm, src))
+    return {"us": t * 1e6, "gbs": gbs}
 
 
 def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
@@ -112,9 +121,10 @@ def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
     es = 2 if fp else 1
     gbs = (M * K * es + N * K * es + M * N * es + 4 * M + 8 * N) / t / 1e9
     hbm = _peaks()[0]
-    print("GeMM^quant %s M=%d K=%d N=%d act=%s: %.1f us, %.0f TOP/s, %.2f of 2 x %s BF16 peak%s; %.0f GB/s, %.2f of copy bandwidth"
-          % ("bf16" if fp else ("e4m3" if f8 else "i8"), M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else "",
-             gbs, gbs / hbm), flush=True)
+    _say("GeMM^quant %s M=%d K=%d N=%d act=%s: %.1f us, %.0f TOP/s, %.2f of 2 x %s BF16 peak%s; %.0f GB/s, %.2f of copy bandwidth"
+         % ("bf16" if fp else ("e4m3" if f8 else "i8"), M, K, N, act, t * 1e6, tops, tops / peak, src, " / 2" if fp else "",
+            gbs, gbs / hbm))
+    return {"us": t * 1e6, "tops": tops, "gbs": gbs}
 
 
 def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static"):
@@ -127,8 +137,9 @@ def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static"):
                                               hero.tensor(out, "fwq", sc), s_q=s, s_k=s, s_v=0.02, s_p=1 / 255, mask=mask,
                                               p_mode=p_mode), 1, iters)
     scores = B * nh * S * S * (0.5 if mask == "causal" else 1.0)
-    print("INT8 attention B=%d S=%d nh=%d dh=%d %s P=%s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
-          % (B, S, nh, dh, mask, p_mode, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12), flush=True)
+    _say("INT8 attention B=%d S=%d nh=%d dh=%d %s P=%s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
+         % (B, S, nh, dh, mask, p_mode, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12))
+    return {"us": t * 1e6, "tscores": scores / t / 1e12}
 
 
 def bench_absmax(h, M, H, iters):

@@ -42,13 +42,22 @@ class Stack:
             ws = layer.workspace
             self.layers.append(layer)
             self.params.append((None, C))
+        self._descs = {}
         # chained activation buffers: input of layer 0 .. output of the last layer
-        self.bufs = []
+        self.bufs = self.make_edges()
+        g0, b0 = self.ln0
+        self.ln0_g = torch.from_numpy(np.asarray(g0, np.float32)).cuda()
+        self.ln0_b = torch.from_numpy(np.asarray(b0, np.float32)).cuda()
+
+    def make_edges(self):
+        """A fresh set of chained activation buffers [(tensor, scale tensor or None, hero.Tensor)] for this stack."""
+        layer_cfgs = self.cfgs
+        bufs = []
         for li in range(len(layer_cfgs) + 1):
             kind = self._edge_kind(li)
             if kind == "fp":
                 t = torch.empty(self.M, self.H, dtype=self.fp_torch, device="cuda")
-                self.bufs.append((t, None, hero.tensor(t)))
+                bufs.append((t, None, hero.tensor(t)))
             else:
                 q8 = torch.float8_e4m3fn if getattr(layer_cfgs[min(li, len(layer_cfgs) - 1)], "payload", "i8") == "f8" else torch.int8
                 t = torch.empty(self.M, self.H, dtype=q8, device="cuda")
@@ -57,10 +66,8 @@ class Stack:
                 else:
                     src = self.layers[li]._bufs["s_in"] if li < len(layer_cfgs) else self.layers[-1]._bufs["s_out"]
                     s = src
-                self.bufs.append((t, s, hero.tensor(t, kind, s)))
-        g0, b0 = self.ln0
-        self.ln0_g = torch.from_numpy(np.asarray(g0, np.float32)).cuda()
-        self.ln0_b = torch.from_numpy(np.asarray(b0, np.float32)).cuda()
+                bufs.append((t, s, hero.tensor(t, kind, s)))
+        return bufs
 
     def _edge_kind(self, li):
         """Type of the tensor between layer li-1 and layer li: 'fp' or an INT8 granularity."""
@@ -81,8 +88,23 @@ class Stack:
         self.h.hero_layernorm_quant(hero.tensor(x_fp), self.ln0_g, self.ln0_b, self.cfgs[0].eps, self.bufs[0][2])
 
     def forward(self, stream=None):
-        for li, layer in enumerate(self.layers):
-            layer.forward(self.bufs[li][2], self.bufs[li + 1][2], stream=stream)
+        """Every layer on the chained buffers: one C call (hero_stack_forward) sequencing the layers' launches."""
+        self.h.hero_stack_forward(self.desc(), self.workspace, stream=stream)
+
+    def desc(self, entry_in=None, edges=None):
+        """The hero_stack_desc of this stack; `entry_in` (a hero.Tensor over an FP activation buffer) adds the entry
+        LN^quant in front, `edges` substitutes other chained buffers (e.g. a second set for an overlapped stream)."""
+        key = (id(entry_in), id(edges))
+        if key not in self._descs:
+            e = [b[2] for b in (edges or self.bufs)]
+            self._descs[key] = hero.stack_desc([l.desc for l in self.layers], e, entry_in,
+                                               self.ln0_g if entry_in is not None else None,
+                                               self.ln0_b if entry_in is not None else None, self.cfgs[0].eps)
+        return self._descs[key]
+
+    @property
+    def workspace(self):
+        return max((l.workspace for l in self.layers), key=lambda w: w.numel())
 
     @property
     def output(self):

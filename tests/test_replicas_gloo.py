@@ -53,3 +53,22 @@ def test_single_process_needs_no_group():
     from paper_2310_17723_b200 import replicas
     assert replicas.max_over_ranks(0.25) == 0.25
     assert replicas.job_throughput(100, 4, 1, 2.0) == 200.0
+
+
+def test_bench_gpus_flag_starts_its_own_ranks():
+    # `python bench.py --gpus 2` outside a torchrun environment launches two ranks itself; without GPUs they meet over
+    # gloo.  --rendezvous-only runs the multi-rank plumbing (process group, barrier, max over ranks, rank 0's line)
+    # without the CUDA workload.
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rendezvous-only"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout                                # rank 0 alone prints
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["rendezvous"] == "ok"
+    assert d["max_over_ranks"] == 2.0                               # rank 1 reported 2.0 s, rank 0 1.0 s
+    assert d["value"] == pytest.approx(2 * 100 / 2.0)
