@@ -32,7 +32,7 @@ def _digest():
         h.update(f.encode())
         with open(f, "rb") as fh:
             h.update(fh.read())
-    h.update(" ".join(NVCC_FLAGS).encode())
+    h.update((" ".join(NVCC_FLAGS) + os.environ.get("HERO_NVCC_EXTRA", "")).encode())
     return h.hexdigest()
 
 
@@ -45,7 +45,7 @@ def build(force=False, verbose=False):
                 return LIB
     objdir = os.path.join(HERE, "build")
     os.makedirs(objdir, exist_ok=True)
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"] + os.environ.get("HERO_NVCC_EXTRA", "").split()
     objs = []
     procs = []
     for src in sources():

@@ -580,12 +580,14 @@ static hero_status attention_impl(hero_handle* h, const hero_attn_args* a, const
   if (probe) {
     HERO_REQUIRE(a->dtype == HERO_I8, HERO_ERR_UNSUPPORTED, "the verification outputs exist for the INT8 core only");
     p.dbg_scores = probe->scores; p.dbg_p = probe->p_codes; p.dbg_acc = probe->acc;
-    if (a->S <= 512) return attn_resident_dispatch(h, a, p, s, true);
+    if (a->S <= 512) return (a->dh == 128 && a->S > 384 ? attn_resident_dispatch : attn_pipe_dispatch)(h, a, p, s, true);
     if (rowmax) return a->dh == 64 ? launch_attn<64, true, false, true>(h, a, p, s) : launch_attn<128, true, false, true>(h, a, p, s);
     return a->dh == 64 ? launch_attn<64, false, false, true>(h, a, p, s) : launch_attn<128, false, false, true>(h, a, p, s);
   }
   if (fp_in) return attn_fp_dispatch(h, a, p, s);
-  if (a->S <= 512) return attn_resident_dispatch(h, a, p, s, false);   // the score row fits tensor memory (INT8 or e4m3)
+  // the score row fits tensor memory (INT8 or e4m3): the pipelined kernel, except for the one shape whose row and
+  // accumulator together exceed it there (dh = 128 with more than 384 keys)
+  if (a->S <= 512) return (a->dh == 128 && a->S > 384 ? attn_resident_dispatch : attn_pipe_dispatch)(h, a, p, s, false);
   if (f8_in) return a->dh == 64 ? launch_attn<64, false, true>(h, a, p, s) : launch_attn<128, false, true>(h, a, p, s);
   if (rowmax) return a->dh == 64 ? launch_attn<64, true>(h, a, p, s) : launch_attn<128, true>(h, a, p, s);
   if (a->dh == 64) return launch_attn<64, false>(h, a, p, s);

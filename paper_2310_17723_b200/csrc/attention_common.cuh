@@ -96,5 +96,7 @@ __device__ __forceinline__ int attn_nkv(const AttnParams& p, int qt, int b, int&
 hero_status attn_fp_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream);
 // INT8 core with the whole score row resident in tensor memory (S <= 512); defined in attention_resident.cu
 hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream, bool probe);
+// INT8 core for S <= 512 as a pipeline of exponential and pack warps; defined in attention_pipe.cu
+hero_status attn_pipe_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream, bool probe);
 
 }  // namespace hero
