@@ -5,11 +5,11 @@
 // steps, and the two steps are given to DIFFERENT warps so that the exponentials of one tile (bound by the
 // special-function unit) run beside the scaling, rounding and packing of the previous tile (FMA and byte-permute work):
 //
-//   warps 0-7   exponential warps: lane quarter w % 4, column half w / 4 of every 64-key score block.  Per block:
-//               e = 2^(t c2 - mp) with mp the running maximum of the thread's pieces so far, written back over the
-//               scores (tcgen05.st); running (max, sum) in registers; mp per block and the final (max, sum) go to
-//               shared memory.  One exponential per score.
-//   warps 8-15  pack warps, same split.  Combine the two halves' statistics, then per block
+//   warps 0-7   exponential warps: lane quarter w % 4; the group w / 4 takes every other 64-key score block of a tile.
+//               Per block: e = 2^(t c2 - mp) with mp the running maximum of the thread's pieces so far, written back
+//               over the scores (tcgen05.st); running (max, sum) in registers; mp per piece and the final (max, sum) go
+//               to shared memory.  One exponential per score.
+//   warps 8-15  pack warps: lane quarter w % 4, column half w / 4 of every block.  Combine the two halves' statistics, then per block
 //               P_u8 = Round(e 2^(mp - m) / (l s_p)) (one FMA with the 1.5 * 2^23 constant, byte permutes) into the UMMA
 //               operand tile in shared memory; afterwards the tile's output stage (Eq. 17) from the accumulator.
 //   warp 16     TMA producer: Q tile, K tiles of 128 keys, V tiles of 64 keys in the order P V consumes them.
@@ -107,13 +107,14 @@ __device__ __forceinline__ bool pipe_wait(uint64_t* bar, uint32_t parity, int* e
   return ptx::mbar_wait(bar, parity, err, code);
 }
 
-// A barrier wait for a whole group of eight warps: ONE warp polls the mbarrier, the others block on a hardware named
+// A barrier wait for a whole group of warps: ONE warp polls the mbarrier, the others block on a hardware named
 // barrier until it has seen the phase complete.  Eight warps polling the same word would spend a third of the SM's issue
-// slots on polling loops.  `id`: the group's named barrier (1 = exponential warps, 2 = pack warps); every warp of the
-// group must make the same sequence of calls.
+// slots on polling loops.  `id`: the group's named barrier (1 and 3: the two groups of exponential warps, 2: the pack warps); every warp
+// of a group must make the same sequence of calls.
+template <int THREADS>
 __device__ __forceinline__ bool pipe_group_wait(bool leader, int id, uint64_t* bar, uint32_t parity, int* err, int code, bool ok) {
   if (leader && ok) ok = pipe_wait(bar, parity, err, code);
-  asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory");
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(THREADS) : "memory");
   return ok;
 }
 
@@ -400,11 +401,16 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   }
   } else if (warp < PIPE_EXP_WARPS) {
     // ------------------------------------------------------------------ exponential warps
+    // Two groups of four warps (one warp per lane quarter each).  A group takes every other block of a tile, all 64
+    // columns of it, so the two warps that share a scheduler are always one block apart: while one waits for its block,
+    // loads it or stores it, the other one's exponentials keep the special-function unit busy.
     reg_inc<PIPE_REGS_EXP>();
-    const int quarter = warp & 3, half = warp >> 2;
+    const int quarter = warp & 3, grp = warp >> 2;
     const int r_loc = quarter * 32 + lane;
-    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * 32;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const float c2 = p.c2;
+    const bool leader = quarter == 0;
+    const int bar_id = 1 + 2 * grp;
     uint32_t wcnt = 0, bcnt = 0;
     bool ok = true;
     for (PipeWalk w(p, blockIdx.x, gridDim.x); w.t < total_tiles; w.next()) {
@@ -417,10 +423,10 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const bool stash = g.nb > NRING;
       // the statistics (and stash) slots of this parity are free: the pack warps are through with the tile two back.
       // (With spare ring slots the exponential warps could otherwise run several tiles ahead of the pack warps.)
-      ok = pipe_group_wait(warp == 0, 1, &t_empty[par], ((wcnt >> 1) & 1) ^ 1, p.err, 0x9400 | par, ok);
+      ok = pipe_group_wait<128>(leader, bar_id, &t_empty[par], ((wcnt >> 1) & 1) ^ 1, p.err, 0x9400 | par, ok);
       // the last key that every row of the tile may attend to
       const int tile_kmax = p.mask == HERO_MASK_CAUSAL ? min(g.klen - 1, g.qt * ATT_BM) : g.klen - 1;
-      float* pm_row = pm_s + ((par * PIPE_MAXB) * 2 + half) * ATT_BM + r_loc;
+      float* pm_row = pm_s + (par * PIPE_MAXB) * 2 * ATT_BM + r_loc;
       const long long probe_row = ((long long)(g.b * p.nh + g.h) * p.S + q) * p.S;
       float m = -INFINITY, l = 0.f;
       auto probe_scores = [&](const uint32_t (&r)[32], int key0) {
@@ -432,69 +438,73 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       };
 #pragma unroll 1
-      for (int k = 0; k < g.nb;) {                           // k: position in Q K^T order; every block takes the next ring slot
+      for (int k = 0; k < g.nb; ++k, ++bcnt) {               // k: position in Q K^T order; every block takes the next ring slot
+        if (((k + (int)wcnt) & 1) != grp) continue;          // the other group's block
         const int j = pipe_qk_block(g.nb, stash, k);
         const int blk = bcnt % NRING;
-        ok = pipe_group_wait(warp == 0, 1, &s_full[blk], (bcnt / NRING) & 1, p.err, 0x9000 | blk, ok);
+        ok = pipe_group_wait<128>(leader, bar_id, &s_full[blk], (bcnt / NRING) & 1, p.err, 0x9000 | blk, ok);
         ptx::tc_fence_after();
-        const int key0 = j * PB + half * 32;
+        const int key0 = j * PB;
         const bool to_stash = stash && k == 0;
-        // two blocks at a time while both are fully valid for every row of the warp (the common case): their 64
-        // exponentials then form one independent stream
-        // (decided per tile, not per warp: the eight warps must agree on the sequence of group waits)
-        const bool pair = !to_stash && k + 1 < g.nb && (j + 2) * PB - 1 <= tile_kmax;
-        if (pair) {
-          const int blk2 = (bcnt + 1) % NRING;
+        float* stash_dst = stash_s + (par * PB) * ATT_BM + r_loc;
+        if ((j + 1) * PB - 1 <= tile_kmax) {
+          // every key of the block is valid for every row of the tile (the common case): 64 independent exponentials
           uint32_t ra[32], rb[32];
           ptx::tmem_ld32(t_lane + blk * PB, ra);
-          ok = pipe_group_wait(warp == 0, 1, &s_full[blk2], ((bcnt + 1) / NRING) & 1, p.err, 0x9000 | blk2, ok);
-          ptx::tc_fence_after();
-          ptx::tmem_ld32(t_lane + blk2 * PB, rb);
+          ptx::tmem_ld32(t_lane + blk * PB + 32, rb);
           ptx::tmem_ld_wait();
-          probe_scores(ra, key0); probe_scores(rb, key0 + PB);
+          probe_scores(ra, key0); probe_scores(rb, key0 + 32);
           float mA;
           pipe_exp_two_full<F8>(ra, rb, c2, m, l, mA);
-          ptx::tmem_st32(t_lane + blk * PB, ra);
-          ptx::tmem_st32(t_lane + blk2 * PB, rb);
-          pm_row[j * 2 * ATT_BM] = mA;                       // the maximum each piece's e values are relative to
-          pm_row[(j + 1) * 2 * ATT_BM] = m;
-          k += 2; bcnt += 2;
-          continue;
-        }
-        uint32_t r[32];
-        ptx::tmem_ld32(t_lane + blk * PB, r);
-        ptx::tmem_ld_wait();
-        probe_scores(r, key0);
-        const int nvalid = kmax - key0 + 1;
-        if (__all_sync(0xffffffffu, nvalid >= 32)) {
-          pipe_exp_piece<F8, true>(r, 32, c2, m, l);
-        } else if (nvalid > 0) {
-          pipe_exp_piece<F8, false>(r, nvalid, c2, m, l);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) r[e] = 0;             // every key of the piece masked
-        }
-        if constexpr (Cfg::STASH) {
-          if (to_stash) {
+          if (Cfg::STASH && to_stash) {
             // the block's e values wait in shared memory ([column][row]: a warp's 32 rows are consecutive words) and
-            // its ring slot goes straight back to the Q K^T issuer
+            // its ring slot goes straight back to the Q K^T issuer (eight arrivals, as from the pack warps: two per
+            // warp of this group)
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&s_free[blk]);
-            float* dst = stash_s + (par * PB + half * 32) * ATT_BM + r_loc;
+            if (lane == 0) { ptx::mbar_arrive(&s_free[blk]); ptx::mbar_arrive(&s_free[blk]); }
 #pragma unroll
-            for (int e = 0; e < 32; ++e) dst[e * ATT_BM] = __uint_as_float(r[e]);
+            for (int e = 0; e < 32; ++e) { stash_dst[e * ATT_BM] = __uint_as_float(ra[e]); stash_dst[(32 + e) * ATT_BM] = __uint_as_float(rb[e]); }
           } else {
-            ptx::tmem_st32(t_lane + blk * PB, r);
+            ptx::tmem_st32(t_lane + blk * PB, ra);
+            ptx::tmem_st32(t_lane + blk * PB + 32, rb);
           }
+          pm_row[(j * 2 + 0) * ATT_BM] = mA;                 // the maximum each half's e values are relative to
+          pm_row[(j * 2 + 1) * ATT_BM] = m;
         } else {
-          ptx::tmem_st32(t_lane + blk * PB, r);
+          // a block that the mask cuts: one 32-column piece after the other
+#pragma unroll 1
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t r[32];
+            ptx::tmem_ld32(t_lane + blk * PB + hh * 32, r);
+            ptx::tmem_ld_wait();
+            probe_scores(r, key0 + hh * 32);
+            const int nvalid = kmax - (key0 + hh * 32) + 1;
+            if (__all_sync(0xffffffffu, nvalid >= 32)) {
+              pipe_exp_piece<F8, true>(r, 32, c2, m, l);
+            } else if (nvalid > 0) {
+              pipe_exp_piece<F8, false>(r, nvalid, c2, m, l);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) r[e] = 0;           // every key of the piece masked
+            }
+            if (Cfg::STASH && to_stash) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) stash_dst[(hh * 32 + e) * ATT_BM] = __uint_as_float(r[e]);
+            } else {
+              ptx::tmem_st32(t_lane + blk * PB + hh * 32, r);
+            }
+            pm_row[(j * 2 + hh) * ATT_BM] = m;
+          }
+          if (Cfg::STASH && to_stash) {
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { ptx::mbar_arrive(&s_free[blk]); ptx::mbar_arrive(&s_free[blk]); }
+          }
         }
-        pm_row[j * 2 * ATT_BM] = m;                          // the maximum the piece's e values are relative to
-        ++k; ++bcnt;
       }
       ptx::tmem_st_wait();
-      st_s[(par * 2 + half) * ATT_BM + r_loc] = make_float2(m, l);
+      st_s[(par * 2 + grp) * ATT_BM + r_loc] = make_float2(m, l);   // this group's blocks: their running maximum and sum
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&t_full[par]);
@@ -549,7 +559,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const int par = wcnt & 1;
       const bool stash = g.nb > NRING;
       const long long probe_row = ((long long)(g.b * p.nh + g.h) * p.S + q) * p.S;
-      ok = pipe_group_wait(warp == PIPE_EXP_WARPS, 2, &t_full[par], (wcnt >> 1) & 1, p.err, 0x9100 | par, ok);
+      ok = pipe_group_wait<256>(warp == PIPE_EXP_WARPS, 2, &t_full[par], (wcnt >> 1) & 1, p.err, 0x9100 | par, ok);
       ptx::tc_fence_after();
       // ---- the row's maximum and sum from the two column halves
       const float2 sa = st_s[(par * 2 + 0) * ATT_BM + r_loc], sb = st_s[(par * 2 + 1) * ATT_BM + r_loc];
@@ -601,7 +611,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&s_free[blk]);     // the block's columns may take the next tile's scores
         }
-        ok = pipe_group_wait(warp == PIPE_EXP_WARPS, 2, &p_empty[pb], ((pcnt / PIPE_NPB) & 1) ^ 1, p.err, 0x9200 | pb, ok);
+        ok = pipe_group_wait<256>(warp == PIPE_EXP_WARPS, 2, &p_empty[pb], ((pcnt / PIPE_NPB) & 1) ^ 1, p.err, 0x9200 | pb, ok);
         uint32_t wd[8];
         pipe_pack32<F8>(r, f, wd);
         probe_codes(wd, j);
@@ -617,7 +627,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&t_empty[par]);        // statistics and stash of this parity may be overwritten
       // ---- output stage (Eq. 17): X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8); OW columns per warp
-      ok = pipe_group_wait(warp == PIPE_EXP_WARPS, 2, o_full, wcnt & 1, p.err, 0x9300, ok);
+      ok = pipe_group_wait<256>(warp == PIPE_EXP_WARPS, 2, o_full, wcnt & 1, p.err, 0x9300, ok);
       ptx::tc_fence_after();
 #pragma unroll
       for (int c0 = 0; c0 < OW; c0 += 32) {
