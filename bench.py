@@ -151,7 +151,15 @@ def kernel_table(shape, cfg, first=False):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernel function that dominates a
 # workload's step, each from one small ncu capture (one kernel, a few launches) recorded under profiles/; keyed by
 # (workload, kernel function).  These are constants of a recorded capture, not values this run measures.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    ("c5", "attention"): {"bytes_per_launch": 101.1e6, "source": "profiles/attention_int8.md: one ncu capture (dram__bytes_read.sum + "
+                          "dram__bytes_write.sum = 25.27 MB + 0) of attn_int8_pipe_kernel on B16 S512 nh16 dh64, a quarter of this workload's "
+                          "batch, scaled by 4 (traffic is proportional to the batch); algorithmic 100.7 MB read + 33.6 MB written, the output "
+                          "stays in L2"},
+    ("c3", "gemm_pair_kernel<int8, no activation>"): {"bytes_per_launch": 28.1e6, "source": "profiles/dram_traffic_c3_layer.md: ncu capture "
+                          "of the three launches (QKV 15.8 MB, attention output 13.7 MB, FC2 54.8 MB), recorded with an earlier build of "
+                          "this unchanged kernel"},
+}
 KERNEL_FUNCTION = {"qkv gemm": "gemm_pair_kernel<int8, no activation>", "attn-out gemm": "gemm_pair_kernel<int8, no activation>",
                    "fc2 gemm": "gemm_pair_kernel<int8, no activation>"}
 INT8_NOMINAL_TOPS = 4500.0          # dense INT8 rate of the part (datasheet figure without sparsity), for context

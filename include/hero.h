@@ -341,6 +341,13 @@ hero_status hero_quantize_weight(hero_handle* h, const float* W, int64_t ldw, in
                                  const float* in_scale, const float* out_scale, const float* bias, int8_t* Wq,
                                  int64_t ldq, float* w_scale, float* bias_out, void* stream);
 
+/* The same fold for the FP8 variant of the method (Sec. 2.1: the approach "carries over to FP8"): the payload is e4m3,
+ * w_scale[n] = max_k |W~[n][k]| / 448 (1 if the row is zero) and Wq[n][k] is the byte of the saturating
+ * round-to-nearest-even conversion of W~[n][k] / w_scale[n].  Arguments as hero_quantize_weight. */
+hero_status hero_quantize_weight_f8(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K,
+                                    const float* in_scale, const float* out_scale, const float* bias, uint8_t* Wq,
+                                    int64_t ldq, float* w_scale, float* bias_out, void* stream);
+
 /* Fill desc->mode from a Table 1 preset (M1, M2, M3) or all-FP. */
 hero_status hero_mode_preset(int32_t preset, int32_t mode_out[5]);
 /* Scratch the layer needs for M tokens. */

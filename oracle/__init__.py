@@ -12,6 +12,8 @@ quant   Sec. 2.1 quantizers (symmetric INT8, column-wise weights, TWQ/FWQ/SQ)
 ops     the quantization-aware operators (LN^quant, GeMM^quant, attention, GELU^quant)
 layer   offline preparation (calibration, Eq. 20-23/32 folding) and the
         layer forward of Sec. 2.2 under the module modes of Table 1
+search  per-module sensitivity and the greedy INT8 -> FP mode search that
+        generalises Table 1's presets (Sec. 2.3), as loops over `layer`
 
 Pins (what fixes each function to something other than itself) live in
 tests/test_oracle_*.py; the whole INT8 layer has no external definition and is

@@ -105,11 +105,12 @@ def calibrate_gpu(h, cfg, params, x_cal, n_seq, return_output=False):
     return (scales, out) if return_output else scales
 
 
-def fold_quantize_gpu(h, W, b, in_scale=None, out_scale=None):
-    """Device counterpart of `prep.fold_quantize` (same arguments and return layout): W is [K, N] (the paper's W[d, m])."""
+def fold_quantize_gpu(h, W, b, in_scale=None, out_scale=None, payload="i8"):
+    """Device counterpart of `prep.fold_quantize` (same arguments and return layout): W is [K, N] (the paper's W[d, m]).
+    payload "f8": e4m3 codes (returned as their bytes, uint8) and absmax / 448 scales, through hero_quantize_weight_f8."""
     Wt = torch.from_numpy(np.ascontiguousarray(np.asarray(W, np.float64).T.astype(np.float32))).cuda()   # [N][K]
     N, K = Wt.shape
-    Wq = torch.empty(N, K, dtype=torch.int8, device="cuda")
+    Wq = torch.empty(N, K, dtype=torch.float8_e4m3fn if payload == "f8" else torch.int8, device="cuda")
     ws = torch.empty(N, dtype=torch.float32, device="cuda")
     bo = torch.empty(N, dtype=torch.float32, device="cuda") if b is not None else None
     h.hero_quantize_weight(Wt, Wq, ws, in_scale=None if in_scale is None else _vec(in_scale),
@@ -117,9 +118,11 @@ def fold_quantize_gpu(h, W, b, in_scale=None, out_scale=None):
                            bias=None if b is None else _vec(b), bias_out=bo)
     h.check()
     torch.cuda.synchronize()
+    if payload == "f8":
+        Wq = Wq.view(torch.uint8)
     return Wq.cpu().numpy(), ws.cpu().numpy(), (None if bo is None else bo.cpu().numpy())
 
 
 def prepare_layer_gpu(h, cfg, params, C):
     """`prep.prepare_layer` with the weight folding and quantization done on the device."""
-    return prep.prepare_layer(cfg, params, C, fold_quantize_fn=lambda W, b, i, o: fold_quantize_gpu(h, W, b, i, o))
+    return prep.prepare_layer(cfg, params, C, fold_quantize_fn=lambda W, b, i, o: fold_quantize_gpu(h, W, b, i, o, cfg.payload))

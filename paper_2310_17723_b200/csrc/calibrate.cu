@@ -103,7 +103,9 @@ __global__ void __launch_bounds__(256) abs_hist_kernel(const uint16_t* __restric
     if (sh[i]) atomicAdd(hist + i, (unsigned long long)sh[i]);
 }
 
-// One CTA per output feature n: row n of W [N][K] (FP32).
+// One CTA per output feature n: row n of W [N][K] (FP32).  F8: the e4m3 payload of the FP8 variant (scale absmax / 448,
+// codes by the saturating round-to-nearest-even conversion) instead of INT8.
+template <bool F8>
 __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __restrict__ W, long long ldw, int N, int K,
                                                               const float* __restrict__ in_scale,
                                                               const float* __restrict__ out_scale,
@@ -130,7 +132,7 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
   __syncthreads();
   m = 0.f;
   for (int w = 0; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, red[w]);
-  const float sw = m > 0.f ? m / 127.0f : 1.0f;                  // Eq. 2
+  const float sw = m > 0.f ? m / (F8 ? 448.0f : 127.0f) : 1.0f;  // Eq. 2
   if (threadIdx.x == 0) {
     w_scale[n] = sw;
     if (bias_out) bias_out[n] = bias ? bias[n] / o : 0.f;
@@ -141,12 +143,16 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
     const float4 w = __ldg(reinterpret_cast<const float4*>(row + k));
     float4 s = make_float4(1.f, 1.f, 1.f, 1.f);
     if (in_scale) s = __ldg(reinterpret_cast<const float4*>(in_scale + k));
-    const int a = __float2int_rn(fminf(fmaxf(w.x * s.x / o / sw, -127.f), 127.f));
-    const int b = __float2int_rn(fminf(fmaxf(w.y * s.y / o / sw, -127.f), 127.f));
-    const int c = __float2int_rn(fminf(fmaxf(w.z * s.z / o / sw, -127.f), 127.f));
-    const int d = __float2int_rn(fminf(fmaxf(w.w * s.w / o / sw, -127.f), 127.f));
-    *reinterpret_cast<uint32_t*>(qrow + k) =
-        (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)d << 24);
+    if constexpr (F8) {
+      *reinterpret_cast<uint32_t*>(qrow + k) = ptx::f32x4_to_e4m3x4(w.x * s.x / o / sw, w.y * s.y / o / sw, w.z * s.z / o / sw, w.w * s.w / o / sw);
+    } else {
+      const int a = __float2int_rn(fminf(fmaxf(w.x * s.x / o / sw, -127.f), 127.f));
+      const int b = __float2int_rn(fminf(fmaxf(w.y * s.y / o / sw, -127.f), 127.f));
+      const int c = __float2int_rn(fminf(fmaxf(w.z * s.z / o / sw, -127.f), 127.f));
+      const int d = __float2int_rn(fminf(fmaxf(w.w * s.w / o / sw, -127.f), 127.f));
+      *reinterpret_cast<uint32_t*>(qrow + k) =
+          (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)d << 24);
+    }
   }
 }
 
@@ -218,10 +224,10 @@ extern "C" hero_status hero_abs_histogram(hero_handle* h, const hero_tensor* x, 
   return HERO_OK;
 }
 
-extern "C" hero_status hero_quantize_weight(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K,
-                                            const float* in_scale, const float* out_scale, const float* bias,
-                                            int8_t* Wq, int64_t ldq, float* w_scale, float* bias_out, void* stream) {
-  using namespace hero;
+namespace hero {
+static hero_status quantize_weight_impl(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K, const float* in_scale,
+                                        const float* out_scale, const float* bias, void* Wq, int64_t ldq, float* w_scale,
+                                        float* bias_out, bool f8, void* stream) {
   HERO_REQUIRE(h && W && Wq && w_scale, HERO_ERR_INVALID_ARG, "hero_quantize_weight: NULL argument");
   HERO_REQUIRE(N >= 0 && K > 0 && K % 4 == 0 && ldw >= K && ldw % 4 == 0 && ldq >= K && ldq % 4 == 0, HERO_ERR_INVALID_ARG,
                "K, ldw and ldq must be positive multiples of 4 with ld >= K");
@@ -231,10 +237,24 @@ extern "C" hero_status hero_quantize_weight(hero_handle* h, const float* W, int6
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   {
     LaunchScope scope(h, s, KERNEL_GEMM);
-    HERO_CUDA(launch_dependent(quantize_weight_kernel, dim3((unsigned)N), dim3(256), 0, s, W, (long long)ldw, (int)N, (int)K,
-                               in_scale, out_scale, bias, Wq, (long long)ldq, w_scale, bias_out));
+    auto kern = f8 ? quantize_weight_kernel<true> : quantize_weight_kernel<false>;
+    HERO_CUDA(launch_dependent(kern, dim3((unsigned)N), dim3(256), 0, s, W, (long long)ldw, (int)N, (int)K, in_scale, out_scale,
+                               bias, static_cast<int8_t*>(Wq), (long long)ldq, w_scale, bias_out));
   }
   pdl_fence_stream(s);   // Wq, w_scale and bias_out are model constants to whatever runs next on this stream
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
+}
+}  // namespace hero
+
+extern "C" hero_status hero_quantize_weight(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K,
+                                            const float* in_scale, const float* out_scale, const float* bias,
+                                            int8_t* Wq, int64_t ldq, float* w_scale, float* bias_out, void* stream) {
+  return hero::quantize_weight_impl(h, W, ldw, N, K, in_scale, out_scale, bias, Wq, ldq, w_scale, bias_out, false, stream);
+}
+
+extern "C" hero_status hero_quantize_weight_f8(hero_handle* h, const float* W, int64_t ldw, int32_t N, int32_t K,
+                                               const float* in_scale, const float* out_scale, const float* bias,
+                                               uint8_t* Wq, int64_t ldq, float* w_scale, float* bias_out, void* stream) {
+  return hero::quantize_weight_impl(h, W, ldw, N, K, in_scale, out_scale, bias, Wq, ldq, w_scale, bias_out, true, stream);
 }

@@ -112,7 +112,7 @@ EXPORTS = ("hero_create", "hero_destroy", "hero_last_error", "hero_check", "hero
            "hero_layer_workspace_bytes", "hero_layer_workspace_layout", "hero_layer_forward", "hero_layer_forward_host", "hero_layer_forward_host_async", "hero_profile_begin",
            "hero_profile_end", "hero_layer_forward_static", "hero_absmax_observe", "hero_quantize_weight", "hero_abs_histogram",
            "hero_int8_decode_attention", "hero_layer_decode", "hero_static_check", "hero_int8_attention_probe", "hero_stack_forward",
-           "hero_stack_forward_host_async")
+           "hero_stack_forward_host_async", "hero_quantize_weight_f8")
 
 _lib = None
 
@@ -142,6 +142,7 @@ def lib():
         L.hero_abs_histogram.argtypes = [C.c_void_p, C.POINTER(Tensor), C.c_float, C.c_void_p, C.c_void_p]
         L.hero_quantize_weight.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.hero_quantize_weight_f8.argtypes = L.hero_quantize_weight.argtypes
         L.hero_layer_workspace_layout.argtypes = [C.POINTER(LayerDesc), C.c_int64, C.POINTER(LayerLayout)]
         L.hero_layer_forward.argtypes = [C.c_void_p, C.POINTER(LayerDesc), C.POINTER(Tensor), C.POINTER(Tensor),
                                          C.POINTER(Tensor), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -278,9 +279,12 @@ class Handle:
         _check(lib().hero_abs_histogram(self._h, C.byref(x), float(bound), C.c_void_p(hist.data_ptr()), _stream(stream)))
 
     def hero_quantize_weight(self, W, Wq, w_scale, in_scale=None, out_scale=None, bias=None, bias_out=None, stream=None):
-        """W: float32 [N, K]; Wq: int8 [N, K]; w_scale: float32 [N]; optional folds in_scale [K], out_scale [N]."""
-        assert W.dim() == 2 and W.stride(1) == 1 and Wq.stride(1) == 1 and W.dtype == torch.float32 and Wq.dtype == torch.int8
-        _check(lib().hero_quantize_weight(self._h, C.c_void_p(W.data_ptr()), W.stride(0), W.shape[0], W.shape[1],
+        """W: float32 [N, K]; Wq: int8 [N, K], or float8_e4m3fn [N, K] for the FP8 variant (hero_quantize_weight_f8);
+        w_scale: float32 [N]; optional folds in_scale [K], out_scale [N]."""
+        assert W.dim() == 2 and W.stride(1) == 1 and Wq.stride(1) == 1 and W.dtype == torch.float32
+        assert Wq.dtype in (torch.int8, torch.float8_e4m3fn)
+        fn = lib().hero_quantize_weight if Wq.dtype == torch.int8 else lib().hero_quantize_weight_f8
+        _check(fn(self._h, C.c_void_p(W.data_ptr()), W.stride(0), W.shape[0], W.shape[1],
                                           _ptr(in_scale), _ptr(out_scale), _ptr(bias), C.c_void_p(Wq.data_ptr()),
                                           Wq.stride(0), _ptr(w_scale), _ptr(bias_out), _stream(stream)))
 

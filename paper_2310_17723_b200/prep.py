@@ -213,13 +213,11 @@ def prepare_layer(cfg: LayerConfig, params, C, fold_quantize_fn=None):
     if cfg.payload not in ("i8", "f8"):
         raise ValueError("payload %r" % (cfg.payload,))
     if cfg.payload == "f8":
-        if fold_quantize_fn is not None:
-            raise NotImplementedError("the device-side fold + quantization emits INT8 weights only")
         if cfg.p_mode != "static":
             raise ValueError("the e4m3 attention core has the static P quantizer only")
         if cfg.mode["attn"] != "int8" and cfg.mode["attn_out"] == "int8":
             raise ValueError("e4m3 payload: an FP attention core cannot feed an 8-bit attention-output linear")
-        fq = lambda W, b, i, o: fold_quantize(W, b, i, o, payload="f8")
+        fq = fold_quantize_fn or (lambda W, b, i, o: fold_quantize(W, b, i, o, payload="f8"))
     else:
         fq = fold_quantize_fn or fold_quantize
     p = {k: np.asarray(v, np.float64) for k, v in params.items()}

@@ -69,6 +69,31 @@ def test_quantize_weight_matches_fold_then_eq2(h, K, N, fold):
     assert ws[3] == 1.0 and not Wq[3].any()
 
 
+@pytest.mark.parametrize("K,N,fold", [(256, 192, "none"), (1024, 3072, "both"), (4096, 1024, "in")])
+def test_quantize_weight_f8_matches_fold_then_e4m3(h, K, N, fold):
+    # the FP8 variant's weights prepared on the device: absmax / 448 scales, saturating round-to-nearest-even e4m3 codes
+    rng = np.random.default_rng(7 * K + N)
+    Wm = rng.standard_normal((K, N)) * 0.02
+    Wm[:, 5] = 0.0
+    b = rng.standard_normal(N) * 0.01
+    s_in = np.exp(rng.standard_normal(K) * 0.5) * 0.03 if fold in ("in", "both") else None
+    s_out = np.exp(rng.standard_normal(N) * 0.5) * 0.05 if fold == "both" else None
+    Wq, ws, bo = CAL.fold_quantize_gpu(h, Wm, b, s_in, s_out, payload="f8")
+    f32 = lambda a: None if a is None else np.asarray(a, np.float64).astype(np.float32).astype(np.float64)
+    W_f8, S_w, b_ref = OL.fold_and_quantize(f32(Wm), f32(b), f32(s_in), f32(s_out), payload="f8")
+    got = torch.from_numpy(Wq).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)        # [N][K] e4m3 values
+    want = np.ascontiguousarray(np.asarray(W_f8).T)
+    np.testing.assert_allclose(ws, np.asarray(S_w, np.float64), rtol=1e-6)
+    np.testing.assert_allclose(bo, b_ref, rtol=1e-6, atol=1e-12)
+    # identical codes except where fp32 and fp64 arithmetic fall on different sides of an e4m3 rounding tie: then the
+    # neighbouring code (one step of 2^-3 relative at most)
+    d = got != want
+    assert d.mean() <= 1e-4, float(d.mean())
+    assert np.all(np.abs(got - want)[d] <= np.abs(want[d]) * 0.126 + 2.0 ** -9)
+    assert ws[5] == 1.0 and not got[5].any()
+    assert np.abs(got).max() == 448.0                               # a column's largest weight lands on the largest code
+
+
 SMALL = dict(B=2, S=128, H=256, nh=4, F=512)
 
 
