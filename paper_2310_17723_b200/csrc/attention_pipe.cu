@@ -102,6 +102,31 @@ struct PipeWalk {
   }
 };
 
+// A position in a ring of N slots with the phase parity of its barriers, advanced without divisions (N is 6 or 7).
+template <int N>
+struct RingPos {
+  int idx = 0;
+  uint32_t par = 0;
+  __device__ __forceinline__ void advance(int n) {          // n <= 2 N
+    idx += n;
+    if (idx >= N) { idx -= N; par ^= 1; }
+    if (idx >= N) { idx -= N; par ^= 1; }
+  }
+  // slot and parity k positions further on (k <= N)
+  __device__ __forceinline__ void at(int k, int& slot, uint32_t& parity) const {
+    slot = idx + k; parity = par;
+    if (slot >= N) { slot -= N; parity ^= 1; }
+  }
+};
+
+// A global load that stays where it is written: the compiler may otherwise sink a load to its first use, which here is a
+// whole tile later, on the critical path.
+__device__ __forceinline__ float ld_nc_here(const float* ptr) {
+  float v;
+  asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(ptr));
+  return v;
+}
+
 // Bounded wait (mbarrier.try_wait with a suspend-time hint inside a bounded loop).
 __device__ __forceinline__ bool pipe_wait(uint64_t* bar, uint32_t parity, int* err, int code) {
   return ptx::mbar_wait(bar, parity, err, code);
@@ -333,7 +358,8 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     // ------------------------------------------------------------------ Q K^T issuer: block after block, tile after tile
     if (lane == 0) {
       constexpr uint64_t kmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // Q, K: K-major rows of DH bytes
-      uint32_t wcnt = 0, kcnt = 0, bcnt = 0;
+      uint32_t wcnt = 0, kcnt = 0;
+      RingPos<NRING> ring;
       bool ok = true;
       for (PipeWalk w(p, blockIdx.x, gridDim.x); w.t < total_tiles && ok; w.next()) {
         PipeTile g;
@@ -341,12 +367,12 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int qb = wcnt & 1;
         if (!pipe_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x8000 | qb)) { ok = false; break; }
         const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::Q_TILE);
-        for (int k = 0; k < g.nb && ok; ++k, ++kcnt, ++bcnt) {
-          const int ks = kcnt % KST, blk = bcnt % NRING;
+        for (int k = 0; k < g.nb && ok; ++k, ++kcnt, ring.advance(1)) {
+          const int ks = kcnt % KST, blk = ring.idx;
           if (!pipe_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8100 | ks)) { ok = false; break; }
           // the ring slot: whoever read the block that was there (the pack warps, or the exponential warps for a block
           // that went to the stash) is through with it
-          if (!pipe_wait(&s_free[blk], ((bcnt / NRING) & 1) ^ 1, p.err, 0x8200 | blk)) { ok = false; break; }
+          if (!pipe_wait(&s_free[blk], ring.par ^ 1, p.err, 0x8200 | blk)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::K_TILE);
 #pragma unroll
@@ -411,7 +437,8 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const float c2 = p.c2;
     const bool leader = quarter == 0;
     const int bar_id = 1 + 2 * grp;
-    uint32_t wcnt = 0, bcnt = 0;
+    uint32_t wcnt = 0;
+    RingPos<NRING> ring;                                     // the ring slot of the tile's first block (Q K^T order)
     bool ok = true;
     for (PipeWalk w(p, blockIdx.x, gridDim.x); w.t < total_tiles; w.next()) {
       PipeTile g;
@@ -437,12 +464,14 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
         }
       };
+      // k: position in Q K^T order; every block takes the next ring slot; this group's blocks are every other one
 #pragma unroll 1
-      for (int k = 0; k < g.nb; ++k, ++bcnt) {               // k: position in Q K^T order; every block takes the next ring slot
-        if (((k + (int)wcnt) & 1) != grp) continue;          // the other group's block
+      for (int k = (grp ^ (int)wcnt) & 1; k < g.nb; k += 2) {
         const int j = pipe_qk_block(g.nb, stash, k);
-        const int blk = bcnt % NRING;
-        ok = pipe_group_wait<128>(leader, bar_id, &s_full[blk], (bcnt / NRING) & 1, p.err, 0x9000 | blk, ok);
+        int blk;
+        uint32_t blk_par;
+        ring.at(k, blk, blk_par);
+        ok = pipe_group_wait<128>(leader, bar_id, &s_full[blk], blk_par, p.err, 0x9000 | blk, ok);
         ptx::tc_fence_after();
         const int key0 = j * PB;
         const bool to_stash = stash && k == 0;
@@ -508,6 +537,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&t_full[par]);
+      ring.advance(g.nb);
       ++wcnt;
     }
   } else {
@@ -517,7 +547,8 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     constexpr int OW = DH / 2;                               // output columns of this warp: half * OW .. + OW - 1
     float* osc = osc_s + (warp - PIPE_EXP_WARPS) * OW;
-    uint32_t wcnt = 0, bcnt = 0, pcnt = 0;
+    uint32_t wcnt = 0, pcnt = 0;
+    RingPos<NRING> ring;                                     // the ring slot of the tile's first block (Q K^T order)
     bool ok = true;
     // the per-column output scales of a tile are fetched one tile ahead (a global load in front of every tile would
     // stand on the pack warps' critical path)
@@ -529,7 +560,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       wk = ww.tile(p, gg);
 #pragma unroll
       for (int c = 0; c < OW / 32; ++c)
-        raw[c] = is_q8(p.out_dt) ? __ldg(p.out_scale + (long long)(gg.h * DH + half * OW + c * 32 + lane) * p.out_scale_stride) : 1.f;
+        raw[c] = is_q8(p.out_dt) ? ld_nc_here(p.out_scale + (long long)(gg.h * DH + half * OW + c * 32 + lane) * p.out_scale_stride) : 1.f;
     };
     PipeWalk w(p, blockIdx.x, gridDim.x);
     fetch(w, gn, work_n, osc_raw_n);
@@ -573,7 +604,6 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const float pscale = lsum > 0.f ? (ROWMAX ? 255.0f : __fdividef(p.inv_sp, lsum)) : 0.f;
       const float rowf = ROWMAX ? (lsum > 0.f ? 1.0f / lsum : 0.f) : 1.0f;
       const float* pm_row = pm_s + ((par * PIPE_MAXB) * 2 + half) * ATT_BM + r_loc;
-      const uint32_t bcnt0 = bcnt;                           // ring counter of the tile's block 0
       const int sw = (r_loc >> 1) & 3;
       // UMMA K-major operand tile with 64-byte rows and the 64-byte swizzle: 16-byte chunk c of row r sits at chunk
       // c ^ ((r >> 1) & 3) of the row; this warp owns chunks 2 half and 2 half + 1
@@ -594,7 +624,9 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll 1
       for (int j = 0; j < g.nb; ++j) {
         const bool from_stash = stash && j == g.nb - 1;      // the block that was computed first and parked in shared memory
-        const int blk = (int)((bcnt0 + (stash ? j + 1 : j)) % NRING);
+        int blk;
+        uint32_t blk_par;
+        ring.at(stash ? j + 1 : j, blk, blk_par);
         const int pb = pcnt % PIPE_NPB;
         uint32_t r[32];
         if (Cfg::STASH && from_stash) {
@@ -623,7 +655,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (lane == 0) ptx::mbar_arrive(&p_full[pb]);
         ++pcnt;
       }
-      bcnt += g.nb;
+      ring.advance(g.nb);
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&t_empty[par]);        // statistics and stash of this parity may be overwritten
       // ---- output stage (Eq. 17): X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8); OW columns per warp
