@@ -85,10 +85,31 @@ __device__ __forceinline__ float4 lds_f4(const float* p) {
 // NC (16 or 32) columns of one output row: v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];
 // INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.  Per-column vectors come from shared memory four at a time,
 // the arithmetic runs on packed FP32 pairs, the row segment leaves in 32-byte stores when the output allows it.
+// How a warp's piece of an 8-bit output tile (32 rows x NC bytes) leaves the SM.  Straight from registers every lane writes
+// its own row: 32 different 128-byte lines per store instruction, which the load/store pipe takes one line at a time,
+// in competition with the tensor core's operand reads from shared memory.  Instead the piece is put together in a small
+// per-warp buffer in shared memory (NC = 32: the 32-byte swizzle of the tensor map, so that the lanes' 16-byte writes
+// spread over all banks) and one lane hands it to the TMA unit as a bulk tensor store, which also clips rows and
+// columns beyond the matrix.  The buffer is reused as soon as the unit has read it.
+struct OutStage {
+  uint8_t* buf;               // this warp's buffer (NULL: direct stores)
+  const CUtensorMap* tm;      // box = 32 rows x NC bytes
+};
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_2d(const CUtensorMap* tm, const void* smem_src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(ptx::smem_u32(smem_src)) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 template <bool INT8, int ACT, int OUTK, int NC>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32_t (&r)[NC], const float* e_cs,
                                                const float* e_bias, const float* e_post, int m, bool row_ok, float rs,
-                                               int col0, bool wide) {
+                                               int col0, bool wide, const OutStage& stage) {
   if constexpr (OUTK == OUT_I32) {
     if (!row_ok) return;
     int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
@@ -143,8 +164,8 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
       if constexpr (OUTK == OUT_I8) {
         // Round (half to even) happened in the float adder: 1.5 * 2^23 + k keeps k in its low byte.  The clip to
         // [-127, 127] is applied only if some value of the chunk needs it.
-        hi = fmaxf(fmaxf(hi, fmaxf(y0.x, y0.y)), fmaxf(y1.x, y1.y));
-        lo = fminf(fminf(lo, fminf(y0.x, y0.y)), fminf(y1.x, y1.y));
+        hi = ptx::max3(ptx::max3(hi, y0.x, y0.y), y1.x, y1.y);
+        lo = ptx::min3(ptx::min3(lo, y0.x, y0.y), y1.x, y1.y);
       }
     }
     if constexpr (OUTK == OUT_I8) {
@@ -153,15 +174,34 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
         for (int j = 0; j < NC; ++j) v[j] = fminf(fmaxf(v[j], ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
       }
     }
-    if (!row_ok) return;
     if constexpr (OUTK == OUT_I8 || OUTK == OUT_F8) {
-      int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
       uint32_t w[NC / 4];
 #pragma unroll
       for (int g = 0; g < NC / 4; ++g) {
         if constexpr (OUTK == OUT_F8) w[g] = ptx::f32x4_to_e4m3x4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);   // saturating RNE
         else w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
       }
+      if (stage.buf) {
+        // every lane takes part (rows past the end are clipped by the store)
+        const int lane = threadIdx.x & 31;
+        if (lane == 0) bulk_store_wait_read();               // the previous piece has left the buffer
+        __syncwarp();
+        const uint32_t row = ptx::smem_u32(stage.buf) + lane * NC;
+        if constexpr (NC == 32) {
+          const uint32_t sw = ((lane >> 2) & 1) << 4;        // 32-byte swizzle: 16-byte half ^= bit 7 of the address
+          sts16(row + sw, w[0], w[1], w[2], w[3]);
+          sts16(row + (sw ^ 16), w[4], w[5], w[6], w[7]);
+        } else {
+          sts16(row, w[0], w[1], w[2], w[3]);
+        }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        // lane 0's row is the piece's first; a piece wholly outside the matrix is not sent
+        if (lane == 0 && row_ok && col0 < p.N) bulk_store_2d(stage.tm, stage.buf, col0, m);
+        return;
+      }
+      if (!row_ok) return;
+      int8_t* dst = reinterpret_cast<int8_t*>(p.out) + (long long)m * p.out_ld + col0;
       if constexpr (NC == 32) {
         if (wide && col0 + 32 <= p.N) {
           st32(dst, w);
@@ -173,6 +213,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
         if (col0 + 16 <= p.N) st16(dst, w[0], w[1], w[2], w[3]);
       }
     } else {
+      if (!row_ok) return;
       uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
       uint32_t w[NC / 2];
 #pragma unroll
@@ -198,7 +239,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
 template <int BN, bool INT8, int ACT, int OUTK, int EW>
 __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const float* e_cs, const float* e_bias,
                                                  const float* e_post, uint32_t taddr, int m, bool row_ok, float rs,
-                                                 int n0, int cpart) {
+                                                 int n0, int cpart, const OutStage& stage) {
   constexpr int CH = BN / (EW / 4);
   // 32-byte stores need a 32-byte aligned row segment: base pointer and row pitch multiples of 32 bytes
   const int es = (OUTK == OUT_I8 || OUTK == OUT_F8) ? 1 : (OUTK == OUT_FP ? 2 : 4);
@@ -213,8 +254,8 @@ __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const floa
       if (c + 1 < NCH) ptx::tmem_ld32(taddr + (c + 1) * 32, (c & 1) ? ra : rb);
       const int jw = c * 32;                // column of the chunk's first element among this warp's columns
       const int jc = cpart * CH + jw;       // ... and inside the tile
-      if (c & 1) epilogue_chunk<INT8, ACT, OUTK, 32>(p, rb, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
-      else epilogue_chunk<INT8, ACT, OUTK, 32>(p, ra, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
+      if (c & 1) epilogue_chunk<INT8, ACT, OUTK, 32>(p, rb, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide, stage);
+      else epilogue_chunk<INT8, ACT, OUTK, 32>(p, ra, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide, stage);
     }
   } else {
     constexpr int NCH = CH / 16;
@@ -226,8 +267,8 @@ __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const floa
       if (c + 1 < NCH) ptx::tmem_ld16(taddr + (c + 1) * 16, (c & 1) ? ra : rb);
       const int jw = c * 16;
       const int jc = cpart * CH + jw;
-      if (c & 1) epilogue_chunk<INT8, ACT, OUTK, 16>(p, rb, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
-      else epilogue_chunk<INT8, ACT, OUTK, 16>(p, ra, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide);
+      if (c & 1) epilogue_chunk<INT8, ACT, OUTK, 16>(p, rb, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide, stage);
+      else epilogue_chunk<INT8, ACT, OUTK, 16>(p, ra, e_cs + jw, e_bias + jw, e_post + jw, m, row_ok, rs, n0 + jc, wide, stage);
     }
   }
 }
@@ -237,8 +278,9 @@ __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const floa
 // waiting on them.  ROWS = output rows per tile (128, or 256 for a CTA pair of which this CTA owns rows row_off..+127).
 template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR, int EW>
 __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, uint64_t* acc_full, uint64_t* acc_empty,
-                                              uint32_t tmem_base, int first_tile, int tile_stride, int row_off) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+                                              uint32_t tmem_base, int first_tile, int tile_stride, int row_off,
+                                              const OutStage& stage, int warp) {   // warp: index among the epilogue warps
+  const int lane = threadIdx.x & 31;
   const int quarter = warp & 3, cpart = warp >> 2;
   constexpr int CH = BN / (EW / 4);          // columns per thread and tile
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;
@@ -303,7 +345,7 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     ptx::tc_fence_after();
     {
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + cpart * CH;
-      epilogue_columns<BN, INT8, ACT, OUTK, EW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart);
+      epilogue_columns<BN, INT8, ACT, OUTK, EW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart, stage);
     }
     // hand the accumulator buffer back to the UMMA issuer
     ptx::tc_fence_before();
@@ -313,6 +355,7 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
       else ptx::mbar_arrive(&acc_empty[as]);
     }
   }
+  if (stage.buf && lane == 0) bulk_store_wait_all();         // the unit is through with this CTA's shared memory
 }
 
 template <int BN, bool INT8, int ACT, int OUTK>
@@ -425,7 +468,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------------ epilogue (warps 0-7)
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
     ptx::pdl_wait();                                     // before this warp's first global access
-    epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0);
+    epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0,
+                                                           OutStage{nullptr, nullptr}, warp);
   }
 
   ptx::tc_fence_before();
@@ -488,11 +532,14 @@ static hero_status dispatch_epilogue(hero_handle* h, const CUtensorMap& tmA, con
 // own 128 rows of A and its own 128 of the 256 W rows (32 KB per k-block instead of 48 KB for the same number
 // of MACs per SM, which is what the L2 -> SM path limits), the leader CTA's elected lane issues M = 256 UMMAs
 // that read both CTAs' shared memory, and each CTA's tensor memory receives its 128 accumulator rows.
-//   full[s]      (leader's copy) : the leader's producer thread loads all four half-tiles (two into the peer's
-//                                  shared memory); every copy completes on this barrier
-//   empty[s]     (every CTA)     : the leader's commit is multicast to both CTAs
+//   full[s]      (leader's copy) : each CTA's producer loads its own two half-tiles into its own shared memory; all
+//                                  four copies complete on this barrier, which the leader arms with the total byte count
+//   empty[s]     (every CTA)     : the leader's commit is multicast to both CTAs (each producer waits on its own copy)
 //   acc_full[a]  (every CTA)     : the leader's commit is multicast to both CTAs
-//   acc_empty[a] (leader's copy) : all 16 epilogue warps of the pair arrive on it
+//   acc_empty[a] (leader's copy) : all epilogue warps of the pair arrive on it
+// The two single-lane loops (producer, UMMA issuer) are serial chains that must turn a k-block around every ~500 cycles
+// beside the epilogue warps: they are kept short (loop-invariant addresses and descriptors computed once, uniform
+// control flow) and the copies are split between the two CTAs' producers.
 // No multicast TMA load is used anywhere.
 // ------------------------------------------------------------------------------------------------------
 struct PairCfg {
@@ -503,18 +550,21 @@ struct PairCfg {
   static constexpr int STAGES = 6;
   static constexpr int TMEM_COLS = 2 * BN;
   static constexpr int EPI_FLOATS = 4 * 2 * 3 * BN;
-  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256;
+  static constexpr int OUT_STAGE_BYTES = 8192;                   // 8 warps x (32 rows x 32 B) or 16 warps x (32 rows x 16 B)
+  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + OUT_STAGE_BYTES + EPI_FLOATS * 4 + 256;
 };
 
 template <bool INT8, int ACT, int OUTK, int EW>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW + 2) * 32, 1)
-gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const GemmParams p) {
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                 const __grid_constant__ CUtensorMap tmO, const GemmParams p) {
   using Cfg = PairCfg;
   constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* tiles = smem;
-  float* epi = reinterpret_cast<float*>(smem + STAGES * Cfg::STAGE_BYTES);
+  uint8_t* out_stage = smem + STAGES * Cfg::STAGE_BYTES;
+  float* epi = reinterpret_cast<float*>(out_stage + Cfg::OUT_STAGE_BYTES);
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi + Cfg::EPI_FLOATS);
   uint64_t* full = bars;
   uint64_t* empty = bars + STAGES;
@@ -524,6 +574,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  constexpr int W_TMA = EW, W_MMA = EW + 1;            // warps 0 .. EW-1: epilogue
   const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;   // 256 x 256 tiles
   const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
@@ -533,11 +584,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 2 * EW); }
     ptx::fence_mbar_init();
   }
-  if (warp == EW + 1) {
+  if (warp == W_MMA) {
     ptx::tmem_alloc_pair(tmem_slot, Cfg::TMEM_COLS);
     ptx::tmem_relinquish_pair();
   }
-  if (warp == EW && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); }
+  if (warp == W_TMA && lane == 0) { ptx::prefetch_tmap(&tmA); ptx::prefetch_tmap(&tmW); if (p.tma_out) ptx::prefetch_tmap(&tmO); }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::cluster_sync();                                   // both CTAs' barriers exist before any remote arrive
@@ -545,13 +596,23 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
   ptx::pdl_launch_dependents();
 
-  if (warp == EW) {
-    // ------------------------------------------------------------------ TMA producer (leader CTA only)
-    // One thread feeds both CTAs: its own halves of A and W go to local shared memory, the peer's halves to the
-    // peer's shared memory, all four copies completing on the leader's `full` barrier.  The peer needs no producer,
-    // so the stage hand-off costs one barrier round trip, not a cross-CTA chain.
-    if (lane == 0 && rank == 0) {
+  if (warp == W_TMA) {
+    // ------------------------------------------------------------------ TMA producer (one in each CTA of the pair)
+    // Each CTA's producer loads its own halves of A and W into its own shared memory; all four copies of a k-block
+    // complete on the LEADER's `full` barrier (the leader arms it with the byte count of both CTAs; bytes that land
+    // before the arming only run the count negative for a moment).  A CTA's stage is free when the leader's commit,
+    // multicast to both CTAs, has arrived on its own `empty` barrier.  One thread can start a bulk tensor copy only
+    // every ~90 cycles: four copies per k-block from one thread took most of the ~500 cycles a k-block lasts on the
+    // tensor core, two from each of two threads run side by side.
+    // The whole warp walks the loop (uniform control flow: the addresses stay in the uniform datapath) and one elected
+    // lane issues; everything that does not change from one k-block to the next is computed once.
+    {
+      const bool issue = ptx::elect_one();
       const int kelems = GEMM_BK_BYTES / p.elem_bytes;
+      // cluster addresses are linear in the offset: one mapping for this CTA's tiles, one for the leader's barriers
+      const uint32_t dst = ptx::mapa(ptx::smem_u32(tiles), rank);
+      const uint32_t bar0 = ptx::mapa(ptx::smem_u32(&full[0]), 0);
+      const int ra = (int)rank * GEMM_BM, rw = (int)rank * (BN / 2);   // this CTA's rows of the A and W tiles
       int stage = 0; uint32_t phase = 0; bool ok = true;
       // The weights are constants of the model: the W halves of the first tile's first stages are requested before the
       // dependency wait, the activation halves after it (all complete the same barrier).
@@ -559,31 +620,32 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (pair_id < num_tiles) {
         int mt, nt; tile_coords(pair_id, p.num_m_tiles, p.num_n_tiles, mt, nt);
         pre = min(p.num_kb, STAGES);
-        for (int kb = 0; kb < pre; ++kb) {
-          const uint32_t b_loc = ptx::smem_u32(tiles + kb * Cfg::STAGE_BYTES) + Cfg::A_BYTES;
-          const uint32_t bar = ptx::mapa(ptx::smem_u32(&full[kb]), 0);
-          ptx::mbar_expect_tx(&full[kb], 2 * Cfg::STAGE_BYTES);
-#pragma unroll
-          for (int r = 0; r < 2; ++r) ptx::tma_load_2d_pair(ptx::mapa(b_loc, r), &tmW, kb * kelems, nt * BN + r * (BN / 2), bar);
+        if (issue) {
+          for (int kb = 0; kb < pre; ++kb) {
+            if (rank == 0) ptx::mbar_expect_tx(&full[kb], 2 * Cfg::STAGE_BYTES);
+            ptx::tma_load_2d_pair(dst + kb * Cfg::STAGE_BYTES + Cfg::A_BYTES, &tmW, kb * kelems, nt * BN + rw, bar0 + 8 * kb);
+          }
         }
       }
       ptx::pdl_wait();                                   // the previous kernel's outputs are complete and visible from here on
+      bool first = true;
       for (int t = pair_id; t < num_tiles && ok; t += num_pairs) {
         int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
-        for (int kb = 0; kb < p.num_kb; ++kb) {
-          const bool early = t == pair_id && kb < pre;   // barrier armed and W requested above
+        const int ya = mt * 256 + ra, yw = nt * BN + rw;
+        int x = 0;
+        for (int kb = 0; kb < p.num_kb; ++kb, x += kelems) {
+          const bool early = first && kb < pre;          // barrier armed and W requested above
           if (!early && !ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x700 | stage)) { ok = false; break; }
-          const uint32_t a_loc = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
-          const uint32_t b_loc = a_loc + Cfg::A_BYTES;
-          const uint32_t bar = ptx::mapa(ptx::smem_u32(&full[stage]), 0);
-          if (!early) ptx::mbar_expect_tx(&full[stage], 2 * Cfg::STAGE_BYTES);
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            ptx::tma_load_2d_pair(ptx::mapa(a_loc, r), &tmA, kb * kelems, mt * 256 + r * GEMM_BM, bar);
-            if (!early) ptx::tma_load_2d_pair(ptx::mapa(b_loc, r), &tmW, kb * kelems, nt * BN + r * (BN / 2), bar);
+          if (issue) {
+            const uint32_t off = stage * Cfg::STAGE_BYTES;
+            const uint32_t bar = bar0 + 8 * stage;
+            if (!early && rank == 0) ptx::mbar_expect_tx(&full[stage], 2 * Cfg::STAGE_BYTES);
+            ptx::tma_load_2d_pair(dst + off, &tmA, x, ya, bar);
+            if (!early) ptx::tma_load_2d_pair(dst + off + Cfg::A_BYTES, &tmW, x, yw, bar);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
+        first = false;
       }
       for (int i = 0; i < STAGES; ++i) {                 // drain: every copy started here has been consumed
         if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x780 | stage)) break;
@@ -591,11 +653,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == EW + 1) {
+  } else if (warp == W_MMA) {
     // ------------------------------------------------------------------ UMMA issuer (leader CTA only)
     ptx::pdl_wait();
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
+      // descriptors differ from stage to stage and k-slice to k-slice only in the start-address field (address >> 4,
+      // far from overflowing its 14 bits): one base per operand, small additions afterwards
+      const uint64_t ad0 = ptx::smem_desc(desc_base, ptx::smem_u32(tiles));
+      const uint64_t bd0 = ptx::smem_desc(desc_base, ptx::smem_u32(tiles) + Cfg::A_BYTES);
       int stage = 0; uint32_t phase = 0; bool ok = true;
       int it = 0;
       for (int t = pair_id; t < num_tiles && ok; t += num_pairs, ++it) {
@@ -607,46 +674,63 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int kb = 0; kb < p.num_kb; ++kb) {
           if (!ptx::mbar_wait(&full[stage], phase, p.err, 0x900 | stage)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t a_addr = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
-          const uint32_t b_addr = a_addr + Cfg::A_BYTES;
+          if (issue) {
+            const uint32_t so = (uint32_t)(stage * Cfg::STAGE_BYTES) >> 4;
 #pragma unroll
-          for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
-            const uint64_t ad = ptx::smem_desc(desc_base, a_addr + k * 32);
-            const uint64_t bd = ptx::smem_desc(desc_base, b_addr + k * 32);
-            if constexpr (INT8) ptx::umma_i8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-            else if (p.f8) ptx::umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-            else ptx::umma_f16_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
+              const uint64_t ad = ad0 + (so + 2 * k), bd = bd0 + (so + 2 * k);
+              if constexpr (INT8) ptx::umma_i8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+              else if (p.f8) ptx::umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+              else ptx::umma_f16_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            }
+            ptx::umma_commit_pair(&empty[stage], 3);     // frees this stage in both CTAs
           }
-          ptx::umma_commit_pair(&empty[stage], 3);       // frees this stage in both CTAs
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        if (ok) ptx::umma_commit_pair(&acc_full[as], 3);  // both CTAs' accumulator halves are complete
+        if (ok && issue) ptx::umma_commit_pair(&acc_full[as], 3);  // both CTAs' accumulator halves are complete
       }
     }
     __syncwarp();
   } else {
     ptx::pdl_wait();                                     // before this warp's first global access
     // ------------------------------------------------------------------ epilogue (warps 0 .. EW-1 of each CTA)
-    epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM);
+    OutStage stage{nullptr, &tmO};
+    if (p.tma_out) stage.buf = out_stage + warp * (Cfg::OUT_STAGE_BYTES / EW);
+    epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM, stage,
+                                                      warp);
   }
 
   ptx::tc_fence_before();
   __syncthreads();
   ptx::cluster_sync();                                   // the peer may still be reading this CTA's shared memory / barriers
-  if (warp == EW + 1) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
+  if (warp == W_MMA) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
 }
 
 template <bool INT8, int ACT, int OUTK, int EW>
-static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmParams& p,
+static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, GemmParams p,
                                        cudaStream_t stream) {
   auto kern = gemm_pair_kernel<INT8, ACT, OUTK, EW>;
+  // an 8-bit output leaves through per-warp bulk tensor stores (box: 32 rows x the bytes one lane holds per piece) when
+  // its base and row pitch allow a tensor map; otherwise, and for wider outputs, every lane stores its own row
+  CUtensorMap tmO;
+  memset(&tmO, 0, sizeof(tmO));
+  p.tma_out = 0;
+  if constexpr (OUTK == OUT_I8 || OUTK == OUT_F8) {
+    constexpr int NC = EW == 8 ? 32 : 16;
+    if (aligned16(p.out) && p.out_ld % 16 == 0) {
+      hero_status st = make_tmap_2d(h, &tmO, p.out, 1, false, false, (uint64_t)p.M, (uint64_t)p.N, (uint64_t)p.out_ld, NC, 32,
+                                    NC == 32 ? 32 : 0);
+      if (st != HERO_OK) return st;
+      p.tma_out = 1;
+    }
+  }
   HERO_SMEM_OPT_IN(h, kern, PairCfg::SMEM_BYTES);
   const int tiles = p.num_m_tiles * p.num_n_tiles;
   const int pairs_max = h->sm_count / 2;
   const int pairs = tiles < pairs_max ? tiles : pairs_max;
   {
     LaunchScope scope(h, stream, KERNEL_GEMM);
-    HERO_CUDA(launch_dependent(kern, dim3(2 * pairs), dim3((EW + 2) * 32), PairCfg::SMEM_BYTES, stream, tmA, tmW, p));
+    HERO_CUDA(launch_dependent(kern, dim3(2 * pairs), dim3((EW + 2) * 32), PairCfg::SMEM_BYTES, stream, tmA, tmW, tmO, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;
@@ -802,3 +886,4 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   if (t128 >= enough) return run_bn<128>(h, a, p, s);
   return run_bn<64>(h, a, p, s);
 }
+

@@ -27,6 +27,7 @@ struct GemmParams {
   uint32_t idesc;
   int elem_bytes;           // 1 (INT8, e4m3) or 2 (F16 / BF16)
   int f8;                   // operands are e4m3 (kind::f8f6f4; FP32 accumulators, scales as for INT8)
+  int tma_out;              // the 8-bit output leaves through bulk tensor stores (CTA-pair kernel)
   int* err;
 };
 
@@ -43,40 +44,40 @@ struct GemmCfg {
 
 constexpr float ROUND_MAGIC = 12582912.0f;   // 1.5 * 2^23
 
-// GELU(v) = v Phi(v) = max(v, 0) - 0.5 |v| E(|v| / sqrt 2) with E(z) = erfc(z) for z >= 0, evaluated with the
-// rational-exponential form erfc(z) ~ (a1 t + ... + a5 t^5) exp(-z^2), t = 1 / (1 + p z) (absolute error
-// below 1.5e-7 for every z >= 0): branch-free, two special-function ops, no cancellation for negative v.
+// GELU(v) = v Phi(v) = max(v, 0) - 0.5 a erfc(a / sqrt 2) with a = |v|.  log2 erfc(a / sqrt 2) is close to a parabola, so
+// a degree-6 polynomial P(a) (fitted on [0, 6] with the weight a erfc: what an error in P does to the result) gives
+// erfc(a / sqrt 2) = 2^P(a) with one special-function op per element and no reciprocal: absolute error of the GELU
+// below 1.5e-7 everywhere (8.4e-8 from the polynomial in FP32 Horner form, the rest from ex2.approx).  Beyond a = 6 the
+// term is below 1e-8 and a is clamped (the polynomial is not meant for larger arguments).  Branch-free, no
+// cancellation for negative v.
+constexpr float GELU_P0 = 6.939127616e-06f, GELU_P1 = -1.151201725e+00f, GELU_P2 = -4.587709606e-01f,
+                GELU_P3 = -5.341210961e-02f, GELU_P4 = 8.080720901e-03f, GELU_P5 = -7.692211657e-04f,
+                GELU_P6 = 3.309298336e-05f;
 __device__ __forceinline__ float gelu_erf_f(float v) {
-  const float av = fabsf(v);
-  float t;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(av, 0.3275911f * 0.70710678118654752440f, 1.0f)));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  poly *= t;
+  const float a = fminf(fabsf(v), 6.0f);
+  float q = fmaf(GELU_P6, a, GELU_P5);
+  q = fmaf(q, a, GELU_P4);
+  q = fmaf(q, a, GELU_P3);
+  q = fmaf(q, a, GELU_P2);
+  q = fmaf(q, a, GELU_P1);
+  q = fmaf(q, a, GELU_P0);
   float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(v * v * -0.72134752044448170368f));   // exp(-v^2 / 2)
-  return fmaf(-0.5f * av, poly * e, fmaxf(v, 0.0f));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(q));                   // erfc(a / sqrt 2)
+  return fmaf(-0.5f * a, e, fmaxf(v, 0.0f));
 }
-// the same on a packed pair: the polynomial and the products run as FFMA2 / FMUL2, two special-function ops per element
+// the same on a packed pair: the polynomial runs as six FFMA2, one special-function op per element
 __device__ __forceinline__ float2 gelu_erf_f2(float2 v) {
-  const float2 av = make_float2(fabsf(v.x), fabsf(v.y));
-  const float kz = 0.3275911f * 0.70710678118654752440f;
-  const float2 d = __ffma2_rn(av, make_float2(kz, kz), make_float2(1.0f, 1.0f));
-  float2 t;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.x) : "f"(d.x));
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.y) : "f"(d.y));
-  float2 poly = __ffma2_rn(make_float2(1.061405429f, 1.061405429f), t, make_float2(-1.453152027f, -1.453152027f));
-  poly = __ffma2_rn(poly, t, make_float2(1.421413741f, 1.421413741f));
-  poly = __ffma2_rn(poly, t, make_float2(-0.284496736f, -0.284496736f));
-  poly = __ffma2_rn(poly, t, make_float2(0.254829592f, 0.254829592f));
-  poly = __fmul2_rn(poly, t);
-  const float2 q = __fmul2_rn(__fmul2_rn(v, make_float2(-0.72134752044448170368f, -0.72134752044448170368f)), v);
+  const float2 a = make_float2(fminf(fabsf(v.x), 6.0f), fminf(fabsf(v.y), 6.0f));
+  float2 q = __ffma2_rn(make_float2(GELU_P6, GELU_P6), a, make_float2(GELU_P5, GELU_P5));
+  q = __ffma2_rn(q, a, make_float2(GELU_P4, GELU_P4));
+  q = __ffma2_rn(q, a, make_float2(GELU_P3, GELU_P3));
+  q = __ffma2_rn(q, a, make_float2(GELU_P2, GELU_P2));
+  q = __ffma2_rn(q, a, make_float2(GELU_P1, GELU_P1));
+  q = __ffma2_rn(q, a, make_float2(GELU_P0, GELU_P0));
   float2 e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(q.x));                // exp(-v^2 / 2)
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(q.x));
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(q.y));
-  const float2 w = __fmul2_rn(__fmul2_rn(av, make_float2(-0.5f, -0.5f)), __fmul2_rn(poly, e));
+  const float2 w = __fmul2_rn(__fmul2_rn(a, make_float2(-0.5f, -0.5f)), e);
   return __fadd2_rn(w, make_float2(fmaxf(v.x, 0.0f), fmaxf(v.y, 0.0f)));
 }
 __device__ __forceinline__ float gelu_tanh_f(float x) {
