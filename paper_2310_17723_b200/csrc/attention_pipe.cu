@@ -325,7 +325,10 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   reg_dec<PIPE_REGS_HELPER>();                             // the helper group (its fourth warp has no work)
   if (warp == PIPE_TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // (The three helper loops are walked by the whole warp, one elected lane issuing: with uniform control flow the
+    // addresses stay in the uniform datapath, and a helper's turn-around time is part of every hand-off.)
+    {
+      const bool issue = ptx::elect_one();
       uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
       bool ok = true;
       for (PipeWalk w(p, blockIdx.x, gridDim.x); w.t < total_tiles && ok; w.next()) {
@@ -334,21 +337,27 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int row_base = g.b * p.S, col0 = g.h * DH;
         const int qb = wcnt & 1;
         if (!pipe_wait(&q_empty[qb], ((wcnt >> 1) & 1) ^ 1, p.err, 0x7000 | qb)) { ok = false; break; }
-        ptx::mbar_expect_tx(&q_full[qb], Cfg::Q_TILE);
-        ptx::tma_load_2d(sQ + qb * Cfg::Q_TILE, &tmQ, col0, row_base + g.qt * ATT_BM, &q_full[qb]);
+        if (issue) {
+          ptx::mbar_expect_tx(&q_full[qb], Cfg::Q_TILE);
+          ptx::tma_load_2d(sQ + qb * Cfg::Q_TILE, &tmQ, col0, row_base + g.qt * ATT_BM, &q_full[qb]);
+        }
         const bool stash = g.nb > NRING;
         for (int k = 0; k < g.nb && ok; ++k, ++kcnt) {       // K blocks of 64 keys in Q K^T order
           const int j = pipe_qk_block(g.nb, stash, k);
           const int ks = kcnt % KST;
           if (!pipe_wait(&k_empty[ks], ((kcnt / KST) & 1) ^ 1, p.err, 0x7100 | ks)) { ok = false; break; }
-          ptx::mbar_expect_tx(&k_full[ks], Cfg::K_TILE);
-          ptx::tma_load_2d(sK + ks * Cfg::K_TILE, &tmK, col0, row_base + j * PB, &k_full[ks]);
+          if (issue) {
+            ptx::mbar_expect_tx(&k_full[ks], Cfg::K_TILE);
+            ptx::tma_load_2d(sK + ks * Cfg::K_TILE, &tmK, col0, row_base + j * PB, &k_full[ks]);
+          }
         }
         for (int j = 0; j < g.nb && ok; ++j, ++vcnt) {       // V blocks of 64 keys in P V order
           const int vs = vcnt % VST;
           if (!pipe_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x7200 | vs)) { ok = false; break; }
-          ptx::mbar_expect_tx(&v_full[vs], Cfg::V_TILE);
-          ptx::tma_load_2d(sV + vs * Cfg::V_TILE, &tmV, col0, row_base + j * PB, &v_full[vs]);
+          if (issue) {
+            ptx::mbar_expect_tx(&v_full[vs], Cfg::V_TILE);
+            ptx::tma_load_2d(sV + vs * Cfg::V_TILE, &tmV, col0, row_base + j * PB, &v_full[vs]);
+          }
         }
         ++wcnt;
       }
@@ -356,8 +365,11 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     __syncwarp();
   } else if (warp == PIPE_QK_WARP) {
     // ------------------------------------------------------------------ Q K^T issuer: block after block, tile after tile
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t kmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // Q, K: K-major rows of DH bytes
+      // descriptors differ only in the start-address field (address >> 4): one base per operand, small additions later
+      const uint64_t qd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sQ)), kd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sK));
       uint32_t wcnt = 0, kcnt = 0;
       RingPos<NRING> ring;
       bool ok = true;
@@ -366,7 +378,7 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (!w.tile(p, g)) continue;
         const int qb = wcnt & 1;
         if (!pipe_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x8000 | qb)) { ok = false; break; }
-        const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::Q_TILE);
+        const uint64_t qd = qd0 + (uint32_t)((qb * Cfg::Q_TILE) >> 4);
         for (int k = 0; k < g.nb && ok; ++k, ++kcnt, ring.advance(1)) {
           const int ks = kcnt % KST, blk = ring.idx;
           if (!pipe_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8100 | ks)) { ok = false; break; }
@@ -374,27 +386,29 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           // that went to the stash) is through with it
           if (!pipe_wait(&s_free[blk], ring.par ^ 1, p.err, 0x8200 | blk)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::K_TILE);
+          if (issue) {
+            const uint64_t kd = kd0 + (uint32_t)((ks * Cfg::K_TILE) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < DH / 32; ++kk) {
-            if constexpr (F8) ptx::umma_f8(tmem_base + blk * PB, ptx::smem_desc(kmaj, q_addr + kk * 32),
-                                           ptx::smem_desc(kmaj, k_addr + kk * 32), p.idesc_qk, kk != 0);
-            else ptx::umma_i8(tmem_base + blk * PB, ptx::smem_desc(kmaj, q_addr + kk * 32),
-                              ptx::smem_desc(kmaj, k_addr + kk * 32), p.idesc_qk, kk != 0);
+            for (int kk = 0; kk < DH / 32; ++kk) {
+              if constexpr (F8) ptx::umma_f8(tmem_base + blk * PB, qd + 2 * kk, kd + 2 * kk, p.idesc_qk, kk != 0);
+              else ptx::umma_i8(tmem_base + blk * PB, qd + 2 * kk, kd + 2 * kk, p.idesc_qk, kk != 0);
+            }
+            ptx::umma_commit(&s_full[blk]);
+            ptx::umma_commit(&k_empty[ks]);
           }
-          ptx::umma_commit(&s_full[blk]);
-          ptx::umma_commit(&k_empty[ks]);
         }
-        if (ok) ptx::umma_commit(&q_empty[qb]);
+        if (ok && issue) ptx::umma_commit(&q_empty[qb]);
         ++wcnt;
       }
     }
     __syncwarp();
   } else if (warp == PIPE_PV_WARP) {
     // ------------------------------------------------------------------ P V issuer
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t pmaj = ptx::smem_desc_base(16, 512, ptx::SWZ_64B);        // P: K-major rows of 64 bytes
       constexpr uint64_t vmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // V: MN-major, 8-key groups
+      const uint64_t pd0 = ptx::smem_desc(pmaj, ptx::smem_u32(sP)), vd0 = ptx::smem_desc(vmaj, ptx::smem_u32(sV));
       uint32_t wcnt = 0, vcnt = 0, pcnt = 0;
       bool ok = true;
       for (PipeWalk w(p, blockIdx.x, gridDim.x); w.t < total_tiles && ok; w.next()) {
@@ -407,19 +421,18 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           if (!pipe_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x8600 | vs)) { ok = false; break; }
           if (!pipe_wait(&p_full[pb], (pcnt / PIPE_NPB) & 1, p.err, 0x8700 | pb)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
-          const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::V_TILE);
+          if (issue) {
+            const uint64_t pd = pd0 + (uint32_t)((pb * Cfg::P_TILE) >> 4), vd = vd0 + (uint32_t)((vs * Cfg::V_TILE) >> 4);
 #pragma unroll
-          for (int k = 0; k < PB / 32; ++k) {
-            if constexpr (F8) ptx::umma_f8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                                           ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
-            else ptx::umma_i8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                              ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
+            for (int k = 0; k < PB / 32; ++k) {
+              if constexpr (F8) ptx::umma_f8(tmem_base + Cfg::O_COL, pd + 2 * k, vd + (uint32_t)((k * 32 * DH) >> 4), p.idesc_pv, (i | k) != 0);
+              else ptx::umma_i8(tmem_base + Cfg::O_COL, pd + 2 * k, vd + (uint32_t)((k * 32 * DH) >> 4), p.idesc_pv, (i | k) != 0);
+            }
+            ptx::umma_commit(&v_empty[vs]);
+            ptx::umma_commit(&p_empty[pb]);
           }
-          ptx::umma_commit(&v_empty[vs]);
-          ptx::umma_commit(&p_empty[pb]);
         }
-        if (ok) ptx::umma_commit(o_full);
+        if (ok && issue) ptx::umma_commit(o_full);
         ++wcnt;
       }
     }
