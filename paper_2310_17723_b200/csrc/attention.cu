@@ -102,8 +102,14 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // ------------------------------------------------------------------ TMA producer
     // The rings run on across tile boundaries, so the next tile's Q and first K blocks are already in
     // flight while the softmax warps finish the current tile.
-    if (lane == 0) {
-      uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
+    // (The helper loops are walked by the whole warp, one elected lane issuing: with uniform control flow the addresses
+    // stay in the uniform datapath; ring positions advance without divisions.  A helper's turn-around time is part of
+    // every hand-off.)
+    {
+      const bool issue = ptx::elect_one();
+      RingPos<KST> kr;
+      RingPos<VST> vr;
+      uint32_t wcnt = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         int qt, h, b, klen; attn_tile(p, t, qt, h, b);
@@ -112,21 +118,27 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int row_base = b * p.S, col0 = h * DH;
         const int qb = wcnt & 1;
         if (!ptx::mbar_wait(&q_empty[qb], ((wcnt >> 1) & 1) ^ 1, p.err, 0x1000 | qb)) { ok = false; break; }
-        ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
-        ptx::tma_load_2d(sQ + qb * Cfg::TILE, &tmQ, col0, row_base + qt * ATT_BM, &q_full[qb]);
+        if (issue) {
+          ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
+          ptx::tma_load_2d(sQ + qb * Cfg::TILE, &tmQ, col0, row_base + qt * ATT_BM, &q_full[qb]);
+        }
         for (int i = 0; i < 2 * nkv; ++i) {
           const int j = i < nkv ? i : i - nkv;
-          const int ks = kcnt % KST;
-          if (!ptx::mbar_wait(&k_empty[ks], ((kcnt / KST) & 1) ^ 1, p.err, 0x1100 | ks)) { ok = false; break; }
-          ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
-          ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
-          ++kcnt;
+          const int ks = kr.idx;
+          if (!ptx::mbar_wait(&k_empty[ks], kr.par ^ 1, p.err, 0x1100 | ks)) { ok = false; break; }
+          if (issue) {
+            ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
+            ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
+          }
+          kr.advance(1);
           if (i >= nkv) {
-            const int vs = vcnt % VST;
-            if (!ptx::mbar_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x1200 | vs)) { ok = false; break; }
-            ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
-            ptx::tma_load_2d(sV + vs * Cfg::TILE, &tmV, col0, row_base + j * ATT_BN, &v_full[vs]);
-            ++vcnt;
+            const int vs = vr.idx;
+            if (!ptx::mbar_wait(&v_empty[vs], vr.par ^ 1, p.err, 0x1200 | vs)) { ok = false; break; }
+            if (issue) {
+              ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
+              ptx::tma_load_2d(sV + vs * Cfg::TILE, &tmV, col0, row_base + j * ATT_BN, &v_full[vs]);
+            }
+            vr.advance(1);
           }
         }
         ++wcnt;
@@ -135,30 +147,36 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncwarp();
   } else if (warp == ATT_MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t kmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // Q, K: K-major rows of DH bytes
       constexpr uint64_t pmaj = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);      // P: K-major rows of 128 bytes
       constexpr uint64_t vmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);       // V: MN-major, 8-key groups
-      uint32_t kcnt = 0, vcnt = 0, scnt = 0, pcnt = 0, wcnt = 0;
+      // descriptors differ only in the start-address field (address >> 4): one base per operand, small additions later
+      const uint64_t qd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sQ)), kd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sK));
+      const uint64_t pd0 = ptx::smem_desc(pmaj, ptx::smem_u32(sP)), vd0 = ptx::smem_desc(vmaj, ptx::smem_u32(sV));
+      RingPos<KST> kr;
+      RingPos<VST> vr;
+      RingPos<ATT_NSB> sr;
+      uint32_t pcnt = 0, wcnt = 0;
       bool ok = true;
 
       auto issue_pv = [&](int j) -> bool {
         if (j == 0 && !ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x2500)) return false;   // previous tile's O read out
-        const int vs = vcnt % VST, pb = pcnt & 1;
-        if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x2100 | vs)) return false;
+        const int vs = vr.idx, pb = pcnt & 1;
+        if (!ptx::mbar_wait(&v_full[vs], vr.par, p.err, 0x2100 | vs)) return false;
         if (!ptx::mbar_wait(&p_full[pb], (pcnt >> 1) & 1, p.err, 0x2200 | pb)) return false;
         ptx::tc_fence_after();
-        const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
-        const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
+        if (issue) {
+          const uint64_t pd = pd0 + (uint32_t)((pb * Cfg::P_TILE) >> 4), vd = vd0 + (uint32_t)((vs * Cfg::TILE) >> 4);
 #pragma unroll
-        for (int k = 0; k < ATT_BN / 32; ++k)
-          if constexpr (F8) ptx::umma_f8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                                         ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (j | k) != 0);
-          else ptx::umma_i8(tmem_base + Cfg::O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                            ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (j | k) != 0);
-        ptx::umma_commit(&v_empty[vs]);
-        ptx::umma_commit(&p_empty[pb]);
-        ++vcnt; ++pcnt;
+          for (int k = 0; k < ATT_BN / 32; ++k)
+            if constexpr (F8) ptx::umma_f8(tmem_base + Cfg::O_COL, pd + 2 * k, vd + (uint32_t)((k * 32 * DH) >> 4), p.idesc_pv, (j | k) != 0);
+            else ptx::umma_i8(tmem_base + Cfg::O_COL, pd + 2 * k, vd + (uint32_t)((k * 32 * DH) >> 4), p.idesc_pv, (j | k) != 0);
+          ptx::umma_commit(&v_empty[vs]);
+          ptx::umma_commit(&p_empty[pb]);
+        }
+        vr.advance(1); ++pcnt;
         return true;
       };
 
@@ -168,27 +186,27 @@ attn_int8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (nkv == 0) continue;
         const int qb = wcnt & 1;
         if (!ptx::mbar_wait(&q_full[qb], (wcnt >> 1) & 1, p.err, 0x2000 | qb)) { ok = false; break; }
-        const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
+        const uint64_t qd = qd0 + (uint32_t)((qb * Cfg::TILE) >> 4);
         for (int i = 0; i < 2 * nkv && ok; ++i) {
-          const int ks = kcnt % KST, sb = scnt % ATT_NSB;
-          if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x2300 | ks)) { ok = false; break; }
-          if (!ptx::mbar_wait(&s_empty[sb], ((scnt / ATT_NSB) & 1) ^ 1, p.err, 0x2400 | sb)) { ok = false; break; }
+          const int ks = kr.idx, sb = sr.idx;
+          if (!ptx::mbar_wait(&k_full[ks], kr.par, p.err, 0x2300 | ks)) { ok = false; break; }
+          if (!ptx::mbar_wait(&s_empty[sb], sr.par ^ 1, p.err, 0x2400 | sb)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+          if (issue) {
+            const uint64_t kd = kd0 + (uint32_t)((ks * Cfg::TILE) >> 4);
 #pragma unroll
-          for (int k = 0; k < DH / 32; ++k)
-            if constexpr (F8) ptx::umma_f8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                                           ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
-            else ptx::umma_i8(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                              ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
-          ptx::umma_commit(&k_empty[ks]);
-          ptx::umma_commit(&s_full[sb]);
-          ++kcnt; ++scnt;
-          if (i == 2 * nkv - 1) ptx::umma_commit(&q_empty[qb]);   // Q buffer free once these MMAs have read it
+            for (int k = 0; k < DH / 32; ++k)
+              if constexpr (F8) ptx::umma_f8(tmem_base + sb * ATT_BN, qd + 2 * k, kd + 2 * k, p.idesc_qk, k != 0);
+              else ptx::umma_i8(tmem_base + sb * ATT_BN, qd + 2 * k, kd + 2 * k, p.idesc_qk, k != 0);
+            ptx::umma_commit(&k_empty[ks]);
+            ptx::umma_commit(&s_full[sb]);
+            if (i == 2 * nkv - 1) ptx::umma_commit(&q_empty[qb]);   // Q buffer free once these MMAs have read it
+          }
+          kr.advance(1); sr.advance(1);
           if (i >= nkv + 1) ok = issue_pv(i - nkv - 1);
         }
         if (ok) ok = issue_pv(nkv - 1);
-        if (ok) ptx::umma_commit(o_full);
+        if (ok && issue) ptx::umma_commit(o_full);
         ++wcnt;
       }
     }

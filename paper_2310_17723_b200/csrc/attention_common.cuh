@@ -99,4 +99,22 @@ hero_status attn_resident_dispatch(hero_handle* h, const hero_attn_args* a, Attn
 // INT8 core for S <= 512 as a pipeline of exponential and pack warps; defined in attention_pipe.cu
 hero_status attn_pipe_dispatch(hero_handle* h, const hero_attn_args* a, AttnParams& p, cudaStream_t stream, bool probe);
 
+// A position in a ring of N slots with the phase parity of its barriers, advanced without divisions (the ring depths here are not powers of two).
+template <int N>
+struct RingPos {
+  int idx = 0;
+  uint32_t par = 0;
+  __device__ __forceinline__ void advance(int n) {          // n <= 2 N
+    idx += n;
+    if (idx >= N) { idx -= N; par ^= 1; }
+    if (idx >= N) { idx -= N; par ^= 1; }
+  }
+  // slot and parity k positions further on (k <= N)
+  __device__ __forceinline__ void at(int k, int& slot, uint32_t& parity) const {
+    slot = idx + k; parity = par;
+    if (slot >= N) { slot -= N; parity ^= 1; }
+  }
+};
+
+
 }  // namespace hero

@@ -80,66 +80,86 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
   if (warp == ATT_TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
+    // (helper loops: whole warp, one elected lane issues, ring positions without divisions; see attention.cu)
+    {
+      const bool issue = ptx::elect_one();
+      RingPos<KST> kr;
+      RingPos<VST> vr;
+      RingPos<QB> qr;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         int qt, h, b, klen; attn_tile(p, t, qt, h, b);
         const int nkv = attn_nkv(p, qt, b, klen);
         if (nkv == 0) continue;
         const int row_base = b * p.S, col0 = h * DH;
-        const int qb = wcnt % QB;
-        if (!ptx::mbar_wait(&q_empty[qb], ((wcnt / QB) & 1) ^ 1, p.err, 0x4000 | qb)) { ok = false; break; }
-        ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
-#pragma unroll
-        for (int sIdx = 0; sIdx < NSUB; ++sIdx)
-          ptx::tma_load_2d(sQ + qb * Cfg::TILE + sIdx * Cfg::SUB, &tmQ, col0 + sIdx * 64, row_base + qt * ATT_BM, &q_full[qb]);
-        for (int i = 0; i < 2 * nkv; ++i) {
-          const int j = i < nkv ? i : i - nkv;
-          const int ks = kcnt % KST;
-          if (!ptx::mbar_wait(&k_empty[ks], ((kcnt / KST) & 1) ^ 1, p.err, 0x4100 | ks)) { ok = false; break; }
-          ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
+        const int qb = qr.idx;
+        if (!ptx::mbar_wait(&q_empty[qb], qr.par ^ 1, p.err, 0x4000 | qb)) { ok = false; break; }
+        if (issue) {
+          ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
 #pragma unroll
           for (int sIdx = 0; sIdx < NSUB; ++sIdx)
-            ptx::tma_load_2d(sK + ks * Cfg::TILE + sIdx * Cfg::SUB, &tmK, col0 + sIdx * 64, row_base + j * ATT_BN, &k_full[ks]);
-          ++kcnt;
-          if (i >= nkv) {
-            const int vs = vcnt % VST;
-            if (!ptx::mbar_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x4200 | vs)) { ok = false; break; }
-            ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
+            ptx::tma_load_2d(sQ + qb * Cfg::TILE + sIdx * Cfg::SUB, &tmQ, col0 + sIdx * 64, row_base + qt * ATT_BM, &q_full[qb]);
+        }
+        for (int i = 0; i < 2 * nkv; ++i) {
+          const int j = i < nkv ? i : i - nkv;
+          const int ks = kr.idx;
+          if (!ptx::mbar_wait(&k_empty[ks], kr.par ^ 1, p.err, 0x4100 | ks)) { ok = false; break; }
+          if (issue) {
+            ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
 #pragma unroll
             for (int sIdx = 0; sIdx < NSUB; ++sIdx)
-              ptx::tma_load_2d(sV + vs * Cfg::TILE + sIdx * Cfg::SUB, &tmV, col0 + sIdx * 64, row_base + j * ATT_BN, &v_full[vs]);
-            ++vcnt;
+              ptx::tma_load_2d(sK + ks * Cfg::TILE + sIdx * Cfg::SUB, &tmK, col0 + sIdx * 64, row_base + j * ATT_BN, &k_full[ks]);
+          }
+          kr.advance(1);
+          if (i >= nkv) {
+            const int vs = vr.idx;
+            if (!ptx::mbar_wait(&v_empty[vs], vr.par ^ 1, p.err, 0x4200 | vs)) { ok = false; break; }
+            if (issue) {
+              ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
+#pragma unroll
+              for (int sIdx = 0; sIdx < NSUB; ++sIdx)
+                ptx::tma_load_2d(sV + vs * Cfg::TILE + sIdx * Cfg::SUB, &tmV, col0 + sIdx * 64, row_base + j * ATT_BN, &v_full[vs]);
+            }
+            vr.advance(1);
           }
         }
-        ++wcnt;
+        qr.advance(1);
       }
     }
     __syncwarp();
   } else if (warp == ATT_MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t kmaj = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);          // Q, K, P: K-major, 128-byte rows
       constexpr uint64_t vmaj = ptx::smem_desc_base(Cfg::SUB, 1024, ptx::SWZ_128B);    // V: MN-major; 64-feature chunks SUB apart
-      uint32_t kcnt = 0, vcnt = 0, scnt = 0, pcnt = 0, wcnt = 0;
+      // descriptors differ only in the start-address field (address >> 4): one base per operand, small additions later
+      const uint64_t qd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sQ)), kd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sK));
+      const uint64_t pd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sP)), vd0 = ptx::smem_desc(vmaj, ptx::smem_u32(sV));
+      RingPos<KST> kr;
+      RingPos<VST> vr;
+      RingPos<ATT_NSB> sr;
+      RingPos<PB> pr;
+      RingPos<QB> qr;
+      uint32_t wcnt = 0;
       bool ok = true;
 
       auto issue_pv = [&](int j) -> bool {
         if (j == 0 && !ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x5500)) return false;
-        const int vs = vcnt % VST, pb = pcnt % PB;
-        if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x5100 | vs)) return false;
-        if (!ptx::mbar_wait(&p_full[pb], (pcnt / PB) & 1, p.err, 0x5200 | pb)) return false;
+        const int vs = vr.idx, pb = pr.idx;
+        if (!ptx::mbar_wait(&v_full[vs], vr.par, p.err, 0x5100 | vs)) return false;
+        if (!ptx::mbar_wait(&p_full[pb], pr.par, p.err, 0x5200 | pb)) return false;
         ptx::tc_fence_after();
-        const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
-        const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
+        if (issue) {
+          const uint64_t pd = pd0 + (uint32_t)((pb * Cfg::P_TILE) >> 4), vd = vd0 + (uint32_t)((vs * Cfg::TILE) >> 4);
 #pragma unroll
-        for (int k = 0; k < ATT_BN / 16; ++k)      // 16 keys per MMA: 2 eight-key groups of V, 32 bytes of a P row
-          ptx::umma_f16(tmem_base + Cfg::O_COL, ptx::smem_desc(kmaj, p_addr + (k >> 2) * Cfg::SUB + (k & 3) * 32),
-                        ptx::smem_desc(vmaj, v_addr + k * 2048), p.idesc_pv, (j | k) != 0);
-        ptx::umma_commit(&v_empty[vs]);
-        ptx::umma_commit(&p_empty[pb]);
-        ++vcnt; ++pcnt;
+          for (int k = 0; k < ATT_BN / 16; ++k)    // 16 keys per MMA: 2 eight-key groups of V, 32 bytes of a P row
+            ptx::umma_f16(tmem_base + Cfg::O_COL, pd + (uint32_t)(((k >> 2) * Cfg::SUB + (k & 3) * 32) >> 4),
+                          vd + (uint32_t)((k * 2048) >> 4), p.idesc_pv, (j | k) != 0);
+          ptx::umma_commit(&v_empty[vs]);
+          ptx::umma_commit(&p_empty[pb]);
+        }
+        vr.advance(1); pr.advance(1);
         return true;
       };
 
@@ -147,27 +167,31 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         int qt, h, b, klen; attn_tile(p, t, qt, h, b);
         const int nkv = attn_nkv(p, qt, b, klen);
         if (nkv == 0) continue;
-        const int qb = wcnt % QB;
-        if (!ptx::mbar_wait(&q_full[qb], (wcnt / QB) & 1, p.err, 0x5000 | qb)) { ok = false; break; }
-        const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
+        const int qb = qr.idx;
+        if (!ptx::mbar_wait(&q_full[qb], qr.par, p.err, 0x5000 | qb)) { ok = false; break; }
+        const uint64_t qd = qd0 + (uint32_t)((qb * Cfg::TILE) >> 4);
         for (int i = 0; i < 2 * nkv && ok; ++i) {
-          const int ks = kcnt % KST, sb = scnt % ATT_NSB;
-          if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x5300 | ks)) { ok = false; break; }
-          if (!ptx::mbar_wait(&s_empty[sb], ((scnt / ATT_NSB) & 1) ^ 1, p.err, 0x5400 | sb)) { ok = false; break; }
+          const int ks = kr.idx, sb = sr.idx;
+          if (!ptx::mbar_wait(&k_full[ks], kr.par, p.err, 0x5300 | ks)) { ok = false; break; }
+          if (!ptx::mbar_wait(&s_empty[sb], sr.par ^ 1, p.err, 0x5400 | sb)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+          if (issue) {
+            const uint64_t kd = kd0 + (uint32_t)((ks * Cfg::TILE) >> 4);
 #pragma unroll
-          for (int k = 0; k < DH / 16; ++k)
-            ptx::umma_f16(tmem_base + sb * ATT_BN, ptx::smem_desc(kmaj, q_addr + (k >> 2) * Cfg::SUB + (k & 3) * 32),
-                          ptx::smem_desc(kmaj, k_addr + (k >> 2) * Cfg::SUB + (k & 3) * 32), p.idesc_qk, k != 0);
-          ptx::umma_commit(&k_empty[ks]);
-          ptx::umma_commit(&s_full[sb]);
-          ++kcnt; ++scnt;
-          if (i == 2 * nkv - 1) ptx::umma_commit(&q_empty[qb]);
+            for (int k = 0; k < DH / 16; ++k) {
+              const uint32_t o = (uint32_t)(((k >> 2) * Cfg::SUB + (k & 3) * 32) >> 4);
+              ptx::umma_f16(tmem_base + sb * ATT_BN, qd + o, kd + o, p.idesc_qk, k != 0);
+            }
+            ptx::umma_commit(&k_empty[ks]);
+            ptx::umma_commit(&s_full[sb]);
+            if (i == 2 * nkv - 1) ptx::umma_commit(&q_empty[qb]);
+          }
+          kr.advance(1); sr.advance(1);
           if (i >= nkv + 1) ok = issue_pv(i - nkv - 1);
         }
         if (ok) ok = issue_pv(nkv - 1);
-        if (ok) ptx::umma_commit(o_full);
+        if (ok && issue) ptx::umma_commit(o_full);
+        qr.advance(1);
         ++wcnt;
       }
     }

@@ -102,23 +102,6 @@ struct PipeWalk {
   }
 };
 
-// A position in a ring of N slots with the phase parity of its barriers, advanced without divisions (N is 6 or 7).
-template <int N>
-struct RingPos {
-  int idx = 0;
-  uint32_t par = 0;
-  __device__ __forceinline__ void advance(int n) {          // n <= 2 N
-    idx += n;
-    if (idx >= N) { idx -= N; par ^= 1; }
-    if (idx >= N) { idx -= N; par ^= 1; }
-  }
-  // slot and parity k positions further on (k <= N)
-  __device__ __forceinline__ void at(int k, int& slot, uint32_t& parity) const {
-    slot = idx + k; parity = par;
-    if (slot >= N) { slot -= N; parity ^= 1; }
-  }
-};
-
 // A global load that stays where it is written: the compiler may otherwise sink a load to its first use, which here is a
 // whole tile later, on the critical path.
 __device__ __forceinline__ float ld_nc_here(const float* ptr) {

@@ -396,7 +396,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (warp == TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // (this loop and the UMMA issuer's are walked by the whole warp, one elected lane issuing: uniform control flow keeps
+    // the addresses in the uniform datapath, and these serial chains have to keep up with the tensor core)
+    {
+      const bool issue = ptx::elect_one();
       const int kelems = GEMM_BK_BYTES / p.elem_bytes;
       int stage = 0; uint32_t phase = 0; bool ok = true;
       // The weights are constants of the model: the W tiles of the first tile's first stages are requested before the
@@ -405,24 +408,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if ((int)blockIdx.x < num_tiles) {
         int mt, nt; tile_coords(blockIdx.x, p.num_m_tiles, p.num_n_tiles, mt, nt);
         pre = min(p.num_kb, STAGES);
-        for (int kb = 0; kb < pre; ++kb) {
-          ptx::mbar_expect_tx(&full[kb], Cfg::STAGE_BYTES);
-          ptx::tma_load_2d(tiles + kb * Cfg::STAGE_BYTES + Cfg::A_BYTES, &tmW, kb * kelems, nt * BN, &full[kb]);
+        if (issue) {
+          for (int kb = 0; kb < pre; ++kb) {
+            ptx::mbar_expect_tx(&full[kb], Cfg::STAGE_BYTES);
+            ptx::tma_load_2d(tiles + kb * Cfg::STAGE_BYTES + Cfg::A_BYTES, &tmW, kb * kelems, nt * BN, &full[kb]);
+          }
         }
       }
       ptx::pdl_wait();                                   // the previous kernel's outputs are complete and visible from here on
+      bool first = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         int mt, nt; tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
-        for (int kb = 0; kb < p.num_kb; ++kb) {
-          const bool early = t == (int)blockIdx.x && kb < pre;   // barrier armed and W requested above
+        const int ya = mt * GEMM_BM, yw = nt * BN;
+        int x = 0;
+        for (int kb = 0; kb < p.num_kb; ++kb, x += kelems) {
+          const bool early = first && kb < pre;          // barrier armed and W requested above
           if (!early && !ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x100 | stage)) { ok = false; break; }
-          uint8_t* a_dst = tiles + stage * Cfg::STAGE_BYTES;
-          uint8_t* b_dst = a_dst + Cfg::A_BYTES;
-          if (!early) ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
-          ptx::tma_load_2d(a_dst, &tmA, kb * kelems, mt * GEMM_BM, &full[stage]);
-          if (!early) ptx::tma_load_2d(b_dst, &tmW, kb * kelems, nt * BN, &full[stage]);
+          if (issue) {
+            uint8_t* a_dst = tiles + stage * Cfg::STAGE_BYTES;
+            if (!early) ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
+            ptx::tma_load_2d(a_dst, &tmA, x, ya, &full[stage]);
+            if (!early) ptx::tma_load_2d(a_dst + Cfg::A_BYTES, &tmW, x, yw, &full[stage]);
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
+        first = false;
       }
       // drain: every copy this thread started has landed before the CTA may exit
       for (int i = 0; i < STAGES; ++i) {
@@ -434,8 +444,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else if (warp == MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
     ptx::pdl_wait();
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
+      // descriptors differ only in the start-address field (address >> 4): one base per operand, small additions later
+      const uint64_t ad0 = ptx::smem_desc(desc_base, ptx::smem_u32(tiles));
+      const uint64_t bd0 = ptx::smem_desc(desc_base, ptx::smem_u32(tiles) + Cfg::A_BYTES);
       int stage = 0; uint32_t phase = 0; bool ok = true;
       int it = 0;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
@@ -447,20 +461,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int kb = 0; kb < p.num_kb; ++kb) {
           if (!ptx::mbar_wait(&full[stage], phase, p.err, 0x300 | stage)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t a_addr = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
-          const uint32_t b_addr = a_addr + Cfg::A_BYTES;
+          if (issue) {
+            const uint32_t so = (uint32_t)(stage * Cfg::STAGE_BYTES) >> 4;
 #pragma unroll
-          for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
-            const uint64_t ad = ptx::smem_desc(desc_base, a_addr + k * 32);
-            const uint64_t bd = ptx::smem_desc(desc_base, b_addr + k * 32);
-            if constexpr (INT8) ptx::umma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-            else if (p.f8) ptx::umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-            else ptx::umma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
+              const uint64_t ad = ad0 + (so + 2 * k), bd = bd0 + (so + 2 * k);
+              if constexpr (INT8) ptx::umma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+              else if (p.f8) ptx::umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+              else ptx::umma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+            }
+            ptx::umma_commit(&empty[stage]);    // frees the smem stage once these MMAs have read it
           }
-          ptx::umma_commit(&empty[stage]);      // frees the smem stage once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        if (ok) ptx::umma_commit(&acc_full[as]);  // accumulator of this tile complete
+        if (ok && issue) ptx::umma_commit(&acc_full[as]);  // accumulator of this tile complete
       }
     }
     __syncwarp();
