@@ -171,11 +171,14 @@ def peak_regime(clocks, peaks):
     if not clocks or not clocks.get("sm_mhz"):
         return "burst", "no clock samples"
     mx = clocks.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0)
-    if "sw_power_cap" in (clocks.get("reasons") or []):
-        return "sustained", "sw_power_cap active during the timed region"
+    capped = "sw_power_cap" in (clocks.get("reasons") or [])
+    # the clock decides: a cap that shows up in some samples while the median clock stays at the maximum has not slowed
+    # the timed region down, and comparing with the sustained figure would flatter the kernel
     if clocks["sm_mhz"] < 0.93 * mx:
-        return "sustained", "median SM clock %.0f MHz below 0.93 x %.0f" % (clocks["sm_mhz"], mx)
-    return "burst", "SM clock at %.0f of %.0f MHz, no power cap" % (clocks["sm_mhz"], mx)
+        return "sustained", "median SM clock %.0f MHz below 0.93 x %.0f%s" % (clocks["sm_mhz"], mx,
+                                                                             ", sw_power_cap active" if capped else "")
+    return "burst", "median SM clock %.0f of %.0f MHz%s" % (clocks["sm_mhz"], mx,
+                                                          " (sw_power_cap seen in some samples)" if capped else "")
 
 
 def dominant_kernel(kern, workload, peaks, peak_kind, clocks):

@@ -85,23 +85,33 @@ __device__ __forceinline__ float4 lds_f4(const float* p) {
 // NC (16 or 32) columns of one output row: v = acc * rs * cs[j] + bias[j];  a = act(v) * post[j];
 // INT8: clip(Round(a)) | FP16 / BF16: a | INT32: acc.  Per-column vectors come from shared memory four at a time,
 // the arithmetic runs on packed FP32 pairs, the row segment leaves in 32-byte stores when the output allows it.
-// How a warp's piece of an 8-bit output tile (32 rows x NC bytes) leaves the SM.  Straight from registers every lane writes
-// its own row: 32 different 128-byte lines per store instruction, which the load/store pipe takes one line at a time,
-// in competition with the tensor core's operand reads from shared memory.  Instead the piece is put together in a small
-// per-warp buffer in shared memory (NC = 32: the 32-byte swizzle of the tensor map, so that the lanes' 16-byte writes
-// spread over all banks) and one lane hands it to the TMA unit as a bulk tensor store, which also clips rows and
-// columns beyond the matrix.  The buffer is reused as soon as the unit has read it.
+// How a CTA's 128 x 256 piece of an 8-bit output tile leaves the SM when the epilogue sets the pace (few k-blocks per
+// tile).  Straight from registers every lane writes its own row: 32 different 128-byte lines per store instruction,
+// which the load/store pipe takes one line at a time.  Instead the epilogue warps put the piece together in shared
+// memory (two halves of 128 rows x 128 bytes in the tensor map's 128-byte swizzle, so that the lanes' 16-byte writes
+// spread over all banks) and meet a store warp on a named barrier; its elected lane hands each half to the TMA unit as a
+// bulk tensor store, which also clips rows and columns beyond the matrix, waits until the unit has read the tile and
+// then arrives on a second named barrier, which the epilogue warps pass before their first write of the next tile
+// (long after, as a rule).  The staging area is the pipeline's last stage, which a launch of this kind leaves unused
+// (five stages feed a short main loop as well as six).
 struct OutStage {
-  uint8_t* buf;               // this warp's buffer (NULL: direct stores)
-  const CUtensorMap* tm;      // box = 32 rows x NC bytes
+  uint8_t* buf;               // the CTA's staging tile (NULL: direct stores)
+  const CUtensorMap* tm;      // box = 128 rows x 128 bytes
+  uint32_t lane_off;          // this lane's row: byte offset of the row in a half, and its swizzle term
+  uint32_t lane_sw;
+  int n0;                     // first column of the tile being processed
+  bool fresh;                 // nothing of the current tile has been staged yet
+  int nthreads;               // threads on the two named barriers: epilogue warps + store warp
 };
+constexpr int BAR_STAGED = 1, BAR_DRAINED = 2;   // named barriers: tile staged (epilogue -> store warp), tile read (back)
+constexpr int OUT_HALF_BYTES = GEMM_BM * 128;
 __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_store_2d(const CUtensorMap* tm, const void* smem_src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(ptx::smem_u32(smem_src)) : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
+__device__ __forceinline__ void bulk_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void sts16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -109,7 +119,7 @@ __device__ __forceinline__ void sts16(uint32_t addr, uint32_t a, uint32_t b, uin
 template <bool INT8, int ACT, int OUTK, int NC>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32_t (&r)[NC], const float* e_cs,
                                                const float* e_bias, const float* e_post, int m, bool row_ok, float rs,
-                                               int col0, bool wide, const OutStage& stage) {
+                                               int col0, bool wide, OutStage& stage) {
   if constexpr (OUTK == OUT_I32) {
     if (!row_ok) return;
     int* dst = reinterpret_cast<int*>(p.out) + (long long)m * p.out_ld + col0;
@@ -182,22 +192,16 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
         else w[g] = low_bytes4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
       }
       if (stage.buf) {
-        // every lane takes part (rows past the end are clipped by the store)
-        const int lane = threadIdx.x & 31;
-        if (lane == 0) bulk_store_wait_read();               // the previous piece has left the buffer
-        __syncwarp();
-        const uint32_t row = ptx::smem_u32(stage.buf) + lane * NC;
-        if constexpr (NC == 32) {
-          const uint32_t sw = ((lane >> 2) & 1) << 4;        // 32-byte swizzle: 16-byte half ^= bit 7 of the address
-          sts16(row + sw, w[0], w[1], w[2], w[3]);
-          sts16(row + (sw ^ 16), w[4], w[5], w[6], w[7]);
-        } else {
-          sts16(row, w[0], w[1], w[2], w[3]);
+        // this lane's NC bytes of its row of the staging tile (rows past the end are clipped by the store)
+        if (stage.fresh) {                                   // the unit has read the previous tile out of the staging area
+          asm volatile("bar.sync %0, %1;" ::"n"(BAR_DRAINED), "r"(stage.nthreads) : "memory");
+          stage.fresh = false;
         }
-        ptx::fence_proxy_async_smem();
-        __syncwarp();
-        // lane 0's row is the piece's first; a piece wholly outside the matrix is not sent
-        if (lane == 0 && row_ok && col0 < p.N) bulk_store_2d(stage.tm, stage.buf, col0, m);
+        const int jc = col0 - stage.n0;                      // column inside the tile
+        const uint32_t half = ptx::smem_u32(stage.buf) + (jc >> 7) * OUT_HALF_BYTES + stage.lane_off;
+        const uint32_t c16 = (jc & 127) >> 4;
+        sts16(half + (((c16) ^ stage.lane_sw) << 4), w[0], w[1], w[2], w[3]);
+        if constexpr (NC == 32) sts16(half + (((c16 + 1) ^ stage.lane_sw) << 4), w[4], w[5], w[6], w[7]);
         return;
       }
       if (!row_ok) return;
@@ -239,7 +243,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
 template <int BN, bool INT8, int ACT, int OUTK, int EW>
 __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const float* e_cs, const float* e_bias,
                                                  const float* e_post, uint32_t taddr, int m, bool row_ok, float rs,
-                                                 int n0, int cpart, const OutStage& stage) {
+                                                 int n0, int cpart, OutStage& stage) {
   constexpr int CH = BN / (EW / 4);
   // 32-byte stores need a 32-byte aligned row segment: base pointer and row pitch multiples of 32 bytes
   const int es = (OUTK == OUT_I8 || OUTK == OUT_F8) ? 1 : (OUTK == OUT_FP ? 2 : 4);
@@ -279,17 +283,18 @@ __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const floa
 template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR, int EW>
 __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, uint64_t* acc_full, uint64_t* acc_empty,
                                               uint32_t tmem_base, int first_tile, int tile_stride, int row_off,
-                                              const OutStage& stage, int warp) {   // warp: index among the epilogue warps
+                                              OutStage stage, int warp) {   // warp: index among the epilogue warps
   const int lane = threadIdx.x & 31;
   const int quarter = warp & 3, cpart = warp >> 2;
   constexpr int CH = BN / (EW / 4);          // columns per thread and tile
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;
   bool ok = true;
 
-  // Every warp stages the per-column vectors of its own CH columns in a shared-memory area of its own (two buffers,
-  // 3 x CH floats each), so the epilogue warps never wait for one another.
+  // Every warp stages the per-column vectors of its own CH columns in a shared-memory area of its own (3 x CH floats:
+  // written at the start of a tile, after the warp's last read of the previous tile's), so the epilogue warps never
+  // wait for one another.
   constexpr int NV = CH / 32;                // values per lane and vector
-  float* epi_w = epi + warp * (2 * 3 * CH);
+  float* epi_w = epi + warp * (3 * CH);
   float ncs[NV], nbias[NV], npost[NV], nrs = 1.0f;
   TileWalk walk;                             // stands at the tile whose vectors are fetched next
   walk.init(first_tile, p.num_m_tiles, p.num_n_tiles);
@@ -313,7 +318,8 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
   };
   auto publish = [&](int it) {               // registers -> this tile's shared-memory vectors
     if constexpr (OUTK != OUT_I32) {
-      float* e = epi_w + (it & 1) * 3 * CH;
+      float* e = epi_w;
+      __syncwarp();                          // every lane is through with the previous tile's vectors
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
         if constexpr (ACT == HERO_ACT_NONE) {    // (acc rs cs + b) post = acc rs (cs post) + b post
@@ -336,13 +342,15 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     const float rs = nrs;
     publish(it);
     if (t + tile_stride < num_tiles) fetch();
-    const float* e_cs = epi_w + (it & 1) * 3 * CH;
+    const float* e_cs = epi_w;
     const int m = mt * ROWS + row_off + quarter * 32 + lane;
     const bool row_ok = m < p.M;
 
     // a wait that gave up has recorded its code; the warp runs on without waiting again so that the kernel ends promptly
     if (ok && !ptx::mbar_wait(&acc_full[as], aphase, p.err, 0x400 | as)) ok = false;
     ptx::tc_fence_after();
+    stage.n0 = n0;
+    stage.fresh = it > 0;                                  // (the first tile finds the staging area unused)
     {
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + cpart * CH;
       epilogue_columns<BN, INT8, ACT, OUTK, EW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart, stage);
@@ -354,8 +362,12 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
       if constexpr (PAIR) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(ptx::smem_u32(&acc_empty[as]), 0));
       else ptx::mbar_arrive(&acc_empty[as]);
     }
+    if (stage.buf) {
+      // this warp's part of the staged tile is complete (writes made visible to the TMA unit)
+      ptx::fence_proxy_async_smem();
+      asm volatile("bar.sync %0, %1;" ::"n"(BAR_STAGED), "r"(stage.nthreads) : "memory");
+    }
   }
-  if (stage.buf && lane == 0) bulk_store_wait_all();         // the unit is through with this CTA's shared memory
 }
 
 template <int BN, bool INT8, int ACT, int OUTK>
@@ -483,7 +495,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
     ptx::pdl_wait();                                     // before this warp's first global access
     epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0,
-                                                           OutStage{nullptr, nullptr}, warp);
+                                                           OutStage{nullptr, nullptr, 0, 0, 0, false, 0}, warp);
   }
 
   ptx::tc_fence_before();
@@ -556,6 +568,34 @@ static hero_status dispatch_epilogue(hero_handle* h, const CUtensorMap& tmA, con
 // control flow) and the copies are split between the two CTAs' producers.
 // No multicast TMA load is used anywhere.
 // ------------------------------------------------------------------------------------------------------
+// The store warp of a launch with staged output: for every tile of this CTA, in the epilogue warps' order, wait until the
+// tile is staged, send its two halves, wait until the unit has read them, tell the epilogue warps.
+template <int ROWS>
+__device__ __forceinline__ void store_warp_loop(const GemmParams& p, const CUtensorMap* tm, uint8_t* buf, int first_tile,
+                                                int tile_stride, int row_off, int nthreads) {
+  const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+  const bool issue = ptx::elect_one();
+  TileWalk walk;
+  walk.init(first_tile, p.num_m_tiles, p.num_n_tiles);
+  for (int t = first_tile; t < num_tiles; t += tile_stride) {
+    int mt, nt; walk.coords(mt, nt);
+    walk.advance(tile_stride);
+    asm volatile("bar.sync %0, %1;" ::"n"(BAR_STAGED), "r"(nthreads) : "memory");
+    if (issue) {
+      const int m0 = mt * ROWS + row_off, n0 = nt * 256;
+      if (m0 < p.M) {
+        bulk_store_2d(tm, buf, n0, m0);
+        if (n0 + 128 < p.N) bulk_store_2d(tm, buf + OUT_HALF_BYTES, n0 + 128, m0);
+      }
+      bulk_store_commit();
+      bulk_store_wait_read();
+    }
+    __syncwarp();
+    if (t + tile_stride < num_tiles) asm volatile("bar.arrive %0, %1;" ::"n"(BAR_DRAINED), "r"(nthreads) : "memory");
+  }
+  if (issue) bulk_store_wait_all();                          // the unit is through with this CTA's shared memory
+}
+
 struct PairCfg {
   static constexpr int BN = 256;
   static constexpr int A_BYTES = GEMM_BM * GEMM_BK_BYTES;        // this CTA's 128 rows of A
@@ -563,38 +603,40 @@ struct PairCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = 6;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int EPI_FLOATS = 4 * 2 * 3 * BN;
-  static constexpr int OUT_STAGE_BYTES = 8192;                   // 8 warps x (32 rows x 32 B) or 16 warps x (32 rows x 16 B)
-  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + OUT_STAGE_BYTES + EPI_FLOATS * 4 + 256;
+  static constexpr int EPI_FLOATS = 4 * 3 * BN;                  // per-warp cs / bias / post
+  static_assert(STAGE_BYTES == 2 * OUT_HALF_BYTES, "the last stage doubles as the output staging tile");
+  static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256;
 };
 
 template <bool INT8, int ACT, int OUTK, int EW>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW + 2) * 32, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW + 3) * 32, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmO, const GemmParams p) {
   using Cfg = PairCfg;
-  constexpr int BN = Cfg::BN, STAGES = Cfg::STAGES;
+  constexpr int BN = Cfg::BN;
+  // with staged output the last pipeline stage is the staging tile
+  const int STAGES = p.tma_out ? Cfg::STAGES - 1 : Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* tiles = smem;
-  uint8_t* out_stage = smem + STAGES * Cfg::STAGE_BYTES;
-  float* epi = reinterpret_cast<float*>(out_stage + Cfg::OUT_STAGE_BYTES);
+  uint8_t* out_stage = smem + (Cfg::STAGES - 1) * Cfg::STAGE_BYTES;
+  float* epi = reinterpret_cast<float*>(smem + Cfg::STAGES * Cfg::STAGE_BYTES);
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi + Cfg::EPI_FLOATS);
   uint64_t* full = bars;
-  uint64_t* empty = bars + STAGES;
-  uint64_t* acc_full = bars + 2 * STAGES;
+  uint64_t* empty = bars + Cfg::STAGES;
+  uint64_t* acc_full = bars + 2 * Cfg::STAGES;
   uint64_t* acc_empty = acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  constexpr int W_TMA = EW, W_MMA = EW + 1;            // warps 0 .. EW-1: epilogue
+  constexpr int W_TMA = EW, W_MMA = EW + 1, W_ST = EW + 2;   // warps 0 .. EW-1: epilogue; W_ST: store warp (staged output)
   const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;   // 256 x 256 tiles
   const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < Cfg::STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 2 * EW); }
     ptx::fence_mbar_init();
   }
@@ -705,11 +747,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
     __syncwarp();
+  } else if (warp == W_ST) {
+    // ------------------------------------------------------------------ store warp
+    if (p.tma_out) store_warp_loop<256>(p, &tmO, out_stage, pair_id, num_pairs, (int)rank * GEMM_BM, (EW + 1) * 32);
   } else {
     ptx::pdl_wait();                                     // before this warp's first global access
     // ------------------------------------------------------------------ epilogue (warps 0 .. EW-1 of each CTA)
-    OutStage stage{nullptr, &tmO};
-    if (p.tma_out) stage.buf = out_stage + warp * (Cfg::OUT_STAGE_BYTES / EW);
+    const int row = (warp & 3) * 32 + lane;                // this lane's row of the CTA's 128
+    OutStage stage{p.tma_out ? out_stage : nullptr, &tmO, (uint32_t)row * 128u, (uint32_t)row & 7u, 0, false, (EW + 1) * 32};
     epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM, stage,
                                                       warp);
   }
@@ -724,16 +769,17 @@ template <bool INT8, int ACT, int OUTK, int EW>
 static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, const CUtensorMap& tmW, GemmParams p,
                                        cudaStream_t stream) {
   auto kern = gemm_pair_kernel<INT8, ACT, OUTK, EW>;
-  // an 8-bit output leaves through per-warp bulk tensor stores (box: 32 rows x the bytes one lane holds per piece) when
-  // its base and row pitch allow a tensor map; otherwise, and for wider outputs, every lane stores its own row
+  // an 8-bit output of a short-K product leaves through a staging tile and bulk tensor stores when its base and row
+  // pitch allow a tensor map; otherwise, and for wider outputs, every lane stores its own row
   CUtensorMap tmO;
   memset(&tmO, 0, sizeof(tmO));
   p.tma_out = 0;
   if constexpr (OUTK == OUT_I8 || OUTK == OUT_F8) {
-    constexpr int NC = EW == 8 ? 32 : 16;
-    if (aligned16(p.out) && p.out_ld % 16 == 0) {
-      hero_status st = make_tmap_2d(h, &tmO, p.out, 1, false, false, (uint64_t)p.M, (uint64_t)p.N, (uint64_t)p.out_ld, NC, 32,
-                                    NC == 32 ? 32 : 0);
+    // worth it where the epilogue sets the pace: few k-blocks per tile (a long main loop hides the direct stores and
+    // keeps all six pipeline stages)
+    if (p.num_kb <= 16 && aligned16(p.out) && p.out_ld % 16 == 0) {
+      hero_status st = make_tmap_2d(h, &tmO, p.out, 1, false, false, (uint64_t)p.M, (uint64_t)p.N, (uint64_t)p.out_ld, 128,
+                                    GEMM_BM, 128);
       if (st != HERO_OK) return st;
       p.tma_out = 1;
     }
@@ -744,7 +790,7 @@ static hero_status launch_gemm_pair_ew(hero_handle* h, const CUtensorMap& tmA, c
   const int pairs = tiles < pairs_max ? tiles : pairs_max;
   {
     LaunchScope scope(h, stream, KERNEL_GEMM);
-    HERO_CUDA(launch_dependent(kern, dim3(2 * pairs), dim3((EW + 2) * 32), PairCfg::SMEM_BYTES, stream, tmA, tmW, tmO, p));
+    HERO_CUDA(launch_dependent(kern, dim3(2 * pairs), dim3((EW + 3) * 32), PairCfg::SMEM_BYTES, stream, tmA, tmW, tmO, p));
   }
   HERO_CUDA(cudaGetLastError());
   return HERO_OK;

@@ -38,7 +38,7 @@ struct GemmCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int EPI_FLOATS = 4 * 2 * 3 * BN;             // per-warp, double-buffered cs / bias / post
+  static constexpr int EPI_FLOATS = 4 * 3 * BN;                 // per-warp cs / bias / post
   static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256 /*barriers*/;
 };
 
@@ -49,36 +49,36 @@ constexpr float ROUND_MAGIC = 12582912.0f;   // 1.5 * 2^23
 // erfc(a / sqrt 2) = 2^P(a) with one special-function op per element and no reciprocal: absolute error of the GELU
 // below 1.5e-7 everywhere (8.4e-8 from the polynomial in FP32 Horner form, the rest from ex2.approx).  Beyond a = 6 the
 // term is below 1e-8 and a is clamped (the polynomial is not meant for larger arguments).  Branch-free, no
-// cancellation for negative v.
+// cancellation for negative v.  Evaluated in n = -a (odd coefficients change sign) with the factor 0.5 folded into the
+// constant term (P0 - 1), so that the result is one fused multiply-add: max(v, 0) + n 2^(P(a) - 1).
 constexpr float GELU_P0 = 6.939127616e-06f, GELU_P1 = -1.151201725e+00f, GELU_P2 = -4.587709606e-01f,
                 GELU_P3 = -5.341210961e-02f, GELU_P4 = 8.080720901e-03f, GELU_P5 = -7.692211657e-04f,
                 GELU_P6 = 3.309298336e-05f;
 __device__ __forceinline__ float gelu_erf_f(float v) {
-  const float a = fminf(fabsf(v), 6.0f);
-  float q = fmaf(GELU_P6, a, GELU_P5);
-  q = fmaf(q, a, GELU_P4);
-  q = fmaf(q, a, GELU_P3);
-  q = fmaf(q, a, GELU_P2);
-  q = fmaf(q, a, GELU_P1);
-  q = fmaf(q, a, GELU_P0);
+  const float n = fmaxf(-fabsf(v), -6.0f);
+  float q = fmaf(GELU_P6, n, -GELU_P5);
+  q = fmaf(q, n, GELU_P4);
+  q = fmaf(q, n, -GELU_P3);
+  q = fmaf(q, n, GELU_P2);
+  q = fmaf(q, n, -GELU_P1);
+  q = fmaf(q, n, GELU_P0 - 1.0f);
   float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(q));                   // erfc(a / sqrt 2)
-  return fmaf(-0.5f * a, e, fmaxf(v, 0.0f));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(q));                   // 0.5 erfc(a / sqrt 2)
+  return fmaf(n, e, fmaxf(v, 0.0f));
 }
-// the same on a packed pair: the polynomial runs as six FFMA2, one special-function op per element
+// the same on a packed pair: seven FFMA2, one special-function op per element
 __device__ __forceinline__ float2 gelu_erf_f2(float2 v) {
-  const float2 a = make_float2(fminf(fabsf(v.x), 6.0f), fminf(fabsf(v.y), 6.0f));
-  float2 q = __ffma2_rn(make_float2(GELU_P6, GELU_P6), a, make_float2(GELU_P5, GELU_P5));
-  q = __ffma2_rn(q, a, make_float2(GELU_P4, GELU_P4));
-  q = __ffma2_rn(q, a, make_float2(GELU_P3, GELU_P3));
-  q = __ffma2_rn(q, a, make_float2(GELU_P2, GELU_P2));
-  q = __ffma2_rn(q, a, make_float2(GELU_P1, GELU_P1));
-  q = __ffma2_rn(q, a, make_float2(GELU_P0, GELU_P0));
+  const float2 n = make_float2(fmaxf(-fabsf(v.x), -6.0f), fmaxf(-fabsf(v.y), -6.0f));
+  float2 q = __ffma2_rn(make_float2(GELU_P6, GELU_P6), n, make_float2(-GELU_P5, -GELU_P5));
+  q = __ffma2_rn(q, n, make_float2(GELU_P4, GELU_P4));
+  q = __ffma2_rn(q, n, make_float2(-GELU_P3, -GELU_P3));
+  q = __ffma2_rn(q, n, make_float2(GELU_P2, GELU_P2));
+  q = __ffma2_rn(q, n, make_float2(-GELU_P1, -GELU_P1));
+  q = __ffma2_rn(q, n, make_float2(GELU_P0 - 1.0f, GELU_P0 - 1.0f));
   float2 e;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(q.x));
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(q.y));
-  const float2 w = __fmul2_rn(__fmul2_rn(a, make_float2(-0.5f, -0.5f)), e);
-  return __fadd2_rn(w, make_float2(fmaxf(v.x, 0.0f), fmaxf(v.y, 0.0f)));
+  return __ffma2_rn(n, e, make_float2(fmaxf(v.x, 0.0f), fmaxf(v.y, 0.0f)));
 }
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   return 0.5f * x * (1.0f + tanhf(0.79788456080286535588f * (x + 0.044715f * x * x * x)));
