@@ -148,6 +148,11 @@ hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* a, void* st
  *          still in flight when the call is made (hero_quantize_weight takes care of this for its own outputs).
  *   out  : [M, N].  A TWQ output is refused (HERO_ERR_UNSUPPORTED): the paper keeps the row
  *          reduction out of GEMM epilogues (Sec. 2.1).
+ *   out_col_absmax : device float[N] or NULL.  Calibration observer fused into the epilogue (Sec. 2.1: the static
+ *          scales come from statistics of the un-quantized layer): out_col_absmax[j] = max(out_col_absmax[j],
+ *          max_i |out[i][j]|) over the values as stored, the same statistic hero_absmax_observe takes from the finished
+ *          tensor, without reading it again.  F16 / BF16 outputs only (HERO_ERR_UNSUPPORTED otherwise); accumulates, so
+ *          zero it before the first calibration batch.
  * K must be a multiple of 16 bytes of elements and N a multiple of 16; M is arbitrary.
  */
 typedef struct {
@@ -160,6 +165,7 @@ typedef struct {
   int32_t act;             /* hero_act */
   const float* post_scale; /* device [N] or NULL */
   hero_tensor out;
+  float* out_col_absmax;   /* device [N] or NULL */
 } hero_linear_args;
 
 hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* a, void* stream);

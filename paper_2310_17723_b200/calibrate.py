@@ -1,6 +1,7 @@
 """Calibration on the device (Sec. 2.1): the un-quantized layer runs in FP16 / BF16 through the library's own
-operators, every tensor at an operator border is observed with hero_absmax_observe (the softmax probabilities by
-the FP attention core), and the weights are folded and quantized column-wise by hero_quantize_weight
+operators; the outputs of the four linear modules are observed by their own epilogues (hero_linear_args.out_col_absmax),
+the softmax probabilities by the FP attention core, the other border tensors (LayerNorm and attention outputs, the
+layer's input) with hero_absmax_observe, and the weights are folded and quantized column-wise by hero_quantize_weight
 (Eq. 2, Eq. 20-23, Eq. 32).  Same statistics and the same result layout as the host-side `prep.calibrate` /
 `prep.fold_quantize`; only argument marshalling happens here."""
 import numpy as np
@@ -46,30 +47,36 @@ def calibrate_gpu(h, cfg, params, x_cal, n_seq, return_output=False):
         if per_tensor:
             stat[name + "_t"] = ct
 
+    def colmax(n):
+        return torch.zeros(n, dtype=torch.float32, device="cuda")
+
     def attn(x_in):
         observe("in", x_in)
         qkv = new(3 * H)
-        h.hero_w8a8_linear(hero.tensor(x_in), Wqkv, hero.tensor(qkv), bias=bqkv)
+        # the outputs of the linear modules are observed by their own epilogues (per-column running maxima; Q, K and V
+        # want one static scale each: the maximum over their column ranges)
+        qkv_f = colmax(3 * H)
+        h.hero_w8a8_linear(hero.tensor(x_in), Wqkv, hero.tensor(qkv), bias=bqkv, out_col_absmax=qkv_f)
         q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
-        for n, t in (("q", q), ("k", k), ("v", v)):
-            observe(n, t, per_feature=False)
+        for i, n in enumerate("qkv"):
+            stat[n + "_t"] = qkv_f[i * H:(i + 1) * H].max().reshape(1)
         xa = new(H)
         stat["p_t"] = torch.zeros(1, dtype=torch.float32, device="cuda")
         h.hero_int8_attention(q, k, v, n_seq, S, nh, dh, hero.tensor(xa), mask=cfg.mask, p_absmax=stat["p_t"])
         observe("attn", xa)
         xo = new(H)
-        h.hero_w8a8_linear(hero.tensor(xa), Wo, hero.tensor(xo), bias=bo)
-        observe("o", xo, per_tensor=False)
+        stat["o_f"] = colmax(H)
+        h.hero_w8a8_linear(hero.tensor(xa), Wo, hero.tensor(xo), bias=bo, out_col_absmax=stat["o_f"])
         return xo
 
     def mlp(x_mid):
         observe("mid", x_mid)
         a = new(F)
-        h.hero_w8a8_linear(hero.tensor(x_mid), W1, hero.tensor(a), bias=b1, act=cfg.act)
-        observe("a", a, per_tensor=False)
+        stat["a_f"] = colmax(F)
+        h.hero_w8a8_linear(hero.tensor(x_mid), W1, hero.tensor(a), bias=b1, act=cfg.act, out_col_absmax=stat["a_f"])
         x2 = new(H)
-        h.hero_w8a8_linear(hero.tensor(a), W2, hero.tensor(x2), bias=b2)
-        observe("x2", x2, per_tensor=False)
+        stat["x2_f"] = colmax(H)
+        h.hero_w8a8_linear(hero.tensor(a), W2, hero.tensor(x2), bias=b2, out_col_absmax=stat["x2_f"])
         return x2
 
     out = new(H)

@@ -217,11 +217,26 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
         if (col0 + 16 <= p.N) st16(dst, w[0], w[1], w[2], w[3]);
       }
     } else {
-      if (!row_ok) return;
-      uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
       uint32_t w[NC / 2];
 #pragma unroll
       for (int g = 0; g < NC / 2; ++g) w[g] = pack2_fp(v[2 * g], v[2 * g + 1], p.out_dt);
+      if (p.obs_col) {
+        // calibration observer: the absolute maximum of every column of this piece over the warp's 32 rows, taken from
+        // the values as stored (non-negative floats order like their bit patterns: an integer warp reduction and an
+        // integer atomic maximum do), lane c reporting column c
+        const int lane = threadIdx.x & 31;
+        uint32_t mine = 0;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          const uint32_t h16 = (w[c >> 1] >> (16 * (c & 1))) & 0x7fffu;          // |x| in the stored 16-bit type
+          const float ax = p.out_dt == HERO_F16 ? __half2float(__ushort_as_half((unsigned short)h16)) : __uint_as_float(h16 << 16);
+          const uint32_t mx = __reduce_max_sync(0xffffffffu, row_ok ? __float_as_uint(ax) : 0u);
+          if (lane == c) mine = mx;
+        }
+        if (lane < NC && col0 + lane < p.N && mine != 0u) atomicMax(reinterpret_cast<unsigned int*>(p.obs_col) + col0 + lane, mine);
+      }
+      if (!row_ok) return;
+      uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + (long long)m * p.out_ld + col0;
       if (wide && col0 + NC <= p.N) {
 #pragma unroll
         for (int g = 0; g < NC / 16; ++g) {
@@ -913,6 +928,8 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   if (q8) HERO_REQUIRE(a->w_scale != nullptr || a->out.dtype == HERO_I32, HERO_ERR_INVALID_ARG, "w_scale is required");
   HERO_REQUIRE(a->act >= HERO_ACT_NONE && a->act <= HERO_ACT_GELU_TANH, HERO_ERR_INVALID_ARG, "unknown activation %d", a->act);
   HERO_REQUIRE(a->A.rows < (1ll << 31) && a->N < (1ll << 31) && K < (1ll << 31), HERO_ERR_UNSUPPORTED, "dimension too large");
+  HERO_REQUIRE(a->out_col_absmax == nullptr || is_fp16ish(a->out.dtype), HERO_ERR_UNSUPPORTED,
+               "out_col_absmax observes an F16 / BF16 output (calibration runs the modules in FP mode)");
   if (a->A.rows == 0) return HERO_OK;
 
   GemmParams p;
@@ -926,12 +943,13 @@ extern "C" hero_status hero_w8a8_linear(hero_handle* h, const hero_linear_args* 
   p.bias = a->bias; p.post = a->post_scale;
   p.out = a->out.data; p.out_ld = a->out.ld; p.out_dt = a->out.dtype;
   p.elem_bytes = eb;
+  p.obs_col = a->out_col_absmax;
   p.err = h->d_error;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // Few rows: streaming W bounds the time.  The tile kernels below give one row-tile N / 64 CTAs at most, each walking
   // the whole K; the few-row kernel splits K over a cluster instead.  It wins whenever M <= 16, and for wider inputs
   // when the tile kernels would leave SMs idle on a long K (measured on the M in {16..128} x K, N in {1024..16384} grid).
-  if (p.M <= GEMM_BM) {
+  if (p.M <= GEMM_BM && p.obs_col == nullptr) {            // (the few-row kernel has no observer)
     const bool idle = (p.N + 63) / 64 < h->sm_count;
     const long long kbytes = K * eb;
     if (p.M <= 16 || (idle && kbytes >= 8192) || (idle && kbytes >= 4096 && p.M <= 32)) return run_skinny(h, a, p, s);

@@ -28,6 +28,7 @@ struct GemmParams {
   int elem_bytes;           // 1 (INT8, e4m3) or 2 (F16 / BF16)
   int f8;                   // operands are e4m3 (kind::f8f6f4; FP32 accumulators, scales as for INT8)
   int tma_out;              // the 8-bit output leaves through bulk tensor stores (CTA-pair kernel)
+  float* obs_col;           // [N] or NULL: running per-column absmax of an FP output (calibration observer)
   int* err;
 };
 

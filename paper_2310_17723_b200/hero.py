@@ -50,7 +50,8 @@ class LnArgs(C.Structure):
 
 class LinearArgs(C.Structure):
     _fields_ = [("A", Tensor), ("W", C.c_void_p), ("N", C.c_int64), ("ldw", C.c_int64), ("w_scale", C.c_void_p),
-                ("bias", C.c_void_p), ("act", C.c_int32), ("post_scale", C.c_void_p), ("out", Tensor)]
+                ("bias", C.c_void_p), ("act", C.c_int32), ("post_scale", C.c_void_p), ("out", Tensor),
+                ("out_col_absmax", C.c_void_p)]
 
 
 class AttnArgs(C.Structure):
@@ -229,11 +230,13 @@ class Handle:
                    fp_out or tensor(None))
         _check(lib().hero_layernorm_quant(self._h, C.byref(a), _stream(stream)))
 
-    def hero_w8a8_linear(self, A, W, out, w_scale=None, bias=None, act="none", post_scale=None, stream=None):
-        """A, out: hero.Tensor; W: torch tensor [N, K] (K contiguous)."""
+    def hero_w8a8_linear(self, A, W, out, w_scale=None, bias=None, act="none", post_scale=None, out_col_absmax=None,
+                         stream=None):
+        """A, out: hero.Tensor; W: torch tensor [N, K] (K contiguous); out_col_absmax: float32 [N] running per-column
+        absolute maximum of an FP16 / BF16 output (calibration observer fused into the epilogue)."""
         assert W.dim() == 2 and W.stride(1) == 1
         a = LinearArgs(A, W.data_ptr(), W.shape[0], W.stride(0), _ptr(w_scale), _ptr(bias),
-                       ACT[act] if isinstance(act, str) else act, _ptr(post_scale), out)
+                       ACT[act] if isinstance(act, str) else act, _ptr(post_scale), out, _ptr(out_col_absmax))
         _check(lib().hero_w8a8_linear(self._h, C.byref(a), _stream(stream)))
 
     def hero_int8_attention(self, q, k, v, B, S, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0, s_p=1.0 / 255,

@@ -51,6 +51,46 @@ def test_absmax_observe_is_exact_and_accumulates(h, dt, rows, cols, pad):
     assert float(t0.item()) == ref.max()
 
 
+# every tile kernel the FP product can take: few rows (1-CTA kernels, three tile widths), many rows (CTA pair), ragged M
+# and N, with and without the GELU, FP16 and BF16
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("M,K,N,act", [(40, 256, 64, "none"), (128, 512, 1024, "gelu_erf"), (300, 1024, 4096, "none"),
+                                       (1300, 512, 2000, "gelu_erf"), (4099, 1024, 3072, "none")])
+def test_linear_epilogue_observer_equals_the_streaming_observer(h, dt, M, K, N, act):
+    # the observer fused into the epilogue sees the values as stored: it must agree exactly with hero_absmax_observe on
+    # the finished tensor, accumulate over calls, and leave columns it was not given alone
+    g = W.rng(9, M + N)
+    t = TORCH_FP[dt]
+    A = torch.from_numpy(g.standard_normal((M, K)).astype(np.float32)).to(t).cuda()
+    Wt = torch.from_numpy((g.standard_normal((N, K)) * 0.05).astype(np.float32)).to(t).cuda()
+    bias = torch.from_numpy((g.standard_normal(N) * 0.1).astype(np.float32)).cuda()
+    out = torch.empty(M, N, dtype=t, device="cuda")
+    fused = torch.zeros(N, dtype=torch.float32, device="cuda")
+    h.hero_w8a8_linear(hero.tensor(A), Wt, hero.tensor(out), bias=bias, act=act, out_col_absmax=fused)
+    ref = torch.zeros(N, dtype=torch.float32, device="cuda")
+    h.hero_absmax_observe(hero.tensor(out), ref, None)
+    h.check()
+    assert torch.equal(fused, ref)
+    assert float(fused.max()) > 0
+    # a second batch: running maxima
+    A2 = (A * 0.5).contiguous()
+    A2[0] = A[0] * 3
+    h.hero_w8a8_linear(hero.tensor(A2), Wt, hero.tensor(out), bias=bias, act=act, out_col_absmax=fused)
+    h.hero_absmax_observe(hero.tensor(out), ref, None)
+    h.check()
+    assert torch.equal(fused, ref)
+
+
+def test_linear_epilogue_observer_refuses_an_int8_output(h):
+    A = torch.zeros(256, 256, dtype=torch.int8, device="cuda")
+    Wt = torch.zeros(256, 256, dtype=torch.int8, device="cuda")
+    out = torch.empty(256, 256, dtype=torch.int8, device="cuda")
+    sc = torch.ones(256, dtype=torch.float32, device="cuda")
+    with pytest.raises(hero.HeroError) as e:
+        h.hero_w8a8_linear(hero.tensor(A), Wt, hero.tensor(out, "fwq", sc), w_scale=sc, out_col_absmax=sc)
+    assert e.value.status == hero.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("K,N,fold", [(256, 192, "none"), (1024, 3072, "both"), (4096, 1024, "in"), (768, 768, "out")])
 def test_quantize_weight_matches_fold_then_eq2(h, K, N, fold):
     rng = np.random.default_rng(K + N)

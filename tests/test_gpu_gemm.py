@@ -58,7 +58,10 @@ def test_int32_extreme_values_bit_exact(h):
     assert np.array_equal(got, O.int_matmul(A, Wt.T.copy()))
 
 
-@pytest.mark.parametrize("M,K,N", [(128, 1024, 4096), (333, 4096, 1024), (16, 1024, 4096), (1024, 1024, 4096), (1500, 256, 4096)])
+# (1300, 512, N): the CTA-pair kernel's staged 8-bit output (short K) with a ragged last row-tile and a last column-tile
+# whose second 128-column half is partly (N = 2000), barely (1936) or not at all (1888) inside the matrix
+@pytest.mark.parametrize("M,K,N", [(128, 1024, 4096), (333, 4096, 1024), (16, 1024, 4096), (1024, 1024, 4096), (1500, 256, 4096),
+                                   (1300, 512, 2000), (1300, 512, 1936), (1300, 512, 1888), (2304, 4096, 1024)])
 def test_requant_epilogue_round_only(h, M, K, N):
     # Eq. 22: dequantize by row and column scale, add the folded bias, Round -> INT8
     A, Wt, rs, cs, bias = W.gemm_case(M, K, N)
