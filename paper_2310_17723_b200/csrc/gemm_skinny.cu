@@ -113,25 +113,33 @@ __global__ void __launch_bounds__(SK_THREADS) gemm_skinny_kernel(const __grid_co
   bool have_acc = false;                    // epilogue warps: this CTA's partial sums reached shared memory
   if (warp == SK_TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // (this loop and the issuer's: whole warp, one elected lane issues; uniform control flow keeps the addresses in the
+    // uniform datapath and the serial chains short)
+    {
+      const bool issue = ptx::elect_one();
       const int kelems = GEMM_BK_BYTES / p.elem_bytes;
       int stage = 0; uint32_t phase = 0;
       // The weights do not depend on the previous kernel of the stream: their first tiles are requested before the
       // dependency wait, the activation tiles after it (both complete the same barrier).
       const int pre = min(kb1 - kb0, STAGES);
-      for (int i = 0; i < pre; ++i) {
-        ptx::mbar_expect_tx(&full[i], Cfg::STAGE_BYTES);
-        ptx::tma_load_2d(tiles + i * Cfg::STAGE_BYTES, &tmW, (kb0 + i) * kelems, n0, &full[i]);
+      if (issue) {
+        for (int i = 0; i < pre; ++i) {
+          ptx::mbar_expect_tx(&full[i], Cfg::STAGE_BYTES);
+          ptx::tma_load_2d(tiles + i * Cfg::STAGE_BYTES, &tmW, (kb0 + i) * kelems, n0, &full[i]);
+        }
       }
       ptx::pdl_wait();
       for (int kb = kb0; kb < kb1; ++kb) {
         uint8_t* w_dst = tiles + stage * Cfg::STAGE_BYTES;
-        if (kb - kb0 >= pre) {
-          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x900 | stage)) break;
-          ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
-          ptx::tma_load_2d(w_dst, &tmW, kb * kelems, n0, &full[stage]);
+        const bool late = kb - kb0 >= pre;
+        if (late && !ptx::mbar_wait(&empty[stage], phase ^ 1, p.err, 0x900 | stage)) break;
+        if (issue) {
+          if (late) {
+            ptx::mbar_expect_tx(&full[stage], Cfg::STAGE_BYTES);
+            ptx::tma_load_2d(w_dst, &tmW, kb * kelems, n0, &full[stage]);
+          }
+          ptx::tma_load_2d(w_dst + Cfg::W_BYTES, &tmX, kb * kelems, 0, &full[stage]);
         }
-        ptx::tma_load_2d(w_dst + Cfg::W_BYTES, &tmX, kb * kelems, 0, &full[stage]);
         if (++stage == STAGES) { stage = 0; phase ^= 1; }
       }
       // drain: every copy this thread started has been consumed before the stages are reused or the CTA exits
@@ -143,27 +151,30 @@ __global__ void __launch_bounds__(SK_THREADS) gemm_skinny_kernel(const __grid_co
     __syncwarp();
   } else if (warp == SK_MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t desc_base = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
+      const uint64_t ad0 = ptx::smem_desc(desc_base, ptx::smem_u32(tiles));
+      const uint64_t bd0 = ptx::smem_desc(desc_base, ptx::smem_u32(tiles) + Cfg::W_BYTES);
       int stage = 0; uint32_t phase = 0; bool ok = true;
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!ptx::mbar_wait(&full[stage], phase, p.err, 0xA00 | stage)) { ok = false; break; }
         ptx::tc_fence_after();
-        const uint32_t w_addr = ptx::smem_u32(tiles + stage * Cfg::STAGE_BYTES);
-        const uint32_t x_addr = w_addr + Cfg::W_BYTES;
+        if (issue) {
+          const uint32_t so = (uint32_t)(stage * Cfg::STAGE_BYTES) >> 4;
 #pragma unroll
-        for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
-          const uint64_t ad = ptx::smem_desc(desc_base, w_addr + k * 32);
-          const uint64_t bd = ptx::smem_desc(desc_base, x_addr + k * 32);
-          const uint32_t accumulate = (kb != kb0 || k != 0) ? 1u : 0u;
-          if constexpr (INT8) ptx::umma_i8(tmem_base, ad, bd, p.idesc, accumulate);
-          else if (p.f8) ptx::umma_f8(tmem_base, ad, bd, p.idesc, accumulate);
-          else ptx::umma_f16(tmem_base, ad, bd, p.idesc, accumulate);
+          for (int k = 0; k < GEMM_BK_BYTES / 32; ++k) {
+            const uint64_t ad = ad0 + (so + 2 * k), bd = bd0 + (so + 2 * k);
+            const uint32_t accumulate = (kb != kb0 || k != 0) ? 1u : 0u;
+            if constexpr (INT8) ptx::umma_i8(tmem_base, ad, bd, p.idesc, accumulate);
+            else if (p.f8) ptx::umma_f8(tmem_base, ad, bd, p.idesc, accumulate);
+            else ptx::umma_f16(tmem_base, ad, bd, p.idesc, accumulate);
+          }
+          ptx::umma_commit(&empty[stage]);
         }
-        ptx::umma_commit(&empty[stage]);
         if (++stage == STAGES) { stage = 0; phase ^= 1; }
       }
-      if (ok) ptx::umma_commit(acc_full);
+      if (ok && issue) ptx::umma_commit(acc_full);
     }
     __syncwarp();
   } else {
