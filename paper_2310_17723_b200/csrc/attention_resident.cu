@@ -178,8 +178,12 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 
   if (warp == ATT_TMA_WARP) {
     // ------------------------------------------------------------------ TMA producer: Q, K blocks, V blocks in P V order
-    if (lane == 0) {
-      uint32_t kcnt = 0, vcnt = 0, wcnt = 0;
+    // (helper loops: whole warp, one elected lane issues, ring positions without divisions; see attention.cu)
+    {
+      const bool issue = ptx::elect_one();
+      RingPos<KST> kr;
+      RingPos<VST> vr;
+      uint32_t wcnt = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         int qt, h, b, klen; attn_tile(p, t, qt, h, b);
@@ -188,20 +192,26 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         const int row_base = b * p.S, col0 = h * DH;
         const int qb = wcnt & 1;
         if (!ptx::mbar_wait(&q_empty[qb], ((wcnt >> 1) & 1) ^ 1, p.err, 0x7000 | qb)) { ok = false; break; }
-        ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
-        ptx::tma_load_2d(sQ + qb * Cfg::TILE, &tmQ, col0, row_base + qt * ATT_BM, &q_full[qb]);
-        for (int j = 0; j < nkv && ok; ++j, ++kcnt) {
-          const int ks = kcnt % KST;
-          if (!ptx::mbar_wait(&k_empty[ks], ((kcnt / KST) & 1) ^ 1, p.err, 0x7100 | ks)) { ok = false; break; }
-          ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
-          ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
+        if (issue) {
+          ptx::mbar_expect_tx(&q_full[qb], Cfg::TILE);
+          ptx::tma_load_2d(sQ + qb * Cfg::TILE, &tmQ, col0, row_base + qt * ATT_BM, &q_full[qb]);
         }
-        for (int i = 0; i < nkv && ok; ++i, ++vcnt) {
+        for (int j = 0; j < nkv && ok; ++j, kr.advance(1)) {
+          const int ks = kr.idx;
+          if (!ptx::mbar_wait(&k_empty[ks], kr.par ^ 1, p.err, 0x7100 | ks)) { ok = false; break; }
+          if (issue) {
+            ptx::mbar_expect_tx(&k_full[ks], Cfg::TILE);
+            ptx::tma_load_2d(sK + ks * Cfg::TILE, &tmK, col0, row_base + j * ATT_BN, &k_full[ks]);
+          }
+        }
+        for (int i = 0; i < nkv && ok; ++i, vr.advance(1)) {
           const int j = res_pv_block(nkv, i);
-          const int vs = vcnt % VST;
-          if (!ptx::mbar_wait(&v_empty[vs], ((vcnt / VST) & 1) ^ 1, p.err, 0x7200 | vs)) { ok = false; break; }
-          ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
-          ptx::tma_load_2d(sV + vs * Cfg::TILE, &tmV, col0, row_base + j * ATT_BN, &v_full[vs]);
+          const int vs = vr.idx;
+          if (!ptx::mbar_wait(&v_empty[vs], vr.par ^ 1, p.err, 0x7200 | vs)) { ok = false; break; }
+          if (issue) {
+            ptx::mbar_expect_tx(&v_full[vs], Cfg::TILE);
+            ptx::tma_load_2d(sV + vs * Cfg::TILE, &tmV, col0, row_base + j * ATT_BN, &v_full[vs]);
+          }
         }
         ++wcnt;
       }
@@ -209,11 +219,17 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     __syncwarp();
   } else if (warp == ATT_MMA_WARP) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    {
+      const bool issue = ptx::elect_one();
       constexpr uint64_t kmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);
       constexpr uint64_t pmaj = ptx::smem_desc_base(16, 1024, ptx::SWZ_128B);
       constexpr uint64_t vmaj = ptx::smem_desc_base(16, Cfg::SBO, Cfg::SWZ);
-      uint32_t kcnt = 0, vcnt = 0, pcnt = 0, wcnt = 0;
+      const uint64_t qd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sQ)), kd0 = ptx::smem_desc(kmaj, ptx::smem_u32(sK));
+      const uint64_t pd0 = ptx::smem_desc(pmaj, ptx::smem_u32(sP)), vd0 = ptx::smem_desc(vmaj, ptx::smem_u32(sV));
+      RingPos<KST> kr;
+      RingPos<VST> vr;
+      RingPos<RES_NP> pr;
+      uint32_t wcnt = 0;
       uint32_t used = 0;                                  // bit j: parity of how often score block j has been filled
       bool ok = true;
 
@@ -221,22 +237,21 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       // which the callers keep equal to the producer's order j = 0, 1, ...
       auto issue_qk = [&](uint32_t w, int j) {
         const int qb = w & 1;
-        const int ks = kcnt % KST;
-        if (!ptx::mbar_wait(&k_full[ks], (kcnt / KST) & 1, p.err, 0x8300 | ks)) { ok = false; return; }
+        const int ks = kr.idx;
+        if (!ptx::mbar_wait(&k_full[ks], kr.par, p.err, 0x8300 | ks)) { ok = false; return; }
         if (!ptx::mbar_wait(&s_free[j], ((used >> j) & 1) ^ 1, p.err, 0x8400 | j)) { ok = false; return; }
         ptx::tc_fence_after();
-        const uint32_t q_addr = ptx::smem_u32(sQ + qb * Cfg::TILE);
-        const uint32_t k_addr = ptx::smem_u32(sK + ks * Cfg::TILE);
+        if (issue) {
+          const uint64_t qd = qd0 + (uint32_t)((qb * Cfg::TILE) >> 4), kd = kd0 + (uint32_t)((ks * Cfg::TILE) >> 4);
 #pragma unroll
-        for (int k = 0; k < DH / 32; ++k) {
-          if constexpr (F8) ptx::umma_f8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                                         ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
-          else ptx::umma_i8(tmem_base + j * ATT_BN, ptx::smem_desc(kmaj, q_addr + k * 32),
-                            ptx::smem_desc(kmaj, k_addr + k * 32), p.idesc_qk, k != 0);
+          for (int k = 0; k < DH / 32; ++k) {
+            if constexpr (F8) ptx::umma_f8(tmem_base + j * ATT_BN, qd + 2 * k, kd + 2 * k, p.idesc_qk, k != 0);
+            else ptx::umma_i8(tmem_base + j * ATT_BN, qd + 2 * k, kd + 2 * k, p.idesc_qk, k != 0);
+          }
+          ptx::umma_commit(&k_empty[ks]);
+          ptx::umma_commit(&s_full[j]);
         }
-        ptx::umma_commit(&k_empty[ks]);
-        ptx::umma_commit(&s_full[j]);
-        ++kcnt; used ^= 1u << j;
+        kr.advance(1); used ^= 1u << j;
       };
       // next tile of this CTA with at least one key block
       auto next_tile = [&](int t, int& nkv) {
@@ -266,29 +281,28 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           issue_qk(wcnt, j);
         }
         if (!ok) break;
-        ptx::umma_commit(&q_empty[qb]);
+        if (issue) ptx::umma_commit(&q_empty[qb]);
         issued = 0; q_ready = false;
         for (int i = 0; i < nkv && ok; ++i) {
-          const int vs = vcnt % VST, pb = pcnt % RES_NP;
-          if (!ptx::mbar_wait(&v_full[vs], (vcnt / VST) & 1, p.err, 0x8100 | vs)) { ok = false; break; }
-          if (!ptx::mbar_wait(&p_full[pb], (pcnt / RES_NP) & 1, p.err, 0x8200 | pb)) { ok = false; break; }
+          const int vs = vr.idx, pb = pr.idx;
+          if (!ptx::mbar_wait(&v_full[vs], vr.par, p.err, 0x8100 | vs)) { ok = false; break; }
+          if (!ptx::mbar_wait(&p_full[pb], pr.par, p.err, 0x8200 | pb)) { ok = false; break; }
           if (!o_free) {
             if (!ptx::mbar_wait(o_empty, (wcnt & 1) ^ 1, p.err, 0x8600)) { ok = false; break; }
             o_free = true;
           }
           ptx::tc_fence_after();
-          const uint32_t p_addr = ptx::smem_u32(sP + pb * Cfg::P_TILE);
-          const uint32_t v_addr = ptx::smem_u32(sV + vs * Cfg::TILE);
+          if (issue) {
+            const uint64_t pd = pd0 + (uint32_t)((pb * Cfg::P_TILE) >> 4), vd = vd0 + (uint32_t)((vs * Cfg::TILE) >> 4);
 #pragma unroll
-          for (int k = 0; k < ATT_BN / 32; ++k) {
-            if constexpr (F8) ptx::umma_f8(tmem_base + RES_O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                                           ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
-            else ptx::umma_i8(tmem_base + RES_O_COL, ptx::smem_desc(pmaj, p_addr + k * 32),
-                              ptx::smem_desc(vmaj, v_addr + k * 32 * DH), p.idesc_pv, (i | k) != 0);
+            for (int k = 0; k < ATT_BN / 32; ++k) {
+              if constexpr (F8) ptx::umma_f8(tmem_base + RES_O_COL, pd + 2 * k, vd + (uint32_t)((k * 32 * DH) >> 4), p.idesc_pv, (i | k) != 0);
+              else ptx::umma_i8(tmem_base + RES_O_COL, pd + 2 * k, vd + (uint32_t)((k * 32 * DH) >> 4), p.idesc_pv, (i | k) != 0);
+            }
+            ptx::umma_commit(&v_empty[vs]);
+            ptx::umma_commit(&p_empty[pb]);
           }
-          ptx::umma_commit(&v_empty[vs]);
-          ptx::umma_commit(&p_empty[pb]);
-          ++vcnt; ++pcnt;
+          vr.advance(1); pr.advance(1);
           // the block just converted to P is free: start the next tile's scores there (block 3 holds the output)
           const int j = res_pv_block(nkv, i);
           if (j == issued && j < 3 && j < nkv_n) {
@@ -301,7 +315,7 @@ attn_int8_resident_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             ++issued;
           }
         }
-        if (ok) ptx::umma_commit(o_full);
+        if (ok && issue) ptx::umma_commit(o_full);
         ++wcnt;
         t = tn; nkv = nkv_n;
       }
