@@ -282,62 +282,89 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # CPU oracle arm (also the cpu_baseline leg)
 # ------------------------------------------------------------------------------------------------
-def oracle_run(name, budget_s=12.0, repeats=1):
-    """Times the oracle, as it stands, on whole sequences of the workload (all of its layers).
-    Returns (tokens/s, cores, sample, seconds)."""
-    import numpy as np
-    from oracle import layer as OL, ops as O
-    from paper_2310_17723_b200 import workloads as W
-    shape, cid, cfgs, desc = workload_spec(name)
-    x_cal = W.activations(shape, cid, n_seq=1, tensor=7).astype(np.float64)
-    layers = []
-    cur = None
-    for li, cfg in enumerate(cfgs):                       # offline preparation of every layer (not timed)
-        spec = OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, act=cfg.act,
-                            eps=cfg.eps, mask=cfg.mask, fp_dtype=cfg.fp_dtype, mode=dict(cfg.mode), gran_in=cfg.gran_in,
-                            gran_mid=cfg.gran_mid, gran_attn=cfg.gran_attn, gran_out=cfg.gran_out)
-        p = W.layer_params(shape, cid * 100 + li)
-        if li == 0:
-            ln0 = (p["ln0_g"], p["ln0_b"])
-            cur = O.layernorm(x_cal, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else x_cal
-        C = OL.calibrate(spec, p, cur, 1)
-        if len(cfgs) > 1:
-            cur = OL.layer_fp64(spec, p, cur, B=1)["x_out"]
-        layers.append((spec, OL.prepare_layer(spec, p, C)))
+class OracleArm:
+    """The oracle, as it stands, on whole sequences of a workload (entry LN^quant and all of its layers).  The offline
+    preparation of the layers (calibration, folding, weight quantization) happens once, in the constructor, and is not
+    timed."""
 
-    def run(n_seq):
-        x = W.activations(shape, cid, n_seq=n_seq)
-        spec0, L0 = layers[0]
-        t0 = time.perf_counter()                              # a step = the entry LN^quant and every layer, as on the GPU
+    def __init__(self, name):
+        import numpy as np
+        from oracle import layer as OL, ops as O
+        from paper_2310_17723_b200 import workloads as W
+        self.OL, self.O, self.W = OL, O, W
+        self.shape, self.cid, cfgs, self.desc = workload_spec(name)
+        shape, cid = self.shape, self.cid
+        x_cal = W.activations(shape, cid, n_seq=1, tensor=7).astype(np.float64)
+        self.layers = []
+        cur = None
+        for li, cfg in enumerate(cfgs):
+            spec = OL.LayerSpec(B=shape.B, S=shape.S, H=shape.H, nh=shape.nh, F=shape.F, arch=shape.arch, act=cfg.act,
+                                eps=cfg.eps, mask=cfg.mask, fp_dtype=cfg.fp_dtype, mode=dict(cfg.mode), gran_in=cfg.gran_in,
+                                gran_mid=cfg.gran_mid, gran_attn=cfg.gran_attn, gran_out=cfg.gran_out)
+            p = W.layer_params(shape, cid * 100 + li)
+            if li == 0:
+                self.ln0 = (p["ln0_g"], p["ln0_b"])
+                cur = O.layernorm(x_cal, p["ln0_g"], p["ln0_b"], spec.eps) if spec.arch == "post_ln" else x_cal
+            C = OL.calibrate(spec, p, cur, 1)
+            if len(cfgs) > 1:
+                cur = OL.layer_fp64(spec, p, cur, B=1)["x_out"]
+            self.layers.append((spec, OL.prepare_layer(spec, p, C)))
+        self.t1 = None                                        # seconds for one sequence (measured by the first run)
+
+    def run(self, n_seq):
+        """Seconds for one pass of n_seq sequences: a step = the entry LN^quant and every layer, as on the GPU."""
+        OL, O, W = self.OL, self.O, self.W
+        x = W.activations(self.shape, self.cid, n_seq=n_seq)
+        spec0, L0 = self.layers[0]
+        t0 = time.perf_counter()
         if spec0.arch == "post_ln":
-            cur_t = OL.entry_ln(O.fp_tensor(x, spec0.fp_dtype), ln0[0], ln0[1], spec0.eps, L0["ln_in_out"])
+            cur_t = OL.entry_ln(O.fp_tensor(x, spec0.fp_dtype), self.ln0[0], self.ln0[1], spec0.eps, L0["ln_in_out"])
         else:
             cur_t = O.fp_tensor(x, spec0.fp_dtype)
-        for spec, Lp in layers:
+        for spec, Lp in self.layers:
             cur_t = OL.layer_forward(Lp, cur_t, B=n_seq)["x_out"]
         return time.perf_counter() - t0
 
-    t1 = run(1)
-    n = int(max(1, min(shape.B, budget_s / max(t1, 1e-3))))
-    best = min(run(n) for _ in range(repeats)) if n > 1 else t1
-    cores = os.cpu_count() or 1
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
-    except Exception:
-        pass
-    sample = "%d of %d sequences (%d tokens) of %s through %d layer(s), one pass" % (n, shape.B, n * shape.S, shape.name, len(layers))
-    return n * shape.S / best, cores, sample, best
+    def step(self, budget_s):
+        """One bounded sample: as many whole sequences as fit `budget_s` (at least one).
+        Returns (tokens/s, cores, sample, seconds)."""
+        if self.t1 is None:
+            self.t1 = self.run(1)
+            n, best = 1, self.t1
+            if budget_s >= 2.0 * self.t1:
+                n = int(max(1, min(self.shape.B, budget_s / max(self.t1, 1e-3))))
+                best = self.run(n) if n > 1 else self.t1
+        else:
+            n = int(max(1, min(self.shape.B, budget_s / max(self.t1, 1e-3))))
+            best = self.run(n)
+        cores = os.cpu_count() or 1
+        try:
+            from threadpoolctl import threadpool_info
+            cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            pass
+        sample = "%d of %d sequences (%d tokens) of %s through %d layer(s), one pass" % (n, self.shape.B, n * self.shape.S,
+                                                                                        self.shape.name, len(self.layers))
+        return n * self.shape.S / best, cores, sample, best
+
+
+def oracle_run(name, budget_s=12.0):
+    """One bounded sample of the oracle on a workload: (tokens/s, cores, sample, seconds)."""
+    return OracleArm(name).step(budget_s)
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    shape, cid, cfgs, desc = workload_spec(args.workload)
+    arm = OracleArm(args.workload)                            # offline preparation, once
+    desc = arm.desc
     vals, ts = [], []
+    # every step is a bounded sample; the whole run (warm-up included) aims at about two minutes of oracle time, with one
+    # whole sequence per step as the floor
+    per_step = max(2.0, 120.0 / max(1, args.warmup + args.steps))
     for i in range(args.warmup + args.steps):
-        v, cores, sample, t = oracle_run(args.workload, budget_s=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
+        v, cores, sample, t = arm.step(per_step)
         if i >= args.warmup:
             vals.append(v)
             ts.append(t)
