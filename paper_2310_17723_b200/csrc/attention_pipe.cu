@@ -173,47 +173,6 @@ __device__ __forceinline__ void pipe_exp_piece(uint32_t (&r)[32], int nvalid, fl
   m = mn;
 }
 
-// Two fully valid 32-column pieces at once: both maxima are found first, so the 64 exponentials are independent of one
-// another and of the bookkeeping.  Piece A's e values are relative to mA = max(m, max A), piece B's to mB = max(mA, max B).
-template <bool F8>
-__device__ __forceinline__ void pipe_exp_two_full(uint32_t (&ra)[32], uint32_t (&rb)[32], float c2, float& m, float& l, float& mA_out) {
-  float pa, pb;
-  if constexpr (F8) {
-    float a0 = __uint_as_float(ra[0]), a1 = __uint_as_float(ra[1]), b0 = __uint_as_float(rb[0]), b1 = __uint_as_float(rb[1]);
-#pragma unroll
-    for (int e = 2; e < 32; e += 2) {
-      a0 = fmaxf(a0, __uint_as_float(ra[e])); a1 = fmaxf(a1, __uint_as_float(ra[e + 1]));
-      b0 = fmaxf(b0, __uint_as_float(rb[e])); b1 = fmaxf(b1, __uint_as_float(rb[e + 1]));
-    }
-    pa = fmaxf(a0, a1) * c2; pb = fmaxf(b0, b1) * c2;
-  } else {
-    int a0 = max((int)ra[0], (int)ra[1]), a1 = max((int)ra[2], (int)ra[3]);
-    int b0 = max((int)rb[0], (int)rb[1]), b1 = max((int)rb[2], (int)rb[3]);
-#pragma unroll
-    for (int e = 4; e < 32; e += 4) {
-      a0 = max(a0, max((int)ra[e], (int)ra[e + 1])); a1 = max(a1, max((int)ra[e + 2], (int)ra[e + 3]));
-      b0 = max(b0, max((int)rb[e], (int)rb[e + 1])); b1 = max(b1, max((int)rb[e + 2], (int)rb[e + 3]));
-    }
-    pa = (float)max(a0, a1) * c2; pb = (float)max(b0, b1) * c2;
-  }
-  const float mA = fmaxf(m, pa), mB = fmaxf(mA, pb);
-  float sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
-#pragma unroll
-  for (int e = 0; e < 32; e += 2) {
-    const float a0 = ex2f(fmaf(F8 ? __uint_as_float(ra[e]) : (float)(int)ra[e], c2, -mA));
-    const float a1 = ex2f(fmaf(F8 ? __uint_as_float(ra[e + 1]) : (float)(int)ra[e + 1], c2, -mA));
-    const float b0 = ex2f(fmaf(F8 ? __uint_as_float(rb[e]) : (float)(int)rb[e], c2, -mB));
-    const float b1 = ex2f(fmaf(F8 ? __uint_as_float(rb[e + 1]) : (float)(int)rb[e + 1], c2, -mB));
-    sA0 += a0; sA1 += a1; sB0 += b0; sB1 += b1;
-    ra[e] = __float_as_uint(a0); ra[e + 1] = __float_as_uint(a1);
-    rb[e] = __float_as_uint(b0); rb[e + 1] = __float_as_uint(b1);
-  }
-  const float sumA = sA0 + sA1, sumB = sB0 + sB1;
-  l = (l * ex2f(m - mA) + sumA) * ex2f(mA - mB) + sumB;       // m = -inf before the first piece: 2^(-inf) = 0
-  m = mB;
-  mA_out = mA;
-}
-
 // 32 values e (FP32 bits in r) times the factor f -> 32 P codes packed into w[8].
 template <bool F8>
 __device__ __forceinline__ void pipe_pack32(const uint32_t (&r)[32], float f, uint32_t (&w)[8]) {
@@ -447,8 +406,6 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       // the statistics (and stash) slots of this parity are free: the pack warps are through with the tile two back.
       // (With spare ring slots the exponential warps could otherwise run several tiles ahead of the pack warps.)
       ok = pipe_group_wait<128>(leader, bar_id, &t_empty[par], ((wcnt >> 1) & 1) ^ 1, p.err, 0x9400 | par, ok);
-      // the last key that every row of the tile may attend to
-      const int tile_kmax = p.mask == HERO_MASK_CAUSAL ? min(g.klen - 1, g.qt * ATT_BM) : g.klen - 1;
       float* pm_row = pm_s + (par * PIPE_MAXB) * 2 * ATT_BM + r_loc;
       const long long probe_row = ((long long)(g.b * p.nh + g.h) * p.S + q) * p.S;
       float m = -INFINITY, l = 0.f;
@@ -472,32 +429,9 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int key0 = j * PB;
         const bool to_stash = stash && k == 0;
         float* stash_dst = stash_s + (par * PB) * ATT_BM + r_loc;
-        if ((j + 1) * PB - 1 <= tile_kmax) {
-          // every key of the block is valid for every row of the tile (the common case): 64 independent exponentials
-          uint32_t ra[32], rb[32];
-          ptx::tmem_ld32(t_lane + blk * PB, ra);
-          ptx::tmem_ld32(t_lane + blk * PB + 32, rb);
-          ptx::tmem_ld_wait();
-          probe_scores(ra, key0); probe_scores(rb, key0 + 32);
-          float mA;
-          pipe_exp_two_full<F8>(ra, rb, c2, m, l, mA);
-          if (Cfg::STASH && to_stash) {
-            // the block's e values wait in shared memory ([column][row]: a warp's 32 rows are consecutive words) and
-            // its ring slot goes straight back to the Q K^T issuer (eight arrivals, as from the pack warps: two per
-            // warp of this group)
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) { ptx::mbar_arrive(&s_free[blk]); ptx::mbar_arrive(&s_free[blk]); }
-#pragma unroll
-            for (int e = 0; e < 32; ++e) { stash_dst[e * ATT_BM] = __uint_as_float(ra[e]); stash_dst[(32 + e) * ATT_BM] = __uint_as_float(rb[e]); }
-          } else {
-            ptx::tmem_st32(t_lane + blk * PB, ra);
-            ptx::tmem_st32(t_lane + blk * PB + 32, rb);
-          }
-          pm_row[(j * 2 + 0) * ATT_BM] = mA;                 // the maximum each half's e values are relative to
-          pm_row[(j * 2 + 1) * ATT_BM] = m;
-        } else {
-          // a block that the mask cuts: one 32-column piece after the other
+        {
+          // one 32-column piece after the other, in a rolled loop: the kernel's five roles share the instruction caches, and
+          // a block's 64 exponentials unrolled as one straight line (twice the code) ran slower than this, not faster
 #pragma unroll 1
           for (int hh = 0; hh < 2; ++hh) {
             uint32_t r[32];
