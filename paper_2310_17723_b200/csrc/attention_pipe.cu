@@ -591,12 +591,13 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       // ---- output stage (Eq. 17): X_attn = acc * s_p s_v (/ S_attn[j] -> Round -> INT8); OW columns per warp
       ok = pipe_group_wait<256>(warp == PIPE_EXP_WARPS, 2, o_full, wcnt & 1, p.err, 0x9300, ok);
       ptx::tc_fence_after();
-#pragma unroll
-      for (int c0 = 0; c0 < OW; c0 += 32) {
-        uint32_t r[32];
-        ptx::tmem_ld32(t_lane + Cfg::O_COL + half * OW + c0, r);
+      // 16 columns at a time in a rolled loop (this stage runs once per tile: its code should be small, not fast)
+#pragma unroll 1
+      for (int c0 = 0; c0 < OW; c0 += 16) {
+        uint32_t r[16];
+        ptx::tmem_ld16(t_lane + Cfg::O_COL + half * OW + c0, r);
         ptx::tmem_ld_wait();
-        if (c0 + 32 >= OW) {                                 // the accumulator is in registers: the next tile may use its columns
+        if (c0 + 16 >= OW) {                                 // the accumulator is in registers: the next tile may use its columns
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(o_empty);
@@ -607,48 +608,42 @@ attn_int8_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             if (p.dbg_acc) {
               int* dst = p.dbg_acc + grow * ((long long)p.nh * p.dh) + gcol;
 #pragma unroll
-              for (int c = 0; c < 32; ++c) dst[c] = (int)r[c];
+              for (int c = 0; c < 16; ++c) dst[c] = (int)r[c];
             }
           }
           const float4* o4 = reinterpret_cast<const float4*>(osc + c0);
           auto acc = [&](int c) -> float { if constexpr (F8) return __uint_as_float(r[c]); else return (float)(int)r[c]; };
           if (p.out_dt == HERO_F8) {
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
+            uint32_t w[4];
 #pragma unroll
-            for (int gq = 0; gq < 2; ++gq) {
-              uint32_t w[4];
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float4 sc = o4[4 * gq + k];
-                const int c = 16 * gq + 4 * k;
-                w[k] = ptx::f32x4_to_e4m3x4(acc(c) * rowf * sc.x, acc(c + 1) * rowf * sc.y, acc(c + 2) * rowf * sc.z, acc(c + 3) * rowf * sc.w);
-              }
-              st_g16(dst + 16 * gq, w[0], w[1], w[2], w[3]);
+            for (int k = 0; k < 4; ++k) {
+              const float4 sc = o4[k];
+              const int c = 4 * k;
+              w[k] = ptx::f32x4_to_e4m3x4(acc(c) * rowf * sc.x, acc(c + 1) * rowf * sc.y, acc(c + 2) * rowf * sc.z, acc(c + 3) * rowf * sc.w);
             }
+            st_g16(dst, w[0], w[1], w[2], w[3]);
           } else if (p.out_dt == HERO_I8) {
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + grow * p.out_ld + gcol;
+            uint32_t w[4];
 #pragma unroll
-            for (int gq = 0; gq < 2; ++gq) {
-              uint32_t w[4];
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float4 sc = o4[4 * gq + k];
-                const int c = 16 * gq + 4 * k;
-                // Round(acc f) in the FMA's single rounding (magic + x), clipped to [-127, 127] on the shifted value (the
-                // order of floats is that of the sums, whatever their size); low byte = two's-complement code
-                const float lo = ATT_MAGIC - 127.0f, hi = ATT_MAGIC + 127.0f;
-                const float a = fminf(fmaxf(fmaf(acc(c), ROWMAX ? rowf * sc.x : sc.x, ATT_MAGIC), lo), hi);
-                const float b = fminf(fmaxf(fmaf(acc(c + 1), ROWMAX ? rowf * sc.y : sc.y, ATT_MAGIC), lo), hi);
-                const float cc = fminf(fmaxf(fmaf(acc(c + 2), ROWMAX ? rowf * sc.z : sc.z, ATT_MAGIC), lo), hi);
-                const float d = fminf(fmaxf(fmaf(acc(c + 3), ROWMAX ? rowf * sc.w : sc.w, ATT_MAGIC), lo), hi);
-                w[k] = low_bytes4_u(a, b, cc, d);
-              }
-              st_g16(dst + 16 * gq, w[0], w[1], w[2], w[3]);
+            for (int k = 0; k < 4; ++k) {
+              const float4 sc = o4[k];
+              const int c = 4 * k;
+              // Round(acc f) in the FMA's single rounding (magic + x), clipped to [-127, 127] on the shifted value (the
+              // order of floats is that of the sums, whatever their size); low byte = two's-complement code
+              const float lo = ATT_MAGIC - 127.0f, hi = ATT_MAGIC + 127.0f;
+              const float a = fminf(fmaxf(fmaf(acc(c), ROWMAX ? rowf * sc.x : sc.x, ATT_MAGIC), lo), hi);
+              const float b = fminf(fmaxf(fmaf(acc(c + 1), ROWMAX ? rowf * sc.y : sc.y, ATT_MAGIC), lo), hi);
+              const float cc = fminf(fmaxf(fmaf(acc(c + 2), ROWMAX ? rowf * sc.z : sc.z, ATT_MAGIC), lo), hi);
+              const float d = fminf(fmaxf(fmaf(acc(c + 3), ROWMAX ? rowf * sc.w : sc.w, ATT_MAGIC), lo), hi);
+              w[k] = low_bytes4_u(a, b, cc, d);
             }
+            st_g16(dst, w[0], w[1], w[2], w[3]);
           } else {
             uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + grow * p.out_ld + gcol;
 #pragma unroll
-            for (int gq = 0; gq < 4; ++gq) {
+            for (int gq = 0; gq < 2; ++gq) {
               float v[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) v[e] = acc(8 * gq + e) * rowf * p.pv_scale;
