@@ -102,6 +102,8 @@ struct OutStage {
   int n0;                     // first column of the tile being processed
   bool fresh;                 // nothing of the current tile has been staged yet
   int nthreads;               // threads on the two named barriers: epilogue warps + store warp
+  bool clip_low;              // GELU: some output factor of this warp's columns is negative or above 700, so that
+                              // GELU(v) * factor >= -0.17 * factor may fall below -127 (otherwise only the upper clip can bite)
 };
 constexpr int BAR_STAGED = 1, BAR_DRAINED = 2;   // named barriers: tile staged (epilogue -> store warp), tile read (back)
 constexpr int OUT_HALF_BYTES = GEMM_BM * 128;
@@ -175,11 +177,12 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
         // Round (half to even) happened in the float adder: 1.5 * 2^23 + k keeps k in its low byte.  The clip to
         // [-127, 127] is applied only if some value of the chunk needs it.
         hi = ptx::max3(ptx::max3(hi, y0.x, y0.y), y1.x, y1.y);
-        lo = ptx::min3(ptx::min3(lo, y0.x, y0.y), y1.x, y1.y);
+        if constexpr (ACT == HERO_ACT_NONE) lo = ptx::min3(ptx::min3(lo, y0.x, y0.y), y1.x, y1.y);
       }
     }
     if constexpr (OUTK == OUT_I8) {
-      if (hi > ROUND_MAGIC + 127.0f || lo < ROUND_MAGIC - 127.0f) {
+      // (after a GELU the lower bound is known from the output factors alone: see OutStage::clip_low)
+      if (hi > ROUND_MAGIC + 127.0f || (ACT == HERO_ACT_NONE ? lo < ROUND_MAGIC - 127.0f : stage.clip_low)) {
 #pragma unroll
         for (int j = 0; j < NC; ++j) v[j] = fminf(fmaxf(v[j], ROUND_MAGIC - 127.0f), ROUND_MAGIC + 127.0f);
       }
@@ -342,6 +345,12 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
         } else {
           e[i * 32 + lane] = ncs[i]; e[CH + i * 32 + lane] = nbias[i]; e[2 * CH + i * 32 + lane] = npost[i];
         }
+      }
+      if constexpr (ACT != HERO_ACT_NONE) {
+        bool odd = false;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) odd = odd || !(npost[i] >= 0.0f && npost[i] <= 700.0f);
+        stage.clip_low = __any_sync(0xffffffffu, odd);
       }
       __syncwarp();
     }
@@ -510,7 +519,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
     ptx::pdl_wait();                                     // before this warp's first global access
     epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0,
-                                                           OutStage{nullptr, nullptr, 0, 0, 0, false, 0}, warp);
+                                                           OutStage{nullptr, nullptr, 0, 0, 0, false, 0, true}, warp);
   }
 
   ptx::tc_fence_before();
@@ -769,7 +778,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::pdl_wait();                                     // before this warp's first global access
     // ------------------------------------------------------------------ epilogue (warps 0 .. EW-1 of each CTA)
     const int row = (warp & 3) * 32 + lane;                // this lane's row of the CTA's 128
-    OutStage stage{p.tma_out ? out_stage : nullptr, &tmO, (uint32_t)row * 128u, (uint32_t)row & 7u, 0, false, (EW + 1) * 32};
+    OutStage stage{p.tma_out ? out_stage : nullptr, &tmO, (uint32_t)row * 128u, (uint32_t)row & 7u, 0, false, (EW + 1) * 32, true};
     epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM, stage,
                                                       warp);
   }

@@ -92,6 +92,25 @@ def test_fc1_gelu_quant_epilogue(h, act, M):
     assert_int8_close(got, want.data, what="GELU^quant")
 
 
+@pytest.mark.parametrize("M,K,N", [(1100, 768, 3072), (200, 512, 256)])
+def test_fc1_gelu_quant_saturates_both_ways(h, M, K, N):
+    # output factors far too large for the data (a mis-calibrated 1 / S_a): GELU(v) / S_a leaves [-127, 127] on both
+    # sides, the lower one only because the factor exceeds 127 / 0.17; the codes must saturate exactly as the oracle's
+    g = W.rng(2, 777 + M)
+    A = g.integers(-127, 128, (M, K), dtype=np.int8)
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    rs = (g.uniform(0.5, 1.5, M) * 0.02).astype(np.float32)
+    cs = (g.uniform(0.5, 1.5, N) * 1.5e-4 / np.sqrt(K / 768)).astype(np.float32)
+    bias = (g.standard_normal(N) * 0.1).astype(np.float32)
+    S_a = np.full(N, 1.0 / 40.0)
+    S_a[::3] = 1.0 / 2000.0                                 # every third column: -0.17 * 2000 < -127
+    x = O.QT("i8", A, row_scale=rs.astype(np.float64))
+    want = O.gemm_quant(x, Wt.T.copy(), cs, bias, "gelu_erf", O.OutSpec("fwq", scale=S_a)).data
+    assert (want == -127).any() and (want == 127).any()
+    got = _linear(h, A, Wt, torch.int8, rs=rs, cs=cs, bias=bias, act="gelu_erf", post=(1.0 / S_a).astype(np.float32)).cpu().numpy()
+    assert_int8_close(got, want, what="GELU^quant, saturating")
+
+
 @pytest.mark.parametrize("fp", ["f16", "bf16"])
 def test_int8_gemm_fp_output(h, fp):
     # an INT8 module whose consumer is in FP mode: dequantize + bias only, stored in FP16 / BF16
