@@ -102,10 +102,11 @@ struct OutStage {
   int n0;                     // first column of the tile being processed
   bool fresh;                 // nothing of the current tile has been staged yet
   int nthreads;               // threads on the two named barriers: epilogue warps + store warp
+  int bar_staged, bar_drained;   // named barriers of this warp's group: tile staged (epilogue -> store warp), tile read (back)
   bool clip_low;              // GELU: some output factor of this warp's columns is negative or above 700, so that
                               // GELU(v) * factor >= -0.17 * factor may fall below -127 (otherwise only the upper clip can bite)
 };
-constexpr int BAR_STAGED = 1, BAR_DRAINED = 2;   // named barriers: tile staged (epilogue -> store warp), tile read (back)
+constexpr int BAR_STAGED = 1, BAR_DRAINED = 3;   // first named barrier of each kind (+ the epilogue group's index)
 constexpr int OUT_HALF_BYTES = GEMM_BM * 128;
 __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -197,7 +198,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
       if (stage.buf) {
         // this lane's NC bytes of its row of the staging tile (rows past the end are clipped by the store)
         if (stage.fresh) {                                   // the unit has read the previous tile out of the staging area
-          asm volatile("bar.sync %0, %1;" ::"n"(BAR_DRAINED), "r"(stage.nthreads) : "memory");
+          asm volatile("bar.sync %0, %1;" ::"r"(stage.bar_drained), "r"(stage.nthreads) : "memory");
           stage.fresh = false;
         }
         const int jc = col0 - stage.n0;                      // column inside the tile
@@ -258,15 +259,14 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const uint32
 // One thread's share of a tile's epilogue: BN / (EW / 4) columns of one output row (EW epilogue warps, EW / 4 per
 // tensor-memory lane quarter).  With 8 warps the columns come 32 at a time, the next 32 already loading while the
 // current ones are processed; with 16 warps (96 registers per thread) 16 at a time.
-template <int BN, bool INT8, int ACT, int OUTK, int EW>
+template <int BN, bool INT8, int ACT, int OUTK, int CH, int CW>
 __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const float* e_cs, const float* e_bias,
                                                  const float* e_post, uint32_t taddr, int m, bool row_ok, float rs,
                                                  int n0, int cpart, OutStage& stage) {
-  constexpr int CH = BN / (EW / 4);
   // 32-byte stores need a 32-byte aligned row segment: base pointer and row pitch multiples of 32 bytes
   const int es = (OUTK == OUT_I8 || OUTK == OUT_F8) ? 1 : (OUTK == OUT_FP ? 2 : 4);
   const bool wide = ((reinterpret_cast<uintptr_t>(p.out) & 31) == 0) && ((p.out_ld * es) % 32 == 0);
-  if constexpr (EW == 8) {
+  if constexpr (CW == 32) {
     constexpr int NCH = CH / 32;
     uint32_t ra[32], rb[32];
     ptx::tmem_ld32(taddr, ra);
@@ -298,15 +298,24 @@ __device__ __forceinline__ void epilogue_columns(const GemmParams& p, const floa
 // The epilogue warps' walk over this CTA's tiles.  The per-column vectors (and the row scale) of the NEXT tile are
 // fetched from global memory into registers while the current tile is being processed, so a tile never starts by
 // waiting on them.  ROWS = output rows per tile (128, or 256 for a CTA pair of which this CTA owns rows row_off..+127).
-template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR, int EW>
+// GROUPS = 2 (16 epilogue warps with a staged output): the warps form two groups of eight that take alternate tiles, each
+// group always the same accumulator buffer and its own staging tile.  The two groups are then half a tile apart in time:
+// while one group's warps wait (for tensor memory, for their barrier) the other's keep the issue slots busy, which 16
+// warps moving through the same chunk in step do not.
+template <int BN, bool INT8, int ACT, int OUTK, int ROWS, bool PAIR, int EW, int GROUPS = 1>
 __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, uint64_t* acc_full, uint64_t* acc_empty,
                                               uint32_t tmem_base, int first_tile, int tile_stride, int row_off,
                                               OutStage stage, int warp) {   // warp: index among the epilogue warps
   const int lane = threadIdx.x & 31;
-  const int quarter = warp & 3, cpart = warp >> 2;
-  constexpr int CH = BN / (EW / 4);          // columns per thread and tile
+  constexpr int EWG = EW / GROUPS;           // warps per group
+  constexpr int CH = BN / (EWG / 4);         // columns per thread and tile
+  constexpr int CW = EW == 8 ? 32 : 16;      // columns per chunk (registers: 8 warps afford 32, 16 warps 16)
+  const int wg = warp / EWG, wl = warp % EWG;
+  const int quarter = warp & 3, cpart = wl >> 2;
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;
   bool ok = true;
+  first_tile += wg * tile_stride;            // this group's tiles: every GROUPS-th of the CTA's
+  tile_stride *= GROUPS;
 
   // Every warp stages the per-column vectors of its own CH columns in a shared-memory area of its own (3 x CH floats:
   // written at the start of a tile, after the warp's last read of the previous tile's), so the epilogue warps never
@@ -360,8 +369,8 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
   int it = 0;
   for (int t = first_tile; t < num_tiles; t += tile_stride, ++it) {
     const int mt = nmt, nt = nnt;
-    const int as = it & 1;
-    const uint32_t aphase = (it >> 1) & 1;
+    const int as = GROUPS == 2 ? wg : (it & 1);
+    const uint32_t aphase = GROUPS == 2 ? (it & 1) : ((it >> 1) & 1);
     const int n0 = nt * BN;
     const float rs = nrs;
     publish(it);
@@ -377,7 +386,7 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     stage.fresh = it > 0;                                  // (the first tile finds the staging area unused)
     {
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN + cpart * CH;
-      epilogue_columns<BN, INT8, ACT, OUTK, EW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart, stage);
+      epilogue_columns<BN, INT8, ACT, OUTK, CH, CW>(p, e_cs, e_cs + CH, e_cs + 2 * CH, taddr, m, row_ok, rs, n0, cpart, stage);
     }
     // hand the accumulator buffer back to the UMMA issuer
     ptx::tc_fence_before();
@@ -389,7 +398,7 @@ __device__ __forceinline__ void epilogue_loop(const GemmParams& p, float* epi, u
     if (stage.buf) {
       // this warp's part of the staged tile is complete (writes made visible to the TMA unit)
       ptx::fence_proxy_async_smem();
-      asm volatile("bar.sync %0, %1;" ::"n"(BAR_STAGED), "r"(stage.nthreads) : "memory");
+      asm volatile("bar.sync %0, %1;" ::"r"(stage.bar_staged), "r"(stage.nthreads) : "memory");
     }
   }
 }
@@ -519,7 +528,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // warp w reads TMEM lanes 32 * (w & 3) .. +31 (one output row per thread) and the column half (w >> 2)
     ptx::pdl_wait();                                     // before this warp's first global access
     epilogue_loop<BN, INT8, ACT, OUTK, GEMM_BM, false, 8>(p, epi, acc_full, acc_empty, tmem_base, blockIdx.x, gridDim.x, 0,
-                                                           OutStage{nullptr, nullptr, 0, 0, 0, false, 0, true}, warp);
+                                                           OutStage{nullptr, nullptr, 0, 0, 0, false, 0, 0, 0, true}, warp);
   }
 
   ptx::tc_fence_before();
@@ -592,30 +601,34 @@ static hero_status dispatch_epilogue(hero_handle* h, const CUtensorMap& tmA, con
 // control flow) and the copies are split between the two CTAs' producers.
 // No multicast TMA load is used anywhere.
 // ------------------------------------------------------------------------------------------------------
-// The store warp of a launch with staged output: for every tile of this CTA, in the epilogue warps' order, wait until the
-// tile is staged, send its two halves, wait until the unit has read them, tell the epilogue warps.
+// The store warp of a launch with staged output: for every tile of this CTA, in the epilogue warps' order (tile i belongs to
+// epilogue group i % groups, which has its own staging tile and barrier pair), wait until the tile is staged, send its two
+// halves, wait until the unit has read them, tell that group.
 template <int ROWS>
 __device__ __forceinline__ void store_warp_loop(const GemmParams& p, const CUtensorMap* tm, uint8_t* buf, int first_tile,
-                                                int tile_stride, int row_off, int nthreads) {
+                                                int tile_stride, int row_off, int nthreads, int groups) {
   const int num_tiles = p.num_m_tiles * p.num_n_tiles;
   const bool issue = ptx::elect_one();
   TileWalk walk;
   walk.init(first_tile, p.num_m_tiles, p.num_n_tiles);
-  for (int t = first_tile; t < num_tiles; t += tile_stride) {
+  int it = 0;
+  for (int t = first_tile; t < num_tiles; t += tile_stride, ++it) {
     int mt, nt; walk.coords(mt, nt);
     walk.advance(tile_stride);
-    asm volatile("bar.sync %0, %1;" ::"n"(BAR_STAGED), "r"(nthreads) : "memory");
+    const int g = groups == 2 ? (it & 1) : 0;
+    uint8_t* tile = buf + g * 2 * OUT_HALF_BYTES;
+    asm volatile("bar.sync %0, %1;" ::"r"(BAR_STAGED + g), "r"(nthreads) : "memory");
     if (issue) {
       const int m0 = mt * ROWS + row_off, n0 = nt * 256;
       if (m0 < p.M) {
-        bulk_store_2d(tm, buf, n0, m0);
-        if (n0 + 128 < p.N) bulk_store_2d(tm, buf + OUT_HALF_BYTES, n0 + 128, m0);
+        bulk_store_2d(tm, tile, n0, m0);
+        if (n0 + 128 < p.N) bulk_store_2d(tm, tile + OUT_HALF_BYTES, n0 + 128, m0);
       }
       bulk_store_commit();
       bulk_store_wait_read();
     }
     __syncwarp();
-    if (t + tile_stride < num_tiles) asm volatile("bar.arrive %0, %1;" ::"n"(BAR_DRAINED), "r"(nthreads) : "memory");
+    if (t + groups * tile_stride < num_tiles) asm volatile("bar.arrive %0, %1;" ::"r"(BAR_DRAINED + g), "r"(nthreads) : "memory");
   }
   if (issue) bulk_store_wait_all();                          // the unit is through with this CTA's shared memory
 }
@@ -627,8 +640,8 @@ struct PairCfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = 6;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int EPI_FLOATS = 4 * 3 * BN;                  // per-warp cs / bias / post
-  static_assert(STAGE_BYTES == 2 * OUT_HALF_BYTES, "the last stage doubles as the output staging tile");
+  static constexpr int EPI_FLOATS = 2 * 4 * 3 * BN;              // per-warp cs / bias / post (two groups of 8 warps: 128 columns each)
+  static_assert(STAGE_BYTES == 2 * OUT_HALF_BYTES, "the last stages double as output staging tiles");
   static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_FLOATS * 4 + 256;
 };
 
@@ -638,12 +651,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmO, const GemmParams p) {
   using Cfg = PairCfg;
   constexpr int BN = Cfg::BN;
-  // with staged output the last pipeline stage is the staging tile
-  const int STAGES = p.tma_out ? Cfg::STAGES - 1 : Cfg::STAGES;
+  // with staged output the last pipeline stage is the staging tile; 16 epilogue warps work as two groups with a staging
+  // tile each (the last two stages)
+  const int groups = (p.tma_out && EW == 16) ? 2 : 1;
+  const int STAGES = p.tma_out ? Cfg::STAGES - groups : Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* tiles = smem;
-  uint8_t* out_stage = smem + (Cfg::STAGES - 1) * Cfg::STAGE_BYTES;
+  uint8_t* out_stage = smem + (Cfg::STAGES - groups) * Cfg::STAGE_BYTES;
   float* epi = reinterpret_cast<float*>(smem + Cfg::STAGES * Cfg::STAGE_BYTES);
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi + Cfg::EPI_FLOATS);
   uint64_t* full = bars;
@@ -661,7 +676,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < Cfg::STAGES; ++i) { ptx::mbar_init(&full[i], 1); ptx::mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 2 * EW); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 2 * EW / groups); }
     ptx::fence_mbar_init();
   }
   if (warp == W_MMA) {
@@ -773,14 +788,26 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncwarp();
   } else if (warp == W_ST) {
     // ------------------------------------------------------------------ store warp
-    if (p.tma_out) store_warp_loop<256>(p, &tmO, out_stage, pair_id, num_pairs, (int)rank * GEMM_BM, (EW + 1) * 32);
+    if (p.tma_out) store_warp_loop<256>(p, &tmO, out_stage, pair_id, num_pairs, (int)rank * GEMM_BM, (EW / groups + 1) * 32, groups);
   } else {
     ptx::pdl_wait();                                     // before this warp's first global access
     // ------------------------------------------------------------------ epilogue (warps 0 .. EW-1 of each CTA)
     const int row = (warp & 3) * 32 + lane;                // this lane's row of the CTA's 128
-    OutStage stage{p.tma_out ? out_stage : nullptr, &tmO, (uint32_t)row * 128u, (uint32_t)row & 7u, 0, false, (EW + 1) * 32, true};
-    epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs, (int)rank * GEMM_BM, stage,
-                                                      warp);
+    const int wg = groups == 2 ? warp / (EW / 2) : 0;      // this warp's epilogue group
+    OutStage stage{p.tma_out ? out_stage + wg * 2 * OUT_HALF_BYTES : nullptr, &tmO, (uint32_t)row * 128u, (uint32_t)row & 7u, 0, false,
+                   (EW / groups + 1) * 32, BAR_STAGED + wg, BAR_DRAINED + wg, true};
+    if constexpr (EW == 16) {
+      if (groups == 2) {
+        epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW, 2>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs,
+                                                             (int)rank * GEMM_BM, stage, warp);
+      } else {
+        epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW, 1>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs,
+                                                             (int)rank * GEMM_BM, stage, warp);
+      }
+    } else {
+      epilogue_loop<BN, INT8, ACT, OUTK, 256, true, EW, 1>(p, epi, acc_full, acc_empty, tmem_base, pair_id, num_pairs,
+                                                           (int)rank * GEMM_BM, stage, warp);
+    }
   }
 
   ptx::tc_fence_before();
