@@ -55,6 +55,19 @@ hero_status make_tmap_2d(const hero_handle* h, CUtensorMap* out, const void* bas
                          bool is_bf16, uint64_t rows, uint64_t cols, uint64_t ld_bytes, uint32_t box_cols,
                          uint32_t box_rows, int swizzle_bytes) {
   HERO_REQUIRE(h && h->encode_tiled, HERO_ERR_CUDA, "tensor-map encoder unavailable");
+  // cache look-up (see hero_tmap_slot)
+  const uint64_t key[5] = {reinterpret_cast<uint64_t>(base), rows, cols, ld_bytes,
+                           (uint64_t)box_cols | ((uint64_t)box_rows << 16) | ((uint64_t)elem_bytes << 32) |
+                               ((uint64_t)(is_bf16 ? 1 : 0) << 40) | ((uint64_t)swizzle_bytes << 44)};
+  uint64_t hsh = 0x9E3779B97F4A7C15ull;
+  for (int i = 0; i < 5; ++i) hsh = (hsh ^ key[i]) * 0xBF58476D1CE4E5B9ull + (hsh >> 29);
+  hero_handle* hm = const_cast<hero_handle*>(h);
+  hero_tmap_slot& slot = hm->tmap[(hsh >> 32) % HERO_TMAP_SLOTS];
+  std::lock_guard<std::mutex> guard(hm->tmap_mu);
+  if (slot.used && memcmp(slot.key, key, sizeof(key)) == 0) {
+    *out = slot.map;
+    return HERO_OK;
+  }
   CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_UINT8;
   if (elem_bytes == 2) dt = is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
   (void)is_fp16;
@@ -72,6 +85,9 @@ hero_status make_tmap_2d(const hero_handle* h, CUtensorMap* out, const void* bas
   HERO_REQUIRE(r == CUDA_SUCCESS, HERO_ERR_CUDA,
                "cuTensorMapEncodeTiled failed (%d): rows=%llu cols=%llu ld_bytes=%llu box=%ux%u", (int)r,
                (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)ld_bytes, box_cols, box_rows);
+  memcpy(slot.key, key, sizeof(key));
+  slot.map = *out;
+  slot.used = true;
   return HERO_OK;
 }
 

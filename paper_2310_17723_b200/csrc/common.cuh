@@ -7,11 +7,22 @@
 #include <cstdio>
 #include <cstring>
 #include <atomic>
+#include <mutex>
 
 #include "../../include/hero.h"
 #ifdef __CUDACC__
 #include <cuda_fp16.h>
 #endif
+
+// A tensor map is a pure function of (base, shape, pitch, box, type, swizzle); encoding one costs about a microsecond of
+// host time, several per launch.  Layers launch the same shapes on the same buffers over and over: a small direct-mapped
+// cache in the handle spares the latency-bound workloads that host time.
+struct hero_tmap_slot {
+  uint64_t key[5];
+  CUtensorMap map;
+  bool used = false;
+};
+constexpr int HERO_TMAP_SLOTS = 128;
 
 struct hero_handle {
   int device;
@@ -25,6 +36,8 @@ struct hero_handle {
   int prof_cap, prof_n;
   cudaEvent_t* prof_ev;   // 2 * prof_cap events
   int32_t* prof_tag;      // kernel family of each recorded launch
+  std::mutex tmap_mu;     // several host threads may share a handle
+  hero_tmap_slot tmap[HERO_TMAP_SLOTS];
 };
 
 namespace hero {
