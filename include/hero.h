@@ -112,6 +112,11 @@ int64_t hero_launch_count(const hero_handle* h);
  *              out.data == NULL skips the normalisation (bare residual add into fp_out).
  *   fp_out   : optional F16 / BF16 copy of r (the FP residual stream of a pre-LN layer); when
  *              present the normalisation reads the stored (rounded) r.
+ *   out_col_absmax : optional calibration observer (Sec. 2.1: FWQ / SQ scales come from calibration), device float[H]
+ *              that the caller zeroes once: after the call entry j is max(old, max_i |t[i,j]|) of the FP tensor the
+ *              call stores, t = out when out is F16 / BF16, t = fp_out when out.data is NULL.  The values observed are
+ *              the stored (rounded) ones, so the result equals hero_absmax_observe on t bit for bit, without the
+ *              second read.  An 8-bit out: HERO_ERR_UNSUPPORTED.
  * H must be a multiple of 16 and at most 16384.  M may be any size, including 0 (no launch).
  */
 typedef struct {
@@ -127,6 +132,7 @@ typedef struct {
   float eps;
   hero_tensor out;
   hero_tensor fp_out;
+  float* out_col_absmax;    /* device [H] or NULL */
 } hero_ln_args;
 
 hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* a, void* stream);
@@ -208,6 +214,10 @@ typedef struct {
                           it once); after the call it is max(old, largest softmax probability seen), from which
                           calibration takes s_p = p_absmax / 255 (Eq. 16).  NULL: not observed. */
   int32_t p_mode;      /* hero_p_mode: how P is quantized (INT8 core only); 0 = the paper's static scale */
+  float* out_col_absmax; /* optional, F16 / BF16 core with an F16 / BF16 out only: device float[nh*dh] of running
+                          per-column maxima of |out| as stored (the caller zeroes it once), equal bit for bit to
+                          hero_absmax_observe on out; calibration takes the FWQ scale of X_attn from it (Eq. 17).
+                          NULL: not observed.  Any other combination: HERO_ERR_UNSUPPORTED. */
 } hero_attn_args;
 
 hero_status hero_int8_attention(hero_handle* h, const hero_attn_args* a, void* stream);

@@ -1,7 +1,7 @@
 """Calibration on the device (Sec. 2.1): the un-quantized layer runs in FP16 / BF16 through the library's own
-operators; the outputs of the four linear modules are observed by their own epilogues (hero_linear_args.out_col_absmax),
-the softmax probabilities by the FP attention core, the other border tensors (LayerNorm and attention outputs, the
-layer's input) with hero_absmax_observe, and the weights are folded and quantized column-wise by hero_quantize_weight
+operators; every border tensor is observed by the kernel that produces it (the out_col_absmax option of the linear,
+LayerNorm and attention calls; the softmax probabilities through p_absmax), only the input of a post-LN layer, which no
+kernel of the layer produces, with hero_absmax_observe, and the weights are folded and quantized column-wise by hero_quantize_weight
 (Eq. 2, Eq. 20-23, Eq. 32).  Same statistics and the same result layout as the host-side `prep.calibrate` /
 `prep.fold_quantize`; only argument marshalling happens here."""
 import numpy as np
@@ -50,8 +50,12 @@ def calibrate_gpu(h, cfg, params, x_cal, n_seq, return_output=False):
     def colmax(n):
         return torch.zeros(n, dtype=torch.float32, device="cuda")
 
+    def fused(name, n):
+        """Registers the per-feature statistic `name`, to be filled by its producer; the per-tensor one is its maximum."""
+        stat[name + "_f"] = colmax(n)
+        return stat[name + "_f"]
+
     def attn(x_in):
-        observe("in", x_in)
         qkv = new(3 * H)
         # the outputs of the linear modules are observed by their own epilogues (per-column running maxima; Q, K and V
         # want one static scale each: the maximum over their column ranges)
@@ -62,15 +66,14 @@ def calibrate_gpu(h, cfg, params, x_cal, n_seq, return_output=False):
             stat[n + "_t"] = qkv_f[i * H:(i + 1) * H].max().reshape(1)
         xa = new(H)
         stat["p_t"] = torch.zeros(1, dtype=torch.float32, device="cuda")
-        h.hero_int8_attention(q, k, v, n_seq, S, nh, dh, hero.tensor(xa), mask=cfg.mask, p_absmax=stat["p_t"])
-        observe("attn", xa)
+        h.hero_int8_attention(q, k, v, n_seq, S, nh, dh, hero.tensor(xa), mask=cfg.mask, p_absmax=stat["p_t"],
+                              out_col_absmax=fused("attn", H))
         xo = new(H)
         stat["o_f"] = colmax(H)
         h.hero_w8a8_linear(hero.tensor(xa), Wo, hero.tensor(xo), bias=bo, out_col_absmax=stat["o_f"])
         return xo
 
     def mlp(x_mid):
-        observe("mid", x_mid)
         a = new(F)
         stat["a_f"] = colmax(F)
         h.hero_w8a8_linear(hero.tensor(x_mid), W1, hero.tensor(a), bias=b1, act=cfg.act, out_col_absmax=stat["a_f"])
@@ -81,20 +84,26 @@ def calibrate_gpu(h, cfg, params, x_cal, n_seq, return_output=False):
 
     out = new(H)
     if cfg.arch == "post_ln":
+        observe("in", x, per_tensor=False)
         xo = attn(x)
         xm = new(H)
-        h.hero_layernorm_quant(hero.tensor(x), g1, be1, cfg.eps, hero.tensor(xm), branch=hero.tensor(xo))
+        h.hero_layernorm_quant(hero.tensor(x), g1, be1, cfg.eps, hero.tensor(xm), branch=hero.tensor(xo),
+                               out_col_absmax=fused("mid", H))
         x2 = mlp(xm)
-        h.hero_layernorm_quant(hero.tensor(xm), g2, be2, cfg.eps, hero.tensor(out), branch=hero.tensor(x2))
+        h.hero_layernorm_quant(hero.tensor(xm), g2, be2, cfg.eps, hero.tensor(out), branch=hero.tensor(x2),
+                               out_col_absmax=fused("out", H))
     else:
         xl = new(H)
-        h.hero_layernorm_quant(hero.tensor(x), g1, be1, cfg.eps, hero.tensor(xl))
+        h.hero_layernorm_quant(hero.tensor(x), g1, be1, cfg.eps, hero.tensor(xl), out_col_absmax=fused("in", H))
         xo = attn(xl)
         xm, h1 = new(H), new(H)
-        h.hero_layernorm_quant(hero.tensor(x), g2, be2, cfg.eps, hero.tensor(xm), branch=hero.tensor(xo), fp_out=hero.tensor(h1))
+        h.hero_layernorm_quant(hero.tensor(x), g2, be2, cfg.eps, hero.tensor(xm), branch=hero.tensor(xo), fp_out=hero.tensor(h1),
+                               out_col_absmax=fused("mid", H))
         x2 = mlp(xm)
-        h.hero_layernorm_quant(hero.tensor(h1), None, None, cfg.eps, None, branch=hero.tensor(x2), fp_out=hero.tensor(out))
-    observe("out", out)
+        h.hero_layernorm_quant(hero.tensor(h1), None, None, cfg.eps, None, branch=hero.tensor(x2), fp_out=hero.tensor(out),
+                               out_col_absmax=fused("out", H))
+    for n in ("in", "attn", "mid", "out"):
+        stat[n + "_t"] = stat[n + "_f"].max().reshape(1)
     h.check()
     torch.cuda.synchronize()
     g = lambda k: stat[k].cpu().numpy().astype(np.float64)

@@ -593,6 +593,9 @@ static hero_status attention_impl(hero_handle* h, const hero_attn_args* a, const
   p.err = h->d_error;
   p.p_absmax = a->p_absmax;
   HERO_REQUIRE(a->p_absmax == nullptr || fp_in, HERO_ERR_UNSUPPORTED, "p_absmax is observed by the F16 / BF16 attention core only");
+  p.obs_col = a->out_col_absmax;
+  HERO_REQUIRE(a->out_col_absmax == nullptr || (fp_in && is_fp16ish(a->out.dtype)), HERO_ERR_UNSUPPORTED,
+               "out_col_absmax is observed by the F16 / BF16 attention core on an F16 / BF16 output only");
   HERO_REQUIRE((long long)p.nqt * a->nh * a->B < (1ll << 31), HERO_ERR_UNSUPPORTED, "too many tiles");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (probe) {

@@ -33,6 +33,7 @@ struct AttnParams {
   uint32_t idesc_qk, idesc_pv;
   int* err;
   float* p_absmax;         // calibration observer of the FP core: running max of the softmax probabilities, or NULL
+  float* obs_col;          // calibration observer of the FP core: per-column running absmax of an FP output, or NULL
   // verification outputs (hero_int8_attention_probe; kernels compiled with PROBE only): raw Q K^T accumulators and
   // P codes [B*nh][S][S], raw P V accumulators [B*S][nh*dh]; each may be NULL
   int* dbg_scores;

@@ -319,6 +319,19 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
         for (int j = 0; j < 32; ++j) r[j] = 0;
       }
+      if (p.obs_col != nullptr && cq * 32 < DH) {
+        // calibration observer: per-column maximum over the tile's 32 rows of this warp, rounded as the store rounds
+        // (rounding is monotonic and symmetric, so the maximum of the rounded values is the rounded maximum)
+        uint32_t mine = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const uint32_t mx = __reduce_max_sync(0xffffffffu, row_ok ? (r[j] & 0x7fffffffu) : 0u);
+          if (lane == j) mine = mx;
+        }
+        const uint32_t h = fp2(__uint_as_float(mine), 0.f, p.out_dt) & 0xffffu;
+        const float stored = p.out_dt == HERO_F16 ? __half2float(__ushort_as_half((unsigned short)h)) : __uint_as_float(h << 16);
+        if (stored > 0.f) atomicMax(reinterpret_cast<int*>(p.obs_col) + col0 + cq * 32 + lane, __float_as_int(stored));
+      }
       if (cq * 32 < DH && row_ok) {
         const long long grow = (long long)(row_base + q);
         const int gcol = col0 + cq * 32;

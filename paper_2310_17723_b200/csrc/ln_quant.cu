@@ -34,6 +34,7 @@ struct LnParams {
   float eps;
   void* out; int out_dt; long long out_ld; int out_gran; float* out_scale;
   void* fp_out; int fp_dt; long long fp_ld;
+  float* obs;             // calibration: per-column running absmax of the FP tensor the call stores, or NULL
   long long M; int H;
   int G;                  // threads per row (multiple of 32)
   int RPC;                // rows per CTA per pass
@@ -197,6 +198,9 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
   const int res_es = is_q8(p.res.dt) ? 1 : 2;
   const int br_es = is_q8(p.br.dt) ? 1 : 2;
   const long long rows_per_trip = (long long)RPC * R;
+  float om[VEC];          // calibration observer: this thread's columns, maximum over the rows it visits
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) om[i] = 0.f;
 
   for (long long base = (long long)blockIdx.x * rows_per_trip; base < p.M; base += (long long)gridDim.x * rows_per_trip) {
     float x[R][VEC];
@@ -273,6 +277,10 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
           for (int i = 0; i < VEC / 2; ++i) w[i] = pack_fp2(x[r][2 * i], x[r][2 * i + 1], p.fp_dt);
           store_words<VEC>(reinterpret_cast<char*>(p.fp_out) + (row[r] * p.fp_ld + c0) * 2, w, VEC / 2);
           unpack<VEC>(w, p.fp_dt, x[r]);
+          if (p.obs && !normalize) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) om[i] = fmaxf(om[i], fabsf(x[r][i]));
+          }
         }
       } else {
 #pragma unroll
@@ -364,8 +372,19 @@ __global__ void __launch_bounds__(1024) ln_quant_kernel(const LnParams p) {
 #pragma unroll
         for (int i = 0; i < VEC / 2; ++i) w[i] = pack_fp2(x[r][2 * i], x[r][2 * i + 1], p.out_dt);
         store_words<VEC>(reinterpret_cast<char*>(p.out) + (row[r] * p.out_ld + c0) * 2, w, VEC / 2);
+        if (p.obs) {        // what is observed is what is stored: the rounded values
+          float y[VEC];
+          unpack<VEC>(w, p.out_dt, y);
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) om[i] = fmaxf(om[i], fabsf(y[i]));
+        }
       }
     }
+  }
+  if (p.obs && active) {    // non-negative floats order like their bit patterns
+#pragma unroll
+    for (int i = 0; i < VEC; ++i)
+      if (om[i] > 0.f) atomicMax(reinterpret_cast<int*>(p.obs) + c0 + i, __float_as_int(om[i]));
   }
 }
 
@@ -1448,13 +1467,20 @@ extern "C" hero_status hero_layernorm_quant(hero_handle* h, const hero_ln_args* 
     p.fp_out = a->fp_out.data; p.fp_dt = a->fp_out.dtype; p.fp_ld = a->fp_out.ld;
   }
   HERO_REQUIRE(p.out || p.fp_out, HERO_ERR_INVALID_ARG, "neither out nor fp_out given");
+  if (a->out_col_absmax) {
+    HERO_REQUIRE(p.out ? is_fp16ish(p.out_dt) : true, HERO_ERR_UNSUPPORTED,
+                 "out_col_absmax observes an F16 / BF16 out (or fp_out when out is absent), not 8-bit codes");
+    p.obs = a->out_col_absmax;
+  }
   if (p.M == 0) return HERO_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   bool taken = false;
-  st = try_wide(h, p, s, &taken);
-  if (taken || st != HERO_OK) return st;
-  st = try_fast(h, p, s, &taken);
-  if (taken || st != HERO_OK) return st;
+  if (!p.obs) {             // the observer lives in the generic kernel only (calibration is an offline pass)
+    st = try_wide(h, p, s, &taken);
+    if (taken || st != HERO_OK) return st;
+    st = try_fast(h, p, s, &taken);
+    if (taken || st != HERO_OK) return st;
+  }
   // generic kernel for the remaining combinations.
   // 16 elements per thread when rows are long (fewer, fatter threads); 8 otherwise.  VEC=16 needs H % 16 == 0.
   if (H % 16 == 0 && H >= 2048) return launch_ln<16, 1>(h, p, s);

@@ -45,7 +45,8 @@ class Tensor(C.Structure):
 class LnArgs(C.Structure):
     _fields_ = [("residual", Tensor), ("branch", Tensor), ("extra", Tensor), ("token_ids", C.c_void_p),
                 ("type_ids", C.c_void_p), ("seq_len", C.c_int32), ("n_tokens", C.c_int64), ("gamma", C.c_void_p),
-                ("beta", C.c_void_p), ("eps", C.c_float), ("out", Tensor), ("fp_out", Tensor)]
+                ("beta", C.c_void_p), ("eps", C.c_float), ("out", Tensor), ("fp_out", Tensor),
+                ("out_col_absmax", C.c_void_p)]
 
 
 class LinearArgs(C.Structure):
@@ -58,7 +59,8 @@ class AttnArgs(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("dtype", C.c_int32), ("ld", C.c_int64),
                 ("B", C.c_int32), ("S", C.c_int32), ("nh", C.c_int32), ("dh", C.c_int32), ("s_q", C.c_float),
                 ("s_k", C.c_float), ("s_v", C.c_float), ("s_p", C.c_float), ("mask", C.c_int32),
-                ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p), ("p_mode", C.c_int32)]
+                ("key_len", C.c_void_p), ("out", Tensor), ("p_absmax", C.c_void_p), ("p_mode", C.c_int32),
+                ("out_col_absmax", C.c_void_p)]
 
 
 class AttnProbe(C.Structure):
@@ -223,11 +225,12 @@ class Handle:
 
     # ---- the four calls of the boundary, same names as the C entry points ----
     def hero_layernorm_quant(self, residual, gamma, beta, eps, out, branch=None, extra=None, fp_out=None,
-                             token_ids=None, type_ids=None, seq_len=0, n_tokens=0, stream=None):
-        """residual / branch / extra / out / fp_out are hero.Tensor structs (see `tensor`)."""
+                             token_ids=None, type_ids=None, seq_len=0, n_tokens=0, out_col_absmax=None, stream=None):
+        """residual / branch / extra / out / fp_out are hero.Tensor structs (see `tensor`); out_col_absmax: float32 [H]
+        running per-column absolute maximum of the FP tensor the call stores (calibration observer)."""
         a = LnArgs(residual, branch or tensor(None), extra or tensor(None), _ptr(token_ids), _ptr(type_ids),
                    int(seq_len), int(n_tokens), _ptr(gamma), _ptr(beta), float(eps), out or tensor(None),
-                   fp_out or tensor(None))
+                   fp_out or tensor(None), _ptr(out_col_absmax))
         _check(lib().hero_layernorm_quant(self._h, C.byref(a), _stream(stream)))
 
     def hero_w8a8_linear(self, A, W, out, w_scale=None, bias=None, act="none", post_scale=None, out_col_absmax=None,
@@ -240,14 +243,15 @@ class Handle:
         _check(lib().hero_w8a8_linear(self._h, C.byref(a), _stream(stream)))
 
     def hero_int8_attention(self, q, k, v, B, S, nh, dh, out, s_q=1.0, s_k=1.0, s_v=1.0, s_p=1.0 / 255,
-                            mask="none", key_len=None, p_absmax=None, p_mode="static", probe=None, stream=None):
+                            mask="none", key_len=None, p_absmax=None, p_mode="static", probe=None, out_col_absmax=None,
+                            stream=None):
         """q, k, v: 2-D torch views [B*S, nh*dh] sharing one leading dimension; out: hero.Tensor; p_absmax: float32[1]
         running maximum of the softmax probabilities (F16 / BF16 core only).  probe = (scores int32 [B*nh, S, S] | None,
         p_codes uint8 [B*nh, S, S] | None, acc int32 [B*S, nh*dh] | None) calls hero_int8_attention_probe instead."""
         assert q.stride(0) == k.stride(0) == v.stride(0) and q.dtype == k.dtype == v.dtype
         a = AttnArgs(q.data_ptr(), k.data_ptr(), v.data_ptr(), _DT[q.dtype], q.stride(0), B, S, nh, dh, s_q, s_k,
                      s_v, s_p, MASK[mask] if isinstance(mask, str) else mask, _ptr(key_len), out, _ptr(p_absmax),
-                     P_MODE[p_mode] if isinstance(p_mode, str) else p_mode)
+                     P_MODE[p_mode] if isinstance(p_mode, str) else p_mode, _ptr(out_col_absmax))
         if probe is not None:
             scores, codes, acc = probe
             pr = AttnProbe(_ptr(scores), _ptr(codes), _ptr(acc))

@@ -91,6 +91,98 @@ def test_linear_epilogue_observer_refuses_an_int8_output(h):
     assert e.value.status == hero.ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("M,H,flavour", [(5, 64, "ln"), (1000, 768, "ln"), (4099, 1024, "add_ln"), (333, 4096, "add_ln"),
+                                         (777, 1024, "add_ln_fp"), (1300, 768, "bare_add")])
+def test_layernorm_observer_equals_the_streaming_observer(h, dt, M, H, flavour):
+    # the observer of the LayerNorm call sees the FP tensor it stores (out; fp_out for the bare residual add) as stored
+    g = W.rng(21, M + H)
+    t = TORCH_FP[dt]
+    mk = lambda s: torch.from_numpy((g.standard_normal((M, H)) * s).astype(np.float32)).to(t).cuda()
+    x, br = mk(1.0), mk(0.3)
+    gam = torch.from_numpy((1 + 0.1 * g.standard_normal(H)).astype(np.float32)).cuda()
+    bet = torch.from_numpy((0.1 * g.standard_normal(H)).astype(np.float32)).cuda()
+    out, fpo = torch.empty(M, H, dtype=t, device="cuda"), torch.empty(M, H, dtype=t, device="cuda")
+    fused = torch.zeros(H, dtype=torch.float32, device="cuda")
+    ref = torch.zeros(H, dtype=torch.float32, device="cuda")
+
+    def run(xx):
+        if flavour == "ln":
+            h.hero_layernorm_quant(hero.tensor(xx), gam, bet, 1e-5, hero.tensor(out), out_col_absmax=fused)
+            return out
+        if flavour == "add_ln":
+            h.hero_layernorm_quant(hero.tensor(xx), gam, bet, 1e-5, hero.tensor(out), branch=hero.tensor(br), out_col_absmax=fused)
+            return out
+        if flavour == "add_ln_fp":
+            h.hero_layernorm_quant(hero.tensor(xx), gam, bet, 1e-5, hero.tensor(out), branch=hero.tensor(br),
+                                   fp_out=hero.tensor(fpo), out_col_absmax=fused)
+            return out
+        h.hero_layernorm_quant(hero.tensor(xx), None, None, 1e-5, None, branch=hero.tensor(br), fp_out=hero.tensor(fpo),
+                               out_col_absmax=fused)
+        return fpo
+
+    for xx in (x, (x * 0.5 + 2.0).contiguous()):                   # the second batch: running maxima
+        seen = run(xx)
+        h.hero_absmax_observe(hero.tensor(seen), ref, None)
+        h.check()
+        assert torch.equal(fused, ref)
+    assert float(fused.min()) > 0
+    # the observed call stores what the unobserved one stores
+    plain = torch.empty_like(seen)
+    if flavour == "bare_add":
+        h.hero_layernorm_quant(hero.tensor(xx), None, None, 1e-5, None, branch=hero.tensor(br), fp_out=hero.tensor(plain))
+    else:
+        h.hero_layernorm_quant(hero.tensor(xx), gam, bet, 1e-5, hero.tensor(plain),
+                               branch=None if flavour == "ln" else hero.tensor(br),
+                               fp_out=hero.tensor(torch.empty_like(fpo)) if flavour == "add_ln_fp" else None)
+    h.check()
+    if flavour == "bare_add":
+        assert torch.equal(plain.view(torch.int16), seen.view(torch.int16))
+    else:                                                          # another kernel: the row sums may round differently
+        assert torch.allclose(plain.float(), seen.float(), rtol=1e-2, atol=1e-2)
+
+
+def test_layernorm_observer_refuses_an_int8_output(h):
+    x = torch.zeros(64, 256, dtype=torch.float16, device="cuda")
+    out = torch.empty(64, 256, dtype=torch.int8, device="cuda")
+    sc = torch.ones(256, dtype=torch.float32, device="cuda")
+    with pytest.raises(hero.HeroError) as e:
+        h.hero_layernorm_quant(hero.tensor(x), sc, sc, 1e-5, hero.tensor(out, "fwq", sc), out_col_absmax=sc)
+    assert e.value.status == hero.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+@pytest.mark.parametrize("B,S,nh,dh,mask,klen", [(2, 128, 4, 64, "none", False), (3, 200, 2, 128, "causal", False),
+                                                   (2, 333, 3, 64, "none", True), (1, 1000, 2, 64, "causal", False)])
+def test_attention_observer_equals_the_streaming_observer(h, dt, B, S, nh, dh, mask, klen):
+    g = W.rng(33, B * S + nh)
+    t = TORCH_FP[dt]
+    H = nh * dh
+    qkv = torch.from_numpy(g.standard_normal((B * S, 3 * H)).astype(np.float32)).to(t).cuda()
+    q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
+    kl = torch.from_numpy(g.integers(1, S + 1, B).astype(np.int32)).cuda() if klen else None
+    out = torch.empty(B * S, H, dtype=t, device="cuda")
+    fused = torch.zeros(H, dtype=torch.float32, device="cuda")
+    ref = torch.zeros(H, dtype=torch.float32, device="cuda")
+    for scale in (1.0, 2.0):                                       # the second batch: running maxima
+        vv = (qkv * scale).contiguous()
+        h.hero_int8_attention(vv[:, :H], vv[:, H:2 * H], vv[:, 2 * H:], B, S, nh, dh, hero.tensor(out), mask=mask,
+                              key_len=kl, out_col_absmax=fused)
+        h.hero_absmax_observe(hero.tensor(out), ref, None)
+        h.check()
+        assert torch.equal(fused, ref)
+    assert float(fused.min()) > 0
+
+
+def test_attention_observer_refuses_the_int8_core(h):
+    q = torch.zeros(128, 64, dtype=torch.int8, device="cuda")
+    out = torch.empty(128, 64, dtype=torch.float16, device="cuda")
+    sc = torch.zeros(64, dtype=torch.float32, device="cuda")
+    with pytest.raises(hero.HeroError) as e:
+        h.hero_int8_attention(q, q, q, 1, 128, 1, 64, hero.tensor(out), out_col_absmax=sc)
+    assert e.value.status == hero.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("K,N,fold", [(256, 192, "none"), (1024, 3072, "both"), (4096, 1024, "in"), (768, 768, "out")])
 def test_quantize_weight_matches_fold_then_eq2(h, K, N, fold):
     rng = np.random.default_rng(K + N)
