@@ -528,6 +528,17 @@ def run_ours(args):
     value = replicas.job_throughput(shape.M, args.steps, world, total_ms * 1e-3)
     # the same steps without the entry LN^quant (the layers alone, their INT8 input already in place)
     layers_only_ms = timed(step_layers_only, args.steps) / args.steps if post else None
+    # host time of the C-ABI call: a burst of calls short enough to stay inside the driver's launch queue, so the host
+    # never waits for the device; wall clock until the last call has returned
+    host_us = None
+    if rank == 0:
+        nburst = max(1, min(64, 512 // max(launches_per_step, 1)))
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(nburst):
+            eager_step()
+        host_us = (time.perf_counter() - t0) / nburst * 1e6
+        torch.cuda.synchronize()
 
     # ---- per-kernel device times (a second, instrumented pass: event pairs around every launch)
     kern = []
@@ -688,6 +699,10 @@ def run_ours(args):
     if layers_only_ms is not None:
         line["without_entry_ln"] = {"ms_per_step": layers_only_ms, "value": shape.M / (layers_only_ms * 1e-3), "unit": UNIT,
                                     "note": "the layers alone, their INT8 input already in place (one rank's device time)"}
+    if host_us is not None:
+        line["host_us_per_step"] = {"value": host_us, "launches": launches_per_step,
+                                    "note": "wall clock of the C-ABI call itself (argument checks, tensor-map lookup, launches), "
+                                            "device not waited for"}
     if mixed_path:
         line["attention_and_ln_bf16_path"] = mixed_path
     if extra:
