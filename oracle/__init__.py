@@ -16,9 +16,12 @@ search  per-module sensitivity and the greedy INT8 -> FP mode search that
         generalises Table 1's presets (Sec. 2.3), as loops over `layer`
 
 Pins (what fixes each function to something other than itself) live in
-tests/test_oracle_*.py; the whole INT8 layer has no external definition and is
-"parity unpinned" as a whole: it is pinned piecewise (integer contractions,
-quantizers, folding identities, LayerNorm/GELU/softmax closed forms, the
-all-FP layer against a library transformer layer) plus a sanity bound against
-the unquantized layer.
+tests/test_oracle_*.py.  The whole INT8 layer has no external definition to
+the last bit; it is pinned in two ways: every rounding decision piecewise
+(integer contractions, quantizers, folding identities, LayerNorm / GELU /
+softmax closed forms, the all-FP layer against a library transformer layer),
+and the wiring of the layer stage by stage: each operator of layer_forward,
+in every mode of Table 1, against the float64 library routine of that operator
+fed the dequantized border the oracle itself fed it, to within the operator's
+quantization steps, plus a bound against the unquantized layer end to end.
 """

@@ -144,6 +144,58 @@ def test_int8_layer_is_close_to_unquantized_layer_and_types_follow_table1(preset
         assert (T[key] is not None) == (m[mod] == "int8")
 
 
+# Largest |difference| / largest |value| allowed per border when a library routine recomputes the stage from the oracle's
+# own (dequantized) input border: the stage's quantization steps (8-bit weights, 8-bit output, 8-bit P) and nothing else.
+# Measured on these seeds: 0.0004 - 0.023; a dropped bias, a scale on the wrong axis, a missing 1 / sqrt(dh) or a
+# transposed weight gives 0.1 or more.
+_STAGE_BAR = {"qkv": 0.02, "x_attn": 0.05, "x_o": 0.025, "h_mid": 0.002, "x_mid": 0.008, "a": 0.04, "x_2": 0.035,
+              "x_out": 0.008, "h_out": 0.002}
+
+
+@pytest.mark.parametrize("preset", ["M1", "M2", "M3"])
+@pytest.mark.parametrize("arch", ["post_ln", "pre_ln"])
+def test_every_stage_of_the_layer_matches_a_library_routine_fed_its_own_input_border(preset, arch):
+    # teacher-forced: each operator of layer_forward, whatever its mode, must agree with the float64 library routine of the
+    # same operator applied to the dequantized tensor the oracle itself fed it, to within that operator's quantization
+    # steps.  This pins the wiring of the whole quantized layer (which border feeds which operator, every folded scale,
+    # bias and dequantization factor) to something other than the oracle.
+    shape = W.tiny_shape(arch=arch, mask="causal" if arch == "pre_ln" else "none", eps=1e-5, n_outlier=2)
+    spec = _spec(shape, mode=dict(L.MODE_PRESETS[preset]))
+    p = W.layer_params(shape, 9)
+    x = W.activations(shape, 9)
+    C = L.calibrate(spec, p, x if arch == "pre_ln" else O.layernorm(x, p["ln0_g"], p["ln0_b"], spec.eps), shape.B)
+    Lp = L.prepare_layer(spec, p, C)
+    x_in = (L.entry_ln(O.fp_tensor(x, "f16"), p["ln0_g"], p["ln0_b"], spec.eps, Lp["ln_in_out"]) if arch == "post_ln"
+            else O.fp_tensor(x, spec.fp_dtype))
+    T = L.layer_forward(Lp, x_in)
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    r = lambda k: t(T[k].real())
+    H, nh, dh, S, B = spec.H, spec.nh, spec.dh, spec.S, shape.B
+    lin = torch.nn.functional.linear
+    ln = lambda v, g, b: torch.nn.functional.layer_norm(v, (H,), t(p[g]), t(p[b]), spec.eps)
+    want = {}
+    want["qkv"] = lin(r("x_in"), t(np.concatenate([p["Wq"], p["Wk"], p["Wv"]], axis=1)).T,
+                      t(np.concatenate([p["bq"], p["bk"], p["bv"]])))
+    q, k, v = (r("qkv")[:, i * H:(i + 1) * H].reshape(B, S, nh, dh).transpose(1, 2) for i in range(3))
+    want["x_attn"] = torch.nn.functional.scaled_dot_product_attention(
+        q, k, v, is_causal=(spec.mask == "causal")).transpose(1, 2).reshape(B * S, H)
+    want["x_o"] = lin(r("x_attn"), t(p["Wo"]).T, t(p["bo"]))
+    if arch == "post_ln":
+        want["x_mid"] = ln(r("x_in") + r("x_o"), "ln1_g", "ln1_b")
+    else:
+        want["h_mid"] = r("h_in") + r("x_o")
+        want["x_mid"] = ln(r("h_mid"), "ln2_g", "ln2_b")
+    want["a"] = torch.nn.functional.gelu(lin(r("x_mid"), t(p["W1"]).T, t(p["b1"])))
+    want["x_2"] = lin(r("a"), t(p["W2"]).T, t(p["b2"]))
+    if arch == "post_ln":
+        want["x_out"] = ln(r("x_mid") + r("x_2"), "ln2_g", "ln2_b")
+    else:
+        want["h_out"] = r("h_mid") + r("x_2")
+    for key, w in want.items():
+        e = float((r(key) - w).abs().max() / w.abs().max())
+        assert e < _STAGE_BAR[key], (key, e)
+
+
 def test_granularity_options_fwq_input_and_sq_attn():
     # FWQ on the LN output feeding QKV (scale folded into the QKV weight rows) and SQ on X_attn
     shape = W.tiny_shape(n_outlier=3, eps=1e-5)
