@@ -1,9 +1,11 @@
 // FP16 / BF16 attention for a module the mode table leaves in FP (Sec. 2.3, Table 1; Eq. 9-11):
 // P = softmax(Q K^T / sqrt(dh)), X_attn = P V with fp32 accumulation, stored in FP16 / BF16 or, when the
 // attention-output linear is INT8, quantized by the calibrated S_attn in the epilogue (no standalone
-// quantize kernel).  Same persistent, two-sweep, TMEM-resident structure as the INT8 core so that the two
-// paths differ only in operand type: kind::f16 MMAs, fp32 scores, P stored as FP16 / BF16 in the UMMA
-// operand layout.  A tile row of 128 features is 256 bytes, i.e. two 128-byte-swizzled sub-tiles.
+// quantize kernel).  Same persistent, two-sweep, TMEM-resident structure as the INT8 core for long sequences: kind::f16
+// MMAs, fp32 scores, P stored as FP16 / BF16 in the UMMA operand layout.  Nothing here quantizes P with a static scale,
+// so the first sweep only needs the row maximum (no exponentials): the second sweep forms e = 2^(t - m) <= 1, sums it in
+// FP32 and feeds the UN-normalised e to P V; the row sum is divided out of the accumulator in the epilogue.  One
+// exponential per score.  A tile row of 128 features is 256 bytes, i.e. two 128-byte-swizzled sub-tiles.
 #include "attention_common.cuh"
 
 namespace hero {
@@ -214,8 +216,8 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       int kmax = klen - 1;
       if (p.mask == HERO_MASK_CAUSAL) kmax = min(kmax, q);
 
-      float m = -INFINITY, l = 0.f;
-      // ---- sweep 1: running row max and row sum (log2 domain)
+      float m = -INFINITY;
+      // ---- sweep 1: running row max (log2 domain)
       for (int i = 0; i < nkv; ++i, ++scnt) {
         const int sb = scnt % ATT_NSB;
         if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x6000 | sb)) ok = false;
@@ -226,16 +228,20 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           ptx::tmem_ld_wait();
           const int kb = i * ATT_BN + cq * 32;
           const int nvalid = min(32, kmax - kb + 1);
-          if (nvalid > 0) {
+          if (__all_sync(0xffffffffu, nvalid >= 32)) {
+            // every key of the piece allowed for every row of the warp: no per-element tests
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              mx0 = ptx::max3(mx0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+              mx1 = ptx::max3(mx1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            }
+            m = fmaxf(m, fmaxf(mx0, mx1) * c2);
+          } else if (nvalid > 0) {
             float smax = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 32; ++j) smax = fmaxf(smax, j < nvalid ? __uint_as_float(r[j]) : -INFINITY);
-            const float m_new = fmaxf(m, smax * c2);
-            float acc = 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc += j < nvalid ? ex2f(fmaf(__uint_as_float(r[j]), c2, -m_new)) : 0.f;
-            l = l * ex2f(m - m_new) + acc;
-            m = m_new;
+            m = fmaxf(m, smax * c2);
           }
         }
         ptx::tc_fence_before();
@@ -243,32 +249,20 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
       }
       float2* st = stats + (wcnt & 1) * 4 * ATT_BM;
-      st[cq * ATT_BM + r_loc] = make_float2(m, l);
+      st[cq * ATT_BM + r_loc] = make_float2(m, 0.f);
       asm volatile("bar.sync 1, 512;" ::: "memory");
       {
         float mf = -INFINITY;
 #pragma unroll
         for (int g = 0; g < 4; ++g) mf = fmaxf(mf, st[g * ATT_BM + r_loc].x);
-        float lf = 0.f;
-        if (mf > -INFINITY) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const float2 o = st[g * ATT_BM + r_loc];
-            if (o.x > -INFINITY) lf += o.y * ex2f(o.x - mf);
-          }
-        }
-        m = mf; l = lf;
+        m = mf;
       }
-      const float inv_l = l > 0.f ? 1.0f / l : 0.f;
-      if (p.p_absmax != nullptr && cq == 0) {
-        // calibration observer (Eq. 16: S_p = max P / 255): the largest probability of a row is 2^0 / l
-        float pm = row_ok ? inv_l : 0.f;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, o));
-        if (lane == 0 && pm > 0.f) atomicMax(reinterpret_cast<unsigned int*>(p.p_absmax), __float_as_uint(pm));
-      }
+      const float mneg = m > -INFINITY ? -m : 0.f;            // a row without keys: every e is masked to 0 below
 
-      // ---- sweep 2: P = 2^(t - m) / l as FP16 / BF16 into shared memory (two 64-key sub-tiles, 128-byte swizzle)
+      // ---- sweep 2: e = 2^(t - m) <= 1 as FP16 / BF16 into shared memory (two 64-key sub-tiles, 128-byte swizzle) and the
+      // row sum of the e in FP32; the sum is divided out of the accumulator in the epilogue (one exponential per score:
+      // the first sweep needs the maximum only)
+      float l2a = 0.f, l2b = 0.f;
       for (int j = 0; j < nkv; ++j, ++scnt, ++pcnt) {
         const int sb = scnt % ATT_NSB, pb = pcnt % PB;
         if (ok && !ptx::mbar_wait(&s_full[sb], (scnt / ATT_NSB) & 1, p.err, 0x6100 | sb)) ok = false;
@@ -282,13 +276,27 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           const int kb = j * ATT_BN + cq * 32;
           const int nvalid = min(32, kmax - kb + 1);
           uint32_t w[16];
+          if (__all_sync(0xffffffffu, nvalid >= 32)) {
+            const float2 c22 = make_float2(c2, c2), nm2 = make_float2(mneg, mneg);
+            float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            float a = ex2f(fmaf(__uint_as_float(r[2 * e]), c2, -m)) * inv_l;
-            float c = ex2f(fmaf(__uint_as_float(r[2 * e + 1]), c2, -m)) * inv_l;
-            if (2 * e >= nvalid) a = 0.f;
-            if (2 * e + 1 >= nvalid) c = 0.f;
-            w[e] = fp2(a, c, in_dt);
+            for (int e = 0; e < 16; ++e) {
+              const float2 tt = __ffma2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), c22, nm2);
+              const float2 ev = make_float2(ex2f(tt.x), ex2f(tt.y));
+              acc2 = __fadd2_rn(acc2, ev);
+              w[e] = fp2(ev.x, ev.y, in_dt);
+            }
+            l2a += acc2.x; l2b += acc2.y;
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              float a = ex2f(fmaf(__uint_as_float(r[2 * e]), c2, mneg));
+              float c = ex2f(fmaf(__uint_as_float(r[2 * e + 1]), c2, mneg));
+              if (2 * e >= nvalid) a = 0.f;
+              if (2 * e + 1 >= nvalid) c = 0.f;
+              l2a += a; l2b += c;
+              w[e] = fp2(a, c, in_dt);
+            }
           }
           const int c16 = (cq & 1) * 4;                      // first 16-byte chunk of this thread's 64 bytes
 #pragma unroll
@@ -299,6 +307,18 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) { ptx::mbar_arrive(&s_empty[sb]); ptx::mbar_arrive(&p_full[pb]); }
+      }
+
+      // ---- the row sum from the four column parts; max P = 1 / l for the calibration observer (Eq. 16)
+      st[cq * ATT_BM + r_loc].y = l2a + l2b;
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      const float l = (st[r_loc].y + st[ATT_BM + r_loc].y) + (st[2 * ATT_BM + r_loc].y + st[3 * ATT_BM + r_loc].y);
+      const float inv_l = l > 0.f ? 1.0f / l : 0.f;
+      if (p.p_absmax != nullptr && cq == 0) {
+        float pm = row_ok ? inv_l : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, o));
+        if (lane == 0 && pm > 0.f) atomicMax(reinterpret_cast<unsigned int*>(p.p_absmax), __float_as_uint(pm));
       }
 
       // ---- epilogue
@@ -318,6 +338,10 @@ attn_fp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       if (nkv == 0) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) r[j] = 0;
+      } else if (cq * 32 < DH) {
+        // the accumulator holds sum_k e V: the row sum is divided out here
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * inv_l);
       }
       if (p.obs_col != nullptr && cq * 32 < DH) {
         // calibration observer: per-column maximum over the tile's 32 rows of this warp, rounded as the store rounds

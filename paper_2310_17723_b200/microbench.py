@@ -127,18 +127,25 @@ def bench_gemm(h, M, K, N, act, fp, iters, f8=False):
     return {"us": t * 1e6, "tops": tops, "gbs": gbs}
 
 
-def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static"):
+def bench_attn(h, B, S, nh, dh, mask, iters, p_mode="static", fp=False):
     H = nh * dh
-    qkv = (torch.randn(B * S, 3 * H, device="cuda") * 40).clamp(-127, 127).to(torch.int8)
-    out = torch.empty(B * S, H, device="cuda", dtype=torch.int8)
-    sc = torch.full((H,), 0.02, device="cuda")
-    s = (1.5 ** 0.5) / 40
-    t = _time(lambda i: h.hero_int8_attention(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh,
-                                              hero.tensor(out, "fwq", sc), s_q=s, s_k=s, s_v=0.02, s_p=1 / 255, mask=mask,
-                                              p_mode=p_mode), 1, iters)
+    if fp:                                     # the FP16 core of a module left in FP mode (Table 1): FP16 in, FP16 out
+        qkv = torch.randn(B * S, 3 * H, device="cuda", dtype=torch.float16)
+        out = torch.empty(B * S, H, device="cuda", dtype=torch.float16)
+        t = _time(lambda i: h.hero_int8_attention(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh, hero.tensor(out),
+                                                  mask=mask), 1, iters)
+    else:
+        qkv = (torch.randn(B * S, 3 * H, device="cuda") * 40).clamp(-127, 127).to(torch.int8)
+        out = torch.empty(B * S, H, device="cuda", dtype=torch.int8)
+        sc = torch.full((H,), 0.02, device="cuda")
+        s = (1.5 ** 0.5) / 40
+        t = _time(lambda i: h.hero_int8_attention(qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:], B, S, nh, dh,
+                                                  hero.tensor(out, "fwq", sc), s_q=s, s_k=s, s_v=0.02, s_p=1 / 255, mask=mask,
+                                                  p_mode=p_mode), 1, iters)
     scores = B * nh * S * S * (0.5 if mask == "causal" else 1.0)
-    _say("INT8 attention B=%d S=%d nh=%d dh=%d %s P=%s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
-         % (B, S, nh, dh, mask, p_mode, t * 1e6, scores / t / 1e12, 4 * scores * dh / t / 1e12))
+    _say("%s attention B=%d S=%d nh=%d dh=%d %s P=%s: %.1f us, %.2f T scores/s, %.0f TOP/s tensor work"
+         % ("FP16" if fp else "INT8", B, S, nh, dh, mask, "fp16" if fp else p_mode, t * 1e6, scores / t / 1e12,
+            4 * scores * dh / t / 1e12))
     return {"us": t * 1e6, "tscores": scores / t / 1e12}
 
 
@@ -312,7 +319,7 @@ def main():
     elif a.kernel == "layer":
         bench_layer(h, a.workload, "f8" if a.f8 else "i8", a.fp, a.iters)
     else:
-        bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters, a.p_mode)
+        bench_attn(h, a.B, a.S, a.nh, a.dh, a.mask, a.iters, a.p_mode, a.fp)
     h.check()
 
 
