@@ -152,12 +152,12 @@ def kernel_table(shape, cfg, first=False):
 # workload's step, each from one small ncu capture (one kernel, a few launches) recorded under profiles/; keyed by
 # (workload, kernel function).  These are constants of a recorded capture, not values this run measures.
 NCU_TRAFFIC = {
-    ("c5", "gemm_pair_kernel<int8, no activation>"): {"bytes_per_launch": 90.3e6, "source": "profiles/launch_list_c5_stack.md: ncu launch "
+    ("c5", "gemm_pair_kernel<int8, no activation>"): {"bytes_per_launch": 90.2e6, "source": "profiles/launch_list_c5_stack.md: ncu launch "
                           "list of this workload at full size (one pass: time + dram__bytes_read.sum + dram__bytes_write.sum), "
-                          "average over the 274 captured launches of the three members (69.9 MB read + 20.4 MB written; "
+                          "average over the 274 captured launches of the three members (69.9 MB read + 20.3 MB written; "
                           "algorithmic average 69.9 MB read + 55.9 MB written: most of an output is still in L2 when its kernel ends)"},
-    ("c5", "attention"): {"bytes_per_launch": 158.1e6, "source": "profiles/launch_list_c5_stack.md: same capture, 92 launches of "
-                          "attn_int8_pipe_kernel (139.2 MB read + 18.9 MB written; algorithmic 100.7 MB read + 33.6 MB written: "
+    ("c5", "attention"): {"bytes_per_launch": 144.7e6, "source": "profiles/launch_list_c5_stack.md: same capture, 92 launches of "
+                          "attn_int8_pipe_kernel (128.0 MB read + 16.7 MB written; algorithmic 100.7 MB read + 33.6 MB written: "
                           "K and V of a head are read again by each of its four query tiles, not always from L2)"},
     ("c3", "gemm_pair_kernel<int8, no activation>"): {"bytes_per_launch": 28.1e6, "source": "profiles/dram_traffic_c3_layer.md: ncu capture "
                           "of the three launches (QKV 15.8 MB, attention output 13.7 MB, FC2 54.8 MB), recorded with an earlier build of "
