@@ -964,21 +964,24 @@ __device__ __forceinline__ void copy_chunk(uint8_t* dst, const char* src) {
 
 // Ring depth of ln_wide_kernel: two CTAs per SM; deep enough that about 128 KB per SM are always on their way,
 // within 100 KB per CTA (ring + staged vectors).
-__host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes, int wpr) {
+__host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes, int wpr, int minb = 2) {
   // (rows of 8192 elements, one per stage, want one stage more: 317 against 334 us on 65536 x 8192 FP16 -> INT8)
-  int stages = 1 + ((wpr == 8 ? 80 : 64) * 1024 + stage_bytes - 1) / stage_bytes;
+  int stages = 1 + ((wpr == 8 ? 80 : 64) * 2 / minb * 1024 + stage_bytes - 1) / stage_bytes;
   if (stages < 3) stages = 3;
   if (stages > 8) stages = 8;
-  while (stages > 3 && stages * stage_bytes + vec_bytes > 100 * 1024) --stages;
+  while (stages > 3 && stages * stage_bytes + vec_bytes > 200 / minb * 1024) --stages;
   return stages;
 }
 
-// GEO 0: a lane owns two chunks of 16 elements (H = 1024 * WPR); GEO 1: three chunks of 8 (H = 768 * WPR).
+// GEO 0: a lane owns two chunks of 16 elements (H = 1024 * WPR); GEO 1: three chunks of 8 (H = 768 * WPR); GEO 3: as GEO 0
+// with gamma / beta read from shared memory instead of held in registers (79 registers instead of 124: three CTAs per SM).
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
-__global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
+__global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(const LnParams p) {
   ptx::pdl_launch_dependents();
-  constexpr int CE = GEO == 0 ? 16 : 8;            // elements per chunk
-  constexpr int CPL = GEO == 0 ? 2 : 3;            // chunks per lane
+  constexpr int CE = GEO == 1 ? 8 : 16;            // elements per chunk
+  constexpr int CPL = GEO == 1 ? 3 : 2;            // chunks per lane
+  constexpr bool GBS = GEO == 3;                   // gamma / beta staged in shared memory (fewer registers: three CTAs per SM)
+  constexpr int MINB = GEO == 3 ? 3 : 2;
   constexpr int NP = CE / 2;                       // float pairs per chunk
   constexpr int H = CE * 32 * CPL * WPR;
   constexpr int SLOTS = 8 / WPR;                   // rows per CTA pass
@@ -991,14 +994,16 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   constexpr bool RES_CS = RES == SRC_I8 && RSC == RS_COL;
   constexpr bool BR_CS = BR == SRC_I8;
   constexpr bool OUT_CS = OUT == O_STATIC;
-  constexpr int VEC_BYTES = H * 4 * ((RES_CS ? 1 : 0) + (BR_CS ? 1 : 0) + (OUT_CS ? 1 : 0));
-  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES, WPR);   // ring depth
+  constexpr int VEC_BYTES = H * 4 * ((RES_CS ? 1 : 0) + (BR_CS ? 1 : 0) + (OUT_CS ? 1 : 0) + (GBS ? 2 : 0));
+  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES, WPR, MINB);   // ring depth
   __shared__ float red[3][8][8];                   // [statistic][row slot][warp in row]
   extern __shared__ __align__(16) uint8_t dyn[];
   float* v_rcs = reinterpret_cast<float*>(dyn);
   float* v_bcs = v_rcs + (RES_CS ? H : 0);
   float* v_ocs = v_bcs + (BR_CS ? H : 0);
-  uint8_t* ring = reinterpret_cast<uint8_t*>(v_ocs + (OUT_CS ? H : 0));
+  float* v_gam = v_ocs + (OUT_CS ? H : 0);
+  float* v_bet = v_gam + (GBS ? H : 0);
+  uint8_t* ring = reinterpret_cast<uint8_t*>(v_bet + (GBS ? H : 0));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int slot = warp / WPR, wr = warp % WPR;
   const int c_first = wr * 32 + lane;              // this lane's first chunk (16-element units)
@@ -1039,9 +1044,10 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     if constexpr (RES_CS) v_rcs[si] = __ldg(p.res.col_scale + i * p.res.col_stride);
     if constexpr (BR_CS) v_bcs[si] = __ldg(p.br.col_scale + i * p.br.col_stride);
     if constexpr (OUT_CS) v_ocs[si] = 1.0f / __ldg(p.out_scale + (p.out_gran == HERO_GRAN_FWQ ? i : 0));   // reciprocal, see the output stage
+    if constexpr (GBS && OUT != O_NONE) { v_gam[si] = __ldg(p.gamma + i); v_bet[si] = __ldg(p.beta + i); }
   }
-  float2 gam[CPL][NP], bet[CPL][NP];
-  if constexpr (OUT != O_NONE) {
+  float2 gam[GBS ? 1 : CPL][NP], bet[GBS ? 1 : CPL][NP];
+  if constexpr (OUT != O_NONE && !GBS) {
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
       const int e0 = (c_first + k * STRIDE) * CE;
@@ -1177,9 +1183,13 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     const float2 r2 = f2(rstd);
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
+      if constexpr (GBS) {
+        lds_vec<H / CE, CE>(v_gam + (c_first + k * STRIDE) * 4, gam[0]);
+        lds_vec<H / CE, CE>(v_bet + (c_first + k * STRIDE) * 4, bet[0]);
+      }
 #pragma unroll
       for (int i = 0; i < NP; ++i) {
-        x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(gam[k][i], r2), bet[k][i]);
+        x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(gam[GBS ? 0 : k][i], r2), bet[GBS ? 0 : k][i]);
         if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fmaxf(fabsf(x[k][i].x), fabsf(x[k][i].y)));
       }
     }
@@ -1262,11 +1272,11 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
 static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream) {
-  constexpr int H = (GEO == 0 ? 1024 : 768) * WPR, SLOTS = 8 / WPR;
+  constexpr int H = (GEO == 1 ? 768 : 1024) * WPR, SLOTS = 8 / WPR;
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2, ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
   constexpr size_t STAGE = (size_t)SLOTS * H * (ES_RES + ES_BR);
-  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0));
-  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR);
+  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0) + (GEO == 3 ? 2 : 0));
+  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR, GEO == 3 ? 3 : 2);
   const size_t smem = (size_t)stages * STAGE + VEC;
   auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8, GEO>;
   HERO_SMEM_OPT_IN(h, kern, 200 * 1024);
@@ -1292,7 +1302,9 @@ template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, bool F8>
 static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) {
   switch (p.H) {
     case 768: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 1>(h, p, s);
-    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 0>(h, p, s);
+    // 8-bit residual: gamma / beta from shared memory, three CTAs per SM (3 - 7 % faster); FP residual: the lighter
+    // loop gains nothing from the extra warps and loses the loads (4 % slower), so gamma / beta stay in registers
+    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, RES == SRC_I8 ? 3 : 0>(h, p, s);
     case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2, F8, 0>(h, p, s);
     case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4, F8, 0>(h, p, s);
     default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8, F8, 0>(h, p, s);
