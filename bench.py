@@ -698,7 +698,9 @@ def run_ours(args):
             "cpu_baseline": cpu, "fp16_path": fp_path, "wall_s_timed_region": wall}
     if layers_only_ms is not None:
         line["without_entry_ln"] = {"ms_per_step": layers_only_ms, "value": shape.M / (layers_only_ms * 1e-3), "unit": UNIT,
-                                    "note": "the layers alone, their INT8 input already in place (one rank's device time)"}
+                                    "note": "the layers alone, their INT8 input already in place (one rank's device time); timed after the main "
+                                            "region, i.e. later under the power cap: compare it with a step time from the same phase, "
+                                            "not with ms_per_step"}
     if host_us is not None:
         line["host_us_per_step"] = {"value": host_us, "launches": launches_per_step,
                                     "note": "wall clock of the C-ABI call itself (argument checks, tensor-map lookup, launches), "
