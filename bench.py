@@ -528,6 +528,7 @@ def run_ours(args):
     value = replicas.job_throughput(shape.M, args.steps, world, total_ms * 1e-3)
     # the same steps without the entry LN^quant (the layers alone, their INT8 input already in place)
     layers_only_ms = timed(step_layers_only, args.steps) / args.steps if post else None
+    full_again_ms = timed(step, args.steps) / args.steps if post else None      # the whole step once more, same phase
     # host time of the C-ABI call: a burst of calls short enough to stay inside the driver's launch queue, so the host
     # never waits for the device; wall clock until the last call has returned
     host_us = None
@@ -698,9 +699,10 @@ def run_ours(args):
             "cpu_baseline": cpu, "fp16_path": fp_path, "wall_s_timed_region": wall}
     if layers_only_ms is not None:
         line["without_entry_ln"] = {"ms_per_step": layers_only_ms, "value": shape.M / (layers_only_ms * 1e-3), "unit": UNIT,
+                                    "whole_step_same_phase_ms": full_again_ms,
                                     "note": "the layers alone, their INT8 input already in place (one rank's device time); timed after the main "
-                                            "region, i.e. later under the power cap: compare it with a step time from the same phase, "
-                                            "not with ms_per_step"}
+                                            "region, i.e. later under the power cap: compare it with whole_step_same_phase_ms, the "
+                                            "whole step timed right after it, not with ms_per_step"}
     if host_us is not None:
         line["host_us_per_step"] = {"value": host_us, "launches": launches_per_step,
                                     "note": "wall clock of the C-ABI call itself (argument checks, tensor-map lookup, launches), "
