@@ -5,6 +5,7 @@ stream is torch's current CUDA stream unless one is passed.
 """
 import ctypes as C
 import os
+import sys
 
 import torch
 
@@ -127,6 +128,13 @@ def lib():
         if not os.path.exists(_LIB_PATH):
             raise RuntimeError("libhero.so is not built (%s); run `python -m paper_2310_17723_b200.build`. "
                                "There is no fallback path." % _LIB_PATH)
+        try:                                     # a library older than its sources is loaded all the same, but said
+            from . import build as _build
+            if os.path.exists(_build.STAMP) and open(_build.STAMP).read().strip() != _build._digest():
+                sys.stderr.write("hero: libhero.so was built from other sources than those in csrc/ now; "
+                                 "run `python -m paper_2310_17723_b200.build`\n")
+        except OSError:
+            pass
         L = C.CDLL(_LIB_PATH)
         L.hero_last_error.restype = C.c_char_p
         L.hero_launch_count.restype = C.c_int64
