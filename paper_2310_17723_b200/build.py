@@ -29,7 +29,7 @@ def _digest():
     files = sources() + sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h")))
     files.append(os.path.join(INCLUDE, "hero.h"))
     for f in files:
-        h.update(f.encode())
+        h.update(os.path.basename(f).encode())     # (not the path: the same tree must hash alike wherever it is mounted)
         with open(f, "rb") as fh:
             h.update(fh.read())
     h.update((" ".join(NVCC_FLAGS) + os.environ.get("HERO_NVCC_EXTRA", "")).encode())
