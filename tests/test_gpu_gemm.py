@@ -49,6 +49,28 @@ def test_int32_accumulators_bit_exact(h, M, K, N):
     assert np.array_equal(got, want)
 
 
+def test_many_distinct_buffers_then_the_first_again(h):
+    # more distinct operand / output buffers than the handle keeps tensor maps for: every call must describe ITS buffers
+    # (a stale or colliding descriptor would read or write another tensor), and coming back to the first buffers, whose
+    # maps have been displaced meanwhile, must give the first result again
+    g = W.rng(2, 4242)
+    M, K, N = 160, 192, 320
+    As = [dev(g.integers(-127, 128, (M, K), dtype=np.int8)) for _ in range(150)]
+    Wt = g.integers(-127, 128, (N, K), dtype=np.int8)
+    tW = dev(Wt)
+    outs = [torch.full((M, N), -77, dtype=torch.int32, device="cuda") for _ in range(len(As))]
+    for a, o in zip(As, outs):
+        h.hero_w8a8_linear(hero.tensor(a), tW, hero.tensor(o))
+    again = torch.full((M, N), -77, dtype=torch.int32, device="cuda")
+    h.hero_w8a8_linear(hero.tensor(As[0]), tW, hero.tensor(again))
+    h.check()
+    Wf = tW.double().T
+    for i in (0, 1, 63, 127, 128, 149):
+        want = (As[i].double() @ Wf).to(torch.int32)                 # exact: |sum| < 2^53
+        assert torch.equal(outs[i], want), i
+    assert torch.equal(again, outs[0])
+
+
 def test_int32_extreme_values_bit_exact(h):
     M, K, N = 130, 16384, 64
     A = np.full((M, K), 127, np.int8)
