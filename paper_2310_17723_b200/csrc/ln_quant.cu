@@ -964,28 +964,47 @@ __device__ __forceinline__ void copy_chunk(uint8_t* dst, const char* src) {
 
 // Ring depth of ln_wide_kernel: two CTAs per SM; deep enough that about 128 KB per SM are always on their way,
 // within 100 KB per CTA (ring + staged vectors).
-__host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes, int wpr, int minb = 2) {
+__host__ __device__ constexpr int ln_wide_stages(int stage_bytes, int vec_bytes, int wpr, int minb = 2, int least = 3) {
   // (rows of 8192 elements, one per stage, want one stage more: 317 against 334 us on 65536 x 8192 FP16 -> INT8)
   int stages = 1 + ((wpr == 8 ? 80 : 64) * 2 / minb * 1024 + stage_bytes - 1) / stage_bytes;
-  if (stages < 3) stages = 3;
+  if (stages < least) stages = least;
   if (stages > 8) stages = 8;
-  while (stages > 3 && stages * stage_bytes + vec_bytes > 200 / minb * 1024) --stages;
+  while (stages > least && stages * stage_bytes + vec_bytes > 200 / minb * 1024) --stages;
   return stages;
 }
+// sums / maxima over the LPR consecutive lanes that share a row (32: the warp; 16: a half-warp)
+template <int LPR> __device__ __forceinline__ float lanes_sum(float v) {
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+template <int LPR> __device__ __forceinline__ float lanes_max(float v) {
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
 
-// GEO 0: a lane owns two chunks of 16 elements (H = 1024 * WPR); GEO 1: three chunks of 8 (H = 768 * WPR); GEO 3: as GEO 0
-// with gamma / beta read from shared memory instead of held in registers (79 registers instead of 124: three CTAs per SM).
+// GEO 0: rows of 1024 * WPR elements, WPR >= 2 warps per row, a lane owns two chunks of 16 elements, gamma / beta in
+// registers.  GEO 5 / 6: rows of 1024 / 768 elements, TWO rows per warp: 16 lanes per row, four / three chunks of 16 per
+// lane, gamma / beta read from shared memory like the scale vectors.  The two halves of a warp then read the same
+// per-column vectors (one broadcast wavefront instead of two) and the row reductions take four shuffle steps for two
+// rows at once: the kernel was bound by the shared-memory pipe (80 % busy, two thirds of its wavefronts the FP32
+// per-column vectors), not by DRAM.
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
-__global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(const LnParams p) {
+__global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
   ptx::pdl_launch_dependents();
-  constexpr int CE = GEO == 1 ? 8 : 16;            // elements per chunk
-  constexpr int CPL = GEO == 1 ? 3 : 2;            // chunks per lane
-  constexpr bool GBS = GEO == 3;                   // gamma / beta staged in shared memory (fewer registers: three CTAs per SM)
-  constexpr int MINB = GEO == 3 ? 3 : 2;
+  constexpr bool HALF = GEO >= 5;                  // two rows per warp, 16 lanes each (WPR = 1); GEO 6: rows of 768
+  static_assert(!HALF || WPR == 1, "half-warp rows are for rows of one warp's width");
+  constexpr int LPR = HALF ? 16 : 32;              // lanes that share a row
+  static_assert(GEO == 0 || GEO == 5 || GEO == 6, "unknown row geometry");
+  constexpr int CE = 16;                           // elements per chunk
+  constexpr int CPL = GEO == 6 ? 3 : (HALF ? 4 : 2);   // chunks per lane
+  constexpr bool GBS = HALF;                       // gamma / beta staged in shared memory
+  constexpr int MINB = 2;
   constexpr int NP = CE / 2;                       // float pairs per chunk
-  constexpr int H = CE * 32 * CPL * WPR;
-  constexpr int SLOTS = 8 / WPR;                   // rows per CTA pass
-  constexpr int STRIDE = WPR * 32;                 // chunk stride between a lane's chunks
+  constexpr int H = CE * LPR * CPL * WPR;
+  constexpr int SLOTS = HALF ? 16 : 8 / WPR;       // rows per CTA pass
+  constexpr int STRIDE = WPR * LPR;                // chunk stride between a lane's chunks
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2;
   constexpr int ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
   constexpr int OFF_BR = H * ES_RES;
@@ -995,7 +1014,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
   constexpr bool BR_CS = BR == SRC_I8;
   constexpr bool OUT_CS = OUT == O_STATIC;
   constexpr int VEC_BYTES = H * 4 * ((RES_CS ? 1 : 0) + (BR_CS ? 1 : 0) + (OUT_CS ? 1 : 0) + (GBS ? 2 : 0));
-  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES, WPR, MINB);   // ring depth
+  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES, WPR, MINB, HALF ? 2 : 3);   // ring depth
   __shared__ float red[3][8][8];                   // [statistic][row slot][warp in row]
   extern __shared__ __align__(16) uint8_t dyn[];
   float* v_rcs = reinterpret_cast<float*>(dyn);
@@ -1005,8 +1024,9 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
   float* v_bet = v_gam + (GBS ? H : 0);
   uint8_t* ring = reinterpret_cast<uint8_t*>(v_bet + (GBS ? H : 0));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int slot = warp / WPR, wr = warp % WPR;
-  const int c_first = wr * 32 + lane;              // this lane's first chunk (16-element units)
+  const int slot = HALF ? warp * 2 + (lane >> 4) : warp / WPR, wr = HALF ? 0 : warp % WPR;
+  const int hl = lane & (LPR - 1);                 // this lane's position among the lanes of its row
+  const int c_first = wr * 32 + hl;                // this lane's first chunk (16-element units)
   const float MAGIC = 12582912.0f;                 // 1.5 * 2^23
   constexpr float fH = (float)H;
 
@@ -1072,15 +1092,18 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
   constexpr bool ROW_SC = RES == SRC_I8 && RSC == RS_ROW;
   float rs_ring = 1.f;
   if constexpr (ROW_SC) {
-    const long long r = first + (long long)lane * row_step;
-    if (lane < STAGES - 1 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+    const long long r = first + (long long)hl * row_step;
+    if (hl < STAGES - 1 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
   }
 
   __syncthreads();
 
   int st = 0;
   // every slot walks its own rows: nothing in the loop is shared between slots (named barriers are per slot)
-  for (long long row = first; row < p.M; row += row_step) {
+  // (half-warp rows: the warp's two rows are consecutive, so the loop runs while the lower one exists and the upper half
+  // computes on stale ring contents, stores nothing, on the last pass of an odd tail; shuffles never cross the halves)
+  for (long long row = first; row - (HALF ? (lane >> 4) : 0) < p.M; row += row_step) {
+    const bool row_in = !HALF || row < p.M;
     {
       int pst = st + STAGES - 1;
       if (pst >= STAGES) pst -= STAGES;
@@ -1089,10 +1112,10 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
     float rs_res = 1.f;
     if constexpr (ROW_SC) {
       // this row's scale sits in lane 0; shift the ring by one lane and let lane STAGES - 2 fetch the newest row's
-      rs_res = __shfl_sync(0xffffffffu, rs_ring, 0);
-      rs_ring = __shfl_down_sync(0xffffffffu, rs_ring, 1);
+      rs_res = __shfl_sync(0xffffffffu, rs_ring, 0, LPR);
+      rs_ring = __shfl_down_sync(0xffffffffu, rs_ring, 1, LPR);
       const long long r = row + (long long)(STAGES - 1) * row_step;
-      if (lane == STAGES - 2 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+      if (hl == STAGES - 2 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
     }
     cp_async_wait<STAGES - 1>();                   // this row's copies are the oldest group still pending
     const uint8_t* src = my_ring + st * STAGE_BYTES;
@@ -1140,7 +1163,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
           char* dst = reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + (c_first + k * STRIDE) * CE) * 2;
 #pragma unroll
           for (int j = 0; j < CE / 8; ++j) {
-            st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            if (row_in) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
             fpx8_to_f2<BF>(make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]), x[k] + 4 * j);
           }
         }
@@ -1151,7 +1174,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
     if constexpr (OUT == O_NONE) continue;
 
     // ---- mean (true division: a constant row must give exactly zero deviations)
-    float s = warp_sum(s2.x + s2.y);
+    float s = lanes_sum<LPR>(s2.x + s2.y);
     if constexpr (WPR > 1) {
       if (lane == 0) red[0][slot][wr] = s;
       asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
@@ -1168,7 +1191,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
 #pragma unroll
       for (int i = 0; i < NP; ++i) { x[k][i] = __fadd2_rn(x[k][i], nm); q2 = __ffma2_rn(x[k][i], x[k][i], q2); }
     }
-    float q = warp_sum(q2.x + q2.y);
+    float q = lanes_sum<LPR>(q2.x + q2.y);
     if constexpr (WPR > 1) {
       if (lane == 0) red[1][slot][wr] = q;
       asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
@@ -1197,7 +1220,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
     if constexpr (OUT == O_TWQ) {
       // Eq. 3: S[i] = absmax / 127 on the fly; the scaled value never leaves [-127, 127], so the magic add
       // alone rounds and range-limits it
-      amax = warp_max(amax);
+      amax = lanes_max<LPR>(amax);
       if constexpr (WPR > 1) {
         if (lane == 0) red[2][slot][wr] = amax;
         asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
@@ -1207,7 +1230,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
       }
       const float sc = amax > 0.f ? amax * (F8 ? 1.0f / 448.0f : 1.0f / 127.0f) : 1.0f;   // within 1 ulp of the quotient
       const float2 inv2 = f2(__fdividef(1.0f, sc)), mg2 = f2(MAGIC);
-      if (wr == 0 && lane == 0) p.out_scale[row] = sc;
+      if (wr == 0 && hl == 0 && row_in) p.out_scale[row] = sc;
       {
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
@@ -1223,8 +1246,10 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
             }
           }
           char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
-          if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
-          else st_global8(dst, w[0], w[1]);
+          if (row_in) {
+            if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
+            else st_global8(dst, w[0], w[1]);
+          }
         }
       }
     } else if constexpr (OUT == O_STATIC) {
@@ -1249,8 +1274,10 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
             }
           }
           char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
-          if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
-          else st_global8(dst, w[0], w[1]);
+          if (row_in) {
+            if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
+            else st_global8(dst, w[0], w[1]);
+          }
         }
       }
     } else {
@@ -1262,7 +1289,7 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
           for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
           char* dst = reinterpret_cast<char*>(p.out) + (row * p.out_ld + (c_first + k * STRIDE) * CE) * 2;
 #pragma unroll
-          for (int j = 0; j < CE / 8; ++j) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+          for (int j = 0; j < CE / 8; ++j) if (row_in) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         }
       }
     }
@@ -1272,11 +1299,11 @@ __global__ void __launch_bounds__(LNF_THREADS, GEO == 3 ? 3 : 2) ln_wide_kernel(
 
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
 static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream) {
-  constexpr int H = (GEO == 1 ? 768 : 1024) * WPR, SLOTS = 8 / WPR;
+  constexpr int H = (GEO == 6 ? 768 : 1024) * WPR, SLOTS = GEO >= 5 ? 16 : 8 / WPR;
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2, ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
   constexpr size_t STAGE = (size_t)SLOTS * H * (ES_RES + ES_BR);
-  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0) + (GEO == 3 ? 2 : 0));
-  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR, GEO == 3 ? 3 : 2);
+  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0) + (GEO >= 5 ? 2 : 0));
+  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR, 2, GEO >= 5 ? 2 : 3);
   const size_t smem = (size_t)stages * STAGE + VEC;
   auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8, GEO>;
   HERO_SMEM_OPT_IN(h, kern, 200 * 1024);
@@ -1301,10 +1328,8 @@ static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream)
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, bool F8>
 static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) {
   switch (p.H) {
-    case 768: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 1>(h, p, s);
-    // 8-bit residual: gamma / beta from shared memory, three CTAs per SM (3 - 7 % faster); FP residual: the lighter
-    // loop gains nothing from the extra warps and loses the loads (4 % slower), so gamma / beta stay in registers
-    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, RES == SRC_I8 ? 3 : 0>(h, p, s);
+    case 768: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 6>(h, p, s);
+    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 5>(h, p, s);
     case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2, F8, 0>(h, p, s);
     case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4, F8, 0>(h, p, s);
     default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8, F8, 0>(h, p, s);
