@@ -985,25 +985,29 @@ template <int LPR> __device__ __forceinline__ float lanes_max(float v) {
 }
 
 // GEO 0: rows of 1024 * WPR elements, WPR >= 2 warps per row, a lane owns two chunks of 16 elements, gamma / beta in
-// registers.  GEO 5 / 6: rows of 1024 / 768 elements, TWO rows per warp: 16 lanes per row, four / three chunks of 16 per
-// lane, gamma / beta read from shared memory like the scale vectors.  The two halves of a warp then read the same
-// per-column vectors (one broadcast wavefront instead of two) and the row reductions take four shuffle steps for two
-// rows at once: the kernel was bound by the shared-memory pipe (80 % busy, two thirds of its wavefronts the FP32
-// per-column vectors), not by DRAM.
+// registers.  Rows of one warp's width are processed two per warp, gamma / beta read from shared memory like the scale
+// vectors (the kernel with one row per warp was bound by the shared-memory pipe, 80 % busy, two thirds of its wavefronts
+// the FP32 per-column vectors, and by its per-row chain):
+// GEO 7: rows of 1024: every lane holds its two chunks of BOTH rows, so a per-column vector is read once for two rows;
+// GEO 6: rows of 768: 16 lanes per row, three chunks of 16 per lane (16-byte copies; 32 lanes would need 8-byte ones), the
+//        row reductions take four shuffle steps for two rows at once.
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
 __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams p) {
   ptx::pdl_launch_dependents();
-  constexpr bool HALF = GEO >= 5;                  // two rows per warp, 16 lanes each (WPR = 1); GEO 6: rows of 768
+  constexpr bool HALF = GEO == 6;                  // two rows per warp, 16 lanes each (WPR = 1): rows of 768
+  constexpr bool DUAL = GEO == 7;                  // two rows per warp, every lane holds its columns of both (WPR = 1)
+  constexpr int RPL = DUAL ? 2 : 1;                // rows per lane
   static_assert(!HALF || WPR == 1, "half-warp rows are for rows of one warp's width");
   constexpr int LPR = HALF ? 16 : 32;              // lanes that share a row
-  static_assert(GEO == 0 || GEO == 5 || GEO == 6, "unknown row geometry");
+  static_assert(GEO == 0 || GEO == 6 || GEO == 7, "unknown row geometry");
+  static_assert(!DUAL || WPR == 1, "two rows per lane are for rows of one warp's width");
   constexpr int CE = 16;                           // elements per chunk
-  constexpr int CPL = GEO == 6 ? 3 : (HALF ? 4 : 2);   // chunks per lane
-  constexpr bool GBS = HALF;                       // gamma / beta staged in shared memory
+  constexpr int CPL = HALF ? 3 : 2;                // chunks per lane
+  constexpr bool GBS = HALF || DUAL;               // gamma / beta staged in shared memory
   constexpr int MINB = 2;
   constexpr int NP = CE / 2;                       // float pairs per chunk
   constexpr int H = CE * LPR * CPL * WPR;
-  constexpr int SLOTS = HALF ? 16 : 8 / WPR;       // rows per CTA pass
+  constexpr int SLOTS = HALF || DUAL ? 16 : 8 / WPR;   // rows per CTA pass
   constexpr int STRIDE = WPR * LPR;                // chunk stride between a lane's chunks
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2;
   constexpr int ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
@@ -1014,7 +1018,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   constexpr bool BR_CS = BR == SRC_I8;
   constexpr bool OUT_CS = OUT == O_STATIC;
   constexpr int VEC_BYTES = H * 4 * ((RES_CS ? 1 : 0) + (BR_CS ? 1 : 0) + (OUT_CS ? 1 : 0) + (GBS ? 2 : 0));
-  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES, WPR, MINB, HALF ? 2 : 3);   // ring depth
+  constexpr int STAGES = ln_wide_stages(STAGE_BYTES, VEC_BYTES, WPR, MINB, HALF || DUAL ? 2 : 3);   // ring depth
   __shared__ float red[3][8][8];                   // [statistic][row slot][warp in row]
   extern __shared__ __align__(16) uint8_t dyn[];
   float* v_rcs = reinterpret_cast<float*>(dyn);
@@ -1024,7 +1028,7 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   float* v_bet = v_gam + (GBS ? H : 0);
   uint8_t* ring = reinterpret_cast<uint8_t*>(v_bet + (GBS ? H : 0));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int slot = HALF ? warp * 2 + (lane >> 4) : warp / WPR, wr = HALF ? 0 : warp % WPR;
+  const int slot = HALF ? warp * 2 + (lane >> 4) : (DUAL ? warp * 2 : warp / WPR), wr = HALF || DUAL ? 0 : warp % WPR;
   const int hl = lane & (LPR - 1);                 // this lane's position among the lanes of its row
   const int c_first = wr * 32 + hl;                // this lane's first chunk (16-element units)
   const float MAGIC = 12582912.0f;                 // 1.5 * 2^23
@@ -1038,17 +1042,21 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 
   // A lane copies exactly the chunks it will later read, so waiting on its own copy groups is all the
   // synchronisation the ring needs.
-  auto prefetch = [&](long long row, int st) {
-    if (row < p.M) {                               // rows past the end still commit an (empty) group
-      const char* gr = g_res + row * pitch_res;
-      uint8_t* d = my_ring + st * STAGE_BYTES;
+  auto prefetch = [&](long long row0, int st) {
 #pragma unroll
-      for (int k = 0; k < CPL; ++k) copy_chunk<CE * ES_RES>(d + k * STRIDE * CE * ES_RES, gr + k * STRIDE * CE * ES_RES);
-      if constexpr (BR != SRC_NONE) {
-        const char* gb = g_br + row * pitch_br;
-        uint8_t* db = my_ring_br + st * STAGE_BYTES;
+    for (int u = 0; u < RPL; ++u) {
+      const long long row = row0 + u;              // (two rows per lane: consecutive rows, consecutive ring slots)
+      if (row < p.M) {                             // rows past the end still commit an (empty) group
+        const char* gr = g_res + row * pitch_res;
+        uint8_t* d = my_ring + st * STAGE_BYTES + u * SLOT_BYTES;
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) copy_chunk<CE * ES_BR>(db + k * STRIDE * CE * ES_BR, gb + k * STRIDE * CE * ES_BR);
+        for (int k = 0; k < CPL; ++k) copy_chunk<CE * ES_RES>(d + k * STRIDE * CE * ES_RES, gr + k * STRIDE * CE * ES_RES);
+        if constexpr (BR != SRC_NONE) {
+          const char* gb = g_br + row * pitch_br;
+          uint8_t* db = my_ring_br + st * STAGE_BYTES + u * SLOT_BYTES;
+#pragma unroll
+          for (int k = 0; k < CPL; ++k) copy_chunk<CE * ES_BR>(db + k * STRIDE * CE * ES_BR, gb + k * STRIDE * CE * ES_BR);
+        }
       }
     }
     cp_async_commit();
@@ -1090,10 +1098,14 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   // the per-row scale of a TWQ residual travels STAGES - 1 rows ahead as well, in a register ring: lane i of a warp
   // holds the scale of the i-th row ahead (STAGES <= 8 < 32)
   constexpr bool ROW_SC = RES == SRC_I8 && RSC == RS_ROW;
-  float rs_ring = 1.f;
-  if constexpr (ROW_SC) {
-    const long long r = first + (long long)hl * row_step;
-    if (hl < STAGES - 1 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+  float rs_ring[RPL];
+#pragma unroll
+  for (int u = 0; u < RPL; ++u) {
+    rs_ring[u] = 1.f;
+    if constexpr (ROW_SC) {
+      const long long r = first + u + (long long)hl * row_step;
+      if (hl < STAGES - 1 && r < p.M) rs_ring[u] = __ldg(p.res.row_scale + r);
+    }
   }
 
   __syncthreads();
@@ -1102,20 +1114,27 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
   // every slot walks its own rows: nothing in the loop is shared between slots (named barriers are per slot)
   // (half-warp rows: the warp's two rows are consecutive, so the loop runs while the lower one exists and the upper half
   // computes on stale ring contents, stores nothing, on the last pass of an odd tail; shuffles never cross the halves)
+  // (two rows per lane: a lane holds its columns of the warp's two rows, so every per-column vector is read once for both)
   for (long long row = first; row - (HALF ? (lane >> 4) : 0) < p.M; row += row_step) {
-    const bool row_in = !HALF || row < p.M;
+    bool row_in[RPL];
+#pragma unroll
+    for (int u = 0; u < RPL; ++u) row_in[u] = !(HALF || DUAL) || row + u < p.M;
     {
       int pst = st + STAGES - 1;
       if (pst >= STAGES) pst -= STAGES;
       prefetch(row + (long long)(STAGES - 1) * row_step, pst);
     }
-    float rs_res = 1.f;
-    if constexpr (ROW_SC) {
-      // this row's scale sits in lane 0; shift the ring by one lane and let lane STAGES - 2 fetch the newest row's
-      rs_res = __shfl_sync(0xffffffffu, rs_ring, 0, LPR);
-      rs_ring = __shfl_down_sync(0xffffffffu, rs_ring, 1, LPR);
-      const long long r = row + (long long)(STAGES - 1) * row_step;
-      if (hl == STAGES - 2 && r < p.M) rs_ring = __ldg(p.res.row_scale + r);
+    float rs_res[RPL];
+#pragma unroll
+    for (int u = 0; u < RPL; ++u) {
+      rs_res[u] = 1.f;
+      if constexpr (ROW_SC) {
+        // this row's scale sits in lane 0; shift the ring by one lane and let lane STAGES - 2 fetch the newest row's
+        rs_res[u] = __shfl_sync(0xffffffffu, rs_ring[u], 0, LPR);
+        rs_ring[u] = __shfl_down_sync(0xffffffffu, rs_ring[u], 1, LPR);
+        const long long r = row + u + (long long)(STAGES - 1) * row_step;
+        if (hl == STAGES - 2 && r < p.M) rs_ring[u] = __ldg(p.res.row_scale + r);
+      }
     }
     cp_async_wait<STAGES - 1>();                   // this row's copies are the oldest group still pending
     const uint8_t* src = my_ring + st * STAGE_BYTES;
@@ -1123,87 +1142,94 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
     if (++st == STAGES) st = 0;
 
     // ---- r = sum of the dequantized addends; running row sum
-    float2 x[CPL][NP];
-    float2 s2 = f2(0.f);
+    float2 x[RPL][CPL][NP];
+    float2 s2[RPL];
+#pragma unroll
+    for (int u = 0; u < RPL; ++u) s2[u] = f2(0.f);
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
-      {
-        if constexpr (RES == SRC_I8) {
-          ring_q8<CE, F8>(src + k * STRIDE * CE, x[k]);
-          if constexpr (RSC == RS_COL) {
-            float2 sc[NP];
-            lds_vec<H / CE, CE>(v_rcs + (c_first + k * STRIDE) * 4, sc);
+      float2 rcs[RES_CS ? NP : 1], bcs[BR_CS ? NP : 1];
+      if constexpr (RES_CS) lds_vec<H / CE, CE>(v_rcs + (c_first + k * STRIDE) * 4, rcs);
+      if constexpr (BR_CS) lds_vec<H / CE, CE>(v_bcs + (c_first + k * STRIDE) * 4, bcs);
 #pragma unroll
-            for (int i = 0; i < NP; ++i) x[k][i] = __fmul2_rn(x[k][i], sc[i]);
+      for (int u = 0; u < RPL; ++u) {
+        if constexpr (RES == SRC_I8) {
+          ring_q8<CE, F8>(src + u * SLOT_BYTES + k * STRIDE * CE, x[u][k]);
+          if constexpr (RSC == RS_COL) {
+#pragma unroll
+            for (int i = 0; i < NP; ++i) x[u][k][i] = __fmul2_rn(x[u][k][i], rcs[i]);
           } else {
 #pragma unroll
-            for (int i = 0; i < NP; ++i) x[k][i] = __fmul2_rn(x[k][i], f2(rs_res));
+            for (int i = 0; i < NP; ++i) x[u][k][i] = __fmul2_rn(x[u][k][i], f2(rs_res[u]));
           }
         } else {
-          ring_fp<CE, BF>(src + k * STRIDE * CE * 2, x[k]);
+          ring_fp<CE, BF>(src + u * SLOT_BYTES + k * STRIDE * CE * 2, x[u][k]);
         }
         if constexpr (BR == SRC_I8) {
-          float2 b[NP], sc[NP];
-          ring_q8<CE, F8>(src_br + k * STRIDE * CE, b);
-          lds_vec<H / CE, CE>(v_bcs + (c_first + k * STRIDE) * 4, sc);
+          float2 b[NP];
+          ring_q8<CE, F8>(src_br + u * SLOT_BYTES + k * STRIDE * CE, b);
 #pragma unroll
-          for (int i = 0; i < NP; ++i) x[k][i] = __ffma2_rn(b[i], sc[i], x[k][i]);
+          for (int i = 0; i < NP; ++i) x[u][k][i] = __ffma2_rn(b[i], bcs[i], x[u][k][i]);
         }
         if constexpr (BR == SRC_FP) {
           float2 b[NP];
-          ring_fp<CE, BF>(src_br + k * STRIDE * CE * 2, b);
+          ring_fp<CE, BF>(src_br + u * SLOT_BYTES + k * STRIDE * CE * 2, b);
 #pragma unroll
-          for (int i = 0; i < NP; ++i) x[k][i] = __fadd2_rn(x[k][i], b[i]);
+          for (int i = 0; i < NP; ++i) x[u][k][i] = __fadd2_rn(x[u][k][i], b[i]);
         }
         if constexpr (FPOUT) {
           // the FP residual stream carries the ROUNDED sum; normalise what is stored
           uint32_t w[NP];
 #pragma unroll
-          for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
-          char* dst = reinterpret_cast<char*>(p.fp_out) + (row * p.fp_ld + (c_first + k * STRIDE) * CE) * 2;
+          for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[u][k][i].x, x[u][k][i].y);
+          char* dst = reinterpret_cast<char*>(p.fp_out) + ((row + u) * p.fp_ld + (c_first + k * STRIDE) * CE) * 2;
 #pragma unroll
           for (int j = 0; j < CE / 8; ++j) {
-            if (row_in) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-            fpx8_to_f2<BF>(make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]), x[k] + 4 * j);
+            if (row_in[u]) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            fpx8_to_f2<BF>(make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]), x[u][k] + 4 * j);
           }
         }
 #pragma unroll
-        for (int i = 0; i < NP; ++i) s2 = __fadd2_rn(s2, x[k][i]);
+        for (int i = 0; i < NP; ++i) s2[u] = __fadd2_rn(s2[u], x[u][k][i]);
       }
     }
     if constexpr (OUT == O_NONE) continue;
 
-    // ---- mean (true division: a constant row must give exactly zero deviations)
-    float s = lanes_sum<LPR>(s2.x + s2.y);
-    if constexpr (WPR > 1) {
-      if (lane == 0) red[0][slot][wr] = s;
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
-      s = 0.f;
+    // ---- mean (true division: a constant row must give exactly zero deviations), then the centred (biased) variance
+    float rstd[RPL];
 #pragma unroll
-      for (int w = 0; w < WPR; ++w) s += red[0][slot][w];
+    for (int u = 0; u < RPL; ++u) {
+      float s = lanes_sum<LPR>(s2[u].x + s2[u].y);
+      if constexpr (WPR > 1) {
+        if (lane == 0) red[0][slot][wr] = s;
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
+        s = 0.f;
+#pragma unroll
+        for (int w = 0; w < WPR; ++w) s += red[0][slot][w];
+      }
+      const float mean = s / fH;
+      float2 q2 = f2(0.f);
+      const float2 nm = f2(-mean);
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) {
+#pragma unroll
+        for (int i = 0; i < NP; ++i) { x[u][k][i] = __fadd2_rn(x[u][k][i], nm); q2 = __ffma2_rn(x[u][k][i], x[u][k][i], q2); }
+      }
+      float q = lanes_sum<LPR>(q2.x + q2.y);
+      if constexpr (WPR > 1) {
+        if (lane == 0) red[1][slot][wr] = q;
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
+        q = 0.f;
+#pragma unroll
+        for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
+      }
+      rstd[u] = rsqrtf(q / fH + p.eps);            // 2 ulp: far below the rounding step of the output
     }
-    const float mean = s / fH;
-    // ---- centred (biased) variance over the registers
-    float2 q2 = f2(0.f);
-    const float2 nm = f2(-mean);
-#pragma unroll
-    for (int k = 0; k < CPL; ++k) {
-#pragma unroll
-      for (int i = 0; i < NP; ++i) { x[k][i] = __fadd2_rn(x[k][i], nm); q2 = __ffma2_rn(x[k][i], x[k][i], q2); }
-    }
-    float q = lanes_sum<LPR>(q2.x + q2.y);
-    if constexpr (WPR > 1) {
-      if (lane == 0) red[1][slot][wr] = q;
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
-      q = 0.f;
-#pragma unroll
-      for (int w = 0; w < WPR; ++w) q += red[1][slot][w];
-    }
-    const float rstd = rsqrtf(q / fH + p.eps);   // 2 ulp: far below the rounding step of the output
 
     // ---- y = d * (rstd * gamma) + beta ; TWQ: row absmax in the same sweep
-    float amax = 0.f;
-    const float2 r2 = f2(rstd);
+    float amax[RPL];
+#pragma unroll
+    for (int u = 0; u < RPL; ++u) amax[u] = 0.f;
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
       if constexpr (GBS) {
@@ -1211,42 +1237,47 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
         lds_vec<H / CE, CE>(v_bet + (c_first + k * STRIDE) * 4, bet[0]);
       }
 #pragma unroll
-      for (int i = 0; i < NP; ++i) {
-        x[k][i] = __ffma2_rn(x[k][i], __fmul2_rn(gam[GBS ? 0 : k][i], r2), bet[GBS ? 0 : k][i]);
-        if constexpr (OUT == O_TWQ) amax = fmaxf(amax, fmaxf(fabsf(x[k][i].x), fabsf(x[k][i].y)));
+      for (int u = 0; u < RPL; ++u) {
+        const float2 r2 = f2(rstd[u]);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+          x[u][k][i] = __ffma2_rn(x[u][k][i], __fmul2_rn(gam[GBS ? 0 : k][i], r2), bet[GBS ? 0 : k][i]);
+          if constexpr (OUT == O_TWQ) amax[u] = fmaxf(amax[u], fmaxf(fabsf(x[u][k][i].x), fabsf(x[u][k][i].y)));
+        }
       }
     }
 
     if constexpr (OUT == O_TWQ) {
       // Eq. 3: S[i] = absmax / 127 on the fly; the scaled value never leaves [-127, 127], so the magic add
       // alone rounds and range-limits it
-      amax = lanes_max<LPR>(amax);
-      if constexpr (WPR > 1) {
-        if (lane == 0) red[2][slot][wr] = amax;
-        asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
-        amax = 0.f;
 #pragma unroll
-        for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, red[2][slot][w]);
-      }
-      const float sc = amax > 0.f ? amax * (F8 ? 1.0f / 448.0f : 1.0f / 127.0f) : 1.0f;   // within 1 ulp of the quotient
-      const float2 inv2 = f2(__fdividef(1.0f, sc)), mg2 = f2(MAGIC);
-      if (wr == 0 && hl == 0 && row_in) p.out_scale[row] = sc;
-      {
+      for (int u = 0; u < RPL; ++u) {
+        float am = lanes_max<LPR>(amax[u]);
+        if constexpr (WPR > 1) {
+          if (lane == 0) red[2][slot][wr] = am;
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + slot), "n"(STRIDE) : "memory");
+          am = 0.f;
+#pragma unroll
+          for (int w = 0; w < WPR; ++w) am = fmaxf(am, red[2][slot][w]);
+        }
+        const float sc = am > 0.f ? am * (F8 ? 1.0f / 448.0f : 1.0f / 127.0f) : 1.0f;   // within 1 ulp of the quotient
+        const float2 inv2 = f2(__fdividef(1.0f, sc)), mg2 = f2(MAGIC);
+        if (wr == 0 && hl == 0 && row_in[u]) p.out_scale[row + u] = sc;
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
           uint32_t w[CE / 4];
 #pragma unroll
           for (int g = 0; g < CE / 4; ++g) {
             if constexpr (F8) {
-              const float2 a = __fmul2_rn(x[k][2 * g], inv2), b = __fmul2_rn(x[k][2 * g + 1], inv2);
+              const float2 a = __fmul2_rn(x[u][k][2 * g], inv2), b = __fmul2_rn(x[u][k][2 * g + 1], inv2);
               w[g] = ptx::f32x4_to_e4m3x4(a.x, a.y, b.x, b.y);
             } else {
-              const float2 a = __ffma2_rn(x[k][2 * g], inv2, mg2), b = __ffma2_rn(x[k][2 * g + 1], inv2, mg2);
+              const float2 a = __ffma2_rn(x[u][k][2 * g], inv2, mg2), b = __ffma2_rn(x[u][k][2 * g + 1], inv2, mg2);
               w[g] = pack_low_bytes(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(b.x), __float_as_uint(b.y));
             }
           }
-          char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
-          if (row_in) {
+          char* dst = reinterpret_cast<char*>(p.out) + (row + u) * p.out_ld + (c_first + k * STRIDE) * CE;
+          if (row_in[u]) {
             if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
             else st_global8(dst, w[0], w[1]);
           }
@@ -1261,22 +1292,25 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
         for (int k = 0; k < CPL; ++k) {
           float2 sc[NP];
           lds_vec<H / CE, CE>(v_ocs + (c_first + k * STRIDE) * 4, sc);
-          uint32_t w[CE / 4];
 #pragma unroll
-          for (int g = 0; g < CE / 4; ++g) {
-            const float2 a = __fmul2_rn(x[k][2 * g], sc[2 * g]), b = __fmul2_rn(x[k][2 * g + 1], sc[2 * g + 1]);
-            if constexpr (F8) {
-              w[g] = ptx::f32x4_to_e4m3x4(a.x, a.y, b.x, b.y);
-            } else {
-              const float a0 = fminf(fmaxf(a.x, lo2.x), hi2.x) + mg2.x, a1 = fminf(fmaxf(a.y, lo2.x), hi2.x) + mg2.x;
-              const float b0 = fminf(fmaxf(b.x, lo2.x), hi2.x) + mg2.x, b1 = fminf(fmaxf(b.y, lo2.x), hi2.x) + mg2.x;
-              w[g] = pack_low_bytes(__float_as_uint(a0), __float_as_uint(a1), __float_as_uint(b0), __float_as_uint(b1));
+          for (int u = 0; u < RPL; ++u) {
+            uint32_t w[CE / 4];
+#pragma unroll
+            for (int g = 0; g < CE / 4; ++g) {
+              const float2 a = __fmul2_rn(x[u][k][2 * g], sc[2 * g]), b = __fmul2_rn(x[u][k][2 * g + 1], sc[2 * g + 1]);
+              if constexpr (F8) {
+                w[g] = ptx::f32x4_to_e4m3x4(a.x, a.y, b.x, b.y);
+              } else {
+                const float a0 = fminf(fmaxf(a.x, lo2.x), hi2.x) + mg2.x, a1 = fminf(fmaxf(a.y, lo2.x), hi2.x) + mg2.x;
+                const float b0 = fminf(fmaxf(b.x, lo2.x), hi2.x) + mg2.x, b1 = fminf(fmaxf(b.y, lo2.x), hi2.x) + mg2.x;
+                w[g] = pack_low_bytes(__float_as_uint(a0), __float_as_uint(a1), __float_as_uint(b0), __float_as_uint(b1));
+              }
             }
-          }
-          char* dst = reinterpret_cast<char*>(p.out) + row * p.out_ld + (c_first + k * STRIDE) * CE;
-          if (row_in) {
-            if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
-            else st_global8(dst, w[0], w[1]);
+            char* dst = reinterpret_cast<char*>(p.out) + (row + u) * p.out_ld + (c_first + k * STRIDE) * CE;
+            if (row_in[u]) {
+              if constexpr (CE == 16) st_global16(dst, w[0], w[1], w[2], w[3]);
+              else st_global8(dst, w[0], w[1]);
+            }
           }
         }
       }
@@ -1284,12 +1318,15 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
       {
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
-          uint32_t w[NP];
 #pragma unroll
-          for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[k][i].x, x[k][i].y);
-          char* dst = reinterpret_cast<char*>(p.out) + (row * p.out_ld + (c_first + k * STRIDE) * CE) * 2;
+          for (int u = 0; u < RPL; ++u) {
+            uint32_t w[NP];
 #pragma unroll
-          for (int j = 0; j < CE / 8; ++j) if (row_in) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            for (int i = 0; i < NP; ++i) w[i] = pack_fpx2<BF>(x[u][k][i].x, x[u][k][i].y);
+            char* dst = reinterpret_cast<char*>(p.out) + ((row + u) * p.out_ld + (c_first + k * STRIDE) * CE) * 2;
+#pragma unroll
+            for (int j = 0; j < CE / 8; ++j) if (row_in[u]) st_global16(dst + 16 * j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+          }
         }
       }
     }
@@ -1299,11 +1336,11 @@ __global__ void __launch_bounds__(LNF_THREADS, 2) ln_wide_kernel(const LnParams 
 
 template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, int WPR, bool F8, int GEO>
 static hero_status launch_wide(hero_handle* h, LnParams& p, cudaStream_t stream) {
-  constexpr int H = (GEO == 6 ? 768 : 1024) * WPR, SLOTS = GEO >= 5 ? 16 : 8 / WPR;
+  constexpr int H = (GEO == 6 ? 768 : 1024) * WPR, SLOTS = GEO >= 6 ? 16 : 8 / WPR;   // (GEO 6, 7: two rows per warp)
   constexpr int ES_RES = (RES == SRC_I8) ? 1 : 2, ES_BR = (BR == SRC_I8) ? 1 : (BR == SRC_FP ? 2 : 0);
   constexpr size_t STAGE = (size_t)SLOTS * H * (ES_RES + ES_BR);
-  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0) + (GEO >= 5 ? 2 : 0));
-  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR, 2, GEO >= 5 ? 2 : 3);
+  constexpr size_t VEC = (size_t)H * 4 * ((RES == SRC_I8 && RSC == RS_COL ? 1 : 0) + (BR == SRC_I8 ? 1 : 0) + (OUT == O_STATIC ? 1 : 0) + (GEO >= 6 ? 2 : 0));
+  constexpr int stages = ln_wide_stages((int)STAGE, (int)VEC, WPR, 2, GEO >= 6 ? 2 : 3);
   const size_t smem = (size_t)stages * STAGE + VEC;
   auto kern = ln_wide_kernel<RES, RSC, BR, OUT, FPOUT, BF, WPR, F8, GEO>;
   HERO_SMEM_OPT_IN(h, kern, 200 * 1024);
@@ -1329,7 +1366,7 @@ template <int RES, int RSC, int BR, int OUT, bool FPOUT, bool BF, bool F8>
 static hero_status launch_wide_wpr(hero_handle* h, LnParams& p, cudaStream_t s) {
   switch (p.H) {
     case 768: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 6>(h, p, s);
-    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 5>(h, p, s);
+    case 1024: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 1, F8, 7>(h, p, s);
     case 2048: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 2, F8, 0>(h, p, s);
     case 4096: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 4, F8, 0>(h, p, s);
     default: return launch_wide<RES, RSC, BR, OUT, FPOUT, BF, 8, F8, 0>(h, p, s);
