@@ -96,6 +96,43 @@ def test_residual_int8_twq_plus_int8_fwq(h, out_kind, H):
     _compare(res, want, None, spec)
 
 
+@pytest.mark.parametrize("out_kind", ["twq", "fwq", "fp"])
+@pytest.mark.parametrize("M,H", [(1, 1024), (33, 1024), (4737, 1024), (1, 768), (33, 768), (4737, 768)])
+def test_two_rows_per_warp_odd_row_counts_and_untouched_tail(h, M, H, out_kind):
+    # rows of 1024 / 768 are processed two per warp: an odd row count leaves the last warp with one row, several passes of
+    # the grid (4737 rows) make that happen in the last pass only; nothing beyond row M - 1 may be written
+    g = W.rng(2, 500 + M + H)
+    x, gamma, beta = W.ln_case(M, H)
+    xin = O.emit(x, O.OutSpec("twq"))
+    s_o = (np.abs(g.standard_normal(H)) * 0.01 + 0.002).astype(np.float32)
+    xo = O.QT("i8", g.integers(-127, 128, (M, H), dtype=np.int8), col_scale=s_o.astype(np.float64))
+    y = O.layernorm(xin.real() + xo.real(), gamma, beta, 1e-12)
+    spec = {"twq": O.OutSpec("twq"), "fwq": O.OutSpec("fwq", scale=Q.calib_scale(np.abs(y).max(0))),
+            "fp": O.OutSpec("fp", dtype="f16")}[out_kind]
+    want, _ = O.ln_quant([xin, xo], gamma, beta, 1e-12, spec)
+    din, do = qt_to_device(xin), qt_to_device(xo)
+    pad = 3
+    if out_kind == "fp":
+        full = torch.full((M + pad, H), 7.0, dtype=torch.float16, device="cuda")
+        desc = hero.tensor(full[:M])
+        sc = None
+    else:
+        full = torch.full((M + pad, H), 77, dtype=torch.int8, device="cuda")
+        sc = torch.full((M + pad,), -5.0, dtype=torch.float32, device="cuda") if out_kind == "twq" else f32(spec.scale)
+        desc = hero.tensor(full[:M], out_kind, sc[:M] if out_kind == "twq" else sc)
+    h.hero_layernorm_quant(din[1], f32(gamma), f32(beta), 1e-12, desc, branch=do[1])
+    h.check()
+    if out_kind == "fp":
+        assert rel_err(full[:M].float().cpu().numpy(), want.data) < 2e-3
+        assert bool((full[M:] == 7.0).all())
+    else:
+        assert_int8_close(full[:M].cpu().numpy(), want.data, what="LN out")
+        assert bool((full[M:] == 77).all())
+        if out_kind == "twq":
+            assert_scales_close(sc[:M].cpu().numpy(), want.row_scale, 1e-6, "LN row scales")
+            assert bool((sc[M:] == -5.0).all())
+
+
 @pytest.mark.parametrize("res_kind,br_kind", [("i8_twq", "f16"), ("f16", "f16"), ("bf16", "i8_fwq"), ("i8_fwq", "i8_fwq"),
                                               ("i8_sq", "bf16")])
 @pytest.mark.parametrize("H", [1024, 768])        # two chunks of 16 elements per lane / three chunks of 8
