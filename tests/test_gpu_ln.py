@@ -159,9 +159,8 @@ def test_mixed_input_types(h, res_kind, br_kind, H):
 
 
 @pytest.mark.parametrize("fp", ["f16", "bf16"])
-@pytest.mark.parametrize("H", [4096, 768])
-def test_pre_ln_dual_output_and_bare_add(h, fp, H):
-    M = 150
+@pytest.mark.parametrize("M,H", [(150, 4096), (150, 768), (151, 1024), (2401, 768)])     # (odd counts: two rows per warp)
+def test_pre_ln_dual_output_and_bare_add(h, fp, M, H):
     g = W.rng(2, 123)
     hres = O.fp_tensor(g.standard_normal((M, H)), fp)
     br = O.QT("i8", g.integers(-127, 128, (M, H), dtype=np.int8),
