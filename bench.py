@@ -391,19 +391,23 @@ def sweep_extra(h, peaks):
     i8_burst = 2.0 * peaks["bf16_tflops"]
     out = {"gemm_int8": [], "ln_quant": [], "peaks": {"int8_tops_burst": i8_burst, "int8_tops_nominal": INT8_NOMINAL_TOPS, "hbm_gbs": peaks["hbm_gbs"]},
            "note": "each kernel timed alone over rotating buffers larger than L2, CUDA events; GEMM epilogue = dequant + bias + "
-                   "requant to INT8; LN^quant algorithmic bytes 3 per element"}
+                   "requant to INT8; LN^quant algorithmic bytes 3 per element, launches timed as CUDA-graph replays"}
     for K, N in W.GEMM_SWEEP_KN:
         for M in (8192, 32768):
             r = MB.bench_gemm(h, M, K, N, "none", False, 10)
             out["gemm_int8"].append({"M": M, "K": K, "N": N, "tops": round(r["tops"], 1), "frac_of_burst": round(r["tops"] / i8_burst, 3),
                                      "frac_of_nominal": round(r["tops"] / INT8_NOMINAL_TOPS, 3)})
             torch.cuda.empty_cache()
+    # LN^quant launches of tens of microseconds are timed as CUDA-graph replays (as in profiles/ln_quant.md): between plain
+    # launches the host's launch gaps are part of the figure and make it wander from run to run
+    MB.GRAPH = True
     for H in W.LN_SWEEP_H:
         for kind in ("f16", "i8"):
-            r = MB.bench_ln(h, 65536, H, kind, 20)
+            r = MB.bench_ln(h, 65536, H, kind, 40)
             out["ln_quant"].append({"M": 65536, "H": H, "inputs": "fp16" if kind == "f16" else "int8 twq + int8 fwq", "gbs": round(r["gbs"], 0),
                                     "frac_of_hbm": round(r["gbs"] / peaks["hbm_gbs"], 3)})
             torch.cuda.empty_cache()
+    MB.GRAPH = False
     try:
         # a library INT8 GEMM of the same size as the driver's BF16 probe, for a MEASURED INT8 figure beside the derived
         # 2 x BF16 one (measurement only: nothing of the product path goes through it)
